@@ -1,0 +1,294 @@
+"""EchoKV decode attention -- plain CPU oracle (numpy, fp64).
+
+TEST INFRASTRUCTURE ONLY.  This module defines what the CUDA library must
+compute; it is slow, un-blocked and un-fused on purpose.  It shares no code
+with the CUDA path and imports nothing from it.  Only the test-suite, the
+smoke check and the benchmark's CPU-baseline leg may import it.
+
+Every function takes real-valued numpy arrays (any float dtype; values that
+were stored as bf16 or fp32 are widened to float64 exactly by the helpers at
+the bottom) and computes in float64 without intermediate rounding.
+
+Notation (paper, Section 3.2 "Network Architecture"):
+  L      tokens in the cache
+  H_kv   KV heads, d head dim, D = H_kv * d  flattened per-token KV width
+  S      group size: layer l is an anchor ("global") layer iff l % S == 0 (Eq. 1)
+  m      retained local dims of a compressed layer: C_local = C[:, :m]  (Eq. 2)
+  W      predictor, shape [D - m, D + m]; C_hat_drop = W [C_global ; C_local] (Eq. 3)
+  C_drop = C[:, m:] is what W predicts (Eq. 4)
+  X_tilde = Reshape([X_local ; X_hat_drop]), X in {K, V}            (Eq. 6)
+  A(Q, K, V) = softmax(Q K^T / sqrt(d)) V                           (Eq. 7, App. D.1)
+
+Readings of points the paper leaves open (all listed in the design notes):
+  * K and V have separate predictors, each seeing only its own kind of cache
+    (Table "Hyperparameter configurations": 1408 = 1024 + 384 inputs).
+  * no bias unless one is passed (Eq. 3 has none).
+  * predictor input order is [global ; local] as written in Eq. 3.
+  * flattening is head-major: flat index = head * d + feature.
+  * query head h attends KV head floor(h / (H_q / H_kv)) (contiguous groups).
+  * every cached token, the newest included, is reconstructed alike.
+
+Pins (tests/test_oracle_*.py): hand-computed softmax case, pure-python brute
+force, torch scaled_dot_product_attention (library routine) for the m = D and
+selector-weight cases, zero-weight closed forms, linearity, softmax shift /
+permutation / log-sum-exp merge invariants, and the paper's printed predictor
+shapes, ratios and parameter totals.  What stays "parity unpinned": nothing in
+the paper prints a numeric attention output, and how well a *trained* W
+approximates the dropped cache cannot be checked without trained weights (it is
+not part of what the kernels compute).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+# ----------------------------------------------------------------------------
+# Configuration arithmetic (Eq. 1, Eq. 2, Appendix "Compression-Ratio
+# Configurations", Table "Hyperparameter configurations")
+# ----------------------------------------------------------------------------
+
+
+def is_anchor_layer(layer: int, group_size: int) -> bool:
+    """Eq. 1: the first layer of each group of S layers keeps its full cache."""
+    return layer % group_size == 0
+
+
+def anchor_of(layer: int, group_size: int) -> int:
+    """Eq. 1: C_global^(k) = C_{k*S}; the anchor of layer k*S+i is layer k*S."""
+    return layer - layer % group_size
+
+
+def predictor_shape(D: int, m: int) -> tuple[int, int]:
+    """(input dim, output dim) of W: input [C_global ; C_local] has D + m
+    features, output C_hat_drop has D - m (Eq. 2-4)."""
+    if not 0 <= m <= D:
+        raise ValueError("need 0 <= m <= D")
+    return D + m, D - m
+
+
+def effective_ratio(D: int, group_size: int, m: int) -> float:
+    """Kept fraction of a group's cache: one full layer plus S-1 layers of m
+    dims, over S full layers (Appendix "Compression-Ratio Configurations")."""
+    return (D + (group_size - 1) * m) / (group_size * D)
+
+
+def n_compressed_layers(n_layers: int, group_size: int) -> int:
+    return sum(0 if is_anchor_layer(l, group_size) else 1 for l in range(n_layers))
+
+
+def total_predictor_params(n_layers: int, group_size: int, D: int, m: int,
+                           bias: bool = False) -> int:
+    """Two predictors (one for K, one for V) per compressed layer."""
+    d_in, d_out = predictor_shape(D, m)
+    per = d_in * d_out + (d_out if bias else 0)
+    return 2 * n_compressed_layers(n_layers, group_size) * per
+
+
+# ----------------------------------------------------------------------------
+# Reconstruction (Eq. 2, 3, 4, 6)
+# ----------------------------------------------------------------------------
+
+
+def predictor_input(c_global: np.ndarray, c_local: np.ndarray) -> np.ndarray:
+    """[C_global ; C_local] per token (Eq. 3): [L, D] and [L, m] -> [L, D + m]."""
+    c_global = np.asarray(c_global, dtype=np.float64)
+    c_local = np.asarray(c_local, dtype=np.float64)
+    if c_global.shape[0] != c_local.shape[0]:
+        raise ValueError("token counts differ")
+    return np.concatenate([c_global, c_local], axis=1)
+
+
+def reconstruct_dropped(W: np.ndarray, c_global: np.ndarray, c_local: np.ndarray,
+                        bias: np.ndarray | None = None) -> np.ndarray:
+    """Eq. 3: C_hat_drop[t, :] = W [C_global[t] ; C_local[t]]  (+ bias if given).
+
+    W is [D - m, D + m] (rows = dropped flat dims m..D-1, columns = the D global
+    dims then the m local dims).  Returns [L, D - m].
+    """
+    W = np.asarray(W, dtype=np.float64)
+    x = predictor_input(c_global, c_local)                     # [L, D + m]
+    if W.shape[1] != x.shape[1]:
+        raise ValueError("W has %d columns, input has %d features" % (W.shape[1], x.shape[1]))
+    c_hat = x @ W.T                                            # [L, D - m]
+    if bias is not None:
+        c_hat = c_hat + np.asarray(bias, dtype=np.float64)[None, :]
+    return c_hat
+
+
+def assemble_cache(c_local: np.ndarray, c_hat_drop: np.ndarray, n_kv_heads: int,
+                   head_dim: int) -> np.ndarray:
+    """Eq. 6: X_tilde = Reshape([X_local ; X_hat_drop]) -> [L, H_kv, d]
+    (head-major flattening: flat index = head * d + feature)."""
+    c_local = np.asarray(c_local, dtype=np.float64)
+    c_hat_drop = np.asarray(c_hat_drop, dtype=np.float64)
+    flat = np.concatenate([c_local, c_hat_drop], axis=1)
+    L, D = flat.shape
+    if D != n_kv_heads * head_dim:
+        raise ValueError("local + dropped widths do not add up to H_kv * d")
+    return flat.reshape(L, n_kv_heads, head_dim)
+
+
+# ----------------------------------------------------------------------------
+# Attention (Eq. 7; softmax as defined in the QK-KL appendix)
+# ----------------------------------------------------------------------------
+
+
+def attention_probabilities(q: np.ndarray, K: np.ndarray, scale: float | None = None
+                            ) -> np.ndarray:
+    """softmax_t(q_h . K[t, kv(h)] * scale) -> [H_q, L], kv(h) = h // (H_q / H_kv)."""
+    q = np.asarray(q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    H_q, d = q.shape
+    L, H_kv, d2 = K.shape
+    if d2 != d or H_q % H_kv != 0:
+        raise ValueError("bad head shapes")
+    if L == 0:
+        raise ValueError("softmax over an empty cache is undefined")
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    g = H_q // H_kv
+    p = np.empty((H_q, L), dtype=np.float64)
+    for h in range(H_q):
+        s = (K[:, h // g, :] @ q[h]) * scale                   # [L]
+        e = np.exp(s - s.max())
+        p[h] = e / e.sum()
+    return p
+
+
+def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None = None
+              ) -> np.ndarray:
+    """Eq. 7 for one decode query per head: out[h] = sum_t p[h, t] V[t, kv(h), :].
+
+    q [H_q, d], K and V [L, H_kv, d] -> [H_q, d].
+    """
+    V = np.asarray(V, dtype=np.float64)
+    p = attention_probabilities(q, K, scale)
+    H_q = p.shape[0]
+    g = H_q // V.shape[1]
+    out = np.empty((H_q, V.shape[2]), dtype=np.float64)
+    for h in range(H_q):
+        out[h] = p[h] @ V[:, h // g, :]
+    return out
+
+
+def full_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
+                   n_kv_heads: int, scale: float | None = None) -> np.ndarray:
+    """Attention of an anchor layer / the uncompressed mode: the stored cache
+    [L, D] is used as it is (Eq. 7 with K_tilde = K, V_tilde = V)."""
+    k_cache = np.asarray(k_cache, dtype=np.float64)
+    v_cache = np.asarray(v_cache, dtype=np.float64)
+    L, D = k_cache.shape
+    d = D // n_kv_heads
+    return attention(q, k_cache.reshape(L, n_kv_heads, d), v_cache.reshape(L, n_kv_heads, d), scale)
+
+
+def decode_attention(q: np.ndarray,
+                     k_global: np.ndarray, v_global: np.ndarray,
+                     k_local: np.ndarray, v_local: np.ndarray,
+                     Wk: np.ndarray, Wv: np.ndarray,
+                     n_kv_heads: int, scale: float | None = None,
+                     bk: np.ndarray | None = None, bv: np.ndarray | None = None
+                     ) -> np.ndarray:
+    """One decode step of a compressed layer for one sequence.
+
+    k_global, v_global [L, D]  full cache of the group's anchor layer   (Eq. 1)
+    k_local,  v_local  [L, m]  retained dims of this layer              (Eq. 2)
+    Wk, Wv [D - m, D + m]      this layer's predictors                  (Eq. 3)
+    q [H_q, d]                 the new token's queries
+    Steps: predict the dropped dims (Eq. 3), rebuild K_tilde, V_tilde (Eq. 6),
+    attend (Eq. 7).  Returns [H_q, d].
+    """
+    k_global = np.asarray(k_global, dtype=np.float64)
+    D = k_global.shape[1]
+    d = D // n_kv_heads
+    k_hat = reconstruct_dropped(Wk, k_global, k_local, bk)
+    v_hat = reconstruct_dropped(Wv, v_global, v_local, bv)
+    K_t = assemble_cache(k_local, k_hat, n_kv_heads, d)
+    V_t = assemble_cache(v_local, v_hat, n_kv_heads, d)
+    return attention(q, K_t, V_t, scale)
+
+
+def decode_attention_query_heads(q: np.ndarray,
+                                 k_global: np.ndarray, v_global: np.ndarray,
+                                 k_local: np.ndarray, v_local: np.ndarray,
+                                 Wk: np.ndarray, Wv: np.ndarray,
+                                 n_kv_heads: int, query_heads, scale: float | None = None
+                                 ) -> dict[int, np.ndarray]:
+    """The same quantity as decode_attention, for a chosen few query heads only.
+
+    Heads are independent in Eq. 7 and each dropped flat dim is one row of W in
+    Eq. 3, so for query head h only the d rows of W that produce KV head kv(h)
+    are evaluated.  Used to check sampled outputs of workloads too large to run
+    in full.  Returns {h: out[h] as [d]}.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k_global = np.asarray(k_global, dtype=np.float64)
+    v_global = np.asarray(v_global, dtype=np.float64)
+    k_local = np.asarray(k_local, dtype=np.float64)
+    v_local = np.asarray(v_local, dtype=np.float64)
+    H_q, d = q.shape
+    D = k_global.shape[1]
+    m = k_local.shape[1]
+    g = H_q // n_kv_heads
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    out = {}
+    for h in query_heads:
+        kv = h // g
+        lo = kv * d                                   # flat dims [lo, lo + d) of K_tilde
+        if lo + d <= m:                               # a retained head: stored values
+            K_h = k_local[:, lo:lo + d]
+            V_h = v_local[:, lo:lo + d]
+        elif lo >= m:                                 # a dropped head: rows lo-m .. of W
+            rows = slice(lo - m, lo - m + d)
+            K_h = predictor_input(k_global, k_local) @ np.asarray(Wk, dtype=np.float64)[rows].T
+            V_h = predictor_input(v_global, v_local) @ np.asarray(Wv, dtype=np.float64)[rows].T
+        else:
+            raise ValueError("m must be head-aligned for per-head evaluation")
+        s = (K_h @ q[h]) * scale
+        e = np.exp(s - s.max())
+        out[h] = (e / e.sum()) @ V_h
+    return out
+
+
+# ----------------------------------------------------------------------------
+# Multi-layer step (Eq. 1): which cache each layer attends over
+# ----------------------------------------------------------------------------
+
+
+def layer_step(layer: int, group_size: int, q: np.ndarray, caches_k, caches_v,
+               weights_k, weights_v, n_kv_heads: int, m: int,
+               scale: float | None = None) -> np.ndarray:
+    """Decode attention of `layer` for one sequence.
+
+    caches_k[l], caches_v[l]: [L, D] full (true) caches of every layer; a
+    compressed layer only ever reads its first m dims, an anchor layer all D.
+    weights_k[l], weights_v[l]: predictors of compressed layers.
+    """
+    if is_anchor_layer(layer, group_size):
+        return full_attention(q, caches_k[layer], caches_v[layer], n_kv_heads, scale)
+    a = anchor_of(layer, group_size)
+    return decode_attention(q, caches_k[a], caches_v[a],
+                            np.asarray(caches_k[layer])[:, :m], np.asarray(caches_v[layer])[:, :m],
+                            weights_k[layer], weights_v[layer], n_kv_heads, scale)
+
+
+# ----------------------------------------------------------------------------
+# Stored-precision helpers (exact widening; no arithmetic of the method here)
+# ----------------------------------------------------------------------------
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """uint16 bf16 bit patterns -> float64, exactly (bf16 is the top half of fp32)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def widen(x) -> np.ndarray:
+    """Widen a stored tensor to float64: uint16 arrays are bf16 bit patterns,
+    float arrays are taken by value."""
+    x = np.asarray(x)
+    if x.dtype == np.uint16:
+        return bf16_bits_to_f64(x)
+    return x.astype(np.float64)
