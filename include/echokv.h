@@ -1,0 +1,183 @@
+/*
+ * echokv.h -- C-ABI of the B200 (sm_100a) EchoKV decode-attention library.
+ *
+ * What the library computes (paper, Section 3.2 "Network Architecture" and Eq. 6-7):
+ * the layers of a model are split into groups of S; the first layer of a group
+ * (the "anchor", Eq. 1) keeps its whole KV cache, every other layer keeps only the
+ * first m = r * head_dim flattened dims of each token's K and V (Eq. 2).  At decode
+ * time the dropped dims of a compressed layer are predicted per token by one linear
+ * map per layer and per kind (K, V),
+ *     C_hat_drop[t] = W [C_anchor[t] ; C_local[t]]                         (Eq. 3)
+ * the cache is rebuilt as Reshape([C_local ; C_hat_drop]) (Eq. 6) and fed to
+ *     out_h = softmax_t(q_h . K~[t, kv(h)] * scale) V~[:, kv(h)]           (Eq. 7)
+ * with kv(h) = h / (n_q_heads / n_kv_heads).  The reconstructed K~/V~ exist only
+ * on chip; they are never written to device memory.
+ *
+ * Conventions
+ *  - Every function returns an int status (ECHOKV_OK = 0, negative = error) and
+ *    never throws, aborts or traps.  echokv_strerror() names a status.
+ *  - "device pointer" = memory of the CUDA device named in the config, allocated by
+ *    the caller (e.g. by PyTorch); the library BORROWS it: it must stay valid until
+ *    echokv_destroy().  "host pointer" = ordinary host memory, read during the call
+ *    only, unless stated otherwise.  The library itself allocates no device memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *    that take a stream only enqueue work on it and return; the *_host calls and
+ *    echokv_get_device_status() synchronise.
+ *  - Flattened KV index = kv_head * head_dim + feature.  Retained heads are heads
+ *    0 .. r-1.  Storage type (cache, weights, queries, new K/V) is the config's
+ *    dtype; accumulation is always fp32; outputs are fp32.
+ *  - Page pools: layer l's K pool and V pool are each
+ *        [n_pages][page_tokens][width(l)]   row-major, width = D for an anchor
+ *        layer, m for a compressed layer (no pool when m = 0),
+ *    and one int32 block table [max_batch][max_pages_per_seq], shared by all layers,
+ *    maps (sequence slot, token / page_tokens) to a page id in [0, n_pages).
+ *  - Predictors: Wk, Wv are [D - m][D + m] row-major; column i < D multiplies anchor
+ *    dim i, column D + i multiplies local dim i; row j produces flat dim m + j.
+ */
+#ifndef ECHOKV_H
+#define ECHOKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct echokv_ctx echokv_ctx;
+
+enum { ECHOKV_BF16 = 0, ECHOKV_FP32 = 1 };
+
+enum {
+  ECHOKV_OK = 0,
+  ECHOKV_EINVAL = -1,         /* NULL pointer, bad dimension, layer out of range          */
+  ECHOKV_ENOTANCHOR = -2,     /* echokv_full_attention on a layer that keeps only m dims   */
+  ECHOKV_ENOTCOMPRESSED = -3, /* echokv_set_weights on an anchor layer                     */
+  ECHOKV_ECAPACITY = -4,      /* batch > max_batch, workspace too small, length > pages    */
+  ECHOKV_ENOWEIGHTS = -5,     /* decode on a compressed layer before echokv_set_weights    */
+  ECHOKV_ECUDA = -6,          /* a CUDA runtime / driver call failed                       */
+  ECHOKV_ETIMEOUT = -7,       /* device status: a bounded on-chip wait ran out             */
+  ECHOKV_EBADPAGE = -8,       /* device status: page id or sequence slot out of range      */
+  ECHOKV_EUNSUPPORTED = -9,   /* shape outside what the kernels handle                     */
+  ECHOKV_ENOTABLE = -10,      /* a call that needs the block table before it was set       */
+  ECHOKV_EBADLENGTH = -11     /* device status: a sequence length < 1 or beyond capacity   */
+};
+
+typedef struct {
+  int32_t n_layers;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;        /* must divide n_q_heads                                      */
+  int32_t head_dim;          /* 64 or 128                                                  */
+  int32_t group_size;        /* S >= 1; layer l is an anchor iff l % S == 0 (Eq. 1)        */
+  int32_t n_retained_heads;  /* r in [0, n_kv_heads]; m = r * head_dim (Eq. 2)             */
+  int32_t page_tokens;       /* tokens per page: 16, 32, 64 or 128                         */
+  int32_t max_batch;         /* rows of the block table                                    */
+  int32_t max_pages_per_seq; /* columns of the block table                                 */
+  int32_t dtype;             /* ECHOKV_BF16 or ECHOKV_FP32                                 */
+  int64_t n_pages;           /* pages per pool                                             */
+  float softmax_scale;       /* 0 -> 1 / sqrt(head_dim) (Eq. 7)                            */
+  int32_t device;            /* CUDA device ordinal                                        */
+} echokv_config;
+
+typedef struct {
+  uint64_t anchor_pool_bytes;     /* one K (or V) pool of an anchor layer                  */
+  uint64_t compressed_pool_bytes; /* one K (or V) pool of a compressed layer (0 if m = 0)  */
+  uint64_t block_table_bytes;
+  uint64_t workspace_bytes;       /* minimum size of echokv_buffers.workspace              */
+  int32_t max_partials;           /* split-K partial results kept per (sequence, head)     */
+  int32_t reserved;
+} echokv_sizes;
+
+typedef struct {
+  void* const* k_pools;      /* host array [n_layers] of device pointers (copied at create) */
+  void* const* v_pools;      /* same for V; entries of compressed layers may be NULL if m=0 */
+  void* workspace;           /* device pointer, >= workspace_bytes, 256-byte aligned        */
+  uint64_t workspace_bytes;
+} echokv_buffers;
+
+/* Sizes implied by a config.  Pure host arithmetic, no CUDA call.
+ * Errors: EINVAL (NULL or inconsistent config), EUNSUPPORTED (head_dim, page size). */
+int echokv_query_sizes(const echokv_config* cfg, echokv_sizes* out);
+
+/* Build a context over caller-owned device buffers (pools, workspace).  Makes `device`
+ * current, clears the workspace's status word (synchronous) and prepares the tensor maps
+ * of every pool.  Errors: EINVAL, EUNSUPPORTED, ECAPACITY (workspace too small), ECUDA. */
+int echokv_create(const echokv_config* cfg, const echokv_buffers* buffers, echokv_ctx** out);
+
+/* Release the context (host memory only; the caller's device buffers are untouched). */
+void echokv_destroy(echokv_ctx* ctx);
+
+/* Install the predictors of compressed layer `layer` (Eq. 3): device pointers Wk, Wv of
+ * [D - m][D + m] elements, optional biases bk, bv of [D - m] (NULL = none, the paper's
+ * Eq. 3 has none).  Borrowed.  Errors: EINVAL, ENOTCOMPRESSED, ECUDA. */
+int echokv_set_weights(echokv_ctx* ctx, int layer, const void* Wk, const void* Wv,
+                       const void* bk, const void* bv);
+
+/* Install the block table: device pointer to int32 [max_batch][max_pages_per_seq].
+ * Borrowed; the caller may change its contents between calls (stream-ordered). */
+int echokv_set_block_table(echokv_ctx* ctx, const int32_t* dev_block_table);
+
+/* Append one new token per sequence to layer `layer`'s cache (Section 3.1: compression is
+ * plain eviction of part of each token's K/V): k_new, v_new are device pointers
+ * [B][n_kv_heads][head_dim];
+ * an anchor layer stores all D dims, a compressed layer only the first m (Eq. 2) -- the rest
+ * is never written anywhere.  dev_positions[b] = token index to write (its page must be in
+ * the block table); dev_seq_slots[b] = row of the block table (NULL = row b).
+ * Bad slot / page / position -> device status EBADPAGE, that token is skipped.
+ * Errors: EINVAL, ECAPACITY, ENOTABLE, ECUDA. */
+int echokv_append_kv(echokv_ctx* ctx, int layer, const void* k_new, const void* v_new,
+                     const int32_t* dev_seq_slots, const int32_t* dev_positions, int B, void* stream);
+
+/* Decode attention of compressed layer `layer` (Eq. 3, 6, 7): q is a device pointer
+ * [B][n_q_heads][head_dim], out a device pointer to fp32 [B][n_q_heads][head_dim],
+ * dev_seq_lens[b] = tokens in the cache (>= 1, newest included).  Heads 0..r-1 attend their
+ * stored K/V; heads r.. attend K/V predicted on chip from the anchor layer's cache and this
+ * layer's retained dims.  Called on an anchor layer it is the same as echokv_full_attention.
+ * Uses the workspace; calls on one context must not overlap on the device.
+ * A length < 1 or beyond max_pages_per_seq * page_tokens -> device status EBADLENGTH and
+ * zeros for that sequence.  Errors: EINVAL, ECAPACITY, ENOWEIGHTS, ENOTABLE, ECUDA. */
+int echokv_decode_attention(echokv_ctx* ctx, int layer, const void* q, float* out,
+                            const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                            void* stream);
+
+/* Attention over a layer that holds its full cache (anchor layers; the uncompressed
+ * short-context mode the paper switches from, Section 5.4): Eq. 7 on the stored K, V.
+ * Same arguments as echokv_decode_attention.  Errors: as above plus ENOTANCHOR. */
+int echokv_full_attention(echokv_ctx* ctx, int layer, const void* q, float* out,
+                          const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                          void* stream);
+
+/* One layer-step driven from HOST memory: copies q, k_new, v_new ([B][heads][head_dim],
+ * storage dtype) and seq_lens (int32 [B], lengths AFTER the append) to the device, appends
+ * at position seq_lens[b]-1 in block-table row b, runs the layer's attention if `attend`
+ * is non-zero (decode for a compressed layer, full for an anchor), copies the fp32 result to
+ * out_host and synchronises the stream.  For best speed the host buffers should be pinned.
+ * q_host / out_host may be NULL when attend == 0.  Errors: as the calls it is made of. */
+int echokv_layer_step_host(echokv_ctx* ctx, int layer, const void* q_host, const void* k_new_host,
+                           const void* v_new_host, float* out_host, const int32_t* seq_lens_host,
+                           int B, int attend, void* stream);
+
+/* Read and clear the device status word (synchronises the device).  *host_out receives
+ * ECHOKV_OK or the first device-side error (ETIMEOUT, EBADPAGE, EBADLENGTH). */
+int echokv_get_device_status(echokv_ctx* ctx, int32_t* host_out);
+
+/* Number of kernels the library has launched on this context since creation. */
+int64_t echokv_launch_count(const echokv_ctx* ctx);
+
+/* Which kernel family serves compressed layers of this context:
+ * 0 = none (no layer is compressed or nothing is dropped), 1 = fp32/bf16 CUDA-core kernel,
+ * 2 = bf16 tcgen05 tensor-core kernel. */
+int echokv_decode_path(const echokv_ctx* ctx);
+
+/* Choose the kernel family for compressed layers: 1 = CUDA-core kernel (always possible),
+ * 2 = tcgen05 kernel (EUNSUPPORTED unless dtype is bf16, head_dim 128).  Contexts start on
+ * the fastest family their shape allows.  Meant for tests that check both against the oracle. */
+int echokv_set_decode_path(echokv_ctx* ctx, int path);
+
+/* Static, human-readable name of a status code. */
+const char* echokv_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ECHOKV_H */

@@ -1,0 +1,237 @@
+"""ctypes binding of libechokv.so: the same names as include/echokv.h, argument
+marshalling only.  Every step of the decode path runs in the library's CUDA
+kernels; PyTorch is used by `Context` for device memory and streams.
+
+The library must have been built (python -m paper_2603_22910_b200.build);
+loading fails loudly otherwise -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libechokv.so")
+
+ECHOKV_BF16, ECHOKV_FP32 = 0, 1
+ECHOKV_OK = 0
+ECHOKV_EINVAL, ECHOKV_ENOTANCHOR, ECHOKV_ENOTCOMPRESSED, ECHOKV_ECAPACITY = -1, -2, -3, -4
+ECHOKV_ENOWEIGHTS, ECHOKV_ECUDA, ECHOKV_ETIMEOUT, ECHOKV_EBADPAGE = -5, -6, -7, -8
+ECHOKV_EUNSUPPORTED, ECHOKV_ENOTABLE, ECHOKV_EBADLENGTH = -9, -10, -11
+
+
+class echokv_config(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("group_size", C.c_int32), ("n_retained_heads", C.c_int32),
+                ("page_tokens", C.c_int32), ("max_batch", C.c_int32), ("max_pages_per_seq", C.c_int32),
+                ("dtype", C.c_int32), ("n_pages", C.c_int64), ("softmax_scale", C.c_float),
+                ("device", C.c_int32)]
+
+
+class echokv_sizes(C.Structure):
+    _fields_ = [("anchor_pool_bytes", C.c_uint64), ("compressed_pool_bytes", C.c_uint64),
+                ("block_table_bytes", C.c_uint64), ("workspace_bytes", C.c_uint64),
+                ("max_partials", C.c_int32), ("reserved", C.c_int32)]
+
+
+class echokv_buffers(C.Structure):
+    _fields_ = [("k_pools", C.POINTER(C.c_void_p)), ("v_pools", C.POINTER(C.c_void_p)),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_uint64)]
+
+
+EXPORTS = {
+    # name: (restype, argtypes)
+    "echokv_query_sizes": (C.c_int, [C.POINTER(echokv_config), C.POINTER(echokv_sizes)]),
+    "echokv_create": (C.c_int, [C.POINTER(echokv_config), C.POINTER(echokv_buffers), C.POINTER(C.c_void_p)]),
+    "echokv_destroy": (None, [C.c_void_p]),
+    "echokv_set_weights": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "echokv_set_block_table": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "echokv_append_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_int, C.c_void_p]),
+    "echokv_decode_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_int, C.c_void_p]),
+    "echokv_full_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_int, C.c_void_p]),
+    "echokv_layer_step_host": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
+    "echokv_get_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
+    "echokv_launch_count": (C.c_int64, [C.c_void_p]),
+    "echokv_decode_path": (C.c_int, [C.c_void_p]),
+    "echokv_set_decode_path": (C.c_int, [C.c_void_p, C.c_int]),
+    "echokv_strerror": (C.c_char_p, [C.c_int]),
+}
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library (loaded once)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libechokv.so is not built: run `python -m paper_2603_22910_b200.build` "
+                               "(there is no fallback implementation)")
+        _lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(_lib, name)
+            fn.restype = res
+            fn.argtypes = args
+    return _lib
+
+
+class EchoKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (%d)" % (where, echokv_strerror(status), status))
+
+
+def echokv_strerror(status: int) -> str:
+    return lib().echokv_strerror(status).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != ECHOKV_OK:
+        raise EchoKVError(status, where)
+
+
+def _ptr(t) -> int | None:
+    """Device / host address of a torch tensor (None stays NULL)."""
+    return None if t is None else t.data_ptr()
+
+
+def _stream_handle(stream) -> int | None:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_retained_heads,
+                page_tokens, max_batch, max_pages_per_seq, n_pages, dtype, softmax_scale=0.0,
+                device=0) -> echokv_config:
+    return echokv_config(n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_retained_heads,
+                         page_tokens, max_batch, max_pages_per_seq, dtype, n_pages, softmax_scale, device)
+
+
+def echokv_query_sizes(cfg: echokv_config) -> echokv_sizes:
+    out = echokv_sizes()
+    _check(lib().echokv_query_sizes(C.byref(cfg), C.byref(out)), "echokv_query_sizes")
+    return out
+
+
+class Context:
+    """A context plus the torch tensors it borrows (pools, workspace, block table).
+
+    Allocation is the only thing done here that is not a direct C-ABI call.
+    """
+
+    def __init__(self, cfg: echokv_config, zero_pools: bool = False):
+        import torch
+        self.torch = torch
+        self.cfg = cfg
+        self.device = torch.device("cuda", cfg.device)
+        self.sizes = echokv_query_sizes(cfg)
+        self.tdtype = torch.bfloat16 if cfg.dtype == ECHOKV_BF16 else torch.float32
+        D = cfg.n_kv_heads * cfg.head_dim
+        m = cfg.n_retained_heads * cfg.head_dim
+        self.D, self.m = D, m
+        alloc = torch.zeros if zero_pools else torch.empty
+        self.k_pools, self.v_pools = [], []
+        for l in range(cfg.n_layers):
+            width = D if l % cfg.group_size == 0 else m
+            if width == 0:
+                self.k_pools.append(None)
+                self.v_pools.append(None)
+            else:
+                shape = (cfg.n_pages, cfg.page_tokens, width)
+                self.k_pools.append(alloc(shape, dtype=self.tdtype, device=self.device))
+                self.v_pools.append(alloc(shape, dtype=self.tdtype, device=self.device))
+        self.workspace = torch.empty(self.sizes.workspace_bytes, dtype=torch.uint8, device=self.device)
+        self.block_table = torch.zeros((cfg.max_batch, cfg.max_pages_per_seq), dtype=torch.int32,
+                                       device=self.device)
+        n = cfg.n_layers
+        self._kp = (C.c_void_p * n)(*[_ptr(t) for t in self.k_pools])
+        self._vp = (C.c_void_p * n)(*[_ptr(t) for t in self.v_pools])
+        buf = echokv_buffers(C.cast(self._kp, C.POINTER(C.c_void_p)), C.cast(self._vp, C.POINTER(C.c_void_p)),
+                             self.workspace.data_ptr(), self.sizes.workspace_bytes)
+        self.handle = C.c_void_p()
+        _check(lib().echokv_create(C.byref(cfg), C.byref(buf), C.byref(self.handle)), "echokv_create")
+        _check(lib().echokv_set_block_table(self.handle, self.block_table.data_ptr()), "echokv_set_block_table")
+        self._weights = {}
+
+    # -- direct wrappers -------------------------------------------------------------
+    def close(self):
+        if self.handle:
+            lib().echokv_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_block_table(self, table) -> None:
+        """Copy a host/device int32 table into the borrowed device block table."""
+        self.block_table[:table.shape[0], :table.shape[1]].copy_(table)
+
+    def set_weights(self, layer: int, Wk, Wv, bk=None, bv=None) -> None:
+        self._weights[layer] = (Wk, Wv, bk, bv)   # keep the borrowed tensors alive
+        _check(lib().echokv_set_weights(self.handle, layer, _ptr(Wk), _ptr(Wv), _ptr(bk), _ptr(bv)),
+               "echokv_set_weights")
+
+    def append_kv(self, layer: int, k_new, v_new, positions, seq_slots=None, stream=None) -> None:
+        _check(lib().echokv_append_kv(self.handle, layer, _ptr(k_new), _ptr(v_new), _ptr(seq_slots),
+                                      _ptr(positions), k_new.shape[0], _stream_handle(stream)),
+               "echokv_append_kv")
+
+    def decode_attention(self, layer: int, q, seq_lens, out=None, seq_slots=None, stream=None):
+        out = self._out(q) if out is None else out
+        _check(lib().echokv_decode_attention(self.handle, layer, _ptr(q), _ptr(out), _ptr(seq_slots),
+                                             _ptr(seq_lens), q.shape[0], _stream_handle(stream)),
+               "echokv_decode_attention")
+        return out
+
+    def full_attention(self, layer: int, q, seq_lens, out=None, seq_slots=None, stream=None):
+        out = self._out(q) if out is None else out
+        _check(lib().echokv_full_attention(self.handle, layer, _ptr(q), _ptr(out), _ptr(seq_slots),
+                                           _ptr(seq_lens), q.shape[0], _stream_handle(stream)),
+               "echokv_full_attention")
+        return out
+
+    def layer_step_host(self, layer: int, q_host, k_new_host, v_new_host, out_host, seq_lens_host,
+                        attend: bool = True, stream=None) -> None:
+        _check(lib().echokv_layer_step_host(self.handle, layer, _ptr(q_host), _ptr(k_new_host),
+                                            _ptr(v_new_host), _ptr(out_host), _ptr(seq_lens_host),
+                                            k_new_host.shape[0], 1 if attend else 0,
+                                            _stream_handle(stream)),
+               "echokv_layer_step_host")
+
+    def device_status(self) -> int:
+        v = C.c_int32(0)
+        _check(lib().echokv_get_device_status(self.handle, C.byref(v)), "echokv_get_device_status")
+        return v.value
+
+    def launch_count(self) -> int:
+        return lib().echokv_launch_count(self.handle)
+
+    def decode_path(self) -> int:
+        return lib().echokv_decode_path(self.handle)
+
+    def set_decode_path(self, path: int) -> None:
+        _check(lib().echokv_set_decode_path(self.handle, path), "echokv_set_decode_path")
+
+    def _out(self, q):
+        return self.torch.empty(q.shape, dtype=self.torch.float32, device=self.device)
+
+
+def config_for(w, n_pages: int | None = None, device: int = 0, max_batch: int | None = None) -> echokv_config:
+    """echokv_config of a synth.Workload."""
+    pages = w.pages_per_seq
+    return make_config(n_layers=w.n_layers, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                       head_dim=w.head_dim, group_size=w.group_size,
+                       n_retained_heads=w.n_retained_heads, page_tokens=w.page_tokens,
+                       max_batch=max_batch or w.batch, max_pages_per_seq=pages,
+                       n_pages=n_pages or w.batch * pages,
+                       dtype=ECHOKV_BF16 if w.dtype == "bf16" else ECHOKV_FP32,
+                       softmax_scale=1.0 / math.sqrt(w.head_dim), device=device)

@@ -1,0 +1,401 @@
+// C-ABI of the EchoKV library: argument checking, workspace layout, kernel selection.
+// All device memory belongs to the caller; nothing here allocates on the device.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kernels.h"
+#include "recon_tc.h"
+
+using namespace echokv;
+
+namespace {
+
+constexpr uint64_t kAlign = 256;
+inline uint64_t align_up(uint64_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Derived {
+  int D, m, d_in, d_drop, g, elem, part_tokens, capacity, max_parts;
+  uint64_t off_status, off_ml, off_o, off_q, off_k, off_v, off_out, off_lens, off_pos, total;
+};
+
+int derive(const echokv_config* c, Derived* d) {
+  if (!c) return ECHOKV_EINVAL;
+  if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->group_size < 1 ||
+      c->max_batch < 1 || c->max_pages_per_seq < 1 || c->n_pages < 1)
+    return ECHOKV_EINVAL;
+  if (c->n_q_heads % c->n_kv_heads != 0) return ECHOKV_EINVAL;
+  if (c->n_retained_heads < 0 || c->n_retained_heads > c->n_kv_heads) return ECHOKV_EINVAL;
+  if (c->dtype != ECHOKV_BF16 && c->dtype != ECHOKV_FP32) return ECHOKV_EINVAL;
+  if (!(c->softmax_scale >= 0.f) || !std::isfinite(c->softmax_scale)) return ECHOKV_EINVAL;
+  if (c->head_dim != 64 && c->head_dim != 128) return ECHOKV_EUNSUPPORTED;
+  if (c->page_tokens != 16 && c->page_tokens != 32 && c->page_tokens != 64 && c->page_tokens != 128)
+    return ECHOKV_EUNSUPPORTED;
+  d->g = c->n_q_heads / c->n_kv_heads;
+  if (d->g != 1 && d->g != 2 && d->g != 4 && d->g != 8) return ECHOKV_EUNSUPPORTED;
+  const long long cap = (long long)c->max_pages_per_seq * c->page_tokens;
+  if (cap > (1ll << 30)) return ECHOKV_EINVAL;
+  d->D = c->n_kv_heads * c->head_dim;
+  d->m = c->n_retained_heads * c->head_dim;
+  d->d_in = d->D + d->m;
+  d->d_drop = d->D - d->m;
+  d->elem = c->dtype == ECHOKV_BF16 ? 2 : 4;
+  d->part_tokens = (c->dtype == ECHOKV_BF16 && c->head_dim == 128) ? kTcPartTokens : kSimtTileTokens;
+  d->capacity = (int)cap;
+  d->max_parts = (d->capacity + d->part_tokens - 1) / d->part_tokens;
+  uint64_t off = 0;
+  d->off_status = off; off += kAlign;
+  const uint64_t n_part = (uint64_t)c->max_batch * c->n_q_heads * d->max_parts;
+  d->off_ml = off; off = align_up(off + n_part * sizeof(float2));
+  d->off_o = off; off = align_up(off + n_part * c->head_dim * sizeof(float));
+  const uint64_t q_bytes = (uint64_t)c->max_batch * c->n_q_heads * c->head_dim * d->elem;
+  const uint64_t kv_bytes = (uint64_t)c->max_batch * d->D * d->elem;
+  d->off_q = off; off = align_up(off + q_bytes);
+  d->off_k = off; off = align_up(off + kv_bytes);
+  d->off_v = off; off = align_up(off + kv_bytes);
+  d->off_out = off; off = align_up(off + (uint64_t)c->max_batch * c->n_q_heads * c->head_dim * 4);
+  d->off_lens = off; off = align_up(off + (uint64_t)c->max_batch * 4);
+  d->off_pos = off; off = align_up(off + (uint64_t)c->max_batch * 4);
+  d->total = off;
+  return ECHOKV_OK;
+}
+
+struct Layer {
+  void* k_pool = nullptr;
+  void* v_pool = nullptr;
+  const void* Wk = nullptr;
+  const void* Wv = nullptr;
+  const void* bk = nullptr;
+  const void* bv = nullptr;
+  bool anchor = false;
+  TcLayerMaps tc;     // tensor maps of the tensor-core path (valid when tc.ready)
+};
+
+}  // namespace
+
+struct echokv_ctx {
+  echokv_config cfg;
+  Derived d;
+  std::vector<Layer> layers;
+  const int32_t* table = nullptr;
+  unsigned char* ws = nullptr;
+  int sm_count = 0;
+  int path = 0;          // see echokv_decode_path
+  bool tc_capable = false;
+  int64_t launches = 0;
+  float scale = 0.f;
+  std::vector<int32_t> pos_scratch;
+};
+
+namespace {
+
+int32_t* status_ptr(echokv_ctx* c) { return reinterpret_cast<int32_t*>(c->ws + c->d.off_status); }
+
+PageGeom geom_of(const echokv_ctx* c) {
+  PageGeom g;
+  g.table = c->table;
+  g.max_batch = c->cfg.max_batch;
+  g.max_pages_per_seq = c->cfg.max_pages_per_seq;
+  g.page_tokens = c->cfg.page_tokens;
+  g.n_pages = c->cfg.n_pages;
+  return g;
+}
+
+AttnArgs attn_args(echokv_ctx* c, const void* q, const int32_t* slots, const int32_t* lens, int B) {
+  AttnArgs a;
+  a.dtype = c->cfg.dtype;
+  a.n_q_heads = c->cfg.n_q_heads;
+  a.n_kv_heads = c->cfg.n_kv_heads;
+  a.head_dim = c->cfg.head_dim;
+  a.batch = B;
+  a.scale_log2e = c->scale * kLog2e;
+  a.q = q;
+  a.slots = slots;
+  a.lens = lens;
+  a.geom = geom_of(c);
+  a.parts.ml = reinterpret_cast<float2*>(c->ws + c->d.off_ml);
+  a.parts.o = reinterpret_cast<float*>(c->ws + c->d.off_o);
+  a.parts.max_parts = c->d.max_parts;
+  a.status = status_ptr(c);
+  return a;
+}
+
+int stored_splits(const echokv_ctx* c, int B, int n_heads) {
+  if (n_heads <= 0) return 1;
+  const int ctas = B * n_heads;
+  int n = (4 * c->sm_count + ctas - 1) / ctas;
+  if (n > c->d.max_parts) n = c->d.max_parts;
+  if (n > c->cfg.max_pages_per_seq) n = c->cfg.max_pages_per_seq;
+  if (n < 1) n = 1;
+  return n;
+}
+
+int check_call(echokv_ctx* c, int layer, const void* q, const float* out, const int32_t* lens, int B) {
+  if (!c || !q || !out || !lens) return ECHOKV_EINVAL;
+  if (layer < 0 || layer >= c->cfg.n_layers || B < 1) return ECHOKV_EINVAL;
+  if (B > c->cfg.max_batch) return ECHOKV_ECAPACITY;
+  if (!c->table) return ECHOKV_ENOTABLE;
+  return ECHOKV_OK;
+}
+
+int attend_stored_layer(echokv_ctx* c, const Layer& L, const void* q, float* out,
+                        const int32_t* slots, const int32_t* lens, int B, cudaStream_t s) {
+  AttnArgs a = attn_args(c, q, slots, lens, B);
+  const int H = c->cfg.n_kv_heads;
+  const int n_splits = stored_splits(c, B, H);
+  if (launch_attn_stored(a, L.k_pool, L.v_pool, c->d.D, H, n_splits, s) != cudaSuccess) return ECHOKV_ECUDA;
+  if (launch_merge(a, out, H, n_splits, c->d.part_tokens, nullptr, s) != cudaSuccess) return ECHOKV_ECUDA;
+  c->launches += 2;
+  return ECHOKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int echokv_query_sizes(const echokv_config* cfg, echokv_sizes* out) {
+  if (!out) return ECHOKV_EINVAL;
+  Derived d;
+  const int rc = derive(cfg, &d);
+  if (rc != ECHOKV_OK) return rc;
+  const uint64_t rows = (uint64_t)cfg->n_pages * cfg->page_tokens;
+  out->anchor_pool_bytes = rows * d.D * d.elem;
+  out->compressed_pool_bytes = rows * d.m * d.elem;
+  out->block_table_bytes = (uint64_t)cfg->max_batch * cfg->max_pages_per_seq * 4;
+  out->workspace_bytes = d.total;
+  out->max_partials = d.max_parts;
+  out->reserved = 0;
+  return ECHOKV_OK;
+}
+
+int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ctx** out) {
+  if (!out) return ECHOKV_EINVAL;
+  *out = nullptr;
+  Derived d;
+  int rc = derive(cfg, &d);
+  if (rc != ECHOKV_OK) return rc;
+  if (!buf || !buf->k_pools || !buf->v_pools || !buf->workspace) return ECHOKV_EINVAL;
+  if (buf->workspace_bytes < d.total) return ECHOKV_ECAPACITY;
+  if (reinterpret_cast<uintptr_t>(buf->workspace) % kAlign != 0) return ECHOKV_EINVAL;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const bool anchor = l % cfg->group_size == 0;
+    const bool needs_pool = anchor || d.m > 0;
+    if (needs_pool && (!buf->k_pools[l] || !buf->v_pools[l])) return ECHOKV_EINVAL;
+    if (needs_pool && (reinterpret_cast<uintptr_t>(buf->k_pools[l]) % 16 != 0 ||
+                       reinterpret_cast<uintptr_t>(buf->v_pools[l]) % 16 != 0))
+      return ECHOKV_EINVAL;
+  }
+  echokv_ctx* c = new (std::nothrow) echokv_ctx();
+  if (!c) return ECHOKV_EINVAL;
+  c->cfg = *cfg;
+  c->d = d;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  c->ws = static_cast<unsigned char*>(buf->workspace);
+  c->layers.resize(cfg->n_layers);
+  bool any_compressed = false;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    c->layers[l].anchor = l % cfg->group_size == 0;
+    c->layers[l].k_pool = buf->k_pools[l];
+    c->layers[l].v_pool = buf->v_pools[l];
+    any_compressed |= !c->layers[l].anchor;
+  }
+  if (cudaSetDevice(cfg->device) != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
+  if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) {
+    delete c;
+    return ECHOKV_ECUDA;
+  }
+  if (cudaMemset(c->ws + d.off_status, 0, kAlign) != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
+  c->tc_capable = tc_shape_supported(cfg->dtype, cfg->head_dim, cfg->page_tokens, d.D, d.m);
+  if (!any_compressed || d.d_drop == 0) c->path = 0;
+  else c->path = c->tc_capable ? 2 : 1;
+  if (c->tc_capable) {
+    // tensor maps of every pool (the predictors' maps follow in echokv_set_weights)
+    for (int l = 0; l < cfg->n_layers; ++l) {
+      Layer& L = c->layers[l];
+      const int width = L.anchor ? d.D : d.m;
+      if (width == 0) continue;
+      const cudaError_t e = tc_encode_pool_maps(&L.tc, L.k_pool, L.v_pool, width,
+                                                (uint64_t)cfg->n_pages * cfg->page_tokens,
+                                                cfg->page_tokens);
+      if (e != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
+    }
+  }
+  *out = c;
+  return ECHOKV_OK;
+}
+
+void echokv_destroy(echokv_ctx* ctx) { delete ctx; }
+
+int echokv_set_weights(echokv_ctx* c, int layer, const void* Wk, const void* Wv, const void* bk,
+                       const void* bv) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return ECHOKV_EINVAL;
+  Layer& L = c->layers[layer];
+  if (L.anchor) return ECHOKV_ENOTCOMPRESSED;
+  if (c->d.d_drop > 0 && (!Wk || !Wv)) return ECHOKV_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(Wk) | reinterpret_cast<uintptr_t>(Wv)) % 16 != 0) return ECHOKV_EINVAL;
+  L.Wk = Wk; L.Wv = Wv; L.bk = bk; L.bv = bv;
+  if (c->tc_capable && c->d.d_drop > 0) {
+    if (tc_encode_weight_maps(&L.tc, Wk, Wv, c->d.d_drop, c->d.d_in) != cudaSuccess) return ECHOKV_ECUDA;
+  }
+  return ECHOKV_OK;
+}
+
+int echokv_set_block_table(echokv_ctx* c, const int32_t* dev_block_table) {
+  if (!c || !dev_block_table) return ECHOKV_EINVAL;
+  c->table = dev_block_table;
+  return ECHOKV_OK;
+}
+
+int echokv_set_decode_path(echokv_ctx* c, int path) {
+  if (!c) return ECHOKV_EINVAL;
+  if (c->path == 0) return path == 0 ? ECHOKV_OK : ECHOKV_EINVAL;
+  if (path == 1) { c->path = 1; return ECHOKV_OK; }
+  if (path == 2) {
+    if (!c->tc_capable) return ECHOKV_EUNSUPPORTED;
+    c->path = 2;
+    return ECHOKV_OK;
+  }
+  return ECHOKV_EINVAL;
+}
+
+int echokv_append_kv(echokv_ctx* c, int layer, const void* k_new, const void* v_new,
+                     const int32_t* dev_seq_slots, const int32_t* dev_positions, int B, void* stream) {
+  if (!c || !k_new || !v_new || !dev_positions) return ECHOKV_EINVAL;
+  if (layer < 0 || layer >= c->cfg.n_layers || B < 1) return ECHOKV_EINVAL;
+  if (B > c->cfg.max_batch) return ECHOKV_ECAPACITY;
+  if (!c->table) return ECHOKV_ENOTABLE;
+  const Layer& L = c->layers[layer];
+  const int width = L.anchor ? c->d.D : c->d.m;
+  if (width == 0) return ECHOKV_OK;   // nothing of this layer is kept (m = 0)
+  const cudaError_t e = launch_append(c->cfg.dtype, L.k_pool, L.v_pool, width, c->d.D, k_new, v_new,
+                                      dev_seq_slots, dev_positions, B, geom_of(c), status_ptr(c),
+                                      static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return ECHOKV_ECUDA;
+  c->launches += 1;
+  return ECHOKV_OK;
+}
+
+int echokv_full_attention(echokv_ctx* c, int layer, const void* q, float* out,
+                          const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                          void* stream) {
+  const int rc = check_call(c, layer, q, out, dev_seq_lens, B);
+  if (rc != ECHOKV_OK) return rc;
+  const Layer& L = c->layers[layer];
+  if (!L.anchor && c->d.d_drop != 0) return ECHOKV_ENOTANCHOR;
+  return attend_stored_layer(c, L, q, out, dev_seq_slots, dev_seq_lens, B,
+                             static_cast<cudaStream_t>(stream));
+}
+
+int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
+                            const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                            void* stream) {
+  const int rc = check_call(c, layer, q, out, dev_seq_lens, B);
+  if (rc != ECHOKV_OK) return rc;
+  const Layer& L = c->layers[layer];
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (L.anchor || c->d.d_drop == 0)
+    return attend_stored_layer(c, L, q, out, dev_seq_slots, dev_seq_lens, B, s);
+  if (!L.Wk || !L.Wv) return ECHOKV_ENOWEIGHTS;
+  const Layer& A = c->layers[layer - layer % c->cfg.group_size];
+  AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
+  const int r = c->cfg.n_retained_heads;
+  // retained heads: Eq. 7 on what is stored (Eq. 6 keeps them as they are)
+  const int n_splits = stored_splits(c, B, r);
+  if (r > 0) {
+    if (launch_attn_stored(a, L.k_pool, L.v_pool, c->d.m, r, n_splits, s) != cudaSuccess) return ECHOKV_ECUDA;
+    c->launches += 1;
+  }
+  // dropped heads: predict (Eq. 3) and attend (Eq. 7) on chip
+  ReconArgs ra;
+  ra.k_anchor = A.k_pool; ra.v_anchor = A.v_pool;
+  ra.k_local = L.k_pool; ra.v_local = L.v_pool;
+  ra.Wk = L.Wk; ra.Wv = L.Wv;
+  ra.D = c->d.D; ra.m = c->d.m;
+  ra.part_tokens = c->d.part_tokens;
+  ra.capacity_tokens = c->d.capacity;
+  cudaError_t e;
+  if (c->path == 2) {
+    e = launch_recon_tc(a, ra, A.tc, L.tc, c->sm_count, s);
+  } else {
+    e = launch_recon_simt(a, ra, s);
+  }
+  if (e != cudaSuccess) return ECHOKV_ECUDA;
+  if (launch_merge(a, out, r, n_splits, c->d.part_tokens, L.bv, s) != cudaSuccess) return ECHOKV_ECUDA;
+  c->launches += 2;
+  return ECHOKV_OK;
+}
+
+int echokv_layer_step_host(echokv_ctx* c, int layer, const void* q_host, const void* k_new_host,
+                           const void* v_new_host, float* out_host, const int32_t* seq_lens_host,
+                           int B, int attend, void* stream) {
+  if (!c || !k_new_host || !v_new_host || !seq_lens_host) return ECHOKV_EINVAL;
+  if (attend && (!q_host || !out_host)) return ECHOKV_EINVAL;
+  if (layer < 0 || layer >= c->cfg.n_layers || B < 1) return ECHOKV_EINVAL;
+  if (B > c->cfg.max_batch) return ECHOKV_ECAPACITY;
+  if (!c->table) return ECHOKV_ENOTABLE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const Derived& d = c->d;
+  void* dq = c->ws + d.off_q;
+  void* dk = c->ws + d.off_k;
+  void* dv = c->ws + d.off_v;
+  float* dout = reinterpret_cast<float*>(c->ws + d.off_out);
+  int32_t* dlens = reinterpret_cast<int32_t*>(c->ws + d.off_lens);
+  int32_t* dpos = reinterpret_cast<int32_t*>(c->ws + d.off_pos);
+  const size_t q_bytes = (size_t)B * c->cfg.n_q_heads * c->cfg.head_dim * d.elem;
+  const size_t kv_bytes = (size_t)B * d.D * d.elem;
+  c->pos_scratch.resize(B);
+  for (int b = 0; b < B; ++b) c->pos_scratch[b] = seq_lens_host[b] - 1;
+  bool ok = true;
+  ok &= cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dlens, seq_lens_host, (size_t)B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dpos, c->pos_scratch.data(), (size_t)B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (attend) ok &= cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (!ok) return ECHOKV_ECUDA;
+  int rc = echokv_append_kv(c, layer, dk, dv, nullptr, dpos, B, stream);
+  if (rc != ECHOKV_OK) return rc;
+  if (attend) {
+    rc = echokv_decode_attention(c, layer, dq, dout, nullptr, dlens, B, stream);
+    if (rc != ECHOKV_OK) return rc;
+    if (cudaMemcpyAsync(out_host, dout, (size_t)B * c->cfg.n_q_heads * c->cfg.head_dim * 4,
+                        cudaMemcpyDeviceToHost, s) != cudaSuccess)
+      return ECHOKV_ECUDA;
+  }
+  if (cudaStreamSynchronize(s) != cudaSuccess) return ECHOKV_ECUDA;
+  return ECHOKV_OK;
+}
+
+int echokv_get_device_status(echokv_ctx* c, int32_t* host_out) {
+  if (!c || !host_out) return ECHOKV_EINVAL;
+  if (cudaDeviceSynchronize() != cudaSuccess) return ECHOKV_ECUDA;
+  int32_t v = 0;
+  if (cudaMemcpy(&v, status_ptr(c), 4, cudaMemcpyDeviceToHost) != cudaSuccess) return ECHOKV_ECUDA;
+  if (v != 0 && cudaMemset(status_ptr(c), 0, 4) != cudaSuccess) return ECHOKV_ECUDA;
+  *host_out = v;
+  return ECHOKV_OK;
+}
+
+int64_t echokv_launch_count(const echokv_ctx* c) { return c ? c->launches : 0; }
+
+int echokv_decode_path(const echokv_ctx* c) { return c ? c->path : 0; }
+
+const char* echokv_strerror(int status) {
+  switch (status) {
+    case ECHOKV_OK: return "ok";
+    case ECHOKV_EINVAL: return "invalid argument";
+    case ECHOKV_ENOTANCHOR: return "layer does not hold a full cache";
+    case ECHOKV_ENOTCOMPRESSED: return "layer is an anchor layer and has no predictor";
+    case ECHOKV_ECAPACITY: return "batch, workspace or length beyond the configured capacity";
+    case ECHOKV_ENOWEIGHTS: return "predictor weights of the layer were not set";
+    case ECHOKV_ECUDA: return "a CUDA call failed";
+    case ECHOKV_ETIMEOUT: return "device: a bounded wait ran out";
+    case ECHOKV_EBADPAGE: return "device: page id or sequence slot out of range";
+    case ECHOKV_EUNSUPPORTED: return "shape not supported by the kernels";
+    case ECHOKV_ENOTABLE: return "block table was not set";
+    case ECHOKV_EBADLENGTH: return "device: sequence length below 1 or beyond capacity";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

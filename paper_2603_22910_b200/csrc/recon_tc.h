@@ -1,0 +1,30 @@
+// Tensor-core (tcgen05 / TMEM / TMA) reconstruct-then-attend path: host interface.
+#pragma once
+
+#include <cuda.h>
+
+#include "kernels.h"
+
+namespace echokv {
+
+// TMA descriptors of one layer: its K and V pools (boxes of one page x 64 features) and, for a
+// compressed layer, its two predictors (boxes of 256 rows x 64 input features).
+struct TcLayerMaps {
+  CUtensorMap k_pool, v_pool, wk, wv;
+  bool pools_ready = false;
+  bool weights_ready = false;
+};
+
+bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m);
+
+cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const void* v_pool, int width,
+                                uint64_t rows, int page_tokens);
+
+cudaError_t tc_encode_weight_maps(TcLayerMaps* maps, const void* Wk, const void* Wv, int d_drop,
+                                  int d_in);
+
+// Dropped heads of one compressed layer: Eq. 3 on the tensor cores, Eq. 7 on the accumulators.
+cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                            const TcLayerMaps& layer, int sm_count, cudaStream_t stream);
+
+}  // namespace echokv

@@ -1,0 +1,499 @@
+// CUDA-core kernels of the EchoKV decode path: cache append, attention over stored heads
+// (anchor layers, retained heads), the fp32-FFMA reconstruct-then-attend kernel that serves the
+// fp32 test mode and shapes the tensor-core kernel does not take, and the split-K merge.
+#include "kernels.h"
+
+namespace echokv {
+
+// ---------------------------------------------------------------------------------------------
+// Append (Section 3.1: the dropped dims of a compressed layer are simply not written; Eq. 2)
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) append_kernel(T* __restrict__ k_pool, T* __restrict__ v_pool,
+                                                     int width, int D, const T* __restrict__ k_new,
+                                                     const T* __restrict__ v_new,
+                                                     const int32_t* __restrict__ slots,
+                                                     const int32_t* __restrict__ positions,
+                                                     PageGeom g, int32_t* status) {
+  const int b = blockIdx.x;
+  const int slot = slots ? slots[b] : b;
+  const int pos = positions[b];
+  if (slot < 0 || slot >= g.max_batch || pos < 0 || pos >= g.max_pages_per_seq * g.page_tokens) {
+    if (threadIdx.x == 0) report(status, ECHOKV_EBADPAGE);
+    return;
+  }
+  const int page = g.table[(size_t)slot * g.max_pages_per_seq + pos / g.page_tokens];
+  if (page < 0 || page >= g.n_pages) {
+    if (threadIdx.x == 0) report(status, ECHOKV_EBADPAGE);
+    return;
+  }
+  const size_t row = ((size_t)page * g.page_tokens + pos % g.page_tokens) * (size_t)width;
+  constexpr int kVec = 16 / sizeof(T);
+  const int n_vec = width / kVec;
+  const uint4* ks = reinterpret_cast<const uint4*>(k_new + (size_t)b * D);
+  const uint4* vs = reinterpret_cast<const uint4*>(v_new + (size_t)b * D);
+  uint4* kd = reinterpret_cast<uint4*>(k_pool + row);
+  uint4* vd = reinterpret_cast<uint4*>(v_pool + row);
+  for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
+    kd[i] = ks[i];
+    vd[i] = vs[i];
+  }
+}
+
+cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int width, int D, const void* k_new,
+                          const void* v_new, const int32_t* slots, const int32_t* positions, int B,
+                          const PageGeom& geom, int32_t* status, cudaStream_t stream) {
+  if (dtype == ECHOKV_BF16) {
+    append_kernel<__nv_bfloat16><<<B, 128, 0, stream>>>(
+        (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, width, D, (const __nv_bfloat16*)k_new,
+        (const __nv_bfloat16*)v_new, slots, positions, geom, status);
+  } else {
+    append_kernel<float><<<B, 128, 0, stream>>>((float*)k_pool, (float*)v_pool, width, D,
+                                                (const float*)k_new, (const float*)v_new, slots,
+                                                positions, geom, status);
+  }
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention over stored heads (Eq. 7 on the cache as stored): one warp per token row.
+// ---------------------------------------------------------------------------------------------
+template <typename T, int EPL>
+__device__ __forceinline__ void load_row_slice(const T* p, float (&out)[EPL]) {
+  if constexpr (sizeof(T) * EPL == 16) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    if constexpr (sizeof(T) == 4) {
+      out[0] = __uint_as_float(v.x); out[1] = __uint_as_float(v.y);
+      out[2] = __uint_as_float(v.z); out[3] = __uint_as_float(v.w);
+    }
+  } else if constexpr (sizeof(T) * EPL == 8) {
+    uint2 v = *reinterpret_cast<const uint2*>(p);
+    if constexpr (sizeof(T) == 4) {
+      out[0] = __uint_as_float(v.x); out[1] = __uint_as_float(v.y);
+    } else {
+      out[0] = __uint_as_float(v.x << 16); out[1] = __uint_as_float(v.x & 0xffff0000u);
+      out[2] = __uint_as_float(v.y << 16); out[3] = __uint_as_float(v.y & 0xffff0000u);
+    }
+  } else {
+    static_assert(sizeof(T) * EPL == 4, "row slice of 4, 8 or 16 bytes");
+    uint32_t v = *reinterpret_cast<const uint32_t*>(p);
+    out[0] = __uint_as_float(v << 16); out[1] = __uint_as_float(v & 0xffff0000u);
+  }
+}
+
+template <typename T, int DH, int G>
+__global__ void __launch_bounds__(128) attn_stored_kernel(AttnArgs a, const T* __restrict__ k_pool,
+                                                          const T* __restrict__ v_pool, int width,
+                                                          int n_splits) {
+  constexpr int EPL = DH / 32;
+  constexpr int U = 4;   // tokens in flight per warp
+  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ float sm_m[4][G], sm_l[4][G];
+  __shared__ float sm_o[4][G][DH];
+
+  int slot, len;
+  {
+    int32_t* st = threadIdx.x == 0 ? a.status : nullptr;
+    slot = a.slots ? a.slots[b] : b;
+    len = a.lens[b];
+    const bool bad_slot = slot < 0 || slot >= a.geom.max_batch;
+    const bool bad_len = len < 1 || len > a.geom.max_pages_per_seq * a.geom.page_tokens;
+    if (bad_slot || bad_len) {
+      if (st) report(st, bad_slot ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
+      return;
+    }
+  }
+  const int P = a.geom.page_tokens;
+  const int n_pages_seq = (len + P - 1) / P;
+  const int pages_per_split = (n_pages_seq + n_splits - 1) / n_splits;
+  const int t0 = split * pages_per_split * P;
+  const int t1 = min(len, (split + 1) * pages_per_split * P);
+  const int32_t* table = a.geom.table + (size_t)slot * a.geom.max_pages_per_seq;
+
+  float qr[G][EPL];
+  const T* q = reinterpret_cast<const T*>(a.q);
+#pragma unroll
+  for (int gi = 0; gi < G; ++gi) {
+    float tmp[EPL];
+    load_row_slice<T, EPL>(q + ((size_t)b * a.n_q_heads + kvh * G + gi) * DH + lane * EPL, tmp);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) qr[gi][e] = tmp[e] * a.scale_log2e;
+  }
+  float m[G], l[G], o[G][EPL];
+#pragma unroll
+  for (int gi = 0; gi < G; ++gi) {
+    m[gi] = -INFINITY;
+    l[gi] = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) o[gi][e] = 0.f;
+  }
+
+  for (int tb = t0 + warp * U; tb < t1; tb += 4 * U) {
+    float kx[U][EPL], vx[U][EPL];
+    bool valid[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int t = tb + u;
+      valid[u] = t < t1;
+      if (valid[u]) {
+        const int page = table[t / P];
+        if (page < 0 || page >= a.geom.n_pages) {
+          if (lane == 0) report(a.status, ECHOKV_EBADPAGE);
+          valid[u] = false;
+        } else {
+          const size_t off = ((size_t)page * P + t % P) * (size_t)width + kvh * DH + lane * EPL;
+          load_row_slice<T, EPL>(k_pool + off, kx[u]);
+          load_row_slice<T, EPL>(v_pool + off, vx[u]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (!valid[u]) continue;   // warp-uniform
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) {
+        float s = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) s = fmaf(qr[gi][e], kx[u][e], s);
+        s = warp_sum(s);
+        const float m_new = fmaxf(m[gi], s);
+        const float alpha = exp2f(m[gi] - m_new);
+        const float p = exp2f(s - m_new);
+        l[gi] = l[gi] * alpha + p;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) o[gi][e] = fmaf(p, vx[u][e], o[gi][e] * alpha);
+        m[gi] = m_new;
+      }
+    }
+  }
+
+#pragma unroll
+  for (int gi = 0; gi < G; ++gi) {
+    if (lane == 0) {
+      sm_m[warp][gi] = m[gi];
+      sm_l[warp][gi] = l[gi];
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) sm_o[warp][gi][lane * EPL + e] = o[gi][e];
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < G * DH; idx += 128) {
+    const int gi = idx / DH, j = idx % DH;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) M = fmaxf(M, sm_m[w][gi]);
+    float L = 0.f, acc = 0.f;
+    if (M > -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float wgt = exp2f(sm_m[w][gi] - M);
+        L += wgt * sm_l[w][gi];
+        acc += wgt * sm_o[w][gi][j];
+      }
+    }
+    const size_t pidx = ((size_t)b * a.n_q_heads + kvh * G + gi) * a.parts.max_parts + split;
+    a.parts.o[pidx * DH + j] = acc;
+    if (j == 0) a.parts.ml[pidx] = make_float2(M, L);
+  }
+}
+
+template <typename T, int DH>
+static cudaError_t launch_attn_stored_g(const AttnArgs& a, const void* k_pool, const void* v_pool,
+                                        int width, int n_heads, int n_splits, cudaStream_t stream) {
+  const int g = a.n_q_heads / a.n_kv_heads;
+  dim3 grid(n_splits, n_heads, a.batch);
+  const T* kp = (const T*)k_pool;
+  const T* vp = (const T*)v_pool;
+  switch (g) {
+    case 1: attn_stored_kernel<T, DH, 1><<<grid, 128, 0, stream>>>(a, kp, vp, width, n_splits); break;
+    case 2: attn_stored_kernel<T, DH, 2><<<grid, 128, 0, stream>>>(a, kp, vp, width, n_splits); break;
+    case 4: attn_stored_kernel<T, DH, 4><<<grid, 128, 0, stream>>>(a, kp, vp, width, n_splits); break;
+    case 8: attn_stored_kernel<T, DH, 8><<<grid, 128, 0, stream>>>(a, kp, vp, width, n_splits); break;
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_stored(const AttnArgs& a, const void* k_pool, const void* v_pool, int width,
+                               int n_heads, int n_splits, cudaStream_t stream) {
+  if (n_heads == 0) return cudaSuccess;
+  if (a.dtype == ECHOKV_BF16) {
+    if (a.head_dim == 128)
+      return launch_attn_stored_g<__nv_bfloat16, 128>(a, k_pool, v_pool, width, n_heads, n_splits, stream);
+    return launch_attn_stored_g<__nv_bfloat16, 64>(a, k_pool, v_pool, width, n_heads, n_splits, stream);
+  }
+  if (a.head_dim == 128)
+    return launch_attn_stored_g<float, 128>(a, k_pool, v_pool, width, n_heads, n_splits, stream);
+  return launch_attn_stored_g<float, 64>(a, k_pool, v_pool, width, n_heads, n_splits, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// CUDA-core reconstruct-then-attend (Eq. 3, 6, 7 for one dropped KV head and one token range)
+// ---------------------------------------------------------------------------------------------
+constexpr int kKc = 32;   // features per staged chunk of the predictor input
+
+template <int DH>
+struct ReconSmem {
+  float Xs[kKc][kSimtTileTokens];          // predictor-input chunk, [feature][token]
+  float Ws[kKc][DH];                       // predictor chunk, [feature][output dim of the head]
+  float Hs[kSimtTileTokens][DH + 1];       // predicted K (then V) tile of the head
+  float Ss[kMaxGroup][kSimtTileTokens];    // scores, then probabilities
+  float qs[kMaxGroup][DH];                 // queries * scale * log2e
+  float m_run[kMaxGroup], l_run[kMaxGroup], alpha[kMaxGroup];
+};
+
+// acc[8 tokens][FPT feats] += X[tile tokens][D_in] * W_head[DH][D_in]^T for one 64-token tile
+template <typename T, int DH>
+__device__ __forceinline__ void predict_tile(ReconSmem<DH>& sm, const T* __restrict__ anchor_pool,
+                                             const T* __restrict__ local_pool,
+                                             const T* __restrict__ W_head, int D, int m,
+                                             const int32_t* __restrict__ table, const PageGeom& g,
+                                             int tile_t0, int len, int32_t* status) {
+  constexpr int FPT = DH / 16;
+  constexpr int KPT = kKc * DH / 128;          // predictor k-values loaded per thread and chunk
+  constexpr int VN = Vec16<T>::N;
+  const int tid = threadIdx.x;
+  const int tx = tid % 16, ty = tid / 16;
+  float acc[8][FPT];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < FPT; ++j) acc[i][j] = 0.f;
+
+  // this thread stages 16 features of token (tid / 2)
+  const int ld_tok = tid / 2, ld_half = tid % 2;
+  const int t_glob = tile_t0 + ld_tok;
+  long long row = -1;   // row index inside a pool, or -1 for a padding token
+  if (t_glob < len) {
+    const int page = table[t_glob / g.page_tokens];
+    if (page < 0 || page >= g.n_pages) {
+      report(status, ECHOKV_EBADPAGE);
+    } else {
+      row = (long long)page * g.page_tokens + t_glob % g.page_tokens;
+    }
+  }
+  const int w_row = tid % DH, w_part = tid / DH;
+  const int d_in = D + m;
+
+  for (int kc = 0; kc < d_in; kc += kKc) {
+    // stage X chunk (transposed) and W chunk (transposed)
+    {
+      float xv[16];
+      if (row >= 0) {
+        const T* src = kc < D ? anchor_pool + row * D + kc : local_pool + row * m + (kc - D);
+        src += ld_half * 16;
+#pragma unroll
+        for (int v = 0; v < 16 / VN; ++v) Vec16<T>::load(src + v * VN, xv + v * VN);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) xv[e] = 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < 16; ++e) sm.Xs[ld_half * 16 + e][ld_tok] = xv[e];
+      float wv[KPT];
+      const T* wsrc = W_head + (size_t)w_row * d_in + kc + w_part * KPT;
+#pragma unroll
+      for (int v = 0; v < KPT / VN; ++v) Vec16<T>::load(wsrc + v * VN, wv + v * VN);
+#pragma unroll
+      for (int e = 0; e < KPT; ++e) sm.Ws[w_part * KPT + e][w_row] = wv[e];
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int k = 0; k < kKc; ++k) {
+      float xr[8], wr[FPT];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) xr[i] = sm.Xs[k][ty * 8 + i];
+#pragma unroll
+      for (int j = 0; j < FPT; ++j) wr[j] = sm.Ws[k][tx * FPT + j];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < FPT; ++j) acc[i][j] = fmaf(xr[i], wr[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < FPT; ++j) sm.Hs[ty * 8 + i][tx * FPT + j] = acc[i][j];
+}
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  ReconSmem<DH>& sm = *reinterpret_cast<ReconSmem<DH>*>(smem_raw);
+  const int part = blockIdx.x, b = blockIdx.z;
+  const int n_ret = r.m / DH;
+  const int kvh = n_ret + blockIdx.y;                 // dropped KV head
+  const int g = a.n_q_heads / a.n_kv_heads;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  const int slot = a.slots ? a.slots[b] : b;
+  const int len = a.lens[b];
+  if (slot < 0 || slot >= a.geom.max_batch) {
+    if (tid == 0) report(a.status, ECHOKV_EBADPAGE);
+    return;
+  }
+  if (len < 1 || len > r.capacity_tokens) {
+    if (tid == 0) report(a.status, ECHOKV_EBADLENGTH);
+    return;
+  }
+  const int part_t0 = part * r.part_tokens;
+  if (part_t0 >= len) return;
+  const int32_t* table = a.geom.table + (size_t)slot * a.geom.max_pages_per_seq;
+
+  const T* q = reinterpret_cast<const T*>(a.q);
+  for (int idx = tid; idx < g * DH; idx += 128) {
+    const int gi = idx / DH, j = idx % DH;
+    sm.qs[gi][j] = to_f32(q[((size_t)b * a.n_q_heads + kvh * g + gi) * DH + j]) * a.scale_log2e;
+  }
+  if (tid < kMaxGroup) {
+    sm.m_run[tid] = -INFINITY;
+    sm.l_run[tid] = 0.f;
+  }
+  float o[kMaxGroup];
+#pragma unroll
+  for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
+  __syncthreads();
+
+  const size_t w_off = (size_t)(kvh - n_ret) * DH * (r.D + r.m);
+  const T* Wk_head = reinterpret_cast<const T*>(r.Wk) + w_off;
+  const T* Wv_head = reinterpret_cast<const T*>(r.Wv) + w_off;
+  const int tiles = r.part_tokens / kSimtTileTokens;
+
+  for (int tile = 0; tile < tiles; ++tile) {
+    const int tile_t0 = part_t0 + tile * kSimtTileTokens;
+    if (tile_t0 >= len) break;
+    // K_hat tile (Eq. 3) -> Hs
+    predict_tile<T, DH>(sm, (const T*)r.k_anchor, (const T*)r.k_local, Wk_head, r.D, r.m, table,
+                        a.geom, tile_t0, len, a.status);
+    __syncthreads();
+    // scores of the group's query heads (Eq. 7), base-2 units
+    {
+      const int t = tid % kSimtTileTokens;
+      for (int gi = tid / kSimtTileTokens; gi < g; gi += 128 / kSimtTileTokens) {
+        float s = 0.f;
+#pragma unroll 8
+        for (int j = 0; j < DH; ++j) s = fmaf(sm.qs[gi][j], sm.Hs[t][j], s);
+        sm.Ss[gi][t] = (tile_t0 + t < len) ? s : -INFINITY;
+      }
+    }
+    __syncthreads();
+    // online softmax update, one warp per query head
+    for (int gi = warp; gi < g; gi += 4) {
+      const float s0 = sm.Ss[gi][lane], s1 = sm.Ss[gi][lane + 32];
+      const float mt = warp_max(fmaxf(s0, s1));
+      const float m_old = sm.m_run[gi];
+      const float m_new = fmaxf(m_old, mt);
+      const float alpha = exp2f(m_old - m_new);
+      const float p0 = exp2f(s0 - m_new), p1 = exp2f(s1 - m_new);
+      const float ls = warp_sum(p0 + p1);
+      sm.Ss[gi][lane] = p0;
+      sm.Ss[gi][lane + 32] = p1;
+      if (lane == 0) {
+        sm.m_run[gi] = m_new;
+        sm.l_run[gi] = sm.l_run[gi] * alpha + ls;
+        sm.alpha[gi] = alpha;
+      }
+    }
+    __syncthreads();   // Hs (K_hat) fully consumed, Ss holds probabilities
+    // V_hat tile (Eq. 3) -> Hs
+    predict_tile<T, DH>(sm, (const T*)r.v_anchor, (const T*)r.v_local, Wv_head, r.D, r.m, table,
+                        a.geom, tile_t0, len, a.status);
+    __syncthreads();
+    if (tid < DH) {
+      for (int gi = 0; gi < g; ++gi) {
+        float acc = o[gi] * sm.alpha[gi];
+#pragma unroll 8
+        for (int t = 0; t < kSimtTileTokens; ++t) acc = fmaf(sm.Ss[gi][t], sm.Hs[t][tid], acc);
+        o[gi] = acc;
+      }
+    }
+    __syncthreads();
+  }
+
+  for (int gi = 0; gi < g; ++gi) {
+    const size_t pidx = ((size_t)b * a.n_q_heads + kvh * g + gi) * a.parts.max_parts + part;
+    if (tid < DH) a.parts.o[pidx * DH + tid] = o[gi];
+    if (tid == 0) a.parts.ml[pidx] = make_float2(sm.m_run[gi], sm.l_run[gi]);
+  }
+}
+
+template <typename T, int DH>
+static cudaError_t launch_recon_simt_t(const AttnArgs& a, const ReconArgs& r, cudaStream_t stream) {
+  const int n_drop = a.n_kv_heads - r.m / DH;
+  const int n_parts = (r.capacity_tokens + r.part_tokens - 1) / r.part_tokens;
+  const size_t smem = sizeof(ReconSmem<DH>);
+  cudaError_t e = cudaFuncSetAttribute(recon_simt_kernel<T, DH>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(n_parts, n_drop, a.batch);
+  recon_simt_kernel<T, DH><<<grid, 128, smem, stream>>>(a, r);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_recon_simt(const AttnArgs& a, const ReconArgs& r, cudaStream_t stream) {
+  if (a.n_q_heads / a.n_kv_heads > kMaxGroup) return cudaErrorInvalidValue;
+  if (a.dtype == ECHOKV_BF16) {
+    if (a.head_dim == 128) return launch_recon_simt_t<__nv_bfloat16, 128>(a, r, stream);
+    return launch_recon_simt_t<__nv_bfloat16, 64>(a, r, stream);
+  }
+  if (a.head_dim == 128) return launch_recon_simt_t<float, 128>(a, r, stream);
+  return launch_recon_simt_t<float, 64>(a, r, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-K merge: log-sum-exp combination of partial (max, sum, weighted V) triples
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads,
+                             int n_stored_parts, int part_tokens, const T* __restrict__ bv) {
+  const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
+  const int DH = a.head_dim;
+  const size_t oidx = ((size_t)b * a.n_q_heads + h) * DH + j;
+  const int slot = a.slots ? a.slots[b] : b;
+  const int len = a.lens[b];
+  if (slot < 0 || slot >= a.geom.max_batch || len < 1 ||
+      len > a.geom.max_pages_per_seq * a.geom.page_tokens) {
+    out[oidx] = 0.f;
+    return;
+  }
+  const int g = a.n_q_heads / a.n_kv_heads;
+  const int kvh = h / g;
+  const bool stored = kvh < n_stored_heads;
+  const int n = stored ? n_stored_parts : (len + part_tokens - 1) / part_tokens;
+  const size_t base = ((size_t)b * a.n_q_heads + h) * a.parts.max_parts;
+  float M = -INFINITY;
+  for (int p = 0; p < n; ++p) M = fmaxf(M, a.parts.ml[base + p].x);
+  float L = 0.f, acc = 0.f;
+  if (M > -INFINITY) {
+    for (int p = 0; p < n; ++p) {
+      const float2 ml = a.parts.ml[base + p];
+      const float w = exp2f(ml.x - M);
+      L = fmaf(w, ml.y, L);
+      acc = fmaf(w, a.parts.o[(base + p) * DH + j], acc);
+    }
+  }
+  float res = L > 0.f ? acc / L : 0.f;
+  // a bias on the V predictor shifts every predicted V row alike, so (sum_t p_t = 1) it adds
+  // to the output unchanged; a bias on the K predictor shifts all scores of a head by the
+  // same amount and cancels in the softmax.
+  if (bv != nullptr && !stored) res += to_f32(bv[(kvh - n_stored_heads) * DH + j]);
+  out[oidx] = res;
+}
+
+cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
+                         int part_tokens, const void* bv, cudaStream_t stream) {
+  dim3 grid(a.n_q_heads, a.batch);
+  if (a.dtype == ECHOKV_BF16) {
+    merge_kernel<__nv_bfloat16><<<grid, a.head_dim, 0, stream>>>(
+        a, out, n_stored_heads, n_stored_parts, part_tokens, (const __nv_bfloat16*)bv);
+  } else {
+    merge_kernel<float><<<grid, a.head_dim, 0, stream>>>(a, out, n_stored_heads, n_stored_parts,
+                                                         part_tokens, (const float*)bv);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace echokv

@@ -1,0 +1,197 @@
+"""GPU parity: the CUDA library (through the C-ABI) against the CPU oracle, element by
+element, on the same seeded stored values."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_22910_b200 import binding, build, synth
+from tests.harness import Case, assert_parity, errors
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.lib()
+
+
+def check_layers(case, what):
+    w = case.w
+    worst = (0.0, 0.0)
+    for l in case.layers:
+        out = case.run(l)
+        ref = case.oracle(l)
+        e = assert_parity(out, ref, w.dtype, "%s layer %d" % (what, l))
+        worst = max(worst, e, key=lambda t: t[1])
+        if w.is_anchor(l):
+            np.testing.assert_array_equal(case.run(l, full=True), out)
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    return worst
+
+
+def test_config0_tiny_fp32_full():
+    case = Case(synth.C0, layers=[0, 1])
+    assert case.ctx.decode_path() == 1
+    check_layers(case, "c0")
+    case.close()
+
+
+SMALL = [
+    # name, base, overrides, lens
+    ("c1_shape", synth.C1, dict(batch=2, context=700), [700, 333]),
+    ("c2_shape", synth.C2, dict(batch=3, context=1000), [1000, 517, 256]),
+    ("c2_shape_pages64", synth.C2, dict(batch=2, context=600, page_tokens=64, random_pages=True), [600, 65]),
+    ("c4_25pct", synth.c4_point(25, 4096, 1), dict(batch=2, context=530), [530, 17]),
+    ("c4_50pct", synth.c4_point(50, 4096, 1), dict(batch=2, context=300, random_pages=True), [300, 299]),
+    ("mha_d64_bf16", synth.C0, dict(dtype="bf16", batch=2, context=200), [200, 77]),
+    ("gqa2_fp32_d128", synth.C0, dict(n_q_heads=8, n_kv_heads=4, head_dim=128, n_retained_heads=1,
+                                      batch=2, context=150), [150, 64]),
+    ("gqa8_bf16", synth.C2, dict(n_q_heads=32, n_kv_heads=4, n_retained_heads=1, batch=1, context=300), [300]),
+]
+
+
+@pytest.mark.parametrize("name,base,over,lens", SMALL, ids=[s[0] for s in SMALL])
+@pytest.mark.parametrize("path", [1, 2])
+def test_small_shapes_against_oracle(name, base, over, lens, path):
+    w = base.replace(**over)
+    case = Case(w, lens=lens, layers=[0, 1])
+    if path == 2 and case.ctx.decode_path() != 2:
+        case.close()
+        pytest.skip("shape is served by the CUDA-core kernel only")
+    case.ctx.set_decode_path(path)
+    check_layers(case, name)
+    case.close()
+
+
+def test_config3_shape_multi_layer_random_pages():
+    # 8 layers = two groups of S = 4; ragged lengths; pool larger than needed, random page order
+    w = synth.C3.replace(n_layers=8, batch=2, context=420)
+    case = Case(w, lens=[420, 131], n_pages=2 * w.pages_per_seq + 13)
+    check_layers(case, "c3_shape")
+    case.close()
+
+
+@pytest.mark.parametrize("r", [0, 8])
+def test_nothing_retained_and_nothing_dropped(r):
+    w = synth.C2.replace(batch=2, context=300, n_retained_heads=r)
+    case = Case(w, lens=[300, 40], layers=[0, 1])
+    assert case.ctx.decode_path() == (0 if r == 8 else case.ctx.decode_path())
+    check_layers(case, "r=%d" % r)
+    if r == 8:   # a layer that drops nothing also serves echokv_full_attention
+        np.testing.assert_array_equal(case.run(1, full=True), case.run(1))
+    case.close()
+
+
+@pytest.mark.parametrize("L", [1, 15, 16, 17, 255, 256, 257])
+def test_short_and_boundary_lengths(L):
+    w = synth.C2.replace(batch=2, context=L + 3, n_retained_heads=4)
+    case = Case(w, lens=[L, L + 3], layers=[0, 1])
+    check_layers(case, "L=%d" % L)
+    case.close()
+
+
+def test_predictor_bias():
+    w = synth.C2.replace(batch=2, context=200)
+    case = Case(w, lens=[200, 31], layers=[1], biases=True)
+    check_layers(case, "bias")
+    nb = Case(w, lens=[200, 31], layers=[1], biases=False)
+    assert errors(case.run(1), nb.run(1))[0] > 1e-3      # the bias is not a no-op
+    case.close(); nb.close()
+
+
+def test_page_order_does_not_change_the_result():
+    w = synth.C2.replace(batch=2, context=333)
+    a = Case(w, lens=[333, 90], layers=[0, 1])
+    b = Case(w.replace(random_pages=True), lens=[333, 90], layers=[0, 1], n_pages=2 * w.pages_per_seq + 5)
+    for l in (0, 1):
+        np.testing.assert_array_equal(a.run(l), b.run(l))
+    a.close(); b.close()
+
+
+def test_sequence_slots_select_block_table_rows():
+    w = synth.C2.replace(batch=3, context=200)
+    case = Case(w, lens=[200, 150, 99], layers=[1])
+    base = case.run(1)
+    dev = case.ctx.device
+    order = [2, 0, 1]
+    slots = torch.tensor(order, dtype=torch.int32, device=dev)
+    q = case.q[1][order].contiguous().to(dev)
+    lens = case.seq_lens[order].contiguous()
+    out = case.ctx.decode_attention(1, q, lens, seq_slots=slots)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out.cpu().numpy(), base[order])
+    case.close()
+
+
+def test_append_writes_only_what_the_layer_keeps():
+    w = synth.C2.replace(batch=2, context=40)
+    case = Case(w, lens=[40, 23], layers=[0, 1])
+    for b, L in enumerate(case.lens):
+        page = int(case.table[b, (L - 1) // w.page_tokens])
+        slot = (L - 1) % w.page_tokens
+        for l, width in ((0, w.D), (1, w.m)):
+            got = case.ctx.k_pools[l][page, slot].cpu()
+            assert got.shape[0] == width
+            assert torch.equal(got, case.host[(l, "k", "new")][b, :width])
+            assert not (got == 777.0).any()
+    case.close()
+
+
+def test_bad_length_and_bad_page_are_reported_not_fatal():
+    w = synth.C2.replace(batch=2, context=100)
+    case = Case(w, lens=[100, 60], layers=[1])
+    good = case.run(1)
+    dev = case.ctx.device
+    q = case.q[1].to(dev)
+    bad_lens = torch.tensor([100, 0], dtype=torch.int32, device=dev)
+    out = case.ctx.decode_attention(1, q, bad_lens)
+    assert case.ctx.device_status() == binding.ECHOKV_EBADLENGTH
+    out = out.cpu().numpy()
+    np.testing.assert_array_equal(out[0], good[0])
+    assert np.all(out[1] == 0.0)
+    too_long = torch.tensor([100, 10 ** 6], dtype=torch.int32, device=dev)
+    case.ctx.decode_attention(1, q, too_long)
+    assert case.ctx.device_status() == binding.ECHOKV_EBADLENGTH
+    # a page id outside the pool: reported, the tokens of that page are skipped, no fault
+    saved = case.ctx.block_table.clone()
+    case.ctx.block_table[1, 1] = 10 ** 6
+    out = case.ctx.decode_attention(1, q, case.seq_lens)
+    assert case.ctx.device_status() == binding.ECHOKV_EBADPAGE
+    assert np.all(np.isfinite(out.cpu().numpy()))
+    case.ctx.block_table.copy_(saved)
+    np.testing.assert_array_equal(case.run(1), good)
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+def test_host_status_codes_on_gpu():
+    w = synth.C2.replace(batch=2, context=64)
+    case = Case(w, lens=[64, 64], layers=[0, 1])
+    ctx, L = case.ctx, binding.lib()
+    q = case.q[1].to(ctx.device)
+    out = torch.empty(q.shape, dtype=torch.float32, device=ctx.device)
+    args = (q.data_ptr(), out.data_ptr(), None, case.seq_lens.data_ptr())
+    assert L.echokv_full_attention(ctx.handle, 1, *args, 2, None) == binding.ECHOKV_ENOTANCHOR
+    assert L.echokv_decode_attention(ctx.handle, 2, *args, 2, None) == binding.ECHOKV_EINVAL
+    assert L.echokv_decode_attention(ctx.handle, 1, *args, 3, None) == binding.ECHOKV_ECAPACITY
+    assert L.echokv_set_weights(ctx.handle, 0, q.data_ptr(), q.data_ptr(), None, None) == binding.ECHOKV_ENOTCOMPRESSED
+    fresh = binding.Context(case.cfg)
+    assert L.echokv_decode_attention(fresh.handle, 1, *args, 2, None) == binding.ECHOKV_ENOWEIGHTS
+    fresh.close(); case.close()
+
+
+def test_layer_step_from_host_memory_matches_device_calls():
+    w = synth.C2.replace(batch=2, context=129)
+    case = Case(w, lens=[129, 70], layers=[0, 1])
+    ref = case.run(1)
+    # replay the last token through the host entry point on a second context
+    other = Case(w, lens=[129, 70], layers=[0, 1])
+    lens_host = torch.tensor(case.lens, dtype=torch.int32).pin_memory()
+    out_host = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32).pin_memory()
+    for l, attend in ((0, False), (1, True)):
+        other.ctx.layer_step_host(l, other.q[1].pin_memory(), other.host[(l, "k", "new")].pin_memory(),
+                                  other.host[(l, "v", "new")].pin_memory(), out_host, lens_host, attend=attend)
+    np.testing.assert_array_equal(out_host.numpy(), ref)
+    case.close(); other.close()
