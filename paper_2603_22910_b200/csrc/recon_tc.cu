@@ -1,8 +1,654 @@
-// placeholder until the tcgen05 kernel lands
+// Fused reconstruct-then-attend on the 5th-generation tensor cores (sm_100a).
+//
+// For every dropped KV head of a compressed layer the predictor of Eq. 3 is a dense
+// contraction over D_in = D + m input features per cached token, so it runs as tcgen05.mma
+// with the accumulators in tensor memory; Eq. 7 is then evaluated straight on the accumulators:
+//
+//   work item  = (sequence b, tile of 256 tokens, pair of dropped heads)
+//   K phase    : acc[half][tok, feat] = X_K[tok, :] . W_K[feat, :]    tokens on TMEM lanes
+//                -> each epilogue thread owns one token row: score = q . row (per query head of
+//                   the group), tile max / exp2 / sum, probabilities go to shared memory
+//   V phase    : acc[head][feat, tok] = W_V[feat, :] . X_V[tok, :]    features on TMEM lanes
+//                -> each epilogue thread owns one output feature: o = sum_tok p[tok] * acc[tok]
+//   result     : one split-K partial (max, sum, o) per item and query head; the merge kernel
+//                combines the tiles of a sequence.
+//
+// Both phases stream the same shared-memory stage: 256 token rows x 64 features of the predictor
+// input (one TMA box per cache page, taken through the block table, from the anchor layer's pool
+// for features < D and from this layer's pool of retained dims after that) and 256 predictor rows
+// x 64 features, all bf16 with the 128-byte swizzle the MMA descriptors expect.  In the K phase the
+// token rows are the A operand (two M = 128 halves) and the predictor rows B (N = 256); in the V
+// phase the roles swap.  The predicted K and V never leave the SM.
+//
+// Warp roles: warp 0 issues TMA, warp 1 issues MMA (and owns the TMEM allocation), warps 2..9 are
+// the epilogue (two per TMEM lane quarter, one per accumulator half).  Every wait is bounded: when
+// one runs out the kernel raises the status word, drains what it started and exits.
 #include "recon_tc.h"
+
+#include <cudaTypedefs.h>
+
 namespace echokv {
-bool tc_shape_supported(int, int, int, int, int) { return false; }
-cudaError_t tc_encode_pool_maps(TcLayerMaps*, const void*, const void*, int, uint64_t, int) { return cudaErrorNotSupported; }
-cudaError_t tc_encode_weight_maps(TcLayerMaps*, const void*, const void*, int, int) { return cudaErrorNotSupported; }
-cudaError_t launch_recon_tc(const AttnArgs&, const ReconArgs&, const TcLayerMaps&, const TcLayerMaps&, int, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kStages = 3;
+constexpr int kTileTokens = kTcPartTokens;           // 256
+constexpr int kChunk = 64;                           // features per stage (128 bytes of bf16)
+constexpr int kRowBytes = kChunk * 2;                // 128
+constexpr int kXBytes = kTileTokens * kRowBytes;     // 32 KiB
+constexpr int kWRows = 256;                          // predictor rows per stage: two heads
+constexpr int kWBytes = kWRows * kRowBytes;          // 32 KiB
+constexpr int kStageBytes = kXBytes + kWBytes;       // 64 KiB
+constexpr int kThreads = 320;
+constexpr int kEpilogueThreads = 256;
+constexpr int kMaxBatchPerLaunch = 256;
+constexpr int kTmemCols = 512;
+constexpr long long kWaitLimitCycles = 2000000000ll;   // ~1 s: far beyond any legitimate wait
+
+struct TcParams {
+  const __nv_bfloat16* q;
+  const int32_t* slots;
+  const int32_t* lens;
+  const int32_t* table;
+  int max_batch, max_pages_per_seq, page_tokens;
+  long long n_pages;
+  float2* part_ml;
+  float* part_o;
+  int max_parts;
+  int32_t* status;
+  int b0, nb;                 // batch entries [b0, b0 + nb) are handled by this launch
+  int n_q_heads, n_ret_heads, n_drop_heads, n_pairs;
+  int kc_anchor, kc_total;    // 64-feature chunks of the predictor input: from the anchor, in all
+  float scale_log2e;
+};
+
+template <int G>
+struct TcSmemTail {
+  float P[2 * G][kTileTokens];       // probabilities of the tile, per (head of the pair, query head)
+  float qs[2][G][128];               // queries * scale * log2e
+  float red_max[8][2 * G];
+  float red_sum[8][2 * G];
+  int cum_tiles[kMaxBatchPerLaunch + 1];
+  unsigned long long full_bar[kStages];
+  unsigned long long empty_bar[kStages];
+  unsigned long long acc_full_bar;
+  unsigned long long acc_empty_bar;
+  unsigned long long drain_bar;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit ran out or another thread already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long start = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - start > kWaitLimitCycles) {
+      *abort_flag = 1;
+      report(status, ECHOKV_ETIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols));
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols));
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns -> 32 registers per thread (thread i = lane i of the quarter)
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(addr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Barrier over the 256 epilogue threads that also ANDs a flag, so that all of them take the same
+// decision after a bounded wait (a warp that left alone would strand the others at a barrier).
+__device__ __forceinline__ bool epilogue_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(ok ? 1u : 0u)
+      : "memory");
+  return r != 0;
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 operand whose rows are 128 bytes (64
+// features) in the 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);          // start address
+  d |= static_cast<uint64_t>(1) << 16;                              // leading byte offset (unused here)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                      // stride between 8-row groups
+  d |= static_cast<uint64_t>(1) << 46;                              // descriptor version of sm_100
+  d |= static_cast<uint64_t>(2) << 61;                              // 128-byte swizzle
+  return d;
+}
+// kind::f16 instruction: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+
+struct Item {
+  int b, tile, pair;
+};
+
+// item -> (sequence, token tile, head pair); tiles of all sequences are numbered consecutively
+template <int G>
+__device__ __forceinline__ Item decode_item(const TcSmemTail<G>& t, int item, int n_pairs, int nb) {
+  Item it;
+  const int tg = item / n_pairs;
+  it.pair = item - tg * n_pairs;
+  int lo = 0, hi = nb;   // largest b with cum_tiles[b] <= tg
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (t.cum_tiles[mid] <= tg) lo = mid; else hi = mid;
+  }
+  it.b = lo;
+  it.tile = tg - t.cum_tiles[lo];
+  return it;
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, 1)
+recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_constant__ CUtensorMap tm_anchor_v,
+                const __grid_constant__ CUtensorMap tm_local_k, const __grid_constant__ CUtensorMap tm_local_v,
+                const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
+                const TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  TcSmemTail<G>& t = *reinterpret_cast<TcSmemTail<G>*>(smem + kStages * kStageBytes);
+  const uint32_t stage_base = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  volatile int* abort_flag = &t.abort_flag;
+
+  // ---- set-up: tile counts per sequence, barriers, tensor memory --------------------------------
+  for (int i = tid; i < p.nb; i += kThreads) {
+    const int b = p.b0 + i;
+    const int slot = p.slots ? p.slots[b] : b;
+    const int len = p.lens[b];
+    int tiles = 0;
+    if (slot < 0 || slot >= p.max_batch) {
+      if (blockIdx.x == 0) report(p.status, ECHOKV_EBADPAGE);
+    } else if (len < 1 || len > p.max_pages_per_seq * p.page_tokens) {
+      if (blockIdx.x == 0) report(p.status, ECHOKV_EBADLENGTH);
+    } else {
+      tiles = (len + kTileTokens - 1) / kTileTokens;
+    }
+    t.cum_tiles[i + 1] = tiles;
+  }
+  if (tid == 0) {
+    t.cum_tiles[0] = 0;
+    t.abort_flag = 0;
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&t.full_bar[s]), 1);
+      mbar_init(smem_u32(&t.empty_bar[s]), 1);
+    }
+    mbar_init(smem_u32(&t.acc_full_bar), 1);
+    mbar_init(smem_u32(&t.acc_empty_bar), 1);
+    mbar_init(smem_u32(&t.drain_bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int i = 0; i < p.nb; ++i) {
+      acc += t.cum_tiles[i + 1];
+      t.cum_tiles[i + 1] = acc;
+    }
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&t.tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = t.tmem_base;
+  const int n_items = t.cum_tiles[p.nb] * p.n_pairs;
+  const int boxes = kTileTokens / p.page_tokens;            // TMA boxes (pages) per token tile
+  const uint32_t page_bytes = p.page_tokens * kRowBytes;
+
+  if (warp == 0) {
+    // =============================== TMA producer ===============================================
+    uint32_t it = 0;
+    uint32_t issued[kStages];
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) issued[s] = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const Item w = decode_item<G>(t, item, p.n_pairs, p.nb);
+      const int b = p.b0 + w.b;
+      const int slot = p.slots ? p.slots[b] : b;
+      const int len = p.lens[b];
+      // page of box `lane` of this tile, or -1 when the box holds no cached token
+      int page = -1;
+      if (lane < boxes) {
+        const int t0 = w.tile * kTileTokens + lane * p.page_tokens;
+        if (t0 < len) {
+          page = p.table[(size_t)slot * p.max_pages_per_seq + t0 / p.page_tokens];
+          if (page < 0 || page >= p.n_pages) {
+            report(p.status, ECHOKV_EBADPAGE);
+            page = -1;
+          }
+        }
+      }
+      const uint32_t n_valid_boxes = __popc(__ballot_sync(0xffffffffu, page >= 0));
+      const uint32_t tx_bytes = n_valid_boxes * page_bytes + kWBytes;
+      for (int phase = 0; phase < 2 && alive; ++phase) {
+        const CUtensorMap* m_anchor = phase == 0 ? &tm_anchor_k : &tm_anchor_v;
+        const CUtensorMap* m_local = phase == 0 ? &tm_local_k : &tm_local_v;
+        const CUtensorMap* m_w = phase == 0 ? &tm_wk : &tm_wv;
+        for (int kc = 0; kc < p.kc_total; ++kc, ++it) {
+          const uint32_t s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          const uint32_t full = smem_u32(&t.full_bar[s]);
+          bool ok = true;
+          if (lane == 0) ok = mbar_wait(smem_u32(&t.empty_bar[s]), ph ^ 1u, abort_flag, p.status);
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          if (!ok) { alive = false; break; }
+          if (lane == 0) mbar_arrive_expect_tx(full, tx_bytes);
+          __syncwarp();
+          const uint32_t x_dst = stage_base + s * kStageBytes;
+          if (page >= 0) {
+            const bool from_anchor = kc < p.kc_anchor;
+            tma_load_2d(x_dst + lane * page_bytes, from_anchor ? m_anchor : m_local,
+                        (from_anchor ? kc : kc - p.kc_anchor) * kChunk, page * p.page_tokens, full);
+          }
+          if (lane == 16) tma_load_2d(x_dst + kXBytes, m_w, kc * kChunk, w.pair * kWRows, full);
+          issued[s] = it + 1;
+        }
+      }
+    }
+    if (!alive && lane == 0) {
+      // drain: let every copy this warp started land before the CTA leaves
+#pragma unroll
+      for (int s = 0; s < kStages; ++s) {
+        if (issued[s] == 0) continue;
+        const uint32_t ph = ((issued[s] - 1) / kStages) & 1u;
+        const long long start = clock64();
+        while (!mbar_try_wait(smem_u32(&t.full_bar[s]), ph) && clock64() - start < kWaitLimitCycles) {
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =============================== MMA issuer ================================================
+    if (lane == 0) {
+      uint32_t it = 0, round = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+        for (int phase = 0; phase < 2 && alive; ++phase, ++round) {
+          // accumulators must have been drained by the epilogue of the previous round
+          if (!mbar_wait(smem_u32(&t.acc_empty_bar), (round & 1u) ^ 1u, abort_flag, p.status)) { alive = false; break; }
+          tc_fence_after();
+          for (int kc = 0; kc < p.kc_total; ++kc, ++it) {
+            const uint32_t s = it % kStages;
+            const uint32_t ph = (it / kStages) & 1u;
+            if (!mbar_wait(smem_u32(&t.full_bar[s]), ph, abort_flag, p.status)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t x_addr = stage_base + s * kStageBytes;
+            const uint32_t w_addr = x_addr + kXBytes;
+            // K phase: A = token rows (two halves of 128), B = 256 predictor rows.
+            // V phase: A = predictor rows (one head of 128 each), B = 256 token rows.
+            const uint32_t a_addr = phase == 0 ? x_addr : w_addr;
+            const uint32_t b_addr = phase == 0 ? w_addr : x_addr;
+#pragma unroll
+            for (int k16 = 0; k16 < kChunk / 16; ++k16) {
+              const uint64_t bd = umma_desc(b_addr + k16 * 32);
+              const uint32_t acc = (kc > 0 || k16 > 0) ? 1u : 0u;
+              tc_mma_bf16(tmem, umma_desc(a_addr + k16 * 32), bd, kIdesc, acc);
+              tc_mma_bf16(tmem + 256, umma_desc(a_addr + 128 * kRowBytes + k16 * 32), bd, kIdesc, acc);
+            }
+            tc_commit(smem_u32(&t.empty_bar[s]));     // stage is free once these MMAs have read it
+          }
+          if (alive) tc_commit(smem_u32(&t.acc_full_bar));
+        }
+      }
+      if (!alive) {
+        // drain: wait (bounded) until every MMA issued so far has retired
+        tc_commit(smem_u32(&t.drain_bar));
+        const long long start = clock64();
+        while (!mbar_try_wait(smem_u32(&t.drain_bar), 0) && clock64() - start < kWaitLimitCycles) {
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // =============================== epilogue (8 warps) ========================================
+    const int ew = warp - 2;                 // 0..7
+    const int quarter = warp & 3;            // TMEM lane quarter this warp may read
+    const int half = ew >> 2;                // which accumulator
+    const int row = quarter * 32 + lane;     // TMEM lane: token (K phase) or feature (V phase)
+    const int et = tid - 64;                 // 0..255
+    const uint32_t t_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + half * 256;
+    uint32_t round = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const Item w = decode_item<G>(t, item, p.n_pairs, p.nb);
+      const int b = p.b0 + w.b;
+      const int len = p.lens[b];
+      const int n_valid = min(kTileTokens, len - w.tile * kTileTokens);
+      const int kvh0 = p.n_ret_heads + w.pair * 2;           // first KV head of the pair
+      const bool second = w.pair * 2 + 1 < p.n_drop_heads;   // does the pair have a second head?
+      // queries of the pair's query heads, pre-scaled
+      for (int idx = et; idx < 2 * G * 128; idx += kEpilogueThreads) {
+        const int hh = idx / (G * 128), rem = idx % (G * 128);
+        float v = 0.f;
+        if (hh == 0 || second)
+          v = __bfloat162float(p.q[((size_t)b * p.n_q_heads + (size_t)(kvh0 + hh) * G) * 128 + rem]) * p.scale_log2e;
+        (&t.qs[0][0][0])[idx] = v;
+      }
+
+      // ---------------- K phase: scores and probabilities ----------------
+      // (the vote is also the barrier that publishes the queries staged above)
+      if (!epilogue_all(mbar_wait(smem_u32(&t.acc_full_bar), round & 1u, abort_flag, p.status))) { alive = false; break; }
+      tc_fence_after();
+      float sc[2][G];
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) sc[hh][gi] = 0.f;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          tmem_ld32(t_addr + hh * 128 + c * 32, v);
+#pragma unroll
+          for (int gi = 0; gi < G; ++gi) {
+            const float4* qv = reinterpret_cast<const float4*>(&t.qs[hh][gi][c * 32]);
+            float acc = sc[hh][gi];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 q4 = qv[j];
+              acc = fmaf(v[4 * j + 0], q4.x, acc);
+              acc = fmaf(v[4 * j + 1], q4.y, acc);
+              acc = fmaf(v[4 * j + 2], q4.z, acc);
+              acc = fmaf(v[4 * j + 3], q4.w, acc);
+            }
+            sc[hh][gi] = acc;
+          }
+        }
+      }
+      const int token = half * 128 + row;
+      const bool tok_valid = token < n_valid;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          if (!tok_valid) sc[hh][gi] = -INFINITY;
+          const float wm = warp_max(sc[hh][gi]);
+          if (lane == 0) t.red_max[ew][hh * G + gi] = wm;
+        }
+      epilogue_sync();
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          float M = t.red_max[0][hh * G + gi];
+#pragma unroll
+          for (int w8 = 1; w8 < 8; ++w8) M = fmaxf(M, t.red_max[w8][hh * G + gi]);
+          const float pr = tok_valid ? exp2f(sc[hh][gi] - M) : 0.f;
+          t.P[hh * G + gi][token] = pr;
+          const float ws = warp_sum(pr);
+          if (lane == 0) t.red_sum[ew][hh * G + gi] = ws;
+          sc[hh][gi] = M;
+        }
+      tc_fence_before();
+      epilogue_sync();       // probabilities visible; every warp is done reading the accumulators
+      if (et == 0) mbar_arrive(smem_u32(&t.acc_empty_bar));
+      if (et < 2 * G) {
+        const int hh = et / G, gi = et % G;
+        if (hh == 0 || second) {
+          float M = t.red_max[0][et], L = 0.f;
+#pragma unroll
+          for (int w8 = 1; w8 < 8; ++w8) M = fmaxf(M, t.red_max[w8][et]);
+#pragma unroll
+          for (int w8 = 0; w8 < 8; ++w8) L += t.red_sum[w8][et];
+          const size_t pidx = ((size_t)b * p.n_q_heads + (size_t)(kvh0 + hh) * G + gi) * p.max_parts + w.tile;
+          p.part_ml[pidx] = make_float2(M, L);
+        }
+      }
+      ++round;
+
+      // ---------------- V phase: weighted sum of predicted V rows ----------------
+      if (!epilogue_all(mbar_wait(smem_u32(&t.acc_full_bar), round & 1u, abort_flag, p.status))) { alive = false; break; }
+      tc_fence_after();
+      float o[G];
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) o[gi] = 0.f;
+      if (half == 0 || second) {
+#pragma unroll 1
+        for (int c = 0; c < kTileTokens / 32; ++c) {
+          if (c * 32 >= n_valid) break;
+          float v[32];
+          tmem_ld32(t_addr + c * 32, v);
+          if ((c + 1) * 32 > n_valid) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c * 32 + j >= n_valid) v[j] = 0.f;     // columns that hold no cached token
+          }
+#pragma unroll
+          for (int gi = 0; gi < G; ++gi) {
+            const float4* pv = reinterpret_cast<const float4*>(&t.P[half * G + gi][c * 32]);
+            float acc = o[gi];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 p4 = pv[j];
+              acc = fmaf(v[4 * j + 0], p4.x, acc);
+              acc = fmaf(v[4 * j + 1], p4.y, acc);
+              acc = fmaf(v[4 * j + 2], p4.z, acc);
+              acc = fmaf(v[4 * j + 3], p4.w, acc);
+            }
+            o[gi] = acc;
+          }
+        }
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          const size_t pidx = ((size_t)b * p.n_q_heads + (size_t)(kvh0 + half) * G + gi) * p.max_parts + w.tile;
+          p.part_o[pidx * 128 + row] = o[gi];
+        }
+      }
+      tc_fence_before();
+      epilogue_sync();
+      if (et == 0) mbar_arrive(smem_u32(&t.acc_empty_bar));
+      ++round;
+    }
+  }
+
+  // ---- teardown ------------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+template <int G>
+constexpr size_t tc_smem_bytes() {
+  return 1024 + (size_t)kStages * kStageBytes + sizeof(TcSmemTail<G>);
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(sym);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows][cols] row-major, boxes of box_rows x 64 columns, 128-byte swizzle
+cudaError_t encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                      CUtensorMapL2promotion promo) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return cudaErrorNotSupported;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {kChunk, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+template <int G>
+cudaError_t launch_g(const CUtensorMap& ak, const CUtensorMap& av, const CUtensorMap& lk, const CUtensorMap& lv,
+                     const CUtensorMap& wk, const CUtensorMap& wv, const TcParams& p, int grid,
+                     cudaStream_t stream) {
+  const size_t smem = tc_smem_bytes<G>();
+  cudaError_t e = cudaFuncSetAttribute(recon_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  recon_tc_kernel<G><<<grid, kThreads, smem, stream>>>(ak, av, lk, lv, wk, wv, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m) {
+  if (dtype != ECHOKV_BF16 || head_dim != 128) return false;
+  if (page_tokens != 16 && page_tokens != 32 && page_tokens != 64 && page_tokens != 128) return false;
+  return D % kChunk == 0 && m % kChunk == 0 && D > m;
+}
+
+cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const void* v_pool, int width,
+                                uint64_t rows, int page_tokens) {
+  cudaError_t e = encode_2d(&maps->k_pool, k_pool, rows, width, page_tokens, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+  if (e != cudaSuccess) return e;
+  e = encode_2d(&maps->v_pool, v_pool, rows, width, page_tokens, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+  if (e != cudaSuccess) return e;
+  maps->pools_ready = true;
+  return cudaSuccess;
+}
+
+cudaError_t tc_encode_weight_maps(TcLayerMaps* maps, const void* Wk, const void* Wv, int d_drop, int d_in) {
+  cudaError_t e = encode_2d(&maps->wk, Wk, d_drop, d_in, kWRows, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+  if (e != cudaSuccess) return e;
+  e = encode_2d(&maps->wv, Wv, d_drop, d_in, kWRows, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+  if (e != cudaSuccess) return e;
+  maps->weights_ready = true;
+  return cudaSuccess;
+}
+
+cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                            const TcLayerMaps& layer, int sm_count, cudaStream_t stream) {
+  if (!anchor.pools_ready || !layer.weights_ready) return cudaErrorInvalidValue;
+  if (r.m > 0 && !layer.pools_ready) return cudaErrorInvalidValue;
+  const int g = a.n_q_heads / a.n_kv_heads;
+  TcParams p;
+  p.q = reinterpret_cast<const __nv_bfloat16*>(a.q);
+  p.slots = a.slots;
+  p.lens = a.lens;
+  p.table = a.geom.table;
+  p.max_batch = a.geom.max_batch;
+  p.max_pages_per_seq = a.geom.max_pages_per_seq;
+  p.page_tokens = a.geom.page_tokens;
+  p.n_pages = a.geom.n_pages;
+  p.part_ml = a.parts.ml;
+  p.part_o = a.parts.o;
+  p.max_parts = a.parts.max_parts;
+  p.status = a.status;
+  p.n_q_heads = a.n_q_heads;
+  p.n_ret_heads = r.m / 128;
+  p.n_drop_heads = a.n_kv_heads - p.n_ret_heads;
+  p.n_pairs = (p.n_drop_heads + 1) / 2;
+  p.kc_anchor = r.D / kChunk;
+  p.kc_total = (r.D + r.m) / kChunk;
+  p.scale_log2e = a.scale_log2e;
+  // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
+  const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;
+  const CUtensorMap& lv = r.m > 0 ? layer.v_pool : anchor.v_pool;
+  const int tiles_cap = (r.capacity_tokens + kTileTokens - 1) / kTileTokens;
+  for (int b0 = 0; b0 < a.batch; b0 += kMaxBatchPerLaunch) {
+    p.b0 = b0;
+    p.nb = a.batch - b0 < kMaxBatchPerLaunch ? a.batch - b0 : kMaxBatchPerLaunch;
+    const long long max_items = (long long)p.nb * tiles_cap * p.n_pairs;
+    const int grid = (int)(max_items < sm_count ? max_items : sm_count);
+    cudaError_t e;
+    switch (g) {
+      case 1: e = launch_g<1>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
+      case 2: e = launch_g<2>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
+      case 4: e = launch_g<4>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
+      case 8: e = launch_g<8>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
+      default: return cudaErrorInvalidValue;
+    }
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace echokv

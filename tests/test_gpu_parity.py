@@ -48,6 +48,8 @@ SMALL = [
     ("mha_d64_bf16", synth.C0, dict(dtype="bf16", batch=2, context=200), [200, 77]),
     ("gqa2_fp32_d128", synth.C0, dict(n_q_heads=8, n_kv_heads=4, head_dim=128, n_retained_heads=1,
                                       batch=2, context=150), [150, 64]),
+    ("one_dropped_head", synth.C2, dict(n_retained_heads=7, batch=2, context=300), [300, 258]),
+    ("pages128", synth.C2, dict(batch=2, context=700, page_tokens=128, random_pages=True), [700, 129]),
     ("gqa8_bf16", synth.C2, dict(n_q_heads=32, n_kv_heads=4, n_retained_heads=1, batch=1, context=300), [300]),
 ]
 
