@@ -174,6 +174,14 @@ int echokv_decode_path(const echokv_ctx* ctx);
  * the fastest family their shape allows.  Meant for tests that check both against the oracle. */
 int echokv_set_decode_path(echokv_ctx* ctx, int path);
 
+/* Device timing of the dominant kernel of each attention call (the fused reconstruct-attend
+ * kernel on compressed layers, the stored-head attention kernel on anchor layers): when enabled,
+ * the library records a CUDA event pair around that kernel on the call's stream.
+ * echokv_read_kernel_timing synchronises the device, returns the summed duration and the number
+ * of timed launches since the last read, and starts over.  Errors: EINVAL, ECUDA. */
+int echokv_set_kernel_timing(echokv_ctx* ctx, int enable);
+int echokv_read_kernel_timing(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
+
 /* Static, human-readable name of a status code. */
 const char* echokv_strerror(int status);
 

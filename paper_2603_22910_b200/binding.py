@@ -59,6 +59,8 @@ EXPORTS = {
     "echokv_launch_count": (C.c_int64, [C.c_void_p]),
     "echokv_decode_path": (C.c_int, [C.c_void_p]),
     "echokv_set_decode_path": (C.c_int, [C.c_void_p, C.c_int]),
+    "echokv_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int]),
+    "echokv_read_kernel_timing": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "echokv_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -220,6 +222,15 @@ class Context:
 
     def set_decode_path(self, path: int) -> None:
         _check(lib().echokv_set_decode_path(self.handle, path), "echokv_set_decode_path")
+
+    def set_kernel_timing(self, enable: bool) -> None:
+        _check(lib().echokv_set_kernel_timing(self.handle, 1 if enable else 0), "echokv_set_kernel_timing")
+
+    def read_kernel_timing(self):
+        """(total milliseconds, launches) of the dominant kernel since the last read."""
+        ms, n = C.c_double(0.0), C.c_int64(0)
+        _check(lib().echokv_read_kernel_timing(self.handle, C.byref(ms), C.byref(n)), "echokv_read_kernel_timing")
+        return ms.value, n.value
 
     def _out(self, q):
         return self.torch.empty(q.shape, dtype=self.torch.float32, device=self.device)

@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "kernels.h"
@@ -86,6 +87,15 @@ struct echokv_ctx {
   int64_t launches = 0;
   float scale = 0.f;
   std::vector<int32_t> pos_scratch;
+  bool timing = false;
+  size_t timed = 0;                                         // event pairs in use
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> events;  // grown on demand, reused
+  ~echokv_ctx() {
+    for (auto& e : events) {
+      cudaEventDestroy(e.first);
+      cudaEventDestroy(e.second);
+    }
+  }
 };
 
 namespace {
@@ -131,6 +141,28 @@ int stored_splits(const echokv_ctx* c, int B, int n_heads) {
   return n;
 }
 
+// Event pair around the dominant kernel of a call (only while timing is enabled).
+struct ScopedKernelTimer {
+  echokv_ctx* c;
+  cudaStream_t s;
+  cudaEvent_t stop = nullptr;
+  ScopedKernelTimer(echokv_ctx* ctx, cudaStream_t stream) : c(ctx), s(stream) {
+    if (!c->timing) return;
+    if (c->timed == c->events.size()) {
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess) return;
+      if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return; }
+      c->events.emplace_back(a, b);
+    }
+    auto& e = c->events[c->timed++];
+    cudaEventRecord(e.first, s);
+    stop = e.second;
+  }
+  ~ScopedKernelTimer() {
+    if (stop) cudaEventRecord(stop, s);
+  }
+};
+
 int check_call(echokv_ctx* c, int layer, const void* q, const float* out, const int32_t* lens, int B) {
   if (!c || !q || !out || !lens) return ECHOKV_EINVAL;
   if (layer < 0 || layer >= c->cfg.n_layers || B < 1) return ECHOKV_EINVAL;
@@ -144,7 +176,10 @@ int attend_stored_layer(echokv_ctx* c, const Layer& L, const void* q, float* out
   AttnArgs a = attn_args(c, q, slots, lens, B);
   const int H = c->cfg.n_kv_heads;
   const int n_splits = stored_splits(c, B, H);
-  if (launch_attn_stored(a, L.k_pool, L.v_pool, c->d.D, H, n_splits, s) != cudaSuccess) return ECHOKV_ECUDA;
+  {
+    ScopedKernelTimer timer(c, s);
+    if (launch_attn_stored(a, L.k_pool, L.v_pool, c->d.D, H, n_splits, s) != cudaSuccess) return ECHOKV_ECUDA;
+  }
   if (launch_merge(a, out, H, n_splits, c->d.part_tokens, nullptr, s) != cudaSuccess) return ECHOKV_ECUDA;
   c->launches += 2;
   return ECHOKV_OK;
@@ -315,10 +350,13 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   ra.part_tokens = c->d.part_tokens;
   ra.capacity_tokens = c->d.capacity;
   cudaError_t e;
-  if (c->path == 2) {
-    e = launch_recon_tc(a, ra, A.tc, L.tc, c->sm_count, s);
-  } else {
-    e = launch_recon_simt(a, ra, s);
+  {
+    ScopedKernelTimer timer(c, s);
+    if (c->path == 2) {
+      e = launch_recon_tc(a, ra, A.tc, L.tc, c->sm_count, s);
+    } else {
+      e = launch_recon_simt(a, ra, s);
+    }
   }
   if (e != cudaSuccess) return ECHOKV_ECUDA;
   if (launch_merge(a, out, r, n_splits, c->d.part_tokens, L.bv, s) != cudaSuccess) return ECHOKV_ECUDA;
@@ -373,6 +411,27 @@ int echokv_get_device_status(echokv_ctx* c, int32_t* host_out) {
   if (cudaMemcpy(&v, status_ptr(c), 4, cudaMemcpyDeviceToHost) != cudaSuccess) return ECHOKV_ECUDA;
   if (v != 0 && cudaMemset(status_ptr(c), 0, 4) != cudaSuccess) return ECHOKV_ECUDA;
   *host_out = v;
+  return ECHOKV_OK;
+}
+
+int echokv_set_kernel_timing(echokv_ctx* c, int enable) {
+  if (!c) return ECHOKV_EINVAL;
+  c->timing = enable != 0;
+  return ECHOKV_OK;
+}
+
+int echokv_read_kernel_timing(echokv_ctx* c, double* total_ms, int64_t* n_launches) {
+  if (!c || !total_ms || !n_launches) return ECHOKV_EINVAL;
+  if (cudaDeviceSynchronize() != cudaSuccess) return ECHOKV_ECUDA;
+  double sum = 0.0;
+  for (size_t i = 0; i < c->timed; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->events[i].first, c->events[i].second) != cudaSuccess) return ECHOKV_ECUDA;
+    sum += ms;
+  }
+  *total_ms = sum;
+  *n_launches = (int64_t)c->timed;
+  c->timed = 0;
   return ECHOKV_OK;
 }
 
