@@ -98,12 +98,14 @@ def torch_dtype(w: Workload) -> torch.dtype:
     return torch.bfloat16 if w.dtype == "bf16" else torch.float32
 
 
-def _gen(seed: int, *stream: int) -> torch.Generator:
-    """Independent sub-stream per (seed, tensor id, layer, ...)."""
+def _gen(seed: int, *stream: int, device="cpu") -> torch.Generator:
+    """Independent sub-stream per (seed, tensor id, layer, ...).  A CUDA generator draws a
+    different (equally deterministic) sequence than the CPU one: workloads too large to draw on
+    the host are drawn on the device and read back where the oracle needs them."""
     s = seed
     for v in stream:
         s = (s * 1000003 + 7919 * (v + 1)) % (2 ** 62)
-    g = torch.Generator(device="cpu")
+    g = torch.Generator(device=device)
     g.manual_seed(s)
     return g
 
@@ -111,27 +113,27 @@ def _gen(seed: int, *stream: int) -> torch.Generator:
 T_ANCHOR_K, T_ANCHOR_V, T_NOISE_K, T_NOISE_V, T_WK, T_WV, T_Q, T_PAGES = range(8)
 
 
-def normal(shape, seed: int, *stream: int) -> torch.Tensor:
-    return torch.randn(shape, generator=_gen(seed, *stream), dtype=torch.float32)
+def normal(shape, seed: int, *stream: int, device="cpu") -> torch.Tensor:
+    return torch.randn(shape, generator=_gen(seed, *stream, device=device), dtype=torch.float32, device=device)
 
 
-def xavier_uniform(d_out: int, d_in: int, seed: int, *stream: int) -> torch.Tensor:
+def xavier_uniform(d_out: int, d_in: int, seed: int, *stream: int, device="cpu") -> torch.Tensor:
     a = math.sqrt(6.0 / (d_in + d_out))
-    u = torch.rand((d_out, d_in), generator=_gen(seed, *stream), dtype=torch.float32)
+    u = torch.rand((d_out, d_in), generator=_gen(seed, *stream, device=device), dtype=torch.float32, device=device)
     return (u * 2.0 - 1.0) * a
 
 
-def anchor_cache(w: Workload, layer: int, kind: str, batch_index: int | None = None) -> torch.Tensor:
+def anchor_cache(w: Workload, layer: int, kind: str, batch_index: int | None = None, device="cpu") -> torch.Tensor:
     """fp32 pre-rounding N(0,1) cache of anchor layer `layer`: [B, L, D]
     (or [L, D] for one sequence).  kind is "k" or "v"."""
     tid = T_ANCHOR_K if kind == "k" else T_ANCHOR_V
     if batch_index is None:
-        return torch.stack([anchor_cache(w, layer, kind, b) for b in range(w.batch)])
-    return normal((w.context, w.D), w.seed, tid, layer, batch_index)
+        return torch.stack([anchor_cache(w, layer, kind, b, device) for b in range(w.batch)])
+    return normal((w.context, w.D), w.seed, tid, layer, batch_index, device=device)
 
 
 def layer_cache(w: Workload, layer: int, kind: str, batch_index: int, width: int | None = None,
-                anchor_f32: torch.Tensor | None = None) -> torch.Tensor:
+                anchor_f32: torch.Tensor | None = None, device="cpu") -> torch.Tensor:
     """Stored-precision cache of `layer` for one sequence: [L, width].
 
     An anchor layer is N(0,1); a compressed layer is rho * anchor + sqrt(1 -
@@ -142,26 +144,26 @@ def layer_cache(w: Workload, layer: int, kind: str, batch_index: int, width: int
     width = w.D if width is None else width
     a_layer = w.anchor_of(layer)
     if anchor_f32 is None:
-        anchor_f32 = anchor_cache(w, a_layer, kind, batch_index)
+        anchor_f32 = anchor_cache(w, a_layer, kind, batch_index, device)
     if layer == a_layer:
         x = anchor_f32[:, :width]
     else:
         tid = T_NOISE_K if kind == "k" else T_NOISE_V
-        noise = normal((w.context, w.D), w.seed, tid, layer, batch_index)[:, :width]
+        noise = normal((w.context, w.D), w.seed, tid, layer, batch_index, device=device)[:, :width]
         x = w.rho * anchor_f32[:, :width] + math.sqrt(1.0 - w.rho * w.rho) * noise
     return x.to(torch_dtype(w)).contiguous()
 
 
-def predictor_weights(w: Workload, layer: int, kind: str) -> torch.Tensor:
+def predictor_weights(w: Workload, layer: int, kind: str, device="cpu") -> torch.Tensor:
     """Stored-precision predictor of a compressed layer: [D_drop, D_in],
     columns = the D anchor dims then the m local dims."""
     tid = T_WK if kind == "k" else T_WV
-    return xavier_uniform(w.d_drop, w.d_in, w.seed, tid, layer).to(torch_dtype(w)).contiguous()
+    return xavier_uniform(w.d_drop, w.d_in, w.seed, tid, layer, device=device).to(torch_dtype(w)).contiguous()
 
 
-def queries(w: Workload, layer: int) -> torch.Tensor:
+def queries(w: Workload, layer: int, device="cpu") -> torch.Tensor:
     """Stored-precision decode queries: [B, H_q, d]."""
-    return normal((w.batch, w.n_q_heads, w.head_dim), w.seed, T_Q, layer).to(torch_dtype(w)).contiguous()
+    return normal((w.batch, w.n_q_heads, w.head_dim), w.seed, T_Q, layer, device=device).to(torch_dtype(w)).contiguous()
 
 
 def block_table(w: Workload, n_pages_total: int | None = None) -> torch.Tensor:
@@ -181,6 +183,7 @@ def block_table(w: Workload, n_pages_total: int | None = None) -> torch.Tensor:
 def to_numpy_stored(x: torch.Tensor) -> np.ndarray:
     """Stored tensor -> numpy without changing a bit: bf16 becomes its uint16
     bit pattern, fp32 stays float32."""
+    x = x.cpu()
     if x.dtype == torch.bfloat16:
         return x.contiguous().view(torch.int16).numpy().view(np.uint16)
     return x.contiguous().numpy()
