@@ -60,7 +60,8 @@ enum {
   ECHOKV_EBADPAGE = -8,       /* device status: page id or sequence slot out of range      */
   ECHOKV_EUNSUPPORTED = -9,   /* shape outside what the kernels handle                     */
   ECHOKV_ENOTABLE = -10,      /* a call that needs the block table before it was set       */
-  ECHOKV_EBADLENGTH = -11     /* device status: a sequence length < 1 or beyond capacity   */
+  ECHOKV_EBADLENGTH = -11,    /* device status: a sequence length < 1 or beyond capacity   */
+  ECHOKV_ESCRATCH = -12       /* problem too large for the fixed scratch of the no-alloc entry */
 };
 
 typedef struct {
@@ -181,6 +182,41 @@ int echokv_set_decode_path(echokv_ctx* ctx, int path);
  * of timed launches since the last read, and starts over.  Errors: EINVAL, ECUDA. */
 int echokv_set_kernel_timing(echokv_ctx* ctx, int enable);
 int echokv_read_kernel_timing(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
+
+/* Full-cache attention for callers that cannot allocate device memory (the paper has no
+ * counterpart to this entry point; it exists for the library's users).
+ *
+ * Every other attention call needs a context whose split-K workspace the caller allocated.  A
+ * caller that is only ever handed raw pointers -- a plug-in running inside another framework's
+ * execution callback where allocation is forbidden, a thread that works out of an arena sized
+ * long ago -- has no way to provide one.  This call needs no context and no workspace: it
+ * computes what echokv_full_attention computes (Eq. 7 on the stored cache of one layer), taking
+ * the layer's pools, the block table, q, out and the lengths directly, and keeps its partial
+ * results in a fixed array inside the library image: echokv_noalloc_scratch_bytes() bytes
+ * (8 MiB), resident on every GPU that loads the library until the process exits.
+ *
+ *  - cfg describes the geometry (heads, head_dim, page_tokens, max_batch, max_pages_per_seq,
+ *    n_pages, dtype, softmax_scale, device); n_layers, group_size, n_retained_heads are ignored.
+ *    k_pool / v_pool: device pointers [n_pages][page_tokens][n_kv_heads * head_dim]; the other
+ *    pointers as in echokv_full_attention.  dev_status_out: optional device int32 that receives
+ *    the device status of this call (ECHOKV_OK, EBADPAGE, EBADLENGTH), stream-ordered.
+ *  - It calls no cudaMalloc / cudaFree and no routine that allocates.  Makes cfg->device current.
+ *  - The FIRST call on each device looks up the device address of the array; make that first
+ *    call before any stream capture begins.
+ *  - Size limit: B * n_q_heads * (8 + 4 * head_dim) + 256 bytes must fit the array (for
+ *    head_dim 128: B * n_q_heads <= 16131); beyond it the call returns ECHOKV_ESCRATCH and does
+ *    nothing.  Fewer sequence splits are used when more would not fit.
+ *  - All calls, on all streams and from all threads, share the one array per device, and it keeps
+ *    whatever the previous call left in it (the call clears the one word it needs cleared).
+ *    Two calls that overlap on the GPU race on it: order them, e.g. on one stream.
+ * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (B > max_batch), ESCRATCH, ECUDA. */
+int echokv_full_attention_noalloc(const echokv_config* cfg, const void* k_pool, const void* v_pool,
+                                  const int32_t* dev_block_table, const void* q, float* out,
+                                  const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                                  int32_t* dev_status_out, void* stream);
+
+/* Size in bytes of the fixed scratch array behind echokv_full_attention_noalloc. */
+uint64_t echokv_noalloc_scratch_bytes(void);
 
 /* Static, human-readable name of a status code. */
 const char* echokv_strerror(int status);

@@ -18,7 +18,7 @@ ECHOKV_BF16, ECHOKV_FP32 = 0, 1
 ECHOKV_OK = 0
 ECHOKV_EINVAL, ECHOKV_ENOTANCHOR, ECHOKV_ENOTCOMPRESSED, ECHOKV_ECAPACITY = -1, -2, -3, -4
 ECHOKV_ENOWEIGHTS, ECHOKV_ECUDA, ECHOKV_ETIMEOUT, ECHOKV_EBADPAGE = -5, -6, -7, -8
-ECHOKV_EUNSUPPORTED, ECHOKV_ENOTABLE, ECHOKV_EBADLENGTH = -9, -10, -11
+ECHOKV_EUNSUPPORTED, ECHOKV_ENOTABLE, ECHOKV_EBADLENGTH, ECHOKV_ESCRATCH = -9, -10, -11, -12
 
 
 class echokv_config(C.Structure):
@@ -61,6 +61,10 @@ EXPORTS = {
     "echokv_set_decode_path": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_read_kernel_timing": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "echokv_full_attention_noalloc": (C.c_int, [C.POINTER(echokv_config), C.c_void_p, C.c_void_p, C.c_void_p,
+                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                                C.c_void_p, C.c_void_p]),
+    "echokv_noalloc_scratch_bytes": (C.c_uint64, []),
     "echokv_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -234,6 +238,18 @@ class Context:
 
     def _out(self, q):
         return self.torch.empty(q.shape, dtype=self.torch.float32, device=self.device)
+
+
+def echokv_full_attention_noalloc(cfg: echokv_config, k_pool, v_pool, block_table, q, out, seq_lens,
+                                  seq_slots=None, status_out=None, stream=None) -> None:
+    """Full-cache attention without a context or a workspace, for callers that cannot allocate
+    device memory: partial results live in a fixed 8 MiB array inside the library.  Tensors are
+    only read for their addresses; nothing is allocated here either.  Calls sharing a device must
+    not overlap on the GPU, and the first call on a device should precede any stream capture."""
+    _check(lib().echokv_full_attention_noalloc(C.byref(cfg), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+                                               _ptr(q), _ptr(out), _ptr(seq_slots), _ptr(seq_lens),
+                                               q.shape[0], _ptr(status_out), _stream_handle(stream)),
+           "echokv_full_attention_noalloc")
 
 
 def config_for(w, n_pages: int | None = None, device: int = 0, max_batch: int | None = None) -> echokv_config:

@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libechokv.so")
-SOURCES = ["echokv_host.cu", "simt_kernels.cu", "recon_tc.cu"]
+SOURCES = ["echokv_host.cu", "simt_kernels.cu", "recon_tc.cu", "noalloc.cu"]
 HEADERS = ["common.cuh", "kernels.h", "recon_tc.h", os.path.join("..", "..", "include", "echokv.h")]
 
 

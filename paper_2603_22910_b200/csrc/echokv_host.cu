@@ -453,6 +453,7 @@ const char* echokv_strerror(int status) {
     case ECHOKV_EUNSUPPORTED: return "shape not supported by the kernels";
     case ECHOKV_ENOTABLE: return "block table was not set";
     case ECHOKV_EBADLENGTH: return "device: sequence length below 1 or beyond capacity";
+    case ECHOKV_ESCRATCH: return "problem does not fit the fixed scratch array of the no-alloc entry point";
     default: return "unknown status";
   }
 }

@@ -105,11 +105,11 @@ def test_create_checks_buffers_before_touching_cuda(lib):
 
 def test_strerror_names_every_code(lib):
     seen = set()
-    for code in range(0, -12, -1):
+    for code in range(0, -13, -1):
         s = binding.echokv_strerror(code)
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 12
+    assert len(seen) == 13
     assert binding.echokv_strerror(-99) == "unknown status"
 
 
