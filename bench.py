@@ -105,7 +105,7 @@ class ClockSampler(threading.Thread):
                 for bit, name in names.items():
                     if mask & bit and name != "gpu_idle":
                         self.reasons.add(name)
-                time.sleep(0.02)
+                time.sleep(0.004)
         except Exception as e:  # NVML missing: report it rather than guess
             self.error = repr(e)
 
@@ -162,7 +162,7 @@ def oracle_inputs(w, layer, b):
     return q, kg, vg, kl, vl, Wk, Wv
 
 
-def time_oracle(w, budget_s, max_seqs=None):
+def time_oracle(w, budget_s, max_seqs=None, full=False):
     """The oracle as it stands on whole sequences of the workload until `budget_s` is used."""
     from oracle import echokv_oracle as O
     layer = 1
@@ -171,7 +171,10 @@ def time_oracle(w, budget_s, max_seqs=None):
     for b in range(w.batch if max_seqs is None else min(w.batch, max_seqs)):
         args = oracle_inputs(w, layer, b)
         t0 = time.perf_counter()
-        outs[b] = O.decode_attention(*args, n_kv_heads=w.n_kv_heads)
+        if full:     # the anchor layer's stored cache
+            outs[b] = O.full_attention(args[0], args[1], args[2], w.n_kv_heads)
+        else:
+            outs[b] = O.decode_attention(*args, n_kv_heads=w.n_kv_heads)
         elapsed += time.perf_counter() - t0
         done += 1
         if elapsed >= budget_s:
@@ -228,13 +231,20 @@ def run_reference(args):
     return 0
 
 
-def workload_config(w):
-    return {"workload": "%s: B=%d L=%d H_q=%d H_kv=%d d=%d retained=%d (D_in=%d -> D_drop=%d), %s, %d-token pages, "
-                        "anchor + compressed layer" % (w.name, w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim,
-                                                       w.n_retained_heads, w.d_in, w.d_drop, w.dtype, w.page_tokens),
-            "global_batch": w.batch, "context": w.context,
-            "l2": "inputs (%.2f GB of cache per step) exceed the 126 MB L2; no flush needed" %
-                  (w.batch * w.context * 2 * w.d_in * (2 if w.dtype == "bf16" else 4) / 1e9),
+def workload_config(w, full=False):
+    elem = 2 if w.dtype == "bf16" else 4
+    if full:
+        what = ("%s, uncompressed: B=%d L=%d H_q=%d H_kv=%d d=%d, %s, %d-token pages, full-cache attention on the "
+                "anchor layer" % (w.name, w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype,
+                                  w.page_tokens))
+        gb = w.batch * w.context * 2 * w.D * elem / 1e9
+    else:
+        what = ("%s: B=%d L=%d H_q=%d H_kv=%d d=%d retained=%d (D_in=%d -> D_drop=%d), %s, %d-token pages, "
+                "anchor + compressed layer" % (w.name, w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim,
+                                               w.n_retained_heads, w.d_in, w.d_drop, w.dtype, w.page_tokens))
+        gb = w.batch * w.context * 2 * w.d_in * elem / 1e9
+    return {"workload": what, "global_batch": w.batch, "context": w.context,
+            "l2": "inputs (%.2f GB of cache per step) exceed the 126 MB L2; no flush needed" % gb,
             "parallelism": "replicas"}
 
 
@@ -302,12 +312,23 @@ def run_ours(args):
     out = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
     t_gen = time.perf_counter() - t_gen
 
+    full = args.mode == "full"
+    if args.stored_path is not None:
+        ctx.set_stored_path(args.stored_path)
+
     def step():
         ctx.append_kv(anchor_l, new_dev[(anchor_l, "k")], new_dev[(anchor_l, "v")], positions)
+        if full:     # the uncompressed mode / an anchor layer: Eq. 7 on the stored full cache
+            ctx.full_attention(anchor_l, q, lens, out=out)
+            return
         ctx.append_kv(layer, new_dev[(layer, "k")], new_dev[(layer, "v")], positions)
         ctx.decode_attention(layer, q, lens, out=out)
 
     def step_host():
+        if full:
+            ctx.layer_step_host(anchor_l, q_host, new[(anchor_l, "k")], new[(anchor_l, "v")], out_host, lens_host,
+                                attend=True)
+            return
         ctx.layer_step_host(anchor_l, None, new[(anchor_l, "k")], new[(anchor_l, "v")], None, lens_host, attend=False)
         ctx.layer_step_host(layer, q_host, new[(layer, "k")], new[(layer, "v")], out_host, lens_host, attend=True)
 
@@ -362,7 +383,9 @@ def run_ours(args):
     sync_all()
     ms_e2e = max_over_ranks(e2.elapsed_time(e3))
     elem = 2 if w.dtype == "bf16" else 4
-    h2d = 2 * 2 * w.batch * w.D * elem + w.batch * w.n_q_heads * w.head_dim * elem + 2 * 2 * w.batch * 4
+    n_host_layers = 1 if full else 2
+    h2d = (n_host_layers * 2 * w.batch * w.D * elem + w.batch * w.n_q_heads * w.head_dim * elem
+           + n_host_layers * 2 * w.batch * 4)
     d2h = w.batch * w.n_q_heads * w.head_dim * 4
     same = bool(torch.equal(out_host, out.cpu()))
 
@@ -373,21 +396,33 @@ def run_ours(args):
     peaks, peaks_kind = load_peaks()
     flops, bytes_ = algorithmic_work(w)
     k_ms = kernel_ms / max(kernel_launches, 1)
-    achieved_tf = flops / (k_ms * 1e-3) / 1e12
-    peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
-    roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": achieved_tf / peak_tf, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                "kernel": "recon_tc_kernel", "kernel_ms": k_ms, "kernel_launches": kernel_launches,
-                "peak_source": "%s (bf16 sustained; kernel timed inside a long step)" % peaks_kind,
-                "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": bytes_,
-                "hbm_frac_of_%s" % peaks_kind: bytes_ / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
-                "frac_of_burst_peak": achieved_tf / float(peaks["bf16_tflops"])}
+    if full:
+        # Eq. 7 on the stored cache: every token's K and V row of every KV head is read once
+        bytes_ = w.batch * w.context * 2.0 * w.D * elem
+        achieved_gbs = bytes_ / (k_ms * 1e-3) / 1e9
+        peak_gbs = float(peaks["hbm_gbs"])
+        roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
+                    "frac": achieved_gbs / peak_gbs, "traffic": NCU_TRAFFIC_BYTES.get(args.workload + "_full"),
+                    "kernel": "attn_stored_mma_kernel" if ctx.stored_path() == 1 else "attn_stored_kernel",
+                    "kernel_ms": k_ms, "kernel_launches": kernel_launches,
+                    "peak_source": "%s (STREAM-style copy)" % peaks_kind,
+                    "algorithmic_bytes_per_launch": bytes_}
+    else:
+        achieved_tf = flops / (k_ms * 1e-3) / 1e12
+        peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+        roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": achieved_tf / peak_tf, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                    "kernel": "recon_tc_kernel", "kernel_ms": k_ms, "kernel_launches": kernel_launches,
+                    "peak_source": "%s (bf16 sustained; kernel timed inside a long step)" % peaks_kind,
+                    "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": bytes_,
+                    "hbm_frac_of_%s" % peaks_kind: bytes_ / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
+                    "frac_of_burst_peak": achieved_tf / float(peaks["bf16_tflops"])}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": workload_config(w),
+        "config": workload_config(w, full),
         "us_per_layer_step": ms_step * 1e3,
         "kv_tokens_scanned_per_s": world * w.batch * w.context / (ms_step * 1e-3),
         "clocks": clocks,
@@ -395,12 +430,12 @@ def run_ours(args):
                 "ms_per_step": ms_e2e / args.steps, "matches_device_path": same},
         "gpu_launches": int(launches),
         "roofline": roofline,
-        "decode_path": ctx.decode_path(),
+        "decode_path": ctx.decode_path(), "stored_path": ctx.stored_path(),
         "input_generation_s": t_gen,
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_seq, t_cpu, outs = time_oracle(w, budget_s=12.0, max_seqs=4)
+        n_seq, t_cpu, outs = time_oracle(w, budget_s=12.0, max_seqs=4, full=full)
         gpu = out.cpu().numpy().astype(np.float64)
         worst_abs, num, den = 0.0, 0.0, 0.0
         for b, ref in outs.items():
@@ -425,6 +460,11 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c1", choices=["c1", "c2"])
+    ap.add_argument("--mode", default="compressed", choices=["compressed", "full"],
+                    help="compressed: decode attention of a compressed layer (the headline); full: the "
+                         "uncompressed path, full-cache attention on the anchor layer")
+    ap.add_argument("--stored-path", type=int, default=None, choices=[0, 1],
+                    help="kernel for stored heads: 0 CUDA-core, 1 TMA + tensor-core (default: the library's choice)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")

@@ -175,6 +175,14 @@ int echokv_decode_path(const echokv_ctx* ctx);
  * the fastest family their shape allows.  Meant for tests that check both against the oracle. */
 int echokv_set_decode_path(echokv_ctx* ctx, int path);
 
+/* Which kernel serves attention over stored heads (anchor layers, retained heads, the
+ * uncompressed mode): 0 = CUDA-core kernel (any supported shape), 1 = TMA + tensor-core kernel
+ * (bf16, head_dim 128).  Contexts start on 1 when their shape allows it.
+ * echokv_set_stored_path: EINVAL (not 0 or 1), EUNSUPPORTED (1 on a shape it does not take).
+ * Meant for tests that check both against the oracle. */
+int echokv_stored_path(const echokv_ctx* ctx);
+int echokv_set_stored_path(echokv_ctx* ctx, int path);
+
 /* Device timing of the dominant kernel of each attention call (the fused reconstruct-attend
  * kernel on compressed layers, the stored-head attention kernel on anchor layers): when enabled,
  * the library records a CUDA event pair around that kernel on the call's stream.

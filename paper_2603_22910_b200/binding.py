@@ -59,6 +59,8 @@ EXPORTS = {
     "echokv_launch_count": (C.c_int64, [C.c_void_p]),
     "echokv_decode_path": (C.c_int, [C.c_void_p]),
     "echokv_set_decode_path": (C.c_int, [C.c_void_p, C.c_int]),
+    "echokv_stored_path": (C.c_int, [C.c_void_p]),
+    "echokv_set_stored_path": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_read_kernel_timing": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "echokv_full_attention_noalloc": (C.c_int, [C.POINTER(echokv_config), C.c_void_p, C.c_void_p, C.c_void_p,
@@ -226,6 +228,12 @@ class Context:
 
     def set_decode_path(self, path: int) -> None:
         _check(lib().echokv_set_decode_path(self.handle, path), "echokv_set_decode_path")
+
+    def stored_path(self) -> int:
+        return lib().echokv_stored_path(self.handle)
+
+    def set_stored_path(self, path: int) -> None:
+        _check(lib().echokv_set_stored_path(self.handle, path), "echokv_set_stored_path")
 
     def set_kernel_timing(self, enable: bool) -> None:
         _check(lib().echokv_set_kernel_timing(self.handle, 1 if enable else 0), "echokv_set_kernel_timing")

@@ -8,6 +8,7 @@
 
 #include "kernels.h"
 #include "recon_tc.h"
+#include "stored_mma.h"
 
 using namespace echokv;
 
@@ -71,6 +72,7 @@ struct Layer {
   const void* bv = nullptr;
   bool anchor = false;
   TcLayerMaps tc;     // tensor maps of the tensor-core path (valid when tc.ready)
+  CUtensorMap stored_k, stored_v;   // tensor maps of the stored-head kernel (valid when ctx.stored_path == 1)
 };
 
 }  // namespace
@@ -84,6 +86,8 @@ struct echokv_ctx {
   int sm_count = 0;
   int path = 0;          // see echokv_decode_path
   bool tc_capable = false;
+  bool stored_capable = false;   // shape served by the TMA + mma.sync stored-head kernel
+  int stored_path = 0;           // 0 = CUDA-core kernel, 1 = TMA + mma.sync kernel
   int64_t launches = 0;
   float scale = 0.f;
   std::vector<int32_t> pos_scratch;
@@ -101,6 +105,9 @@ struct echokv_ctx {
 namespace {
 
 int32_t* status_ptr(echokv_ctx* c) { return reinterpret_cast<int32_t*>(c->ws + c->d.off_status); }
+// item sizes the stored-head kernel publishes for the merge kernel: kStoredMaxLaunches words that
+// share the status word's 256-byte block
+int32_t* item_tokens_ptr(echokv_ctx* c) { return reinterpret_cast<int32_t*>(c->ws + c->d.off_status + 64); }
 
 PageGeom geom_of(const echokv_ctx* c) {
   PageGeom g;
@@ -171,17 +178,35 @@ int check_call(echokv_ctx* c, int layer, const void* q, const float* out, const 
   return ECHOKV_OK;
 }
 
+// Eq. 7 for the stored KV heads 0 .. n_heads-1 of layer L (pool row width `width`), as split-K
+// partials.  *item_tokens receives the device array the merge kernel reads the partial count
+// from (null: n_splits partials per head).
+cudaError_t attend_stored_heads(echokv_ctx* c, const AttnArgs& a, const Layer& L, int width, int n_heads,
+                                int n_splits, const int32_t** item_tokens, cudaStream_t s) {
+  *item_tokens = nullptr;
+  if (n_heads == 0) return cudaSuccess;
+  c->launches += 1;
+  if (c->stored_path == 1) {
+    *item_tokens = item_tokens_ptr(c);
+    return launch_attn_stored_mma(a, L.stored_k, L.stored_v, n_heads, item_tokens_ptr(c), c->sm_count, s);
+  }
+  return launch_attn_stored(a, L.k_pool, L.v_pool, width, n_heads, n_splits, s);
+}
+
 int attend_stored_layer(echokv_ctx* c, const Layer& L, const void* q, float* out,
                         const int32_t* slots, const int32_t* lens, int B, cudaStream_t s) {
   AttnArgs a = attn_args(c, q, slots, lens, B);
   const int H = c->cfg.n_kv_heads;
   const int n_splits = stored_splits(c, B, H);
+  const int32_t* item_tokens = nullptr;
   {
     ScopedKernelTimer timer(c, s);
-    if (launch_attn_stored(a, L.k_pool, L.v_pool, c->d.D, H, n_splits, s) != cudaSuccess) return ECHOKV_ECUDA;
+    if (attend_stored_heads(c, a, L, c->d.D, H, n_splits, &item_tokens, s) != cudaSuccess) return ECHOKV_ECUDA;
   }
-  if (launch_merge(a, out, H, n_splits, c->d.part_tokens, nullptr, s) != cudaSuccess) return ECHOKV_ECUDA;
-  c->launches += 2;
+  if (launch_merge(a, out, H, n_splits, item_tokens, kStoredMaxBatchPerLaunch, c->d.part_tokens, nullptr, s) !=
+      cudaSuccess)
+    return ECHOKV_ECUDA;
+  c->launches += 1;
   return ECHOKV_OK;
 }
 
@@ -256,6 +281,22 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
       if (e != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
     }
   }
+  c->stored_capable = stored_mma_supported(cfg->dtype, cfg->head_dim, d.g, cfg->max_batch);
+  if (c->stored_capable) {
+    const int box_rows = stored_rows_per_box(cfg->page_tokens);
+    for (int l = 0; l < cfg->n_layers; ++l) {
+      Layer& L = c->layers[l];
+      const int width = L.anchor ? d.D : d.m;
+      if (width == 0) continue;
+      const uint64_t rows = (uint64_t)cfg->n_pages * cfg->page_tokens;
+      if (encode_pool_box_map(&L.stored_k, L.k_pool, width, rows, box_rows) != cudaSuccess ||
+          encode_pool_box_map(&L.stored_v, L.v_pool, width, rows, box_rows) != cudaSuccess) {
+        delete c;
+        return ECHOKV_ECUDA;
+      }
+    }
+    c->stored_path = 1;
+  }
   *out = c;
   return ECHOKV_OK;
 }
@@ -292,6 +333,15 @@ int echokv_set_decode_path(echokv_ctx* c, int path) {
     return ECHOKV_OK;
   }
   return ECHOKV_EINVAL;
+}
+
+int echokv_stored_path(const echokv_ctx* c) { return c ? c->stored_path : 0; }
+
+int echokv_set_stored_path(echokv_ctx* c, int path) {
+  if (!c || (path != 0 && path != 1)) return ECHOKV_EINVAL;
+  if (path == 1 && !c->stored_capable) return ECHOKV_EUNSUPPORTED;
+  c->stored_path = path;
+  return ECHOKV_OK;
 }
 
 int echokv_append_kv(echokv_ctx* c, int layer, const void* k_new, const void* v_new,
@@ -337,10 +387,8 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   const int r = c->cfg.n_retained_heads;
   // retained heads: Eq. 7 on what is stored (Eq. 6 keeps them as they are)
   const int n_splits = stored_splits(c, B, r);
-  if (r > 0) {
-    if (launch_attn_stored(a, L.k_pool, L.v_pool, c->d.m, r, n_splits, s) != cudaSuccess) return ECHOKV_ECUDA;
-    c->launches += 1;
-  }
+  const int32_t* item_tokens = nullptr;
+  if (attend_stored_heads(c, a, L, c->d.m, r, n_splits, &item_tokens, s) != cudaSuccess) return ECHOKV_ECUDA;
   // dropped heads: predict (Eq. 3) and attend (Eq. 7) on chip
   ReconArgs ra;
   ra.k_anchor = A.k_pool; ra.v_anchor = A.v_pool;
@@ -359,7 +407,9 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     }
   }
   if (e != cudaSuccess) return ECHOKV_ECUDA;
-  if (launch_merge(a, out, r, n_splits, c->d.part_tokens, L.bv, s) != cudaSuccess) return ECHOKV_ECUDA;
+  if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, c->d.part_tokens, L.bv, s) !=
+      cudaSuccess)
+    return ECHOKV_ECUDA;
   c->launches += 2;
   return ECHOKV_OK;
 }

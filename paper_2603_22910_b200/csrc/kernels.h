@@ -41,10 +41,13 @@ struct ReconArgs {
 // dropped KV heads; one partial per part_tokens tokens.
 cudaError_t launch_recon_simt(const AttnArgs& a, const ReconArgs& r, cudaStream_t stream);
 
-// Merge split-K partials into out[B][H_q][d]; heads with KV head < n_stored_heads have
-// n_stored_parts partials, the others ceil(len / part_tokens).  bv (may be null): bias of the
-// V predictor, fp32-converted on the fly, added to dropped heads ([D - m] in storage dtype).
+// Merge split-K partials into out[B][H_q][d].  Heads with KV head < n_stored_heads have
+// n_stored_parts partials or, when stored_item_tokens is given (device; one entry per
+// stored_batch_per_slot sequences, written by the stored-head kernel), ceil(len / that entry);
+// the others ceil(len / part_tokens).  bv (may be null): bias of the V predictor, fp32-converted
+// on the fly, added to dropped heads ([D - m] in storage dtype).
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
-                         int part_tokens, const void* bv, cudaStream_t stream);
+                         const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
+                         const void* bv, cudaStream_t stream);
 
 }  // namespace echokv

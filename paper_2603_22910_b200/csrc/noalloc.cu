@@ -113,7 +113,7 @@ extern "C" int echokv_full_attention_noalloc(const echokv_config* cfg, const voi
   a.status = status;
   const int D = cfg->n_kv_heads * cfg->head_dim;
   if (launch_attn_stored(a, k_pool, v_pool, D, cfg->n_kv_heads, n_splits, s) != cudaSuccess) return ECHOKV_ECUDA;
-  if (launch_merge(a, out, cfg->n_kv_heads, n_splits, /*part_tokens=*/1, nullptr, s) != cudaSuccess)
+  if (launch_merge(a, out, cfg->n_kv_heads, n_splits, nullptr, 1, /*part_tokens=*/1, nullptr, s) != cudaSuccess)
     return ECHOKV_ECUDA;
   if (dev_status_out &&
       cudaMemcpyAsync(dev_status_out, status, sizeof(int32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)

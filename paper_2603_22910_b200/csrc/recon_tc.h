@@ -15,6 +15,9 @@ struct TcLayerMaps {
   bool weights_ready = false;
 };
 
+// TMA descriptor of a bf16 pool [rows][width]: boxes of box_rows token rows x 64 features, 128-byte swizzle.
+cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows);
+
 bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m);
 
 cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const void* v_pool, int width,

@@ -448,7 +448,8 @@ cudaError_t launch_recon_simt(const AttnArgs& a, const ReconArgs& r, cudaStream_
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads,
-                             int n_stored_parts, int part_tokens, const T* __restrict__ bv) {
+                             int n_stored_parts, const int32_t* __restrict__ stored_item_tokens,
+                             int stored_batch_per_slot, int part_tokens, const T* __restrict__ bv) {
   const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
   const int DH = a.head_dim;
   const size_t oidx = ((size_t)b * a.n_q_heads + h) * DH + j;
@@ -462,7 +463,15 @@ __global__ void merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_h
   const int g = a.n_q_heads / a.n_kv_heads;
   const int kvh = h / g;
   const bool stored = kvh < n_stored_heads;
-  const int n = stored ? n_stored_parts : (len + part_tokens - 1) / part_tokens;
+  int n;
+  if (!stored) {
+    n = (len + part_tokens - 1) / part_tokens;
+  } else if (stored_item_tokens != nullptr) {
+    const int item_tokens = stored_item_tokens[b / stored_batch_per_slot];
+    n = (len + item_tokens - 1) / item_tokens;
+  } else {
+    n = n_stored_parts;
+  }
   const size_t base = ((size_t)b * a.n_q_heads + h) * a.parts.max_parts;
   float M = -INFINITY;
   for (int p = 0; p < n; ++p) M = fmaxf(M, a.parts.ml[base + p].x);
@@ -484,13 +493,16 @@ __global__ void merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_h
 }
 
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
-                         int part_tokens, const void* bv, cudaStream_t stream) {
+                         const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
+                         const void* bv, cudaStream_t stream) {
   dim3 grid(a.n_q_heads, a.batch);
   if (a.dtype == ECHOKV_BF16) {
     merge_kernel<__nv_bfloat16><<<grid, a.head_dim, 0, stream>>>(
-        a, out, n_stored_heads, n_stored_parts, part_tokens, (const __nv_bfloat16*)bv);
+        a, out, n_stored_heads, n_stored_parts, stored_item_tokens, stored_batch_per_slot, part_tokens,
+        (const __nv_bfloat16*)bv);
   } else {
     merge_kernel<float><<<grid, a.head_dim, 0, stream>>>(a, out, n_stored_heads, n_stored_parts,
+                                                         stored_item_tokens, stored_batch_per_slot,
                                                          part_tokens, (const float*)bv);
   }
   return cudaGetLastError();

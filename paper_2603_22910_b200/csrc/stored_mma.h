@@ -1,0 +1,25 @@
+// Tensor-core (mma.sync) + TMA attention over stored bf16 heads of 128 dims: host interface.
+#pragma once
+
+#include <cuda.h>
+
+#include "kernels.h"
+
+namespace echokv {
+
+constexpr int kStoredMaxBatchPerLaunch = 512;   // sequences one launch indexes in shared memory
+constexpr int kStoredMaxLaunches = 32;          // launches (and published item sizes) per call
+
+bool stored_mma_supported(int dtype, int head_dim, int group, int max_batch);
+
+// Token rows per TMA box of the pool maps this kernel wants: min(page_tokens, 64); 64 features wide.
+int stored_rows_per_box(int page_tokens);
+
+// Eq. 7 for the query heads of KV heads 0 .. n_heads-1 of the pool behind k_map / v_map.  One
+// split-K partial per (sequence, item, query head), item = a range of item_tokens tokens; the
+// kernel chooses item_tokens and writes it to item_tokens_slots[launch index] (one launch per
+// kStoredMaxBatchPerLaunch sequences) for the merge kernel.
+cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, const CUtensorMap& v_map,
+                                   int n_heads, int32_t* item_tokens_slots, int sm_count, cudaStream_t stream);
+
+}  // namespace echokv

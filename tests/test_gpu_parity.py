@@ -67,6 +67,53 @@ def test_small_shapes_against_oracle(name, base, over, lens, path):
     case.close()
 
 
+STORED = [
+    # name, base, overrides, lens: shapes of the stored-head attention (anchor layer 0, retained heads of layer 1)
+    ("mha", synth.C1, dict(batch=3, context=2100), [2100, 1025, 64]),
+    ("gqa4", synth.C2, dict(batch=3, context=1500, n_retained_heads=3, random_pages=True), [1500, 257, 1]),
+    ("gqa2_pages32", synth.C2, dict(n_q_heads=16, batch=2, context=900, page_tokens=32, random_pages=True), [900, 33]),
+    ("gqa8_pages64", synth.C2, dict(n_q_heads=32, n_kv_heads=4, n_retained_heads=2, batch=2, context=700,
+                                    page_tokens=64), [700, 65]),
+    ("gqa4_pages128", synth.C2, dict(batch=2, context=1000, page_tokens=128, n_retained_heads=5,
+                                     random_pages=True), [1000, 129]),
+]
+
+
+@pytest.mark.parametrize("name,base,over,lens", STORED, ids=[s[0] for s in STORED])
+@pytest.mark.parametrize("stored_path", [0, 1])
+def test_stored_head_kernels_against_oracle(name, base, over, lens, stored_path):
+    w = base.replace(**over)
+    case = Case(w, lens=lens, layers=[0, 1])
+    assert case.ctx.stored_path() == 1        # bf16, head_dim 128: the TMA + tensor-core kernel by default
+    case.ctx.set_stored_path(stored_path)
+    check_layers(case, "%s stored_path %d" % (name, stored_path))
+    case.close()
+
+
+def test_slots_that_hold_no_token_may_contain_anything():
+    # cache slots past a sequence's length, and pages no sequence uses, were never written: fill
+    # them with NaN and huge values; the result must not change
+    w = synth.C2.replace(batch=2, context=600, n_retained_heads=3, random_pages=True)
+    lens = [600, 70]
+    n_pages = 2 * w.pages_per_seq + 9
+    case = Case(w, lens=lens, layers=[0, 1], n_pages=n_pages)
+    clean = {l: case.run(l) for l in (0, 1)}
+    used = torch.zeros((n_pages, w.page_tokens), dtype=torch.bool)
+    for b, L in enumerate(lens):
+        for t in range(L):
+            used[int(case.table[b, t // w.page_tokens]), t % w.page_tokens] = True
+    junk = torch.tensor([float("nan"), float("inf"), -3.0e38, 1.0e30], dtype=torch.float32)
+    for l in (0, 1):
+        for pool in (case.ctx.k_pools[l], case.ctx.v_pools[l]):
+            fill = junk[torch.arange(pool.shape[-1]) % 4].to(pool.dtype).to(pool.device)
+            pool[(~used).to(pool.device)] = fill
+    for l in (0, 1):
+        np.testing.assert_array_equal(case.run(l), clean[l])
+        assert_parity(case.run(l), case.oracle(l), w.dtype, "junk in unused slots, layer %d" % l)
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
 def test_config3_shape_multi_layer_random_pages():
     # 8 layers = two groups of S = 4; ragged lengths; pool larger than needed, random page order
     w = synth.C3.replace(n_layers=8, batch=2, context=420)
