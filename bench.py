@@ -1,20 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the EchoKV decode path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4] [--mode compressed|full]
+                    [--impl ours|reference]
 
-One "step" = one pass of the whole hot path over one batch of synthetic input:
-append the new token to the anchor layer and to the compressed layer (which keeps
-only the retained heads), then decode attention on the compressed layer -- retained
-heads from the cache, dropped heads reconstructed on chip -- including the split-K
-merge.  `value` is decode tokens per second (sequences advanced per second) with the
-caches resident in HBM; `e2e` is the same step driven from pinned host buffers
-through echokv_layer_step_host.  With N > 1 every rank runs an independent replica
-of the batch (the path has no exchange step): weak scaling, no collective on the
-data path.
+One "step" = one pass of the whole hot path over one batch of synthetic input.  For the
+single-layer workloads (c1, the default and the headline; c2; a point of the c4 sweep) that is:
+append the new token to the anchor layer and to the compressed layer (which keeps only the
+retained heads), then decode attention on the compressed layer -- retained heads from the
+cache, dropped heads reconstructed on chip -- including the split-K merge.  For c3 it is the
+whole 32-layer decode step: per layer an append and the layer's attention (full-cache on the
+8 anchor layers, reconstruct-then-attend on the 24 compressed ones).  --mode full times the
+uncompressed path instead (full-cache attention on the anchor layer).
 
---impl reference times the CPU oracle (numpy, fp64) on a bounded sample of the same
-workload.
+`value` is decode tokens per second (sequences advanced per second) with the caches resident
+in HBM; `e2e` is the same step driven from pinned host buffers through
+echokv_layer_step_host.  With N > 1 every rank runs an independent replica of the batch (the
+path has no exchange step): weak scaling, no collective on the data path.
+
+--impl reference times the CPU oracle (numpy, fp64) on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
@@ -34,7 +38,7 @@ UNIT = "tokens/s"
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu captures summarised under profiles/; None until a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": None}
+NCU_TRAFFIC_BYTES = {}
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -47,9 +51,15 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def workload_by_name(name, batch=0, context=0):
+def workload_by_name(name, batch=0, context=0, page_tokens=0, random_pages=False, ratio=75):
     from paper_2603_22910_b200 import synth
-    w = {"c1": synth.C1, "c2": synth.C2, "c0": synth.C0}[name]
+    if name == "c4":
+        return synth.c4_point(ratio, context or 16384, batch or 8)
+    w = {"c1": synth.C1, "c2": synth.C2, "c3": synth.C3}[name]
+    if page_tokens:
+        w = w.replace(page_tokens=page_tokens, name=w.name + "_P%d" % page_tokens)
+    if random_pages:
+        w = w.replace(random_pages=True, name=w.name + "_randpages")
     if batch:
         w = w.replace(batch=batch, name=w.name + "_B%d" % batch)
     if context:
@@ -58,8 +68,9 @@ def workload_by_name(name, batch=0, context=0):
 
 
 def algorithmic_work(w):
-    """Per launch of the fused kernel: FLOPs of Eq. 3 (both predictors) plus Eq. 7 on the dropped
-    heads, and the bytes the method must move (predictor inputs once, predictors once)."""
+    """Per launch of the fused kernel (one compressed layer): FLOPs of Eq. 3 (both predictors) plus
+    Eq. 7 on the dropped heads, and the bytes the method must move (predictor inputs once,
+    predictors once)."""
     tokens = w.batch * w.context
     g = w.n_q_heads // w.n_kv_heads
     n_drop_q = (w.n_kv_heads - w.n_retained_heads) * g
@@ -130,6 +141,95 @@ def physical_gpu_index(local_index):
 
 
 # --------------------------------------------------------------------------------------------
+# Workload state on the GPU
+# --------------------------------------------------------------------------------------------
+class State:
+    """A workload resident on one GPU: pools filled through the block table from the seeded
+    generators (drawn on the device: the largest workloads do not fit host memory), predictors,
+    one decode query per layer, and the newest token of every layer (re-appended by each step)."""
+
+    def __init__(self, w, local_rank, layers):
+        import torch
+        from paper_2603_22910_b200 import binding, synth
+        self.w, self.layers = w, layers
+        self.dev = dev = torch.device("cuda", local_rank)
+        self.ctx = ctx = binding.Context(binding.config_for(w, device=local_rank))
+        self.table = synth.block_table(w)
+        ctx.set_block_table(self.table)
+        t0 = time.perf_counter()
+        needed = sorted(set(layers) | {w.anchor_of(l) for l in layers})
+        tdt = synth.torch_dtype(w)
+        self.new_dev, self.new_host, self.q_dev, self.q_host = {}, {}, {}, {}
+        for l in needed:
+            width = w.D if w.is_anchor(l) else w.m
+            for kind, pools in (("k", ctx.k_pools), ("v", ctx.v_pools)):
+                newest = torch.zeros((w.batch, w.D), dtype=tdt, device=dev)
+                for b in range(w.batch):
+                    if width == 0:
+                        continue
+                    ids = self.table[b].long().to(dev)
+                    x = synth.layer_cache(w, l, kind, b, width=width, device=dev)
+                    pad = w.pages_per_seq * w.page_tokens - w.context
+                    if pad:
+                        x = torch.cat([x, torch.zeros((pad, width), dtype=tdt, device=dev)])
+                    pools[l][ids] = x.reshape(w.pages_per_seq, w.page_tokens, width)
+                    newest[b, :width] = x[w.context - 1]
+                    del x
+                self.new_dev[(l, kind)] = newest
+                self.new_host[(l, kind)] = newest.cpu().pin_memory()
+            if not w.is_anchor(l):
+                Wk = synth.predictor_weights(w, l, "k", device=dev)
+                Wv = synth.predictor_weights(w, l, "v", device=dev)
+                ctx.set_weights(l, Wk, Wv)
+            self.q_dev[l] = synth.queries(w, l, device=dev)
+            self.q_host[l] = self.q_dev[l].cpu().pin_memory()
+        self.lens_host = torch.full((w.batch,), w.context, dtype=torch.int32).pin_memory()
+        self.lens = self.lens_host.to(dev)
+        self.positions = self.lens - 1
+        shape = (w.batch, w.n_q_heads, w.head_dim)
+        self.out = {l: torch.empty(shape, dtype=torch.float32, device=dev) for l in layers}
+        self.out_host = {l: torch.empty(shape, dtype=torch.float32).pin_memory() for l in layers}
+        torch.cuda.synchronize()
+        self.gen_s = time.perf_counter() - t0
+
+    def stored_sequence(self, layer, kind, b):
+        """Stored values [L, width] of one sequence, gathered back from the pool (oracle input)."""
+        pools = self.ctx.k_pools if kind == "k" else self.ctx.v_pools
+        if pools[layer] is None:
+            import torch
+            return torch.zeros((self.w.context, 0), dtype=self.ctx.tdtype)
+        ids = self.table[b].long().to(self.dev)
+        x = pools[layer][ids].reshape(-1, pools[layer].shape[-1])[: self.w.context]
+        return x.cpu()
+
+    def oracle_inputs(self, layer, b):
+        """Widened (float64) oracle inputs of sequence b at `layer`, from what the GPU holds."""
+        from oracle import echokv_oracle as O
+        from paper_2603_22910_b200 import synth
+        w = self.w
+        st = synth.to_numpy_stored
+        a = w.anchor_of(layer)
+        q = O.widen(st(self.q_host[layer]))[b]
+        kg = O.widen(st(self.stored_sequence(a, "k", b)))
+        vg = O.widen(st(self.stored_sequence(a, "v", b)))
+        if w.is_anchor(layer):
+            return q, kg, vg
+        kl = O.widen(st(self.stored_sequence(layer, "k", b)))
+        vl = O.widen(st(self.stored_sequence(layer, "v", b)))
+        Wk, Wv = (O.widen(st(t)) for t in self.ctx._weights[layer][:2])
+        return q, kg, vg, kl, vl, Wk, Wv
+
+
+def plan_layers(w, mode):
+    """(layers resident on the GPU, [(layer, attend?)] of one step)."""
+    if mode == "full":
+        return [0], [(0, True)]
+    if w.n_layers > 2:                     # the whole multi-layer decode step
+        return list(range(w.n_layers)), [(l, True) for l in range(w.n_layers)]
+    return [0, 1], [(0, False), (1, True)]  # the anchor only receives its token; layer 1 attends
+
+
+# --------------------------------------------------------------------------------------------
 # CPU oracle legs
 # --------------------------------------------------------------------------------------------
 def oracle_threads():
@@ -146,40 +246,46 @@ def oracle_threads():
         return os.cpu_count() or 1
 
 
-def oracle_inputs(w, layer, b):
-    """Widened (float64) oracle inputs of sequence b from the seeded generators."""
+def oracle_layer(inputs, w):
     from oracle import echokv_oracle as O
-    from paper_2603_22910_b200 import synth
-    a = w.anchor_of(layer)
-    st = synth.to_numpy_stored
-    kg = O.widen(st(synth.layer_cache(w, a, "k", b)))
-    vg = O.widen(st(synth.layer_cache(w, a, "v", b)))
-    kl = O.widen(st(synth.layer_cache(w, layer, "k", b, width=w.m)))
-    vl = O.widen(st(synth.layer_cache(w, layer, "v", b, width=w.m)))
-    Wk = O.widen(st(synth.predictor_weights(w, layer, "k")))
-    Wv = O.widen(st(synth.predictor_weights(w, layer, "v")))
-    q = O.widen(st(synth.queries(w, layer)))[b]
-    return q, kg, vg, kl, vl, Wk, Wv
+    if len(inputs) == 3:
+        return O.full_attention(inputs[0], inputs[1], inputs[2], w.n_kv_heads)
+    return O.decode_attention(*inputs, n_kv_heads=w.n_kv_heads)
 
 
-def time_oracle(w, budget_s, max_seqs=None, full=False):
-    """The oracle as it stands on whole sequences of the workload until `budget_s` is used."""
-    from oracle import echokv_oracle as O
-    layer = 1
-    done, elapsed = 0, 0.0
-    outs = {}
-    for b in range(w.batch if max_seqs is None else min(w.batch, max_seqs)):
-        args = oracle_inputs(w, layer, b)
+def time_oracle(state, step_layers, budget_s):
+    """The oracle as it stands on a bounded sample of the workload.  Returns (tokens/s of the
+    oracle scaled to the whole step, sample description, {(layer, b): oracle output})."""
+    w = state.w
+    attend = [l for l, a in step_layers if a]
+    outs, elapsed = {}, 0.0
+    if len(attend) == 1:
+        # whole sequences of the batch, all heads, all tokens, until the budget is used
+        layer = attend[0]
+        for b in range(min(w.batch, 4)):
+            inputs = state.oracle_inputs(layer, b)
+            t0 = time.perf_counter()
+            outs[(layer, b)] = oracle_layer(inputs, w)
+            elapsed += time.perf_counter() - t0
+            if elapsed >= budget_s:
+                break
+        n_seq = len(outs)
+        return n_seq / elapsed, ("%d of %d sequences of the batch, all heads, all %d tokens (%.1f s)"
+                                 % (n_seq, w.batch, w.context, elapsed)), outs
+    # multi-layer step: one group of S consecutive layers (an anchor and the layers that lean on
+    # it) for one sequence; every group costs the same, so the step takes n_groups times as long
+    S = w.group_size
+    group = [l for l in attend if l < S]
+    b = 0
+    for l in group:
+        inputs = state.oracle_inputs(l, b)
         t0 = time.perf_counter()
-        if full:     # the anchor layer's stored cache
-            outs[b] = O.full_attention(args[0], args[1], args[2], w.n_kv_heads)
-        else:
-            outs[b] = O.decode_attention(*args, n_kv_heads=w.n_kv_heads)
+        outs[(l, b)] = oracle_layer(inputs, w)
         elapsed += time.perf_counter() - t0
-        done += 1
-        if elapsed >= budget_s:
-            break
-    return done, elapsed, outs
+    scale = len(attend) / float(len(group))
+    return 1.0 / (elapsed * scale), ("sequence 0 of %d, layers 0..%d (one group of S = %d), all heads, all %d "
+                                     "tokens (%.1f s); extrapolated x%.0f to the %d layers"
+                                     % (w.batch, S - 1, S, w.context, elapsed, scale, len(attend))), outs
 
 
 def run_reference(args):
@@ -188,41 +294,59 @@ def run_reference(args):
     if rank != 0:
         return 0
     from oracle import echokv_oracle as O
-    w = workload_by_name(args.workload, args.batch, args.context)
-    layer = 1
+    from paper_2603_22910_b200 import synth
+    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio)
+    st = synth.to_numpy_stored
+    full = args.mode == "full"
+    layer = 0 if full else 1
+    a = w.anchor_of(layer)
+    q = O.widen(st(synth.queries(w, layer)))[0]
+    kg = O.widen(st(synth.layer_cache(w, a, "k", 0)))
+    vg = O.widen(st(synth.layer_cache(w, a, "v", 0)))
     g = w.n_q_heads // w.n_kv_heads
-    dropped_q = list(range(w.n_retained_heads * g, w.n_q_heads))
-    inputs = oracle_inputs(w, layer, 0)
-    # probe: one dropped KV head's query heads on sequence 0
-    probe_heads = dropped_q[:g]
-    t0 = time.perf_counter()
-    O.decode_attention_query_heads(*inputs, n_kv_heads=w.n_kv_heads, query_heads=probe_heads)
-    t_head = time.perf_counter() - t0
     total = args.steps + args.warmup
     budget = 150.0
-    n_kv_sample = max(1, min(w.n_kv_heads - w.n_retained_heads, int(budget / max(total * t_head, 1e-9))))
-    heads = dropped_q[: n_kv_sample * g]
+    if full:
+        n_units, heads = w.n_kv_heads, list(range(w.n_q_heads))
+        d = w.head_dim
+
+        def run(n_kv):   # the first n_kv KV heads of the stored cache
+            return O.full_attention(q[: n_kv * g], kg[:, : n_kv * d], vg[:, : n_kv * d], n_kv)
+    else:
+        kl = O.widen(st(synth.layer_cache(w, layer, "k", 0, width=w.m)))
+        vl = O.widen(st(synth.layer_cache(w, layer, "v", 0, width=w.m)))
+        Wk = O.widen(st(synth.predictor_weights(w, layer, "k")))
+        Wv = O.widen(st(synth.predictor_weights(w, layer, "v")))
+        n_units = w.n_kv_heads - w.n_retained_heads
+        heads = list(range(w.n_retained_heads * g, w.n_q_heads))
+
+        def run(n_kv):   # the first n_kv dropped KV heads (the retained ones cost next to nothing)
+            return O.decode_attention_query_heads(q, kg, vg, kl, vl, Wk, Wv, n_kv_heads=w.n_kv_heads,
+                                                  query_heads=heads[: n_kv * g])
+    t0 = time.perf_counter()
+    run(1)
+    t_head = time.perf_counter() - t0
+    n_sample = max(1, min(n_units, int(budget / max(total * t_head, 1e-9))))
     times = []
     for i in range(total):
         t0 = time.perf_counter()
-        O.decode_attention_query_heads(*inputs, n_kv_heads=w.n_kv_heads, query_heads=heads)
+        run(n_sample)
         dt = time.perf_counter() - t0
         if i >= args.warmup:
             times.append(dt)
-    # a step covers n_kv_sample of the (H_kv - r) dropped heads of ONE of the B sequences; the
-    # retained heads cost next to nothing beside them, so a whole batch step takes about
-    # B * (H_kv - r) / n_kv_sample times as long
-    frac = n_kv_sample / float(w.n_kv_heads - w.n_retained_heads)
+    # a step covers n_sample of the n_units KV heads of ONE of the B sequences of ONE layer
+    n_attend = w.n_layers if (w.n_layers > 2 and not full) else 1
     t_step = sum(times) / len(times)
-    t_batch = t_step / frac * w.batch
+    t_batch = t_step / (n_sample / float(n_units)) * w.batch * n_attend
     value = w.batch / t_batch
-    sample = ("sequence 0 of %d, %d of %d dropped KV heads per step (all %d tokens), scaled to the full batch"
-              % (w.batch, n_kv_sample, w.n_kv_heads - w.n_retained_heads, w.context))
+    sample = ("sequence 0 of %d, %d of %d %s KV heads per step (all %d tokens), one layer; scaled to the full "
+              "batch%s" % (w.batch, n_sample, n_units, "stored" if full else "dropped", w.context,
+                           " and to %d layers" % n_attend if n_attend > 1 else ""))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_batch * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": workload_config(w),
+        "data": "synthetic", "config": workload_config(w, full),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -233,18 +357,25 @@ def run_reference(args):
 
 def workload_config(w, full=False):
     elem = 2 if w.dtype == "bf16" else 4
+    pages = "%d-token pages%s" % (w.page_tokens, " in a random order" if w.random_pages else "")
     if full:
-        what = ("%s, uncompressed: B=%d L=%d H_q=%d H_kv=%d d=%d, %s, %d-token pages, full-cache attention on the "
-                "anchor layer" % (w.name, w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype,
-                                  w.page_tokens))
+        what = ("%s, uncompressed: B=%d L=%d H_q=%d H_kv=%d d=%d, %s, %s, full-cache attention on the "
+                "anchor layer" % (w.name, w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, pages))
         gb = w.batch * w.context * 2 * w.D * elem / 1e9
+    elif w.n_layers > 2:
+        n_anchor = (w.n_layers + w.group_size - 1) // w.group_size
+        what = ("%s: %d layers (S=%d: %d anchor + %d compressed), B=%d L=%d H_q=%d H_kv=%d d=%d retained=%d "
+                "(D_in=%d -> D_drop=%d), %s, %s" % (w.name, w.n_layers, w.group_size, n_anchor, w.n_layers - n_anchor,
+                                                   w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim,
+                                                   w.n_retained_heads, w.d_in, w.d_drop, w.dtype, pages))
+        gb = w.batch * w.context * 2 * elem * (n_anchor * w.D + (w.n_layers - n_anchor) * w.d_in) / 1e9
     else:
-        what = ("%s: B=%d L=%d H_q=%d H_kv=%d d=%d retained=%d (D_in=%d -> D_drop=%d), %s, %d-token pages, "
+        what = ("%s: B=%d L=%d H_q=%d H_kv=%d d=%d retained=%d (D_in=%d -> D_drop=%d), %s, %s, "
                 "anchor + compressed layer" % (w.name, w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim,
-                                               w.n_retained_heads, w.d_in, w.d_drop, w.dtype, w.page_tokens))
+                                               w.n_retained_heads, w.d_in, w.d_drop, w.dtype, pages))
         gb = w.batch * w.context * 2 * w.d_in * elem / 1e9
     return {"workload": what, "global_batch": w.batch, "context": w.context,
-            "l2": "inputs (%.2f GB of cache per step) exceed the 126 MB L2; no flush needed" % gb,
+            "l2": "inputs (%.2f GB of cache read per step) exceed the 126 MB L2; no flush needed" % gb,
             "parallelism": "replicas"}
 
 
@@ -254,7 +385,7 @@ def workload_config(w, full=False):
 def run_ours(args):
     import numpy as np
     import torch
-    from paper_2603_22910_b200 import binding, build, synth
+    from paper_2603_22910_b200 import binding, build
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -274,63 +405,33 @@ def run_ours(args):
         dist.barrier()
     binding.lib()
 
-    w = workload_by_name(args.workload, args.batch, args.context)
+    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio)
     if world > 1:
         w = w.replace(seed=w.seed + 7919 * rank)   # every replica has its own batch
-    dev = torch.device("cuda", local_rank)
-    cfg = binding.config_for(w, device=local_rank)
-    ctx = binding.Context(cfg)
-    table = synth.block_table(w)
-    ctx.set_block_table(table)
-    anchor_l, layer = 0, 1
-    # caches: generated per sequence on the host with the seeded generators, laid out in pages
-    t_gen = time.perf_counter()
-    new = {(l, kind): torch.zeros((w.batch, w.D), dtype=synth.torch_dtype(w)) for l in (anchor_l, layer)
-           for kind in ("k", "v")}
-    for kind, pools in (("k", ctx.k_pools), ("v", ctx.v_pools)):
-        for b in range(w.batch):
-            anchor_f32 = synth.anchor_cache(w, anchor_l, kind, b)
-            ids = table[b].long().to(dev)
-            for l, width in ((anchor_l, w.D), (layer, w.m)):
-                if width == 0:
-                    continue
-                x = synth.layer_cache(w, l, kind, b, width=width, anchor_f32=anchor_f32)
-                pools[l][ids] = x.reshape(w.pages_per_seq, w.page_tokens, width).to(dev)
-                new[(l, kind)][b, :width] = x[-1]      # the step re-appends the newest token
-            del anchor_f32
-    new = {k: v.pin_memory() for k, v in new.items()}
-    Wk = synth.predictor_weights(w, layer, "k").to(dev)
-    Wv = synth.predictor_weights(w, layer, "v").to(dev)
-    ctx.set_weights(layer, Wk, Wv)
-    q_host = synth.queries(w, layer).pin_memory()
-    lens_host = torch.full((w.batch,), w.context, dtype=torch.int32).pin_memory()
-    out_host = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32).pin_memory()
-    q = q_host.to(dev)
-    new_dev = {k: v.to(dev) for k, v in new.items()}
-    lens = lens_host.to(dev)
-    positions = lens - 1
-    out = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
-    t_gen = time.perf_counter() - t_gen
-
     full = args.mode == "full"
+    resident, step_layers = plan_layers(w, args.mode)
+    st = State(w, local_rank, resident)
+    ctx, dev = st.ctx, st.dev
     if args.stored_path is not None:
         ctx.set_stored_path(args.stored_path)
+    last = [l for l, a in step_layers if a][-1]
+
+    def attend(l):
+        if full or w.is_anchor(l):   # the uncompressed mode / an anchor layer: Eq. 7 on the stored full cache
+            ctx.full_attention(l, st.q_dev[l], st.lens, out=st.out[l])
+        else:
+            ctx.decode_attention(l, st.q_dev[l], st.lens, out=st.out[l])
 
     def step():
-        ctx.append_kv(anchor_l, new_dev[(anchor_l, "k")], new_dev[(anchor_l, "v")], positions)
-        if full:     # the uncompressed mode / an anchor layer: Eq. 7 on the stored full cache
-            ctx.full_attention(anchor_l, q, lens, out=out)
-            return
-        ctx.append_kv(layer, new_dev[(layer, "k")], new_dev[(layer, "v")], positions)
-        ctx.decode_attention(layer, q, lens, out=out)
+        for l, a in step_layers:
+            ctx.append_kv(l, st.new_dev[(l, "k")], st.new_dev[(l, "v")], st.positions)
+            if a:
+                attend(l)
 
     def step_host():
-        if full:
-            ctx.layer_step_host(anchor_l, q_host, new[(anchor_l, "k")], new[(anchor_l, "v")], out_host, lens_host,
-                                attend=True)
-            return
-        ctx.layer_step_host(anchor_l, None, new[(anchor_l, "k")], new[(anchor_l, "v")], None, lens_host, attend=False)
-        ctx.layer_step_host(layer, q_host, new[(layer, "k")], new[(layer, "v")], out_host, lens_host, attend=True)
+        for l, a in step_layers:
+            ctx.layer_step_host(l, st.q_host[l] if a else None, st.new_host[(l, "k")], st.new_host[(l, "v")],
+                                st.out_host[l] if a else None, st.lens_host, attend=a)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -365,7 +466,7 @@ def run_ours(args):
     sync_all()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     launches = ctx.launch_count() - launches0
-    kernel_ms, kernel_launches = ctx.read_kernel_timing()
+    timing = ctx.read_kernel_timing_by_kind()
     ctx.set_kernel_timing(False)
     clocks = sampler.stop()
     status = ctx.device_status()
@@ -383,11 +484,11 @@ def run_ours(args):
     sync_all()
     ms_e2e = max_over_ranks(e2.elapsed_time(e3))
     elem = 2 if w.dtype == "bf16" else 4
-    n_host_layers = 1 if full else 2
-    h2d = (n_host_layers * 2 * w.batch * w.D * elem + w.batch * w.n_q_heads * w.head_dim * elem
-           + n_host_layers * 2 * w.batch * 4)
-    d2h = w.batch * w.n_q_heads * w.head_dim * 4
-    same = bool(torch.equal(out_host, out.cpu()))
+    n_attend = sum(1 for _, a in step_layers if a)
+    h2d = (len(step_layers) * (2 * w.batch * w.D * elem + 2 * w.batch * 4)
+           + n_attend * w.batch * w.n_q_heads * w.head_dim * elem)
+    d2h = n_attend * w.batch * w.n_q_heads * w.head_dim * 4
+    same = bool(torch.equal(st.out_host[last], st.out[last].cpu()))
 
     ms_step = ms_total / args.steps
     value = world * w.batch / (ms_step * 1e-3)
@@ -395,57 +496,69 @@ def run_ours(args):
 
     peaks, peaks_kind = load_peaks()
     flops, bytes_ = algorithmic_work(w)
-    k_ms = kernel_ms / max(kernel_launches, 1)
-    if full:
-        # Eq. 7 on the stored cache: every token's K and V row of every KV head is read once
-        bytes_ = w.batch * w.context * 2.0 * w.D * elem
-        achieved_gbs = bytes_ / (k_ms * 1e-3) / 1e9
-        peak_gbs = float(peaks["hbm_gbs"])
-        roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
-                    "frac": achieved_gbs / peak_gbs, "traffic": NCU_TRAFFIC_BYTES.get(args.workload + "_full"),
-                    "kernel": "attn_stored_mma_kernel" if ctx.stored_path() == 1 else "attn_stored_kernel",
-                    "kernel_ms": k_ms, "kernel_launches": kernel_launches,
-                    "peak_source": "%s (STREAM-style copy)" % peaks_kind,
-                    "algorithmic_bytes_per_launch": bytes_}
-    else:
+    stored_ms, stored_n = timing["stored"]
+    recon_ms, recon_n = timing["recon"]
+    full_bytes = w.batch * w.context * 2.0 * w.D * elem   # a stored layer: every K and V row once
+    stored_info = None
+    if stored_n:
+        k_ms = stored_ms / stored_n
+        stored_info = {"kernel": "attn_stored_mma_kernel" if ctx.stored_path() == 1 else "attn_stored_kernel",
+                       "kernel_ms": k_ms, "kernel_launches": stored_n, "achieved_gbs": full_bytes / (k_ms * 1e-3) / 1e9,
+                       "frac_of_%s_hbm" % peaks_kind: full_bytes / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"])}
+    if recon_n:
+        k_ms = recon_ms / recon_n
         achieved_tf = flops / (k_ms * 1e-3) / 1e12
         peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
         roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                     "frac": achieved_tf / peak_tf, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                    "kernel": "recon_tc_kernel", "kernel_ms": k_ms, "kernel_launches": kernel_launches,
+                    "kernel": "recon_tc_kernel" if ctx.decode_path() == 2 else "recon_simt_kernel",
+                    "kernel_ms": k_ms, "kernel_launches": recon_n,
+                    "share_of_step": recon_ms / ms_total,
                     "peak_source": "%s (bf16 sustained; kernel timed inside a long step)" % peaks_kind,
                     "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": bytes_,
                     "hbm_frac_of_%s" % peaks_kind: bytes_ / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
                     "frac_of_burst_peak": achieved_tf / float(peaks["bf16_tflops"])}
+        if stored_info:
+            roofline["anchor_layers"] = stored_info
+    else:
+        k_ms = stored_ms / max(stored_n, 1)
+        achieved_gbs = full_bytes / (k_ms * 1e-3) / 1e9
+        peak_gbs = float(peaks["hbm_gbs"])
+        roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
+                    "frac": achieved_gbs / peak_gbs, "traffic": NCU_TRAFFIC_BYTES.get(args.workload + "_full"),
+                    "kernel": stored_info["kernel"] if stored_info else None,
+                    "kernel_ms": k_ms, "kernel_launches": stored_n, "share_of_step": stored_ms / ms_total,
+                    "peak_source": "%s (STREAM-style copy)" % peaks_kind,
+                    "algorithmic_bytes_per_launch": full_bytes}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
         "config": workload_config(w, full),
-        "us_per_layer_step": ms_step * 1e3,
-        "kv_tokens_scanned_per_s": world * w.batch * w.context / (ms_step * 1e-3),
+        "us_per_layer_step": ms_step * 1e3 / n_attend,
+        "kv_tokens_scanned_per_s": world * w.batch * w.context * n_attend / (ms_step * 1e-3),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps, "matches_device_path": same},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "decode_path": ctx.decode_path(), "stored_path": ctx.stored_path(),
-        "input_generation_s": t_gen,
+        "input_generation_s": st.gen_s,
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_seq, t_cpu, outs = time_oracle(w, budget_s=12.0, max_seqs=4, full=full)
-        gpu = out.cpu().numpy().astype(np.float64)
+        cpu_value, sample, outs = time_oracle(st, step_layers, budget_s=12.0)
         worst_abs, num, den = 0.0, 0.0, 0.0
-        for b, ref in outs.items():
-            worst_abs = max(worst_abs, float(np.max(np.abs(gpu[b] - ref))))
-            num += float(np.sum((gpu[b] - ref) ** 2))
+        for (l, b), ref in outs.items():
+            gpu = st.out[l][b].cpu().numpy().astype(np.float64)
+            worst_abs = max(worst_abs, float(np.max(np.abs(gpu - ref))))
+            num += float(np.sum((gpu - ref) ** 2))
             den += float(np.sum(ref ** 2))
-        line["cpu_baseline"] = {"value": n_seq / t_cpu, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                                "sample": "%d of %d sequences of the batch, all heads, all %d tokens (%.1f s)"
-                                          % (n_seq, w.batch, w.context, t_cpu)}
-        line["parity_vs_oracle"] = {"sequences": n_seq, "max_abs": worst_abs, "rel_l2": (num / max(den, 1e-300)) ** 0.5}
+        line["cpu_baseline"] = {"value": cpu_value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                                "sample": sample}
+        line["parity_vs_oracle"] = {"outputs": sorted(outs.keys()), "max_abs": worst_abs,
+                                    "rel_l2": (num / max(den, 1e-300)) ** 0.5}
     if rank == 0:
         print(json.dumps(line))
     ctx.close()
@@ -459,7 +572,10 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c1", choices=["c1", "c2"])
+    ap.add_argument("--workload", default="c1", choices=["c1", "c2", "c3", "c4"],
+                    help="c1 (default, the headline): Llama-2-7B-shaped layer; c2: Llama-3-8B-shaped GQA layer; "
+                         "c3: 32-layer Llama-2-7B-shaped decode step; c4: one point of the GQA sweep "
+                         "(--ratio, --context, --batch)")
     ap.add_argument("--mode", default="compressed", choices=["compressed", "full"],
                     help="compressed: decode attention of a compressed layer (the headline); full: the "
                          "uncompressed path, full-cache attention on the anchor layer")
@@ -469,8 +585,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
+    ap.add_argument("--ratio", type=int, default=75, choices=[25, 50, 75],
+                    help="c4 only: percent of the layer's KV heads discarded")
+    ap.add_argument("--page-tokens", type=int, default=0, choices=[0, 16, 32, 64, 128],
+                    help="override the tokens per cache page (default 16)")
+    ap.add_argument("--random-pages", action="store_true", help="pages of the pool in a seeded random order")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.workload == "c3" and args.steps == 50 and args.impl == "ours":
+        args.steps = 10      # a 32-layer step is ~25x a single layer-step
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

@@ -191,6 +191,12 @@ int echokv_set_stored_path(echokv_ctx* ctx, int path);
 int echokv_set_kernel_timing(echokv_ctx* ctx, int enable);
 int echokv_read_kernel_timing(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
 
+/* The same reading split by kernel: total_ms and n_launches are host arrays of
+ * ECHOKV_TIMED_KINDS entries, indexed by ECHOKV_TIMED_STORED (stored-head attention of an
+ * anchor / uncompressed layer) and ECHOKV_TIMED_RECON (fused reconstruct-attend kernel). */
+enum { ECHOKV_TIMED_STORED = 0, ECHOKV_TIMED_RECON = 1, ECHOKV_TIMED_KINDS = 2 };
+int echokv_read_kernel_timing_by_kind(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
+
 /* Full-cache attention for callers that cannot allocate device memory (the paper has no
  * counterpart to this entry point; it exists for the library's users).
  *

@@ -63,6 +63,7 @@ EXPORTS = {
     "echokv_set_stored_path": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_read_kernel_timing": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "echokv_read_kernel_timing_by_kind": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "echokv_full_attention_noalloc": (C.c_int, [C.POINTER(echokv_config), C.c_void_p, C.c_void_p, C.c_void_p,
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                                 C.c_void_p, C.c_void_p]),
@@ -243,6 +244,12 @@ class Context:
         ms, n = C.c_double(0.0), C.c_int64(0)
         _check(lib().echokv_read_kernel_timing(self.handle, C.byref(ms), C.byref(n)), "echokv_read_kernel_timing")
         return ms.value, n.value
+
+    def read_kernel_timing_by_kind(self):
+        """{"stored": (ms, launches), "recon": (ms, launches)} since the last read."""
+        ms, n = (C.c_double * 2)(), (C.c_int64 * 2)()
+        _check(lib().echokv_read_kernel_timing_by_kind(self.handle, ms, n), "echokv_read_kernel_timing_by_kind")
+        return {"stored": (ms[0], n[0]), "recon": (ms[1], n[1])}
 
     def _out(self, q):
         return self.torch.empty(q.shape, dtype=self.torch.float32, device=self.device)

@@ -94,6 +94,7 @@ struct echokv_ctx {
   bool timing = false;
   size_t timed = 0;                                         // event pairs in use
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> events;  // grown on demand, reused
+  std::vector<int> event_kind;                              // ECHOKV_TIMED_* of each pair
   ~echokv_ctx() {
     for (auto& e : events) {
       cudaEventDestroy(e.first);
@@ -153,14 +154,16 @@ struct ScopedKernelTimer {
   echokv_ctx* c;
   cudaStream_t s;
   cudaEvent_t stop = nullptr;
-  ScopedKernelTimer(echokv_ctx* ctx, cudaStream_t stream) : c(ctx), s(stream) {
+  ScopedKernelTimer(echokv_ctx* ctx, cudaStream_t stream, int kind) : c(ctx), s(stream) {
     if (!c->timing) return;
     if (c->timed == c->events.size()) {
       cudaEvent_t a, b;
       if (cudaEventCreate(&a) != cudaSuccess) return;
       if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return; }
       c->events.emplace_back(a, b);
+      c->event_kind.push_back(kind);
     }
+    c->event_kind[c->timed] = kind;
     auto& e = c->events[c->timed++];
     cudaEventRecord(e.first, s);
     stop = e.second;
@@ -200,7 +203,7 @@ int attend_stored_layer(echokv_ctx* c, const Layer& L, const void* q, float* out
   const int n_splits = stored_splits(c, B, H);
   const int32_t* item_tokens = nullptr;
   {
-    ScopedKernelTimer timer(c, s);
+    ScopedKernelTimer timer(c, s, ECHOKV_TIMED_STORED);
     if (attend_stored_heads(c, a, L, c->d.D, H, n_splits, &item_tokens, s) != cudaSuccess) return ECHOKV_ECUDA;
   }
   if (launch_merge(a, out, H, n_splits, item_tokens, kStoredMaxBatchPerLaunch, c->d.part_tokens, nullptr, s) !=
@@ -399,7 +402,7 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   ra.capacity_tokens = c->d.capacity;
   cudaError_t e;
   {
-    ScopedKernelTimer timer(c, s);
+    ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
     if (c->path == 2) {
       e = launch_recon_tc(a, ra, A.tc, L.tc, c->sm_count, s);
     } else {
@@ -470,18 +473,35 @@ int echokv_set_kernel_timing(echokv_ctx* c, int enable) {
   return ECHOKV_OK;
 }
 
-int echokv_read_kernel_timing(echokv_ctx* c, double* total_ms, int64_t* n_launches) {
+int echokv_read_kernel_timing_by_kind(echokv_ctx* c, double* total_ms, int64_t* n_launches) {
   if (!c || !total_ms || !n_launches) return ECHOKV_EINVAL;
   if (cudaDeviceSynchronize() != cudaSuccess) return ECHOKV_ECUDA;
-  double sum = 0.0;
+  for (int k = 0; k < ECHOKV_TIMED_KINDS; ++k) {
+    total_ms[k] = 0.0;
+    n_launches[k] = 0;
+  }
   for (size_t i = 0; i < c->timed; ++i) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, c->events[i].first, c->events[i].second) != cudaSuccess) return ECHOKV_ECUDA;
-    sum += ms;
+    total_ms[c->event_kind[i]] += ms;
+    n_launches[c->event_kind[i]] += 1;
   }
-  *total_ms = sum;
-  *n_launches = (int64_t)c->timed;
   c->timed = 0;
+  return ECHOKV_OK;
+}
+
+int echokv_read_kernel_timing(echokv_ctx* c, double* total_ms, int64_t* n_launches) {
+  if (!c || !total_ms || !n_launches) return ECHOKV_EINVAL;
+  double ms[ECHOKV_TIMED_KINDS];
+  int64_t n[ECHOKV_TIMED_KINDS];
+  const int rc = echokv_read_kernel_timing_by_kind(c, ms, n);
+  if (rc != ECHOKV_OK) return rc;
+  *total_ms = 0.0;
+  *n_launches = 0;
+  for (int k = 0; k < ECHOKV_TIMED_KINDS; ++k) {
+    *total_ms += ms[k];
+    *n_launches += n[k];
+  }
   return ECHOKV_OK;
 }
 
