@@ -38,9 +38,21 @@ UNIT = "tokens/s"
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu captures summarised under profiles/; None until a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    "c1": 4 * 619.0e6,        # recon_tc_kernel: B = 2 capture x 4 (tokens)
+    "c2": 8 * 346.8e6,        # recon_tc_kernel: B = 2 capture x 8
+    "c1_full": 4 * 275.0e6,   # attn_stored_mma_kernel: B = 2 capture x 4
+    "c2_full": 8 * 273.8e6,   # attn_stored_mma_kernel: B = 2 capture x 8
+}
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def traffic_of(args, key):
+    """The stored ncu figure, only for the exact workload it was scaled to."""
+    if args.batch or args.context or args.page_tokens or args.random_pages:
+        return None
+    return NCU_TRAFFIC_BYTES.get(key)
 
 
 def load_peaks():
@@ -510,7 +522,7 @@ def run_ours(args):
         achieved_tf = flops / (k_ms * 1e-3) / 1e12
         peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
         roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                    "frac": achieved_tf / peak_tf, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                    "frac": achieved_tf / peak_tf, "traffic": traffic_of(args, args.workload),
                     "kernel": "recon_tc_kernel" if ctx.decode_path() == 2 else "recon_simt_kernel",
                     "kernel_ms": k_ms, "kernel_launches": recon_n,
                     "share_of_step": recon_ms / ms_total,
@@ -525,7 +537,7 @@ def run_ours(args):
         achieved_gbs = full_bytes / (k_ms * 1e-3) / 1e9
         peak_gbs = float(peaks["hbm_gbs"])
         roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
-                    "frac": achieved_gbs / peak_gbs, "traffic": NCU_TRAFFIC_BYTES.get(args.workload + "_full"),
+                    "frac": achieved_gbs / peak_gbs, "traffic": traffic_of(args, args.workload + "_full"),
                     "kernel": stored_info["kernel"] if stored_info else None,
                     "kernel_ms": k_ms, "kernel_launches": stored_n, "share_of_step": stored_ms / ms_total,
                     "peak_source": "%s (STREAM-style copy)" % peaks_kind,
