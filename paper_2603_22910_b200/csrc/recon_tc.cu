@@ -44,6 +44,7 @@ constexpr int kStageBytes = kXBytes + kWBytes;       // 64 KiB
 constexpr int kThreads = 320;
 constexpr int kEpilogueThreads = 256;
 constexpr int kMaxBatchPerLaunch = 256;
+constexpr int kRunTokens = 64;                       // token rows of a tall box over consecutive pages
 constexpr int kTmemCols = 512;
 
 struct TcParams {
@@ -60,6 +61,7 @@ struct TcParams {
   int b0, nb;                 // batch entries [b0, b0 + nb) are handled by this launch
   int n_q_heads, n_ret_heads, n_drop_heads, n_pairs;
   int kc_anchor, kc_total;    // 64-feature chunks of the predictor input: from the anchor, in all
+  int run_pages;              // pages per tall box (kRunTokens / page_tokens), 1 = no tall boxes
   float scale_log2e;
 };
 
@@ -133,6 +135,8 @@ template <int G>
 __global__ void __launch_bounds__(kThreads, 1)
 recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_constant__ CUtensorMap tm_anchor_v,
                 const __grid_constant__ CUtensorMap tm_local_k, const __grid_constant__ CUtensorMap tm_local_v,
+                const __grid_constant__ CUtensorMap tm_anchor_k_run, const __grid_constant__ CUtensorMap tm_anchor_v_run,
+                const __grid_constant__ CUtensorMap tm_local_k_run, const __grid_constant__ CUtensorMap tm_local_v_run,
                 const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
                 const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
@@ -216,9 +220,26 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
       }
       const uint32_t n_valid_boxes = __popc(__ballot_sync(0xffffffffu, page >= 0));
       const uint32_t tx_bytes = n_valid_boxes * page_bytes + kWBytes;
+      // Pages that follow one another in the pool are fetched together: when the run_pages pages of
+      // an aligned group (kRunTokens token rows) are consecutive, the group's first lane issues one
+      // tall box for all of them -- far fewer TMA operations than one per 16-token page.
+      bool run_lead = false, run_member = false;
+      if (p.run_pages > 1) {
+        bool consecutive = page >= 0;
+        for (int k = 1; k < p.run_pages; ++k) {
+          const int pk = __shfl_down_sync(0xffffffffu, page, k);
+          consecutive = consecutive && pk == page + k;
+        }
+        const int lead = lane - lane % p.run_pages;
+        const bool group_run = __shfl_sync(0xffffffffu, consecutive ? 1 : 0, lead) != 0;
+        run_lead = group_run && lane == lead && lane < boxes;
+        run_member = group_run && lane != lead && lane < boxes;
+      }
       for (int phase = 0; phase < 2 && alive; ++phase) {
         const CUtensorMap* m_anchor = phase == 0 ? &tm_anchor_k : &tm_anchor_v;
         const CUtensorMap* m_local = phase == 0 ? &tm_local_k : &tm_local_v;
+        const CUtensorMap* m_anchor_run = phase == 0 ? &tm_anchor_k_run : &tm_anchor_v_run;
+        const CUtensorMap* m_local_run = phase == 0 ? &tm_local_k_run : &tm_local_v_run;
         const CUtensorMap* m_w = phase == 0 ? &tm_wk : &tm_wv;
         for (int kc = 0; kc < p.kc_total; ++kc, ++it) {
           const uint32_t s = it % kStages;
@@ -231,10 +252,12 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
           if (lane == 0) mbar_arrive_expect_tx(full, tx_bytes);
           __syncwarp();
           const uint32_t x_dst = stage_base + s * kStageBytes;
-          if (page >= 0) {
+          if (page >= 0 && !run_member) {
             const bool from_anchor = kc < p.kc_anchor;
-            tma_load_2d(x_dst + lane * page_bytes, from_anchor ? m_anchor : m_local,
-                        (from_anchor ? kc : kc - p.kc_anchor) * kChunk, page * p.page_tokens, full);
+            const CUtensorMap* m = run_lead ? (from_anchor ? m_anchor_run : m_local_run)
+                                            : (from_anchor ? m_anchor : m_local);
+            tma_load_2d(x_dst + lane * page_bytes, m, (from_anchor ? kc : kc - p.kc_anchor) * kChunk,
+                        page * p.page_tokens, full);
           }
           if (lane == 16) tma_load_2d(x_dst + kXBytes, m_w, kc * kChunk, w.pair * kWRows, full);
           issued[s] = it + 1;
@@ -481,12 +504,13 @@ cudaError_t encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_
 
 template <int G>
 cudaError_t launch_g(const CUtensorMap& ak, const CUtensorMap& av, const CUtensorMap& lk, const CUtensorMap& lv,
+                     const CUtensorMap& akr, const CUtensorMap& avr, const CUtensorMap& lkr, const CUtensorMap& lvr,
                      const CUtensorMap& wk, const CUtensorMap& wv, const TcParams& p, int grid,
                      cudaStream_t stream) {
   const size_t smem = tc_smem_bytes<G>();
   cudaError_t e = cudaFuncSetAttribute(recon_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  recon_tc_kernel<G><<<grid, kThreads, smem, stream>>>(ak, av, lk, lv, wk, wv, p);
+  recon_tc_kernel<G><<<grid, kThreads, smem, stream>>>(ak, av, lk, lv, akr, avr, lkr, lvr, wk, wv, p);
   return cudaGetLastError();
 }
 
@@ -507,6 +531,12 @@ cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const voi
   cudaError_t e = encode_2d(&maps->k_pool, k_pool, rows, width, page_tokens, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (e != cudaSuccess) return e;
   e = encode_2d(&maps->v_pool, v_pool, rows, width, page_tokens, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+  if (e != cudaSuccess) return e;
+  // tall boxes over runs of consecutive pages (the same maps again when a page is already that tall)
+  const int run_rows = page_tokens < kRunTokens ? kRunTokens : page_tokens;
+  e = encode_2d(&maps->k_pool_run, k_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+  if (e != cudaSuccess) return e;
+  e = encode_2d(&maps->v_pool_run, v_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (e != cudaSuccess) return e;
   maps->pools_ready = true;
   return cudaSuccess;
@@ -546,9 +576,12 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
   p.kc_anchor = r.D / kChunk;
   p.kc_total = (r.D + r.m) / kChunk;
   p.scale_log2e = a.scale_log2e;
+  p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;
   const CUtensorMap& lv = r.m > 0 ? layer.v_pool : anchor.v_pool;
+  const CUtensorMap& lkr = r.m > 0 ? layer.k_pool_run : anchor.k_pool_run;
+  const CUtensorMap& lvr = r.m > 0 ? layer.v_pool_run : anchor.v_pool_run;
   const int tiles_cap = (r.capacity_tokens + kTileTokens - 1) / kTileTokens;
   for (int b0 = 0; b0 < a.batch; b0 += kMaxBatchPerLaunch) {
     p.b0 = b0;
@@ -557,10 +590,14 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
     const int grid = (int)(max_items < sm_count ? max_items : sm_count);
     cudaError_t e;
     switch (g) {
-      case 1: e = launch_g<1>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
-      case 2: e = launch_g<2>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
-      case 4: e = launch_g<4>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
-      case 8: e = launch_g<8>(anchor.k_pool, anchor.v_pool, lk, lv, layer.wk, layer.wv, p, grid, stream); break;
+      case 1: e = launch_g<1>(anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run, anchor.v_pool_run, lkr, lvr,
+                                layer.wk, layer.wv, p, grid, stream); break;
+      case 2: e = launch_g<2>(anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run, anchor.v_pool_run, lkr, lvr,
+                                layer.wk, layer.wv, p, grid, stream); break;
+      case 4: e = launch_g<4>(anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run, anchor.v_pool_run, lkr, lvr,
+                                layer.wk, layer.wv, p, grid, stream); break;
+      case 8: e = launch_g<8>(anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run, anchor.v_pool_run, lkr, lvr,
+                                layer.wk, layer.wv, p, grid, stream); break;
       default: return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;

@@ -11,6 +11,7 @@ namespace echokv {
 // compressed layer, its two predictors (boxes of 256 rows x 64 input features).
 struct TcLayerMaps {
   CUtensorMap k_pool, v_pool, wk, wv;
+  CUtensorMap k_pool_run, v_pool_run;   // the pools again, in boxes of 64 token rows (runs of consecutive pages)
   bool pools_ready = false;
   bool weights_ready = false;
 };
