@@ -426,6 +426,8 @@ def run_ours(args):
     ctx, dev = st.ctx, st.dev
     if args.stored_path is not None:
         ctx.set_stored_path(args.stored_path)
+    if args.decode_path is not None and not full:
+        ctx.set_decode_path(args.decode_path)
     last = [l for l, a in step_layers if a][-1]
 
     def attend(l):
@@ -523,7 +525,7 @@ def run_ours(args):
         peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
         roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                     "frac": achieved_tf / peak_tf, "traffic": traffic_of(args, args.workload),
-                    "kernel": "recon_tc_kernel" if ctx.decode_path() == 2 else "recon_simt_kernel",
+                    "kernel": {3: "recon_pair_kernel", 2: "recon_tc_kernel"}.get(ctx.decode_path(), "recon_simt_kernel"),
                     "kernel_ms": k_ms, "kernel_launches": recon_n,
                     "share_of_step": recon_ms / ms_total,
                     "peak_source": "%s (bf16 sustained; kernel timed inside a long step)" % peaks_kind,
@@ -593,6 +595,8 @@ def main():
                          "uncompressed path, full-cache attention on the anchor layer")
     ap.add_argument("--stored-path", type=int, default=None, choices=[0, 1],
                     help="kernel for stored heads: 0 CUDA-core, 1 TMA + tensor-core (default: the library's choice)")
+    ap.add_argument("--decode-path", type=int, default=None, choices=[1, 2, 3],
+                    help="kernel family for compressed layers (default: the library's choice)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")

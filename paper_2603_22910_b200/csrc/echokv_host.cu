@@ -43,7 +43,7 @@ int derive(const echokv_config* c, Derived* d) {
   d->d_in = d->D + d->m;
   d->d_drop = d->D - d->m;
   d->elem = c->dtype == ECHOKV_BF16 ? 2 : 4;
-  d->part_tokens = (c->dtype == ECHOKV_BF16 && c->head_dim == 128) ? kTcPartTokens : kSimtTileTokens;
+  d->part_tokens = (c->dtype == ECHOKV_BF16 && c->head_dim == 128) ? kPairPartTokens : kSimtTileTokens;
   d->capacity = (int)cap;
   d->max_parts = (d->capacity + d->part_tokens - 1) / d->part_tokens;
   uint64_t off = 0;
@@ -271,7 +271,7 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
   if (cudaMemset(c->ws + d.off_status, 0, kAlign) != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
   c->tc_capable = tc_shape_supported(cfg->dtype, cfg->head_dim, cfg->page_tokens, d.D, d.m);
   if (!any_compressed || d.d_drop == 0) c->path = 0;
-  else c->path = c->tc_capable ? 2 : 1;
+  else c->path = c->tc_capable ? 3 : 1;
   if (c->tc_capable) {
     // tensor maps of every pool (the predictors' maps follow in echokv_set_weights)
     for (int l = 0; l < cfg->n_layers; ++l) {
@@ -330,9 +330,9 @@ int echokv_set_decode_path(echokv_ctx* c, int path) {
   if (!c) return ECHOKV_EINVAL;
   if (c->path == 0) return path == 0 ? ECHOKV_OK : ECHOKV_EINVAL;
   if (path == 1) { c->path = 1; return ECHOKV_OK; }
-  if (path == 2) {
+  if (path == 2 || path == 3) {
     if (!c->tc_capable) return ECHOKV_EUNSUPPORTED;
-    c->path = 2;
+    c->path = path;
     return ECHOKV_OK;
   }
   return ECHOKV_EINVAL;
@@ -403,14 +403,17 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   cudaError_t e;
   {
     ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
-    if (c->path == 2) {
+    if (c->path == 3) {
+      e = launch_recon_pair(a, ra, A.tc, L.tc, c->sm_count, s);
+    } else if (c->path == 2) {
       e = launch_recon_tc(a, ra, A.tc, L.tc, c->sm_count, s);
     } else {
       e = launch_recon_simt(a, ra, s);
     }
   }
   if (e != cudaSuccess) return ECHOKV_ECUDA;
-  if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, c->d.part_tokens, L.bv, s) !=
+  const int recon_part_tokens = c->path == 2 ? kTcPartTokens : c->d.part_tokens;
+  if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, recon_part_tokens, L.bv, s) !=
       cudaSuccess)
     return ECHOKV_ECUDA;
   c->launches += 2;

@@ -12,6 +12,7 @@ namespace echokv {
 struct TcLayerMaps {
   CUtensorMap k_pool, v_pool, wk, wv;
   CUtensorMap k_pool_run, v_pool_run;   // the pools again, in boxes of 64 token rows (runs of consecutive pages)
+  CUtensorMap wk_half, wv_half;         // the predictors in boxes of 128 rows (one head): CTA-pair kernel
   bool pools_ready = false;
   bool weights_ready = false;
 };
@@ -30,5 +31,11 @@ cudaError_t tc_encode_weight_maps(TcLayerMaps* maps, const void* Wk, const void*
 // Dropped heads of one compressed layer: Eq. 3 on the tensor cores, Eq. 7 on the accumulators.
 cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
                             const TcLayerMaps& layer, int sm_count, cudaStream_t stream);
+
+// The same on pairs of CTAs (cta_group::2, M = 256): one split-K partial per kPairPartTokens tokens.
+cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                              const TcLayerMaps& layer, int sm_count, cudaStream_t stream);
+
+constexpr int kPairPartTokens = 128;
 
 }  // namespace echokv

@@ -51,17 +51,21 @@ SMALL = [
     ("one_dropped_head", synth.C2, dict(n_retained_heads=7, batch=2, context=300), [300, 258]),
     ("pages128", synth.C2, dict(batch=2, context=700, page_tokens=128, random_pages=True), [700, 129]),
     ("gqa8_bf16", synth.C2, dict(n_q_heads=32, n_kv_heads=4, n_retained_heads=1, batch=1, context=300), [300]),
+    ("many_tiles_ragged", synth.C2, dict(batch=5, context=2000, random_pages=True), [2000, 129, 128, 1153, 1]),
+    ("mha_three_dropped", synth.C1.replace(n_q_heads=4, n_kv_heads=4), dict(n_retained_heads=1, batch=2, context=600),
+     [600, 385]),
 ]
 
 
 @pytest.mark.parametrize("name,base,over,lens", SMALL, ids=[s[0] for s in SMALL])
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 2, 3])
 def test_small_shapes_against_oracle(name, base, over, lens, path):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1])
-    if path == 2 and case.ctx.decode_path() != 2:
+    if path >= 2 and case.ctx.decode_path() < 2:
         case.close()
         pytest.skip("shape is served by the CUDA-core kernel only")
+    assert case.ctx.decode_path() in (1, 3)    # a context starts on the fastest family its shape allows
     case.ctx.set_decode_path(path)
     check_layers(case, name)
     case.close()
