@@ -271,7 +271,14 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
   if (cudaMemset(c->ws + d.off_status, 0, kAlign) != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
   c->tc_capable = tc_shape_supported(cfg->dtype, cfg->head_dim, cfg->page_tokens, d.D, d.m);
   if (!any_compressed || d.d_drop == 0) c->path = 0;
-  else c->path = c->tc_capable ? 3 : 1;
+  else if (!c->tc_capable) c->path = 1;
+  else {
+    // Long contractions (many 64-feature chunks per phase, few query heads per KV head) hide the
+    // epilogue by themselves and run best one CTA per SM; short ones need the CTA-pair kernel's
+    // double-buffered accumulators.
+    const int chunks = d.d_in / 64;
+    c->path = chunks <= 12 * d.g ? 3 : 2;
+  }
   if (c->tc_capable) {
     // tensor maps of every pool (the predictors' maps follow in echokv_set_weights)
     for (int l = 0; l < cfg->n_layers; ++l) {

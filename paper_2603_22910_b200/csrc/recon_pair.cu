@@ -5,9 +5,11 @@
 //
 //   work item  = (sequence b, tile of 256 tokens, pair of dropped heads), one per CTA pair;
 //                CTA r of the pair owns tokens [128 r, 128 r + 128) of the tile and head r of the pair
-//   stage      = per CTA 128 token rows and the 128 predictor rows of its head, kStageChunks x 64
-//                features of each; every MMA reads the token rows of both CTAs and the predictor
-//                rows of both CTAs, so each operand byte is fetched into shared memory once per pair
+//   stage      = per CTA 128 token rows and the 128 predictor rows of its head, two 64-feature chunks
+//                of each (64 KiB, 3 deep); every MMA reads the token rows of both CTAs and the predictor
+//                rows of both CTAs, so each operand byte is fetched into shared memory once per pair.
+//                When the CTA's 128 tokens lie consecutively in the pool a stage is two TMA copies
+//                (tokens, predictor); otherwise 64-row runs or single pages are copied chunk by chunk
 //   K phase    : acc0[tok, feat] (M = tokens: 128 per CTA, N = 256 features of both heads)
 //                -> a thread owns (token, head): scores of the head's G query heads, tile max / exp2 /
 //                   sum over the CTA's 128 tokens; the probabilities go to the CTA that owns the
@@ -39,8 +41,8 @@ constexpr int kStages = 3;
 constexpr int kXBytes = kCtaTokens * kRowBytes;      // 16 KiB: token rows of one chunk
 constexpr int kWRows = 128;                          // predictor rows per CTA: one head
 constexpr int kWBytes = kWRows * kRowBytes;          // 16 KiB: predictor rows of one chunk
-constexpr int kChunkBytes = kXBytes + kWBytes;       // 32 KiB
-constexpr int kStageBytes = kStageChunks * kChunkBytes;
+constexpr int kStageXBytes = kStageChunks * kXBytes;  // token rows: chunk 0, chunk 1
+constexpr int kStageBytes = kStageChunks * (kXBytes + kWBytes);   // then predictor rows: chunk 0, chunk 1
 constexpr int kThreads = 320;
 constexpr int kEpilogueThreads = 256;
 constexpr int kMaxBatchPerLaunch = 256;
@@ -136,6 +138,8 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
                   const __grid_constant__ CUtensorMap tm_local_k, const __grid_constant__ CUtensorMap tm_local_v,
                   const __grid_constant__ CUtensorMap tm_anchor_k_run, const __grid_constant__ CUtensorMap tm_anchor_v_run,
                   const __grid_constant__ CUtensorMap tm_local_k_run, const __grid_constant__ CUtensorMap tm_local_v_run,
+                  const __grid_constant__ CUtensorMap tm_anchor_k_128, const __grid_constant__ CUtensorMap tm_anchor_v_128,
+                  const __grid_constant__ CUtensorMap tm_local_k_128, const __grid_constant__ CUtensorMap tm_local_v_128,
                   const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
                   const PairParams p) {
   extern __shared__ unsigned char smem_raw[];
@@ -198,7 +202,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
   const int boxes = kCtaTokens / p.page_tokens;             // TMA boxes (pages) of this CTA's tokens
   const uint32_t page_bytes = p.page_tokens * kRowBytes;
   const uint32_t peer_abort = mapa_u32(smem_u32(&t.abort_flag), rank ^ 1u);
-  const int n_steps = (p.kc_total + kStageChunks - 1) / kStageChunks;   // stages per phase
+  const int n_steps = p.kc_total / kStageChunks;            // stages per phase (kc_total is even)
   bool gave_up = false;
 
   if (warp == 0) {
@@ -223,7 +227,10 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
         }
       }
       const uint32_t n_valid_boxes = __popc(__ballot_sync(0xffffffffu, page >= 0));
-      const uint32_t chunk_tx = n_valid_boxes * page_bytes + kWBytes;
+      const uint32_t stage_tx = kStageChunks * (n_valid_boxes * page_bytes + kWBytes);
+      // all of this CTA's 128 tokens cached and consecutive in the pool: one copy per stage
+      const int page0 = __shfl_sync(0xffffffffu, page, 0);
+      const bool run128 = __all_sync(0xffffffffu, lane >= boxes || (page >= 0 && page == page0 + lane));
       // runs of consecutive pages are fetched as one tall box
       bool run_lead = false, run_member = false;
       if (p.run_pages > 1) {
@@ -242,6 +249,8 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
         const CUtensorMap* m_local = phase == 0 ? &tm_local_k : &tm_local_v;
         const CUtensorMap* m_anchor_run = phase == 0 ? &tm_anchor_k_run : &tm_anchor_v_run;
         const CUtensorMap* m_local_run = phase == 0 ? &tm_local_k_run : &tm_local_v_run;
+        const CUtensorMap* m_anchor_128 = phase == 0 ? &tm_anchor_k_128 : &tm_anchor_v_128;
+        const CUtensorMap* m_local_128 = phase == 0 ? &tm_local_k_128 : &tm_local_v_128;
         const CUtensorMap* m_w = phase == 0 ? &tm_wk : &tm_wv;
         for (int step = 0; step < n_steps; ++step, ++it) {
           const uint32_t s = it % kStages;
@@ -252,23 +261,25 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
           if (lane == 0) ok = mbar_wait(smem_u32(&t.empty_bar[s]), ph ^ 1u, abort_flag, p.status);
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
           if (!ok) { alive = false; break; }
-          const int kc0 = step * kStageChunks;
-          const int n_chunks = min(kStageChunks, p.kc_total - kc0);
-          if (lane == 0) mbar_arrive_expect_tx_cluster(full, chunk_tx * n_chunks);
+          const int kc0 = step * kStageChunks;              // both chunks come from the same pool (D / 64 is even)
+          const bool from_anchor = kc0 < p.kc_anchor;
+          const int kx0 = from_anchor ? kc0 : kc0 - p.kc_anchor;   // chunk index inside that pool's rows
+          if (lane == 0) mbar_arrive_expect_tx_cluster(full, stage_tx);
           __syncwarp();
-          for (int j = 0; j < n_chunks; ++j) {
-            const int kc = kc0 + j;
-            const uint32_t x_dst = stage_base + s * kStageBytes + j * kChunkBytes;
-            if (page >= 0 && !run_member) {
-              const bool from_anchor = kc < p.kc_anchor;
-              const CUtensorMap* m = run_lead ? (from_anchor ? m_anchor_run : m_local_run)
-                                              : (from_anchor ? m_anchor : m_local);
-              tma_load_2d_pair(x_dst + lane * page_bytes, m, (from_anchor ? kc : kc - p.kc_anchor) * kChunk,
-                               page * p.page_tokens, full);
-            }
-            if (lane == 16)
-              tma_load_2d_pair(x_dst + kXBytes, m_w, kc * kChunk, w.pair * 2 * kWRows + (int)rank * kWRows, full);
+          const uint32_t x_dst = stage_base + s * kStageBytes;
+          if (run128) {
+            if (lane == 0)
+              tma_load_3d_pair(x_dst, from_anchor ? m_anchor_128 : m_local_128, 0, page * p.page_tokens, kx0, full);
+          } else if (page >= 0 && !run_member) {
+            const CUtensorMap* m = run_lead ? (from_anchor ? m_anchor_run : m_local_run)
+                                            : (from_anchor ? m_anchor : m_local);
+#pragma unroll
+            for (int j = 0; j < kStageChunks; ++j)
+              tma_load_2d_pair(x_dst + j * kXBytes + lane * page_bytes, m, (kx0 + j) * kChunk, page * p.page_tokens,
+                               full);
           }
+          if (lane == 16)
+            tma_load_3d_pair(x_dst + kStageXBytes, m_w, 0, w.pair * 2 * kWRows + (int)rank * kWRows, kc0, full);
         }
       }
     }
@@ -292,10 +303,10 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
             const uint32_t ph = (it / kStages) & 1u;
             if (!mbar_wait(smem_u32(&t.full_bar[s]), ph, abort_flag, p.status)) { alive = false; break; }
             tc_fence_after();
-            const int n_chunks = min(kStageChunks, p.kc_total - step * kStageChunks);
-            for (int j = 0; j < n_chunks; ++j) {
-              const uint32_t x_addr = stage_base + s * kStageBytes + j * kChunkBytes;
-              const uint32_t w_addr = x_addr + kXBytes;
+#pragma unroll
+            for (int j = 0; j < kStageChunks; ++j) {
+              const uint32_t x_addr = stage_base + s * kStageBytes + j * kXBytes;
+              const uint32_t w_addr = stage_base + s * kStageBytes + kStageXBytes + j * kWBytes;
               // K phase: A = token rows (128 per CTA), B = predictor rows (128 per CTA: 256 features).
               // V phase: A = predictor rows (head r on CTA r), B = token rows (128 per CTA: 256 tokens).
               const uint64_t a_desc = umma_desc(phase == 0 ? x_addr : w_addr);
@@ -491,8 +502,8 @@ constexpr size_t pair_smem_bytes() {
 
 template <int G>
 cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUtensorMap& lv, const CUtensorMap& lkr,
-                     const CUtensorMap& lvr, const TcLayerMaps& layer, const PairParams& p, int n_clusters,
-                     cudaStream_t stream) {
+                     const CUtensorMap& lvr, const CUtensorMap& lk8, const CUtensorMap& lv8, const TcLayerMaps& layer,
+                     const PairParams& p, int n_clusters, cudaStream_t stream) {
   const size_t smem = pair_smem_bytes<G>();
   cudaError_t e = cudaFuncSetAttribute(recon_pair_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
@@ -519,7 +530,8 @@ cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUt
   if (n_clusters > resident_pairs) n_clusters = resident_pairs;
   cfg.gridDim = dim3(2 * n_clusters, 1, 1);
   return cudaLaunchKernelEx(&cfg, recon_pair_kernel<G>, anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run,
-                            anchor.v_pool_run, lkr, lvr, layer.wk_half, layer.wv_half, p);
+                            anchor.v_pool_run, lkr, lvr, anchor.k_pool_run128, anchor.v_pool_run128, lk8, lv8,
+                            layer.wk_half, layer.wv_half, p);
 }
 
 }  // namespace
@@ -555,6 +567,9 @@ cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLay
   const CUtensorMap& lv = r.m > 0 ? layer.v_pool : anchor.v_pool;
   const CUtensorMap& lkr = r.m > 0 ? layer.k_pool_run : anchor.k_pool_run;
   const CUtensorMap& lvr = r.m > 0 ? layer.v_pool_run : anchor.v_pool_run;
+  const CUtensorMap& lk8 = r.m > 0 ? layer.k_pool_run128 : anchor.k_pool_run128;
+  const CUtensorMap& lv8 = r.m > 0 ? layer.v_pool_run128 : anchor.v_pool_run128;
+  if (p.kc_total % kStageChunks != 0 || p.kc_anchor % kStageChunks != 0) return cudaErrorInvalidValue;
   const int tiles_cap = (r.capacity_tokens + kTileTokens - 1) / kTileTokens;
   for (int b0 = 0; b0 < a.batch; b0 += kMaxBatchPerLaunch) {
     p.b0 = b0;
@@ -563,10 +578,10 @@ cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLay
     const int n_clusters = (int)(max_items < sm_count / 2 ? max_items : sm_count / 2);
     cudaError_t e;
     switch (g) {
-      case 1: e = launch_g<1>(anchor, lk, lv, lkr, lvr, layer, p, n_clusters, stream); break;
-      case 2: e = launch_g<2>(anchor, lk, lv, lkr, lvr, layer, p, n_clusters, stream); break;
-      case 4: e = launch_g<4>(anchor, lk, lv, lkr, lvr, layer, p, n_clusters, stream); break;
-      case 8: e = launch_g<8>(anchor, lk, lv, lkr, lvr, layer, p, n_clusters, stream); break;
+      case 1: e = launch_g<1>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream); break;
+      case 2: e = launch_g<2>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream); break;
+      case 4: e = launch_g<4>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream); break;
+      case 8: e = launch_g<8>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream); break;
       default: return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;

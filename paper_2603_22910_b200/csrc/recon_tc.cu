@@ -522,6 +522,22 @@ bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m) 
   return D % kChunk == 0 && m % kChunk == 0 && D > m;
 }
 
+// The same matrix seen as [cols / 64][rows][64]: a box of box_chunks x box_rows x 64 lands in shared memory
+// as box_chunks consecutive swizzled sub-tiles of box_rows rows, one per 64-column chunk.
+cudaError_t encode_3d_chunks(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                             uint32_t box_chunks, CUtensorMapL2promotion promo) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return cudaErrorNotSupported;
+  cuuint64_t dims[3] = {kChunk, rows, cols / kChunk};
+  cuuint64_t strides[2] = {cols * 2, kChunk * 2};
+  cuuint32_t box[3] = {kChunk, box_rows, box_chunks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows) {
   return encode_2d(map, pool, rows, width, box_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
@@ -538,6 +554,11 @@ cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const voi
   if (e != cudaSuccess) return e;
   e = encode_2d(&maps->v_pool_run, v_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (e != cudaSuccess) return e;
+  // CTA-pair kernel: 128 consecutive token rows x two 64-feature chunks in one copy
+  e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+  if (e != cudaSuccess) return e;
+  e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+  if (e != cudaSuccess) return e;
   maps->pools_ready = true;
   return cudaSuccess;
 }
@@ -547,9 +568,9 @@ cudaError_t tc_encode_weight_maps(TcLayerMaps* maps, const void* Wk, const void*
   if (e != cudaSuccess) return e;
   e = encode_2d(&maps->wv, Wv, d_drop, d_in, kWRows, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
   if (e != cudaSuccess) return e;
-  e = encode_2d(&maps->wk_half, Wk, d_drop, d_in, kWRows / 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+  e = encode_3d_chunks(&maps->wk_half, Wk, d_drop, d_in, kWRows / 2, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
   if (e != cudaSuccess) return e;
-  e = encode_2d(&maps->wv_half, Wv, d_drop, d_in, kWRows / 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+  e = encode_3d_chunks(&maps->wv_half, Wv, d_drop, d_in, kWRows / 2, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
   if (e != cudaSuccess) return e;
   maps->weights_ready = true;
   return cudaSuccess;

@@ -12,7 +12,10 @@ namespace echokv {
 struct TcLayerMaps {
   CUtensorMap k_pool, v_pool, wk, wv;
   CUtensorMap k_pool_run, v_pool_run;   // the pools again, in boxes of 64 token rows (runs of consecutive pages)
-  CUtensorMap wk_half, wv_half;         // the predictors in boxes of 128 rows (one head): CTA-pair kernel
+  // CTA-pair kernel: three-dimensional views [64-column chunk][row][64] whose boxes hold two chunks of
+  // 128 rows each: of the pools (128 consecutive token rows) and of the predictors (one head)
+  CUtensorMap k_pool_run128, v_pool_run128;
+  CUtensorMap wk_half, wv_half;
   bool pools_ready = false;
   bool weights_ready = false;
 };
