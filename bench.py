@@ -40,7 +40,7 @@ UNIT = "tokens/s"
 # the ncu captures summarised under profiles/; None until a capture of that workload exists.
 NCU_TRAFFIC_BYTES = {
     "c1": 4 * 619.0e6,        # recon_tc_kernel: B = 2 capture x 4 (tokens)
-    "c2": 8 * 346.8e6,        # recon_tc_kernel: B = 2 capture x 8
+    "c2": 8 * 347.9e6,        # recon_pair_kernel: B = 2 capture x 8
     "c1_full": 4 * 275.0e6,   # attn_stored_mma_kernel: B = 2 capture x 4
     "c2_full": 8 * 273.8e6,   # attn_stored_mma_kernel: B = 2 capture x 8
 }

@@ -446,18 +446,22 @@ cudaError_t launch_recon_simt(const AttnArgs& a, const ReconArgs& r, cudaStream_
 // ---------------------------------------------------------------------------------------------
 // Split-K merge: log-sum-exp combination of partial (max, sum, weighted V) triples
 // ---------------------------------------------------------------------------------------------
+constexpr int kMergeGroups = 4;   // partials are dealt round-robin to this many thread groups
+
 template <typename T>
-__global__ void merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads,
-                             int n_stored_parts, const int32_t* __restrict__ stored_item_tokens,
-                             int stored_batch_per_slot, int part_tokens, const T* __restrict__ bv) {
-  const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
-  const int DH = a.head_dim;
+__global__ void __launch_bounds__(128 * kMergeGroups)
+merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stored_parts,
+             const int32_t* __restrict__ stored_item_tokens, int stored_batch_per_slot, int part_tokens,
+             const T* __restrict__ bv) {
+  const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x, grp = threadIdx.y;
+  const int DH = a.head_dim;                      // == blockDim.x
+  const int tid = grp * DH + j, n_threads = DH * kMergeGroups;
   const size_t oidx = ((size_t)b * a.n_q_heads + h) * DH + j;
   const int slot = a.slots ? a.slots[b] : b;
   const int len = a.lens[b];
   if (slot < 0 || slot >= a.geom.max_batch || len < 1 ||
-      len > a.geom.max_pages_per_seq * a.geom.page_tokens) {
-    out[oidx] = 0.f;
+      len > a.geom.max_pages_per_seq * a.geom.page_tokens) {      // (the same for the whole block)
+    if (grp == 0) out[oidx] = 0.f;
     return;
   }
   const int g = a.n_q_heads / a.n_kv_heads;
@@ -473,16 +477,36 @@ __global__ void merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_h
     n = n_stored_parts;
   }
   const size_t base = ((size_t)b * a.n_q_heads + h) * a.parts.max_parts;
+  __shared__ float s_max[16];
+  __shared__ float s_l[kMergeGroups];
+  __shared__ float s_acc[kMergeGroups][128];
+  // pass 1: the largest partial maximum, all threads of the block together
+  float m = -INFINITY;
+  for (int p = tid; p < n; p += n_threads) m = fmaxf(m, a.parts.ml[base + p].x);
+  m = warp_max(m);
+  if ((tid & 31) == 0) s_max[tid >> 5] = m;
+  __syncthreads();
   float M = -INFINITY;
-  for (int p = 0; p < n; ++p) M = fmaxf(M, a.parts.ml[base + p].x);
+  for (int w = 0; w < n_threads / 32; ++w) M = fmaxf(M, s_max[w]);
+  // pass 2: each group sums every kMergeGroups-th partial
   float L = 0.f, acc = 0.f;
   if (M > -INFINITY) {
-    for (int p = 0; p < n; ++p) {
+#pragma unroll 4
+    for (int p = grp; p < n; p += kMergeGroups) {
       const float2 ml = a.parts.ml[base + p];
       const float w = exp2f(ml.x - M);
       L = fmaf(w, ml.y, L);
       acc = fmaf(w, a.parts.o[(base + p) * DH + j], acc);
     }
+  }
+  s_acc[grp][j] = acc;
+  if (j == 0) s_l[grp] = L;
+  __syncthreads();
+  if (grp != 0) return;
+#pragma unroll
+  for (int k = 1; k < kMergeGroups; ++k) {
+    acc += s_acc[k][j];
+    L += s_l[k];
   }
   float res = L > 0.f ? acc / L : 0.f;
   // a bias on the V predictor shifts every predicted V row alike, so (sum_t p_t = 1) it adds
@@ -497,11 +521,11 @@ cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int 
                          const void* bv, cudaStream_t stream) {
   dim3 grid(a.n_q_heads, a.batch);
   if (a.dtype == ECHOKV_BF16) {
-    merge_kernel<__nv_bfloat16><<<grid, a.head_dim, 0, stream>>>(
+    merge_kernel<__nv_bfloat16><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(
         a, out, n_stored_heads, n_stored_parts, stored_item_tokens, stored_batch_per_slot, part_tokens,
         (const __nv_bfloat16*)bv);
   } else {
-    merge_kernel<float><<<grid, a.head_dim, 0, stream>>>(a, out, n_stored_heads, n_stored_parts,
+    merge_kernel<float><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(a, out, n_stored_heads, n_stored_parts,
                                                          stored_item_tokens, stored_batch_per_slot,
                                                          part_tokens, (const float*)bv);
   }
