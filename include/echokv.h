@@ -176,6 +176,32 @@ int echokv_decode_path(const echokv_ctx* ctx);
  * the fastest family their shape allows.  Meant for tests that check all against the oracle. */
 int echokv_set_decode_path(echokv_ctx* ctx, int path);
 
+/* Absorbed-predictor decode mode.  Eq. 3 is linear, so Eq. 7 over a predicted head can be evaluated
+ * without forming the predicted K and V:
+ *     q . (Wk x_t) = (Wk^T q) . x_t          sum_t p_t (Wv x_t) = Wv (sum_t p_t x_t)
+ * with x_t = [anchor dims ; retained dims] of token t.  The library then streams the K features once
+ * (scores of all query heads against "absorbed queries" Wk^T q), the V features once (probability-
+ * weighted sums of x_t) and applies Wv at the end: the same function of the same inputs as
+ * echokv_decode_attention's default (explicit) mode up to rounding, at about D_drop / (2 n_q_heads)
+ * times fewer FLOPs, bound by HBM bandwidth instead of the tensor cores.  The paper does not describe
+ * this evaluation order; it follows from the linearity of its predictor (Section 3.2, Eq. 3).
+ *
+ *  - echokv_absorbed_workspace_bytes: size of the extra device workspace the mode needs (scores and
+ *    probabilities of every cached token and head, absorbed queries, partial sums).
+ *    EUNSUPPORTED unless dtype is bf16, head_dim 128, n_q_heads in {16, 32, 64}, at least one head is
+ *    dropped and max_batch <= 256.
+ *  - echokv_enable_absorbed: hands the library that workspace (device pointer, 256-byte aligned,
+ *    borrowed until echokv_destroy) and switches the context to the absorbed mode.
+ *    Errors: EINVAL, EUNSUPPORTED, ECAPACITY (workspace too small), ECUDA.
+ *  - echokv_set_decode_mode: 0 = explicit reconstruction, 1 = absorbed (EUNSUPPORTED before
+ *    echokv_enable_absorbed).  Anchor layers and echokv_full_attention are not affected.
+ *  In this mode a page id outside the pool is still reported (EBADPAGE) but the output of that
+ *  sequence is unspecified. */
+int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out);
+int echokv_enable_absorbed(echokv_ctx* ctx, void* workspace, uint64_t workspace_bytes);
+int echokv_decode_mode(const echokv_ctx* ctx);
+int echokv_set_decode_mode(echokv_ctx* ctx, int mode);
+
 /* Which kernel serves attention over stored heads (anchor layers, retained heads, the
  * uncompressed mode): 0 = CUDA-core kernel (any supported shape), 1 = TMA + tensor-core kernel
  * (bf16, head_dim 128).  Contexts start on 1 when their shape allows it.
@@ -194,8 +220,14 @@ int echokv_read_kernel_timing(echokv_ctx* ctx, double* total_ms, int64_t* n_laun
 
 /* The same reading split by kernel: total_ms and n_launches are host arrays of
  * ECHOKV_TIMED_KINDS entries, indexed by ECHOKV_TIMED_STORED (stored-head attention of an
- * anchor / uncompressed layer) and ECHOKV_TIMED_RECON (fused reconstruct-attend kernel). */
-enum { ECHOKV_TIMED_STORED = 0, ECHOKV_TIMED_RECON = 1, ECHOKV_TIMED_KINDS = 2 };
+ * anchor / uncompressed layer), ECHOKV_TIMED_RECON (fused reconstruct-attend kernel) and the two
+ * streaming kernels of the absorbed mode. */
+enum {
+  ECHOKV_TIMED_STORED = 0, ECHOKV_TIMED_RECON = 1,
+  ECHOKV_TIMED_ABSORB_K = 2,   /* absorbed mode: the pass over the K features (scores)          */
+  ECHOKV_TIMED_ABSORB_V = 3,   /* absorbed mode: the pass over the V features (weighted sums)   */
+  ECHOKV_TIMED_KINDS = 4
+};
 int echokv_read_kernel_timing_by_kind(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
 
 /* Full-cache attention for callers that cannot allocate device memory (the paper has no

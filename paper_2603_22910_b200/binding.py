@@ -59,6 +59,10 @@ EXPORTS = {
     "echokv_launch_count": (C.c_int64, [C.c_void_p]),
     "echokv_decode_path": (C.c_int, [C.c_void_p]),
     "echokv_set_decode_path": (C.c_int, [C.c_void_p, C.c_int]),
+    "echokv_absorbed_workspace_bytes": (C.c_int, [C.POINTER(echokv_config), C.POINTER(C.c_uint64)]),
+    "echokv_enable_absorbed": (C.c_int, [C.c_void_p, C.c_void_p, C.c_uint64]),
+    "echokv_decode_mode": (C.c_int, [C.c_void_p]),
+    "echokv_set_decode_mode": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_stored_path": (C.c_int, [C.c_void_p]),
     "echokv_set_stored_path": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int]),
@@ -230,6 +234,20 @@ class Context:
     def set_decode_path(self, path: int) -> None:
         _check(lib().echokv_set_decode_path(self.handle, path), "echokv_set_decode_path")
 
+    def enable_absorbed(self) -> None:
+        """Allocate the absorbed mode's workspace and switch the context to that mode."""
+        n = C.c_uint64(0)
+        _check(lib().echokv_absorbed_workspace_bytes(C.byref(self.cfg), C.byref(n)), "echokv_absorbed_workspace_bytes")
+        self.workspace_absorbed = self.torch.empty(n.value, dtype=self.torch.uint8, device=self.device)
+        _check(lib().echokv_enable_absorbed(self.handle, self.workspace_absorbed.data_ptr(), n.value),
+               "echokv_enable_absorbed")
+
+    def decode_mode(self) -> int:
+        return lib().echokv_decode_mode(self.handle)
+
+    def set_decode_mode(self, mode: int) -> None:
+        _check(lib().echokv_set_decode_mode(self.handle, mode), "echokv_set_decode_mode")
+
     def stored_path(self) -> int:
         return lib().echokv_stored_path(self.handle)
 
@@ -247,9 +265,9 @@ class Context:
 
     def read_kernel_timing_by_kind(self):
         """{"stored": (ms, launches), "recon": (ms, launches)} since the last read."""
-        ms, n = (C.c_double * 2)(), (C.c_int64 * 2)()
+        ms, n = (C.c_double * 4)(), (C.c_int64 * 4)()
         _check(lib().echokv_read_kernel_timing_by_kind(self.handle, ms, n), "echokv_read_kernel_timing_by_kind")
-        return {"stored": (ms[0], n[0]), "recon": (ms[1], n[1])}
+        return {"stored": (ms[0], n[0]), "recon": (ms[1], n[1]), "absorb_k": (ms[2], n[2]), "absorb_v": (ms[3], n[3])}
 
     def _out(self, q):
         return self.torch.empty(q.shape, dtype=self.torch.float32, device=self.device)

@@ -1,0 +1,895 @@
+// Absorbed-predictor decode of a compressed layer (bf16, head_dim 128).
+//
+// Eq. 3 is linear, so Eq. 7 over predicted heads needs neither K_hat nor V_hat:
+//     q . (W_k x_t)           = (W_k^T q) . x_t            "absorbed query"  q~ = W_k^T q
+//     sum_t p_t (W_v x_t)     = W_v (sum_t p_t x_t)         project after the weighted sum
+// with x_t = [anchor dims ; retained dims] of token t (D_in values).  A retained head fits the
+// same form with a q~ that selects its own dims, so all H_q query heads attend over the same
+// per-token vectors and the layer becomes two streams over the cache plus small projections:
+//
+//   1. absorb_query_kernel   q~[b][h][:] for every head, scaled, split into two bf16 halves
+//   2. absorb_scores_kernel  S[b][h][t] = q~ . x^K_t        tcgen05: M = 128 tokens, N = 2 H_q, K = D_in
+//   3. absorb_softmax_kernel (max, sum) per head; p = 2^(S - max) split into two bf16 halves
+//   4. absorb_pv_kernel      y[b][h][:] = sum_t p_t x^V_t   tcgen05: M = 128 features (the V tile
+//                            is the M-major A operand), N = 2 H_q, K = tokens; split over token
+//                            ranges and 256-feature slices
+//   5. absorb_out_kernel     out = W_v y / sum (+ b_v) for predicted heads, y's own dims / sum for
+//                            retained heads
+//
+// The same result as the explicit path (Eq. 3, 6, 7) up to rounding, at 4 D_in bytes and
+// 8 H_q D_in FLOP per token instead of 4 D_in D_drop FLOP: the two tcgen05 kernels are HBM-bound.
+// Every wait is bounded.
+#include "absorbed.h"
+
+#include <cudaTypedefs.h>
+
+#include "ptx_sm100.cuh"
+
+namespace echokv {
+
+namespace {
+
+constexpr int kChunk = 64;
+constexpr int kRowBytes = 128;
+constexpr int kMaxStages = 6;
+constexpr int kThreads = 256;            // warp 0 TMA, 1 MMA, 2 helper, 3 idle, 4..7 epilogue
+constexpr int kMaxBatchPerLaunch = 256;
+constexpr int kRunTokens = 64;
+constexpr int kSmemBudget = 200 * 1024;
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ bool epi_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(ok ? 1u : 0u)
+      : "memory");
+  return r != 0;
+}
+
+// K-major bf16 operand: 128-byte rows in the 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// M-major bf16 operand made of [K rows][64 M-elements] tiles in the 128-byte swizzle (what a TMA box
+// of token rows x 64 features is when tokens are the contraction index): 8-row groups along K are
+// 1024 bytes apart, successive 64-element blocks along M are `block_bytes` apart
+__device__ __forceinline__ uint64_t desc_mmajor(uint32_t smem_addr, uint32_t block_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
+  d |= static_cast<uint64_t>(block_bytes >> 4) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// kind::f16, bf16 x bf16 -> fp32, M = 128; a_mmajor: the A operand is M-major (B always K-major)
+inline uint32_t make_idesc(int n, bool a_mmajor) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (a_mmajor ? (1u << 15) : 0u) | ((uint32_t)(n >> 3) << 17) |
+         ((128u >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------------
+// 1. absorbed queries
+// ---------------------------------------------------------------------------------------------
+constexpr int kQGroup = 8;   // (sequence, query head of the group) pairs per block
+
+__global__ void __launch_bounds__(256)
+absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ Wk,
+                    __nv_bfloat16* __restrict__ q2, int B, int n_q_heads, int g, int n_ret, int D, int d_in,
+                    float scale_log2e) {
+  __shared__ float qs[kQGroup][128];
+  const int i = blockIdx.x * 256 + threadIdx.x;     // input feature (column of W_k)
+  const int kv = blockIdx.y;
+  const int first = blockIdx.z * kQGroup;
+  const int n_pairs = B * g;
+  for (int idx = threadIdx.x; idx < kQGroup * 128; idx += 256) {
+    const int k = idx >> 7, j = idx & 127;
+    const int pr = first + k;
+    float v = 0.f;
+    if (pr < n_pairs) {
+      const int b = pr / g, gi = pr - b * g;
+      v = __bfloat162float(q[((size_t)b * n_q_heads + kv * g + gi) * 128 + j]) * scale_log2e;
+    }
+    qs[k][j] = v;
+  }
+  __syncthreads();
+  if (i >= d_in) return;
+  float acc[kQGroup];
+#pragma unroll
+  for (int k = 0; k < kQGroup; ++k) acc[k] = 0.f;
+  if (kv < n_ret) {
+    // a retained head reads its own stored dims: q~ is q placed at the head's local dims
+    const int j = i - (D + kv * 128);
+    if (j >= 0 && j < 128) {
+#pragma unroll
+      for (int k = 0; k < kQGroup; ++k) acc[k] = qs[k][j];
+    }
+  } else {
+    const __nv_bfloat16* w = Wk + (size_t)(kv - n_ret) * 128 * d_in + i;
+#pragma unroll 4
+    for (int j = 0; j < 128; ++j) {
+      const float wv = __bfloat162float(w[(size_t)j * d_in]);
+#pragma unroll
+      for (int k = 0; k < kQGroup; ++k) acc[k] = fmaf(wv, qs[k][j], acc[k]);
+    }
+  }
+  const int nh2 = 2 * n_q_heads;
+#pragma unroll
+  for (int k = 0; k < kQGroup; ++k) {
+    const int pr = first + k;
+    if (pr >= n_pairs) break;
+    const int b = pr / g, gi = pr - b * g;
+    const int h = kv * g + gi;
+    const __nv_bfloat16 hi = __float2bfloat16_rn(acc[k]);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(acc[k] - __bfloat162float(hi));
+    q2[((size_t)b * nh2 + h) * d_in + i] = hi;
+    q2[((size_t)b * nh2 + n_q_heads + h) * d_in + i] = lo;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// shared pieces of the two tcgen05 kernels
+// ---------------------------------------------------------------------------------------------
+struct StreamParams {
+  const int32_t* slots;
+  const int32_t* lens;
+  const int32_t* table;
+  int max_batch, max_pages_per_seq, page_tokens;
+  long long n_pages;
+  int32_t* status;
+  int b0, nb;
+  int n_q_heads, nh2;
+  int kc_anchor, kc_total;      // 64-feature chunks: from the anchor pool, in all
+  int run_pages;                // pages per 64-row run box, 1 = none
+  int l_cap;
+  int n_stages;
+  uint32_t stage_bytes;
+  uint32_t idesc;
+  float* s_out;                 // scores kernel: S
+  float* y_out;                 // pv kernel: partial y
+  int d_in;
+  int range_tokens;             // pv kernel: tokens per range
+  int n_slices;                 // pv kernel: 256-feature slices
+  int v_tile_ok;                // pv kernel: the 4-chunk V maps exist for (anchor, local)
+};
+
+struct StreamSmemTail {
+  int cum[kMaxBatchPerLaunch + 1];
+  unsigned long long full_bar[kMaxStages];
+  unsigned long long empty_bar[kMaxStages];
+  unsigned long long clean_bar[kMaxStages];
+  unsigned long long acc_full_bar[2];
+  unsigned long long acc_empty_bar[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ int find_seq(const StreamSmemTail& t, int unit, int nb) {
+  int lo = 0, hi = nb;   // largest b with cum[b] <= unit
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (t.cum[mid] <= unit) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// Per-sequence unit counts -> exclusive prefix sums in t.cum; barriers; tensor memory.
+template <typename CountFn>
+__device__ __forceinline__ void stream_setup(StreamSmemTail& t, const StreamParams& p, uint32_t tmem_cols,
+                                             CountFn count) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  for (int i = tid; i < p.nb; i += kThreads) {
+    const int b = p.b0 + i;
+    const int slot = p.slots ? p.slots[b] : b;
+    const int len = p.lens[b];
+    int n = 0;
+    if (slot < 0 || slot >= p.max_batch) {
+      if (blockIdx.x == 0) report(p.status, ECHOKV_EBADPAGE);
+    } else if (len < 1 || len > p.max_pages_per_seq * p.page_tokens) {
+      if (blockIdx.x == 0) report(p.status, ECHOKV_EBADLENGTH);
+    } else {
+      n = count(len);
+    }
+    t.cum[i + 1] = n;
+  }
+  if (tid == 0) {
+    t.cum[0] = 0;
+    t.abort_flag = 0;
+    for (int s = 0; s < kMaxStages; ++s) {
+      mbar_init(smem_u32(&t.full_bar[s]), 1);
+      mbar_init(smem_u32(&t.empty_bar[s]), 1);
+      mbar_init(smem_u32(&t.clean_bar[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&t.acc_full_bar[i]), 1);
+      mbar_init(smem_u32(&t.acc_empty_bar[i]), 1);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int i = 0; i < p.nb; ++i) {
+      acc += t.cum[i + 1];
+      t.cum[i + 1] = acc;
+    }
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&t.tmem_base), tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+}
+
+// Pages of `n_boxes` consecutive page-sized boxes starting at token t0 of the sequence in block-table
+// row `slot` (lane i holds box i; -1 = no cached token there or a bad page id), whether they form one
+// consecutive run, and for 64-row sub-runs which lane leads / follows.
+struct PageSet {
+  int page;
+  bool all_run;        // every box valid and consecutive in the pool
+  bool run_lead, run_member;
+  uint32_t n_valid;
+};
+__device__ __forceinline__ PageSet lookup_pages(const StreamParams& p, int slot, int len, int t0, int n_boxes,
+                                                int lane) {
+  PageSet r;
+  r.page = -1;
+  if (lane < n_boxes) {
+    const int tb = t0 + lane * p.page_tokens;
+    if (tb < len) {
+      const int pg = p.table[(size_t)slot * p.max_pages_per_seq + tb / p.page_tokens];
+      if (pg < 0 || pg >= p.n_pages) report(p.status, ECHOKV_EBADPAGE);
+      else r.page = pg;
+    }
+  }
+  r.n_valid = __popc(__ballot_sync(0xffffffffu, r.page >= 0));
+  const int page0 = __shfl_sync(0xffffffffu, r.page, 0);
+  r.all_run = __all_sync(0xffffffffu, lane >= n_boxes || (r.page >= 0 && r.page == page0 + lane));
+  r.run_lead = r.run_member = false;
+  if (p.run_pages > 1) {
+    bool consecutive = r.page >= 0;
+    for (int k = 1; k < p.run_pages; ++k) {
+      const int pk = __shfl_down_sync(0xffffffffu, r.page, k);
+      consecutive = consecutive && pk == r.page + k;
+    }
+    const int lead = lane - lane % p.run_pages;
+    const bool group_run = __shfl_sync(0xffffffffu, consecutive ? 1 : 0, lead) != 0;
+    r.run_lead = group_run && lane == lead && lane < n_boxes;
+    r.run_member = group_run && lane != lead && lane < n_boxes;
+  }
+  return r;
+}
+
+// ---------------------------------------------------------------------------------------------
+// 2. scores: S[b][h][t] = q~[b][h] . x^K_t
+// ---------------------------------------------------------------------------------------------
+constexpr int kScoreTokens = 128;                    // tokens per work item
+constexpr int kScoreXBytes = kScoreTokens * kRowBytes;   // one chunk of the token rows
+
+__global__ void __launch_bounds__(kThreads, 1)
+absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_constant__ CUtensorMap tm_local,
+                     const __grid_constant__ CUtensorMap tm_anchor_run, const __grid_constant__ CUtensorMap tm_local_run,
+                     const __grid_constant__ CUtensorMap tm_anchor_128, const __grid_constant__ CUtensorMap tm_local_128,
+                     const __grid_constant__ CUtensorMap tm_q2, const StreamParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  StreamSmemTail& t = *reinterpret_cast<StreamSmemTail*>(smem + (size_t)p.n_stages * p.stage_bytes);
+  const uint32_t stage_base = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  volatile int* abort_flag = &t.abort_flag;
+  stream_setup(t, p, 256u, [](int len) { return (len + kScoreTokens - 1) / kScoreTokens; });
+  const uint32_t tmem = t.tmem_base;
+  const int n_items = t.cum[p.nb];
+  const int n_steps = p.kc_total / 2;                     // stages per item: two chunks each
+  const int boxes = kScoreTokens / p.page_tokens;
+  const uint32_t page_bytes = p.page_tokens * kRowBytes;
+  const uint32_t q_chunk_bytes = (uint32_t)p.nh2 * kRowBytes;
+
+  if (warp == 0) {
+    // =============================== TMA producer ===============================================
+    uint32_t it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const int bi = find_seq(t, item, p.nb);
+      const int b = p.b0 + bi;
+      const int tile = item - t.cum[bi];
+      const int slot = p.slots ? p.slots[b] : b;
+      const int len = p.lens[b];
+      const PageSet ps = lookup_pages(p, slot, len, tile * kScoreTokens, boxes, lane);
+      const uint32_t stage_tx = 2u * (ps.n_valid * page_bytes + q_chunk_bytes);
+      for (int step = 0; step < n_steps; ++step, ++it) {
+        const uint32_t s = it % p.n_stages;
+        const uint32_t ph = (it / p.n_stages) & 1u;
+        const uint32_t full = smem_u32(&t.full_bar[s]);
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(smem_u32(&t.empty_bar[s]), ph ^ 1u, abort_flag, p.status);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) { alive = false; break; }
+        const int kc0 = step * 2;                           // both chunks come from the same pool
+        const bool from_anchor = kc0 < p.kc_anchor;
+        const int kx0 = from_anchor ? kc0 : kc0 - p.kc_anchor;
+        if (lane == 0) mbar_arrive_expect_tx(full, stage_tx);
+        __syncwarp();
+        const uint32_t x_dst = stage_base + s * p.stage_bytes;
+        if (ps.all_run) {
+          if (lane == 0)
+            tma_load_3d(x_dst, from_anchor ? &tm_anchor_128 : &tm_local_128, 0, ps.page * p.page_tokens, kx0, full);
+        } else if (ps.page >= 0 && !ps.run_member) {
+          const CUtensorMap* m = ps.run_lead ? (from_anchor ? &tm_anchor_run : &tm_local_run)
+                                             : (from_anchor ? &tm_anchor : &tm_local);
+#pragma unroll
+          for (int j = 0; j < 2; ++j)
+            tma_load_2d(x_dst + j * kScoreXBytes + lane * page_bytes, m, (kx0 + j) * kChunk,
+                        ps.page * p.page_tokens, full);
+        }
+        if (lane == 16) tma_load_3d(x_dst + 2 * kScoreXBytes, &tm_q2, 0, b * p.nh2, kc0, full);
+      }
+    }
+  } else if (warp == 1) {
+    // =============================== MMA issuer ================================================
+    if (lane == 0) {
+      uint32_t it = 0, n = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++n) {
+        const uint32_t buf = n & 1u;
+        if (!mbar_wait(smem_u32(&t.acc_empty_bar[buf]), ((n >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem + buf * 128u;
+        for (int step = 0; step < n_steps; ++step, ++it) {
+          const uint32_t s = it % p.n_stages;
+          const uint32_t ph = (it / p.n_stages) & 1u;
+          if (!mbar_wait(smem_u32(&t.full_bar[s]), ph, abort_flag, p.status)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t x_addr = stage_base + s * p.stage_bytes;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint64_t a_desc = desc_kmajor(x_addr + j * kScoreXBytes);
+            const uint64_t b_desc = desc_kmajor(x_addr + 2 * kScoreXBytes + j * q_chunk_bytes);
+#pragma unroll
+            for (int k16 = 0; k16 < 4; ++k16)
+              tc_mma_bf16(d_tmem, a_desc + 2 * k16, b_desc + 2 * k16, p.idesc, (step > 0 || j > 0 || k16 > 0) ? 1u : 0u);
+          }
+          tc_commit(smem_u32(&t.empty_bar[s]));
+        }
+        if (alive) tc_commit(smem_u32(&t.acc_full_bar[buf]));
+      }
+    }
+    __syncwarp();
+  } else if (warp >= 4) {
+    // =============================== epilogue (4 warps) ========================================
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;                 // TMEM lane = token of the tile
+    uint32_t n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const int bi = find_seq(t, item, p.nb);
+      const int b = p.b0 + bi;
+      const int tile = item - t.cum[bi];
+      const int len = p.lens[b];
+      const uint32_t buf = n & 1u;
+      if (!epi_all(mbar_wait(smem_u32(&t.acc_full_bar[buf]), (n >> 1) & 1u, abort_flag, p.status))) break;
+      tc_fence_after();
+      const int token = tile * kScoreTokens + row;
+      const bool valid = token < len;
+      const uint32_t addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 128u;
+      float* dst = p.s_out + (size_t)b * p.n_q_heads * p.l_cap + token;
+      for (int hb = 0; hb < p.n_q_heads; hb += 16) {
+        float hi[16], lo[16];
+        tmem_ld16(addr + hb, hi);
+        tmem_ld16(addr + p.n_q_heads + hb, lo);
+#pragma unroll
+        for (int k = 0; k < 16; ++k)
+          dst[(size_t)(hb + k) * p.l_cap] = valid ? hi[k] + lo[k] : -INFINITY;
+      }
+      tc_fence_before();
+      epi_sync();
+      if (tid == 128) mbar_arrive(smem_u32(&t.acc_empty_bar[buf]));
+    }
+  }
+
+  if (t.abort_flag) {     // a wait ran out: give copies and MMAs already started ample time to land
+    const long long start = clock64();
+    while (clock64() - start < 4000000ll) {
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 256u);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 3. softmax statistics and probabilities
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+absorb_softmax_kernel(const float* __restrict__ S, __nv_bfloat16* __restrict__ p2, float2* __restrict__ ml,
+                      const int32_t* __restrict__ slots, const int32_t* __restrict__ lens, int max_batch,
+                      int capacity, int n_q_heads, int l_cap) {
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int slot = slots ? slots[b] : b;
+  const int len = lens[b];
+  if (slot < 0 || slot >= max_batch || len < 1 || len > capacity) {
+    if (tid == 0) ml[(size_t)b * n_q_heads + h] = make_float2(-INFINITY, 0.f);
+    return;
+  }
+  __shared__ float red[8];
+  const float* s = S + ((size_t)b * n_q_heads + h) * l_cap;
+  const int n4 = (len + 3) / 4;                  // (entries past len hold -inf up to the next 128)
+  float m = -INFINITY;
+  for (int i = tid; i < n4; i += 256) {
+    const float4 v = reinterpret_cast<const float4*>(s)[i];
+    m = fmaxf(fmaxf(m, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+  }
+  m = warp_max(m);
+  if ((tid & 31) == 0) red[tid >> 5] = m;
+  __syncthreads();
+  float M = red[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) M = fmaxf(M, red[w]);
+  __syncthreads();
+  const int nh2 = 2 * n_q_heads;
+  __nv_bfloat16* hi = p2 + ((size_t)b * nh2 + h) * l_cap;
+  __nv_bfloat16* lo = p2 + ((size_t)b * nh2 + n_q_heads + h) * l_cap;
+  const int n4_pad = ((len + 63) / 64) * 16;     // the V pass reads whole 64-token blocks
+  float L = 0.f;
+  for (int i = tid; i < n4_pad; i += 256) {
+    const float4 v = reinterpret_cast<const float4*>(s)[i];
+    const float pv[4] = {exp2f(v.x - M), exp2f(v.y - M), exp2f(v.z - M), exp2f(v.w - M)};   // 2^(-inf) = 0
+    L += (pv[0] + pv[1]) + (pv[2] + pv[3]);
+    const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
+    const __nv_bfloat162 h23 = __floats2bfloat162_rn(pv[2], pv[3]);
+    const __nv_bfloat162 l01 = __floats2bfloat162_rn(pv[0] - __low2float(h01), pv[1] - __high2float(h01));
+    const __nv_bfloat162 l23 = __floats2bfloat162_rn(pv[2] - __low2float(h23), pv[3] - __high2float(h23));
+    uint2 uh, ul;
+    uh.x = *reinterpret_cast<const uint32_t*>(&h01); uh.y = *reinterpret_cast<const uint32_t*>(&h23);
+    ul.x = *reinterpret_cast<const uint32_t*>(&l01); ul.y = *reinterpret_cast<const uint32_t*>(&l23);
+    reinterpret_cast<uint2*>(hi)[i] = uh;
+    reinterpret_cast<uint2*>(lo)[i] = ul;
+  }
+  L = warp_sum(L);
+  if ((tid & 31) == 0) red[tid >> 5] = L;
+  __syncthreads();
+  if (tid == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    ml[(size_t)b * n_q_heads + h] = make_float2(M, tot);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 4. y[b][h][:] = sum_t p[b][h][t] x^V_t, per (sequence, token range, 256-feature slice)
+// ---------------------------------------------------------------------------------------------
+constexpr int kPvTokens = 64;                        // tokens per stage
+constexpr int kPvTileBytes = kPvTokens * kRowBytes;  // 64 token rows x 64 features
+constexpr int kPvVBytes = 4 * kPvTileBytes;          // four chunks
+
+__global__ void __launch_bounds__(kThreads, 1)
+absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_constant__ CUtensorMap tm_local,
+                 const __grid_constant__ CUtensorMap tm_anchor_run, const __grid_constant__ CUtensorMap tm_local_run,
+                 const __grid_constant__ CUtensorMap tm_anchor_4, const __grid_constant__ CUtensorMap tm_local_4,
+                 const __grid_constant__ CUtensorMap tm_p2, const StreamParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  StreamSmemTail& t = *reinterpret_cast<StreamSmemTail*>(smem + (size_t)p.n_stages * p.stage_bytes);
+  const uint32_t stage_base = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  volatile int* abort_flag = &t.abort_flag;
+  const int range_tokens = p.range_tokens, n_slices = p.n_slices;
+  stream_setup(t, p, 512u, [range_tokens, n_slices](int len) {
+    return ((len + range_tokens - 1) / range_tokens) * n_slices;
+  });
+  const uint32_t tmem = t.tmem_base;
+  const int n_items = t.cum[p.nb];
+  const int boxes = kPvTokens / p.page_tokens;              // page boxes per chunk and stage (>= 1)
+  const uint32_t page_bytes = p.page_tokens * kRowBytes;
+  const uint32_t p_tile_bytes = (uint32_t)p.nh2 * kRowBytes;
+
+  // item -> (sequence, range, slice); its token span and chunk span
+  struct Work { int b, slot, len, range, slice, t_begin, n_steps, kc0, n_chunks; bool from_anchor; };
+  auto decode = [&](int item) {
+    Work w;
+    const int bi = find_seq(t, item, p.nb);
+    w.b = p.b0 + bi;
+    const int local = item - t.cum[bi];
+    w.range = local / n_slices;
+    w.slice = local - w.range * n_slices;
+    w.slot = p.slots ? p.slots[w.b] : w.b;
+    w.len = p.lens[w.b];
+    w.t_begin = w.range * range_tokens;
+    const int t_end = min(w.len, w.t_begin + range_tokens);
+    w.n_steps = (t_end - w.t_begin + kPvTokens - 1) / kPvTokens;
+    w.kc0 = w.slice * 4;
+    w.n_chunks = min(4, p.kc_total - w.kc0);
+    w.from_anchor = w.kc0 < p.kc_anchor;   // (D / 64 is a multiple of 4 when the tiled maps are in use)
+    return w;
+  };
+
+  if (warp == 0) {
+    // =============================== TMA producer ===============================================
+    uint32_t it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const Work w = decode(item);
+      const bool one_pool = w.kc0 + w.n_chunks <= p.kc_anchor || w.kc0 >= p.kc_anchor;
+      for (int step = 0; step < w.n_steps; ++step, ++it) {
+        const uint32_t s = it % p.n_stages;
+        const uint32_t ph = (it / p.n_stages) & 1u;
+        const uint32_t full = smem_u32(&t.full_bar[s]);
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(smem_u32(&t.empty_bar[s]), ph ^ 1u, abort_flag, p.status);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) { alive = false; break; }
+        const int t0 = w.t_begin + step * kPvTokens;
+        const PageSet ps = lookup_pages(p, w.slot, w.len, t0, boxes, lane);
+        if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)w.n_chunks * ps.n_valid * page_bytes + p_tile_bytes);
+        __syncwarp();
+        const uint32_t v_dst = stage_base + s * p.stage_bytes;
+        if (ps.all_run && w.n_chunks == 4 && one_pool && p.v_tile_ok) {
+          if (lane == 0)
+            tma_load_3d(v_dst, w.from_anchor ? &tm_anchor_4 : &tm_local_4, 0, ps.page * p.page_tokens,
+                        w.from_anchor ? w.kc0 : w.kc0 - p.kc_anchor, full);
+        } else if (ps.page >= 0 && !ps.run_member) {
+          for (int c = 0; c < w.n_chunks; ++c) {
+            const int kc = w.kc0 + c;
+            const bool fa = kc < p.kc_anchor;
+            const CUtensorMap* m = ps.run_lead ? (fa ? &tm_anchor_run : &tm_local_run) : (fa ? &tm_anchor : &tm_local);
+            tma_load_2d(v_dst + c * kPvTileBytes + lane * page_bytes, m, (fa ? kc : kc - p.kc_anchor) * kChunk,
+                        ps.page * p.page_tokens, full);
+          }
+        }
+        if (lane == 16) tma_load_2d(v_dst + kPvVBytes, &tm_p2, t0, w.b * p.nh2, full);
+      }
+    }
+  } else if (warp == 1) {
+    // =============================== MMA issuer ================================================
+    if (lane == 0) {
+      uint32_t it = 0, n = 0;
+      uint32_t clean_uses[kMaxStages];
+#pragma unroll
+      for (int s = 0; s < kMaxStages; ++s) clean_uses[s] = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++n) {
+        const Work w = decode(item);
+        const uint32_t buf = n & 1u;
+        if (!mbar_wait(smem_u32(&t.acc_empty_bar[buf]), ((n >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
+        tc_fence_after();
+        const int n_mtiles = w.n_chunks / 2;
+        for (int step = 0; step < w.n_steps; ++step, ++it) {
+          const uint32_t s = it % p.n_stages;
+          const uint32_t ph = (it / p.n_stages) & 1u;
+          if (!mbar_wait(smem_u32(&t.full_bar[s]), ph, abort_flag, p.status)) { alive = false; break; }
+          if (w.t_begin + (step + 1) * kPvTokens > w.len) {
+            // a block with slots that hold no token: wait until the helper warp has zeroed them
+            if (!mbar_wait(smem_u32(&t.clean_bar[s]), clean_uses[s] & 1u, abort_flag, p.status)) { alive = false; break; }
+            ++clean_uses[s];
+          }
+          tc_fence_after();
+          const uint32_t v_addr = stage_base + s * p.stage_bytes;
+          const uint64_t b_desc = desc_kmajor(v_addr + kPvVBytes);
+          for (int mt = 0; mt < n_mtiles; ++mt) {
+            // A: 128 features (two 64-feature tiles, kPvTileBytes apart) x 16 tokens per MMA, M-major
+            const uint64_t a_desc = desc_mmajor(v_addr + mt * 2 * kPvTileBytes, kPvTileBytes);
+            const uint32_t d_tmem = tmem + buf * 256u + mt * (uint32_t)p.nh2;
+#pragma unroll
+            for (int k16 = 0; k16 < 4; ++k16)   // 16 tokens = 2048 bytes of A rows, 32 bytes along B's K
+              tc_mma_bf16(d_tmem, a_desc + 128 * k16, b_desc + 2 * k16, p.idesc, (step > 0 || k16 > 0) ? 1u : 0u);
+          }
+          tc_commit(smem_u32(&t.empty_bar[s]));
+        }
+        if (alive) tc_commit(smem_u32(&t.acc_full_bar[buf]));
+      }
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ============ helper: zero V rows of slots that hold no token (never written, or a skipped page) ====
+    uint32_t it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const Work w = decode(item);
+      for (int step = 0; step < w.n_steps; ++step, ++it) {
+        const uint32_t s = it % p.n_stages;
+        const uint32_t ph = (it / p.n_stages) & 1u;
+        const bool got = mbar_wait(smem_u32(&t.full_bar[s]), ph, abort_flag, p.status);
+        if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
+        const int n_tok = w.len - (w.t_begin + step * kPvTokens);
+        if (n_tok >= kPvTokens) continue;
+        const uint32_t v_addr = stage_base + s * p.stage_bytes;
+        const int n_rows = kPvTokens - n_tok;                 // rows n_tok .. 63 of every chunk tile
+        for (int idx = lane; idx < w.n_chunks * n_rows * 8; idx += 32) {
+          const int piece = idx & 7, rr = (idx >> 3) % n_rows, c = (idx >> 3) / n_rows;
+          const uint32_t a = v_addr + c * kPvTileBytes + (n_tok + rr) * kRowBytes + piece * 16;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&t.clean_bar[s]));
+      }
+    }
+  } else if (warp >= 4) {
+    // =============================== epilogue (4 warps) ========================================
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;                 // TMEM lane = feature of the 128-feature tile
+    uint32_t n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const Work w = decode(item);
+      const uint32_t buf = n & 1u;
+      if (!epi_all(mbar_wait(smem_u32(&t.acc_full_bar[buf]), (n >> 1) & 1u, abort_flag, p.status))) break;
+      tc_fence_after();
+      const int n_mtiles = w.n_chunks / 2;
+      for (int mt = 0; mt < n_mtiles; ++mt) {
+        const uint32_t addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256u + mt * (uint32_t)p.nh2;
+        const int feature = w.kc0 * kChunk + mt * 128 + row;
+        float* dst = p.y_out + (((size_t)w.b * kAbsorbMaxRanges + w.range) * p.n_q_heads) * p.d_in + feature;
+        for (int hb = 0; hb < p.n_q_heads; hb += 16) {
+          float hi[16], lo[16];
+          tmem_ld16(addr + hb, hi);
+          tmem_ld16(addr + p.n_q_heads + hb, lo);
+#pragma unroll
+          for (int k = 0; k < 16; ++k) dst[(size_t)(hb + k) * p.d_in] = hi[k] + lo[k];
+        }
+      }
+      tc_fence_before();
+      epi_sync();
+      if (tid == 128) mbar_arrive(smem_u32(&t.acc_empty_bar[buf]));
+    }
+  }
+
+  if (t.abort_flag) {
+    const long long start = clock64();
+    while (clock64() - start < 4000000ll) {
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512u);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 5. output projection
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+absorb_out_kernel(const float* __restrict__ y, const float2* __restrict__ ml, const __nv_bfloat16* __restrict__ Wv,
+                  const __nv_bfloat16* __restrict__ bv, float* __restrict__ out, const int32_t* __restrict__ slots,
+                  const int32_t* __restrict__ lens, int max_batch, int capacity, int n_q_heads, int g, int n_ret,
+                  int D, int d_in, int range_tokens) {
+  extern __shared__ float ys[];     // [g][d_in]: sum_t p_t x^V_t of the group's query heads
+  const int kv = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int slot = slots ? slots[b] : b;
+  const int len = lens[b];
+  float* o = out + ((size_t)b * n_q_heads + kv * g) * 128;
+  if (slot < 0 || slot >= max_batch || len < 1 || len > capacity) {
+    for (int idx = tid; idx < g * 128; idx += 256) o[idx] = 0.f;
+    return;
+  }
+  const int n_ranges = (len + range_tokens - 1) / range_tokens;
+  const float* yb = y + ((size_t)b * kAbsorbMaxRanges * n_q_heads + kv * g) * d_in;
+  const size_t range_stride = (size_t)n_q_heads * d_in;
+  if (kv < n_ret) {
+    // a retained head: its own stored dims of y
+    for (int idx = tid; idx < g * 128; idx += 256) {
+      const int gi = idx >> 7, j = idx & 127;
+      float acc = 0.f;
+      for (int r = 0; r < n_ranges; ++r) acc += yb[r * range_stride + (size_t)gi * d_in + D + kv * 128 + j];
+      const float L = ml[(size_t)b * n_q_heads + kv * g + gi].y;
+      o[idx] = L > 0.f ? acc / L : 0.f;
+    }
+    return;
+  }
+  for (int idx = tid; idx < g * d_in; idx += 256) {
+    float acc = 0.f;
+    for (int r = 0; r < n_ranges; ++r) acc += yb[r * range_stride + idx];
+    ys[idx] = acc;
+  }
+  __syncthreads();
+  const __nv_bfloat16* W = Wv + (size_t)(kv - n_ret) * 128 * d_in;
+  for (int j = warp; j < 128; j += 8) {
+    float acc[kMaxGroup];
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
+    const __nv_bfloat16* wrow = W + (size_t)j * d_in;
+    for (int i = lane * 8; i < d_in; i += 256) {
+      float wv[8];
+      Vec16<__nv_bfloat16>::load(wrow + i, wv);
+#pragma unroll
+      for (int gi = 0; gi < kMaxGroup; ++gi) {
+        if (gi < g) {
+          const float* yy = ys + (size_t)gi * d_in + i;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[gi] = fmaf(wv[e], yy[e], acc[gi]);
+        }
+      }
+    }
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi) {
+      if (gi < g) {
+        const float tot = warp_sum(acc[gi]);
+        if (lane == 0) {
+          const float L = ml[(size_t)b * n_q_heads + kv * g + gi].y;
+          float res = L > 0.f ? tot / L : 0.f;
+          if (bv != nullptr) res += __bfloat162float(bv[(kv - n_ret) * 128 + j]);
+          o[gi * 128 + j] = res;
+        }
+      }
+    }
+  }
+}
+
+int round_up(int v, int a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+bool absorbed_supported(int dtype, int head_dim, int n_q_heads, int n_kv_heads, int n_retained, int page_tokens) {
+  if (dtype != ECHOKV_BF16 || head_dim != 128) return false;
+  if (n_q_heads != 16 && n_q_heads != 32 && n_q_heads != 64) return false;   // 2 H_q accumulator columns
+  if (n_q_heads / n_kv_heads > kMaxGroup) return false;
+  if (n_retained >= n_kv_heads) return false;
+  return page_tokens == 16 || page_tokens == 32 || page_tokens == 64 || page_tokens == 128;
+}
+
+void absorbed_layout(int max_batch, int n_q_heads, int d_in, int capacity_tokens, AbsorbLayout* out) {
+  auto align = [](uint64_t v) { return (v + 255) / 256 * 256; };
+  out->nh2 = 2 * n_q_heads;
+  out->l_cap = round_up(capacity_tokens, kAbsorbTokAlign);
+  uint64_t off = 0;
+  out->off_q2 = off; off = align(off + (uint64_t)max_batch * out->nh2 * d_in * 2);
+  out->off_s = off; off = align(off + (uint64_t)max_batch * n_q_heads * out->l_cap * 4);
+  out->off_p2 = off; off = align(off + (uint64_t)max_batch * out->nh2 * out->l_cap * 2);
+  out->off_ml = off; off = align(off + (uint64_t)max_batch * n_q_heads * 8);
+  out->off_y = off; off = align(off + (uint64_t)max_batch * kAbsorbMaxRanges * n_q_heads * d_in * 4);
+  out->total = off;
+}
+
+cudaError_t absorbed_encode_maps(AbsorbMaps* maps, unsigned char* ws, const AbsorbLayout& lay, int max_batch, int d_in) {
+  cudaError_t e = encode_chunked_3d_map(&maps->q2, ws + lay.off_q2, (uint64_t)max_batch * lay.nh2, d_in, lay.nh2, 2);
+  if (e != cudaSuccess) return e;
+  e = encode_pool_box_map(&maps->p2, ws + lay.off_p2, lay.l_cap, (uint64_t)max_batch * lay.nh2, lay.nh2);
+  if (e != cudaSuccess) return e;
+  maps->ready = true;
+  return cudaSuccess;
+}
+
+cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const AbsorbMaps& maps, const TcLayerMaps& anchor,
+                            const TcLayerMaps& layer, float* out, int sm_count, cudaStream_t stream,
+                            cudaEvent_t* ev) {
+  if (!maps.ready || !anchor.pools_ready) return cudaErrorInvalidValue;
+  if (r.m > 0 && !layer.pools_ready) return cudaErrorInvalidValue;
+  if (a.batch > kMaxBatchPerLaunch) return cudaErrorInvalidValue;
+  const int g = a.n_q_heads / a.n_kv_heads;
+  const int d_in = r.D + r.m;
+  const int n_ret = r.m / 128;
+  const AbsorbLayout& lay = r.lay;
+  __nv_bfloat16* q2 = reinterpret_cast<__nv_bfloat16*>(r.ws + lay.off_q2);
+  float* S = reinterpret_cast<float*>(r.ws + lay.off_s);
+  __nv_bfloat16* p2 = reinterpret_cast<__nv_bfloat16*>(r.ws + lay.off_p2);
+  float2* ml = reinterpret_cast<float2*>(r.ws + lay.off_ml);
+  float* y = reinterpret_cast<float*>(r.ws + lay.off_y);
+  cudaError_t e;
+
+  // 1. absorbed queries
+  {
+    dim3 grid((d_in + 255) / 256, a.n_kv_heads, (a.batch * g + kQGroup - 1) / kQGroup);
+    absorb_query_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q),
+                                                  reinterpret_cast<const __nv_bfloat16*>(r.Wk), q2, a.batch,
+                                                  a.n_q_heads, g, n_ret, r.D, d_in, a.scale_log2e);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+
+  StreamParams p;
+  p.slots = a.slots;
+  p.lens = a.lens;
+  p.table = a.geom.table;
+  p.max_batch = a.geom.max_batch;
+  p.max_pages_per_seq = a.geom.max_pages_per_seq;
+  p.page_tokens = a.geom.page_tokens;
+  p.n_pages = a.geom.n_pages;
+  p.status = a.status;
+  p.b0 = 0;
+  p.nb = a.batch;
+  p.n_q_heads = a.n_q_heads;
+  p.nh2 = lay.nh2;
+  p.kc_anchor = r.D / kChunk;
+  p.kc_total = d_in / kChunk;
+  p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
+  p.l_cap = lay.l_cap;
+  p.s_out = S;
+  p.y_out = y;
+  p.d_in = d_in;
+  // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
+  const TcLayerMaps& loc = r.m > 0 ? layer : anchor;
+  const int capacity = r.capacity_tokens;
+
+  // 2. scores
+  {
+    p.stage_bytes = 2u * (kScoreXBytes + (uint32_t)lay.nh2 * kRowBytes);
+    p.n_stages = (int)(kSmemBudget / p.stage_bytes);
+    if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;
+    p.idesc = make_idesc(lay.nh2, false);
+    p.range_tokens = 0; p.n_slices = 0; p.v_tile_ok = 0;
+    const size_t smem = 1024 + (size_t)p.n_stages * p.stage_bytes + sizeof(StreamSmemTail);
+    if ((e = cudaFuncSetAttribute(absorb_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+        cudaSuccess)
+      return e;
+    const long long max_items = (long long)a.batch * ((capacity + kScoreTokens - 1) / kScoreTokens);
+    const int grid = (int)(max_items < sm_count ? max_items : sm_count);
+    if (ev) cudaEventRecord(ev[0], stream);
+    absorb_scores_kernel<<<grid, kThreads, smem, stream>>>(anchor.k_pool, loc.k_pool, anchor.k_pool_run, loc.k_pool_run,
+                                                           anchor.k_pool_run128, loc.k_pool_run128, maps.q2, p);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (ev) cudaEventRecord(ev[1], stream);
+  }
+
+  // 3. softmax statistics and probabilities
+  {
+    dim3 grid(a.n_q_heads, a.batch);
+    absorb_softmax_kernel<<<grid, 256, 0, stream>>>(S, p2, ml, a.slots, a.lens, a.geom.max_batch, capacity,
+                                                    a.n_q_heads, lay.l_cap);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+
+  // 4. probability-weighted inputs
+  int range_tokens;
+  {
+    p.n_slices = (p.kc_total + 3) / 4;
+    int ranges = (4 * sm_count + p.n_slices * a.batch - 1) / (p.n_slices * a.batch);
+    if (ranges > kAbsorbMaxRanges) ranges = kAbsorbMaxRanges;
+    if (ranges < 1) ranges = 1;
+    range_tokens = round_up((capacity + ranges - 1) / ranges, kPvTokens);
+    p.range_tokens = range_tokens;
+    p.stage_bytes = kPvVBytes + (uint32_t)lay.nh2 * kRowBytes;
+    p.n_stages = (int)(kSmemBudget / p.stage_bytes);
+    if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;
+    p.idesc = make_idesc(lay.nh2, true);
+    // the 4-chunk maps exist for pools whose width is a multiple of 256, and a slice must not straddle pools
+    p.v_tile_ok = (r.D % 256 == 0 && (r.m == 0 || r.m % 256 == 0)) ? 1 : 0;
+    const size_t smem = 1024 + (size_t)p.n_stages * p.stage_bytes + sizeof(StreamSmemTail);
+    if ((e = cudaFuncSetAttribute(absorb_pv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+        cudaSuccess)
+      return e;
+    const long long max_items = (long long)a.batch * ((capacity + range_tokens - 1) / range_tokens) * p.n_slices;
+    const int grid = (int)(max_items < sm_count ? max_items : sm_count);
+    const CUtensorMap& a4 = p.v_tile_ok ? anchor.v_pool_tok64x4 : anchor.v_pool_run;
+    const CUtensorMap& l4 = p.v_tile_ok && r.m > 0 ? loc.v_pool_tok64x4 : a4;
+    if (ev) cudaEventRecord(ev[2], stream);
+    absorb_pv_kernel<<<grid, kThreads, smem, stream>>>(anchor.v_pool, loc.v_pool, anchor.v_pool_run, loc.v_pool_run, a4,
+                                                       l4, maps.p2, p);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (ev) cudaEventRecord(ev[3], stream);
+  }
+
+  // 5. output projection
+  {
+    const size_t smem = (size_t)g * d_in * sizeof(float);
+    if ((e = cudaFuncSetAttribute(absorb_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+        cudaSuccess)
+      return e;
+    dim3 grid(a.n_kv_heads, a.batch);
+    absorb_out_kernel<<<grid, 256, smem, stream>>>(y, ml, reinterpret_cast<const __nv_bfloat16*>(r.Wv),
+                                                   reinterpret_cast<const __nv_bfloat16*>(r.bv), out, a.slots, a.lens,
+                                                   a.geom.max_batch, capacity, a.n_q_heads, g, n_ret, r.D, d_in,
+                                                   range_tokens);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace echokv

@@ -1,0 +1,55 @@
+// Absorbed-predictor decode: host interface.
+//
+// Eq. 3 is linear, so Eq. 7 over predicted heads can be evaluated without ever forming the
+// predicted K and V:  q . (W_k x_t) = (W_k^T q) . x_t   and   sum_t p_t (W_v x_t) = W_v (sum_t p_t x_t).
+// Every query head then attends over the same per-token vector x_t = [anchor dims ; retained dims]
+// (a retained head's "absorbed query" simply selects its own dims), which makes the layer one
+// stream over the K features, one stream over the V features and two small projections.
+#pragma once
+
+#include <cuda.h>
+
+#include "recon_tc.h"
+
+namespace echokv {
+
+constexpr int kAbsorbMaxRanges = 4;      // token ranges the V pass may split a sequence into
+constexpr int kAbsorbTokAlign = 128;     // score rows are padded to this many tokens
+
+struct AbsorbLayout {
+  int nh2;          // rows of the absorbed-query / probability matrices per sequence: 2 * n_q_heads (hi, lo)
+  int l_cap;        // tokens per score row
+  uint64_t off_q2;  // bf16 [max_batch * nh2][D_in]      absorbed queries, split into two bf16 halves
+  uint64_t off_s;   // fp32 [max_batch][n_q_heads][l_cap] scores (base-2 units)
+  uint64_t off_p2;  // bf16 [max_batch * nh2][l_cap]     probabilities, split into two bf16 halves
+  uint64_t off_ml;  // float2 [max_batch][n_q_heads]      (max, sum) of every head
+  uint64_t off_y;   // fp32 [max_batch][ranges][n_q_heads][D_in]  partial probability-weighted inputs
+  uint64_t total;
+};
+
+bool absorbed_supported(int dtype, int head_dim, int n_q_heads, int n_kv_heads, int n_retained, int page_tokens);
+void absorbed_layout(int max_batch, int n_q_heads, int d_in, int capacity_tokens, AbsorbLayout* out);
+
+struct AbsorbMaps {
+  CUtensorMap q2;   // [chunk][row][64] view of the absorbed queries, boxes of 2 chunks x nh2 rows
+  CUtensorMap p2;   // probabilities, boxes of nh2 rows x 64 tokens
+  bool ready = false;
+};
+
+cudaError_t absorbed_encode_maps(AbsorbMaps* maps, unsigned char* ws, const AbsorbLayout& lay, int max_batch, int d_in);
+
+struct AbsorbArgs {
+  unsigned char* ws;            // the absorbed-mode workspace
+  AbsorbLayout lay;
+  const void* Wk; const void* Wv; const void* bv;     // predictors of the layer ([D - m][D + m]), V bias or null
+  int D, m;
+  int capacity_tokens;
+  double* kernel_ms;            // unused
+};
+
+// One compressed layer, all query heads: out[B][H_q][d].
+cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const AbsorbMaps& maps, const TcLayerMaps& anchor,
+                            const TcLayerMaps& layer, float* out, int sm_count, cudaStream_t stream,
+                            cudaEvent_t* timing_events /* 4 events or null: around the K pass and the V pass */);
+
+}  // namespace echokv

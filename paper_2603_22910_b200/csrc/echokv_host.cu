@@ -9,6 +9,7 @@
 #include "kernels.h"
 #include "recon_tc.h"
 #include "stored_mma.h"
+#include "absorbed.h"
 
 using namespace echokv;
 
@@ -86,6 +87,11 @@ struct echokv_ctx {
   int sm_count = 0;
   int path = 0;          // see echokv_decode_path
   bool tc_capable = false;
+  bool absorbed_capable = false;  // shape served by the absorbed-predictor kernels
+  int decode_mode = 0;            // 0 = explicit reconstruction (Eq. 3, 6, 7 as written), 1 = absorbed predictors
+  unsigned char* ws_absorbed = nullptr;
+  AbsorbLayout alay;
+  AbsorbMaps amaps;
   bool stored_capable = false;   // shape served by the TMA + mma.sync stored-head kernel
   int stored_path = 0;           // 0 = CUDA-core kernel, 1 = TMA + mma.sync kernel
   int64_t launches = 0;
@@ -172,6 +178,23 @@ struct ScopedKernelTimer {
     if (stop) cudaEventRecord(stop, s);
   }
 };
+
+// An event pair of the given kind for a kernel the callee launches itself (null while timing is off).
+bool timed_pair(echokv_ctx* c, int kind, cudaEvent_t* start, cudaEvent_t* stop) {
+  if (!c->timing) return false;
+  if (c->timed == c->events.size()) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess) return false;
+    if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return false; }
+    c->events.emplace_back(a, b);
+    c->event_kind.push_back(kind);
+  }
+  c->event_kind[c->timed] = kind;
+  *start = c->events[c->timed].first;
+  *stop = c->events[c->timed].second;
+  ++c->timed;
+  return true;
+}
 
 int check_call(echokv_ctx* c, int layer, const void* q, const float* out, const int32_t* lens, int B) {
   if (!c || !q || !out || !lens) return ECHOKV_EINVAL;
@@ -345,6 +368,46 @@ int echokv_set_decode_path(echokv_ctx* c, int path) {
   return ECHOKV_EINVAL;
 }
 
+int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out) {
+  if (!out) return ECHOKV_EINVAL;
+  Derived d;
+  const int rc = derive(cfg, &d);
+  if (rc != ECHOKV_OK) return rc;
+  if (!absorbed_supported(cfg->dtype, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, cfg->n_retained_heads,
+                          cfg->page_tokens) || cfg->max_batch > 256)
+    return ECHOKV_EUNSUPPORTED;
+  AbsorbLayout lay;
+  absorbed_layout(cfg->max_batch, cfg->n_q_heads, d.d_in, d.capacity, &lay);
+  *out = lay.total;
+  return ECHOKV_OK;
+}
+
+int echokv_enable_absorbed(echokv_ctx* c, void* workspace, uint64_t workspace_bytes) {
+  if (!c || !workspace) return ECHOKV_EINVAL;
+  uint64_t need = 0;
+  const int rc = echokv_absorbed_workspace_bytes(&c->cfg, &need);
+  if (rc != ECHOKV_OK) return rc;
+  if (!c->tc_capable) return ECHOKV_EUNSUPPORTED;
+  if (workspace_bytes < need) return ECHOKV_ECAPACITY;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign != 0) return ECHOKV_EINVAL;
+  c->ws_absorbed = static_cast<unsigned char*>(workspace);
+  absorbed_layout(c->cfg.max_batch, c->cfg.n_q_heads, c->d.d_in, c->d.capacity, &c->alay);
+  if (absorbed_encode_maps(&c->amaps, c->ws_absorbed, c->alay, c->cfg.max_batch, c->d.d_in) != cudaSuccess)
+    return ECHOKV_ECUDA;
+  c->absorbed_capable = true;
+  c->decode_mode = 1;
+  return ECHOKV_OK;
+}
+
+int echokv_decode_mode(const echokv_ctx* c) { return c ? c->decode_mode : 0; }
+
+int echokv_set_decode_mode(echokv_ctx* c, int mode) {
+  if (!c || (mode != 0 && mode != 1)) return ECHOKV_EINVAL;
+  if (mode == 1 && !c->absorbed_capable) return ECHOKV_EUNSUPPORTED;
+  c->decode_mode = mode;
+  return ECHOKV_OK;
+}
+
 int echokv_stored_path(const echokv_ctx* c) { return c ? c->stored_path : 0; }
 
 int echokv_set_stored_path(echokv_ctx* c, int path) {
@@ -394,6 +457,24 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   if (!L.Wk || !L.Wv) return ECHOKV_ENOWEIGHTS;
   const Layer& A = c->layers[layer - layer % c->cfg.group_size];
   AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
+  if (c->decode_mode == 1) {
+    // absorbed predictors: every query head in one pass over [anchor dims ; retained dims]
+    if (B > 256) return ECHOKV_EUNSUPPORTED;
+    AbsorbArgs aa;
+    aa.ws = c->ws_absorbed;
+    aa.lay = c->alay;
+    aa.Wk = L.Wk; aa.Wv = L.Wv; aa.bv = L.bv;
+    aa.D = c->d.D; aa.m = c->d.m;
+    aa.capacity_tokens = c->d.capacity;
+    aa.kernel_ms = nullptr;
+    cudaEvent_t ev[4];
+    const bool timed = timed_pair(c, ECHOKV_TIMED_ABSORB_K, &ev[0], &ev[1]) &&
+                       timed_pair(c, ECHOKV_TIMED_ABSORB_V, &ev[2], &ev[3]);
+    if (launch_absorbed(a, aa, c->amaps, A.tc, L.tc, out, c->sm_count, s, timed ? ev : nullptr) != cudaSuccess)
+      return ECHOKV_ECUDA;
+    c->launches += 5;
+    return ECHOKV_OK;
+  }
   const int r = c->cfg.n_retained_heads;
   // retained heads: Eq. 7 on what is stored (Eq. 6 keeps them as they are)
   const int n_splits = stored_splits(c, B, r);

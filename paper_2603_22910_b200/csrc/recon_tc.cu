@@ -538,6 +538,11 @@ cudaError_t encode_3d_chunks(CUtensorMap* map, const void* base, uint64_t rows, 
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+cudaError_t encode_chunked_3d_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int box_rows,
+                                  int box_chunks) {
+  return encode_3d_chunks(map, base, rows, cols, box_rows, box_chunks, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+}
+
 cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows) {
   return encode_2d(map, pool, rows, width, box_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
@@ -559,6 +564,11 @@ cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const voi
   if (e != cudaSuccess) return e;
   e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (e != cudaSuccess) return e;
+  // absorbed mode, V side: 64 consecutive token rows x four 64-feature chunks in one copy
+  if (width % 256 == 0) {
+    e = encode_3d_chunks(&maps->v_pool_tok64x4, v_pool, rows, width, 64, 4, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    if (e != cudaSuccess) return e;
+  }
   maps->pools_ready = true;
   return cudaSuccess;
 }

@@ -16,12 +16,18 @@ struct TcLayerMaps {
   // 128 rows each: of the pools (128 consecutive token rows) and of the predictors (one head)
   CUtensorMap k_pool_run128, v_pool_run128;
   CUtensorMap wk_half, wv_half;
+  CUtensorMap v_pool_tok64x4;           // [chunk][row][64] view of the V pool, boxes of 4 chunks x 64 rows
   bool pools_ready = false;
   bool weights_ready = false;
 };
 
 // TMA descriptor of a bf16 pool [rows][width]: boxes of box_rows token rows x 64 features, 128-byte swizzle.
 cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows);
+
+// The matrix [rows][cols] seen as [cols / 64][rows][64]: boxes of box_chunks x box_rows x 64 land in shared
+// memory as box_chunks consecutive swizzled sub-tiles of box_rows rows.
+cudaError_t encode_chunked_3d_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int box_rows,
+                                  int box_chunks);
 
 bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m);
 
