@@ -13,8 +13,8 @@
 //   4. absorb_pv_kernel      y[b][h][:] = sum_t p_t x^V_t   tcgen05: M = 128 features (the V tile
 //                            is the M-major A operand), N = 2 H_q, K = tokens; split over token
 //                            ranges and 256-feature slices
-//   5. absorb_out_kernel     out = W_v y / sum (+ b_v) for predicted heads, y's own dims / sum for
-//                            retained heads
+//   5. absorb_ysum_kernel    y summed over the ranges and divided by the softmax sum;
+//      absorb_out_kernel     out = W_v y (+ b_v) for predicted heads, y's own dims for retained heads
 //
 // The same result as the explicit path (Eq. 3, 6, 7) up to rounding, at 4 D_in bytes and
 // 8 H_q D_in FLOP per token instead of 4 D_in D_drop FLOP: the two tcgen05 kernels are HBM-bound.
@@ -117,7 +117,7 @@ absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     }
   } else {
     const __nv_bfloat16* w = Wk + (size_t)(kv - n_ret) * 128 * d_in + i;
-#pragma unroll 4
+#pragma unroll 16
     for (int j = 0; j < 128; ++j) {
       const float wv = __bfloat162float(w[(size_t)j * d_in]);
 #pragma unroll
@@ -243,17 +243,19 @@ struct PageSet {
   bool run_lead, run_member;
   uint32_t n_valid;
 };
-__device__ __forceinline__ PageSet lookup_pages(const StreamParams& p, int slot, int len, int t0, int n_boxes,
-                                                int lane) {
+// Block-table entry of box `lane` (only the load: callers issue it a stage ahead of its use)
+__device__ __forceinline__ int load_page(const StreamParams& p, int slot, int len, int t0, int n_boxes, int lane) {
+  const int tb = t0 + lane * p.page_tokens;
+  if (lane < n_boxes && tb < len) return p.table[(size_t)slot * p.max_pages_per_seq + tb / p.page_tokens];
+  return -1;
+}
+__device__ __forceinline__ PageSet make_page_set(const StreamParams& p, int raw_page, int len, int t0, int n_boxes,
+                                                 int lane) {
   PageSet r;
   r.page = -1;
-  if (lane < n_boxes) {
-    const int tb = t0 + lane * p.page_tokens;
-    if (tb < len) {
-      const int pg = p.table[(size_t)slot * p.max_pages_per_seq + tb / p.page_tokens];
-      if (pg < 0 || pg >= p.n_pages) report(p.status, ECHOKV_EBADPAGE);
-      else r.page = pg;
-    }
+  if (lane < n_boxes && t0 + lane * p.page_tokens < len) {
+    if (raw_page < 0 || raw_page >= p.n_pages) report(p.status, ECHOKV_EBADPAGE);
+    else r.page = raw_page;
   }
   r.n_valid = __popc(__ballot_sync(0xffffffffu, r.page >= 0));
   const int page0 = __shfl_sync(0xffffffffu, r.page, 0);
@@ -271,6 +273,10 @@ __device__ __forceinline__ PageSet lookup_pages(const StreamParams& p, int slot,
     r.run_member = group_run && lane != lead && lane < n_boxes;
   }
   return r;
+}
+__device__ __forceinline__ PageSet lookup_pages(const StreamParams& p, int slot, int len, int t0, int n_boxes,
+                                                int lane) {
+  return make_page_set(p, load_page(p, slot, len, t0, n_boxes, lane), len, t0, n_boxes, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -528,7 +534,10 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       const Work w = decode(item);
       const bool one_pool = w.kc0 + w.n_chunks <= p.kc_anchor || w.kc0 >= p.kc_anchor;
+      int raw_next = load_page(p, w.slot, w.len, w.t_begin, boxes, lane);
       for (int step = 0; step < w.n_steps; ++step, ++it) {
+        const int raw = raw_next;      // this stage's block-table entries were requested a stage ago
+        if (step + 1 < w.n_steps) raw_next = load_page(p, w.slot, w.len, w.t_begin + (step + 1) * kPvTokens, boxes, lane);
         const uint32_t s = it % p.n_stages;
         const uint32_t ph = (it / p.n_stages) & 1u;
         const uint32_t full = smem_u32(&t.full_bar[s]);
@@ -537,7 +546,7 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) { alive = false; break; }
         const int t0 = w.t_begin + step * kPvTokens;
-        const PageSet ps = lookup_pages(p, w.slot, w.len, t0, boxes, lane);
+        const PageSet ps = make_page_set(p, raw, w.len, t0, boxes, lane);
         if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)w.n_chunks * ps.n_valid * page_bytes + p_tile_bytes);
         __syncwarp();
         const uint32_t v_dst = stage_base + s * p.stage_bytes;
@@ -665,70 +674,97 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------
-// 5. output projection
+// 5. output: sum the ranges, normalise, project
 // ---------------------------------------------------------------------------------------------
+// ysum[b][h][i] = (sum over the sequence's ranges of y[b][range][h][i]) / softmax sum of (b, h)
 __global__ void __launch_bounds__(256)
-absorb_out_kernel(const float* __restrict__ y, const float2* __restrict__ ml, const __nv_bfloat16* __restrict__ Wv,
-                  const __nv_bfloat16* __restrict__ bv, float* __restrict__ out, const int32_t* __restrict__ slots,
-                  const int32_t* __restrict__ lens, int max_batch, int capacity, int n_q_heads, int g, int n_ret,
-                  int D, int d_in, int range_tokens) {
-  extern __shared__ float ys[];     // [g][d_in]: sum_t p_t x^V_t of the group's query heads
-  const int kv = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+absorb_ysum_kernel(const float* __restrict__ y, const float2* __restrict__ ml, float* __restrict__ ysum,
+                   const int32_t* __restrict__ slots, const int32_t* __restrict__ lens, int max_batch, int capacity,
+                   int n_q_heads, int d_in, int range_tokens) {
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int i4 = blockIdx.x * 256 + threadIdx.x;        // float4 index inside the row
+  if (i4 * 4 >= d_in) return;
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
-  float* o = out + ((size_t)b * n_q_heads + kv * g) * 128;
-  if (slot < 0 || slot >= max_batch || len < 1 || len > capacity) {
-    for (int idx = tid; idx < g * 128; idx += 256) o[idx] = 0.f;
-    return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (slot >= 0 && slot < max_batch && len >= 1 && len <= capacity) {
+    const int n_ranges = (len + range_tokens - 1) / range_tokens;
+    const float4* src = reinterpret_cast<const float4*>(y + (((size_t)b * kAbsorbMaxRanges) * n_q_heads + h) * d_in) + i4;
+    const size_t range_stride4 = (size_t)n_q_heads * d_in / 4;
+    for (int r = 0; r < n_ranges; ++r) {
+      const float4 v = src[r * range_stride4];
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    const float L = ml[(size_t)b * n_q_heads + h].y;
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
   }
-  const int n_ranges = (len + range_tokens - 1) / range_tokens;
-  const float* yb = y + ((size_t)b * kAbsorbMaxRanges * n_q_heads + kv * g) * d_in;
-  const size_t range_stride = (size_t)n_q_heads * d_in;
+  reinterpret_cast<float4*>(ysum + ((size_t)b * n_q_heads + h) * d_in)[i4] = acc;
+}
+
+constexpr int kOutRows = 16;     // output features per block (two per warp)
+constexpr int kOutPairs = 8;     // (sequence, query head of the group) pairs per block
+
+// out[b][h][j] = W_v[row of (kv, j)] . ysum[b][h]  (+ b_v) for predicted heads; ysum's own dims for retained heads
+__global__ void __launch_bounds__(256)
+absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restrict__ Wv,
+                  const __nv_bfloat16* __restrict__ bv, float* __restrict__ out, int B, int n_q_heads, int g,
+                  int n_ret, int D, int d_in) {
+  const int kv = blockIdx.x, jt = blockIdx.y, first = blockIdx.z * kOutPairs;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_pairs = B * g;
   if (kv < n_ret) {
-    // a retained head: its own stored dims of y
-    for (int idx = tid; idx < g * 128; idx += 256) {
-      const int gi = idx >> 7, j = idx & 127;
-      float acc = 0.f;
-      for (int r = 0; r < n_ranges; ++r) acc += yb[r * range_stride + (size_t)gi * d_in + D + kv * 128 + j];
-      const float L = ml[(size_t)b * n_q_heads + kv * g + gi].y;
-      o[idx] = L > 0.f ? acc / L : 0.f;
+    // a retained head: its own stored dims
+    for (int idx = tid; idx < kOutPairs * kOutRows; idx += 256) {
+      const int k = idx / kOutRows, j = jt * kOutRows + idx % kOutRows;
+      const int pr = first + k;
+      if (pr >= n_pairs) continue;
+      const int b = pr / g, h = kv * g + (pr - b * g);
+      out[((size_t)b * n_q_heads + h) * 128 + j] = ysum[((size_t)b * n_q_heads + h) * d_in + D + kv * 128 + j];
     }
     return;
   }
-  for (int idx = tid; idx < g * d_in; idx += 256) {
-    float acc = 0.f;
-    for (int r = 0; r < n_ranges; ++r) acc += yb[r * range_stride + idx];
-    ys[idx] = acc;
+  const float* yrow[kOutPairs];
+#pragma unroll
+  for (int k = 0; k < kOutPairs; ++k) {
+    const int pr = min(first + k, n_pairs - 1);       // (rows past the end repeat the last pair; not stored)
+    const int b = pr / g, h = kv * g + (pr - b * g);
+    yrow[k] = ysum + ((size_t)b * n_q_heads + h) * d_in;
   }
-  __syncthreads();
-  const __nv_bfloat16* W = Wv + (size_t)(kv - n_ret) * 128 * d_in;
-  for (int j = warp; j < 128; j += 8) {
-    float acc[kMaxGroup];
+  const int j0 = jt * kOutRows + warp * 2;
+  const __nv_bfloat16* w0 = Wv + ((size_t)(kv - n_ret) * 128 + j0) * d_in;
+  const __nv_bfloat16* w1 = w0 + d_in;
+  float acc[2][kOutPairs];
 #pragma unroll
-    for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
-    const __nv_bfloat16* wrow = W + (size_t)j * d_in;
-    for (int i = lane * 8; i < d_in; i += 256) {
-      float wv[8];
-      Vec16<__nv_bfloat16>::load(wrow + i, wv);
+  for (int k = 0; k < kOutPairs; ++k) acc[0][k] = acc[1][k] = 0.f;
+  for (int i = lane * 8; i < d_in; i += 256) {
+    float wa[8], wb[8];
+    Vec16<__nv_bfloat16>::load(w0 + i, wa);
+    Vec16<__nv_bfloat16>::load(w1 + i, wb);
 #pragma unroll
-      for (int gi = 0; gi < kMaxGroup; ++gi) {
-        if (gi < g) {
-          const float* yy = ys + (size_t)gi * d_in + i;
+    for (int k = 0; k < kOutPairs; ++k) {
+      const float4 y0 = *reinterpret_cast<const float4*>(yrow[k] + i);
+      const float4 y1 = *reinterpret_cast<const float4*>(yrow[k] + i + 4);
+      const float yy[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[gi] = fmaf(wv[e], yy[e], acc[gi]);
-        }
+      for (int e = 0; e < 8; ++e) {
+        acc[0][k] = fmaf(wa[e], yy[e], acc[0][k]);
+        acc[1][k] = fmaf(wb[e], yy[e], acc[1][k]);
       }
     }
+  }
 #pragma unroll
-    for (int gi = 0; gi < kMaxGroup; ++gi) {
-      if (gi < g) {
-        const float tot = warp_sum(acc[gi]);
-        if (lane == 0) {
-          const float L = ml[(size_t)b * n_q_heads + kv * g + gi].y;
-          float res = L > 0.f ? tot / L : 0.f;
-          if (bv != nullptr) res += __bfloat162float(bv[(kv - n_ret) * 128 + j]);
-          o[gi * 128 + j] = res;
-        }
+  for (int rr = 0; rr < 2; ++rr) {
+#pragma unroll
+    for (int k = 0; k < kOutPairs; ++k) {
+      const float tot = warp_sum(acc[rr][k]);
+      const int pr = first + k;
+      if (lane == 0 && pr < n_pairs) {
+        const int b = pr / g, h = kv * g + (pr - b * g);
+        const int j = j0 + rr;
+        float res = tot;
+        if (bv != nullptr) res += __bfloat162float(bv[(kv - n_ret) * 128 + j]);
+        out[((size_t)b * n_q_heads + h) * 128 + j] = res;
       }
     }
   }
@@ -756,6 +792,7 @@ void absorbed_layout(int max_batch, int n_q_heads, int d_in, int capacity_tokens
   out->off_p2 = off; off = align(off + (uint64_t)max_batch * out->nh2 * out->l_cap * 2);
   out->off_ml = off; off = align(off + (uint64_t)max_batch * n_q_heads * 8);
   out->off_y = off; off = align(off + (uint64_t)max_batch * kAbsorbMaxRanges * n_q_heads * d_in * 4);
+  out->off_ysum = off; off = align(off + (uint64_t)max_batch * n_q_heads * d_in * 4);
   out->total = off;
 }
 
@@ -783,6 +820,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   __nv_bfloat16* p2 = reinterpret_cast<__nv_bfloat16*>(r.ws + lay.off_p2);
   float2* ml = reinterpret_cast<float2*>(r.ws + lay.off_ml);
   float* y = reinterpret_cast<float*>(r.ws + lay.off_y);
+  float* ysum = reinterpret_cast<float*>(r.ws + lay.off_ysum);
   cudaError_t e;
 
   // 1. absorbed queries
@@ -850,10 +888,13 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   int range_tokens;
   {
     p.n_slices = (p.kc_total + 3) / 4;
-    int ranges = (4 * sm_count + p.n_slices * a.batch - 1) / (p.n_slices * a.batch);
+    // about ten items per CTA so that the persistent grid ends evenly, but ranges of >= 1024 tokens so that
+    // the partial results stay small next to what a range reads
+    int ranges = (10 * sm_count + p.n_slices * a.batch - 1) / (p.n_slices * a.batch);
     if (ranges > kAbsorbMaxRanges) ranges = kAbsorbMaxRanges;
     if (ranges < 1) ranges = 1;
     range_tokens = round_up((capacity + ranges - 1) / ranges, kPvTokens);
+    if (range_tokens < 1024) range_tokens = 1024;
     p.range_tokens = range_tokens;
     p.stage_bytes = kPvVBytes + (uint32_t)lay.nh2 * kRowBytes;
     p.n_stages = (int)(kSmemBudget / p.stage_bytes);
@@ -876,17 +917,16 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     if (ev) cudaEventRecord(ev[3], stream);
   }
 
-  // 5. output projection
+  // 5. sum the ranges, normalise, project
   {
-    const size_t smem = (size_t)g * d_in * sizeof(float);
-    if ((e = cudaFuncSetAttribute(absorb_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
-        cudaSuccess)
-      return e;
-    dim3 grid(a.n_kv_heads, a.batch);
-    absorb_out_kernel<<<grid, 256, smem, stream>>>(y, ml, reinterpret_cast<const __nv_bfloat16*>(r.Wv),
-                                                   reinterpret_cast<const __nv_bfloat16*>(r.bv), out, a.slots, a.lens,
-                                                   a.geom.max_batch, capacity, a.n_q_heads, g, n_ret, r.D, d_in,
-                                                   range_tokens);
+    dim3 grid1((d_in / 4 + 255) / 256, a.n_q_heads, a.batch);
+    absorb_ysum_kernel<<<grid1, 256, 0, stream>>>(y, ml, ysum, a.slots, a.lens, a.geom.max_batch, capacity,
+                                                  a.n_q_heads, d_in, range_tokens);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    dim3 grid2(a.n_kv_heads, 128 / kOutRows, (a.batch * g + kOutPairs - 1) / kOutPairs);
+    absorb_out_kernel<<<grid2, 256, 0, stream>>>(ysum, reinterpret_cast<const __nv_bfloat16*>(r.Wv),
+                                                 reinterpret_cast<const __nv_bfloat16*>(r.bv), out, a.batch,
+                                                 a.n_q_heads, g, n_ret, r.D, d_in);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;

@@ -13,7 +13,7 @@
 
 namespace echokv {
 
-constexpr int kAbsorbMaxRanges = 4;      // token ranges the V pass may split a sequence into
+constexpr int kAbsorbMaxRanges = 16;     // token ranges the V pass may split a sequence into
 constexpr int kAbsorbTokAlign = 128;     // score rows are padded to this many tokens
 
 struct AbsorbLayout {
@@ -24,6 +24,7 @@ struct AbsorbLayout {
   uint64_t off_p2;  // bf16 [max_batch * nh2][l_cap]     probabilities, split into two bf16 halves
   uint64_t off_ml;  // float2 [max_batch][n_q_heads]      (max, sum) of every head
   uint64_t off_y;   // fp32 [max_batch][ranges][n_q_heads][D_in]  partial probability-weighted inputs
+  uint64_t off_ysum; // fp32 [max_batch][n_q_heads][D_in]         their sum over ranges, divided by the softmax sum
   uint64_t total;
 };
 

@@ -472,7 +472,7 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
                        timed_pair(c, ECHOKV_TIMED_ABSORB_V, &ev[2], &ev[3]);
     if (launch_absorbed(a, aa, c->amaps, A.tc, L.tc, out, c->sm_count, s, timed ? ev : nullptr) != cudaSuccess)
       return ECHOKV_ECUDA;
-    c->launches += 5;
+    c->launches += 6;
     return ECHOKV_OK;
   }
   const int r = c->cfg.n_retained_heads;
