@@ -234,38 +234,41 @@ __device__ __forceinline__ void stream_setup(StreamSmemTail& t, const StreamPara
   tc_fence_after();
 }
 
-// Pages of `n_boxes` consecutive page-sized boxes starting at token t0 of the sequence in block-table
-// row `slot` (lane i holds box i; -1 = no cached token there or a bad page id), whether they form one
-// consecutive run, and for 64-row sub-runs which lane leads / follows.
+// The `n_boxes` boxes of `box_tokens` token rows (a page, or part of a page when pages are taller than the
+// span wanted) that start at token t0 of the sequence in block-table row `slot`: lane i holds the pool row
+// where box i starts (-1 = no cached token there or a bad page id); whether the boxes form one
+// consecutive run in the pool; and for 64-row sub-runs which lane leads / follows.
 struct PageSet {
-  int page;
+  int row;
   bool all_run;        // every box valid and consecutive in the pool
   bool run_lead, run_member;
   uint32_t n_valid;
 };
-// Block-table entry of box `lane` (only the load: callers issue it a stage ahead of its use)
-__device__ __forceinline__ int load_page(const StreamParams& p, int slot, int len, int t0, int n_boxes, int lane) {
-  const int tb = t0 + lane * p.page_tokens;
+// Block-table entry of box `lane` (only the load: callers may issue it a stage ahead of its use)
+__device__ __forceinline__ int load_page(const StreamParams& p, int slot, int len, int t0, int n_boxes,
+                                         int box_tokens, int lane) {
+  const int tb = t0 + lane * box_tokens;
   if (lane < n_boxes && tb < len) return p.table[(size_t)slot * p.max_pages_per_seq + tb / p.page_tokens];
   return -1;
 }
 __device__ __forceinline__ PageSet make_page_set(const StreamParams& p, int raw_page, int len, int t0, int n_boxes,
-                                                 int lane) {
+                                                 int box_tokens, int lane) {
   PageSet r;
-  r.page = -1;
-  if (lane < n_boxes && t0 + lane * p.page_tokens < len) {
+  r.row = -1;
+  const int tb = t0 + lane * box_tokens;
+  if (lane < n_boxes && tb < len) {
     if (raw_page < 0 || raw_page >= p.n_pages) report(p.status, ECHOKV_EBADPAGE);
-    else r.page = raw_page;
+    else r.row = raw_page * p.page_tokens + tb % p.page_tokens;
   }
-  r.n_valid = __popc(__ballot_sync(0xffffffffu, r.page >= 0));
-  const int page0 = __shfl_sync(0xffffffffu, r.page, 0);
-  r.all_run = __all_sync(0xffffffffu, lane >= n_boxes || (r.page >= 0 && r.page == page0 + lane));
+  r.n_valid = __popc(__ballot_sync(0xffffffffu, r.row >= 0));
+  const int row0 = __shfl_sync(0xffffffffu, r.row, 0);
+  r.all_run = __all_sync(0xffffffffu, lane >= n_boxes || (r.row >= 0 && r.row == row0 + lane * box_tokens));
   r.run_lead = r.run_member = false;
   if (p.run_pages > 1) {
-    bool consecutive = r.page >= 0;
+    bool consecutive = r.row >= 0;
     for (int k = 1; k < p.run_pages; ++k) {
-      const int pk = __shfl_down_sync(0xffffffffu, r.page, k);
-      consecutive = consecutive && pk == r.page + k;
+      const int rk = __shfl_down_sync(0xffffffffu, r.row, k);
+      consecutive = consecutive && rk == r.row + k * box_tokens;
     }
     const int lead = lane - lane % p.run_pages;
     const bool group_run = __shfl_sync(0xffffffffu, consecutive ? 1 : 0, lead) != 0;
@@ -275,8 +278,8 @@ __device__ __forceinline__ PageSet make_page_set(const StreamParams& p, int raw_
   return r;
 }
 __device__ __forceinline__ PageSet lookup_pages(const StreamParams& p, int slot, int len, int t0, int n_boxes,
-                                                int lane) {
-  return make_page_set(p, load_page(p, slot, len, t0, n_boxes, lane), len, t0, n_boxes, lane);
+                                                int box_tokens, int lane) {
+  return make_page_set(p, load_page(p, slot, len, t0, n_boxes, box_tokens, lane), len, t0, n_boxes, box_tokens, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -301,8 +304,9 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
   const uint32_t tmem = t.tmem_base;
   const int n_items = t.cum[p.nb];
   const int n_steps = p.kc_total / 2;                     // stages per item: two chunks each
-  const int boxes = kScoreTokens / p.page_tokens;
-  const uint32_t page_bytes = p.page_tokens * kRowBytes;
+  const int box_tokens = min(p.page_tokens, kScoreTokens);
+  const int boxes = kScoreTokens / box_tokens;
+  const uint32_t page_bytes = box_tokens * kRowBytes;
   const uint32_t q_chunk_bytes = (uint32_t)p.nh2 * kRowBytes;
 
   if (warp == 0) {
@@ -315,7 +319,7 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
       const int tile = item - t.cum[bi];
       const int slot = p.slots ? p.slots[b] : b;
       const int len = p.lens[b];
-      const PageSet ps = lookup_pages(p, slot, len, tile * kScoreTokens, boxes, lane);
+      const PageSet ps = lookup_pages(p, slot, len, tile * kScoreTokens, boxes, box_tokens, lane);
       const uint32_t stage_tx = 2u * (ps.n_valid * page_bytes + q_chunk_bytes);
       for (int step = 0; step < n_steps; ++step, ++it) {
         const uint32_t s = it % p.n_stages;
@@ -333,14 +337,13 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
         const uint32_t x_dst = stage_base + s * p.stage_bytes;
         if (ps.all_run) {
           if (lane == 0)
-            tma_load_3d(x_dst, from_anchor ? &tm_anchor_128 : &tm_local_128, 0, ps.page * p.page_tokens, kx0, full);
-        } else if (ps.page >= 0 && !ps.run_member) {
+            tma_load_3d(x_dst, from_anchor ? &tm_anchor_128 : &tm_local_128, 0, ps.row, kx0, full);
+        } else if (ps.row >= 0 && !ps.run_member) {
           const CUtensorMap* m = ps.run_lead ? (from_anchor ? &tm_anchor_run : &tm_local_run)
                                              : (from_anchor ? &tm_anchor : &tm_local);
 #pragma unroll
           for (int j = 0; j < 2; ++j)
-            tma_load_2d(x_dst + j * kScoreXBytes + lane * page_bytes, m, (kx0 + j) * kChunk,
-                        ps.page * p.page_tokens, full);
+            tma_load_2d(x_dst + j * kScoreXBytes + lane * page_bytes, m, (kx0 + j) * kChunk, ps.row, full);
         }
         if (lane == 16) tma_load_3d(x_dst + 2 * kScoreXBytes, &tm_q2, 0, b * p.nh2, kc0, full);
       }
@@ -503,8 +506,9 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
   });
   const uint32_t tmem = t.tmem_base;
   const int n_items = t.cum[p.nb];
-  const int boxes = kPvTokens / p.page_tokens;              // page boxes per chunk and stage (>= 1)
-  const uint32_t page_bytes = p.page_tokens * kRowBytes;
+  const int box_tokens = min(p.page_tokens, kPvTokens);     // (a taller page is read 64 rows at a time)
+  const int boxes = kPvTokens / box_tokens;                 // boxes per chunk and stage
+  const uint32_t page_bytes = box_tokens * kRowBytes;
   const uint32_t p_tile_bytes = (uint32_t)p.nh2 * kRowBytes;
 
   // item -> (sequence, range, slice); its token span and chunk span
@@ -534,10 +538,11 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       const Work w = decode(item);
       const bool one_pool = w.kc0 + w.n_chunks <= p.kc_anchor || w.kc0 >= p.kc_anchor;
-      int raw_next = load_page(p, w.slot, w.len, w.t_begin, boxes, lane);
+      int raw_next = load_page(p, w.slot, w.len, w.t_begin, boxes, box_tokens, lane);
       for (int step = 0; step < w.n_steps; ++step, ++it) {
         const int raw = raw_next;      // this stage's block-table entries were requested a stage ago
-        if (step + 1 < w.n_steps) raw_next = load_page(p, w.slot, w.len, w.t_begin + (step + 1) * kPvTokens, boxes, lane);
+        if (step + 1 < w.n_steps)
+          raw_next = load_page(p, w.slot, w.len, w.t_begin + (step + 1) * kPvTokens, boxes, box_tokens, lane);
         const uint32_t s = it % p.n_stages;
         const uint32_t ph = (it / p.n_stages) & 1u;
         const uint32_t full = smem_u32(&t.full_bar[s]);
@@ -546,21 +551,23 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) { alive = false; break; }
         const int t0 = w.t_begin + step * kPvTokens;
-        const PageSet ps = make_page_set(p, raw, w.len, t0, boxes, lane);
+        const PageSet ps = make_page_set(p, raw, w.len, t0, boxes, box_tokens, lane);
         if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)w.n_chunks * ps.n_valid * page_bytes + p_tile_bytes);
         __syncwarp();
         const uint32_t v_dst = stage_base + s * p.stage_bytes;
         if (ps.all_run && w.n_chunks == 4 && one_pool && p.v_tile_ok) {
           if (lane == 0)
-            tma_load_3d(v_dst, w.from_anchor ? &tm_anchor_4 : &tm_local_4, 0, ps.page * p.page_tokens,
+            tma_load_3d(v_dst, w.from_anchor ? &tm_anchor_4 : &tm_local_4, 0, ps.row,
                         w.from_anchor ? w.kc0 : w.kc0 - p.kc_anchor, full);
-        } else if (ps.page >= 0 && !ps.run_member) {
+        } else if (ps.row >= 0 && !ps.run_member) {
           for (int c = 0; c < w.n_chunks; ++c) {
             const int kc = w.kc0 + c;
             const bool fa = kc < p.kc_anchor;
-            const CUtensorMap* m = ps.run_lead ? (fa ? &tm_anchor_run : &tm_local_run) : (fa ? &tm_anchor : &tm_local);
-            tma_load_2d(v_dst + c * kPvTileBytes + lane * page_bytes, m, (fa ? kc : kc - p.kc_anchor) * kChunk,
-                        ps.page * p.page_tokens, full);
+            // (pages of 64 tokens or more: the 64-row maps are the box of one stage)
+            const bool tall = ps.run_lead || p.page_tokens >= kPvTokens;
+            const CUtensorMap* m = tall ? (fa ? &tm_anchor_run : &tm_local_run) : (fa ? &tm_anchor : &tm_local);
+            tma_load_2d(v_dst + c * kPvTileBytes + lane * page_bytes, m, (fa ? kc : kc - p.kc_anchor) * kChunk, ps.row,
+                        full);
           }
         }
         if (lane == 16) tma_load_2d(v_dst + kPvVBytes, &tm_p2, t0, w.b * p.nh2, full);

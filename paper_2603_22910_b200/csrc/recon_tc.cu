@@ -553,8 +553,8 @@ cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const voi
   if (e != cudaSuccess) return e;
   e = encode_2d(&maps->v_pool, v_pool, rows, width, page_tokens, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (e != cudaSuccess) return e;
-  // tall boxes over runs of consecutive pages (the same maps again when a page is already that tall)
-  const int run_rows = page_tokens < kRunTokens ? kRunTokens : page_tokens;
+  // boxes of 64 token rows: runs of consecutive pages, or part of a page that is taller
+  const int run_rows = kRunTokens;
   e = encode_2d(&maps->k_pool_run, k_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (e != cudaSuccess) return e;
   e = encode_2d(&maps->v_pool_run, v_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
