@@ -392,6 +392,50 @@ def workload_config(w, full=False):
 
 
 # --------------------------------------------------------------------------------------------
+# Replicas: the path has no exchange step, so N GPUs run N independent copies of the batch
+# --------------------------------------------------------------------------------------------
+class Replicas:
+    """One process per GPU.  The only communication is the timing protocol: a barrier on both sides
+    of the timed region and the maximum of the measured time over the ranks."""
+
+    def __init__(self, backend="nccl", device=None):
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.device = device
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            self.dist = dist
+            kw = {"device_id": device} if (backend == "nccl" and device is not None) else {}
+            dist.init_process_group(backend, **kw)
+
+    def seed_for(self, base_seed):
+        """Every replica draws its own batch."""
+        return base_seed + 7919 * self.rank
+
+    def barrier(self):
+        if self.dist:
+            self.dist.barrier()
+
+    def max_over_ranks(self, ms):
+        if not self.dist:
+            return ms
+        import torch
+        t = torch.tensor([ms], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def job_value(self, units_per_rank, ms_step):
+        """Whole-job throughput: what all ranks processed divided by the slowest rank's time."""
+        return self.world * units_per_rank / (ms_step * 1e-3)
+
+    def close(self):
+        if self.dist:
+            self.dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------------
 # GPU arm
 # --------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -399,27 +443,19 @@ def run_ours(args):
     import torch
     from paper_2603_22910_b200 import binding, build
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
+    rep = Replicas("nccl", torch.device("cuda", local_rank))
+    rank, world, dist = rep.rank, rep.world, rep.dist
     if rank == 0:
         build.build()
-    if dist:
-        dist.barrier()
+    rep.barrier()
     binding.lib()
 
     w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio)
-    if world > 1:
-        w = w.replace(seed=w.seed + 7919 * rank)   # every replica has its own batch
+    w = w.replace(seed=rep.seed_for(w.seed))
     full = args.mode == "full"
     resident, step_layers = plan_layers(w, args.mode)
     st = State(w, local_rank, resident)
@@ -453,15 +489,10 @@ def run_ours(args):
     def sync_all():
         torch.cuda.synchronize()
         if dist:
-            dist.barrier()
+            rep.barrier()
             torch.cuda.synchronize()
 
-    def max_over_ranks(ms):
-        if not dist:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    max_over_ranks = rep.max_over_ranks
 
     for _ in range(args.warmup):
         step()
@@ -508,8 +539,8 @@ def run_ours(args):
     same = bool(torch.equal(st.out_host[last], st.out[last].cpu()))
 
     ms_step = ms_total / args.steps
-    value = world * w.batch / (ms_step * 1e-3)
-    e2e_value = world * w.batch / (ms_e2e / args.steps * 1e-3)
+    value = rep.job_value(w.batch, ms_step)
+    e2e_value = rep.job_value(w.batch, ms_e2e / args.steps)
 
     peaks, peaks_kind = load_peaks()
     flops, bytes_ = algorithmic_work(w)
@@ -598,8 +629,7 @@ def run_ours(args):
     if rank == 0:
         print(json.dumps(line))
     ctx.close()
-    if dist:
-        dist.destroy_process_group()
+    rep.close()
     return 0
 
 

@@ -1,0 +1,94 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the workloads
+are too large for the oracle to evaluate whole, so a seeded sample of (layer, sequence, query head)
+outputs is recomputed one by one (heads are independent in Eq. 7, and a predicted head needs only
+its own rows of W in Eq. 3).  Inputs are drawn on the device by the seeded generators and read back
+from the pools for the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from oracle import echokv_oracle as O
+from paper_2603_22910_b200 import binding, build, synth
+from tests.harness import TOL
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.lib()
+
+
+def sampled_check(w, mode, samples, absorbed, seed=7):
+    resident, step_layers = bench.plan_layers(w, mode)
+    st = bench.State(w, 0, resident)
+    ctx = st.ctx
+    if absorbed:
+        ctx.enable_absorbed()
+    for l, attend in step_layers:          # exactly bench.py's step
+        ctx.append_kv(l, st.new_dev[(l, "k")], st.new_dev[(l, "v")], st.positions)
+        if attend:
+            if mode == "full" or w.is_anchor(l):
+                ctx.full_attention(l, st.q_dev[l], st.lens, out=st.out[l])
+            else:
+                ctx.decode_attention(l, st.q_dev[l], st.lens, out=st.out[l])
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.ECHOKV_OK
+    rng = np.random.default_rng(seed)
+    attend_layers = [l for l, a in step_layers if a]
+    tol = TOL[w.dtype]
+    worst = 0.0
+    num = den = 0.0
+    for _ in range(samples):
+        l = int(rng.choice(attend_layers))
+        b = int(rng.integers(w.batch))
+        h = int(rng.integers(w.n_q_heads))
+        inputs = st.oracle_inputs(l, b)
+        if len(inputs) == 3:                # a stored (anchor / uncompressed) layer: only the head's own dims
+            q, kg, vg = inputs
+            kv = h // (w.n_q_heads // w.n_kv_heads)
+            d = w.head_dim
+            ref = O.attention(q[h:h + 1], kg[:, None, kv * d:(kv + 1) * d], vg[:, None, kv * d:(kv + 1) * d])[0]
+        else:
+            ref = O.decode_attention_query_heads(*inputs, n_kv_heads=w.n_kv_heads, query_heads=[h])[h]
+        got = st.out[l][b, h].cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got))
+        worst = max(worst, float(np.max(np.abs(got - ref))))
+        num += float(np.sum((got - ref) ** 2))
+        den += float(np.sum(ref ** 2))
+    rel = (num / max(den, 1e-300)) ** 0.5
+    ctx.close()
+    del st
+    torch.cuda.empty_cache()
+    assert worst <= tol["max_abs"] and rel <= tol["rel_l2"], (worst, rel)
+    return worst, rel
+
+
+@pytest.mark.parametrize("absorbed", [False, True], ids=["explicit", "absorbed"])
+def test_config1_full_size_sampled(absorbed):
+    sampled_check(synth.C1, "compressed", samples=6, absorbed=absorbed)
+
+
+@pytest.mark.parametrize("absorbed", [False, True], ids=["explicit", "absorbed"])
+def test_config2_full_size_sampled(absorbed):
+    sampled_check(synth.C2, "compressed", samples=6, absorbed=absorbed)
+
+
+@pytest.mark.parametrize("absorbed", [False, True], ids=["explicit", "absorbed"])
+def test_config3_full_size_32_layers_sampled(absorbed):
+    sampled_check(synth.C3, "compressed", samples=8, absorbed=absorbed)
+
+
+def test_config4_sweep_points_sampled():
+    # one point per compression ratio, at the long-context end that still keeps the run short
+    for ratio, context, batch in ((25, 65536, 4), (50, 131072, 2), (75, 16384, 32)):
+        sampled_check(synth.c4_point(ratio, context, batch), "compressed", samples=3, absorbed=False)
+    sampled_check(synth.c4_point(75, 131072, 2), "compressed", samples=3, absorbed=True)
+
+
+def test_uncompressed_path_full_size_sampled():
+    sampled_check(synth.C1, "full", samples=4, absorbed=False)
+    sampled_check(synth.C2, "full", samples=4, absorbed=False)
