@@ -83,13 +83,14 @@ inline uint32_t make_idesc(int n, bool a_mmajor) {
 // 1. absorbed queries
 // ---------------------------------------------------------------------------------------------
 constexpr int kQGroup = 8;   // (sequence, query head of the group) pairs per block
+constexpr int kQCols = 512;  // input features per block: two adjacent ones per thread
 
 __global__ void __launch_bounds__(256)
 absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ Wk,
                     __nv_bfloat16* __restrict__ q2, int B, int n_q_heads, int g, int n_ret, int D, int d_in,
                     float scale_log2e) {
   __shared__ float qs[kQGroup][128];
-  const int i = blockIdx.x * 256 + threadIdx.x;     // input feature (column of W_k)
+  const int i = blockIdx.x * kQCols + threadIdx.x * 2;     // first of this thread's two input features
   const int kv = blockIdx.y;
   const int first = blockIdx.z * kQGroup;
   const int n_pairs = B * g;
@@ -105,23 +106,30 @@ absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   }
   __syncthreads();
   if (i >= d_in) return;
-  float acc[kQGroup];
+  float acc[kQGroup][2];
 #pragma unroll
-  for (int k = 0; k < kQGroup; ++k) acc[k] = 0.f;
+  for (int k = 0; k < kQGroup; ++k) acc[k][0] = acc[k][1] = 0.f;
   if (kv < n_ret) {
     // a retained head reads its own stored dims: q~ is q placed at the head's local dims
     const int j = i - (D + kv * 128);
     if (j >= 0 && j < 128) {
 #pragma unroll
-      for (int k = 0; k < kQGroup; ++k) acc[k] = qs[k][j];
+      for (int k = 0; k < kQGroup; ++k) {
+        acc[k][0] = qs[k][j];
+        acc[k][1] = qs[k][j + 1];
+      }
     }
   } else {
     const __nv_bfloat16* w = Wk + (size_t)(kv - n_ret) * 128 * d_in + i;
 #pragma unroll 16
     for (int j = 0; j < 128; ++j) {
-      const float wv = __bfloat162float(w[(size_t)j * d_in]);
+      const uint32_t raw = *reinterpret_cast<const uint32_t*>(w + (size_t)j * d_in);
+      const float w0 = __uint_as_float(raw << 16), w1 = __uint_as_float(raw & 0xffff0000u);
 #pragma unroll
-      for (int k = 0; k < kQGroup; ++k) acc[k] = fmaf(wv, qs[k][j], acc[k]);
+      for (int k = 0; k < kQGroup; ++k) {
+        acc[k][0] = fmaf(w0, qs[k][j], acc[k][0]);
+        acc[k][1] = fmaf(w1, qs[k][j], acc[k][1]);
+      }
     }
   }
   const int nh2 = 2 * n_q_heads;
@@ -131,10 +139,10 @@ absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     if (pr >= n_pairs) break;
     const int b = pr / g, gi = pr - b * g;
     const int h = kv * g + gi;
-    const __nv_bfloat16 hi = __float2bfloat16_rn(acc[k]);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(acc[k] - __bfloat162float(hi));
-    q2[((size_t)b * nh2 + h) * d_in + i] = hi;
-    q2[((size_t)b * nh2 + n_q_heads + h) * d_in + i] = lo;
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(acc[k][0], acc[k][1]);
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[k][0] - __low2float(hi), acc[k][1] - __high2float(hi));
+    *reinterpret_cast<__nv_bfloat162*>(q2 + ((size_t)b * nh2 + h) * d_in + i) = hi;
+    *reinterpret_cast<__nv_bfloat162*>(q2 + ((size_t)b * nh2 + n_q_heads + h) * d_in + i) = lo;
   }
 }
 
@@ -709,14 +717,17 @@ absorb_ysum_kernel(const float* __restrict__ y, const float2* __restrict__ ml, f
   reinterpret_cast<float4*>(ysum + ((size_t)b * n_q_heads + h) * d_in)[i4] = acc;
 }
 
-constexpr int kOutRows = 16;     // output features per block (two per warp)
+constexpr int kOutRows = 16;     // output features per block
 constexpr int kOutPairs = 8;     // (sequence, query head of the group) pairs per block
 
-// out[b][h][j] = W_v[row of (kv, j)] . ysum[b][h]  (+ b_v) for predicted heads; ysum's own dims for retained heads
+// out[b][h][j] = W_v[row of (kv, j)] . ysum[b][h]  (+ b_v) for predicted heads; ysum's own dims for retained
+// heads.  A block takes 16 output features x 8 (sequence, head) pairs; its 8 warps split the contraction,
+// so every y value loaded is used for all 16 rows.
 __global__ void __launch_bounds__(256)
 absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restrict__ Wv,
                   const __nv_bfloat16* __restrict__ bv, float* __restrict__ out, int B, int n_q_heads, int g,
                   int n_ret, int D, int d_in) {
+  __shared__ float red[8][kOutRows][kOutPairs];
   const int kv = blockIdx.x, jt = blockIdx.y, first = blockIdx.z * kOutPairs;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_pairs = B * g;
@@ -734,45 +745,54 @@ absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restric
   const float* yrow[kOutPairs];
 #pragma unroll
   for (int k = 0; k < kOutPairs; ++k) {
-    const int pr = min(first + k, n_pairs - 1);       // (rows past the end repeat the last pair; not stored)
+    const int pr = min(first + k, n_pairs - 1);       // (pairs past the end repeat the last one; not stored)
     const int b = pr / g, h = kv * g + (pr - b * g);
     yrow[k] = ysum + ((size_t)b * n_q_heads + h) * d_in;
   }
-  const int j0 = jt * kOutRows + warp * 2;
-  const __nv_bfloat16* w0 = Wv + ((size_t)(kv - n_ret) * 128 + j0) * d_in;
-  const __nv_bfloat16* w1 = w0 + d_in;
-  float acc[2][kOutPairs];
+  const __nv_bfloat16* w = Wv + ((size_t)(kv - n_ret) * 128 + jt * kOutRows) * d_in;
+  float acc[kOutRows][kOutPairs];
 #pragma unroll
-  for (int k = 0; k < kOutPairs; ++k) acc[0][k] = acc[1][k] = 0.f;
-  for (int i = lane * 8; i < d_in; i += 256) {
-    float wa[8], wb[8];
-    Vec16<__nv_bfloat16>::load(w0 + i, wa);
-    Vec16<__nv_bfloat16>::load(w1 + i, wb);
+  for (int r = 0; r < kOutRows; ++r)
+#pragma unroll
+    for (int k = 0; k < kOutPairs; ++k) acc[r][k] = 0.f;
+  // warp w takes columns [w * 32 * 4, ...) in steps of 8 warps x 32 lanes x 4 columns
+  for (int i = (warp * 32 + lane) * 4; i < d_in; i += 8 * 32 * 4) {
+    float yy[kOutPairs][4];
 #pragma unroll
     for (int k = 0; k < kOutPairs; ++k) {
-      const float4 y0 = *reinterpret_cast<const float4*>(yrow[k] + i);
-      const float4 y1 = *reinterpret_cast<const float4*>(yrow[k] + i + 4);
-      const float yy[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+      const float4 v = *reinterpret_cast<const float4*>(yrow[k] + i);
+      yy[k][0] = v.x; yy[k][1] = v.y; yy[k][2] = v.z; yy[k][3] = v.w;
+    }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        acc[0][k] = fmaf(wa[e], yy[e], acc[0][k]);
-        acc[1][k] = fmaf(wb[e], yy[e], acc[1][k]);
-      }
+    for (int r = 0; r < kOutRows; ++r) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(w + (size_t)r * d_in + i);
+      const float wv[4] = {__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
+                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u)};
+#pragma unroll
+      for (int k = 0; k < kOutPairs; ++k)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[r][k] = fmaf(wv[e], yy[k][e], acc[r][k]);
     }
   }
 #pragma unroll
-  for (int rr = 0; rr < 2; ++rr) {
+  for (int r = 0; r < kOutRows; ++r)
 #pragma unroll
     for (int k = 0; k < kOutPairs; ++k) {
-      const float tot = warp_sum(acc[rr][k]);
-      const int pr = first + k;
-      if (lane == 0 && pr < n_pairs) {
-        const int b = pr / g, h = kv * g + (pr - b * g);
-        const int j = j0 + rr;
-        float res = tot;
-        if (bv != nullptr) res += __bfloat162float(bv[(kv - n_ret) * 128 + j]);
-        out[((size_t)b * n_q_heads + h) * 128 + j] = res;
-      }
+      const float tot = warp_sum(acc[r][k]);
+      if (lane == 0) red[warp][r][k] = tot;
+    }
+  __syncthreads();
+  if (tid < kOutRows * kOutPairs) {
+    const int r = tid / kOutPairs, k = tid % kOutPairs;
+    const int pr = first + k;
+    if (pr < n_pairs) {
+      float res = 0.f;
+#pragma unroll
+      for (int ww = 0; ww < 8; ++ww) res += red[ww][r][k];
+      const int b = pr / g, h = kv * g + (pr - b * g);
+      const int j = jt * kOutRows + r;
+      if (bv != nullptr) res += __bfloat162float(bv[(kv - n_ret) * 128 + j]);
+      out[((size_t)b * n_q_heads + h) * 128 + j] = res;
     }
   }
 }
@@ -832,7 +852,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
 
   // 1. absorbed queries
   {
-    dim3 grid((d_in + 255) / 256, a.n_kv_heads, (a.batch * g + kQGroup - 1) / kQGroup);
+    dim3 grid((d_in + kQCols - 1) / kQCols, a.n_kv_heads, (a.batch * g + kQGroup - 1) / kQGroup);
     absorb_query_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q),
                                                   reinterpret_cast<const __nv_bfloat16*>(r.Wk), q2, a.batch,
                                                   a.n_q_heads, g, n_ret, r.D, d_in, a.scale_log2e);
