@@ -26,7 +26,8 @@ Readings of points the paper leaves open (all listed in the design notes):
   * predictor input order is [global ; local] as written in Eq. 3.
   * flattening is head-major: flat index = head * d + feature.
   * query head h attends KV head floor(h / (H_q / H_kv)) (contiguous groups).
-  * every cached token, the newest included, is reconstructed alike.
+  * every cached token, the newest included, is reconstructed alike, unless a
+    sink / recent window is asked for (Section 5.1): those tokens keep all dims.
 
 Pins (tests/test_oracle_*.py): hand-computed softmax case, pure-python brute
 force, torch scaled_dot_product_attention (library routine) for the m = D and
@@ -213,7 +214,8 @@ def decode_attention_query_heads(q: np.ndarray,
                                  k_global: np.ndarray, v_global: np.ndarray,
                                  k_local: np.ndarray, v_local: np.ndarray,
                                  Wk: np.ndarray, Wv: np.ndarray,
-                                 n_kv_heads: int, query_heads, scale: float | None = None
+                                 n_kv_heads: int, query_heads, scale: float | None = None,
+                                 k_true_drop=None, v_true_drop=None, n_sink: int = 0, n_window: int = 0
                                  ) -> dict[int, np.ndarray]:
     """The same quantity as decode_attention, for a chosen few query heads only.
 
@@ -244,12 +246,58 @@ def decode_attention_query_heads(q: np.ndarray,
             rows = slice(lo - m, lo - m + d)
             K_h = predictor_input(k_global, k_local) @ np.asarray(Wk, dtype=np.float64)[rows].T
             V_h = predictor_input(v_global, v_local) @ np.asarray(Wv, dtype=np.float64)[rows].T
+            if n_sink or n_window:       # sink / window tokens keep their true dims
+                keep = full_precision_tokens(K_h.shape[0], n_sink, n_window)
+                K_h = overlay_true_dims(K_h, np.asarray(k_true_drop, dtype=np.float64)[:, rows], keep)
+                V_h = overlay_true_dims(V_h, np.asarray(v_true_drop, dtype=np.float64)[:, rows], keep)
         else:
             raise ValueError("m must be head-aligned for per-head evaluation")
         s = (K_h @ q[h]) * scale
         e = np.exp(s - s.max())
         out[h] = (e / e.sum()) @ V_h
     return out
+
+
+# ----------------------------------------------------------------------------
+# Sink and recent-window tokens kept at full precision (Section 5.1, "Implement
+# details": 4 sink tokens and a local window of 128 tokens)
+# ----------------------------------------------------------------------------
+
+
+def full_precision_tokens(L: int, n_sink: int, n_window: int) -> np.ndarray:
+    """Boolean [L]: token t keeps its whole K / V (nothing of it is predicted) iff it
+    is one of the first n_sink tokens or one of the last n_window tokens."""
+    if n_sink < 0 or n_window < 0:
+        raise ValueError("negative sink / window size")
+    t = np.arange(L)
+    return (t < n_sink) | (t >= L - n_window)
+
+
+def overlay_true_dims(c_hat_drop: np.ndarray, c_true_drop: np.ndarray, keep: np.ndarray) -> np.ndarray:
+    """Dropped dims of every token: the stored true values where keep[t], the
+    predicted ones elsewhere.  Rows of c_true_drop outside `keep` are never read."""
+    out = np.array(c_hat_drop, dtype=np.float64, copy=True)
+    keep = np.asarray(keep, dtype=bool)
+    out[keep] = np.asarray(c_true_drop, dtype=np.float64)[keep]
+    return out
+
+
+def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n_kv_heads: int,
+                              k_true_drop, v_true_drop, n_sink: int, n_window: int,
+                              scale: float | None = None, bk=None, bv=None) -> np.ndarray:
+    """decode_attention with the sink and recent-window tokens at full precision:
+    for those tokens the dropped dims come from k_true_drop / v_true_drop ([L, D - m],
+    the layer's own dims m..D-1), for all others from Eq. 3.  Returns [H_q, d]."""
+    q = np.asarray(q, dtype=np.float64)
+    d = q.shape[1]
+    L = np.asarray(k_global).shape[0]
+    if L < 1:
+        raise ValueError("empty cache: softmax over no token is undefined")
+    keep = full_precision_tokens(L, n_sink, n_window)
+    k_drop = overlay_true_dims(reconstruct_dropped(Wk, k_global, k_local, bk), k_true_drop, keep)
+    v_drop = overlay_true_dims(reconstruct_dropped(Wv, v_global, v_local, bv), v_true_drop, keep)
+    return attention(q, assemble_cache(k_local, k_drop, n_kv_heads, d),
+                     assemble_cache(v_local, v_drop, n_kv_heads, d), scale)
 
 
 # ----------------------------------------------------------------------------

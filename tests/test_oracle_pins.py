@@ -414,3 +414,95 @@ def test_planted_mistakes_are_caught(monkeypatch):
     _expect_caught(monkeypatch, "attention_probabilities", wrong_group, pins)
     _expect_caught(monkeypatch, "reconstruct_dropped", dropped_local_block, pins)
     _expect_caught(monkeypatch, "reconstruct_dropped", transposed_square_W, pins)
+
+
+# --------------------------------------------------------------------------
+# Sink and recent-window tokens at full precision (Section 5.1)
+# --------------------------------------------------------------------------
+def true_dropped(c, seed):
+    """A layer's own dims m..D-1 (what the predictor stands in for), unrelated to W on purpose."""
+    rng = np.random.default_rng(1000 + seed)
+    return rng.standard_normal((c["L"], c["D"] - c["m"])), rng.standard_normal((c["L"], c["D"] - c["m"]))
+
+
+def run_windowed(c, kt, vt, n_sink, n_window, scale=None):
+    return O.decode_attention_windowed(c["q"], c["kg"], c["vg"], c["kl"], c["vl"], c["Wk"], c["Wv"], c["H_kv"],
+                                       kt, vt, n_sink, n_window, scale)
+
+
+def brute_force_windowed(c, kt, vt, n_sink, n_window):
+    """Index by index: a sink / window token reads its stored dims, any other token the predicted ones."""
+    q, kg, vg, kl, vl, Wk, Wv = (c[k].tolist() for k in ("q", "kg", "vg", "kl", "vl", "Wk", "Wv"))
+    H_q, H_kv, d, m, D, L = c["H_q"], c["H_kv"], c["d"], c["m"], c["D"], c["L"]
+    grp = H_q // H_kv
+
+    def value(glob, loc, W, true, t, flat):
+        if flat < m:
+            return loc[t][flat]
+        if t < n_sink or t > L - 1 - n_window:
+            return true[t][flat - m]
+        row = W[flat - m]
+        return math.fsum([row[i] * glob[t][i] for i in range(D)] + [row[D + i] * loc[t][i] for i in range(m)])
+    out = []
+    for h in range(H_q):
+        kv = h // grp
+        s = [math.fsum(q[h][j] * value(kg, kl, Wk, kt.tolist(), t, kv * d + j) for j in range(d)) / math.sqrt(d)
+             for t in range(L)]
+        mx = max(s)
+        e = [math.exp(v - mx) for v in s]
+        z = math.fsum(e)
+        out.append([math.fsum(e[t] / z * value(vg, vl, Wv, vt.tolist(), t, kv * d + j) for t in range(L))
+                    for j in range(d)])
+    return np.array(out)
+
+
+@pytest.mark.parametrize("seed,L,H_q,H_kv,d,r,n_sink,n_window", [
+    (11, 9, 4, 2, 4, 1, 2, 3), (12, 7, 2, 2, 4, 0, 1, 0), (13, 8, 6, 3, 2, 2, 0, 2), (14, 5, 2, 2, 4, 1, 4, 4)])
+def test_windowed_brute_force_tiny(seed, L, H_q, H_kv, d, r, n_sink, n_window):
+    c = rand_case(seed, L, H_q, H_kv, d, r)
+    kt, vt = true_dropped(c, seed)
+    np.testing.assert_allclose(run_windowed(c, kt, vt, n_sink, n_window),
+                               brute_force_windowed(c, kt, vt, n_sink, n_window), rtol=1e-12, atol=1e-13)
+
+
+def test_windowed_limits():
+    c = rand_case(21, 10, 4, 2, 4, 1)
+    kt, vt = true_dropped(c, 21)
+    # no sink, no window: the plain method
+    np.testing.assert_array_equal(run_windowed(c, kt, vt, 0, 0), run(c))
+    # everything inside sink + window: standard attention on the layer's true cache (library routine)
+    K = np.concatenate([c["kl"], kt], axis=1).reshape(c["L"], c["H_kv"], c["d"])
+    V = np.concatenate([c["vl"], vt], axis=1).reshape(c["L"], c["H_kv"], c["d"])
+    for n_sink, n_window in ((4, 6), (0, 10), (10, 0), (3, 128)):
+        np.testing.assert_allclose(run_windowed(c, kt, vt, n_sink, n_window), sdpa(c["q"], K, V), rtol=1e-12, atol=1e-13)
+    # rows of the true dims outside sink / window are never read
+    poisoned_k, poisoned_v = kt.copy(), vt.copy()
+    poisoned_k[2:7] = np.nan
+    poisoned_v[2:7] = np.nan
+    np.testing.assert_array_equal(run_windowed(c, poisoned_k, poisoned_v, 2, 3), run_windowed(c, kt, vt, 2, 3))
+    # the per-head evaluation agrees
+    per = O.decode_attention_query_heads(c["q"], c["kg"], c["vg"], c["kl"], c["vl"], c["Wk"], c["Wv"], c["H_kv"],
+                                         range(c["H_q"]), k_true_drop=kt, v_true_drop=vt, n_sink=2, n_window=3)
+    full = run_windowed(c, kt, vt, 2, 3)
+    for h in range(c["H_q"]):
+        np.testing.assert_allclose(per[h], full[h], rtol=1e-12, atol=1e-14)
+
+
+def test_windowed_planted_mistakes_are_caught(monkeypatch):
+    good = O.full_precision_tokens
+
+    def window_at_the_front(L, n_sink, n_window):               # the window must be the LAST tokens
+        t = np.arange(L)
+        return (t < n_sink) | ((t >= n_sink) & (t < n_sink + n_window))
+
+    def off_by_one(L, n_sink, n_window):
+        t = np.arange(L)
+        return (t < n_sink) | (t > L - n_window)
+
+    def sink_forgotten(L, n_sink, n_window):
+        return good(L, 0, n_window)
+
+    pins = [lambda: test_windowed_brute_force_tiny(11, 9, 4, 2, 4, 1, 2, 3),
+            lambda: test_windowed_brute_force_tiny(13, 8, 6, 3, 2, 2, 0, 2)]
+    for bad in (window_at_the_front, off_by_one, sink_forgotten):
+        _expect_caught(monkeypatch, "full_precision_tokens", bad, pins)
