@@ -176,6 +176,25 @@ int echokv_decode_path(const echokv_ctx* ctx);
  * the fastest family their shape allows.  Meant for tests that check all against the oracle. */
 int echokv_set_decode_path(echokv_ctx* ctx, int path);
 
+/* Sink and recent-window tokens at full precision (Section 5.1, "Implement details": the paper keeps
+ * 4 sink tokens and a local window of 128 tokens uncompressed).  With (n_sink, n_window) set, the first
+ * n_sink and the last n_window tokens of every sequence are never predicted: the dims m .. D-1 of those
+ * tokens are kept in per-layer side buffers and Eq. 7 uses them as stored; every other token is
+ * reconstructed by Eq. 3 as before.
+ *  - echokv_side_buffer_bytes: size of ONE side buffer: [max_batch][n_sink + n_window][D - m] elements
+ *    of the storage dtype.  EUNSUPPORTED if n_sink + n_window > 4096.
+ *  - echokv_set_full_precision_window: k_side / v_side are host arrays [n_layers] of device pointers
+ *    (16-byte aligned, borrowed; entries of anchor layers are ignored and may be NULL).  From then on
+ *    echokv_append_kv on a compressed layer also writes the new token's dims m .. D-1 to the side buffers
+ *    (slot `position` while position < n_sink, and ring slot n_sink + position % n_window), and
+ *    echokv_decode_attention attends the sink / window tokens from there.  Set it before the first
+ *    append, or fill the slots of the tokens already cached yourself.  (0, 0) switches it off.
+ *    Not available together with the absorbed mode (echokv_decode_attention returns EUNSUPPORTED).
+ *    Errors: EINVAL, EUNSUPPORTED. */
+int echokv_side_buffer_bytes(const echokv_config* cfg, int n_sink, int n_window, uint64_t* out);
+int echokv_set_full_precision_window(echokv_ctx* ctx, int n_sink, int n_window, void* const* k_side,
+                                     void* const* v_side);
+
 /* Absorbed-predictor decode mode.  Eq. 3 is linear, so Eq. 7 over a predicted head can be evaluated
  * without forming the predicted K and V:
  *     q . (Wk x_t) = (Wk^T q) . x_t          sum_t p_t (Wv x_t) = Wv (sum_t p_t x_t)

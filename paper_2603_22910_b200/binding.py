@@ -59,6 +59,9 @@ EXPORTS = {
     "echokv_launch_count": (C.c_int64, [C.c_void_p]),
     "echokv_decode_path": (C.c_int, [C.c_void_p]),
     "echokv_set_decode_path": (C.c_int, [C.c_void_p, C.c_int]),
+    "echokv_side_buffer_bytes": (C.c_int, [C.POINTER(echokv_config), C.c_int, C.c_int, C.POINTER(C.c_uint64)]),
+    "echokv_set_full_precision_window": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p),
+                                                   C.POINTER(C.c_void_p)]),
     "echokv_absorbed_workspace_bytes": (C.c_int, [C.POINTER(echokv_config), C.POINTER(C.c_uint64)]),
     "echokv_enable_absorbed": (C.c_int, [C.c_void_p, C.c_void_p, C.c_uint64]),
     "echokv_decode_mode": (C.c_int, [C.c_void_p]),
@@ -233,6 +236,27 @@ class Context:
 
     def set_decode_path(self, path: int) -> None:
         _check(lib().echokv_set_decode_path(self.handle, path), "echokv_set_decode_path")
+
+    def set_full_precision_window(self, n_sink: int, n_window: int) -> None:
+        """Keep the first n_sink and the last n_window tokens of every sequence uncompressed: allocates the
+        side buffers of the compressed layers ([max_batch][n_sink + n_window][D - m]) and hands them over."""
+        cfg, n = self.cfg, self.cfg.n_layers
+        self.k_side, self.v_side = [], []
+        for l in range(n):
+            if l % cfg.group_size == 0 or self.D == self.m or n_sink + n_window == 0:
+                self.k_side.append(None)
+                self.v_side.append(None)
+            else:
+                shape = (cfg.max_batch, n_sink + n_window, self.D - self.m)
+                self.k_side.append(self.torch.zeros(shape, dtype=self.tdtype, device=self.device))
+                self.v_side.append(self.torch.zeros(shape, dtype=self.tdtype, device=self.device))
+        self._ks = (C.c_void_p * n)(*[_ptr(t) for t in self.k_side])
+        self._vs = (C.c_void_p * n)(*[_ptr(t) for t in self.v_side])
+        _check(lib().echokv_set_full_precision_window(self.handle, n_sink, n_window,
+                                                      C.cast(self._ks, C.POINTER(C.c_void_p)),
+                                                      C.cast(self._vs, C.POINTER(C.c_void_p))),
+               "echokv_set_full_precision_window")
+        self.n_sink, self.n_window = n_sink, n_window
 
     def enable_absorbed(self) -> None:
         """Allocate the absorbed mode's workspace and switch the context to that mode."""

@@ -46,7 +46,7 @@ int derive(const echokv_config* c, Derived* d) {
   d->elem = c->dtype == ECHOKV_BF16 ? 2 : 4;
   d->part_tokens = (c->dtype == ECHOKV_BF16 && c->head_dim == 128) ? kPairPartTokens : kSimtTileTokens;
   d->capacity = (int)cap;
-  d->max_parts = (d->capacity + d->part_tokens - 1) / d->part_tokens;
+  d->max_parts = (d->capacity + d->part_tokens - 1) / d->part_tokens + 1;   // + the sink / window partial
   uint64_t off = 0;
   d->off_status = off; off += kAlign;
   const uint64_t n_part = (uint64_t)c->max_batch * c->n_q_heads * d->max_parts;
@@ -72,6 +72,8 @@ struct Layer {
   const void* bk = nullptr;
   const void* bv = nullptr;
   bool anchor = false;
+  void* k_side = nullptr;   // dropped dims of the sink and recent-window tokens (compressed layers)
+  void* v_side = nullptr;
   TcLayerMaps tc;     // tensor maps of the tensor-core path (valid when tc.ready)
   CUtensorMap stored_k, stored_v;   // tensor maps of the stored-head kernel (valid when ctx.stored_path == 1)
 };
@@ -87,6 +89,7 @@ struct echokv_ctx {
   int sm_count = 0;
   int path = 0;          // see echokv_decode_path
   bool tc_capable = false;
+  int n_sink = 0, n_window = 0;   // tokens kept at full precision (0, 0 = none)
   bool absorbed_capable = false;  // shape served by the absorbed-predictor kernels
   int decode_mode = 0;            // 0 = explicit reconstruction (Eq. 3, 6, 7 as written), 1 = absorbed predictors
   unsigned char* ws_absorbed = nullptr;
@@ -194,6 +197,28 @@ bool timed_pair(echokv_ctx* c, int kind, cudaEvent_t* start, cudaEvent_t* stop) 
   *stop = c->events[c->timed].second;
   ++c->timed;
   return true;
+}
+
+bool side_active(const echokv_ctx* c, const Layer& L) {
+  return !L.anchor && c->d.d_drop > 0 && (c->n_sink > 0 || c->n_window > 0);
+}
+
+SideArgs side_args(const echokv_ctx* c, const Layer& L) {
+  SideArgs s;
+  s.k_side = L.k_side; s.v_side = L.v_side;
+  s.n_sink = c->n_sink; s.n_window = c->n_window; s.d_drop = c->d.d_drop;
+  return s;
+}
+
+// The new token's dropped dims of a compressed layer go to the side buffers while a sink / window is set.
+int append_side(echokv_ctx* c, const Layer& L, const void* k_new, const void* v_new, const int32_t* slots,
+                const int32_t* positions, int B, cudaStream_t s) {
+  if (!side_active(c, L)) return ECHOKV_OK;
+  if (launch_append_side(c->cfg.dtype, side_args(c, L), c->d.m, c->d.D, k_new, v_new, slots, positions, B,
+                         c->cfg.max_batch, status_ptr(c), s) != cudaSuccess)
+    return ECHOKV_ECUDA;
+  c->launches += 1;
+  return ECHOKV_OK;
 }
 
 int check_call(echokv_ctx* c, int layer, const void* q, const float* out, const int32_t* lens, int B) {
@@ -368,6 +393,39 @@ int echokv_set_decode_path(echokv_ctx* c, int path) {
   return ECHOKV_EINVAL;
 }
 
+int echokv_side_buffer_bytes(const echokv_config* cfg, int n_sink, int n_window, uint64_t* out) {
+  if (!out || n_sink < 0 || n_window < 0) return ECHOKV_EINVAL;
+  Derived d;
+  const int rc = derive(cfg, &d);
+  if (rc != ECHOKV_OK) return rc;
+  if (n_sink + n_window > 4096) return ECHOKV_EUNSUPPORTED;
+  *out = (uint64_t)cfg->max_batch * (uint64_t)(n_sink + n_window) * d.d_drop * d.elem;
+  return ECHOKV_OK;
+}
+
+int echokv_set_full_precision_window(echokv_ctx* c, int n_sink, int n_window, void* const* k_side,
+                                     void* const* v_side) {
+  if (!c || n_sink < 0 || n_window < 0) return ECHOKV_EINVAL;
+  if (n_sink + n_window > 4096) return ECHOKV_EUNSUPPORTED;
+  const bool on = (n_sink > 0 || n_window > 0) && c->d.d_drop > 0;
+  if (on) {
+    if (!k_side || !v_side) return ECHOKV_EINVAL;
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+      if (c->layers[l].anchor) continue;
+      if (!k_side[l] || !v_side[l]) return ECHOKV_EINVAL;
+      if ((reinterpret_cast<uintptr_t>(k_side[l]) | reinterpret_cast<uintptr_t>(v_side[l])) % 16 != 0)
+        return ECHOKV_EINVAL;
+    }
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+      c->layers[l].k_side = c->layers[l].anchor ? nullptr : k_side[l];
+      c->layers[l].v_side = c->layers[l].anchor ? nullptr : v_side[l];
+    }
+  }
+  c->n_sink = on ? n_sink : 0;
+  c->n_window = on ? n_window : 0;
+  return ECHOKV_OK;
+}
+
 int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out) {
   if (!out) return ECHOKV_EINVAL;
   Derived d;
@@ -425,13 +483,14 @@ int echokv_append_kv(echokv_ctx* c, int layer, const void* k_new, const void* v_
   if (!c->table) return ECHOKV_ENOTABLE;
   const Layer& L = c->layers[layer];
   const int width = L.anchor ? c->d.D : c->d.m;
-  if (width == 0) return ECHOKV_OK;   // nothing of this layer is kept (m = 0)
+  if (width == 0)                     // nothing of this layer is kept in the pools (m = 0)
+    return append_side(c, L, k_new, v_new, dev_seq_slots, dev_positions, B, static_cast<cudaStream_t>(stream));
   const cudaError_t e = launch_append(c->cfg.dtype, L.k_pool, L.v_pool, width, c->d.D, k_new, v_new,
                                       dev_seq_slots, dev_positions, B, geom_of(c), status_ptr(c),
                                       static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return ECHOKV_ECUDA;
   c->launches += 1;
-  return ECHOKV_OK;
+  return append_side(c, L, k_new, v_new, dev_seq_slots, dev_positions, B, static_cast<cudaStream_t>(stream));
 }
 
 int echokv_full_attention(echokv_ctx* c, int layer, const void* q, float* out,
@@ -457,6 +516,8 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   if (!L.Wk || !L.Wv) return ECHOKV_ENOWEIGHTS;
   const Layer& A = c->layers[layer - layer % c->cfg.group_size];
   AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
+  const bool side = side_active(c, L);
+  if (c->decode_mode == 1 && side) return ECHOKV_EUNSUPPORTED;   // (the absorbed mode has no sink / window yet)
   if (c->decode_mode == 1) {
     // absorbed predictors: every query head in one pass over [anchor dims ; retained dims]
     if (B > 256) return ECHOKV_EUNSUPPORTED;
@@ -488,6 +549,8 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   ra.D = c->d.D; ra.m = c->d.m;
   ra.part_tokens = c->d.part_tokens;
   ra.capacity_tokens = c->d.capacity;
+  ra.n_sink = side ? c->n_sink : 0;
+  ra.n_window = side ? c->n_window : 0;
   cudaError_t e;
   {
     ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
@@ -501,8 +564,13 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   }
   if (e != cudaSuccess) return ECHOKV_ECUDA;
   const int recon_part_tokens = c->path == 2 ? kTcPartTokens : c->d.part_tokens;
-  if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, recon_part_tokens, L.bv, s) !=
-      cudaSuccess)
+  if (side) {
+    // sink and recent-window tokens: Eq. 7 on their stored dims, one more partial per query head
+    if (launch_attn_side(a, side_args(c, L), r, recon_part_tokens, s) != cudaSuccess) return ECHOKV_ECUDA;
+    c->launches += 1;
+  }
+  if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, recon_part_tokens, L.bv, s,
+                   side ? 1 : 0) != cudaSuccess)
     return ECHOKV_ECUDA;
   c->launches += 2;
   return ECHOKV_OK;

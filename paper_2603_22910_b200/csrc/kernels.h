@@ -35,7 +35,37 @@ struct ReconArgs {
   int D, m;
   int part_tokens;                              // tokens per partial
   int capacity_tokens;                          // max_pages_per_seq * page_tokens
+  int n_sink = 0, n_window = 0;                 // tokens kept at full precision: the first n_sink and the last
+                                                // n_window of a sequence are NOT predicted here (they are
+                                                // attended from the side buffers, see launch_attn_side)
 };
+
+// Tokens of a sequence of `len` tokens that are predicted: [lo, hi) (Section 5.1: sink and recent-window
+// tokens keep all their dims).
+__host__ __device__ inline int predicted_lo(int len, int n_sink) { return n_sink < len ? n_sink : len; }
+__host__ __device__ inline int predicted_hi(int len, int n_sink, int n_window) {
+  const int lo = predicted_lo(len, n_sink);
+  const int hi = len - n_window;
+  return hi > lo ? hi : lo;
+}
+
+// Side buffers of one compressed layer: the dropped dims (m .. D-1) of the sink and recent-window tokens,
+// [max_batch][n_sink + n_window][D - m] in the storage dtype; slot of token t: t if t < n_sink, and
+// n_sink + t % n_window while it is inside the window.
+struct SideArgs {
+  void* k_side; void* v_side;
+  int n_sink, n_window, d_drop;
+};
+
+// Append: the new token's dropped dims go to its side slots.
+cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, const void* k_new, const void* v_new,
+                               const int32_t* slots, const int32_t* positions, int B, int max_batch,
+                               int32_t* status, cudaStream_t stream);
+
+// Eq. 7 over the sink and window tokens of the dropped heads, from the side buffers: one split-K partial per
+// (sequence, query head of a dropped KV head), written at partial index ceil(len / part_tokens).
+cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int n_ret_heads, int part_tokens,
+                             cudaStream_t stream);
 
 // CUDA-core reconstruct-then-attend (fp32 or bf16 storage, fp32 FFMA): Eq. 3, 6, 7 for the
 // dropped KV heads; one partial per part_tokens tokens.
@@ -48,6 +78,6 @@ cudaError_t launch_recon_simt(const AttnArgs& a, const ReconArgs& r, cudaStream_
 // on the fly, added to dropped heads ([D - m] in storage dtype).
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
                          const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-                         const void* bv, cudaStream_t stream);
+                         const void* bv, cudaStream_t stream, int extra_recon_part = 0);
 
 }  // namespace echokv

@@ -65,6 +65,7 @@ struct PairParams {
   int n_q_heads, n_ret_heads, n_drop_heads, n_pairs;
   int kc_anchor, kc_total;    // 64-feature chunks of the predictor input: from the anchor, in all
   int run_pages;              // pages per tall box (kRunTokens / page_tokens), 1 = no tall boxes
+  int n_sink, n_window;       // sink / recent-window tokens are not predicted (masked here)
   float scale_log2e;
 };
 
@@ -382,7 +383,9 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
         }
       }
       const int token = (int)rank * kCtaTokens + row;        // token of the tile
-      const bool tok_valid = token < n_valid;
+      // predicted tokens only: sink and recent-window tokens are attended from the side buffers
+      const int t_seq = w.tile * kTileTokens + token;
+      const bool tok_valid = t_seq >= predicted_lo(len, p.n_sink) && t_seq < predicted_hi(len, p.n_sink, p.n_window);
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) {
         if (!tok_valid) sc[gi] = -INFINITY;
@@ -561,6 +564,8 @@ cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLay
   p.kc_anchor = r.D / kChunk;
   p.kc_total = (r.D + r.m) / kChunk;
   p.scale_log2e = a.scale_log2e;
+  p.n_sink = r.n_sink;
+  p.n_window = r.n_window;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;

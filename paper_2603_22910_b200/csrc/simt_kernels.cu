@@ -376,7 +376,9 @@ __global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r
         float s = 0.f;
 #pragma unroll 8
         for (int j = 0; j < DH; ++j) s = fmaf(sm.qs[gi][j], sm.Hs[t][j], s);
-        sm.Ss[gi][t] = (tile_t0 + t < len) ? s : -INFINITY;
+        const int t_seq = tile_t0 + t;     // predicted tokens only (sink / window tokens come from the side buffers)
+        sm.Ss[gi][t] = (t_seq >= predicted_lo(len, r.n_sink) && t_seq < predicted_hi(len, r.n_sink, r.n_window))
+                           ? s : -INFINITY;
       }
     }
     __syncthreads();
@@ -386,8 +388,9 @@ __global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r
       const float mt = warp_max(fmaxf(s0, s1));
       const float m_old = sm.m_run[gi];
       const float m_new = fmaxf(m_old, mt);
-      const float alpha = exp2f(m_old - m_new);
-      const float p0 = exp2f(s0 - m_new), p1 = exp2f(s1 - m_new);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;     // nothing predicted so far: every p is 0
+      const float alpha = exp2f(m_old - m_use);
+      const float p0 = exp2f(s0 - m_use), p1 = exp2f(s1 - m_use);
       const float ls = warp_sum(p0 + p1);
       sm.Ss[gi][lane] = p0;
       sm.Ss[gi][lane + 32] = p1;
@@ -452,7 +455,7 @@ template <typename T>
 __global__ void __launch_bounds__(128 * kMergeGroups)
 merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stored_parts,
              const int32_t* __restrict__ stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-             const T* __restrict__ bv) {
+             const T* __restrict__ bv, int extra_recon_part) {
   const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x, grp = threadIdx.y;
   const int DH = a.head_dim;                      // == blockDim.x
   const int tid = grp * DH + j, n_threads = DH * kMergeGroups;
@@ -469,7 +472,7 @@ merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stor
   const bool stored = kvh < n_stored_heads;
   int n;
   if (!stored) {
-    n = (len + part_tokens - 1) / part_tokens;
+    n = (len + part_tokens - 1) / part_tokens + extra_recon_part;   // (+ the sink / window partial)
   } else if (stored_item_tokens != nullptr) {
     const int item_tokens = stored_item_tokens[b / stored_batch_per_slot];
     n = (len + item_tokens - 1) / item_tokens;
@@ -518,18 +521,190 @@ merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stor
 
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
                          const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-                         const void* bv, cudaStream_t stream) {
+                         const void* bv, cudaStream_t stream, int extra_recon_part) {
   dim3 grid(a.n_q_heads, a.batch);
   if (a.dtype == ECHOKV_BF16) {
     merge_kernel<__nv_bfloat16><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(
         a, out, n_stored_heads, n_stored_parts, stored_item_tokens, stored_batch_per_slot, part_tokens,
-        (const __nv_bfloat16*)bv);
+        (const __nv_bfloat16*)bv, extra_recon_part);
   } else {
     merge_kernel<float><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(a, out, n_stored_heads, n_stored_parts,
                                                          stored_item_tokens, stored_batch_per_slot,
-                                                         part_tokens, (const float*)bv);
+                                                         part_tokens, (const float*)bv, extra_recon_part);
   }
   return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sink and recent-window tokens at full precision (Section 5.1): their dropped dims live in small
+// side buffers; these two kernels write and attend them.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) append_side_kernel(T* __restrict__ k_side, T* __restrict__ v_side, int n_sink,
+                                                          int n_window, int d_drop, int m, int D,
+                                                          const T* __restrict__ k_new, const T* __restrict__ v_new,
+                                                          const int32_t* __restrict__ slots,
+                                                          const int32_t* __restrict__ positions, int max_batch,
+                                                          int32_t* status) {
+  const int b = blockIdx.x;
+  const int slot = slots ? slots[b] : b;
+  const int pos = positions[b];
+  if (slot < 0 || slot >= max_batch || pos < 0) {
+    if (threadIdx.x == 0) report(status, ECHOKV_EBADPAGE);
+    return;
+  }
+  constexpr int kVec = 16 / sizeof(T);
+  const int n_vec = d_drop / kVec;
+  const uint4* ks = reinterpret_cast<const uint4*>(k_new + (size_t)b * D + m);
+  const uint4* vs = reinterpret_cast<const uint4*>(v_new + (size_t)b * D + m);
+  const size_t seq_base = (size_t)slot * (n_sink + n_window);
+  // a token inside the sink is written there; every token also enters the window ring
+  for (int which = 0; which < 2; ++which) {
+    int idx;
+    if (which == 0) { if (pos >= n_sink) continue; idx = pos; }
+    else { if (n_window == 0) continue; idx = n_sink + pos % n_window; }
+    uint4* kd = reinterpret_cast<uint4*>(k_side + (seq_base + idx) * d_drop);
+    uint4* vd = reinterpret_cast<uint4*>(v_side + (seq_base + idx) * d_drop);
+    for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
+      kd[i] = ks[i];
+      vd[i] = vs[i];
+    }
+  }
+}
+
+cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, const void* k_new, const void* v_new,
+                               const int32_t* slots, const int32_t* positions, int B, int max_batch,
+                               int32_t* status, cudaStream_t stream) {
+  if (dtype == ECHOKV_BF16) {
+    append_side_kernel<__nv_bfloat16><<<B, 128, 0, stream>>>(
+        (__nv_bfloat16*)side.k_side, (__nv_bfloat16*)side.v_side, side.n_sink, side.n_window, side.d_drop, m, D,
+        (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, slots, positions, max_batch, status);
+  } else {
+    append_side_kernel<float><<<B, 128, 0, stream>>>((float*)side.k_side, (float*)side.v_side, side.n_sink,
+                                                     side.n_window, side.d_drop, m, D, (const float*)k_new,
+                                                     (const float*)v_new, slots, positions, max_batch, status);
+  }
+  return cudaGetLastError();
+}
+
+// One block per (dropped KV head, sequence): scores of the <= n_sink + n_window full-precision tokens against
+// the group's query heads, softmax, weighted V; one partial per query head.
+template <typename T, int DH>
+__global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __restrict__ k_side,
+                                                        const T* __restrict__ v_side, int n_sink, int n_window,
+                                                        int d_drop, int n_ret, int part_tokens) {
+  extern __shared__ float side_smem[];
+  const int dh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = a.n_q_heads / a.n_kv_heads;
+  const int kvh = n_ret + dh;
+  const int n_side = n_sink + n_window;
+  float* qs = side_smem;                      // [g][DH]
+  float* sc = qs + kMaxGroup * DH;            // [g][n_side]
+  __shared__ float red[4][kMaxGroup];
+  __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
+  const int slot = a.slots ? a.slots[b] : b;
+  const int len = a.lens[b];
+  if (slot < 0 || slot >= a.geom.max_batch || len < 1 ||
+      len > a.geom.max_pages_per_seq * a.geom.page_tokens)
+    return;                                    // (reported by the other kernels of the call; merge writes zeros)
+  const int lo = predicted_lo(len, n_sink), hi = predicted_hi(len, n_sink, n_window);
+  const int n_tok = lo + (len - hi);          // sink tokens [0, lo) then window tokens [hi, len)
+  const T* q = reinterpret_cast<const T*>(a.q);
+  for (int idx = tid; idx < g * DH; idx += 128)
+    qs[idx] = to_f32(q[((size_t)b * a.n_q_heads + kvh * g) * DH + idx]) * a.scale_log2e;
+  __syncthreads();
+  const size_t seq_base = (size_t)slot * n_side;
+  auto side_row = [&](int i) {                 // i-th full-precision token -> row of the side buffers
+    const int t = i < lo ? i : hi + (i - lo);
+    return (seq_base + (t < lo ? t : n_sink + t % n_window)) * (size_t)d_drop + (size_t)dh * DH;
+  };
+  // scores: one token per thread
+  for (int i = tid; i < n_tok; i += 128) {
+    const T* kr = k_side + side_row(i);
+    float acc[kMaxGroup];
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
+    for (int j = 0; j < DH; j += Vec16<T>::N) {
+      float kv[Vec16<T>::N];
+      Vec16<T>::load(kr + j, kv);
+#pragma unroll
+      for (int gi = 0; gi < kMaxGroup; ++gi)
+        if (gi < g) {
+#pragma unroll
+          for (int e = 0; e < Vec16<T>::N; ++e) acc[gi] = fmaf(kv[e], qs[gi * DH + j + e], acc[gi]);
+        }
+    }
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi)
+      if (gi < g) sc[gi * n_side + i] = acc[gi];
+  }
+  __syncthreads();
+  // max and sum per query head
+  for (int gi = 0; gi < g; ++gi) {
+    float m = -INFINITY;
+    for (int i = tid; i < n_tok; i += 128) m = fmaxf(m, sc[gi * n_side + i]);
+    m = warp_max(m);
+    if (lane == 0) red[warp][gi] = m;
+  }
+  __syncthreads();
+  if (tid < g) s_m[tid] = fmaxf(fmaxf(red[0][tid], red[1][tid]), fmaxf(red[2][tid], red[3][tid]));
+  __syncthreads();
+  for (int gi = 0; gi < g; ++gi) {
+    const float M = s_m[gi];
+    float l = 0.f;
+    for (int i = tid; i < n_tok; i += 128) {
+      const float pv = exp2f(sc[gi * n_side + i] - M);
+      sc[gi * n_side + i] = pv;
+      l += pv;
+    }
+    l = warp_sum(l);
+    if (lane == 0) red[warp][gi] = l;
+  }
+  __syncthreads();
+  if (tid < g) s_l[tid] = (red[0][tid] + red[1][tid]) + (red[2][tid] + red[3][tid]);
+  __syncthreads();
+  // weighted V: one output feature per thread
+  const int part = (len + part_tokens - 1) / part_tokens;
+  if (tid < DH) {
+    float o[kMaxGroup];
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
+    for (int i = 0; i < n_tok; ++i) {
+      const float vv = to_f32(v_side[side_row(i) + tid]);
+#pragma unroll
+      for (int gi = 0; gi < kMaxGroup; ++gi)
+        if (gi < g) o[gi] = fmaf(sc[gi * n_side + i], vv, o[gi]);
+    }
+    for (int gi = 0; gi < g; ++gi) {
+      const size_t pidx = ((size_t)b * a.n_q_heads + kvh * g + gi) * a.parts.max_parts + part;
+      a.parts.o[pidx * DH + tid] = o[gi];
+      if (tid == 0) a.parts.ml[pidx] = make_float2(s_m[gi], s_l[gi]);
+    }
+  }
+}
+
+template <typename T, int DH>
+static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, int n_ret, int part_tokens,
+                                      cudaStream_t stream) {
+  const int n_drop = a.n_kv_heads - n_ret;
+  const int n_side = side.n_sink + side.n_window;
+  const size_t smem = (size_t)(kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(attn_side_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(n_drop, a.batch);
+  attn_side_kernel<T, DH><<<grid, 128, smem, stream>>>(a, (const T*)side.k_side, (const T*)side.v_side, side.n_sink,
+                                                       side.n_window, side.d_drop, n_ret, part_tokens);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int n_ret_heads, int part_tokens,
+                             cudaStream_t stream) {
+  if (a.dtype == ECHOKV_BF16) {
+    if (a.head_dim == 128) return launch_attn_side_t<__nv_bfloat16, 128>(a, side, n_ret_heads, part_tokens, stream);
+    return launch_attn_side_t<__nv_bfloat16, 64>(a, side, n_ret_heads, part_tokens, stream);
+  }
+  if (a.head_dim == 128) return launch_attn_side_t<float, 128>(a, side, n_ret_heads, part_tokens, stream);
+  return launch_attn_side_t<float, 64>(a, side, n_ret_heads, part_tokens, stream);
 }
 
 }  // namespace echokv

@@ -16,7 +16,8 @@ class Case:
     """One workload resident on the GPU (all layers), plus the host copies the oracle reads."""
 
     def __init__(self, w: synth.Workload, lens=None, n_pages=None, layers=None, keep_host=True,
-                 biases=False):
+                 biases=False, window=None):
+        """window = (n_sink, n_window): those tokens of every sequence keep all their dims (Section 5.1)."""
         self.w = w
         self.lens = list(lens) if lens is not None else [w.context] * w.batch
         assert len(self.lens) == w.batch and max(self.lens) <= w.context
@@ -26,6 +27,10 @@ class Case:
         self.table = synth.block_table(w, n_pages)
         self.ctx.set_block_table(self.table)
         self.layers = list(range(w.n_layers)) if layers is None else layers
+        self.window = window
+        if window:
+            self.ctx.set_full_precision_window(*window)
+        self.true_drop = {}  # (layer, kind, b) -> the layer's own dims m..D-1 [len_b, D - m] (window tests)
         self.host = {}       # (layer, kind, b) -> stored-precision tensor [len_b, width]
         self.weights = {}    # layer -> (Wk, Wv, bk, bv) device tensors
         self.host_w = {}
@@ -50,6 +55,21 @@ class Case:
                     newest[b, :width] = seqs[b][-1]
                     if width < w.D:
                         newest[b, width:] = 777.0   # must never reach the cache
+                if window and not w.is_anchor(l) and w.D > w.m:
+                    # the sink / window tokens' own dims m..D-1: all but the newest are placed in the side
+                    # buffers here, the newest goes through the library's append
+                    n_sink, n_window = window
+                    side = (self.ctx.k_side if kind == "k" else self.ctx.v_side)[l]
+                    for b in range(w.batch):
+                        L = self.lens[b]
+                        full = synth.layer_cache(w, l, kind, b, width=w.D)[:L]
+                        self.true_drop[(l, kind, b)] = full[:, w.m:]
+                        newest[b, w.m:] = full[-1, w.m:]
+                        for t in range(L - 1):
+                            if t < n_sink:
+                                side[b, t] = full[t, w.m:].to(dev)
+                            if n_window and t >= L - 1 - n_window:      # still inside the ring after the append
+                                side[b, n_sink + t % n_window] = full[t, w.m:].to(dev)
                 self.host[(l, kind, "new")] = newest
             if not w.is_anchor(l):
                 Wk = synth.predictor_weights(w, l, "k")
@@ -103,7 +123,13 @@ class Case:
             vl = self._stored(layer, "v", b) if w.m else np.zeros((L, 0))
             Wk, Wv, bk, bv = (None if t is None else O.widen(synth.to_numpy_stored(t))
                               for t in self.host_w[layer])
-            if query_heads is None:
+            if self.window and w.D > w.m:
+                kt = O.widen(synth.to_numpy_stored(self.true_drop[(layer, "k", b)]))
+                vt = O.widen(synth.to_numpy_stored(self.true_drop[(layer, "v", b)]))
+                assert query_heads is None
+                res[b] = O.decode_attention_windowed(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, kt, vt,
+                                                     self.window[0], self.window[1], bk=bk, bv=bv)
+            elif query_heads is None:
                 res[b] = O.decode_attention(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv)
             else:
                 per = O.decode_attention_query_heads(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, query_heads)

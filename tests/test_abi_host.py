@@ -40,12 +40,12 @@ def test_query_sizes_c1(lib):
     assert s.anchor_pool_bytes == rows * w.D * 2
     assert s.compressed_pool_bytes == rows * w.m * 2
     assert s.block_table_bytes == w.batch * w.pages_per_seq * 4
-    assert s.max_partials == w.context // 128      # one partial per 128 tokens (CTA-pair kernel)
+    assert s.max_partials == w.context // 128 + 1  # one partial per 128 tokens, one for sink / window tokens
     part = w.batch * w.n_q_heads * s.max_partials
     assert s.workspace_bytes >= part * (8 + 4 * w.head_dim)
     w0 = synth.C0
     s0 = binding.echokv_query_sizes(binding.config_for(w0))
-    assert s0.max_partials == w0.context // 64
+    assert s0.max_partials == w0.context // 64 + 1
     assert s0.anchor_pool_bytes == w0.context * w0.D * 4
 
 
