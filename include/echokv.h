@@ -189,8 +189,7 @@ int echokv_set_decode_path(echokv_ctx* ctx, int path);
  *    (slot `position` while position < n_sink, and ring slot n_sink + position % n_window), and
  *    echokv_decode_attention attends the sink / window tokens from there.  Set it before the first
  *    append, or fill the slots of the tokens already cached yourself.  (0, 0) switches it off.
- *    Not available together with the absorbed mode (echokv_decode_attention returns EUNSUPPORTED).
- *    Errors: EINVAL, EUNSUPPORTED. */
+ *    Works in both decode modes.  Errors: EINVAL, EUNSUPPORTED. */
 int echokv_side_buffer_bytes(const echokv_config* cfg, int n_sink, int n_window, uint64_t* out);
 int echokv_set_full_precision_window(echokv_ctx* ctx, int n_sink, int n_window, void* const* k_side,
                                      void* const* v_side);

@@ -170,6 +170,7 @@ struct StreamParams {
   int range_tokens;             // pv kernel: tokens per range
   int n_slices;                 // pv kernel: 256-feature slices
   int v_tile_ok;                // pv kernel: the 4-chunk V maps exist for (anchor, local)
+  int n_sink, n_window;         // scores kernel: sink / recent-window tokens are left to the side kernel
 };
 
 struct StreamSmemTail {
@@ -400,7 +401,7 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
       if (!epi_all(mbar_wait(smem_u32(&t.acc_full_bar[buf]), (n >> 1) & 1u, abort_flag, p.status))) break;
       tc_fence_after();
       const int token = tile * kScoreTokens + row;
-      const bool valid = token < len;
+      const bool valid = token >= predicted_lo(len, p.n_sink) && token < predicted_hi(len, p.n_sink, p.n_window);
       const uint32_t addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 128u;
       float* dst = p.s_out + (size_t)b * p.n_q_heads * p.l_cap + token;
       for (int hb = 0; hb < p.n_q_heads; hb += 16) {
@@ -459,6 +460,8 @@ absorb_softmax_kernel(const float* __restrict__ S, __nv_bfloat16* __restrict__ p
 #pragma unroll
   for (int w = 1; w < 8; ++w) M = fmaxf(M, red[w]);
   __syncthreads();
+  const float M_out = M;
+  if (M == -INFINITY) M = 0.f;     // every token is a sink / window token: all probabilities are 0 here
   const int nh2 = 2 * n_q_heads;
   __nv_bfloat16* hi = p2 + ((size_t)b * nh2 + h) * l_cap;
   __nv_bfloat16* lo = p2 + ((size_t)b * nh2 + n_q_heads + h) * l_cap;
@@ -485,7 +488,7 @@ absorb_softmax_kernel(const float* __restrict__ S, __nv_bfloat16* __restrict__ p
     float tot = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
-    ml[(size_t)b * n_q_heads + h] = make_float2(M, tot);
+    ml[(size_t)b * n_q_heads + h] = make_float2(M_out, tot);
   }
 }
 
@@ -797,6 +800,23 @@ absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restric
   }
 }
 
+// out[b][h][:] holds the normalised result over the predicted tokens, ml[b][h] its (max, sum); parts hold the
+// partial over the sink / window tokens at index 0.  Combine the two by log-sum-exp.
+__global__ void __launch_bounds__(128)
+absorb_combine_kernel(float* __restrict__ out, const float2* __restrict__ ml, Partials parts, int n_q_heads) {
+  const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
+  const size_t bh = (size_t)b * n_q_heads + h;
+  const float2 mid = ml[bh];
+  const float2 side = parts.ml[bh * parts.max_parts];
+  const float M = fmaxf(mid.x, side.x);
+  if (M == -INFINITY) return;      // (an unusable sequence: zeros were written already)
+  const float w_mid = mid.y > 0.f ? exp2f(mid.x - M) * mid.y : 0.f;      // weight of the normalised mid result
+  const float w_side = exp2f(side.x - M);
+  const float denom = w_mid + w_side * side.y;
+  const float o_side = parts.o[bh * parts.max_parts * 128 + j];
+  out[bh * 128 + j] = denom > 0.f ? (w_mid * out[bh * 128 + j] + w_side * o_side) / denom : 0.f;
+}
+
 int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
 }  // namespace
@@ -876,6 +896,8 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   p.kc_total = d_in / kChunk;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   p.l_cap = lay.l_cap;
+  p.n_sink = r.n_sink;
+  p.n_window = r.n_window;
   p.s_out = S;
   p.y_out = y;
   p.d_in = d_in;
@@ -954,6 +976,19 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     absorb_out_kernel<<<grid2, 256, 0, stream>>>(ysum, reinterpret_cast<const __nv_bfloat16*>(r.Wv),
                                                  reinterpret_cast<const __nv_bfloat16*>(r.bv), out, a.batch,
                                                  a.n_q_heads, g, n_ret, r.D, d_in);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  // 6. sink and recent-window tokens (Section 5.1): attended at full precision by the side kernel, then
+  //    combined with the result over the predicted tokens
+  if (r.n_sink > 0 || r.n_window > 0) {
+    SideArgs side;
+    side.k_side = r.k_side; side.v_side = r.v_side;
+    side.n_sink = r.n_sink; side.n_window = r.n_window; side.d_drop = r.D - r.m;
+    SidePool pool;
+    pool.k_pool = r.k_local; pool.v_pool = r.v_local; pool.width = r.m; pool.part = 0;
+    if ((e = launch_attn_side(a, side, n_ret, 1, stream, &pool)) != cudaSuccess) return e;
+    dim3 grid(a.n_q_heads, a.batch);
+    absorb_combine_kernel<<<grid, 128, 0, stream>>>(out, ml, a.parts, a.n_q_heads);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;

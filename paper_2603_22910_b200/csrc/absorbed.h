@@ -45,6 +45,9 @@ struct AbsorbArgs {
   const void* Wk; const void* Wv; const void* bv;     // predictors of the layer ([D - m][D + m]), V bias or null
   int D, m;
   int capacity_tokens;
+  int n_sink = 0, n_window = 0; // sink / recent-window tokens kept at full precision (0, 0 = none) ...
+  void* k_side = nullptr; void* v_side = nullptr;            // ... their dropped dims (side buffers of the layer)
+  const void* k_local = nullptr; const void* v_local = nullptr;   // ... and the layer's pools (retained dims)
   double* kernel_ms;            // unused
 };
 

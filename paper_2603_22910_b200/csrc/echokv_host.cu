@@ -517,7 +517,6 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   const Layer& A = c->layers[layer - layer % c->cfg.group_size];
   AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
   const bool side = side_active(c, L);
-  if (c->decode_mode == 1 && side) return ECHOKV_EUNSUPPORTED;   // (the absorbed mode has no sink / window yet)
   if (c->decode_mode == 1) {
     // absorbed predictors: every query head in one pass over [anchor dims ; retained dims]
     if (B > 256) return ECHOKV_EUNSUPPORTED;
@@ -528,12 +527,17 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     aa.D = c->d.D; aa.m = c->d.m;
     aa.capacity_tokens = c->d.capacity;
     aa.kernel_ms = nullptr;
+    if (side) {
+      aa.n_sink = c->n_sink; aa.n_window = c->n_window;
+      aa.k_side = L.k_side; aa.v_side = L.v_side;
+      aa.k_local = L.k_pool; aa.v_local = L.v_pool;
+    }
     cudaEvent_t ev[4];
     const bool timed = timed_pair(c, ECHOKV_TIMED_ABSORB_K, &ev[0], &ev[1]) &&
                        timed_pair(c, ECHOKV_TIMED_ABSORB_V, &ev[2], &ev[3]);
     if (launch_absorbed(a, aa, c->amaps, A.tc, L.tc, out, c->sm_count, s, timed ? ev : nullptr) != cudaSuccess)
       return ECHOKV_ECUDA;
-    c->launches += 6;
+    c->launches += side ? 8 : 6;
     return ECHOKV_OK;
   }
   const int r = c->cfg.n_retained_heads;

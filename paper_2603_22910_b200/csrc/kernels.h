@@ -64,8 +64,15 @@ cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, co
 
 // Eq. 7 over the sink and window tokens of the dropped heads, from the side buffers: one split-K partial per
 // (sequence, query head of a dropped KV head), written at partial index ceil(len / part_tokens).
+// With `pool` given (the absorbed mode), the retained heads are covered too, from their stored dims in the
+// layer's pool, and every partial goes to index pool->part.
+struct SidePool {
+  const void* k_pool; const void* v_pool;   // the layer's pools (row width `width` = m)
+  int width;
+  int part;
+};
 cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int n_ret_heads, int part_tokens,
-                             cudaStream_t stream);
+                             cudaStream_t stream, const SidePool* pool = nullptr);
 
 // CUDA-core reconstruct-then-attend (fp32 or bf16 storage, fp32 FFMA): Eq. 3, 6, 7 for the
 // dropped KV heads; one partial per part_tokens tokens.

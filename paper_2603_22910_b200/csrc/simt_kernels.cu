@@ -587,16 +587,21 @@ cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, co
   return cudaGetLastError();
 }
 
-// One block per (dropped KV head, sequence): scores of the <= n_sink + n_window full-precision tokens against
-// the group's query heads, softmax, weighted V; one partial per query head.
+// One block per (KV head, sequence): scores of the <= n_sink + n_window full-precision tokens against the
+// group's query heads, softmax, weighted V; one partial per query head.  A dropped head reads the side
+// buffers; a retained head (only asked for by the absorbed mode, first_head = 0) reads its stored dims
+// from the layer's pool.  The partial goes to index fixed_part, or ceil(len / part_tokens) if that is < 0.
 template <typename T, int DH>
 __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __restrict__ k_side,
                                                         const T* __restrict__ v_side, int n_sink, int n_window,
-                                                        int d_drop, int n_ret, int part_tokens) {
+                                                        int d_drop, int n_ret, int part_tokens, int first_head,
+                                                        int fixed_part, const T* __restrict__ k_pool,
+                                                        const T* __restrict__ v_pool, int pool_width) {
   extern __shared__ float side_smem[];
-  const int dh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = a.n_q_heads / a.n_kv_heads;
-  const int kvh = n_ret + dh;
+  const int kvh = first_head + blockIdx.x;
+  const int dh = kvh - n_ret;                  // index among the dropped heads (< 0: a retained head)
   const int n_side = n_sink + n_window;
   float* qs = side_smem;                      // [g][DH]
   float* sc = qs + kMaxGroup * DH;            // [g][n_side]
@@ -614,13 +619,22 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     qs[idx] = to_f32(q[((size_t)b * a.n_q_heads + kvh * g) * DH + idx]) * a.scale_log2e;
   __syncthreads();
   const size_t seq_base = (size_t)slot * n_side;
-  auto side_row = [&](int i) {                 // i-th full-precision token -> row of the side buffers
+  const T* k_src = dh >= 0 ? k_side : k_pool;
+  const T* v_src = dh >= 0 ? v_side : v_pool;
+  const int32_t* table = a.geom.table + (size_t)slot * a.geom.max_pages_per_seq;
+  auto side_row = [&](int i) -> size_t {       // i-th full-precision token -> offset of its head's dims
     const int t = i < lo ? i : hi + (i - lo);
-    return (seq_base + (t < lo ? t : n_sink + t % n_window)) * (size_t)d_drop + (size_t)dh * DH;
+    if (dh >= 0) return (seq_base + (t < lo ? t : n_sink + t % n_window)) * (size_t)d_drop + (size_t)dh * DH;
+    int page = table[t / a.geom.page_tokens];
+    if (page < 0 || page >= a.geom.n_pages) {
+      report(a.status, ECHOKV_EBADPAGE);
+      page = 0;
+    }
+    return ((size_t)page * a.geom.page_tokens + t % a.geom.page_tokens) * (size_t)pool_width + (size_t)kvh * DH;
   };
   // scores: one token per thread
   for (int i = tid; i < n_tok; i += 128) {
-    const T* kr = k_side + side_row(i);
+    const T* kr = k_src + side_row(i);
     float acc[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
@@ -664,13 +678,13 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
   if (tid < g) s_l[tid] = (red[0][tid] + red[1][tid]) + (red[2][tid] + red[3][tid]);
   __syncthreads();
   // weighted V: one output feature per thread
-  const int part = (len + part_tokens - 1) / part_tokens;
+  const int part = fixed_part >= 0 ? fixed_part : (len + part_tokens - 1) / part_tokens;
   if (tid < DH) {
     float o[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
     for (int i = 0; i < n_tok; ++i) {
-      const float vv = to_f32(v_side[side_row(i) + tid]);
+      const float vv = to_f32(v_src[side_row(i) + tid]);
 #pragma unroll
       for (int gi = 0; gi < kMaxGroup; ++gi)
         if (gi < g) o[gi] = fmaf(sc[gi * n_side + i], vv, o[gi]);
@@ -685,26 +699,30 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
 
 template <typename T, int DH>
 static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, int n_ret, int part_tokens,
-                                      cudaStream_t stream) {
-  const int n_drop = a.n_kv_heads - n_ret;
+                                      cudaStream_t stream, const SidePool* pool) {
+  const int first_head = pool ? 0 : n_ret;
+  const int n_heads = a.n_kv_heads - first_head;
   const int n_side = side.n_sink + side.n_window;
   const size_t smem = (size_t)(kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(attn_side_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid(n_drop, a.batch);
-  attn_side_kernel<T, DH><<<grid, 128, smem, stream>>>(a, (const T*)side.k_side, (const T*)side.v_side, side.n_sink,
-                                                       side.n_window, side.d_drop, n_ret, part_tokens);
+  dim3 grid(n_heads, a.batch);
+  attn_side_kernel<T, DH><<<grid, 128, smem, stream>>>(
+      a, (const T*)side.k_side, (const T*)side.v_side, side.n_sink, side.n_window, side.d_drop, n_ret, part_tokens,
+      first_head, pool ? pool->part : -1, pool ? (const T*)pool->k_pool : nullptr,
+      pool ? (const T*)pool->v_pool : nullptr, pool ? pool->width : 0);
   return cudaGetLastError();
 }
 
 cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int n_ret_heads, int part_tokens,
-                             cudaStream_t stream) {
+                             cudaStream_t stream, const SidePool* pool) {
   if (a.dtype == ECHOKV_BF16) {
-    if (a.head_dim == 128) return launch_attn_side_t<__nv_bfloat16, 128>(a, side, n_ret_heads, part_tokens, stream);
-    return launch_attn_side_t<__nv_bfloat16, 64>(a, side, n_ret_heads, part_tokens, stream);
+    if (a.head_dim == 128)
+      return launch_attn_side_t<__nv_bfloat16, 128>(a, side, n_ret_heads, part_tokens, stream, pool);
+    return launch_attn_side_t<__nv_bfloat16, 64>(a, side, n_ret_heads, part_tokens, stream, pool);
   }
-  if (a.head_dim == 128) return launch_attn_side_t<float, 128>(a, side, n_ret_heads, part_tokens, stream);
-  return launch_attn_side_t<float, 64>(a, side, n_ret_heads, part_tokens, stream);
+  if (a.head_dim == 128) return launch_attn_side_t<float, 128>(a, side, n_ret_heads, part_tokens, stream, pool);
+  return launch_attn_side_t<float, 64>(a, side, n_ret_heads, part_tokens, stream, pool);
 }
 
 }  // namespace echokv

@@ -42,6 +42,11 @@ def test_window_against_oracle(name, base, over, lens, window):
         assert_parity(case.run(1), case.oracle(1), w.dtype, "%s path %d" % (name, path))
     # the anchor layer is served as before
     assert_parity(case.run(0), case.oracle(0), w.dtype, name + " anchor")
+    # and the absorbed-predictor mode gives the same, where the shape has it
+    n = C.c_uint64(0)
+    if binding.lib().echokv_absorbed_workspace_bytes(C.byref(case.cfg), C.byref(n)) == binding.ECHOKV_OK:
+        case.ctx.enable_absorbed()
+        assert_parity(case.run(1), case.oracle(1), w.dtype, name + " absorbed")
     assert case.ctx.device_status() == binding.ECHOKV_OK
     case.close()
 
@@ -99,12 +104,4 @@ def test_window_status_codes():
     assert L.echokv_side_buffer_bytes(C.byref(case.cfg), -1, 0, C.byref(n)) == binding.ECHOKV_EINVAL
     assert L.echokv_set_full_precision_window(case.ctx.handle, 4, 128, None, None) == binding.ECHOKV_EINVAL
     assert L.echokv_set_full_precision_window(case.ctx.handle, 0, 0, None, None) == binding.ECHOKV_OK
-    # the absorbed mode does not take a window
-    case.ctx.set_full_precision_window(4, 8)
-    case.ctx.enable_absorbed()
-    q = case.q[1].to(case.ctx.device)
-    out = torch.empty(q.shape, dtype=torch.float32, device=case.ctx.device)
-    rc = L.echokv_decode_attention(case.ctx.handle, 1, q.data_ptr(), out.data_ptr(), None, case.seq_lens.data_ptr(),
-                                   2, None)
-    assert rc == binding.ECHOKV_EUNSUPPORTED
     case.close()
