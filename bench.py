@@ -160,12 +160,16 @@ class State:
     generators (drawn on the device: the largest workloads do not fit host memory), predictors,
     one decode query per layer, and the newest token of every layer (re-appended by each step)."""
 
-    def __init__(self, w, local_rank, layers):
+    def __init__(self, w, local_rank, layers, window=None):
         import torch
         from paper_2603_22910_b200 import binding, synth
         self.w, self.layers = w, layers
+        self.window = window if (window and w.D > w.m) else None
         self.dev = dev = torch.device("cuda", local_rank)
         self.ctx = ctx = binding.Context(binding.config_for(w, device=local_rank))
+        if self.window:
+            ctx.set_full_precision_window(*self.window)
+        self.true_rows = {}   # (layer, kind, b) -> (token indices, their dims m..D-1): sink and window tokens
         self.table = synth.block_table(w)
         ctx.set_block_table(self.table)
         t0 = time.perf_counter()
@@ -180,12 +184,29 @@ class State:
                     if width == 0:
                         continue
                     ids = self.table[b].long().to(dev)
-                    x = synth.layer_cache(w, l, kind, b, width=width, device=dev)
+                    x = synth.layer_cache(w, l, kind, b, width=w.D if self.window else width, device=dev)
+                    if self.window and not w.is_anchor(l):
+                        # sink and recent-window tokens keep their dims m..D-1 in the side buffers
+                        n_sink, n_window = self.window
+                        L = w.context
+                        toks = [t for t in range(L) if t < n_sink or t >= L - n_window]
+                        tt = torch.tensor(toks, device=dev)
+                        rows = x[tt, w.m:]
+                        side = (ctx.k_side if kind == "k" else ctx.v_side)[l]
+                        slots = torch.tensor([t if t < n_sink else n_sink + t % n_window for t in toks], device=dev)
+                        side[b, slots] = rows          # (a sink token inside the window: same values twice)
+                        self.true_rows[(l, kind, b)] = (toks, rows.cpu())
+                        newest_full = x[w.context - 1].clone()
+                        x = x[:, :width].contiguous()
+                    else:
+                        newest_full = None
                     pad = w.pages_per_seq * w.page_tokens - w.context
                     if pad:
                         x = torch.cat([x, torch.zeros((pad, width), dtype=tdt, device=dev)])
                     pools[l][ids] = x.reshape(w.pages_per_seq, w.page_tokens, width)
                     newest[b, :width] = x[w.context - 1]
+                    if newest_full is not None:
+                        newest[b] = newest_full        # the step re-appends the newest token, all its dims
                     del x
                 self.new_dev[(l, kind)] = newest
                 self.new_host[(l, kind)] = newest.cpu().pin_memory()
@@ -231,6 +252,16 @@ class State:
         Wk, Wv = (O.widen(st(t)) for t in self.ctx._weights[layer][:2])
         return q, kg, vg, kl, vl, Wk, Wv
 
+    def true_dropped(self, layer, kind, b):
+        """[L, D - m] with the sink / window tokens' own dims m..D-1 (NaN elsewhere: never read)."""
+        import numpy as np
+        from oracle import echokv_oracle as O
+        from paper_2603_22910_b200 import synth
+        toks, rows = self.true_rows[(layer, kind, b)]
+        out = np.full((self.w.context, self.w.D - self.w.m), np.nan)
+        out[toks] = O.widen(synth.to_numpy_stored(rows))
+        return out
+
 
 def plan_layers(w, mode):
     """(layers resident on the GPU, [(layer, attend?)] of one step)."""
@@ -258,10 +289,13 @@ def oracle_threads():
         return os.cpu_count() or 1
 
 
-def oracle_layer(inputs, w):
+def oracle_layer(inputs, w, state=None, layer=None, b=None):
     from oracle import echokv_oracle as O
     if len(inputs) == 3:
         return O.full_attention(inputs[0], inputs[1], inputs[2], w.n_kv_heads)
+    if state is not None and state.window:
+        return O.decode_attention_windowed(*inputs, w.n_kv_heads, state.true_dropped(layer, "k", b),
+                                           state.true_dropped(layer, "v", b), state.window[0], state.window[1])
     return O.decode_attention(*inputs, n_kv_heads=w.n_kv_heads)
 
 
@@ -277,7 +311,7 @@ def time_oracle(state, step_layers, budget_s):
         for b in range(min(w.batch, 4)):
             inputs = state.oracle_inputs(layer, b)
             t0 = time.perf_counter()
-            outs[(layer, b)] = oracle_layer(inputs, w)
+            outs[(layer, b)] = oracle_layer(inputs, w, state, layer, b)
             elapsed += time.perf_counter() - t0
             if elapsed >= budget_s:
                 break
@@ -292,7 +326,7 @@ def time_oracle(state, step_layers, budget_s):
     for l in group:
         inputs = state.oracle_inputs(l, b)
         t0 = time.perf_counter()
-        outs[(l, b)] = oracle_layer(inputs, w)
+        outs[(l, b)] = oracle_layer(inputs, w, state, l, b)
         elapsed += time.perf_counter() - t0
     scale = len(attend) / float(len(group))
     return 1.0 / (elapsed * scale), ("sequence 0 of %d, layers 0..%d (one group of S = %d), all heads, all %d "
@@ -458,7 +492,10 @@ def run_ours(args):
     w = w.replace(seed=rep.seed_for(w.seed))
     full = args.mode == "full"
     resident, step_layers = plan_layers(w, args.mode)
-    st = State(w, local_rank, resident)
+    window = None
+    if args.window and not full:
+        window = tuple(int(v) for v in args.window.split(","))
+    st = State(w, local_rank, resident, window)
     ctx, dev = st.ctx, st.dev
     if args.stored_path is not None:
         ctx.set_stored_path(args.stored_path)
@@ -611,6 +648,7 @@ def run_ours(args):
         "roofline": roofline,
         "decode_path": ctx.decode_path(), "stored_path": ctx.stored_path(),
         "decode_mode": "absorbed" if absorbed else "explicit",
+        "full_precision_tokens": {"sink": window[0], "window": window[1]} if window else None,
         "input_generation_s": st.gen_s,
     }
 
@@ -652,6 +690,8 @@ def main():
     ap.add_argument("--decode-mode", default="explicit", choices=["explicit", "absorbed"],
                     help="explicit: reconstruct-then-attend as the paper states it (the headline); absorbed: the "
                          "predictors folded into the queries and the output (same outputs, HBM-bound)")
+    ap.add_argument("--window", default="", help="n_sink,n_window: tokens kept at full precision, e.g. 4,128 (the "
+                                                 "paper's setting); default none, as the benchmark configs state")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")

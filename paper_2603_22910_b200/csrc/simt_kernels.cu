@@ -605,6 +605,7 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
   const int n_side = n_sink + n_window;
   float* qs = side_smem;                      // [g][DH]
   float* sc = qs + kMaxGroup * DH;            // [g][n_side]
+  unsigned long long* rows = reinterpret_cast<unsigned long long*>(sc + kMaxGroup * n_side);   // [n_side]
   __shared__ float red[4][kMaxGroup];
   __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
   const int slot = a.slots ? a.slots[b] : b;
@@ -632,9 +633,12 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     }
     return ((size_t)page * a.geom.page_tokens + t % a.geom.page_tokens) * (size_t)pool_width + (size_t)kvh * DH;
   };
+  // where each full-precision token lives (looked up once: the loops below must not chase the block table)
+  for (int i = tid; i < n_tok; i += 128) rows[i] = side_row(i);
+  __syncthreads();
   // scores: one token per thread
   for (int i = tid; i < n_tok; i += 128) {
-    const T* kr = k_src + side_row(i);
+    const T* kr = k_src + rows[i];
     float acc[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
@@ -683,8 +687,9 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     float o[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
+#pragma unroll 4
     for (int i = 0; i < n_tok; ++i) {
-      const float vv = to_f32(v_src[side_row(i) + tid]);
+      const float vv = to_f32(v_src[rows[i] + tid]);
 #pragma unroll
       for (int gi = 0; gi < kMaxGroup; ++gi)
         if (gi < g) o[gi] = fmaf(sc[gi * n_side + i], vv, o[gi]);
@@ -703,7 +708,7 @@ static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, i
   const int first_head = pool ? 0 : n_ret;
   const int n_heads = a.n_kv_heads - first_head;
   const int n_side = side.n_sink + side.n_window;
-  const size_t smem = (size_t)(kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float);
+  const size_t smem = (size_t)(kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float) + (size_t)n_side * 8 + 8;
   cudaError_t e = cudaFuncSetAttribute(attn_side_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(n_heads, a.batch);
