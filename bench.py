@@ -63,10 +63,14 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def workload_by_name(name, batch=0, context=0, page_tokens=0, random_pages=False, ratio=75):
+def workload_by_name(name, batch=0, context=0, page_tokens=0, random_pages=False, ratio=75, retained_dims=0):
     from paper_2603_22910_b200 import synth
     if name == "c4":
-        return synth.c4_point(ratio, context or 16384, batch or 8)
+        w = synth.c4_point(ratio, context or 16384, batch or 8)
+        if retained_dims:   # the paper's own settings, e.g. m = 64: half of the first head (absorbed mode only)
+            w = w.replace(n_retained_dims=retained_dims, n_retained_heads=retained_dims // w.head_dim,
+                          name="c4_m%d_L%d_B%d" % (retained_dims, w.context, w.batch))
+        return w
     w = {"c1": synth.C1, "c2": synth.C2, "c3": synth.C3}[name]
     if page_tokens:
         w = w.replace(page_tokens=page_tokens, name=w.name + "_P%d" % page_tokens)
@@ -85,7 +89,7 @@ def algorithmic_work(w):
     predictors once)."""
     tokens = w.batch * w.context
     g = w.n_q_heads // w.n_kv_heads
-    n_drop_q = (w.n_kv_heads - w.n_retained_heads) * g
+    n_drop_q = (w.n_kv_heads - w.m // w.head_dim) * g
     flops = tokens * (4.0 * w.d_in * w.d_drop + 4.0 * n_drop_q * w.head_dim)
     elem = 2 if w.dtype == "bf16" else 4
     bytes_ = tokens * 2.0 * w.d_in * elem + 2.0 * w.d_in * w.d_drop * elem
@@ -341,7 +345,8 @@ def run_reference(args):
         return 0
     from oracle import echokv_oracle as O
     from paper_2603_22910_b200 import synth
-    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio)
+    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio,
+                         args.retained_dims)
     st = synth.to_numpy_stored
     full = args.mode == "full"
     layer = 0 if full else 1
@@ -488,13 +493,16 @@ def run_ours(args):
     rep.barrier()
     binding.lib()
 
-    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio)
+    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio,
+                         args.retained_dims)
     w = w.replace(seed=rep.seed_for(w.seed))
     full = args.mode == "full"
     resident, step_layers = plan_layers(w, args.mode)
     window = None
     if args.window and not full:
         window = tuple(int(v) for v in args.window.split(","))
+        if sum(window) == 0:
+            window = None
     st = State(w, local_rank, resident, window)
     ctx, dev = st.ctx, st.dev
     if args.stored_path is not None:
@@ -698,6 +706,9 @@ def main():
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
     ap.add_argument("--ratio", type=int, default=75, choices=[25, 50, 75],
                     help="c4 only: percent of the layer's KV heads discarded")
+    ap.add_argument("--retained-dims", type=int, default=0,
+                    help="c4 only: m in flat dims instead of --ratio, e.g. 64 or 384 (the paper's settings); a value "
+                         "that splits a head needs --decode-mode absorbed")
     ap.add_argument("--page-tokens", type=int, default=0, choices=[0, 16, 32, 64, 128],
                     help="override the tokens per cache page (default 16)")
     ap.add_argument("--random-pages", action="store_true", help="pages of the pool in a seeded random order")

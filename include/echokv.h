@@ -78,6 +78,12 @@ typedef struct {
   int64_t n_pages;           /* pages per pool                                             */
   float softmax_scale;       /* 0 -> 1 / sqrt(head_dim) (Eq. 7)                            */
   int32_t device;            /* CUDA device ordinal                                        */
+  int32_t n_retained_dims;   /* 0: m = n_retained_heads * head_dim.  Otherwise m itself, in flat dims: a
+                                multiple of 64 in [0, D] that need not end on a head boundary (the paper's
+                                m = 64 keeps half of head 0); n_retained_heads is then ignored.  A partly
+                                retained head is served by the absorbed mode only: echokv_create succeeds
+                                where that mode is available (EUNSUPPORTED otherwise) and
+                                echokv_decode_attention returns EUNSUPPORTED until echokv_enable_absorbed */
 } echokv_config;
 
 typedef struct {

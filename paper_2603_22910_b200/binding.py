@@ -26,7 +26,7 @@ class echokv_config(C.Structure):
                 ("head_dim", C.c_int32), ("group_size", C.c_int32), ("n_retained_heads", C.c_int32),
                 ("page_tokens", C.c_int32), ("max_batch", C.c_int32), ("max_pages_per_seq", C.c_int32),
                 ("dtype", C.c_int32), ("n_pages", C.c_int64), ("softmax_scale", C.c_float),
-                ("device", C.c_int32)]
+                ("device", C.c_int32), ("n_retained_dims", C.c_int32)]
 
 
 class echokv_sizes(C.Structure):
@@ -124,9 +124,10 @@ def _stream_handle(stream) -> int | None:
 
 def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_retained_heads,
                 page_tokens, max_batch, max_pages_per_seq, n_pages, dtype, softmax_scale=0.0,
-                device=0) -> echokv_config:
+                device=0, n_retained_dims=0) -> echokv_config:
     return echokv_config(n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_retained_heads,
-                         page_tokens, max_batch, max_pages_per_seq, dtype, n_pages, softmax_scale, device)
+                         page_tokens, max_batch, max_pages_per_seq, dtype, n_pages, softmax_scale, device,
+                         n_retained_dims)
 
 
 def echokv_query_sizes(cfg: echokv_config) -> echokv_sizes:
@@ -149,7 +150,7 @@ class Context:
         self.sizes = echokv_query_sizes(cfg)
         self.tdtype = torch.bfloat16 if cfg.dtype == ECHOKV_BF16 else torch.float32
         D = cfg.n_kv_heads * cfg.head_dim
-        m = cfg.n_retained_heads * cfg.head_dim
+        m = cfg.n_retained_dims if cfg.n_retained_dims else cfg.n_retained_heads * cfg.head_dim
         self.D, self.m = D, m
         alloc = torch.zeros if zero_pools else torch.empty
         self.k_pools, self.v_pools = [], []
@@ -318,4 +319,5 @@ def config_for(w, n_pages: int | None = None, device: int = 0, max_batch: int | 
                        max_batch=max_batch or w.batch, max_pages_per_seq=pages,
                        n_pages=n_pages or w.batch * pages,
                        dtype=ECHOKV_BF16 if w.dtype == "bf16" else ECHOKV_FP32,
-                       softmax_scale=1.0 / math.sqrt(w.head_dim), device=device)
+                       softmax_scale=1.0 / math.sqrt(w.head_dim), device=device,
+                       n_retained_dims=w.n_retained_dims)

@@ -87,7 +87,7 @@ constexpr int kQCols = 512;  // input features per block: two adjacent ones per 
 
 __global__ void __launch_bounds__(256)
 absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ Wk,
-                    __nv_bfloat16* __restrict__ q2, int B, int n_q_heads, int g, int n_ret, int D, int d_in,
+                    __nv_bfloat16* __restrict__ q2, int B, int n_q_heads, int g, int m, int D, int d_in,
                     float scale_log2e) {
   __shared__ float qs[kQGroup][128];
   const int i = blockIdx.x * kQCols + threadIdx.x * 2;     // first of this thread's two input features
@@ -109,21 +109,24 @@ absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   float acc[kQGroup][2];
 #pragma unroll
   for (int k = 0; k < kQGroup; ++k) acc[k][0] = acc[k][1] = 0.f;
-  if (kv < n_ret) {
-    // a retained head reads its own stored dims: q~ is q placed at the head's local dims
+  // dims kv * 128 + j of this head with flat index < m are stored (the head reads them as they are: q~ is q
+  // placed at those local dims); the others are predicted by row (flat index - m) of W_k
+  const int n_stored = max(0, min(128, m - kv * 128));
+  {
     const int j = i - (D + kv * 128);
-    if (j >= 0 && j < 128) {
+    if (j >= 0 && j < n_stored) {
 #pragma unroll
       for (int k = 0; k < kQGroup; ++k) {
         acc[k][0] = qs[k][j];
         acc[k][1] = qs[k][j + 1];
       }
     }
-  } else {
-    const __nv_bfloat16* w = Wk + (size_t)(kv - n_ret) * 128 * d_in + i;
+  }
+  if (n_stored < 128) {
+    const __nv_bfloat16* w = Wk + ((size_t)kv * 128 + n_stored - m) * d_in + i;
 #pragma unroll 16
-    for (int j = 0; j < 128; ++j) {
-      const uint32_t raw = *reinterpret_cast<const uint32_t*>(w + (size_t)j * d_in);
+    for (int j = n_stored; j < 128; ++j, w += d_in) {
+      const uint32_t raw = *reinterpret_cast<const uint32_t*>(w);
       const float w0 = __uint_as_float(raw << 16), w1 = __uint_as_float(raw & 0xffff0000u);
 #pragma unroll
       for (int k = 0; k < kQGroup; ++k) {
@@ -169,7 +172,7 @@ struct StreamParams {
   int d_in;
   int range_tokens;             // pv kernel: tokens per range
   int n_slices;                 // pv kernel: 256-feature slices
-  int v_tile_ok;                // pv kernel: the 4-chunk V maps exist for (anchor, local)
+  int v_tile_ok;                // pv kernel: the 4-chunk V maps exist (bit 0: anchor pool, bit 1: local pool)
   int n_sink, n_window;         // scores kernel: sink / recent-window tokens are left to the side kernel
 };
 
@@ -312,7 +315,7 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
   stream_setup(t, p, 256u, [](int len) { return (len + kScoreTokens - 1) / kScoreTokens; });
   const uint32_t tmem = t.tmem_base;
   const int n_items = t.cum[p.nb];
-  const int n_steps = p.kc_total / 2;                     // stages per item: two chunks each
+  const int n_steps = (p.kc_total + 1) / 2;               // stages per item: two chunks each (the last maybe one)
   const int box_tokens = min(p.page_tokens, kScoreTokens);
   const int boxes = kScoreTokens / box_tokens;
   const uint32_t page_bytes = box_tokens * kRowBytes;
@@ -329,7 +332,6 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
       const int slot = p.slots ? p.slots[b] : b;
       const int len = p.lens[b];
       const PageSet ps = lookup_pages(p, slot, len, tile * kScoreTokens, boxes, box_tokens, lane);
-      const uint32_t stage_tx = 2u * (ps.n_valid * page_bytes + q_chunk_bytes);
       for (int step = 0; step < n_steps; ++step, ++it) {
         const uint32_t s = it % p.n_stages;
         const uint32_t ph = (it / p.n_stages) & 1u;
@@ -339,19 +341,20 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) { alive = false; break; }
         const int kc0 = step * 2;                           // both chunks come from the same pool
+        const int n_chunks = min(2, p.kc_total - kc0);
         const bool from_anchor = kc0 < p.kc_anchor;
         const int kx0 = from_anchor ? kc0 : kc0 - p.kc_anchor;
-        if (lane == 0) mbar_arrive_expect_tx(full, stage_tx);
+        // (the absorbed-query box always brings two chunks: past the last one it is filled with zeros)
+        if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)n_chunks * ps.n_valid * page_bytes + 2u * q_chunk_bytes);
         __syncwarp();
         const uint32_t x_dst = stage_base + s * p.stage_bytes;
-        if (ps.all_run) {
+        if (ps.all_run && n_chunks == 2) {
           if (lane == 0)
             tma_load_3d(x_dst, from_anchor ? &tm_anchor_128 : &tm_local_128, 0, ps.row, kx0, full);
         } else if (ps.row >= 0 && !ps.run_member) {
           const CUtensorMap* m = ps.run_lead ? (from_anchor ? &tm_anchor_run : &tm_local_run)
                                              : (from_anchor ? &tm_anchor : &tm_local);
-#pragma unroll
-          for (int j = 0; j < 2; ++j)
+          for (int j = 0; j < n_chunks; ++j)
             tma_load_2d(x_dst + j * kScoreXBytes + lane * page_bytes, m, (kx0 + j) * kChunk, ps.row, full);
         }
         if (lane == 16) tma_load_3d(x_dst + 2 * kScoreXBytes, &tm_q2, 0, b * p.nh2, kc0, full);
@@ -373,8 +376,8 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
           if (!mbar_wait(smem_u32(&t.full_bar[s]), ph, abort_flag, p.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t x_addr = stage_base + s * p.stage_bytes;
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
+          const int n_chunks = min(2, p.kc_total - step * 2);
+          for (int j = 0; j < n_chunks; ++j) {
             const uint64_t a_desc = desc_kmajor(x_addr + j * kScoreXBytes);
             const uint64_t b_desc = desc_kmajor(x_addr + 2 * kScoreXBytes + j * q_chunk_bytes);
 #pragma unroll
@@ -566,7 +569,7 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
         if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)w.n_chunks * ps.n_valid * page_bytes + p_tile_bytes);
         __syncwarp();
         const uint32_t v_dst = stage_base + s * p.stage_bytes;
-        if (ps.all_run && w.n_chunks == 4 && one_pool && p.v_tile_ok) {
+        if (ps.all_run && w.n_chunks == 4 && one_pool && (p.v_tile_ok & (w.from_anchor ? 1 : 2))) {
           if (lane == 0)
             tma_load_3d(v_dst, w.from_anchor ? &tm_anchor_4 : &tm_local_4, 0, ps.row,
                         w.from_anchor ? w.kc0 : w.kc0 - p.kc_anchor, full);
@@ -597,7 +600,7 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
         const uint32_t buf = n & 1u;
         if (!mbar_wait(smem_u32(&t.acc_empty_bar[buf]), ((n >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
         tc_fence_after();
-        const int n_mtiles = w.n_chunks / 2;
+        const int n_mtiles = (w.n_chunks + 1) / 2;   // (a last tile may be half filled: its upper rows are unused)
         for (int step = 0; step < w.n_steps; ++step, ++it) {
           const uint32_t s = it % p.n_stages;
           const uint32_t ph = (it / p.n_stages) & 1u;
@@ -659,10 +662,11 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
       const uint32_t buf = n & 1u;
       if (!epi_all(mbar_wait(smem_u32(&t.acc_full_bar[buf]), (n >> 1) & 1u, abort_flag, p.status))) break;
       tc_fence_after();
-      const int n_mtiles = w.n_chunks / 2;
+      const int n_mtiles = (w.n_chunks + 1) / 2;
       for (int mt = 0; mt < n_mtiles; ++mt) {
         const uint32_t addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256u + mt * (uint32_t)p.nh2;
         const int feature = w.kc0 * kChunk + mt * 128 + row;
+        if (feature >= p.d_in) continue;          // (rows of a half-filled tile that stand for no feature)
         float* dst = p.y_out + (((size_t)w.b * kAbsorbMaxRanges + w.range) * p.n_q_heads) * p.d_in + feature;
         for (int hb = 0; hb < p.n_q_heads; hb += 16) {
           float hi[16], lo[16];
@@ -729,13 +733,14 @@ constexpr int kOutPairs = 8;     // (sequence, query head of the group) pairs pe
 __global__ void __launch_bounds__(256)
 absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restrict__ Wv,
                   const __nv_bfloat16* __restrict__ bv, float* __restrict__ out, int B, int n_q_heads, int g,
-                  int n_ret, int D, int d_in) {
+                  int m, int D, int d_in) {
   __shared__ float red[8][kOutRows][kOutPairs];
   const int kv = blockIdx.x, jt = blockIdx.y, first = blockIdx.z * kOutPairs;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_pairs = B * g;
-  if (kv < n_ret) {
-    // a retained head: its own stored dims
+  const int row0 = kv * 128 + jt * kOutRows;        // flat dim of this block's first output feature
+  if (row0 < m) {
+    // stored dims (m is a multiple of the block's 16 features): read back as they are
     for (int idx = tid; idx < kOutPairs * kOutRows; idx += 256) {
       const int k = idx / kOutRows, j = jt * kOutRows + idx % kOutRows;
       const int pr = first + k;
@@ -752,7 +757,7 @@ absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restric
     const int b = pr / g, h = kv * g + (pr - b * g);
     yrow[k] = ysum + ((size_t)b * n_q_heads + h) * d_in;
   }
-  const __nv_bfloat16* w = Wv + ((size_t)(kv - n_ret) * 128 + jt * kOutRows) * d_in;
+  const __nv_bfloat16* w = Wv + (size_t)(row0 - m) * d_in;
   float acc[kOutRows][kOutPairs];
 #pragma unroll
   for (int r = 0; r < kOutRows; ++r)
@@ -794,7 +799,7 @@ absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restric
       for (int ww = 0; ww < 8; ++ww) res += red[ww][r][k];
       const int b = pr / g, h = kv * g + (pr - b * g);
       const int j = jt * kOutRows + r;
-      if (bv != nullptr) res += __bfloat162float(bv[(kv - n_ret) * 128 + j]);
+      if (bv != nullptr) res += __bfloat162float(bv[row0 - m + r]);
       out[((size_t)b * n_q_heads + h) * 128 + j] = res;
     }
   }
@@ -821,11 +826,11 @@ int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
-bool absorbed_supported(int dtype, int head_dim, int n_q_heads, int n_kv_heads, int n_retained, int page_tokens) {
+bool absorbed_supported(int dtype, int head_dim, int n_q_heads, int n_kv_heads, int m, int page_tokens) {
   if (dtype != ECHOKV_BF16 || head_dim != 128) return false;
   if (n_q_heads != 16 && n_q_heads != 32 && n_q_heads != 64) return false;   // 2 H_q accumulator columns
   if (n_q_heads / n_kv_heads > kMaxGroup) return false;
-  if (n_retained >= n_kv_heads) return false;
+  if (m < 0 || m % 64 != 0 || m >= n_kv_heads * head_dim) return false;
   return page_tokens == 16 || page_tokens == 32 || page_tokens == 64 || page_tokens == 128;
 }
 
@@ -860,7 +865,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   if (a.batch > kMaxBatchPerLaunch) return cudaErrorInvalidValue;
   const int g = a.n_q_heads / a.n_kv_heads;
   const int d_in = r.D + r.m;
-  const int n_ret = r.m / 128;
+  const int n_ret = r.m / 128;           // (whole retained heads; used by the sink / window side kernel only)
   const AbsorbLayout& lay = r.lay;
   __nv_bfloat16* q2 = reinterpret_cast<__nv_bfloat16*>(r.ws + lay.off_q2);
   float* S = reinterpret_cast<float*>(r.ws + lay.off_s);
@@ -875,7 +880,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     dim3 grid((d_in + kQCols - 1) / kQCols, a.n_kv_heads, (a.batch * g + kQGroup - 1) / kQGroup);
     absorb_query_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q),
                                                   reinterpret_cast<const __nv_bfloat16*>(r.Wk), q2, a.batch,
-                                                  a.n_q_heads, g, n_ret, r.D, d_in, a.scale_log2e);
+                                                  a.n_q_heads, g, r.m, r.D, d_in, a.scale_log2e);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
 
@@ -949,16 +954,16 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     p.n_stages = (int)(kSmemBudget / p.stage_bytes);
     if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;
     p.idesc = make_idesc(lay.nh2, true);
-    // the 4-chunk maps exist for pools whose width is a multiple of 256, and a slice must not straddle pools
-    p.v_tile_ok = (r.D % 256 == 0 && (r.m == 0 || r.m % 256 == 0)) ? 1 : 0;
+    // the 4-chunk maps exist for pools at least 256 dims wide (bit 0: anchor pool, bit 1: this layer's pool)
+    p.v_tile_ok = (r.D >= 256 ? 1 : 0) | (r.m >= 256 ? 2 : 0);
     const size_t smem = 1024 + (size_t)p.n_stages * p.stage_bytes + sizeof(StreamSmemTail);
     if ((e = cudaFuncSetAttribute(absorb_pv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
         cudaSuccess)
       return e;
     const long long max_items = (long long)a.batch * ((capacity + range_tokens - 1) / range_tokens) * p.n_slices;
     const int grid = (int)(max_items < sm_count ? max_items : sm_count);
-    const CUtensorMap& a4 = p.v_tile_ok ? anchor.v_pool_tok64x4 : anchor.v_pool_run;
-    const CUtensorMap& l4 = p.v_tile_ok && r.m > 0 ? loc.v_pool_tok64x4 : a4;
+    const CUtensorMap& a4 = (p.v_tile_ok & 1) ? anchor.v_pool_tok64x4 : anchor.v_pool_run;
+    const CUtensorMap& l4 = (p.v_tile_ok & 2) ? loc.v_pool_tok64x4 : a4;
     if (ev) cudaEventRecord(ev[2], stream);
     absorb_pv_kernel<<<grid, kThreads, smem, stream>>>(anchor.v_pool, loc.v_pool, anchor.v_pool_run, loc.v_pool_run, a4,
                                                        l4, maps.p2, p);
@@ -975,7 +980,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     dim3 grid2(a.n_kv_heads, 128 / kOutRows, (a.batch * g + kOutPairs - 1) / kOutPairs);
     absorb_out_kernel<<<grid2, 256, 0, stream>>>(ysum, reinterpret_cast<const __nv_bfloat16*>(r.Wv),
                                                  reinterpret_cast<const __nv_bfloat16*>(r.bv), out, a.batch,
-                                                 a.n_q_heads, g, n_ret, r.D, d_in);
+                                                 a.n_q_heads, g, r.m, r.D, d_in);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   // 6. sink and recent-window tokens (Section 5.1): attended at full precision by the side kernel, then

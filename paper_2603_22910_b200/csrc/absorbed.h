@@ -28,7 +28,8 @@ struct AbsorbLayout {
   uint64_t total;
 };
 
-bool absorbed_supported(int dtype, int head_dim, int n_q_heads, int n_kv_heads, int n_retained, int page_tokens);
+// m = retained flat dims per token: any multiple of 64 below D (it need not end on a head boundary)
+bool absorbed_supported(int dtype, int head_dim, int n_q_heads, int n_kv_heads, int m, int page_tokens);
 void absorbed_layout(int max_batch, int n_q_heads, int d_in, int capacity_tokens, AbsorbLayout* out);
 
 struct AbsorbMaps {

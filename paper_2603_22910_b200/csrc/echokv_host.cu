@@ -20,6 +20,7 @@ inline uint64_t align_up(uint64_t v) { return (v + kAlign - 1) / kAlign * kAlign
 
 struct Derived {
   int D, m, d_in, d_drop, g, elem, part_tokens, capacity, max_parts;
+  bool head_aligned;   // m ends on a head boundary (the explicit kernels need it; the absorbed mode does not)
   uint64_t off_status, off_ml, off_o, off_q, off_k, off_v, off_out, off_lens, off_pos, total;
 };
 
@@ -41,6 +42,13 @@ int derive(const echokv_config* c, Derived* d) {
   if (cap > (1ll << 30)) return ECHOKV_EINVAL;
   d->D = c->n_kv_heads * c->head_dim;
   d->m = c->n_retained_heads * c->head_dim;
+  if (c->n_retained_dims != 0) {
+    // m given in flat dims (the paper's m = 64: half of the first head): any multiple of 64 up to D
+    if (c->n_retained_dims < 0 || c->n_retained_dims > d->D) return ECHOKV_EINVAL;
+    if (c->n_retained_dims % 64 != 0) return ECHOKV_EUNSUPPORTED;
+    d->m = c->n_retained_dims;
+  }
+  d->head_aligned = d->m % c->head_dim == 0;
   d->d_in = d->D + d->m;
   d->d_drop = d->D - d->m;
   d->elem = c->dtype == ECHOKV_BF16 ? 2 : 4;
@@ -319,6 +327,14 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
   if (cudaMemset(c->ws + d.off_status, 0, kAlign) != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
   c->tc_capable = tc_shape_supported(cfg->dtype, cfg->head_dim, cfg->page_tokens, d.D, d.m);
   if (!any_compressed || d.d_drop == 0) c->path = 0;
+  else if (!d.head_aligned) {
+    // a partly retained head: served by the absorbed mode only
+    if (!absorbed_supported(cfg->dtype, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, d.m, cfg->page_tokens)) {
+      delete c;
+      return ECHOKV_EUNSUPPORTED;
+    }
+    c->path = 0;
+  }
   else if (!c->tc_capable) c->path = 1;
   else {
     // Long contractions (many 64-feature chunks per phase, few query heads per KV head) hide the
@@ -407,6 +423,7 @@ int echokv_set_full_precision_window(echokv_ctx* c, int n_sink, int n_window, vo
                                      void* const* v_side) {
   if (!c || n_sink < 0 || n_window < 0) return ECHOKV_EINVAL;
   if (n_sink + n_window > 4096) return ECHOKV_EUNSUPPORTED;
+  if (!c->d.head_aligned && (n_sink > 0 || n_window > 0)) return ECHOKV_EUNSUPPORTED;   // (side buffers are per head)
   const bool on = (n_sink > 0 || n_window > 0) && c->d.d_drop > 0;
   if (on) {
     if (!k_side || !v_side) return ECHOKV_EINVAL;
@@ -431,8 +448,8 @@ int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out) {
   Derived d;
   const int rc = derive(cfg, &d);
   if (rc != ECHOKV_OK) return rc;
-  if (!absorbed_supported(cfg->dtype, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, cfg->n_retained_heads,
-                          cfg->page_tokens) || cfg->max_batch > 256)
+  if (!absorbed_supported(cfg->dtype, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, d.m, cfg->page_tokens) ||
+      cfg->max_batch > 256)
     return ECHOKV_EUNSUPPORTED;
   AbsorbLayout lay;
   absorbed_layout(cfg->max_batch, cfg->n_q_heads, d.d_in, d.capacity, &lay);
@@ -540,7 +557,8 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     c->launches += side ? 8 : 6;
     return ECHOKV_OK;
   }
-  const int r = c->cfg.n_retained_heads;
+  if (!c->d.head_aligned) return ECHOKV_EUNSUPPORTED;   // explicit reconstruction needs whole heads: use the absorbed mode
+  const int r = c->d.m / c->cfg.head_dim;
   // retained heads: Eq. 7 on what is stored (Eq. 6 keeps them as they are)
   const int n_splits = stored_splits(c, B, r);
   const int32_t* item_tokens = nullptr;

@@ -563,12 +563,17 @@ cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const voi
   e = encode_2d(&maps->v_pool_run, v_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (e != cudaSuccess) return e;
   // CTA-pair kernel: 128 consecutive token rows x two 64-feature chunks in one copy
-  e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-  if (e != cudaSuccess) return e;
-  e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-  if (e != cudaSuccess) return e;
+  if (width >= 128) {     // (a pool one chunk wide is never read two chunks at a time)
+    e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    if (e != cudaSuccess) return e;
+    e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    if (e != cudaSuccess) return e;
+  } else {
+    maps->k_pool_run128 = maps->k_pool_run;
+    maps->v_pool_run128 = maps->v_pool_run;
+  }
   // absorbed mode, V side: 64 consecutive token rows x four 64-feature chunks in one copy
-  if (width % 256 == 0) {
+  if (width >= 256) {
     e = encode_3d_chunks(&maps->v_pool_tok64x4, v_pool, rows, width, 64, 4, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (e != cudaSuccess) return e;
   }

@@ -44,6 +44,7 @@ class Workload:
     page_tokens: int = 16
     random_pages: bool = False
     seed: int = 1000
+    n_retained_dims: int = 0   # if non-zero: m itself, in flat dims (need not end on a head boundary)
 
     @property
     def D(self) -> int:
@@ -51,7 +52,7 @@ class Workload:
 
     @property
     def m(self) -> int:
-        return self.n_retained_heads * self.head_dim
+        return self.n_retained_dims if self.n_retained_dims else self.n_retained_heads * self.head_dim
 
     @property
     def d_in(self) -> int:

@@ -62,6 +62,40 @@ def test_absorbed_mode_against_oracle(name, base, over, lens):
     case.close()
 
 
+RAGGED = [
+    # the paper's own settings for 8 KV heads x 128 (Appendix "Compression-Ratio Configurations"): m need not end
+    # on a head boundary.  name, overrides, lens
+    ("paper_S4_m64", dict(n_retained_dims=64, n_retained_heads=0, batch=2, context=700, group_size=4, n_layers=4),
+     [700, 129]),
+    ("paper_S2_m384", dict(n_retained_dims=384, n_retained_heads=3, batch=2, context=400, random_pages=True), [400, 65]),
+    ("m320_pages64", dict(n_retained_dims=320, n_retained_heads=2, batch=2, context=500, page_tokens=64), [500, 64]),
+    ("m960_one_half_head_dropped", dict(n_retained_dims=960, n_retained_heads=7, batch=2, context=300), [300, 7]),
+]
+
+
+@pytest.mark.parametrize("name,over,lens", RAGGED, ids=[r[0] for r in RAGGED])
+def test_retained_dims_that_split_a_head(name, over, lens):
+    w = synth.C2.replace(**over)
+    layers = [l for l in range(w.n_layers) if not w.is_anchor(l)][:2]
+    case = Case(w, lens=lens, layers=layers)
+    L = binding.lib()
+    dev = case.ctx.device
+    l0 = layers[0]
+    q = case.q[l0].to(dev)
+    out = torch.empty(q.shape, dtype=torch.float32, device=dev)
+    if w.m % w.head_dim:
+        # explicit reconstruction works on whole heads only
+        assert case.ctx.decode_path() == 0
+        rc = L.echokv_decode_attention(case.ctx.handle, l0, q.data_ptr(), out.data_ptr(), None,
+                                       case.seq_lens.data_ptr(), w.batch, None)
+        assert rc == binding.ECHOKV_EUNSUPPORTED
+    case.ctx.enable_absorbed()
+    for l in layers:
+        assert_parity(case.run(l), case.oracle(l), w.dtype, "%s layer %d" % (name, l))
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
 def test_absorbed_multi_layer_random_pages():
     w = synth.C3.replace(n_layers=8, batch=2, context=420)
     case = Case(w, lens=[420, 131], n_pages=2 * w.pages_per_seq + 13)
