@@ -248,3 +248,49 @@ def test_layer_step_from_host_memory_matches_device_calls():
                                   other.host[(l, "v", "new")].pin_memory(), out_host, lens_host, attend=attend)
     np.testing.assert_array_equal(out_host.numpy(), ref)
     case.close(); other.close()
+
+
+@pytest.mark.parametrize("absorbed", [False, True], ids=["explicit", "absorbed"])
+def test_layer_step_replayed_from_a_cuda_graph(absorbed):
+    # every call only enqueues kernels on the caller's stream, so a whole step can be captured once and replayed
+    w = synth.C2.replace(batch=2, context=600)
+    case = Case(w, lens=[600, 333], layers=[0, 1])
+    ctx, dev = case.ctx, case.ctx.device
+    if absorbed:
+        ctx.enable_absorbed()
+    q = {l: case.q[l].to(dev) for l in (0, 1)}
+    out = {l: torch.empty(q[l].shape, dtype=torch.float32, device=dev) for l in (0, 1)}
+    new = {(l, kind): case.host[(l, kind, "new")].to(dev) for l in (0, 1) for kind in ("k", "v")}
+
+    def step():
+        for l in (0, 1):
+            ctx.append_kv(l, new[(l, "k")], new[(l, "v")], case.positions)
+            ctx.decode_attention(l, q[l], case.seq_lens, out=out[l])
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step()                       # first-use set-up happens here, outside the capture
+        side.synchronize()
+        eager = {l: out[l].clone() for l in (0, 1)}
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.current_stream().wait_stream(side)
+    for l in (0, 1):
+        out[l].fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    for l in (0, 1):
+        assert torch.equal(out[l], eager[l])
+    # new queries through the same graph: the captured kernels read the tensors, not copies of them
+    q2 = synth.queries(w.replace(seed=w.seed + 5), 1).to(dev)
+    q[1].copy_(q2)
+    graph.replay()
+    torch.cuda.synchronize()
+    replayed = out[1].clone()
+    direct = ctx.decode_attention(1, q2, case.seq_lens)
+    torch.cuda.synchronize()
+    assert torch.equal(replayed, direct)
+    assert ctx.device_status() == binding.ECHOKV_OK
+    case.close()
