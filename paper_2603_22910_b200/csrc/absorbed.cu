@@ -9,11 +9,11 @@
 //
 //   1. absorb_query_kernel   q~[b][h][:] for every head, scaled, split into two bf16 halves
 //   2. absorb_scores_kernel  S[b][h][t] = q~ . x^K_t        tcgen05: M = 128 tokens, N = 2 H_q, K = D_in
-//   3. absorb_softmax_kernel (max, sum) per head; p = 2^(S - max) split into two bf16 halves
+//   3. absorb_softmax_kernel (max, sum) per head and token range; p = 2^(S - max of the range) as two bf16 halves
 //   4. absorb_pv_kernel      y[b][h][:] = sum_t p_t x^V_t   tcgen05: M = 128 features (the V tile
 //                            is the M-major A operand), N = 2 H_q, K = tokens; split over token
 //                            ranges and 256-feature slices
-//   5. absorb_ysum_kernel    y summed over the ranges and divided by the softmax sum;
+//   5. absorb_ysum_kernel    y of the ranges merged by log-sum-exp and divided by the softmax sum;
 //      absorb_out_kernel     out = W_v y (+ b_v) for predicted heads, y's own dims for retained heads
 //
 // The same result as the explicit path (Eq. 3, 6, 7) up to rounding, at 4 D_in bytes and
@@ -437,20 +437,22 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
 // ---------------------------------------------------------------------------------------------
 // 3. softmax statistics and probabilities
 // ---------------------------------------------------------------------------------------------
+// One block per (query head, sequence, token range of the V pass): the range's own maximum and sum, and its
+// probabilities relative to that maximum; the ranges are merged by log-sum-exp in absorb_ysum_kernel.
 __global__ void __launch_bounds__(256)
-absorb_softmax_kernel(const float* __restrict__ S, __nv_bfloat16* __restrict__ p2, float2* __restrict__ ml,
+absorb_softmax_kernel(const float* __restrict__ S, __nv_bfloat16* __restrict__ p2, float2* __restrict__ ml_range,
                       const int32_t* __restrict__ slots, const int32_t* __restrict__ lens, int max_batch,
-                      int capacity, int n_q_heads, int l_cap) {
-  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+                      int capacity, int n_q_heads, int l_cap, int range_tokens) {
+  const int h = blockIdx.x, b = blockIdx.y, range = blockIdx.z, tid = threadIdx.x;
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
-  if (slot < 0 || slot >= max_batch || len < 1 || len > capacity) {
-    if (tid == 0) ml[(size_t)b * n_q_heads + h] = make_float2(-INFINITY, 0.f);
-    return;
-  }
+  if (slot < 0 || slot >= max_batch || len < 1 || len > capacity) return;   // (absorb_ysum_kernel writes zeros)
+  const int t_begin = range * range_tokens;
+  if (t_begin >= len) return;
+  const int t_end = min(len, t_begin + range_tokens);
   __shared__ float red[8];
-  const float* s = S + ((size_t)b * n_q_heads + h) * l_cap;
-  const int n4 = (len + 3) / 4;                  // (entries past len hold -inf up to the next 128)
+  const float* s = S + ((size_t)b * n_q_heads + h) * l_cap + t_begin;
+  const int n4 = (t_end - t_begin + 3) / 4;      // (entries past len hold -inf up to the next 128)
   float m = -INFINITY;
   for (int i = tid; i < n4; i += 256) {
     const float4 v = reinterpret_cast<const float4*>(s)[i];
@@ -464,11 +466,11 @@ absorb_softmax_kernel(const float* __restrict__ S, __nv_bfloat16* __restrict__ p
   for (int w = 1; w < 8; ++w) M = fmaxf(M, red[w]);
   __syncthreads();
   const float M_out = M;
-  if (M == -INFINITY) M = 0.f;     // every token is a sink / window token: all probabilities are 0 here
+  if (M == -INFINITY) M = 0.f;     // every token of the range is a sink / window token: all probabilities are 0
   const int nh2 = 2 * n_q_heads;
-  __nv_bfloat16* hi = p2 + ((size_t)b * nh2 + h) * l_cap;
-  __nv_bfloat16* lo = p2 + ((size_t)b * nh2 + n_q_heads + h) * l_cap;
-  const int n4_pad = ((len + 63) / 64) * 16;     // the V pass reads whole 64-token blocks
+  __nv_bfloat16* hi = p2 + ((size_t)b * nh2 + h) * l_cap + t_begin;
+  __nv_bfloat16* lo = p2 + ((size_t)b * nh2 + n_q_heads + h) * l_cap + t_begin;
+  const int n4_pad = ((t_end - t_begin + 63) / 64) * 16;     // the V pass reads whole 64-token blocks
   float L = 0.f;
   for (int i = tid; i < n4_pad; i += 256) {
     const float4 v = reinterpret_cast<const float4*>(s)[i];
@@ -491,7 +493,7 @@ absorb_softmax_kernel(const float* __restrict__ S, __nv_bfloat16* __restrict__ p
     float tot = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
-    ml[(size_t)b * n_q_heads + h] = make_float2(M_out, tot);
+    ml_range[((size_t)b * n_q_heads + h) * kAbsorbMaxRanges + range] = make_float2(M_out, tot);
   }
 }
 
@@ -698,30 +700,42 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
 // ---------------------------------------------------------------------------------------------
 // 5. output: sum the ranges, normalise, project
 // ---------------------------------------------------------------------------------------------
-// ysum[b][h][i] = (sum over the sequence's ranges of y[b][range][h][i]) / softmax sum of (b, h)
+// ysum[b][h][i] = log-sum-exp merge over the sequence's ranges of y[b][range][h][i] (each relative to its
+// range's maximum), divided by the merged softmax sum; ml[b][h] receives the merged (max, sum)
 __global__ void __launch_bounds__(256)
-absorb_ysum_kernel(const float* __restrict__ y, const float2* __restrict__ ml, float* __restrict__ ysum,
-                   const int32_t* __restrict__ slots, const int32_t* __restrict__ lens, int max_batch, int capacity,
-                   int n_q_heads, int d_in, int range_tokens) {
+absorb_ysum_kernel(const float* __restrict__ y, const float2* __restrict__ ml_range, float2* __restrict__ ml,
+                   float* __restrict__ ysum, const int32_t* __restrict__ slots, const int32_t* __restrict__ lens,
+                   int max_batch, int capacity, int n_q_heads, int d_in, int range_tokens) {
   const int h = blockIdx.y, b = blockIdx.z;
   const int i4 = blockIdx.x * 256 + threadIdx.x;        // float4 index inside the row
-  if (i4 * 4 >= d_in) return;
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
+  const bool usable = slot >= 0 && slot < max_batch && len >= 1 && len <= capacity;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (slot >= 0 && slot < max_batch && len >= 1 && len <= capacity) {
+  float M = -INFINITY, L = 0.f;
+  if (usable) {
     const int n_ranges = (len + range_tokens - 1) / range_tokens;
-    const float4* src = reinterpret_cast<const float4*>(y + (((size_t)b * kAbsorbMaxRanges) * n_q_heads + h) * d_in) + i4;
-    const size_t range_stride4 = (size_t)n_q_heads * d_in / 4;
-    for (int r = 0; r < n_ranges; ++r) {
-      const float4 v = src[r * range_stride4];
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    const float2* mr = ml_range + ((size_t)b * n_q_heads + h) * kAbsorbMaxRanges;
+    for (int r = 0; r < n_ranges; ++r) M = fmaxf(M, mr[r].x);
+    if (M > -INFINITY && i4 * 4 < d_in) {
+      const float4* src = reinterpret_cast<const float4*>(y + (((size_t)b * kAbsorbMaxRanges) * n_q_heads + h) * d_in) + i4;
+      const size_t range_stride4 = (size_t)n_q_heads * d_in / 4;
+      for (int r = 0; r < n_ranges; ++r) {
+        const float2 m = mr[r];
+        const float w = exp2f(m.x - M);
+        L = fmaf(w, m.y, L);
+        const float4 v = src[r * range_stride4];
+        acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
+        acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+      }
+      const float inv = L > 0.f ? 1.f / L : 0.f;
+      acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    } else if (M > -INFINITY) {
+      for (int r = 0; r < n_ranges; ++r) L = fmaf(exp2f(mr[r].x - M), mr[r].y, L);
     }
-    const float L = ml[(size_t)b * n_q_heads + h].y;
-    const float inv = L > 0.f ? 1.f / L : 0.f;
-    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
   }
-  reinterpret_cast<float4*>(ysum + ((size_t)b * n_q_heads + h) * d_in)[i4] = acc;
+  if (blockIdx.x == 0 && threadIdx.x == 0) ml[(size_t)b * n_q_heads + h] = make_float2(M, L);
+  if (i4 * 4 < d_in) reinterpret_cast<float4*>(ysum + ((size_t)b * n_q_heads + h) * d_in)[i4] = acc;
 }
 
 constexpr int kOutRows = 16;     // output features per block
@@ -843,6 +857,7 @@ void absorbed_layout(int max_batch, int n_q_heads, int d_in, int capacity_tokens
   out->off_s = off; off = align(off + (uint64_t)max_batch * n_q_heads * out->l_cap * 4);
   out->off_p2 = off; off = align(off + (uint64_t)max_batch * out->nh2 * out->l_cap * 2);
   out->off_ml = off; off = align(off + (uint64_t)max_batch * n_q_heads * 8);
+  out->off_ml_range = off; off = align(off + (uint64_t)max_batch * n_q_heads * kAbsorbMaxRanges * 8);
   out->off_y = off; off = align(off + (uint64_t)max_batch * kAbsorbMaxRanges * n_q_heads * d_in * 4);
   out->off_ysum = off; off = align(off + (uint64_t)max_batch * n_q_heads * d_in * 4);
   out->total = off;
@@ -871,6 +886,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   float* S = reinterpret_cast<float*>(r.ws + lay.off_s);
   __nv_bfloat16* p2 = reinterpret_cast<__nv_bfloat16*>(r.ws + lay.off_p2);
   float2* ml = reinterpret_cast<float2*>(r.ws + lay.off_ml);
+  float2* ml_range = reinterpret_cast<float2*>(r.ws + lay.off_ml_range);
   float* y = reinterpret_cast<float*>(r.ws + lay.off_y);
   float* ysum = reinterpret_cast<float*>(r.ws + lay.off_ysum);
   cudaError_t e;
@@ -930,15 +946,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     if (ev) cudaEventRecord(ev[1], stream);
   }
 
-  // 3. softmax statistics and probabilities
-  {
-    dim3 grid(a.n_q_heads, a.batch);
-    absorb_softmax_kernel<<<grid, 256, 0, stream>>>(S, p2, ml, a.slots, a.lens, a.geom.max_batch, capacity,
-                                                    a.n_q_heads, lay.l_cap);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  }
-
-  // 4. probability-weighted inputs
+  // the V pass splits every sequence into token ranges; the softmax works range by range as well
   int range_tokens;
   {
     p.n_slices = (p.kc_total + 3) / 4;
@@ -949,6 +957,18 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     if (ranges < 1) ranges = 1;
     range_tokens = round_up((capacity + ranges - 1) / ranges, kPvTokens);
     if (range_tokens < 1024) range_tokens = 1024;
+  }
+
+  // 3. per range: maximum, sum, probabilities
+  {
+    dim3 grid(a.n_q_heads, a.batch, (capacity + range_tokens - 1) / range_tokens);
+    absorb_softmax_kernel<<<grid, 256, 0, stream>>>(S, p2, ml_range, a.slots, a.lens, a.geom.max_batch, capacity,
+                                                    a.n_q_heads, lay.l_cap, range_tokens);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+
+  // 4. probability-weighted inputs
+  {
     p.range_tokens = range_tokens;
     p.stage_bytes = kPvVBytes + (uint32_t)lay.nh2 * kRowBytes;
     p.n_stages = (int)(kSmemBudget / p.stage_bytes);
@@ -974,7 +994,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   // 5. sum the ranges, normalise, project
   {
     dim3 grid1((d_in / 4 + 255) / 256, a.n_q_heads, a.batch);
-    absorb_ysum_kernel<<<grid1, 256, 0, stream>>>(y, ml, ysum, a.slots, a.lens, a.geom.max_batch, capacity,
+    absorb_ysum_kernel<<<grid1, 256, 0, stream>>>(y, ml_range, ml, ysum, a.slots, a.lens, a.geom.max_batch, capacity,
                                                   a.n_q_heads, d_in, range_tokens);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     dim3 grid2(a.n_kv_heads, 128 / kOutRows, (a.batch * g + kOutPairs - 1) / kOutPairs);

@@ -23,6 +23,7 @@ struct AbsorbLayout {
   uint64_t off_s;   // fp32 [max_batch][n_q_heads][l_cap] scores (base-2 units)
   uint64_t off_p2;  // bf16 [max_batch * nh2][l_cap]     probabilities, split into two bf16 halves
   uint64_t off_ml;  // float2 [max_batch][n_q_heads]      (max, sum) of every head
+  uint64_t off_ml_range;  // float2 [max_batch][n_q_heads][ranges]  the same per token range
   uint64_t off_y;   // fp32 [max_batch][ranges][n_q_heads][D_in]  partial probability-weighted inputs
   uint64_t off_ysum; // fp32 [max_batch][n_q_heads][D_in]         their sum over ranges, divided by the softmax sum
   uint64_t total;
