@@ -32,7 +32,7 @@ namespace {
 constexpr int kChunk = 64;
 constexpr int kRowBytes = 128;
 constexpr int kMaxStages = 6;
-constexpr int kThreads = 256;            // warp 0 TMA, 1 MMA, 2 helper, 3 idle, 4..7 epilogue
+constexpr int kThreads = 256;            // warp 0 TMA, 1 MMA, 2 helper, 3 second TMA warp (V pass), 4..7 epilogue
 constexpr int kMaxBatchPerLaunch = 256;
 constexpr int kRunTokens = 64;
 constexpr int kSmemBudget = 200 * 1024;
@@ -321,8 +321,9 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
   const uint32_t page_bytes = box_tokens * kRowBytes;
   const uint32_t q_chunk_bytes = (uint32_t)p.nh2 * kRowBytes;
 
-  if (warp == 0) {
-    // =============================== TMA producer ===============================================
+  if (warp == 0 || warp == 3) {
+    // =============================== TMA producers (alternate stages) ===========================
+    const uint32_t mine = warp == 0 ? 0u : 1u;
     uint32_t it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
@@ -333,6 +334,7 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
       const int len = p.lens[b];
       const PageSet ps = lookup_pages(p, slot, len, tile * kScoreTokens, boxes, box_tokens, lane);
       for (int step = 0; step < n_steps; ++step, ++it) {
+        if ((it & 1u) != mine) continue;
         const uint32_t s = it % p.n_stages;
         const uint32_t ph = (it / p.n_stages) & 1u;
         const uint32_t full = smem_u32(&t.full_bar[s]);
@@ -547,18 +549,25 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
     return w;
   };
 
-  if (warp == 0) {
-    // =============================== TMA producer ===============================================
+  if (warp == 0 || warp == 3) {
+    // =============================== TMA producers ==============================================
+    // Two warps take alternate stages: what one thread must do per stage (block-table entries, run
+    // detection, two copies) is what limits a single producer here, not the memory system.
+    const uint32_t mine = warp == 0 ? 0u : 1u;
     uint32_t it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       const Work w = decode(item);
       const bool one_pool = w.kc0 + w.n_chunks <= p.kc_anchor || w.kc0 >= p.kc_anchor;
-      int raw_next = load_page(p, w.slot, w.len, w.t_begin, boxes, box_tokens, lane);
+      // block-table entries are requested one own stage (two stages) ahead of their use
+      const int first = ((it & 1u) == mine) ? 0 : 1;
+      int raw_next = first < w.n_steps
+                         ? load_page(p, w.slot, w.len, w.t_begin + first * kPvTokens, boxes, box_tokens, lane) : -1;
       for (int step = 0; step < w.n_steps; ++step, ++it) {
-        const int raw = raw_next;      // this stage's block-table entries were requested a stage ago
-        if (step + 1 < w.n_steps)
-          raw_next = load_page(p, w.slot, w.len, w.t_begin + (step + 1) * kPvTokens, boxes, box_tokens, lane);
+        if ((it & 1u) != mine) continue;
+        const int raw = raw_next;
+        if (step + 2 < w.n_steps)
+          raw_next = load_page(p, w.slot, w.len, w.t_begin + (step + 2) * kPvTokens, boxes, box_tokens, lane);
         const uint32_t s = it % p.n_stages;
         const uint32_t ph = (it / p.n_stages) & 1u;
         const uint32_t full = smem_u32(&t.full_bar[s]);
