@@ -84,6 +84,7 @@ struct Layer {
   void* v_side = nullptr;
   TcLayerMaps tc;     // tensor maps of the tensor-core path (valid when tc.ready)
   CUtensorMap stored_k, stored_v;   // tensor maps of the stored-head kernel (valid when ctx.stored_path == 1)
+  CUtensorMap stored_k_run, stored_v_run;   // the same pools in boxes of 64 token rows
 };
 
 }  // namespace
@@ -247,7 +248,8 @@ cudaError_t attend_stored_heads(echokv_ctx* c, const AttnArgs& a, const Layer& L
   c->launches += 1;
   if (c->stored_path == 1) {
     *item_tokens = item_tokens_ptr(c);
-    return launch_attn_stored_mma(a, L.stored_k, L.stored_v, n_heads, item_tokens_ptr(c), c->sm_count, s);
+    return launch_attn_stored_mma(a, L.stored_k, L.stored_v, L.stored_k_run, L.stored_v_run, n_heads,
+                                  item_tokens_ptr(c), c->sm_count, s);
   }
   return launch_attn_stored(a, L.k_pool, L.v_pool, width, n_heads, n_splits, s);
 }
@@ -364,7 +366,9 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
       if (width == 0) continue;
       const uint64_t rows = (uint64_t)cfg->n_pages * cfg->page_tokens;
       if (encode_pool_box_map(&L.stored_k, L.k_pool, width, rows, box_rows) != cudaSuccess ||
-          encode_pool_box_map(&L.stored_v, L.v_pool, width, rows, box_rows) != cudaSuccess) {
+          encode_pool_box_map(&L.stored_v, L.v_pool, width, rows, box_rows) != cudaSuccess ||
+          encode_pool_box_map(&L.stored_k_run, L.k_pool, width, rows, 64) != cudaSuccess ||
+          encode_pool_box_map(&L.stored_v_run, L.v_pool, width, rows, 64) != cudaSuccess) {
         delete c;
         return ECHOKV_ECUDA;
       }

@@ -115,6 +115,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 template <int G>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                       const __grid_constant__ CUtensorMap tm_k_run, const __grid_constant__ CUtensorMap tm_v_run,
                        const StoredParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
@@ -211,7 +212,15 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
       const int t_end = min(len, t_begin + item_tokens);
       const int n_iter = (t_end - t_begin + kStageTokens - 1) / kStageTokens;
       const int32_t* table = p.table + (size_t)slot * p.max_pages_per_seq;
+      // block-table entry of this lane's box of stage j (requested one stage ahead of its use)
+      auto load_page = [&](int j) {
+        const int tb = t_begin + j * kStageTokens + sub * rpb;
+        return (lane < n_boxes && tb < t_end) ? table[tb / p.page_tokens] : -1;
+      };
+      int page_next = load_page(0);
       for (int j = 0; j < n_iter; ++j, ++it) {
+        const int page = page_next;
+        if (j + 1 < n_iter) page_next = load_page(j + 1);
         const uint32_t s = it % kStages;
         const uint32_t ph = (it / kStages) & 1u;
         bool ok = true;
@@ -221,7 +230,6 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
         const int tb = t_begin + j * kStageTokens + sub * rpb;      // first token of this lane's box
         long long row = -1;
         if (lane < n_boxes && tb < t_end) {
-          const int page = table[tb / p.page_tokens];
           if (page < 0 || page >= p.n_pages) {
             report(p.status, ECHOKV_EBADPAGE);
           } else {
@@ -229,13 +237,21 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
           }
         }
         const uint32_t ok_mask = __ballot_sync(0xffffffffu, row >= 0);
+        // all boxes of the stage cached and consecutive in the pool: one 64-row copy per kind instead of one
+        // per page (lanes 0..3 hold the first page's row for the four kinds)
+        const long long row0 = __shfl_sync(0xffffffffu, row, kind);
+        const bool run = n_boxes > 4 && __all_sync(0xffffffffu, lane >= n_boxes || (row >= 0 && row == row0 + sub * rpb));
         const uint32_t full = smem_u32(&t.full_bar[s]);
         if (lane == 0) {
           t.box_ok[s] = ok_mask;
           mbar_arrive_expect_tx(full, __popc(ok_mask) * (uint32_t)rpb * 128u);
         }
         __syncwarp();
-        if (row >= 0) {
+        if (run) {
+          if (lane < 4)
+            tma_load_2d(stage_base + s * kStageBytes + kind * kBlockBytes, kind < 2 ? &tm_k_run : &tm_v_run,
+                        w.kvh * 128 + (kind & 1) * 64, (int)row, full);
+        } else if (row >= 0) {
           tma_load_2d(stage_base + s * kStageBytes + kind * kBlockBytes + sub * rpb * 128,
                       kind < 2 ? &tm_k : &tm_v, w.kvh * 128 + (kind & 1) * 64, (int)row, full);
         }
@@ -428,8 +444,8 @@ constexpr size_t stored_smem_bytes() {
 }
 
 template <int G>
-cudaError_t launch_g(const CUtensorMap& k, const CUtensorMap& v, const StoredParams& p, int sm_count,
-                     cudaStream_t stream) {
+cudaError_t launch_g(const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& k_run, const CUtensorMap& v_run,
+                     const StoredParams& p, int sm_count, cudaStream_t stream) {
   const size_t smem = stored_smem_bytes<G>();
   cudaError_t e = cudaFuncSetAttribute(attn_stored_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
@@ -447,7 +463,7 @@ cudaError_t launch_g(const CUtensorMap& k, const CUtensorMap& v, const StoredPar
   long long grid = (long long)resident * sm_count;
   if (grid > cap_items) grid = cap_items;
   if (grid < 1) grid = 1;
-  attn_stored_mma_kernel<G><<<(int)grid, kThreads, smem, stream>>>(k, v, p);
+  attn_stored_mma_kernel<G><<<(int)grid, kThreads, smem, stream>>>(k, v, k_run, v_run, p);
   return cudaGetLastError();
 }
 
@@ -462,7 +478,7 @@ bool stored_mma_supported(int dtype, int head_dim, int group, int max_batch) {
 int stored_rows_per_box(int page_tokens) { return page_tokens < kStageTokens ? page_tokens : kStageTokens; }
 
 cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, const CUtensorMap& v_map,
-                                   int n_heads, int32_t* item_tokens_slots, int sm_count, cudaStream_t stream) {
+                                   const CUtensorMap& k_run_map, const CUtensorMap& v_run_map, int n_heads, int32_t* item_tokens_slots, int sm_count, cudaStream_t stream) {
   if (n_heads == 0) return cudaSuccess;
   StoredParams p;
   p.q = reinterpret_cast<const __nv_bfloat16*>(a.q);
@@ -489,10 +505,10 @@ cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, 
     p.item_tokens_out = item_tokens_slots + launch;
     cudaError_t e;
     switch (g) {
-      case 1: e = launch_g<1>(k_map, v_map, p, sm_count, stream); break;
-      case 2: e = launch_g<2>(k_map, v_map, p, sm_count, stream); break;
-      case 4: e = launch_g<4>(k_map, v_map, p, sm_count, stream); break;
-      case 8: e = launch_g<8>(k_map, v_map, p, sm_count, stream); break;
+      case 1: e = launch_g<1>(k_map, v_map, k_run_map, v_run_map, p, sm_count, stream); break;
+      case 2: e = launch_g<2>(k_map, v_map, k_run_map, v_run_map, p, sm_count, stream); break;
+      case 4: e = launch_g<4>(k_map, v_map, k_run_map, v_run_map, p, sm_count, stream); break;
+      case 8: e = launch_g<8>(k_map, v_map, k_run_map, v_run_map, p, sm_count, stream); break;
       default: return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;

@@ -19,7 +19,8 @@ int stored_rows_per_box(int page_tokens);
 // split-K partial per (sequence, item, query head), item = a range of item_tokens tokens; the
 // kernel chooses item_tokens and writes it to item_tokens_slots[launch index] (one launch per
 // kStoredMaxBatchPerLaunch sequences) for the merge kernel.
+// k_run_map / v_run_map: the same pools in boxes of 64 token rows (used when a stage's pages are consecutive).
 cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, const CUtensorMap& v_map,
-                                   int n_heads, int32_t* item_tokens_slots, int sm_count, cudaStream_t stream);
+                                   const CUtensorMap& k_run_map, const CUtensorMap& v_run_map, int n_heads, int32_t* item_tokens_slots, int sm_count, cudaStream_t stream);
 
 }  // namespace echokv
