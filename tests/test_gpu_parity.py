@@ -294,3 +294,30 @@ def test_layer_step_replayed_from_a_cuda_graph(absorbed):
     assert torch.equal(replayed, direct)
     assert ctx.device_status() == binding.ECHOKV_OK
     case.close()
+
+
+def test_more_sequences_than_one_launch_indexes():
+    # the tcgen05 kernels index at most 256 sequences per launch and the stored-head kernel 512: a larger
+    # batch is split over several launches
+    w = synth.C2.replace(batch=600, context=48, n_kv_heads=2, n_q_heads=8, n_retained_heads=1)
+    rng = np.random.default_rng(3)
+    lens = [int(v) for v in rng.integers(1, 49, size=w.batch)]
+    case = Case(w, lens=lens, layers=[0, 1])
+    for path in (2, 3):
+        case.ctx.set_decode_path(path)
+        assert_parity(case.run(1), case.oracle(1), w.dtype, "batch 600, path %d" % path)
+    assert_parity(case.run(0), case.oracle(0), w.dtype, "batch 600, anchor")
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+def test_every_sequence_unusable_gives_zeros_and_a_status():
+    w = synth.C2.replace(batch=2, context=64)
+    case = Case(w, lens=[64, 64], layers=[0, 1])
+    dev = case.ctx.device
+    bad = torch.tensor([0, -5], dtype=torch.int32, device=dev)
+    for l in (0, 1):
+        out = case.ctx.decode_attention(l, case.q[l].to(dev), bad)
+        assert case.ctx.device_status() == binding.ECHOKV_EBADLENGTH
+        assert np.all(out.cpu().numpy() == 0.0)
+    case.close()
