@@ -28,12 +28,19 @@ Readings of points the paper leaves open (all listed in the design notes):
   * query head h attends KV head floor(h / (H_q / H_kv)) (contiguous groups).
   * every cached token, the newest included, is reconstructed alike, unless a
     sink / recent window is asked for (Section 5.1): those tokens keep all dims.
+  * the predictors see keys BEFORE the rotary position embedding (Section 3.2), so a
+    cache of such keys must be rotated when it is read: with rope_theta given, every
+    row t of K_tilde (retained, predicted or full-precision alike) is rotated to
+    position t (half-split pairing of feature j with j + d/2, frequencies
+    rope_theta^(-2j/d)) before q . k; q arrives already rotated; V is untouched.
+    Without rope_theta (all printed configurations) K_tilde is used as it is.
 
 Pins (tests/test_oracle_*.py): hand-computed softmax case, pure-python brute
 force, torch scaled_dot_product_attention (library routine) for the m = D and
 selector-weight cases, zero-weight closed forms, linearity, softmax shift /
-permutation / log-sum-exp merge invariants, and the paper's printed predictor
-shapes, ratios and parameter totals.  What stays "parity unpinned": nothing in
+permutation / log-sum-exp merge invariants, the paper's printed predictor
+shapes, ratios and parameter totals; for the rotation: hand values, the complex-
+number form, a library rotary routine, and the relative-position property.  What stays "parity unpinned": nothing in
 the paper prints a numeric attention output, and how well a *trained* W
 approximates the dropped cache cannot be checked without trained weights (it is
 not part of what the kernels compute).
@@ -131,15 +138,47 @@ def assemble_cache(c_local: np.ndarray, c_hat_drop: np.ndarray, n_kv_heads: int,
 
 
 # ----------------------------------------------------------------------------
+# Rotary position embedding applied when the cache is read (Section 3.2: the
+# predictor inputs, hence the cached keys, are keys prior to RoPE)
+# ----------------------------------------------------------------------------
+
+
+def rope_angles(L: int, d: int, rope_theta: float) -> np.ndarray:
+    """angle[t, j] = t * rope_theta^(-2 j / d) for positions t = 0..L-1 and the d/2
+    frequency indices j (RoFormer's frequencies; position = index in the cache)."""
+    if d % 2:
+        raise ValueError("head dim must be even")
+    j = np.arange(d // 2, dtype=np.float64)
+    inv_freq = np.power(float(rope_theta), -2.0 * j / d)
+    return np.arange(L, dtype=np.float64)[:, None] * inv_freq[None, :]
+
+
+def rotate_keys(K: np.ndarray, rope_theta: float) -> np.ndarray:
+    """Rotate row t of every head of K [L, H, d] to position t.  Feature j < d/2 is
+    paired with feature j + d/2 (the "rotate half" layout of the Llama family):
+        out[j]       = k[j] cos(a_tj) - k[j + d/2] sin(a_tj)
+        out[j + d/2] = k[j + d/2] cos(a_tj) + k[j] sin(a_tj)
+    """
+    K = np.asarray(K, dtype=np.float64)
+    L, H, d = K.shape
+    a = rope_angles(L, d, rope_theta)[:, None, :]              # [L, 1, d/2]
+    lo, hi = K[:, :, :d // 2], K[:, :, d // 2:]
+    return np.concatenate([lo * np.cos(a) - hi * np.sin(a), hi * np.cos(a) + lo * np.sin(a)], axis=2)
+
+
+# ----------------------------------------------------------------------------
 # Attention (Eq. 7; softmax as defined in the QK-KL appendix)
 # ----------------------------------------------------------------------------
 
 
-def attention_probabilities(q: np.ndarray, K: np.ndarray, scale: float | None = None
-                            ) -> np.ndarray:
-    """softmax_t(q_h . K[t, kv(h)] * scale) -> [H_q, L], kv(h) = h // (H_q / H_kv)."""
+def attention_probabilities(q: np.ndarray, K: np.ndarray, scale: float | None = None,
+                            rope_theta: float | None = None) -> np.ndarray:
+    """softmax_t(q_h . K[t, kv(h)] * scale) -> [H_q, L], kv(h) = h // (H_q / H_kv).
+    With rope_theta, K holds un-rotated keys and row t is rotated to position t first."""
     q = np.asarray(q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
+    if rope_theta is not None:
+        K = rotate_keys(K, rope_theta)
     H_q, d = q.shape
     L, H_kv, d2 = K.shape
     if d2 != d or H_q % H_kv != 0:
@@ -157,14 +196,14 @@ def attention_probabilities(q: np.ndarray, K: np.ndarray, scale: float | None = 
     return p
 
 
-def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None = None
-              ) -> np.ndarray:
+def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None = None,
+              rope_theta: float | None = None) -> np.ndarray:
     """Eq. 7 for one decode query per head: out[h] = sum_t p[h, t] V[t, kv(h), :].
 
     q [H_q, d], K and V [L, H_kv, d] -> [H_q, d].
     """
     V = np.asarray(V, dtype=np.float64)
-    p = attention_probabilities(q, K, scale)
+    p = attention_probabilities(q, K, scale, rope_theta)
     H_q = p.shape[0]
     g = H_q // V.shape[1]
     out = np.empty((H_q, V.shape[2]), dtype=np.float64)
@@ -174,14 +213,16 @@ def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None =
 
 
 def full_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
-                   n_kv_heads: int, scale: float | None = None) -> np.ndarray:
+                   n_kv_heads: int, scale: float | None = None,
+                   rope_theta: float | None = None) -> np.ndarray:
     """Attention of an anchor layer / the uncompressed mode: the stored cache
     [L, D] is used as it is (Eq. 7 with K_tilde = K, V_tilde = V)."""
     k_cache = np.asarray(k_cache, dtype=np.float64)
     v_cache = np.asarray(v_cache, dtype=np.float64)
     L, D = k_cache.shape
     d = D // n_kv_heads
-    return attention(q, k_cache.reshape(L, n_kv_heads, d), v_cache.reshape(L, n_kv_heads, d), scale)
+    return attention(q, k_cache.reshape(L, n_kv_heads, d), v_cache.reshape(L, n_kv_heads, d), scale,
+                     rope_theta)
 
 
 def decode_attention(q: np.ndarray,
@@ -189,8 +230,8 @@ def decode_attention(q: np.ndarray,
                      k_local: np.ndarray, v_local: np.ndarray,
                      Wk: np.ndarray, Wv: np.ndarray,
                      n_kv_heads: int, scale: float | None = None,
-                     bk: np.ndarray | None = None, bv: np.ndarray | None = None
-                     ) -> np.ndarray:
+                     bk: np.ndarray | None = None, bv: np.ndarray | None = None,
+                     rope_theta: float | None = None) -> np.ndarray:
     """One decode step of a compressed layer for one sequence.
 
     k_global, v_global [L, D]  full cache of the group's anchor layer   (Eq. 1)
@@ -198,7 +239,7 @@ def decode_attention(q: np.ndarray,
     Wk, Wv [D - m, D + m]      this layer's predictors                  (Eq. 3)
     q [H_q, d]                 the new token's queries
     Steps: predict the dropped dims (Eq. 3), rebuild K_tilde, V_tilde (Eq. 6),
-    attend (Eq. 7).  Returns [H_q, d].
+    (rotate K_tilde by position if rope_theta is given), attend (Eq. 7).  Returns [H_q, d].
     """
     k_global = np.asarray(k_global, dtype=np.float64)
     D = k_global.shape[1]
@@ -207,7 +248,7 @@ def decode_attention(q: np.ndarray,
     v_hat = reconstruct_dropped(Wv, v_global, v_local, bv)
     K_t = assemble_cache(k_local, k_hat, n_kv_heads, d)
     V_t = assemble_cache(v_local, v_hat, n_kv_heads, d)
-    return attention(q, K_t, V_t, scale)
+    return attention(q, K_t, V_t, scale, rope_theta)
 
 
 def decode_attention_query_heads(q: np.ndarray,
@@ -215,8 +256,8 @@ def decode_attention_query_heads(q: np.ndarray,
                                  k_local: np.ndarray, v_local: np.ndarray,
                                  Wk: np.ndarray, Wv: np.ndarray,
                                  n_kv_heads: int, query_heads, scale: float | None = None,
-                                 k_true_drop=None, v_true_drop=None, n_sink: int = 0, n_window: int = 0
-                                 ) -> dict[int, np.ndarray]:
+                                 k_true_drop=None, v_true_drop=None, n_sink: int = 0, n_window: int = 0,
+                                 rope_theta: float | None = None) -> dict[int, np.ndarray]:
     """The same quantity as decode_attention, for a chosen few query heads only.
 
     Heads are independent in Eq. 7 and each dropped flat dim is one row of W in
@@ -252,6 +293,8 @@ def decode_attention_query_heads(q: np.ndarray,
                 V_h = overlay_true_dims(V_h, np.asarray(v_true_drop, dtype=np.float64)[:, rows], keep)
         else:
             raise ValueError("m must be head-aligned for per-head evaluation")
+        if rope_theta is not None:
+            K_h = rotate_keys(K_h[:, None, :], rope_theta)[:, 0, :]
         s = (K_h @ q[h]) * scale
         e = np.exp(s - s.max())
         out[h] = (e / e.sum()) @ V_h
@@ -284,7 +327,8 @@ def overlay_true_dims(c_hat_drop: np.ndarray, c_true_drop: np.ndarray, keep: np.
 
 def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n_kv_heads: int,
                               k_true_drop, v_true_drop, n_sink: int, n_window: int,
-                              scale: float | None = None, bk=None, bv=None) -> np.ndarray:
+                              scale: float | None = None, bk=None, bv=None,
+                              rope_theta: float | None = None) -> np.ndarray:
     """decode_attention with the sink and recent-window tokens at full precision:
     for those tokens the dropped dims come from k_true_drop / v_true_drop ([L, D - m],
     the layer's own dims m..D-1), for all others from Eq. 3.  Returns [H_q, d]."""
@@ -297,7 +341,7 @@ def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n
     k_drop = overlay_true_dims(reconstruct_dropped(Wk, k_global, k_local, bk), k_true_drop, keep)
     v_drop = overlay_true_dims(reconstruct_dropped(Wv, v_global, v_local, bv), v_true_drop, keep)
     return attention(q, assemble_cache(k_local, k_drop, n_kv_heads, d),
-                     assemble_cache(v_local, v_drop, n_kv_heads, d), scale)
+                     assemble_cache(v_local, v_drop, n_kv_heads, d), scale, rope_theta)
 
 
 # ----------------------------------------------------------------------------
@@ -307,7 +351,7 @@ def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n
 
 def layer_step(layer: int, group_size: int, q: np.ndarray, caches_k, caches_v,
                weights_k, weights_v, n_kv_heads: int, m: int,
-               scale: float | None = None) -> np.ndarray:
+               scale: float | None = None, rope_theta: float | None = None) -> np.ndarray:
     """Decode attention of `layer` for one sequence.
 
     caches_k[l], caches_v[l]: [L, D] full (true) caches of every layer; a
@@ -315,11 +359,11 @@ def layer_step(layer: int, group_size: int, q: np.ndarray, caches_k, caches_v,
     weights_k[l], weights_v[l]: predictors of compressed layers.
     """
     if is_anchor_layer(layer, group_size):
-        return full_attention(q, caches_k[layer], caches_v[layer], n_kv_heads, scale)
+        return full_attention(q, caches_k[layer], caches_v[layer], n_kv_heads, scale, rope_theta)
     a = anchor_of(layer, group_size)
     return decode_attention(q, caches_k[a], caches_v[a],
                             np.asarray(caches_k[layer])[:, :m], np.asarray(caches_v[layer])[:, :m],
-                            weights_k[layer], weights_v[layer], n_kv_heads, scale)
+                            weights_k[layer], weights_v[layer], n_kv_heads, scale, rope_theta=rope_theta)
 
 
 # ----------------------------------------------------------------------------

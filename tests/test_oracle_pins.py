@@ -385,10 +385,10 @@ def test_planted_mistakes_are_caught(monkeypatch):
     def swapped_concat(c_global, c_local):                       # [local ; global]
         return np.concatenate([np.asarray(c_local, float), np.asarray(c_global, float)], axis=1)
 
-    def no_scale(q, K, scale=None):                              # forgot 1/sqrt(d)
+    def no_scale(q, K, scale=None, rope_theta=None):                              # forgot 1/sqrt(d)
         return good_probs(q, K, 1.0 if scale is None else scale)
 
-    def wrong_group(q, K, scale=None):                           # h % H_kv instead of h // g
+    def wrong_group(q, K, scale=None, rope_theta=None):                           # h % H_kv instead of h // g
         K = np.asarray(K, float)
         H_q, H_kv = np.asarray(q).shape[0], K.shape[1]
         g = H_q // H_kv
