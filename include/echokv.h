@@ -200,6 +200,27 @@ int echokv_side_buffer_bytes(const echokv_config* cfg, int n_sink, int n_window,
 int echokv_set_full_precision_window(echokv_ctx* ctx, int n_sink, int n_window, void* const* k_side,
                                      void* const* v_side);
 
+/* Rotary position embedding applied when the cache is read.  Section 3.2 feeds the predictors keys PRIOR
+ * to RoPE, so a backbone that follows the paper caches un-rotated keys and the rotation has to happen between
+ * reconstruction and q . k.  With a rotary table set, every attention call of the context rotates row t of
+ * K~ (stored, predicted, sink / window alike; anchor layers and echokv_full_attention included) to position
+ * t before the dot product:  feature j < head_dim/2 pairs with feature j + head_dim/2 (the Llama layout),
+ *     k'[j] = k[j] cos(a) - k[j + d/2] sin(a),  k'[j + d/2] = k[j + d/2] cos(a) + k[j] sin(a),
+ *     a = t * theta^(-2 j / head_dim),  t = index of the token in its sequence.
+ * q must arrive already rotated to its own position; V is never rotated.  The paper does not say where the
+ * rotation is re-applied at inference; this is the reading that keeps Eq. 3 on un-rotated keys.
+ *  - echokv_rope_table_bytes: size of the table, [head_dim / 2][max_pages_per_seq * page_tokens] pairs
+ *    (cos, sin) of fp32.
+ *  - echokv_set_rope: `table` is a device pointer of at least that size (16-byte aligned, borrowed until
+ *    echokv_destroy or until rope is switched off); the call enqueues one kernel on `stream` that fills it
+ *    (angles and sin / cos in fp64, rounded to fp32 once) and switches rotation on for later calls.
+ *    theta = 0 with table = NULL switches it off.  Not available together with the absorbed mode (a
+ *    rotation that depends on the token cannot be folded into the queries) nor with n_retained_dims that
+ *    split a head: EUNSUPPORTED.  Errors: EINVAL (theta < 1, misaligned), ECAPACITY, EUNSUPPORTED, ECUDA. */
+int echokv_rope_table_bytes(const echokv_config* cfg, uint64_t* out);
+int echokv_set_rope(echokv_ctx* ctx, double theta, void* table, uint64_t table_bytes, void* stream);
+int echokv_rope_enabled(const echokv_ctx* ctx);
+
 /* Absorbed-predictor decode mode.  Eq. 3 is linear, so Eq. 7 over a predicted head can be evaluated
  * without forming the predicted K and V:
  *     q . (Wk x_t) = (Wk^T q) . x_t          sum_t p_t (Wv x_t) = Wv (sum_t p_t x_t)
@@ -218,7 +239,7 @@ int echokv_set_full_precision_window(echokv_ctx* ctx, int n_sink, int n_window, 
  *    borrowed until echokv_destroy) and switches the context to the absorbed mode.
  *    Errors: EINVAL, EUNSUPPORTED, ECAPACITY (workspace too small), ECUDA.
  *  - echokv_set_decode_mode: 0 = explicit reconstruction, 1 = absorbed (EUNSUPPORTED before
- *    echokv_enable_absorbed).  Anchor layers and echokv_full_attention are not affected.
+ *    echokv_enable_absorbed, and while a rotary table is set).  Anchor layers and echokv_full_attention are not affected.
  *  In this mode a page id outside the pool is still reported (EBADPAGE) but the output of that
  *  sequence is unspecified. */
 int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out);

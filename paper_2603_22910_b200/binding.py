@@ -62,6 +62,9 @@ EXPORTS = {
     "echokv_side_buffer_bytes": (C.c_int, [C.POINTER(echokv_config), C.c_int, C.c_int, C.POINTER(C.c_uint64)]),
     "echokv_set_full_precision_window": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p),
                                                    C.POINTER(C.c_void_p)]),
+    "echokv_rope_table_bytes": (C.c_int, [C.POINTER(echokv_config), C.POINTER(C.c_uint64)]),
+    "echokv_set_rope": (C.c_int, [C.c_void_p, C.c_double, C.c_void_p, C.c_uint64, C.c_void_p]),
+    "echokv_rope_enabled": (C.c_int, [C.c_void_p]),
     "echokv_absorbed_workspace_bytes": (C.c_int, [C.POINTER(echokv_config), C.POINTER(C.c_uint64)]),
     "echokv_enable_absorbed": (C.c_int, [C.c_void_p, C.c_void_p, C.c_uint64]),
     "echokv_decode_mode": (C.c_int, [C.c_void_p]),
@@ -258,6 +261,22 @@ class Context:
                                                       C.cast(self._vs, C.POINTER(C.c_void_p))),
                "echokv_set_full_precision_window")
         self.n_sink, self.n_window = n_sink, n_window
+
+    def set_rope(self, theta: float, stream=None) -> None:
+        """Rotate cached keys to their positions when they are read (the cache holds un-rotated keys):
+        allocates the (cos, sin) table and has the library fill it.  theta = 0 switches it off."""
+        if not theta:
+            _check(lib().echokv_set_rope(self.handle, 0.0, None, 0, None), "echokv_set_rope")
+            self.rope_table = None
+            return
+        n = C.c_uint64(0)
+        _check(lib().echokv_rope_table_bytes(C.byref(self.cfg), C.byref(n)), "echokv_rope_table_bytes")
+        self.rope_table = self.torch.empty(n.value, dtype=self.torch.uint8, device=self.device)
+        _check(lib().echokv_set_rope(self.handle, float(theta), self.rope_table.data_ptr(), n.value,
+                                     _stream_handle(stream)), "echokv_set_rope")
+
+    def rope_enabled(self) -> bool:
+        return bool(lib().echokv_rope_enabled(self.handle))
 
     def enable_absorbed(self) -> None:
         """Allocate the absorbed mode's workspace and switch the context to that mode."""

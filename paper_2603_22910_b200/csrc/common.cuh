@@ -33,6 +33,14 @@ struct PageGeom {
   long long n_pages;
 };
 
+// Rotary position embedding applied when the cache is read (Section 3.2: the predictors, hence the
+// cache, hold keys prior to RoPE).  cs[j * stride + t] = (cos, sin)(t * theta^(-2 j / d)) for the d/2
+// frequency indices j and positions t < stride; feature j pairs with feature j + d/2.  cs == null: off.
+struct RopeTable {
+  const float2* cs = nullptr;
+  int stride = 0;
+};
+
 __device__ __forceinline__ void report(int32_t* status, int code) {
   // keep the first error; 0 means "none yet"
   atomicCAS(status, 0, code);

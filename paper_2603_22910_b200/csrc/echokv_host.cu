@@ -99,6 +99,7 @@ struct echokv_ctx {
   int path = 0;          // see echokv_decode_path
   bool tc_capable = false;
   int n_sink = 0, n_window = 0;   // tokens kept at full precision (0, 0 = none)
+  RopeTable rope;                 // rotate-on-read of un-rotated cached keys (off while rope.cs is null)
   bool absorbed_capable = false;  // shape served by the absorbed-predictor kernels
   int decode_mode = 0;            // 0 = explicit reconstruction (Eq. 3, 6, 7 as written), 1 = absorbed predictors
   unsigned char* ws_absorbed = nullptr;
@@ -154,6 +155,7 @@ AttnArgs attn_args(echokv_ctx* c, const void* q, const int32_t* slots, const int
   a.parts.o = reinterpret_cast<float*>(c->ws + c->d.off_o);
   a.parts.max_parts = c->d.max_parts;
   a.status = status_ptr(c);
+  a.rope = c->rope;
   return a;
 }
 
@@ -447,6 +449,41 @@ int echokv_set_full_precision_window(echokv_ctx* c, int n_sink, int n_window, vo
   return ECHOKV_OK;
 }
 
+int echokv_rope_table_bytes(const echokv_config* cfg, uint64_t* out) {
+  if (!out) return ECHOKV_EINVAL;
+  Derived d;
+  const int rc = derive(cfg, &d);
+  if (rc != ECHOKV_OK) return rc;
+  *out = (uint64_t)d.capacity * (uint64_t)(cfg->head_dim / 2) * sizeof(float2);
+  return ECHOKV_OK;
+}
+
+int echokv_set_rope(echokv_ctx* c, double theta, void* table, uint64_t table_bytes, void* stream) {
+  if (!c) return ECHOKV_EINVAL;
+  if (table == nullptr || !(theta > 0.0)) {      // off
+    if (table != nullptr || theta != 0.0) return ECHOKV_EINVAL;
+    c->rope = RopeTable();
+    return ECHOKV_OK;
+  }
+  if (!std::isfinite(theta) || theta < 1.0) return ECHOKV_EINVAL;
+  // a rotation that depends on the token cannot be folded into the queries
+  if (c->decode_mode == 1 || !c->d.head_aligned) return ECHOKV_EUNSUPPORTED;
+  uint64_t need = 0;
+  const int rc = echokv_rope_table_bytes(&c->cfg, &need);
+  if (rc != ECHOKV_OK) return rc;
+  if (table_bytes < need) return ECHOKV_ECAPACITY;
+  if (reinterpret_cast<uintptr_t>(table) % 16 != 0) return ECHOKV_EINVAL;
+  if (launch_rope_table(static_cast<float2*>(table), c->d.capacity, c->cfg.head_dim, theta,
+                        static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return ECHOKV_ECUDA;
+  c->launches += 1;
+  c->rope.cs = static_cast<const float2*>(table);
+  c->rope.stride = c->d.capacity;
+  return ECHOKV_OK;
+}
+
+int echokv_rope_enabled(const echokv_ctx* c) { return c && c->rope.cs != nullptr ? 1 : 0; }
+
 int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out) {
   if (!out) return ECHOKV_EINVAL;
   Derived d;
@@ -466,7 +503,7 @@ int echokv_enable_absorbed(echokv_ctx* c, void* workspace, uint64_t workspace_by
   uint64_t need = 0;
   const int rc = echokv_absorbed_workspace_bytes(&c->cfg, &need);
   if (rc != ECHOKV_OK) return rc;
-  if (!c->tc_capable) return ECHOKV_EUNSUPPORTED;
+  if (!c->tc_capable || c->rope.cs != nullptr) return ECHOKV_EUNSUPPORTED;
   if (workspace_bytes < need) return ECHOKV_ECAPACITY;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign != 0) return ECHOKV_EINVAL;
   c->ws_absorbed = static_cast<unsigned char*>(workspace);
@@ -482,7 +519,7 @@ int echokv_decode_mode(const echokv_ctx* c) { return c ? c->decode_mode : 0; }
 
 int echokv_set_decode_mode(echokv_ctx* c, int mode) {
   if (!c || (mode != 0 && mode != 1)) return ECHOKV_EINVAL;
-  if (mode == 1 && !c->absorbed_capable) return ECHOKV_EUNSUPPORTED;
+  if (mode == 1 && (!c->absorbed_capable || c->rope.cs != nullptr)) return ECHOKV_EUNSUPPORTED;
   c->decode_mode = mode;
   return ECHOKV_OK;
 }

@@ -16,7 +16,11 @@ struct AttnArgs {
   PageGeom geom;
   Partials parts;
   int32_t* status;
+  RopeTable rope;            // rotate every key row to its position before q . k (off unless set)
 };
+
+// Fill a rotary table (see RopeTable) for head_dim d and `stride` positions; angles in fp64.
+cudaError_t launch_rope_table(float2* table, int stride, int head_dim, double theta, cudaStream_t stream);
 
 // Append one token per sequence: writes the first `width` flat dims of k_new / v_new.
 cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int width, int D, const void* k_new,

@@ -67,6 +67,7 @@ struct PairParams {
   int run_pages;              // pages per tall box (kRunTokens / page_tokens), 1 = no tall boxes
   int n_sink, n_window;       // sink / recent-window tokens are not predicted (masked here)
   float scale_log2e;
+  RopeTable rope;             // read by the ROPE instantiations only
 };
 
 template <int G>
@@ -133,7 +134,9 @@ __device__ __forceinline__ Item decode_item(const PairSmemTail<G>& t, int item, 
   return it;
 }
 
-template <int G>
+// ROPE: the predicted key rows are rotated to their positions before q . k (Section 3.2: the predictors
+// produce keys prior to the rotary embedding).
+template <int G, bool ROPE>
 __global__ void __launch_bounds__(kThreads, 1)
 recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_constant__ CUtensorMap tm_anchor_v,
                   const __grid_constant__ CUtensorMap tm_local_k, const __grid_constant__ CUtensorMap tm_local_v,
@@ -363,6 +366,28 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
       float sc[G];
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) sc[gi] = 0.f;
+      if constexpr (ROPE) {
+        // this thread's row is token t_rot: features j and j + 64 of the head turn by t_rot * theta^(-2j/128)
+        const int t_rot = min(w.tile * kTileTokens + (int)rank * kCtaTokens + row, p.rope.stride - 1);
+        const float2* cs_row = p.rope.cs + t_rot;
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          float2 cs[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) cs[j] = cs_row[(size_t)(cb * 16 + j) * p.rope.stride];
+          float lo[16], hi[16];
+          tmem_ld16(lane_addr + sel * 128 + cb * 16, lo);
+          tmem_ld16(lane_addr + sel * 128 + 64 + cb * 16, hi);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float r_lo = lo[j] * cs[j].x - hi[j] * cs[j].y;
+            const float r_hi = hi[j] * cs[j].x + lo[j] * cs[j].y;
+#pragma unroll
+            for (int gi = 0; gi < G; ++gi)
+              sc[gi] = fmaf(r_hi, t.qs[sel][gi][64 + cb * 16 + j], fmaf(r_lo, t.qs[sel][gi][cb * 16 + j], sc[gi]));
+          }
+        }
+      } else {
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float v[32];
@@ -381,6 +406,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
           }
           sc[gi] = acc;
         }
+      }
       }
       const int token = (int)rank * kCtaTokens + row;        // token of the tile
       // predicted tokens only: sink and recent-window tokens are attended from the side buffers
@@ -503,12 +529,12 @@ constexpr size_t pair_smem_bytes() {
   return 1024 + (size_t)kStages * kStageBytes + sizeof(PairSmemTail<G>);
 }
 
-template <int G>
+template <int G, bool ROPE>
 cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUtensorMap& lv, const CUtensorMap& lkr,
                      const CUtensorMap& lvr, const CUtensorMap& lk8, const CUtensorMap& lv8, const TcLayerMaps& layer,
                      const PairParams& p, int n_clusters, cudaStream_t stream) {
   const size_t smem = pair_smem_bytes<G>();
-  cudaError_t e = cudaFuncSetAttribute(recon_pair_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(recon_pair_kernel<G, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -526,15 +552,23 @@ cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUt
   if (resident_pairs == 0) {
     cfg.gridDim = dim3(2 * n_clusters, 1, 1);
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, recon_pair_kernel<G>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, recon_pair_kernel<G, ROPE>, &cfg);
     if (e != cudaSuccess) return e;
     resident_pairs = n < 1 ? 1 : n;
   }
   if (n_clusters > resident_pairs) n_clusters = resident_pairs;
   cfg.gridDim = dim3(2 * n_clusters, 1, 1);
-  return cudaLaunchKernelEx(&cfg, recon_pair_kernel<G>, anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run,
+  return cudaLaunchKernelEx(&cfg, recon_pair_kernel<G, ROPE>, anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run,
                             anchor.v_pool_run, lkr, lvr, anchor.k_pool_run128, anchor.v_pool_run128, lk8, lv8,
                             layer.wk_half, layer.wv_half, p);
+}
+
+template <int G>
+cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUtensorMap& lv, const CUtensorMap& lkr,
+                     const CUtensorMap& lvr, const CUtensorMap& lk8, const CUtensorMap& lv8, const TcLayerMaps& layer,
+                     const PairParams& p, int n_clusters, cudaStream_t stream) {
+  if (p.rope.cs != nullptr) return launch_g<G, true>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
+  return launch_g<G, false>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
 }
 
 }  // namespace
@@ -566,6 +600,7 @@ cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLay
   p.scale_log2e = a.scale_log2e;
   p.n_sink = r.n_sink;
   p.n_window = r.n_window;
+  p.rope = a.rope;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;

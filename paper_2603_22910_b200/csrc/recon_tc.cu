@@ -64,6 +64,7 @@ struct TcParams {
   int run_pages;              // pages per tall box (kRunTokens / page_tokens), 1 = no tall boxes
   int n_sink, n_window;       // sink / recent-window tokens are not predicted (masked here)
   float scale_log2e;
+  RopeTable rope;             // read by the ROPE instantiations only
 };
 
 template <int G>
@@ -132,7 +133,9 @@ __device__ __forceinline__ Item decode_item(const TcSmemTail<G>& t, int item, in
   return it;
 }
 
-template <int G>
+// ROPE: the predicted key rows are rotated to their positions before q . k (Section 3.2: the predictors
+// produce keys prior to the rotary embedding).
+template <int G, bool ROPE>
 __global__ void __launch_bounds__(kThreads, 1)
 recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_constant__ CUtensorMap tm_anchor_v,
                 const __grid_constant__ CUtensorMap tm_local_k, const __grid_constant__ CUtensorMap tm_local_v,
@@ -353,6 +356,32 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
       for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
         for (int gi = 0; gi < G; ++gi) sc[hh][gi] = 0.f;
+      if constexpr (ROPE) {
+        // this thread's row is token t_rot: features j and j + 64 of a head turn by t_rot * theta^(-2j/128);
+        // 16 frequencies at a time, shared by the two heads of the pair
+        const int t_rot = min(w.tile * kTileTokens + half * 128 + row, p.rope.stride - 1);
+        const float2* cs_row = p.rope.cs + t_rot;
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          float2 cs[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) cs[j] = cs_row[(size_t)(cb * 16 + j) * p.rope.stride];
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            float lo[16], hi[16];
+            tmem_ld16(t_addr + hh * 128 + cb * 16, lo);
+            tmem_ld16(t_addr + hh * 128 + 64 + cb * 16, hi);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float r_lo = lo[j] * cs[j].x - hi[j] * cs[j].y;
+              const float r_hi = hi[j] * cs[j].x + lo[j] * cs[j].y;
+#pragma unroll
+              for (int gi = 0; gi < G; ++gi)
+                sc[hh][gi] = fmaf(r_hi, t.qs[hh][gi][64 + cb * 16 + j], fmaf(r_lo, t.qs[hh][gi][cb * 16 + j], sc[hh][gi]));
+            }
+          }
+        }
+      } else {
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
 #pragma unroll 1
@@ -374,6 +403,7 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
             sc[hh][gi] = acc;
           }
         }
+      }
       }
       const int token = half * 128 + row;
       // predicted tokens only: sink and recent-window tokens are attended from the side buffers
@@ -505,16 +535,25 @@ cudaError_t encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <int G>
+template <int G, bool ROPE>
 cudaError_t launch_g(const CUtensorMap& ak, const CUtensorMap& av, const CUtensorMap& lk, const CUtensorMap& lv,
                      const CUtensorMap& akr, const CUtensorMap& avr, const CUtensorMap& lkr, const CUtensorMap& lvr,
                      const CUtensorMap& wk, const CUtensorMap& wv, const TcParams& p, int grid,
                      cudaStream_t stream) {
   const size_t smem = tc_smem_bytes<G>();
-  cudaError_t e = cudaFuncSetAttribute(recon_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(recon_tc_kernel<G, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  recon_tc_kernel<G><<<grid, kThreads, smem, stream>>>(ak, av, lk, lv, akr, avr, lkr, lvr, wk, wv, p);
+  recon_tc_kernel<G, ROPE><<<grid, kThreads, smem, stream>>>(ak, av, lk, lv, akr, avr, lkr, lvr, wk, wv, p);
   return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_g(const CUtensorMap& ak, const CUtensorMap& av, const CUtensorMap& lk, const CUtensorMap& lv,
+                     const CUtensorMap& akr, const CUtensorMap& avr, const CUtensorMap& lkr, const CUtensorMap& lvr,
+                     const CUtensorMap& wk, const CUtensorMap& wv, const TcParams& p, int grid,
+                     cudaStream_t stream) {
+  if (p.rope.cs != nullptr) return launch_g<G, true>(ak, av, lk, lv, akr, avr, lkr, lvr, wk, wv, p, grid, stream);
+  return launch_g<G, false>(ak, av, lk, lv, akr, avr, lkr, lvr, wk, wv, p, grid, stream);
 }
 
 }  // namespace
@@ -621,6 +660,7 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
   p.scale_log2e = a.scale_log2e;
   p.n_sink = r.n_sink;
   p.n_window = r.n_window;
+  p.rope = a.rope;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;

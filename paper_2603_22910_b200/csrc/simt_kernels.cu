@@ -6,6 +6,29 @@
 namespace echokv {
 
 // ---------------------------------------------------------------------------------------------
+// Rotary table (Section 3.2: keys are cached un-rotated and rotated to their position when read)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) rope_table_kernel(float2* __restrict__ table, int stride, int head_dim,
+                                                         double theta) {
+  const long long n = (long long)(head_dim / 2) * stride;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
+    const int j = (int)(i / stride), t = (int)(i % stride);
+    const double angle = (double)t * pow(theta, -2.0 * (double)j / (double)head_dim);
+    double sn, cs;
+    sincos(angle, &sn, &cs);
+    table[i] = make_float2((float)cs, (float)sn);
+  }
+}
+
+cudaError_t launch_rope_table(float2* table, int stride, int head_dim, double theta, cudaStream_t stream) {
+  const long long n = (long long)(head_dim / 2) * stride;
+  long long blocks = (n + 255) / 256;
+  if (blocks > 4096) blocks = 4096;
+  rope_table_kernel<<<(int)blocks, 256, 0, stream>>>(table, stride, head_dim, theta);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Append (Section 3.1: the dropped dims of a compressed layer are simply not written; Eq. 2)
 // ---------------------------------------------------------------------------------------------
 template <typename T>
@@ -120,6 +143,15 @@ __global__ void __launch_bounds__(128) attn_stored_kernel(AttnArgs a, const T* _
 #pragma unroll
     for (int e = 0; e < EPL; ++e) qr[gi][e] = tmp[e] * a.scale_log2e;
   }
+  // rotate-on-read: q . (R_t k) = sum_j k_j (q_j cos + sgn_j q_partner(j) sin), partner = j +- DH/2, which
+  // lives 16 lanes away; sgn = +1 in the lower half of the head, -1 in the upper half
+  const bool rope = a.rope.cs != nullptr;
+  float qp[G][EPL];
+#pragma unroll
+  for (int gi = 0; gi < G; ++gi)
+#pragma unroll
+    for (int e = 0; e < EPL; ++e)
+      qp[gi][e] = (lane < 16 ? 1.f : -1.f) * __shfl_xor_sync(0xffffffffu, qr[gi][e], 16);
   float m[G], l[G], o[G][EPL];
 #pragma unroll
   for (int gi = 0; gi < G; ++gi) {
@@ -151,11 +183,21 @@ __global__ void __launch_bounds__(128) attn_stored_kernel(AttnArgs a, const T* _
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       if (!valid[u]) continue;   // warp-uniform
+      float2 cs[EPL];
+      if (rope) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) cs[e] = a.rope.cs[(size_t)((lane & 15) * EPL + e) * a.rope.stride + tb + u];
+      }
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) {
         float s = 0.f;
+        if (rope) {
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) s = fmaf(qr[gi][e], kx[u][e], s);
+          for (int e = 0; e < EPL; ++e) s = fmaf(kx[u][e], fmaf(qr[gi][e], cs[e].x, qp[gi][e] * cs[e].y), s);
+        } else {
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) s = fmaf(qr[gi][e], kx[u][e], s);
+        }
         s = warp_sum(s);
         const float m_new = fmaxf(m[gi], s);
         const float alpha = exp2f(m[gi] - m_new);
@@ -373,10 +415,22 @@ __global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r
     {
       const int t = tid % kSimtTileTokens;
       for (int gi = tid / kSimtTileTokens; gi < g; gi += 128 / kSimtTileTokens) {
-        float s = 0.f;
-#pragma unroll 8
-        for (int j = 0; j < DH; ++j) s = fmaf(sm.qs[gi][j], sm.Hs[t][j], s);
         const int t_seq = tile_t0 + t;     // predicted tokens only (sink / window tokens come from the side buffers)
+        float s = 0.f;
+        if (a.rope.cs != nullptr) {
+          // the predicted key row is rotated to position t_seq before q . k
+          const float2* cs = a.rope.cs + min(t_seq, a.rope.stride - 1);
+#pragma unroll 8
+          for (int j = 0; j < DH / 2; ++j) {
+            const float2 w = cs[(size_t)j * a.rope.stride];
+            const float k_lo = sm.Hs[t][j], k_hi = sm.Hs[t][j + DH / 2];
+            s = fmaf(sm.qs[gi][j], k_lo * w.x - k_hi * w.y, s);
+            s = fmaf(sm.qs[gi][j + DH / 2], k_hi * w.x + k_lo * w.y, s);
+          }
+        } else {
+#pragma unroll 8
+          for (int j = 0; j < DH; ++j) s = fmaf(sm.qs[gi][j], sm.Hs[t][j], s);
+        }
         sm.Ss[gi][t] = (t_seq >= predicted_lo(len, r.n_sink) && t_seq < predicted_hi(len, r.n_sink, r.n_window))
                            ? s : -INFINITY;
       }
@@ -642,15 +696,33 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     float acc[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
-    for (int j = 0; j < DH; j += Vec16<T>::N) {
-      float kv[Vec16<T>::N];
-      Vec16<T>::load(kr + j, kv);
+    if (a.rope.cs != nullptr) {
+      // the key row is rotated to its position before q . k
+      const float2* cs = a.rope.cs + (i < lo ? i : hi + (i - lo));
+      for (int j = 0; j < DH / 2; j += Vec16<T>::N) {
+        float k_lo[Vec16<T>::N], k_hi[Vec16<T>::N];
+        Vec16<T>::load(kr + j, k_lo);
+        Vec16<T>::load(kr + DH / 2 + j, k_hi);
 #pragma unroll
-      for (int gi = 0; gi < kMaxGroup; ++gi)
-        if (gi < g) {
+        for (int e = 0; e < Vec16<T>::N; ++e) {
+          const float2 w = cs[(size_t)(j + e) * a.rope.stride];
+          const float r_lo = k_lo[e] * w.x - k_hi[e] * w.y, r_hi = k_hi[e] * w.x + k_lo[e] * w.y;
 #pragma unroll
-          for (int e = 0; e < Vec16<T>::N; ++e) acc[gi] = fmaf(kv[e], qs[gi * DH + j + e], acc[gi]);
+          for (int gi = 0; gi < kMaxGroup; ++gi)
+            if (gi < g) acc[gi] = fmaf(r_hi, qs[gi * DH + DH / 2 + j + e], fmaf(r_lo, qs[gi * DH + j + e], acc[gi]));
         }
+      }
+    } else {
+      for (int j = 0; j < DH; j += Vec16<T>::N) {
+        float kv[Vec16<T>::N];
+        Vec16<T>::load(kr + j, kv);
+#pragma unroll
+        for (int gi = 0; gi < kMaxGroup; ++gi)
+          if (gi < g) {
+#pragma unroll
+            for (int e = 0; e < Vec16<T>::N; ++e) acc[gi] = fmaf(kv[e], qs[gi * DH + j + e], acc[gi]);
+          }
+      }
     }
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi)

@@ -55,6 +55,7 @@ struct StoredParams {
   int n_q_heads, n_heads;     // query heads in all; stored KV heads attended (0 .. n_heads - 1)
   int rows_per_box;           // token rows per TMA box: min(page_tokens, 64)
   float scale_log2e;
+  RopeTable rope;             // read by the ROPE instantiations only
 };
 
 template <int G>
@@ -112,7 +113,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int G>
+// two packed bf16 -> fp32
+__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+// (x0, x1) as a packed bf16 pair plus the packed pair of what the rounding dropped
+__device__ __forceinline__ void split_bf16(float x0, float x1, uint32_t& head, uint32_t& rest) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  head = *reinterpret_cast<const uint32_t*>(&h);
+  rest = pack_bf16(x0 - __low2float(h), x1 - __high2float(h));
+}
+
+// ROPE: every key row is rotated to its position before q . k (Section 3.2: the cache holds keys prior to
+// the rotary embedding).  The rotated rows are formed in fp32 from the fragments and fed to the tensor
+// cores as bf16 head + remainder, so the rotation costs no precision.
+template <int G, bool ROPE>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                        const __grid_constant__ CUtensorMap tm_k_run, const __grid_constant__ CUtensorMap tm_v_run,
@@ -339,6 +353,37 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
           for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) sc[nt][e] = 0.f;
+          if constexpr (ROPE) {
+            // fragment element (register i, half e) of step ks: token tile i >> 1, feature pair index
+            // jj = 16 ks + 8 (i & 1) + qd + e, which pairs feature jj (first 64-feature block) with jj + 64
+            const int tok_a = min(t0 + cw * kWarpTokens + (lane >> 2), p.rope.stride - 1);
+            const int tok_b = min(t0 + cw * kWarpTokens + 8 + (lane >> 2), p.rope.stride - 1);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const int c0 = ks * 2 + ((lane >> 3) & 1);
+              const uint32_t off = tok_k * 128 + ((c0 ^ (tok_k & 7)) << 4);
+              uint32_t a[4], b[4];
+              ldsm_x4(sb + off, a[0], a[1], a[2], a[3]);
+              ldsm_x4(sb + kBlockBytes + off, b[0], b[1], b[2], b[3]);
+              uint32_t lo_h[4], lo_r[4], hi_h[4], hi_r[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2* cs = p.rope.cs + (size_t)(ks * 16 + (i & 1) * 8 + qd) * p.rope.stride + ((i >> 1) ? tok_b : tok_a);
+                const float2 w0 = cs[0], w1 = cs[p.rope.stride];
+                const float a0 = bf16_lo(a[i]), a1 = bf16_hi(a[i]), b0 = bf16_lo(b[i]), b1 = bf16_hi(b[i]);
+                split_bf16(a0 * w0.x - b0 * w0.y, a1 * w1.x - b1 * w1.y, lo_h[i], lo_r[i]);
+                split_bf16(b0 * w0.x + a0 * w0.y, b1 * w1.x + a1 * w1.y, hi_h[i], hi_r[i]);
+              }
+              mma_m16n8k16_bf16(sc[0], qa0[ks], 0u, qa2[ks], 0u, lo_h[0], lo_h[1]);
+              mma_m16n8k16_bf16(sc[1], qa0[ks], 0u, qa2[ks], 0u, lo_h[2], lo_h[3]);
+              mma_m16n8k16_bf16(sc[0], qa0[ks + 4], 0u, qa2[ks + 4], 0u, hi_h[0], hi_h[1]);
+              mma_m16n8k16_bf16(sc[1], qa0[ks + 4], 0u, qa2[ks + 4], 0u, hi_h[2], hi_h[3]);
+              mma_m16n8k16_bf16(sc[0], qa0[ks], 0u, qa2[ks], 0u, lo_r[0], lo_r[1]);
+              mma_m16n8k16_bf16(sc[1], qa0[ks], 0u, qa2[ks], 0u, lo_r[2], lo_r[3]);
+              mma_m16n8k16_bf16(sc[0], qa0[ks + 4], 0u, qa2[ks + 4], 0u, hi_r[0], hi_r[1]);
+              mma_m16n8k16_bf16(sc[1], qa0[ks + 4], 0u, qa2[ks + 4], 0u, hi_r[2], hi_r[3]);
+            }
+          } else {
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             const int c0 = (ks & 3) * 2 + ((lane >> 3) & 1);
@@ -346,6 +391,7 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
             ldsm_x4(sb + (ks >> 2) * kBlockBytes + tok_k * 128 + ((c0 ^ (tok_k & 7)) << 4), r0, r1, r2, r3);
             mma_m16n8k16_bf16(sc[0], qa0[ks], 0u, qa2[ks], 0u, r0, r1);
             mma_m16n8k16_bf16(sc[1], qa0[ks], 0u, qa2[ks], 0u, r2, r3);
+          }
           }
 
           // ---- online softmax on row `row` (c0, c1 of both tiles) ----
@@ -443,18 +489,18 @@ constexpr size_t stored_smem_bytes() {
   return 1024 + (size_t)kStages * kStageBytes + sizeof(StoredSmemTail<G>);
 }
 
-template <int G>
+template <int G, bool ROPE>
 cudaError_t launch_g(const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& k_run, const CUtensorMap& v_run,
                      const StoredParams& p, int sm_count, cudaStream_t stream) {
   const size_t smem = stored_smem_bytes<G>();
-  cudaError_t e = cudaFuncSetAttribute(attn_stored_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attn_stored_mma_kernel<G, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
   // as many CTAs as stay resident, but never more than the items there can be
   static int resident = 0;   // per instantiation; the answer depends only on the kernel and the device type
   if (resident == 0) {
     int n = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_stored_mma_kernel<G>, kThreads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_stored_mma_kernel<G, ROPE>, kThreads, smem);
     if (e != cudaSuccess) return e;
     resident = n < 1 ? 1 : n;
   }
@@ -463,8 +509,15 @@ cudaError_t launch_g(const CUtensorMap& k, const CUtensorMap& v, const CUtensorM
   long long grid = (long long)resident * sm_count;
   if (grid > cap_items) grid = cap_items;
   if (grid < 1) grid = 1;
-  attn_stored_mma_kernel<G><<<(int)grid, kThreads, smem, stream>>>(k, v, k_run, v_run, p);
+  attn_stored_mma_kernel<G, ROPE><<<(int)grid, kThreads, smem, stream>>>(k, v, k_run, v_run, p);
   return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_g(const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& k_run, const CUtensorMap& v_run,
+                     const StoredParams& p, int sm_count, cudaStream_t stream) {
+  if (p.rope.cs != nullptr) return launch_g<G, true>(k, v, k_run, v_run, p, sm_count, stream);
+  return launch_g<G, false>(k, v, k_run, v_run, p, sm_count, stream);
 }
 
 }  // namespace
@@ -497,6 +550,7 @@ cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, 
   p.n_heads = n_heads;
   p.rows_per_box = stored_rows_per_box(a.geom.page_tokens);
   p.scale_log2e = a.scale_log2e;
+  p.rope = a.rope;
   const int g = a.n_q_heads / a.n_kv_heads;
   for (int b0 = 0, launch = 0; b0 < a.batch; b0 += kStoredMaxBatchPerLaunch, ++launch) {
     if (launch >= kStoredMaxLaunches) return cudaErrorInvalidValue;

@@ -16,8 +16,9 @@ class Case:
     """One workload resident on the GPU (all layers), plus the host copies the oracle reads."""
 
     def __init__(self, w: synth.Workload, lens=None, n_pages=None, layers=None, keep_host=True,
-                 biases=False, window=None):
-        """window = (n_sink, n_window): those tokens of every sequence keep all their dims (Section 5.1)."""
+                 biases=False, window=None, rope=None):
+        """window = (n_sink, n_window): those tokens of every sequence keep all their dims (Section 5.1).
+        rope = theta: the cache holds un-rotated keys that are rotated to their positions when read."""
         self.w = w
         self.lens = list(lens) if lens is not None else [w.context] * w.batch
         assert len(self.lens) == w.batch and max(self.lens) <= w.context
@@ -30,6 +31,9 @@ class Case:
         self.window = window
         if window:
             self.ctx.set_full_precision_window(*window)
+        self.rope = rope
+        if rope:
+            self.ctx.set_rope(rope)
         self.true_drop = {}  # (layer, kind, b) -> the layer's own dims m..D-1 [len_b, D - m] (window tests)
         self.host = {}       # (layer, kind, b) -> stored-precision tensor [len_b, width]
         self.weights = {}    # layer -> (Wk, Wv, bk, bv) device tensors
@@ -110,9 +114,9 @@ class Case:
             if w.is_anchor(layer):
                 kk, vv = self._stored(layer, "k", b), self._stored(layer, "v", b)
                 if query_heads is None:
-                    res[b] = O.full_attention(qn[b], kk, vv, w.n_kv_heads)
+                    res[b] = O.full_attention(qn[b], kk, vv, w.n_kv_heads, rope_theta=self.rope)
                 else:
-                    full = O.full_attention(qn[b], kk, vv, w.n_kv_heads)
+                    full = O.full_attention(qn[b], kk, vv, w.n_kv_heads, rope_theta=self.rope)
                     for h in query_heads:
                         res[(b, h)] = full[h]
                 continue
@@ -128,11 +132,14 @@ class Case:
                 vt = O.widen(synth.to_numpy_stored(self.true_drop[(layer, "v", b)]))
                 assert query_heads is None
                 res[b] = O.decode_attention_windowed(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, kt, vt,
-                                                     self.window[0], self.window[1], bk=bk, bv=bv)
+                                                     self.window[0], self.window[1], bk=bk, bv=bv,
+                                                     rope_theta=self.rope)
             elif query_heads is None:
-                res[b] = O.decode_attention(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv)
+                res[b] = O.decode_attention(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv,
+                                            rope_theta=self.rope)
             else:
-                per = O.decode_attention_query_heads(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, query_heads)
+                per = O.decode_attention_query_heads(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, query_heads,
+                                                     rope_theta=self.rope)
                 for h, v in per.items():
                     res[(b, h)] = v
         return res

@@ -1,0 +1,112 @@
+"""GPU parity with rotate-on-read (Section 3.2: the predictors, hence the cache, hold keys prior to the
+rotary position embedding): every kernel family that computes q . k against the oracle's rotation."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_22910_b200 import binding, build, synth
+from tests.harness import Case, assert_parity, errors
+
+pytestmark = pytest.mark.gpu
+
+THETA = 10000.0
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.lib()
+
+
+CASES = [
+    # name, base, overrides, lens, window
+    ("tiny_fp32_d64", synth.C0, {}, None, None),
+    ("fp32_d128_gqa2", synth.C0, dict(n_q_heads=8, n_kv_heads=4, head_dim=128, n_retained_heads=1, batch=2,
+                                      context=150), [150, 64], None),
+    ("c2_shape", synth.C2, dict(batch=3, context=1000), [1000, 517, 256], None),
+    ("c1_shape", synth.C1, dict(batch=2, context=700), [700, 333], None),
+    ("c2_pages64_random", synth.C2, dict(batch=2, context=600, page_tokens=64, random_pages=True), [600, 65], None),
+    ("gqa8", synth.C2, dict(n_q_heads=32, n_kv_heads=4, n_retained_heads=1, batch=1, context=300), [300], None),
+    ("ragged_many_tiles", synth.C2, dict(batch=5, context=2000, random_pages=True), [2000, 129, 128, 1153, 1], None),
+    ("c2_window", synth.C2, dict(batch=3, context=1000, random_pages=True), [1000, 517, 100], (4, 128)),
+    ("fp32_d64_window", synth.C0, dict(batch=2, context=200), [200, 50], (2, 16)),
+    ("bf16_d64", synth.C0, dict(dtype="bf16", batch=2, context=200), [200, 77], None),
+]
+
+
+@pytest.mark.parametrize("name,base,over,lens,window", CASES, ids=[c[0] for c in CASES])
+def test_rope_against_oracle(name, base, over, lens, window):
+    w = base.replace(**over)
+    case = Case(w, lens=lens, layers=[0, 1], window=window, rope=THETA)
+    assert case.ctx.rope_enabled()
+    paths = [1, 2, 3] if case.ctx.decode_path() >= 2 else [1]
+    stored_paths = [0, 1] if case.ctx.stored_path() == 1 else [0]
+    ref0, ref1 = case.oracle(0), case.oracle(1)
+    for stored_path in stored_paths:
+        case.ctx.set_stored_path(stored_path)
+        out0 = case.run(0)
+        assert_parity(out0, ref0, w.dtype, "%s anchor stored_path %d" % (name, stored_path))
+        np.testing.assert_array_equal(case.run(0, full=True), out0)
+        for path in paths:
+            case.ctx.set_decode_path(path)
+            assert_parity(case.run(1), ref1, w.dtype, "%s path %d stored_path %d" % (name, path, stored_path))
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    # switched off again, the context computes the un-rotated result
+    case.ctx.set_rope(0)
+    assert not case.ctx.rope_enabled()
+    case.rope = None
+    assert_parity(case.run(1), case.oracle(1), w.dtype, name + " rope off")
+    assert errors(case.oracle(1), ref1)[1] > 1e-2          # (and the rotation is no small change)
+    case.close()
+
+
+def test_rope_and_absorbed_mode_exclude_each_other():
+    w = synth.C2.replace(batch=1, context=300)
+    case = Case(w, lens=[300], layers=[1], rope=THETA)
+    n = C.c_uint64(0)
+    assert binding.lib().echokv_absorbed_workspace_bytes(C.byref(case.cfg), C.byref(n)) == binding.ECHOKV_OK
+    buf = torch.empty(n.value, dtype=torch.uint8, device="cuda")
+    assert binding.lib().echokv_enable_absorbed(case.ctx.handle, buf.data_ptr(), n.value) == binding.ECHOKV_EUNSUPPORTED
+    case.ctx.set_rope(0)
+    case.ctx.enable_absorbed()
+    with pytest.raises(binding.EchoKVError) as e:
+        case.ctx.set_rope(THETA)
+    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
+    case.ctx.set_decode_mode(0)
+    case.ctx.set_rope(THETA)
+    with pytest.raises(binding.EchoKVError) as e:
+        case.ctx.set_decode_mode(1)
+    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
+    case.rope = THETA
+    assert_parity(case.run(1), case.oracle(1), w.dtype, "explicit mode with rope after the switches")
+    case.close()
+
+
+def test_rope_argument_checks():
+    w = synth.C0
+    case = Case(w, layers=[1])
+    lib, h = binding.lib(), case.ctx.handle
+    n = C.c_uint64(0)
+    assert lib.echokv_rope_table_bytes(C.byref(case.cfg), C.byref(n)) == binding.ECHOKV_OK
+    assert n.value == w.pages_per_seq * w.page_tokens * (w.head_dim // 2) * 8
+    buf = torch.empty(n.value + 16, dtype=torch.uint8, device="cuda")
+    assert lib.echokv_set_rope(h, 10000.0, buf.data_ptr(), n.value - 1, None) == binding.ECHOKV_ECAPACITY
+    assert lib.echokv_set_rope(h, 0.5, buf.data_ptr(), n.value, None) == binding.ECHOKV_EINVAL
+    assert lib.echokv_set_rope(h, float("nan"), buf.data_ptr(), n.value, None) == binding.ECHOKV_EINVAL
+    assert lib.echokv_set_rope(h, 10000.0, buf.data_ptr() + 8, n.value, None) == binding.ECHOKV_EINVAL
+    assert lib.echokv_set_rope(h, 10000.0, None, 0, None) == binding.ECHOKV_EINVAL
+    assert not case.ctx.rope_enabled()
+    assert lib.echokv_set_rope(h, 10000.0, buf.data_ptr(), n.value, None) == binding.ECHOKV_OK
+    assert case.ctx.rope_enabled()
+    # the table the library wrote: (cos, sin)(t * theta^(-2j/d)), [d/2][capacity]
+    torch.cuda.synchronize()
+    tab = buf[: n.value].view(torch.float32).view(w.head_dim // 2, -1, 2).cpu().numpy().astype(np.float64)
+    t = np.arange(tab.shape[1], dtype=np.float64)
+    for j in (0, 1, w.head_dim // 2 - 1):
+        a = t * 10000.0 ** (-2.0 * j / w.head_dim)
+        np.testing.assert_allclose(tab[j, :, 0], np.cos(a), atol=1e-7)
+        np.testing.assert_allclose(tab[j, :, 1], np.sin(a), atol=1e-7)
+    case.close()
