@@ -295,12 +295,14 @@ def oracle_threads():
 
 def oracle_layer(inputs, w, state=None, layer=None, b=None):
     from oracle import echokv_oracle as O
+    rope = getattr(state, "rope", None) or None
     if len(inputs) == 3:
-        return O.full_attention(inputs[0], inputs[1], inputs[2], w.n_kv_heads)
+        return O.full_attention(inputs[0], inputs[1], inputs[2], w.n_kv_heads, rope_theta=rope)
     if state is not None and state.window:
         return O.decode_attention_windowed(*inputs, w.n_kv_heads, state.true_dropped(layer, "k", b),
-                                           state.true_dropped(layer, "v", b), state.window[0], state.window[1])
-    return O.decode_attention(*inputs, n_kv_heads=w.n_kv_heads)
+                                           state.true_dropped(layer, "v", b), state.window[0], state.window[1],
+                                           rope_theta=rope)
+    return O.decode_attention(*inputs, n_kv_heads=w.n_kv_heads, rope_theta=rope)
 
 
 def time_oracle(state, step_layers, budget_s):
@@ -362,7 +364,8 @@ def run_reference(args):
         d = w.head_dim
 
         def run(n_kv):   # the first n_kv KV heads of the stored cache
-            return O.full_attention(q[: n_kv * g], kg[:, : n_kv * d], vg[:, : n_kv * d], n_kv)
+            return O.full_attention(q[: n_kv * g], kg[:, : n_kv * d], vg[:, : n_kv * d], n_kv,
+                                    rope_theta=args.rope or None)
     else:
         kl = O.widen(st(synth.layer_cache(w, layer, "k", 0, width=w.m)))
         vl = O.widen(st(synth.layer_cache(w, layer, "v", 0, width=w.m)))
@@ -373,7 +376,7 @@ def run_reference(args):
 
         def run(n_kv):   # the first n_kv dropped KV heads (the retained ones cost next to nothing)
             return O.decode_attention_query_heads(q, kg, vg, kl, vl, Wk, Wv, n_kv_heads=w.n_kv_heads,
-                                                  query_heads=heads[: n_kv * g])
+                                                  query_heads=heads[: n_kv * g], rope_theta=args.rope or None)
     t0 = time.perf_counter()
     run(1)
     t_head = time.perf_counter() - t0
@@ -512,6 +515,9 @@ def run_ours(args):
     absorbed = args.decode_mode == "absorbed" and not full
     if absorbed:
         ctx.enable_absorbed()
+    st.rope = args.rope
+    if args.rope:
+        ctx.set_rope(args.rope)      # (the library refuses it together with the absorbed mode)
     last = [l for l, a in step_layers if a][-1]
 
     def attend(l):
@@ -680,6 +686,7 @@ def run_ours(args):
         "decode_mode": "absorbed" if absorbed else "explicit",
         "cuda_graph": {"ms_per_step_eager": ms_eager / args.steps} if args.graph else None,
         "full_precision_tokens": {"sink": window[0], "window": window[1]} if window else None,
+        "rope_theta": args.rope or None,
         "input_generation_s": st.gen_s,
     }
 
@@ -725,6 +732,8 @@ def main():
                     help="time the step replayed from a CUDA graph (launch gaps removed) instead of eager launches")
     ap.add_argument("--window", default="", help="n_sink,n_window: tokens kept at full precision, e.g. 4,128 (the "
                                                  "paper's setting); default none, as the benchmark configs state")
+    ap.add_argument("--rope", type=float, default=0.0, help="theta of a rotary embedding applied when the cache is "
+                    "read (the cache then holds un-rotated keys); 0 = none, as in the paper's configurations")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")

@@ -36,10 +36,16 @@ struct PageGeom {
 // Rotary position embedding applied when the cache is read (Section 3.2: the predictors, hence the
 // cache, hold keys prior to RoPE).  cs[j * stride + t] = (cos, sin)(t * theta^(-2 j / d)) for the d/2
 // frequency indices j and positions t < stride; feature j pairs with feature j + d/2.  cs == null: off.
+// The same angles factored as position = 16 u + r:  coarse[u * (d/2) + j] = (cos, sin)(16 u * w_j) for
+// u < stride / 16 and fine[r * (d/2) + j] = (cos, sin)(r * w_j) for r < 16 (the stored-head kernel multiplies
+// the two: a 64-token stage then needs 2 KiB of table instead of 32 KiB).
 struct RopeTable {
   const float2* cs = nullptr;
   int stride = 0;
+  const float2* coarse = nullptr;
+  const float2* fine = nullptr;
 };
+constexpr int kRopeFineRows = 16;
 
 __device__ __forceinline__ void report(int32_t* status, int code) {
   // keep the first error; 0 means "none yet"

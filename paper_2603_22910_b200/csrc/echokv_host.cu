@@ -454,7 +454,7 @@ int echokv_rope_table_bytes(const echokv_config* cfg, uint64_t* out) {
   Derived d;
   const int rc = derive(cfg, &d);
   if (rc != ECHOKV_OK) return rc;
-  *out = (uint64_t)d.capacity * (uint64_t)(cfg->head_dim / 2) * sizeof(float2);
+  *out = (uint64_t)rope_table_pairs(d.capacity, cfg->head_dim) * sizeof(float2);
   return ECHOKV_OK;
 }
 
@@ -476,9 +476,8 @@ int echokv_set_rope(echokv_ctx* c, double theta, void* table, uint64_t table_byt
   if (launch_rope_table(static_cast<float2*>(table), c->d.capacity, c->cfg.head_dim, theta,
                         static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return ECHOKV_ECUDA;
-  c->launches += 1;
-  c->rope.cs = static_cast<const float2*>(table);
-  c->rope.stride = c->d.capacity;
+  c->launches += 3;
+  c->rope = rope_table_view(static_cast<const float2*>(table), c->d.capacity, c->cfg.head_dim);
   return ECHOKV_OK;
 }
 

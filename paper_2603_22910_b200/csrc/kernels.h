@@ -19,8 +19,12 @@ struct AttnArgs {
   RopeTable rope;            // rotate every key row to its position before q . k (off unless set)
 };
 
-// Fill a rotary table (see RopeTable) for head_dim d and `stride` positions; angles in fp64.
-cudaError_t launch_rope_table(float2* table, int stride, int head_dim, double theta, cudaStream_t stream);
+// The three parts of a rotary table (see RopeTable) live in one buffer: [d/2][stride], then [stride/16][d/2],
+// then [16][d/2] pairs.  rope_table_pairs: pairs in all; rope_table_view: the RopeTable over such a buffer;
+// launch_rope_table: fill it (angles and sin / cos in fp64; three launches).
+size_t rope_table_pairs(int stride, int head_dim);
+RopeTable rope_table_view(const float2* buffer, int stride, int head_dim);
+cudaError_t launch_rope_table(float2* buffer, int stride, int head_dim, double theta, cudaStream_t stream);
 
 // Append one token per sequence: writes the first `width` flat dims of k_new / v_new.
 cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int width, int D, const void* k_new,

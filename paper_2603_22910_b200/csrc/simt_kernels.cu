@@ -8,24 +8,52 @@ namespace echokv {
 // ---------------------------------------------------------------------------------------------
 // Rotary table (Section 3.2: keys are cached un-rotated and rotated to their position when read)
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) rope_table_kernel(float2* __restrict__ table, int stride, int head_dim,
-                                                         double theta) {
-  const long long n = (long long)(head_dim / 2) * stride;
+// out[i] = (cos, sin)(pos * theta^(-2 j / d)); layout 0: i = j * n_pos + pos (positions 0 .. n_pos-1);
+// layout 1: i = u * (d/2) + j with pos = pos_step * u.
+__global__ void __launch_bounds__(256) rope_table_kernel(float2* __restrict__ out, long long n, int n_pos,
+                                                         int head_dim, double theta, int layout, int pos_step) {
+  const int half = head_dim / 2;
   for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
-    const int j = (int)(i / stride), t = (int)(i % stride);
-    const double angle = (double)t * pow(theta, -2.0 * (double)j / (double)head_dim);
+    int j, pos;
+    if (layout == 0) { j = (int)(i / n_pos); pos = (int)(i % n_pos); }
+    else { j = (int)(i % half); pos = (int)(i / half) * pos_step; }
+    const double angle = (double)pos * pow(theta, -2.0 * (double)j / (double)head_dim);
     double sn, cs;
     sincos(angle, &sn, &cs);
-    table[i] = make_float2((float)cs, (float)sn);
+    out[i] = make_float2((float)cs, (float)sn);
   }
 }
 
-cudaError_t launch_rope_table(float2* table, int stride, int head_dim, double theta, cudaStream_t stream) {
-  const long long n = (long long)(head_dim / 2) * stride;
-  long long blocks = (n + 255) / 256;
-  if (blocks > 4096) blocks = 4096;
-  rope_table_kernel<<<(int)blocks, 256, 0, stream>>>(table, stride, head_dim, theta);
-  return cudaGetLastError();
+size_t rope_table_pairs(int stride, int head_dim) {
+  const size_t half = head_dim / 2;
+  return half * stride + (size_t)(stride / kRopeFineRows) * half + (size_t)kRopeFineRows * half;
+}
+
+RopeTable rope_table_view(const float2* buffer, int stride, int head_dim) {
+  const size_t half = head_dim / 2;
+  RopeTable t;
+  t.cs = buffer;
+  t.stride = stride;
+  t.coarse = buffer + half * stride;
+  t.fine = t.coarse + (size_t)(stride / kRopeFineRows) * half;
+  return t;
+}
+
+cudaError_t launch_rope_table(float2* buffer, int stride, int head_dim, double theta, cudaStream_t stream) {
+  const RopeTable t = rope_table_view(buffer, stride, head_dim);
+  const long long half = head_dim / 2;
+  const long long n[3] = {half * stride, (long long)(stride / kRopeFineRows) * half, (long long)kRopeFineRows * half};
+  float2* dst[3] = {buffer, const_cast<float2*>(t.coarse), const_cast<float2*>(t.fine)};
+  const int layout[3] = {0, 1, 1}, step[3] = {1, kRopeFineRows, 1};
+  for (int k = 0; k < 3; ++k) {
+    if (n[k] == 0) continue;
+    long long blocks = (n[k] + 255) / 256;
+    if (blocks > 4096) blocks = 4096;
+    rope_table_kernel<<<(int)blocks, 256, 0, stream>>>(dst[k], n[k], stride, head_dim, theta, layout[k], step[k]);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 // ---------------------------------------------------------------------------------------------

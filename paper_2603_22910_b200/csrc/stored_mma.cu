@@ -28,7 +28,13 @@ namespace echokv {
 
 namespace {
 
-constexpr int kStages = 3;
+constexpr int kStages = 3;                           // stage barriers in shared memory (stages in use: StoredStages)
+constexpr int kFineRowPairs = 72;                    // (cos, sin) pairs per row of the in-CTA offset table: 64 + 8 of
+                                                     // padding, so that two rows fill the 32 banks exactly
+// Stages of 32 KiB per CTA.  The rotating variant also keeps a 9 KiB table; with many query heads per KV
+// head (a large merge area) it runs on two stages so that two CTAs still fit an SM.
+template <int G, bool ROPE>
+struct StoredStages { static constexpr int value = (ROPE && G >= 4) ? 2 : 3; };
 constexpr int kStageTokens = 64;
 constexpr int kBlockBytes = kStageTokens * 128;      // 64 token rows x 64 features (128 bytes)
 constexpr int kStageBytes = 4 * kBlockBytes;         // K lo, K hi, V lo, V hi
@@ -134,7 +140,14 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  StoredSmemTail<G>& t = *reinterpret_cast<StoredSmemTail<G>*>(smem + kStages * kStageBytes);
+  constexpr int NS = StoredStages<G, ROPE>::value;
+  StoredSmemTail<G>& t = *reinterpret_cast<StoredSmemTail<G>*>(smem + NS * kStageBytes);
+  // ROPE: (cos, sin)(r * w_j) for the 16 offsets r inside a warp's token slice, rows padded (see kFineRowPairs)
+  float2* fine = reinterpret_cast<float2*>(smem + NS * kStageBytes + ((sizeof(StoredSmemTail<G>) + 15) / 16) * 16);
+  if constexpr (ROPE) {
+    for (int i = threadIdx.x; i < kRopeFineRows * 64; i += kThreads)
+      fine[(i >> 6) * kFineRowPairs + (i & 63)] = p.rope.fine[i];
+  }
   const uint32_t stage_base = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &t.abort_flag;
@@ -145,7 +158,7 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
     t.total_tokens = 0ull;
     t.abort_flag = 0;
     t.cum_items[0] = 0;
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < NS; ++s) {
       mbar_init(smem_u32(&t.full_bar[s]), 1);
       mbar_init(smem_u32(&t.empty_bar[s]), kConsumers);
     }
@@ -212,9 +225,9 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
   if (warp == 0) {
     // =============================== TMA producer ===============================================
     uint32_t it = 0;
-    uint32_t issued[kStages];
+    uint32_t issued[NS];
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) issued[s] = 0;
+    for (int s = 0; s < NS; ++s) issued[s] = 0;
     bool alive = true;
     const int sub = lane >> 2, kind = lane & 3;    // box row group inside the stage; K lo, K hi, V lo, V hi
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
@@ -235,8 +248,8 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
       for (int j = 0; j < n_iter; ++j, ++it) {
         const int page = page_next;
         if (j + 1 < n_iter) page_next = load_page(j + 1);
-        const uint32_t s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1u;
+        const uint32_t s = it % NS;
+        const uint32_t ph = (it / NS) & 1u;
         bool ok = true;
         if (lane == 0) ok = mbar_wait(smem_u32(&t.empty_bar[s]), ph ^ 1u, abort_flag, p.status);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -275,8 +288,8 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
     if (!alive && lane == 0) {
       // let every copy this warp started land before the CTA leaves
 #pragma unroll
-      for (int s = 0; s < kStages; ++s)
-        if (issued[s] != 0) mbar_drain(smem_u32(&t.full_bar[s]), ((issued[s] - 1) / kStages) & 1u);
+      for (int s = 0; s < NS; ++s)
+        if (issued[s] != 0) mbar_drain(smem_u32(&t.full_bar[s]), ((issued[s] - 1) / NS) & 1u);
     }
   } else {
     // =============================== consumers (4 warps) ========================================
@@ -311,9 +324,24 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
 #pragma unroll
         for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
 
+      // ROPE: the angle of token 16 u + r is the sum of a coarse angle (row u of the coarse table, fetched a
+      // stage ahead of its use) and a fine one (row r of the table in shared memory).  base[2 ks + h] holds the
+      // coarse (cos, sin) of this thread's frequency indices 16 ks + 8 h + qd and + 1, which pair feature jj of
+      // the first 64-feature block with feature jj + 64.
+      float4 base[ROPE ? 8 : 1];
+      auto load_base = [&](int stage_t0) {
+        if constexpr (ROPE) {
+          const int u = min(stage_t0 / kRopeFineRows + cw, p.rope.stride / kRopeFineRows - 1);
+          const float4* src = reinterpret_cast<const float4*>(p.rope.coarse + (size_t)u * 64 + qd);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) base[k] = __ldg(src + k * 4);
+        }
+      };
+      load_base(t_begin);
+
       for (int j = 0; j < n_iter; ++j, ++it) {
-        const uint32_t s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1u;
+        const uint32_t s = it % NS;
+        const uint32_t ph = (it / NS) & 1u;
         const bool got = mbar_wait(smem_u32(&t.full_bar[s]), ph, abort_flag, p.status);
         if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
         const uint32_t sb = stage_base + s * kStageBytes;
@@ -354,10 +382,10 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
 #pragma unroll
             for (int e = 0; e < 4; ++e) sc[nt][e] = 0.f;
           if constexpr (ROPE) {
-            // fragment element (register i, half e) of step ks: token tile i >> 1, feature pair index
-            // jj = 16 ks + 8 (i & 1) + qd + e, which pairs feature jj (first 64-feature block) with jj + 64
-            const int tok_a = min(t0 + cw * kWarpTokens + (lane >> 2), p.rope.stride - 1);
-            const int tok_b = min(t0 + cw * kWarpTokens + 8 + (lane >> 2), p.rope.stride - 1);
+            // register i of step ks: token tile i >> 1 (slice offsets lane / 4 and lane / 4 + 8), frequency
+            // indices 16 ks + 8 (i & 1) + qd and + 1
+            const float4* fine_a = reinterpret_cast<const float4*>(fine + (lane >> 2) * kFineRowPairs + qd);
+            const float4* fine_b = reinterpret_cast<const float4*>(fine + ((lane >> 2) + 8) * kFineRowPairs + qd);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
               const int c0 = ks * 2 + ((lane >> 3) & 1);
@@ -368,11 +396,13 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
               uint32_t lo_h[4], lo_r[4], hi_h[4], hi_r[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                const float2* cs = p.rope.cs + (size_t)(ks * 16 + (i & 1) * 8 + qd) * p.rope.stride + ((i >> 1) ? tok_b : tok_a);
-                const float2 w0 = cs[0], w1 = cs[p.rope.stride];
+                const float4 bw = base[ks * 2 + (i & 1)];
+                const float4 fw = ((i >> 1) ? fine_b : fine_a)[ks * 8 + (i & 1) * 4];
+                const float c0w = bw.x * fw.x - bw.y * fw.y, s0w = bw.y * fw.x + bw.x * fw.y;
+                const float c1w = bw.z * fw.z - bw.w * fw.w, s1w = bw.w * fw.z + bw.z * fw.w;
                 const float a0 = bf16_lo(a[i]), a1 = bf16_hi(a[i]), b0 = bf16_lo(b[i]), b1 = bf16_hi(b[i]);
-                split_bf16(a0 * w0.x - b0 * w0.y, a1 * w1.x - b1 * w1.y, lo_h[i], lo_r[i]);
-                split_bf16(b0 * w0.x + a0 * w0.y, b1 * w1.x + a1 * w1.y, hi_h[i], hi_r[i]);
+                split_bf16(a0 * c0w - b0 * s0w, a1 * c1w - b1 * s1w, lo_h[i], lo_r[i]);
+                split_bf16(b0 * c0w + a0 * s0w, b1 * c1w + a1 * s1w, hi_h[i], hi_r[i]);
               }
               mma_m16n8k16_bf16(sc[0], qa0[ks], 0u, qa2[ks], 0u, lo_h[0], lo_h[1]);
               mma_m16n8k16_bf16(sc[1], qa0[ks], 0u, qa2[ks], 0u, lo_h[2], lo_h[3]);
@@ -383,6 +413,7 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
               mma_m16n8k16_bf16(sc[0], qa0[ks + 4], 0u, qa2[ks + 4], 0u, hi_r[0], hi_r[1]);
               mma_m16n8k16_bf16(sc[1], qa0[ks + 4], 0u, qa2[ks + 4], 0u, hi_r[2], hi_r[3]);
             }
+            if (j + 1 < n_iter) load_base(t0 + kStageTokens);   // in flight during the rest of this stage
           } else {
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
@@ -442,6 +473,8 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
             mma_m16n8k16_bf16(o[2 * dp + 1], p_hi[0], p_lo[0], p_hi[1], p_lo[1], r2, r3);
           }
           if (!all_valid) fence_proxy_async_smem();   // the zeroed rows, before TMA writes there again
+        } else if (ROPE && j + 1 < n_iter) {
+          load_base(t0 + kStageTokens);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&t.empty_bar[s]));
@@ -484,15 +517,16 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
   }
 }
 
-template <int G>
+template <int G, bool ROPE>
 constexpr size_t stored_smem_bytes() {
-  return 1024 + (size_t)kStages * kStageBytes + sizeof(StoredSmemTail<G>);
+  return 1024 + (size_t)StoredStages<G, ROPE>::value * kStageBytes + ((sizeof(StoredSmemTail<G>) + 15) / 16) * 16 +
+         (ROPE ? (size_t)kRopeFineRows * kFineRowPairs * sizeof(float2) : 0);
 }
 
 template <int G, bool ROPE>
 cudaError_t launch_g(const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& k_run, const CUtensorMap& v_run,
                      const StoredParams& p, int sm_count, cudaStream_t stream) {
-  const size_t smem = stored_smem_bytes<G>();
+  const size_t smem = stored_smem_bytes<G, ROPE>();
   cudaError_t e = cudaFuncSetAttribute(attn_stored_mma_kernel<G, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;

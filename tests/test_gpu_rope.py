@@ -91,7 +91,8 @@ def test_rope_argument_checks():
     lib, h = binding.lib(), case.ctx.handle
     n = C.c_uint64(0)
     assert lib.echokv_rope_table_bytes(C.byref(case.cfg), C.byref(n)) == binding.ECHOKV_OK
-    assert n.value == w.pages_per_seq * w.page_tokens * (w.head_dim // 2) * 8
+    cap, half = w.pages_per_seq * w.page_tokens, w.head_dim // 2
+    assert n.value == (cap * half + (cap // 16) * half + 16 * half) * 8     # full, every 16th position, offsets 0..15
     buf = torch.empty(n.value + 16, dtype=torch.uint8, device="cuda")
     assert lib.echokv_set_rope(h, 10000.0, buf.data_ptr(), n.value - 1, None) == binding.ECHOKV_ECAPACITY
     assert lib.echokv_set_rope(h, 0.5, buf.data_ptr(), n.value, None) == binding.ECHOKV_EINVAL
@@ -103,10 +104,16 @@ def test_rope_argument_checks():
     assert case.ctx.rope_enabled()
     # the table the library wrote: (cos, sin)(t * theta^(-2j/d)), [d/2][capacity]
     torch.cuda.synchronize()
-    tab = buf[: n.value].view(torch.float32).view(w.head_dim // 2, -1, 2).cpu().numpy().astype(np.float64)
-    t = np.arange(tab.shape[1], dtype=np.float64)
-    for j in (0, 1, w.head_dim // 2 - 1):
-        a = t * 10000.0 ** (-2.0 * j / w.head_dim)
-        np.testing.assert_allclose(tab[j, :, 0], np.cos(a), atol=1e-7)
-        np.testing.assert_allclose(tab[j, :, 1], np.sin(a), atol=1e-7)
+    flat = buf[: n.value].view(torch.float32).view(-1, 2).cpu().numpy().astype(np.float64)
+    tab = flat[: cap * half].reshape(half, cap, 2)
+    coarse = flat[cap * half: cap * half + (cap // 16) * half].reshape(cap // 16, half, 2)
+    fine = flat[cap * half + (cap // 16) * half:].reshape(16, half, 2)
+    t = np.arange(cap, dtype=np.float64)
+    for j in (0, 1, half - 1):
+        wj = 10000.0 ** (-2.0 * j / w.head_dim)
+        np.testing.assert_allclose(tab[j, :, 0], np.cos(t * wj), atol=1e-7)
+        np.testing.assert_allclose(tab[j, :, 1], np.sin(t * wj), atol=1e-7)
+        np.testing.assert_allclose(coarse[:, j, 0], np.cos(t[::16] * wj), atol=1e-7)
+        np.testing.assert_allclose(coarse[:, j, 1], np.sin(t[::16] * wj), atol=1e-7)
+        np.testing.assert_allclose(fine[:, j, 1], np.sin(t[:16] * wj), atol=1e-7)
     case.close()
