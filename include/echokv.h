@@ -135,6 +135,21 @@ int echokv_set_block_table(echokv_ctx* ctx, const int32_t* dev_block_table);
 int echokv_append_kv(echokv_ctx* ctx, int layer, const void* k_new, const void* v_new,
                      const int32_t* dev_seq_slots, const int32_t* dev_positions, int B, void* stream);
 
+/* The switch from full-cache generation to compressed inference (Section 3.1: compression is evicting part
+ * of each token's K / V, at the moment memory runs short; Section 5.4: or already during prefill).  The caller
+ * has cached layer `layer` at full width in pools of its own, k_full / v_full: device pointers
+ * [n_pages][page_tokens][D] (16-byte aligned) addressed by the same block table.  For tokens
+ * dev_seq_begins[b] .. dev_seq_lens[b]-1 of each of the B sequences the call copies dims 0 .. m-1 of K and V
+ * into the layer's own pools (Eq. 2) and, while a sink / window is set, dims m .. D-1 of the sink tokens and of
+ * the last n_window tokens before dev_seq_lens[b] into the side buffers; afterwards echokv_decode_attention
+ * serves the layer and the caller may release the full-width pools.  dev_seq_begins = NULL means 0; with a
+ * prefill done in chunks, call it once per chunk with the chunk's range.  The copies are bit-exact.
+ * Bad slot / page -> device status EBADPAGE, bad length or begin -> EBADLENGTH; that sequence is skipped.
+ * Errors: EINVAL, ENOTCOMPRESSED (anchor layers keep everything), ECAPACITY, ENOTABLE, ECUDA. */
+int echokv_compress_layer(echokv_ctx* ctx, int layer, const void* k_full, const void* v_full,
+                          const int32_t* dev_seq_slots, const int32_t* dev_seq_begins,
+                          const int32_t* dev_seq_lens, int B, void* stream);
+
 /* Decode attention of compressed layer `layer` (Eq. 3, 6, 7): q is a device pointer
  * [B][n_q_heads][head_dim], out a device pointer to fp32 [B][n_q_heads][head_dim],
  * dev_seq_lens[b] = tokens in the cache (>= 1, newest included).  Heads 0..r-1 attend their

@@ -98,6 +98,23 @@ def total_predictor_params(n_layers: int, group_size: int, D: int, m: int,
 # ----------------------------------------------------------------------------
 
 
+def retained_dims(c: np.ndarray, m: int) -> np.ndarray:
+    """Eq. 2: C_local = C[:, :m], what a compressed layer keeps of each token ([L, D] -> [L, m]).
+    Compression is nothing but this eviction (Section 3.1)."""
+    c = np.asarray(c)
+    if not 0 <= m <= c.shape[1]:
+        raise ValueError("need 0 <= m <= D")
+    return c[:, :m]
+
+
+def dropped_dims(c: np.ndarray, m: int) -> np.ndarray:
+    """Eq. 4: C_drop = C[:, m:], what is evicted and later predicted ([L, D] -> [L, D - m])."""
+    c = np.asarray(c)
+    if not 0 <= m <= c.shape[1]:
+        raise ValueError("need 0 <= m <= D")
+    return c[:, m:]
+
+
 def predictor_input(c_global: np.ndarray, c_local: np.ndarray) -> np.ndarray:
     """[C_global ; C_local] per token (Eq. 3): [L, D] and [L, m] -> [L, D + m]."""
     c_global = np.asarray(c_global, dtype=np.float64)

@@ -49,6 +49,8 @@ EXPORTS = {
     "echokv_set_block_table": (C.c_int, [C.c_void_p, C.c_void_p]),
     "echokv_append_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_int, C.c_void_p]),
+    "echokv_compress_layer": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_int, C.c_void_p]),
     "echokv_decode_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_int, C.c_void_p]),
     "echokv_full_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -204,6 +206,12 @@ class Context:
         _check(lib().echokv_append_kv(self.handle, layer, _ptr(k_new), _ptr(v_new), _ptr(seq_slots),
                                       _ptr(positions), k_new.shape[0], _stream_handle(stream)),
                "echokv_append_kv")
+
+    def compress_layer(self, layer: int, k_full, v_full, seq_lens, seq_begins=None, seq_slots=None, stream=None) -> None:
+        """Evict a layer cached at full width ([n_pages][page_tokens][D] pools) down to its retained dims."""
+        _check(lib().echokv_compress_layer(self.handle, layer, _ptr(k_full), _ptr(v_full), _ptr(seq_slots),
+                                           _ptr(seq_begins), _ptr(seq_lens), seq_lens.shape[0],
+                                           _stream_handle(stream)), "echokv_compress_layer")
 
     def decode_attention(self, layer: int, q, seq_lens, out=None, seq_slots=None, stream=None):
         out = self._out(q) if out is None else out

@@ -550,6 +550,27 @@ int echokv_append_kv(echokv_ctx* c, int layer, const void* k_new, const void* v_
   return append_side(c, L, k_new, v_new, dev_seq_slots, dev_positions, B, static_cast<cudaStream_t>(stream));
 }
 
+int echokv_compress_layer(echokv_ctx* c, int layer, const void* k_full, const void* v_full,
+                          const int32_t* dev_seq_slots, const int32_t* dev_seq_begins,
+                          const int32_t* dev_seq_lens, int B, void* stream) {
+  if (!c || !k_full || !v_full || !dev_seq_lens) return ECHOKV_EINVAL;
+  if (layer < 0 || layer >= c->cfg.n_layers || B < 1) return ECHOKV_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(k_full) | reinterpret_cast<uintptr_t>(v_full)) % 16 != 0) return ECHOKV_EINVAL;
+  if (B > c->cfg.max_batch) return ECHOKV_ECAPACITY;
+  if (!c->table) return ECHOKV_ENOTABLE;
+  const Layer& L = c->layers[layer];
+  if (L.anchor) return ECHOKV_ENOTCOMPRESSED;
+  const bool side = side_active(c, L);
+  if (c->d.m == 0 && !side) return ECHOKV_OK;          // nothing of this layer is kept
+  const SideArgs sa = side_args(c, L);
+  if (launch_compress(c->d.elem, k_full, v_full, L.k_pool, L.v_pool, side ? &sa : nullptr, c->d.D, c->d.m,
+                      dev_seq_slots, dev_seq_begins, dev_seq_lens, B, geom_of(c), status_ptr(c),
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return ECHOKV_ECUDA;
+  c->launches += 1;
+  return ECHOKV_OK;
+}
+
 int echokv_full_attention(echokv_ctx* c, int layer, const void* q, float* out,
                           const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
                           void* stream) {

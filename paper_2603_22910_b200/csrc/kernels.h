@@ -70,6 +70,13 @@ cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, co
                                const int32_t* slots, const int32_t* positions, int B, int max_batch,
                                int32_t* status, cudaStream_t stream);
 
+// Evict a full-width cache ([n_pages][page_tokens][D], same block table) down to what a compressed layer keeps:
+// dims 0 .. m-1 of tokens [begins[b], lens[b]) into k_local / v_local (skipped when m == 0), dims m .. D-1 of the
+// sink / window tokens (window relative to lens[b]) into the side buffers (side may be null).  Bit-exact copies.
+cudaError_t launch_compress(int elem_bytes, const void* k_full, const void* v_full, void* k_local, void* v_local,
+                            const SideArgs* side, int D, int m, const int32_t* slots, const int32_t* begins,
+                            const int32_t* lens, int B, const PageGeom& geom, int32_t* status, cudaStream_t stream);
+
 // Eq. 7 over the sink and window tokens of the dropped heads, from the side buffers: one split-K partial per
 // (sequence, query head of a dropped KV head), written at partial index ceil(len / part_tokens).
 // With `pool` given (the absorbed mode), the retained heads are covered too, from their stored dims in the

@@ -107,6 +107,80 @@ cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int width, int 
 }
 
 // ---------------------------------------------------------------------------------------------
+// The switch from full-cache generation to compressed inference (Section 3.1: compression is evicting
+// part of each token's K / V; Section 5.4: done only once memory runs short, or during prefill): rows of a
+// full-width cache are cut down to what a compressed layer keeps.  One block per (page of a sequence):
+// dims 0 .. m-1 of every token go to the layer's pools (Eq. 2), dims m .. D-1 of sink / window tokens to the
+// side buffers.  Plain 16-byte copies: bit-exact.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) compress_kernel(const uint4* __restrict__ k_full, const uint4* __restrict__ v_full,
+                                                       uint4* __restrict__ k_local, uint4* __restrict__ v_local,
+                                                       uint4* __restrict__ k_side, uint4* __restrict__ v_side,
+                                                       int d_vec, int m_vec, int n_sink, int n_window,
+                                                       const int32_t* __restrict__ slots,
+                                                       const int32_t* __restrict__ begins,
+                                                       const int32_t* __restrict__ lens, PageGeom g, int32_t* status) {
+  const int b = blockIdx.y, page_idx = blockIdx.x, P = g.page_tokens;
+  const int slot = slots ? slots[b] : b;
+  const int len = lens[b];
+  const int begin = begins ? begins[b] : 0;
+  if (slot < 0 || slot >= g.max_batch) {
+    if (threadIdx.x == 0 && page_idx == 0) report(status, ECHOKV_EBADPAGE);
+    return;
+  }
+  if (len < 1 || len > g.max_pages_per_seq * P || begin < 0 || begin > len) {
+    if (threadIdx.x == 0 && page_idx == 0) report(status, ECHOKV_EBADLENGTH);
+    return;
+  }
+  const int t0 = page_idx * P;
+  const int r_lo = max(begin - t0, 0), r_hi = min(len - t0, P);     // rows of this page to evict
+  if (r_lo >= r_hi) return;
+  const int page = g.table[(size_t)slot * g.max_pages_per_seq + page_idx];
+  if (page < 0 || page >= g.n_pages) {
+    if (threadIdx.x == 0) report(status, ECHOKV_EBADPAGE);
+    return;
+  }
+  const size_t row0 = (size_t)page * P;
+  if (m_vec > 0) {
+    for (int idx = r_lo * m_vec + threadIdx.x; idx < r_hi * m_vec; idx += blockDim.x) {
+      const int r = idx / m_vec, v = idx - r * m_vec;
+      k_local[(row0 + r) * m_vec + v] = k_full[(row0 + r) * d_vec + v];
+      v_local[(row0 + r) * m_vec + v] = v_full[(row0 + r) * d_vec + v];
+    }
+  }
+  const int drop_vec = d_vec - m_vec;
+  if (k_side != nullptr && drop_vec > 0 && (t0 + r_lo < n_sink || t0 + r_hi > len - n_window)) {
+    const size_t seq_base = (size_t)slot * (n_sink + n_window);
+    for (int idx = r_lo * drop_vec + threadIdx.x; idx < r_hi * drop_vec; idx += blockDim.x) {
+      const int r = idx / drop_vec, v = idx - r * drop_vec;
+      const int t = t0 + r;
+      const uint4 kv = k_full[(row0 + r) * d_vec + m_vec + v];
+      const uint4 vv = v_full[(row0 + r) * d_vec + m_vec + v];
+      if (t < n_sink) {
+        k_side[(seq_base + t) * drop_vec + v] = kv;
+        v_side[(seq_base + t) * drop_vec + v] = vv;
+      }
+      if (n_window > 0 && t >= len - n_window) {
+        k_side[(seq_base + n_sink + t % n_window) * drop_vec + v] = kv;
+        v_side[(seq_base + n_sink + t % n_window) * drop_vec + v] = vv;
+      }
+    }
+  }
+}
+
+cudaError_t launch_compress(int elem_bytes, const void* k_full, const void* v_full, void* k_local, void* v_local,
+                            const SideArgs* side, int D, int m, const int32_t* slots, const int32_t* begins,
+                            const int32_t* lens, int B, const PageGeom& geom, int32_t* status, cudaStream_t stream) {
+  const int d_vec = D * elem_bytes / 16, m_vec = m * elem_bytes / 16;
+  dim3 grid(geom.max_pages_per_seq, B);
+  compress_kernel<<<grid, 256, 0, stream>>>(
+      (const uint4*)k_full, (const uint4*)v_full, (uint4*)k_local, (uint4*)v_local,
+      side ? (uint4*)side->k_side : nullptr, side ? (uint4*)side->v_side : nullptr, d_vec, m_vec,
+      side ? side->n_sink : 0, side ? side->n_window : 0, slots, begins, lens, geom, status);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Attention over stored heads (Eq. 7 on the cache as stored): one warp per token row.
 // ---------------------------------------------------------------------------------------------
 template <typename T, int EPL>

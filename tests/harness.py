@@ -43,17 +43,19 @@ class Case:
         for l in sorted(needed):
             width = w.D if w.is_anchor(l) else w.m
             for kind in ("k", "v"):
-                if width == 0:
+                side_only = width == 0 and bool(window) and not w.is_anchor(l)
+                if width == 0 and not side_only:
                     continue
                 seqs = []
                 for b in range(w.batch):
-                    x = synth.layer_cache(w, l, kind, b, width=width)[: self.lens[b]]
+                    x = synth.layer_cache(w, l, kind, b, width=max(width, 1))[: self.lens[b]][:, :width]
                     seqs.append(x)
-                    if keep_host:
+                    if keep_host and width:
                         self.host[(l, kind, b)] = x
                 # all tokens but the last go in directly; the last one is appended by the library
-                pool = synth.paged_pool(w, [s[:-1] for s in seqs], self.table, n_pages, width)
-                (self.ctx.k_pools if kind == "k" else self.ctx.v_pools)[l].copy_(pool)
+                if width:
+                    pool = synth.paged_pool(w, [s[:-1] for s in seqs], self.table, n_pages, width)
+                    (self.ctx.k_pools if kind == "k" else self.ctx.v_pools)[l].copy_(pool)
                 newest = torch.zeros((w.batch, w.D), dtype=synth.torch_dtype(w))
                 for b in range(w.batch):
                     newest[b, :width] = seqs[b][-1]

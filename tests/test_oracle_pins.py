@@ -69,6 +69,22 @@ def test_paper_predictor_shapes_ratios_and_param_totals():
     assert O.effective_ratio(1024, 4, 64) == 0.296875
 
 
+def test_eviction_eq2_eq4_matches_the_printed_shapes():
+    # the table's rows: what is kept (m) plus the anchor's D dims is the predictor's input width, what is
+    # dropped its output width; kept and dropped together are the token's cache again
+    g = rng(77)
+    for ratio, S, m, d_in, d_out, _, _ in load_table():
+        D = 1024
+        c = g.standard_normal((5, D))
+        kept, dropped = O.retained_dims(c, m), O.dropped_dims(c, m)
+        assert kept.shape == (5, m) and dropped.shape == (5, d_out)
+        assert O.predictor_input(c, kept).shape == (5, d_in)
+        np.testing.assert_array_equal(np.concatenate([kept, dropped], axis=1), c)
+        np.testing.assert_array_equal(O.assemble_cache(kept, dropped, 8, 128).reshape(5, D), c)
+    with pytest.raises(ValueError):
+        O.retained_dims(np.zeros((2, 8)), 9)
+
+
 def test_anchor_assignment_eq1():
     S = 4
     assert [O.is_anchor_layer(l, S) for l in range(9)] == [True, False, False, False, True, False, False, False, True]
