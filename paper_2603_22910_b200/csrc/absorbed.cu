@@ -83,18 +83,25 @@ inline uint32_t make_idesc(int n, bool a_mmajor) {
 // 1. absorbed queries
 // ---------------------------------------------------------------------------------------------
 constexpr int kQGroup = 8;   // (sequence, query head of the group) pairs per block
-constexpr int kQCols = 512;  // input features per block: two adjacent ones per thread
+constexpr int kQCols = 256;  // input features per block: eight adjacent ones per lane
+constexpr size_t kQuerySmemBytes = (size_t)(kQGroup * 128 + 8 * kQGroup * kQCols) * sizeof(float);
 
+// Block = (256 input features, KV head, 8 (sequence, query head) pairs).  The head's predictor rows are dealt
+// round-robin to the 8 warps, each lane reading 16 bytes (8 features) of a row, so a thread has all its
+// loads in flight at once; the warps' partial sums meet in shared memory.
 __global__ void __launch_bounds__(256)
 absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ Wk,
                     __nv_bfloat16* __restrict__ q2, int B, int n_q_heads, int g, int m, int D, int d_in,
                     float scale_log2e) {
-  __shared__ float qs[kQGroup][128];
-  const int i = blockIdx.x * kQCols + threadIdx.x * 2;     // first of this thread's two input features
+  extern __shared__ __align__(16) float query_smem[];
+  float (*qs)[128] = reinterpret_cast<float (*)[128]>(query_smem);          // [kQGroup][128]
+  float* red = query_smem + kQGroup * 128;                                  // [8 warps][kQGroup][kQCols]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int col0 = blockIdx.x * kQCols;
   const int kv = blockIdx.y;
   const int first = blockIdx.z * kQGroup;
   const int n_pairs = B * g;
-  for (int idx = threadIdx.x; idx < kQGroup * 128; idx += 256) {
+  for (int idx = tid; idx < kQGroup * 128; idx += 256) {
     const int k = idx >> 7, j = idx & 127;
     const int pr = first + k;
     float v = 0.f;
@@ -105,47 +112,58 @@ absorb_query_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     qs[k][j] = v;
   }
   __syncthreads();
-  if (i >= d_in) return;
-  float acc[kQGroup][2];
-#pragma unroll
-  for (int k = 0; k < kQGroup; ++k) acc[k][0] = acc[k][1] = 0.f;
   // dims kv * 128 + j of this head with flat index < m are stored (the head reads them as they are: q~ is q
   // placed at those local dims); the others are predicted by row (flat index - m) of W_k
   const int n_stored = max(0, min(128, m - kv * 128));
-  {
-    const int j = i - (D + kv * 128);
-    if (j >= 0 && j < n_stored) {
+  float acc[kQGroup][8];
+#pragma unroll
+  for (int k = 0; k < kQGroup; ++k)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[k][c] = 0.f;
+  const int i8 = col0 + lane * 8;                    // this lane's eight input features (d_in is a multiple of 8)
+  if (i8 < d_in && n_stored < 128) {
+    const __nv_bfloat16* w = Wk + (size_t)(kv * 128 + n_stored + warp - m) * d_in + i8;
+#pragma unroll 8
+    for (int j = n_stored + warp; j < 128; j += 8, w += (size_t)8 * d_in) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(w);
+      const uint32_t r4[4] = {raw.x, raw.y, raw.z, raw.w};
+      float wv[8];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        wv[2 * c] = __uint_as_float(r4[c] << 16);
+        wv[2 * c + 1] = __uint_as_float(r4[c] & 0xffff0000u);
+      }
 #pragma unroll
       for (int k = 0; k < kQGroup; ++k) {
-        acc[k][0] = qs[k][j];
-        acc[k][1] = qs[k][j + 1];
+        const float qv = qs[k][j];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[k][c] = fmaf(wv[c], qv, acc[k][c]);
       }
     }
   }
-  if (n_stored < 128) {
-    const __nv_bfloat16* w = Wk + ((size_t)kv * 128 + n_stored - m) * d_in + i;
-#pragma unroll 16
-    for (int j = n_stored; j < 128; ++j, w += d_in) {
-      const uint32_t raw = *reinterpret_cast<const uint32_t*>(w);
-      const float w0 = __uint_as_float(raw << 16), w1 = __uint_as_float(raw & 0xffff0000u);
 #pragma unroll
-      for (int k = 0; k < kQGroup; ++k) {
-        acc[k][0] = fmaf(w0, qs[k][j], acc[k][0]);
-        acc[k][1] = fmaf(w1, qs[k][j], acc[k][1]);
-      }
-    }
+  for (int k = 0; k < kQGroup; ++k) {
+    float4* dst = reinterpret_cast<float4*>(red + (size_t)(warp * kQGroup + k) * kQCols + lane * 8);
+    dst[0] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+    dst[1] = make_float4(acc[k][4], acc[k][5], acc[k][6], acc[k][7]);
   }
+  __syncthreads();
+  const int i = col0 + tid;                          // one input feature per thread from here on
+  if (i >= d_in) return;
+  const int j_stored = i - (D + kv * 128);
   const int nh2 = 2 * n_q_heads;
 #pragma unroll
   for (int k = 0; k < kQGroup; ++k) {
     const int pr = first + k;
     if (pr >= n_pairs) break;
+    float v = (j_stored >= 0 && j_stored < n_stored) ? qs[k][j_stored] : 0.f;
+#pragma unroll
+    for (int w8 = 0; w8 < 8; ++w8) v += red[(size_t)(w8 * kQGroup + k) * kQCols + tid];
     const int b = pr / g, gi = pr - b * g;
     const int h = kv * g + gi;
-    const __nv_bfloat162 hi = __floats2bfloat162_rn(acc[k][0], acc[k][1]);
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[k][0] - __low2float(hi), acc[k][1] - __high2float(hi));
-    *reinterpret_cast<__nv_bfloat162*>(q2 + ((size_t)b * nh2 + h) * d_in + i) = hi;
-    *reinterpret_cast<__nv_bfloat162*>(q2 + ((size_t)b * nh2 + n_q_heads + h) * d_in + i) = lo;
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    q2[((size_t)b * nh2 + h) * d_in + i] = hi;
+    q2[((size_t)b * nh2 + n_q_heads + h) * d_in + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
   }
 }
 
@@ -903,7 +921,10 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   // 1. absorbed queries
   {
     dim3 grid((d_in + kQCols - 1) / kQCols, a.n_kv_heads, (a.batch * g + kQGroup - 1) / kQGroup);
-    absorb_query_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q),
+    if ((e = cudaFuncSetAttribute(absorb_query_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)kQuerySmemBytes)) != cudaSuccess)
+      return e;
+    absorb_query_kernel<<<grid, 256, kQuerySmemBytes, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q),
                                                   reinterpret_cast<const __nv_bfloat16*>(r.Wk), q2, a.batch,
                                                   a.n_q_heads, g, r.m, r.D, d_in, a.scale_log2e);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
