@@ -40,9 +40,11 @@ UNIT = "tokens/s"
 # the ncu captures summarised under profiles/; None until a capture of that workload exists.
 NCU_TRAFFIC_BYTES = {
     "c1": 4 * 619.0e6,        # recon_tc_kernel: B = 2 capture x 4 (tokens)
-    "c2": 8 * 347.9e6,        # recon_pair_kernel: B = 2 capture x 8
-    "c1_full": 4 * 275.0e6,   # attn_stored_mma_kernel: B = 2 capture x 4
-    "c2_full": 8 * 273.8e6,   # attn_stored_mma_kernel: B = 2 capture x 8
+    "c2": 8 * 348.1e6,        # recon_pair_kernel: B = 2 capture x 8
+    "c1_full": 4 * 272.9e6,   # attn_stored_mma_kernel: B = 2 capture x 4
+    "c2_full": 8 * 274.5e6,   # attn_stored_mma_kernel: B = 2 capture x 8
+    "c1_absorbed": 4 * 418.8e6,   # absorb_scores_kernel + absorb_pv_kernel (one launch each): B = 2 capture x 4
+    "c2_absorbed": 8 * 354.3e6,   # the same: B = 2 capture x 8
 }
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -52,6 +54,8 @@ def traffic_of(args, key):
     """The stored ncu figure, only for the exact workload it was scaled to."""
     if args.batch or args.context or args.page_tokens or args.random_pages:
         return None
+    if args.rope or args.window or args.retained_dims or args.decode_path is not None or args.stored_path is not None:
+        return None          # another kernel (instantiation) than the captured one
     return NCU_TRAFFIC_BYTES.get(key)
 
 
@@ -635,7 +639,8 @@ def run_ours(args):
         achieved_gbs = bytes_ / (k_ms * 1e-3) / 1e9
         peak_gbs = float(peaks["hbm_gbs"])
         roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
-                    "frac": achieved_gbs / peak_gbs, "traffic": None,
+                    "frac": achieved_gbs / peak_gbs,
+                    "traffic": traffic_of(args, args.workload + "_absorbed"),
                     "kernel": "absorb_scores_kernel + absorb_pv_kernel", "kernel_ms": k_ms,
                     "kernel_ms_k_pass": ak_ms / max(ak_n, 1), "kernel_ms_v_pass": av_ms / max(av_n, 1),
                     "kernel_launches": ak_n + av_n, "share_of_step": (ak_ms + av_ms) / ms_eager,
