@@ -76,7 +76,7 @@ class Workload:
         return dataclasses.replace(self, **kw)
 
 
-# The five benchmark configurations (BASELINE.json "configs"), in order.
+# The five benchmark configurations, in order.
 C0 = Workload("c0_tiny_fp32", "fp32", 1, 512, 8, 8, 64, 4, 0.8, seed=1000)
 C1 = Workload("c1_llama2_7b_layer", "bf16", 8, 8192, 32, 32, 128, 16, 0.8, seed=1001)
 C2 = Workload("c2_llama3_8b_gqa_layer", "bf16", 16, 32768, 32, 8, 128, 2, 0.7, seed=1002)
