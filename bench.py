@@ -647,6 +647,23 @@ def run_ours(args):
                     "peak_source": "%s (STREAM-style copy)" % peaks_kind,
                     "algorithmic_bytes_per_launch": bytes_,
                     "mode": "absorbed predictors: the same outputs as the explicit path, a separate roofline row"}
+        if args.rope:
+            # rotated keys: the K side is explicit (Eq. 3 for the keys on the tensor cores, rotation, scores), only
+            # the V side is absorbed; the K pass is the dominant kernel and tensor-bound
+            tokens = float(w.batch) * w.context
+            k_flops = tokens * 2.0 * w.d_in * w.d_drop
+            k_pass_ms = ak_ms / max(ak_n, 1)
+            achieved_tf = k_flops / (k_pass_ms * 1e-3) / 1e12
+            peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+            roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                        "frac": achieved_tf / peak_tf, "traffic": None,
+                        "kernel": "recon_pair_kernel (key scores) + key_scores_stored_kernel", "kernel_ms": k_pass_ms,
+                        "kernel_ms_k_pass": k_pass_ms, "kernel_ms_v_pass": av_ms / max(av_n, 1),
+                        "kernel_launches": ak_n, "share_of_step": ak_ms / ms_eager,
+                        "peak_source": "%s (cuBLAS bf16 GEMM, sustained)" % peaks_kind,
+                        "algorithmic_flops_per_launch": k_flops,
+                        "v_pass_frac_of_hbm": (bytes_ / 2) / (av_ms / max(av_n, 1) * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
+                        "mode": "rotated keys: K side explicit, V side with absorbed predictors"}
         if stored_info:
             roofline["anchor_layers"] = stored_info
     elif recon_n:

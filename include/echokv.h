@@ -229,9 +229,11 @@ int echokv_set_full_precision_window(echokv_ctx* ctx, int n_sink, int n_window, 
  *  - echokv_set_rope: `table` is a device pointer of at least that size (16-byte aligned, borrowed until
  *    echokv_destroy or until rope is switched off); the call enqueues one kernel on `stream` that fills it
  *    (angles and sin / cos in fp64, rounded to fp32 once) and switches rotation on for later calls.
- *    theta = 0 with table = NULL switches it off.  Not available together with the absorbed mode (a
- *    rotation that depends on the token cannot be folded into the queries) nor with n_retained_dims that
- *    split a head: EUNSUPPORTED.  Errors: EINVAL (theta < 1, misaligned), ECAPACITY, EUNSUPPORTED, ECUDA. */
+ *    theta = 0 with table = NULL switches it off.  Not available with n_retained_dims that split a head
+ *    (EUNSUPPORTED).  In the absorbed mode a rotation that depends on the token cannot be folded into the
+ *    queries: with a table set that mode evaluates the K side explicitly (predicted keys on the tensor cores,
+ *    rotated, scored) and keeps the absorbed form for the V side only -- about half the tensor work of the
+ *    explicit mode.  Errors: EINVAL (theta < 1, misaligned), ECAPACITY, EUNSUPPORTED, ECUDA. */
 int echokv_rope_table_bytes(const echokv_config* cfg, uint64_t* out);
 int echokv_set_rope(echokv_ctx* ctx, double theta, void* table, uint64_t table_bytes, void* stream);
 int echokv_rope_enabled(const echokv_ctx* ctx);
@@ -254,7 +256,7 @@ int echokv_rope_enabled(const echokv_ctx* ctx);
  *    borrowed until echokv_destroy) and switches the context to the absorbed mode.
  *    Errors: EINVAL, EUNSUPPORTED, ECAPACITY (workspace too small), ECUDA.
  *  - echokv_set_decode_mode: 0 = explicit reconstruction, 1 = absorbed (EUNSUPPORTED before
- *    echokv_enable_absorbed, and while a rotary table is set).  Anchor layers and echokv_full_attention are not affected.
+ *    echokv_enable_absorbed).  Anchor layers and echokv_full_attention are not affected.
  *  In this mode a page id outside the pool is still reported (EBADPAGE) but the output of that
  *  sequence is unspecified. */
 int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out);

@@ -918,11 +918,18 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   float* ysum = reinterpret_cast<float*>(r.ws + lay.off_ysum);
   cudaError_t e;
 
+  const bool rotated = a.rope.cs != nullptr;
+  if (rotated && (r.m % 128 != 0 || !layer.weights_ready)) return cudaErrorInvalidValue;
+
   // 1. absorbed queries
-  {
+  if (!rotated) {
     dim3 grid((d_in + kQCols - 1) / kQCols, a.n_kv_heads, (a.batch * g + kQGroup - 1) / kQGroup);
     if ((e = cudaFuncSetAttribute(absorb_query_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)kQuerySmemBytes)) != cudaSuccess)
+      return e;
+    // several blocks per SM: ask for the largest shared-memory carve-out (the default sizes it for one block)
+    if ((e = cudaFuncSetAttribute(absorb_query_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                  cudaSharedmemCarveoutMaxShared)) != cudaSuccess)
       return e;
     absorb_query_kernel<<<grid, 256, kQuerySmemBytes, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q),
                                                   reinterpret_cast<const __nv_bfloat16*>(r.Wk), q2, a.batch,
@@ -957,7 +964,22 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   const int capacity = r.capacity_tokens;
 
   // 2. scores
-  {
+  if (rotated) {
+    // keys rotated by position: predicted heads on the tensor cores (Eq. 3, rotation, q . k), stored heads from
+    // the layer's pool; both write the score rows the softmax below reads
+    ReconArgs ra;
+    ra.k_anchor = nullptr; ra.v_anchor = nullptr; ra.k_local = r.k_local; ra.v_local = r.v_local;
+    ra.Wk = r.Wk; ra.Wv = r.Wv; ra.bk = r.bk;
+    ra.D = r.D; ra.m = r.m;
+    ra.part_tokens = 0;
+    ra.capacity_tokens = capacity;
+    ra.n_sink = r.n_sink; ra.n_window = r.n_window;
+    if (ev) cudaEventRecord(ev[0], stream);
+    if ((e = launch_recon_pair_key_scores(a, ra, anchor, layer, S, lay.l_cap, sm_count, stream)) != cudaSuccess) return e;
+    if ((e = launch_key_scores_stored(a, r.k_local, r.m, n_ret, S, lay.l_cap, r.n_sink, r.n_window, stream)) != cudaSuccess)
+      return e;
+    if (ev) cudaEventRecord(ev[1], stream);
+  } else {
     p.stage_bytes = 2u * (kScoreXBytes + (uint32_t)lay.nh2 * kRowBytes);
     p.n_stages = (int)(kSmemBudget / p.stage_bytes);
     if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;

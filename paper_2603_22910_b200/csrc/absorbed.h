@@ -45,15 +45,20 @@ struct AbsorbArgs {
   unsigned char* ws;            // the absorbed-mode workspace
   AbsorbLayout lay;
   const void* Wk; const void* Wv; const void* bv;     // predictors of the layer ([D - m][D + m]), V bias or null
+  const void* bk = nullptr;     // K bias or null; read only when the keys are rotated (a.rope set): it cancels otherwise
   int D, m;
   int capacity_tokens;
   int n_sink = 0, n_window = 0; // sink / recent-window tokens kept at full precision (0, 0 = none) ...
   void* k_side = nullptr; void* v_side = nullptr;            // ... their dropped dims (side buffers of the layer)
-  const void* k_local = nullptr; const void* v_local = nullptr;   // ... and the layer's pools (retained dims)
+  const void* k_local = nullptr; const void* v_local = nullptr;   // ... and the layer's pools (retained dims); also
+                                                                 // read when the keys are rotated
   double* kernel_ms;            // unused
 };
 
-// One compressed layer, all query heads: out[B][H_q][d].
+// One compressed layer, all query heads: out[B][H_q][d].  With a.rope set (keys cached before the rotary embedding) a
+// rotation that depends on the token sits between Eq. 3 and q . k, so W_k cannot be folded into the queries: the K
+// side is then explicit (predicted keys on the tensor cores, rotated, scored; stored heads scored from the pool; m
+// must be head-aligned) and only the V side uses the absorbed form.
 cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const AbsorbMaps& maps, const TcLayerMaps& anchor,
                             const TcLayerMaps& layer, float* out, int sm_count, cudaStream_t stream,
                             cudaEvent_t* timing_events /* 4 events or null: around the K pass and the V pass */);

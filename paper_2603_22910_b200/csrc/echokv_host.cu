@@ -466,8 +466,9 @@ int echokv_set_rope(echokv_ctx* c, double theta, void* table, uint64_t table_byt
     return ECHOKV_OK;
   }
   if (!std::isfinite(theta) || theta < 1.0) return ECHOKV_EINVAL;
-  // a rotation that depends on the token cannot be folded into the queries
-  if (c->decode_mode == 1 || !c->d.head_aligned) return ECHOKV_EUNSUPPORTED;
+  // a rotation that depends on the token cannot be folded into the queries: the K side stays explicit, which
+  // needs whole heads
+  if (!c->d.head_aligned) return ECHOKV_EUNSUPPORTED;
   uint64_t need = 0;
   const int rc = echokv_rope_table_bytes(&c->cfg, &need);
   if (rc != ECHOKV_OK) return rc;
@@ -502,7 +503,7 @@ int echokv_enable_absorbed(echokv_ctx* c, void* workspace, uint64_t workspace_by
   uint64_t need = 0;
   const int rc = echokv_absorbed_workspace_bytes(&c->cfg, &need);
   if (rc != ECHOKV_OK) return rc;
-  if (!c->tc_capable || c->rope.cs != nullptr) return ECHOKV_EUNSUPPORTED;
+  if (!c->tc_capable) return ECHOKV_EUNSUPPORTED;
   if (workspace_bytes < need) return ECHOKV_ECAPACITY;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign != 0) return ECHOKV_EINVAL;
   c->ws_absorbed = static_cast<unsigned char*>(workspace);
@@ -518,7 +519,7 @@ int echokv_decode_mode(const echokv_ctx* c) { return c ? c->decode_mode : 0; }
 
 int echokv_set_decode_mode(echokv_ctx* c, int mode) {
   if (!c || (mode != 0 && mode != 1)) return ECHOKV_EINVAL;
-  if (mode == 1 && (!c->absorbed_capable || c->rope.cs != nullptr)) return ECHOKV_EUNSUPPORTED;
+  if (mode == 1 && !c->absorbed_capable) return ECHOKV_EUNSUPPORTED;
   c->decode_mode = mode;
   return ECHOKV_OK;
 }
@@ -602,6 +603,8 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     aa.ws = c->ws_absorbed;
     aa.lay = c->alay;
     aa.Wk = L.Wk; aa.Wv = L.Wv; aa.bv = L.bv;
+    aa.bk = c->rope.cs != nullptr ? L.bk : nullptr;
+    aa.k_local = L.k_pool; aa.v_local = L.v_pool;
     aa.D = c->d.D; aa.m = c->d.m;
     aa.capacity_tokens = c->d.capacity;
     aa.kernel_ms = nullptr;
@@ -615,7 +618,7 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
                        timed_pair(c, ECHOKV_TIMED_ABSORB_V, &ev[2], &ev[3]);
     if (launch_absorbed(a, aa, c->amaps, A.tc, L.tc, out, c->sm_count, s, timed ? ev : nullptr) != cudaSuccess)
       return ECHOKV_ECUDA;
-    c->launches += side ? 8 : 6;
+    c->launches += (c->rope.cs != nullptr ? 5 + (c->d.m > 0 ? 1 : 0) : 6) + (side ? 2 : 0);
     return ECHOKV_OK;
   }
   if (!c->d.head_aligned) return ECHOKV_EUNSUPPORTED;   // explicit reconstruction needs whole heads: use the absorbed mode
@@ -629,6 +632,7 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   ra.k_anchor = A.k_pool; ra.v_anchor = A.v_pool;
   ra.k_local = L.k_pool; ra.v_local = L.v_pool;
   ra.Wk = L.Wk; ra.Wv = L.Wv;
+  ra.bk = c->rope.cs != nullptr ? L.bk : nullptr;
   ra.D = c->d.D; ra.m = c->d.m;
   ra.part_tokens = c->d.part_tokens;
   ra.capacity_tokens = c->d.capacity;

@@ -68,12 +68,16 @@ struct PairParams {
   int n_sink, n_window;       // sink / recent-window tokens are not predicted (masked here)
   float scale_log2e;
   RopeTable rope;             // read by the ROPE instantiations only
+  const __nv_bfloat16* bk;    // bias of the K predictor or null (ROPE instantiations only: otherwise it cancels)
+  float* s_out;               // KS instantiations: scores [b][query head][l_cap], base-2 units
+  int l_cap;
 };
 
 template <int G>
 struct PairSmemTail {
   float P[2][G][kTileTokens];        // [item parity][query head][token of the tile]: this CTA's head
   float qs[2][G][128];               // queries of both heads of the pair * scale * log2e
+  float kb[2][128];                  // bias of the K predictor for the pair's heads (rotating variant)
   float red_max[8][G];
   float red_sum[8][G];
   int cum_tiles[kMaxBatchPerLaunch + 1];
@@ -136,7 +140,10 @@ __device__ __forceinline__ Item decode_item(const PairSmemTail<G>& t, int item, 
 
 // ROPE: the predicted key rows are rotated to their positions before q . k (Section 3.2: the predictors
 // produce keys prior to the rotary embedding).
-template <int G, bool ROPE>
+// KS ("key scores only"): the K phase alone, its scores written out instead of being turned into
+// probabilities; successive work items alternate between the two accumulators, so the epilogue of one item runs
+// under the MMAs of the next.  Used when the V side is evaluated with absorbed predictors.
+template <int G, bool ROPE, bool KS>
 __global__ void __launch_bounds__(kThreads, 1)
 recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_constant__ CUtensorMap tm_anchor_v,
                   const __grid_constant__ CUtensorMap tm_local_k, const __grid_constant__ CUtensorMap tm_local_v,
@@ -248,7 +255,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
         run_lead = group_run && lane == lead && lane < boxes;
         run_member = group_run && lane != lead && lane < boxes;
       }
-      for (int phase = 0; phase < 2 && alive; ++phase) {
+      for (int phase = 0; phase < (KS ? 1 : 2) && alive; ++phase) {
         const CUtensorMap* m_anchor = phase == 0 ? &tm_anchor_k : &tm_anchor_v;
         const CUtensorMap* m_local = phase == 0 ? &tm_local_k : &tm_local_v;
         const CUtensorMap* m_anchor_run = phase == 0 ? &tm_anchor_k_run : &tm_anchor_v_run;
@@ -294,14 +301,16 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
       uint32_t it = 0, n = 0;
       bool alive = true;
       for (int item = pair_id; item < n_items && alive; item += n_clusters, ++n) {
-        for (int phase = 0; phase < 2 && alive; ++phase) {
-          // this phase's accumulator must have been drained by both CTAs' epilogues of the previous item
-          if (!mbar_wait_cluster(smem_u32(&t.acc_empty_bar[phase]), (n & 1u) ^ 1u, abort_flag, p.status)) {
+        for (int phase = 0; phase < (KS ? 1 : 2) && alive; ++phase) {
+          // this accumulator must have been drained by both CTAs' epilogues of its previous use
+          const uint32_t acc = KS ? (n & 1u) : (uint32_t)phase;
+          const uint32_t use = KS ? (n >> 1) : n;            // how often this accumulator was used before
+          if (!mbar_wait_cluster(smem_u32(&t.acc_empty_bar[acc]), (use & 1u) ^ 1u, abort_flag, p.status)) {
             alive = false;
             break;
           }
           tc_fence_after();
-          const uint32_t d_tmem = tmem + phase * kAccCols;
+          const uint32_t d_tmem = tmem + acc * kAccCols;
           for (int step = 0; step < n_steps; ++step, ++it) {
             const uint32_t s = it % kStages;
             const uint32_t ph = (it / kStages) & 1u;
@@ -322,7 +331,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
             }
             tc_commit_pair(smem_u32(&t.empty_bar[s]));     // the stage is free in both CTAs
           }
-          if (alive) tc_commit_pair(smem_u32(&t.acc_full_bar[phase]));
+          if (alive) tc_commit_pair(smem_u32(&t.acc_full_bar[acc]));
         }
       }
       gave_up = !alive;
@@ -350,6 +359,9 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
       const int kvh0 = p.n_ret_heads + w.pair * 2;           // first KV head of the pair
       const bool second = w.pair * 2 + 1 < p.n_drop_heads;   // does the pair have a second head?
       const uint32_t par = n & 1u;
+      const uint32_t k_acc = KS ? (n & 1u) : 0u;             // accumulator holding this item's predicted keys
+      const uint32_t k_par = KS ? ((n >> 1) & 1u) : par;
+      const uint32_t k_addr = lane_addr + k_acc * kAccCols;
       // queries of the pair's query heads, pre-scaled (the previous item's K epilogue is long done)
       for (int idx = et; idx < 2 * G * 128; idx += kEpilogueThreads) {
         const int hh = idx / (G * 128), rem = idx % (G * 128);
@@ -358,10 +370,16 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
           v = __bfloat162float(p.q[((size_t)b * p.n_q_heads + (size_t)(kvh0 + hh) * G) * 128 + rem]) * p.scale_log2e;
         (&t.qs[0][0][0])[idx] = v;
       }
+      if constexpr (ROPE) {
+        // a bias on predicted keys is rotated with them, so it no longer cancels in the softmax
+        const int hh = et >> 7, j = et & 127;
+        t.kb[hh][j] = (p.bk != nullptr && (hh == 0 || second))
+                          ? __bfloat162float(p.bk[(size_t)(w.pair * 2 + hh) * 128 + j]) : 0.f;
+      }
 
       // ---------------- K phase: scores and probabilities of (token `row`, head `sel`) ----------------
       // (the vote is also the barrier that publishes the queries staged above)
-      if (!epilogue_all(mbar_wait(smem_u32(&t.acc_full_bar[0]), par, abort_flag, p.status))) { alive = false; break; }
+      if (!epilogue_all(mbar_wait(smem_u32(&t.acc_full_bar[k_acc]), k_par, abort_flag, p.status))) { alive = false; break; }
       tc_fence_after();
       float sc[G];
 #pragma unroll
@@ -376,12 +394,13 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
 #pragma unroll
           for (int j = 0; j < 16; ++j) cs[j] = cs_row[(size_t)(cb * 16 + j) * p.rope.stride];
           float lo[16], hi[16];
-          tmem_ld16(lane_addr + sel * 128 + cb * 16, lo);
-          tmem_ld16(lane_addr + sel * 128 + 64 + cb * 16, hi);
+          tmem_ld16(k_addr + sel * 128 + cb * 16, lo);
+          tmem_ld16(k_addr + sel * 128 + 64 + cb * 16, hi);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const float r_lo = lo[j] * cs[j].x - hi[j] * cs[j].y;
-            const float r_hi = hi[j] * cs[j].x + lo[j] * cs[j].y;
+            const float k_lo = lo[j] + t.kb[sel][cb * 16 + j], k_hi = hi[j] + t.kb[sel][64 + cb * 16 + j];
+            const float r_lo = k_lo * cs[j].x - k_hi * cs[j].y;
+            const float r_hi = k_hi * cs[j].x + k_lo * cs[j].y;
 #pragma unroll
             for (int gi = 0; gi < G; ++gi)
               sc[gi] = fmaf(r_hi, t.qs[sel][gi][64 + cb * 16 + j], fmaf(r_lo, t.qs[sel][gi][cb * 16 + j], sc[gi]));
@@ -391,7 +410,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float v[32];
-        tmem_ld32(lane_addr + sel * 128 + c * 32, v);
+        tmem_ld32(k_addr + sel * 128 + c * 32, v);
 #pragma unroll
         for (int gi = 0; gi < G; ++gi) {
           const float4* qv = reinterpret_cast<const float4*>(&t.qs[sel][gi][c * 32]);
@@ -412,6 +431,17 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
       // predicted tokens only: sink and recent-window tokens are attended from the side buffers
       const int t_seq = w.tile * kTileTokens + token;
       const bool tok_valid = t_seq >= predicted_lo(len, p.n_sink) && t_seq < predicted_hi(len, p.n_sink, p.n_window);
+      if constexpr (KS) {
+        tc_fence_before();
+        epilogue_sync();       // every warp is done reading the accumulator (and the staged queries)
+        if (et == 0) mbar_arrive_cluster(k_acc ? acc_empty1 : acc_empty0);
+        // scores of every token slot of the tile; slots without a predicted token read as -inf downstream
+        if (t_seq < p.l_cap && (sel == 0 || second)) {
+          float* dst = p.s_out + ((size_t)b * p.n_q_heads + (size_t)(kvh0 + sel) * G) * p.l_cap + t_seq;
+#pragma unroll
+          for (int gi = 0; gi < G; ++gi) dst[(size_t)gi * p.l_cap] = tok_valid ? sc[gi] : -INFINITY;
+        }
+      } else {
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) {
         if (!tok_valid) sc[gi] = -INFINITY;
@@ -503,6 +533,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
       tc_fence_before();
       epilogue_sync();       // every warp is done reading acc1 and P[par]
       if (et == 0) mbar_arrive_cluster(acc_empty1);
+      }
     }
     gave_up = !alive;
   }
@@ -529,12 +560,12 @@ constexpr size_t pair_smem_bytes() {
   return 1024 + (size_t)kStages * kStageBytes + sizeof(PairSmemTail<G>);
 }
 
-template <int G, bool ROPE>
+template <int G, bool ROPE, bool KS>
 cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUtensorMap& lv, const CUtensorMap& lkr,
                      const CUtensorMap& lvr, const CUtensorMap& lk8, const CUtensorMap& lv8, const TcLayerMaps& layer,
                      const PairParams& p, int n_clusters, cudaStream_t stream) {
   const size_t smem = pair_smem_bytes<G>();
-  cudaError_t e = cudaFuncSetAttribute(recon_pair_kernel<G, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(recon_pair_kernel<G, ROPE, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -552,13 +583,13 @@ cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUt
   if (resident_pairs == 0) {
     cfg.gridDim = dim3(2 * n_clusters, 1, 1);
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, recon_pair_kernel<G, ROPE>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, recon_pair_kernel<G, ROPE, KS>, &cfg);
     if (e != cudaSuccess) return e;
     resident_pairs = n < 1 ? 1 : n;
   }
   if (n_clusters > resident_pairs) n_clusters = resident_pairs;
   cfg.gridDim = dim3(2 * n_clusters, 1, 1);
-  return cudaLaunchKernelEx(&cfg, recon_pair_kernel<G, ROPE>, anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run,
+  return cudaLaunchKernelEx(&cfg, recon_pair_kernel<G, ROPE, KS>, anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run,
                             anchor.v_pool_run, lkr, lvr, anchor.k_pool_run128, anchor.v_pool_run128, lk8, lv8,
                             layer.wk_half, layer.wv_half, p);
 }
@@ -567,14 +598,19 @@ template <int G>
 cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUtensorMap& lv, const CUtensorMap& lkr,
                      const CUtensorMap& lvr, const CUtensorMap& lk8, const CUtensorMap& lv8, const TcLayerMaps& layer,
                      const PairParams& p, int n_clusters, cudaStream_t stream) {
-  if (p.rope.cs != nullptr) return launch_g<G, true>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
-  return launch_g<G, false>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
+  if (p.s_out != nullptr) {
+    if (p.rope.cs == nullptr) return cudaErrorInvalidValue;     // (only built for rotated keys)
+    return launch_g<G, true, true>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
+  }
+  if (p.rope.cs != nullptr) return launch_g<G, true, false>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
+  return launch_g<G, false, false>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
 }
 
 }  // namespace
 
-cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
-                              const TcLayerMaps& layer, int sm_count, cudaStream_t stream) {
+static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                                    const TcLayerMaps& layer, int sm_count, cudaStream_t stream, float* s_out,
+                                    int l_cap) {
   if (!anchor.pools_ready || !layer.weights_ready) return cudaErrorInvalidValue;
   if (r.m > 0 && !layer.pools_ready) return cudaErrorInvalidValue;
   const int g = a.n_q_heads / a.n_kv_heads;
@@ -601,6 +637,9 @@ cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLay
   p.n_sink = r.n_sink;
   p.n_window = r.n_window;
   p.rope = a.rope;
+  p.bk = reinterpret_cast<const __nv_bfloat16*>(r.bk);
+  p.s_out = s_out;
+  p.l_cap = l_cap;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;
@@ -627,6 +666,18 @@ cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLay
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                              const TcLayerMaps& layer, int sm_count, cudaStream_t stream) {
+  return launch_pair_impl(a, r, anchor, layer, sm_count, stream, nullptr, 0);
+}
+
+cudaError_t launch_recon_pair_key_scores(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                                         const TcLayerMaps& layer, float* scores, int l_cap, int sm_count,
+                                         cudaStream_t stream) {
+  if (scores == nullptr) return cudaErrorInvalidValue;
+  return launch_pair_impl(a, r, anchor, layer, sm_count, stream, scores, l_cap);
 }
 
 }  // namespace echokv

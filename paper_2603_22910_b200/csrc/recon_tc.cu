@@ -65,12 +65,14 @@ struct TcParams {
   int n_sink, n_window;       // sink / recent-window tokens are not predicted (masked here)
   float scale_log2e;
   RopeTable rope;             // read by the ROPE instantiations only
+  const __nv_bfloat16* bk;    // bias of the K predictor or null (ROPE instantiations only: otherwise it cancels)
 };
 
 template <int G>
 struct TcSmemTail {
   float P[2 * G][kTileTokens];       // probabilities of the tile, per (head of the pair, query head)
   float qs[2][G][128];               // queries * scale * log2e
+  float kb[2][128];                  // bias of the K predictor for the pair's heads (rotating variant)
   float red_max[8][2 * G];
   float red_sum[8][2 * G];
   int cum_tiles[kMaxBatchPerLaunch + 1];
@@ -346,6 +348,12 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
           v = __bfloat162float(p.q[((size_t)b * p.n_q_heads + (size_t)(kvh0 + hh) * G) * 128 + rem]) * p.scale_log2e;
         (&t.qs[0][0][0])[idx] = v;
       }
+      if constexpr (ROPE) {
+        // a bias on predicted keys is rotated with them, so it no longer cancels in the softmax
+        const int hh = et >> 7, j = et & 127;
+        t.kb[hh][j] = (p.bk != nullptr && (hh == 0 || second))
+                          ? __bfloat162float(p.bk[(size_t)(w.pair * 2 + hh) * 128 + j]) : 0.f;
+      }
 
       // ---------------- K phase: scores and probabilities ----------------
       // (the vote is also the barrier that publishes the queries staged above)
@@ -373,8 +381,9 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
             tmem_ld16(t_addr + hh * 128 + 64 + cb * 16, hi);
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const float r_lo = lo[j] * cs[j].x - hi[j] * cs[j].y;
-              const float r_hi = hi[j] * cs[j].x + lo[j] * cs[j].y;
+              const float k_lo = lo[j] + t.kb[hh][cb * 16 + j], k_hi = hi[j] + t.kb[hh][64 + cb * 16 + j];
+              const float r_lo = k_lo * cs[j].x - k_hi * cs[j].y;
+              const float r_hi = k_hi * cs[j].x + k_lo * cs[j].y;
 #pragma unroll
               for (int gi = 0; gi < G; ++gi)
                 sc[hh][gi] = fmaf(r_hi, t.qs[hh][gi][64 + cb * 16 + j], fmaf(r_lo, t.qs[hh][gi][cb * 16 + j], sc[hh][gi]));
@@ -661,6 +670,7 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
   p.n_sink = r.n_sink;
   p.n_window = r.n_window;
   p.rope = a.rope;
+  p.bk = reinterpret_cast<const __nv_bfloat16*>(r.bk);
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;

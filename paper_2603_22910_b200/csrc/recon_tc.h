@@ -45,6 +45,14 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
 cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
                               const TcLayerMaps& layer, int sm_count, cudaStream_t stream);
 
+// The K half of the same kernel for rotated keys (a.rope must be set): Eq. 3 for the dropped heads' keys, the
+// rotation, q . k -- and the scores go to scores[b][query head][l_cap] (base-2 units; token slots that hold no
+// predicted token get -inf, whole 256-token tiles are written) instead of into a softmax.  The V side is then
+// evaluated with absorbed predictors.
+cudaError_t launch_recon_pair_key_scores(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                                         const TcLayerMaps& layer, float* scores, int l_cap, int sm_count,
+                                         cudaStream_t stream);
+
 constexpr int kPairPartTokens = 128;
 
 }  // namespace echokv

@@ -373,6 +373,154 @@ cudaError_t launch_attn_stored(const AttnArgs& a, const void* k_pool, const void
 }
 
 // ---------------------------------------------------------------------------------------------
+// Scores of stored heads whose keys are rotated when read: S[b][h][t] = q_h . R_t k_t (base-2 units) for the
+// query heads of KV heads 0 .. n_heads-1, one thread per token; token slots that hold no predicted token get
+// -inf.  Feeds the softmax of the absorbed V side when the K side has to be explicit (rotated keys).
+// ---------------------------------------------------------------------------------------------
+// Shared memory of key_scores_stored_kernel: everything the per-token loop reads, so that loop never waits on
+// global memory.
+template <int DH>
+struct KeyScoresSmem {
+  static constexpr int kRowPad = DH * 2 + 16;        // staged key rows: 16-byte reads of successive rows hit all banks
+  static constexpr int kFinePad = DH / 2 + 1;        // fine-angle rows: 8-byte reads of successive rows hit all banks
+  float qs[kMaxGroup][DH];
+  float2 fine[kRopeFineRows][kFinePad];              // (cos, sin) of offsets 0 .. 15
+  float2 coarse[128 / kRopeFineRows][DH / 2];        // (cos, sin) of the block's eight 16-token groups
+  long long rows[128];                               // pool row of each token, -1 = nothing to read
+  __align__(16) unsigned char ks[128 * kRowPad];     // the block's 128 key rows of this head
+};
+
+template <int DH, int G>
+__global__ void __launch_bounds__(128) key_scores_stored_kernel(AttnArgs a, const __nv_bfloat16* __restrict__ k_pool,
+                                                                int width, float* __restrict__ S, int l_cap,
+                                                                int n_sink, int n_window) {
+  extern __shared__ __align__(16) unsigned char key_scores_smem[];
+  KeyScoresSmem<DH>& sm = *reinterpret_cast<KeyScoresSmem<DH>*>(key_scores_smem);
+  constexpr int kRowPad = KeyScoresSmem<DH>::kRowPad;
+  // heads fastest: the blocks that run together read neighbouring pieces of the same cache rows
+  const int b = blockIdx.z, kvh = blockIdx.x, tid = threadIdx.x;
+  const int t0 = blockIdx.y * 128, t = t0 + tid;
+  constexpr int g = G;
+  const int slot = a.slots ? a.slots[b] : b;
+  const int len = a.lens[b];
+  if (slot < 0 || slot >= a.geom.max_batch || len < 1 || len > a.geom.max_pages_per_seq * a.geom.page_tokens)
+    return;                                    // (reported by the other kernels of the call)
+  if (t0 >= ((len + 255) / 256) * 256) return;     // whole 256-token tiles are written, no more
+  const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
+  for (int idx = tid; idx < g * DH; idx += 128)
+    sm.qs[idx / DH][idx % DH] = __bfloat162float(q[((size_t)b * a.n_q_heads + (size_t)kvh * g) * DH + idx]) * a.scale_log2e;
+  // the angle of token 16 u + r is the sum of a coarse one (row u) and a fine one (row r)
+  for (int idx = tid; idx < kRopeFineRows * (DH / 2); idx += 128)
+    sm.fine[idx / (DH / 2)][idx % (DH / 2)] = a.rope.fine[idx];
+  for (int idx = tid; idx < (128 / kRopeFineRows) * (DH / 2); idx += 128) {
+    const int u = min(t0 / kRopeFineRows + idx / (DH / 2), a.rope.stride / kRopeFineRows - 1);
+    sm.coarse[idx / (DH / 2)][idx % (DH / 2)] = a.rope.coarse[(size_t)u * (DH / 2) + idx % (DH / 2)];
+  }
+  const bool valid = t < l_cap && t >= predicted_lo(len, n_sink) && t < predicted_hi(len, n_sink, n_window);
+  long long row = -1;
+  if (valid) {
+    const int page = a.geom.table[(size_t)slot * a.geom.max_pages_per_seq + t / a.geom.page_tokens];
+    if (page < 0 || page >= a.geom.n_pages) report(a.status, ECHOKV_EBADPAGE);
+    else row = (long long)page * a.geom.page_tokens + t % a.geom.page_tokens;
+  }
+  sm.rows[tid] = row;
+  __syncthreads();
+  // stage the rows with coalesced reads, 16 lanes x 16 bytes per row; all of a thread's loads are issued before
+  // the first store so that they overlap
+  constexpr int kVecPerRow = DH * 2 / 16;
+  static_assert(kVecPerRow == 16, "one row per 16 lanes");
+  {
+    const int v = tid % kVecPerRow, r0 = tid / kVecPerRow;
+    uint4 buf[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const long long src_row = sm.rows[r0 + 8 * i];
+      buf[i] = src_row >= 0 ? __ldg(reinterpret_cast<const uint4*>(k_pool + (size_t)src_row * width + (size_t)kvh * DH) + v)
+                            : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) *reinterpret_cast<uint4*>(sm.ks + (r0 + 8 * i) * kRowPad + v * 16) = buf[i];
+  }
+  __syncthreads();
+  if (t >= l_cap) return;
+  float acc[G];
+#pragma unroll
+  for (int gi = 0; gi < G; ++gi) acc[gi] = 0.f;
+  if (row >= 0) {
+    const unsigned char* kr = sm.ks + tid * kRowPad;
+    const float2* fine = sm.fine[tid % kRopeFineRows];
+    const float4* coarse = reinterpret_cast<const float4*>(sm.coarse[tid / kRopeFineRows]);
+#pragma unroll 2
+    for (int j = 0; j < DH / 2; j += 8) {
+      const uint4 lo4 = *reinterpret_cast<const uint4*>(kr + j * 2);
+      const uint4 hi4 = *reinterpret_cast<const uint4*>(kr + DH + j * 2);
+      const uint32_t lw[4] = {lo4.x, lo4.y, lo4.z, lo4.w}, hw[4] = {hi4.x, hi4.y, hi4.z, hi4.w};
+      float r_lo[8], r_hi[8];          // the eight rotated feature pairs
+#pragma unroll
+      for (int e2 = 0; e2 < 4; ++e2) {
+        const float4 cw = coarse[j / 2 + e2];            // coarse (cos, sin) of frequency indices j + 2 e2 and + 1
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int e = 2 * e2 + h;
+          const float k_lo = h ? __uint_as_float(lw[e2] & 0xffff0000u) : __uint_as_float(lw[e2] << 16);
+          const float k_hi = h ? __uint_as_float(hw[e2] & 0xffff0000u) : __uint_as_float(hw[e2] << 16);
+          const float2 fw = fine[j + e];
+          const float cc = h ? cw.z : cw.x, cs_ = h ? cw.w : cw.y;
+          const float c = cc * fw.x - cs_ * fw.y, sn = cs_ * fw.x + cc * fw.y;
+          r_lo[e] = k_lo * c - k_hi * sn;
+          r_hi[e] = k_hi * c + k_lo * sn;
+        }
+      }
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) {
+        const float4* ql = reinterpret_cast<const float4*>(&sm.qs[gi][j]);
+        const float4* qh = reinterpret_cast<const float4*>(&sm.qs[gi][DH / 2 + j]);
+        const float4 l0 = ql[0], l1 = ql[1], h0 = qh[0], h1 = qh[1];
+        float v = acc[gi];
+        v = fmaf(r_lo[0], l0.x, v); v = fmaf(r_lo[1], l0.y, v); v = fmaf(r_lo[2], l0.z, v); v = fmaf(r_lo[3], l0.w, v);
+        v = fmaf(r_lo[4], l1.x, v); v = fmaf(r_lo[5], l1.y, v); v = fmaf(r_lo[6], l1.z, v); v = fmaf(r_lo[7], l1.w, v);
+        v = fmaf(r_hi[0], h0.x, v); v = fmaf(r_hi[1], h0.y, v); v = fmaf(r_hi[2], h0.z, v); v = fmaf(r_hi[3], h0.w, v);
+        v = fmaf(r_hi[4], h1.x, v); v = fmaf(r_hi[5], h1.y, v); v = fmaf(r_hi[6], h1.z, v); v = fmaf(r_hi[7], h1.w, v);
+        acc[gi] = v;
+      }
+    }
+  }
+#pragma unroll
+  for (int gi = 0; gi < G; ++gi)
+    S[((size_t)b * a.n_q_heads + (size_t)kvh * G + gi) * l_cap + t] = row >= 0 ? acc[gi] : -INFINITY;
+}
+
+template <int G>
+static cudaError_t launch_key_scores_stored_g(const AttnArgs& a, const void* k_pool, int width, int n_heads, float* S,
+                                              int l_cap, int n_sink, int n_window, cudaStream_t stream) {
+  const size_t smem = sizeof(KeyScoresSmem<128>);
+  cudaError_t e = cudaFuncSetAttribute(key_scores_stored_kernel<128, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  // several blocks per SM: ask for the largest shared-memory carve-out
+  e = cudaFuncSetAttribute(key_scores_stored_kernel<128, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared);
+  if (e != cudaSuccess) return e;
+  dim3 grid(n_heads, (l_cap + 127) / 128, a.batch);
+  key_scores_stored_kernel<128, G><<<grid, 128, smem, stream>>>(a, reinterpret_cast<const __nv_bfloat16*>(k_pool), width,
+                                                                S, l_cap, n_sink, n_window);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_key_scores_stored(const AttnArgs& a, const void* k_pool, int width, int n_heads, float* S,
+                                     int l_cap, int n_sink, int n_window, cudaStream_t stream) {
+  if (n_heads == 0) return cudaSuccess;
+  if (a.dtype != ECHOKV_BF16 || a.head_dim != 128 || a.rope.cs == nullptr) return cudaErrorInvalidValue;
+  switch (a.n_q_heads / a.n_kv_heads) {
+    case 1: return launch_key_scores_stored_g<1>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
+    case 2: return launch_key_scores_stored_g<2>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
+    case 4: return launch_key_scores_stored_g<4>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
+    case 8: return launch_key_scores_stored_g<8>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // CUDA-core reconstruct-then-attend (Eq. 3, 6, 7 for one dropped KV head and one token range)
 // ---------------------------------------------------------------------------------------------
 constexpr int kKc = 32;   // features per staged chunk of the predictor input
@@ -384,6 +532,7 @@ struct ReconSmem {
   float Hs[kSimtTileTokens][DH + 1];       // predicted K (then V) tile of the head
   float Ss[kMaxGroup][kSimtTileTokens];    // scores, then probabilities
   float qs[kMaxGroup][DH];                 // queries * scale * log2e
+  float kb[DH];                            // bias of the K predictor for this head (only with a rotation)
   float m_run[kMaxGroup], l_run[kMaxGroup], alpha[kMaxGroup];
 };
 
@@ -496,6 +645,9 @@ __global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r
     sm.m_run[tid] = -INFINITY;
     sm.l_run[tid] = 0.f;
   }
+  // (a bias on predicted keys is rotated with them, so it does not cancel in the softmax then)
+  for (int j = tid; j < DH; j += 128)
+    sm.kb[j] = r.bk != nullptr ? to_f32(reinterpret_cast<const T*>(r.bk)[(size_t)(kvh - n_ret) * DH + j]) : 0.f;
   float o[kMaxGroup];
 #pragma unroll
   for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
@@ -525,7 +677,7 @@ __global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r
 #pragma unroll 8
           for (int j = 0; j < DH / 2; ++j) {
             const float2 w = cs[(size_t)j * a.rope.stride];
-            const float k_lo = sm.Hs[t][j], k_hi = sm.Hs[t][j + DH / 2];
+            const float k_lo = sm.Hs[t][j] + sm.kb[j], k_hi = sm.Hs[t][j + DH / 2] + sm.kb[j + DH / 2];
             s = fmaf(sm.qs[gi][j], k_lo * w.x - k_hi * w.y, s);
             s = fmaf(sm.qs[gi][j + DH / 2], k_hi * w.x + k_lo * w.y, s);
           }

@@ -63,26 +63,69 @@ def test_rope_against_oracle(name, base, over, lens, window):
     case.close()
 
 
-def test_rope_and_absorbed_mode_exclude_each_other():
-    w = synth.C2.replace(batch=1, context=300)
-    case = Case(w, lens=[300], layers=[1], rope=THETA)
-    n = C.c_uint64(0)
-    assert binding.lib().echokv_absorbed_workspace_bytes(C.byref(case.cfg), C.byref(n)) == binding.ECHOKV_OK
-    buf = torch.empty(n.value, dtype=torch.uint8, device="cuda")
-    assert binding.lib().echokv_enable_absorbed(case.ctx.handle, buf.data_ptr(), n.value) == binding.ECHOKV_EUNSUPPORTED
-    case.ctx.set_rope(0)
-    case.ctx.enable_absorbed()
-    with pytest.raises(binding.EchoKVError) as e:
-        case.ctx.set_rope(THETA)
-    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
-    case.ctx.set_decode_mode(0)
-    case.ctx.set_rope(THETA)
-    with pytest.raises(binding.EchoKVError) as e:
-        case.ctx.set_decode_mode(1)
-    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
-    case.rope = THETA
-    assert_parity(case.run(1), case.oracle(1), w.dtype, "explicit mode with rope after the switches")
+@pytest.mark.parametrize("base,over,lens", [
+    (synth.C2, dict(batch=2, context=600), [600, 131]),
+    (synth.C0, dict(batch=2, context=200), [200, 50]),
+], ids=["bf16_gqa", "fp32_d64"])
+def test_rope_with_predictor_biases(base, over, lens):
+    # a bias on the K predictor is rotated with the predicted keys: it does not cancel in the softmax any more
+    w = base.replace(**over)
+    case = Case(w, lens=lens, layers=[0, 1], biases=True, rope=THETA)
+    ref = case.oracle(1)
+    for path in ([1, 2, 3] if case.ctx.decode_path() >= 2 else [1]):
+        case.ctx.set_decode_path(path)
+        assert_parity(case.run(1), ref, w.dtype, "biases path %d" % path)
+    Wk, Wv, bk, bv = case.weights[1]
+    case.ctx.set_weights(1, Wk, Wv, None, bv)
+    assert errors(case.run(1), ref)[1] > 1e-3          # without the K bias the result is another one
+    assert case.ctx.device_status() == binding.ECHOKV_OK
     case.close()
+
+
+MIXED = [
+    # name, base, overrides, lens, window, biases
+    ("c2_shape", synth.C2, dict(batch=3, context=1000), [1000, 517, 256], None, False),
+    ("c1_shape", synth.C1, dict(batch=2, context=700), [700, 333], None, False),
+    ("pages64_random", synth.C2, dict(batch=2, context=600, page_tokens=64, random_pages=True), [600, 65], None, False),
+    ("ragged_many_tiles", synth.C2, dict(batch=5, context=2000, random_pages=True), [2000, 129, 128, 1153, 1], None, True),
+    ("window", synth.C2, dict(batch=3, context=1000, random_pages=True), [1000, 517, 100], (4, 128), False),
+    ("nothing_retained", synth.C2, dict(batch=2, context=700, n_retained_heads=0), [700, 300], None, True),
+    ("one_dropped_head", synth.C2, dict(batch=2, context=400, n_retained_heads=7), [400, 258], (2, 40), False),
+]
+
+
+@pytest.mark.parametrize("name,base,over,lens,window,biases", MIXED, ids=[c[0] for c in MIXED])
+def test_rotated_keys_with_the_absorbed_value_side(name, base, over, lens, window, biases):
+    # with rotated keys the absorbed mode keeps the K side explicit and absorbs the V side only
+    w = base.replace(**over)
+    case = Case(w, lens=lens, layers=[0, 1], window=window, biases=biases, rope=THETA)
+    ref = case.oracle(1)
+    assert_parity(case.run(1), ref, w.dtype, name + " explicit")
+    case.ctx.enable_absorbed()
+    assert case.ctx.decode_mode() == 1 and case.ctx.rope_enabled()
+    out = case.run(1)
+    assert_parity(out, ref, w.dtype, name + " K explicit, V absorbed")
+    np.testing.assert_array_equal(case.run(1), out)             # and it is repeatable
+    assert_parity(case.run(0), case.oracle(0), w.dtype, name + " anchor")
+    # the order of the two switches does not matter, and without the table the mode is the fully absorbed one
+    case.ctx.set_rope(0)
+    case.rope = None
+    assert_parity(case.run(1), case.oracle(1), w.dtype, name + " absorbed, no rotation")
+    case.ctx.set_rope(THETA)
+    case.rope = THETA
+    assert_parity(case.run(1), ref, w.dtype, name + " table set after the mode")
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+def test_rope_needs_whole_heads():
+    w = synth.C2.replace(batch=1, context=300, n_retained_dims=64)
+    cfg = binding.config_for(w)
+    ctx = binding.Context(cfg)
+    with pytest.raises(binding.EchoKVError) as e:
+        ctx.set_rope(THETA)
+    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
+    ctx.close()
 
 
 def test_rope_argument_checks():
