@@ -355,51 +355,49 @@ def run_reference(args):
                          args.retained_dims)
     st = synth.to_numpy_stored
     full = args.mode == "full"
-    layer = 0 if full else 1
-    a = w.anchor_of(layer)
-    q = O.widen(st(synth.queries(w, layer)))[0]
-    kg = O.widen(st(synth.layer_cache(w, a, "k", 0)))
-    vg = O.widen(st(synth.layer_cache(w, a, "v", 0)))
-    g = w.n_q_heads // w.n_kv_heads
-    total = args.steps + args.warmup
-    budget = 150.0
-    if full:
-        n_units, heads = w.n_kv_heads, list(range(w.n_q_heads))
-        d = w.head_dim
+    rope = args.rope or None
+    # The same sampling as the cpu_baseline leg: whole sequences, all heads, all tokens.  A step evaluates
+    # sequence 0 of the batch for one layer (single-layer workloads) or for one group of S consecutive layers
+    # (the 32-layer workload: every group costs the same); the result is scaled to the batch and the layers.
+    multi = w.n_layers > 2 and not full
+    layers = list(range(w.group_size)) if multi else [0 if full else 1]
+    inputs = {}
+    for l in layers:
+        a = w.anchor_of(l)
+        q = O.widen(st(synth.queries(w, l)))[0]
+        kg = O.widen(st(synth.layer_cache(w, a, "k", 0)))
+        vg = O.widen(st(synth.layer_cache(w, a, "v", 0)))
+        if full or w.is_anchor(l):
+            inputs[l] = (q, kg, vg)
+        else:
+            inputs[l] = (q, kg, vg,
+                         O.widen(st(synth.layer_cache(w, l, "k", 0, width=w.m))),
+                         O.widen(st(synth.layer_cache(w, l, "v", 0, width=w.m))),
+                         O.widen(st(synth.predictor_weights(w, l, "k"))),
+                         O.widen(st(synth.predictor_weights(w, l, "v"))))
 
-        def run(n_kv):   # the first n_kv KV heads of the stored cache
-            return O.full_attention(q[: n_kv * g], kg[:, : n_kv * d], vg[:, : n_kv * d], n_kv,
-                                    rope_theta=args.rope or None)
-    else:
-        kl = O.widen(st(synth.layer_cache(w, layer, "k", 0, width=w.m)))
-        vl = O.widen(st(synth.layer_cache(w, layer, "v", 0, width=w.m)))
-        Wk = O.widen(st(synth.predictor_weights(w, layer, "k")))
-        Wv = O.widen(st(synth.predictor_weights(w, layer, "v")))
-        n_units = w.n_kv_heads - w.n_retained_heads
-        heads = list(range(w.n_retained_heads * g, w.n_q_heads))
+    def run():
+        for l in layers:
+            x = inputs[l]
+            if len(x) == 3:
+                O.full_attention(x[0], x[1], x[2], w.n_kv_heads, rope_theta=rope)
+            else:
+                O.decode_attention(*x, n_kv_heads=w.n_kv_heads, rope_theta=rope)
 
-        def run(n_kv):   # the first n_kv dropped KV heads (the retained ones cost next to nothing)
-            return O.decode_attention_query_heads(q, kg, vg, kl, vl, Wk, Wv, n_kv_heads=w.n_kv_heads,
-                                                  query_heads=heads[: n_kv * g], rope_theta=args.rope or None)
-    t0 = time.perf_counter()
-    run(1)
-    t_head = time.perf_counter() - t0
-    n_sample = max(1, min(n_units, int(budget / max(total * t_head, 1e-9))))
     times = []
-    for i in range(total):
+    for i in range(args.steps + args.warmup):
         t0 = time.perf_counter()
-        run(n_sample)
+        run()
         dt = time.perf_counter() - t0
         if i >= args.warmup:
             times.append(dt)
-    # a step covers n_sample of the n_units KV heads of ONE of the B sequences of ONE layer
-    n_attend = w.n_layers if (w.n_layers > 2 and not full) else 1
     t_step = sum(times) / len(times)
-    t_batch = t_step / (n_sample / float(n_units)) * w.batch * n_attend
+    n_attend = w.n_layers if multi else 1
+    t_batch = t_step * w.batch * (n_attend / float(len(layers)))
     value = w.batch / t_batch
-    sample = ("sequence 0 of %d, %d of %d %s KV heads per step (all %d tokens), one layer; scaled to the full "
-              "batch%s" % (w.batch, n_sample, n_units, "stored" if full else "dropped", w.context,
-                           " and to %d layers" % n_attend if n_attend > 1 else ""))
+    sample = ("sequence 0 of %d per step, %s, all heads, all %d tokens; scaled to the full batch%s"
+              % (w.batch, "layers 0..%d (one group of S = %d)" % (w.group_size - 1, w.group_size) if multi
+                 else "one layer", w.context, " and to %d layers" % n_attend if multi else ""))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_batch * 1e3,
