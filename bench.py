@@ -54,7 +54,8 @@ def traffic_of(args, key):
     """The stored ncu figure, only for the exact workload it was scaled to."""
     if args.batch or args.context or args.page_tokens or args.random_pages:
         return None
-    if args.rope or args.window or args.retained_dims or args.decode_path is not None or args.stored_path is not None:
+    if (args.rope or args.window or args.retained_dims or args.save_k or args.decode_path is not None
+            or args.stored_path is not None):
         return None          # another kernel (instantiation) than the captured one
     return NCU_TRAFFIC_BYTES.get(key)
 
@@ -67,8 +68,12 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def workload_by_name(name, batch=0, context=0, page_tokens=0, random_pages=False, ratio=75, retained_dims=0):
+def workload_by_name(name, batch=0, context=0, page_tokens=0, random_pages=False, ratio=75, retained_dims=0,
+                     save_k=False):
     from paper_2603_22910_b200 import synth
+    if save_k:    # keys kept whole on compressed layers, only the values predicted (the paper's "save K" setting)
+        w = workload_by_name(name, batch, context, page_tokens, random_pages, ratio, retained_dims)
+        return w.replace(save_k=True, name=w.name + "_saveK")
     if name == "c4":
         w = synth.c4_point(ratio, context or 16384, batch or 8)
         if retained_dims:   # the paper's own settings, e.g. m = 64: half of the first head (absorbed mode only)
@@ -185,8 +190,8 @@ class State:
         tdt = synth.torch_dtype(w)
         self.new_dev, self.new_host, self.q_dev, self.q_host = {}, {}, {}, {}
         for l in needed:
-            width = w.D if w.is_anchor(l) else w.m
             for kind, pools in (("k", ctx.k_pools), ("v", ctx.v_pools)):
+                width = w.D if w.is_anchor(l) else (w.mk if kind == "k" else w.m)
                 newest = torch.zeros((w.batch, w.D), dtype=tdt, device=dev)
                 for b in range(w.batch):
                     if width == 0:
@@ -221,7 +226,7 @@ class State:
             if not w.is_anchor(l):
                 Wk = synth.predictor_weights(w, l, "k", device=dev)
                 Wv = synth.predictor_weights(w, l, "v", device=dev)
-                ctx.set_weights(l, Wk, Wv)
+                ctx.set_weights(l, None if w.save_k else Wk, Wv)
             self.q_dev[l] = synth.queries(w, l, device=dev)
             self.q_host[l] = self.q_dev[l].cpu().pin_memory()
         self.lens_host = torch.full((w.batch,), w.context, dtype=torch.int32).pin_memory()
@@ -255,10 +260,18 @@ class State:
         vg = O.widen(st(self.stored_sequence(a, "v", b)))
         if w.is_anchor(layer):
             return q, kg, vg
-        kl = O.widen(st(self.stored_sequence(layer, "k", b)))
+        kl = O.widen(st(self.stored_sequence(layer, "k", b)))[:, :w.m]
         vl = O.widen(st(self.stored_sequence(layer, "v", b)))
-        Wk, Wv = (O.widen(st(t)) for t in self.ctx._weights[layer][:2])
+        Wk, Wv = (None if t is None else O.widen(st(t)) for t in self.ctx._weights[layer][:2])
         return q, kg, vg, kl, vl, Wk, Wv
+
+    def true_keys(self, layer, b):
+        """The layer's whole keys [L, D] where it keeps them ("save K"), else None."""
+        from oracle import echokv_oracle as O
+        from paper_2603_22910_b200 import synth
+        if not self.w.save_k or self.w.is_anchor(layer):
+            return None
+        return O.widen(synth.to_numpy_stored(self.stored_sequence(layer, "k", b)))
 
     def true_dropped(self, layer, kind, b):
         """[L, D - m] with the sink / window tokens' own dims m..D-1 (NaN elsewhere: never read)."""
@@ -306,7 +319,8 @@ def oracle_layer(inputs, w, state=None, layer=None, b=None):
         return O.decode_attention_windowed(*inputs, w.n_kv_heads, state.true_dropped(layer, "k", b),
                                            state.true_dropped(layer, "v", b), state.window[0], state.window[1],
                                            rope_theta=rope)
-    return O.decode_attention(*inputs, n_kv_heads=w.n_kv_heads, rope_theta=rope)
+    k_true = state.true_keys(layer, b) if state is not None else None
+    return O.decode_attention(*inputs, n_kv_heads=w.n_kv_heads, rope_theta=rope, k_true=k_true)
 
 
 def time_oracle(state, step_layers, budget_s):
@@ -352,7 +366,7 @@ def run_reference(args):
     from oracle import echokv_oracle as O
     from paper_2603_22910_b200 import synth
     w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio,
-                         args.retained_dims)
+                         args.retained_dims, args.save_k)
     st = synth.to_numpy_stored
     full = args.mode == "full"
     rope = args.rope or None
@@ -361,7 +375,7 @@ def run_reference(args):
     # (the 32-layer workload: every group costs the same); the result is scaled to the batch and the layers.
     multi = w.n_layers > 2 and not full
     layers = list(range(w.group_size)) if multi else [0 if full else 1]
-    inputs = {}
+    inputs, k_true = {}, {}
     for l in layers:
         a = w.anchor_of(l)
         q = O.widen(st(synth.queries(w, l)))[0]
@@ -370,6 +384,7 @@ def run_reference(args):
         if full or w.is_anchor(l):
             inputs[l] = (q, kg, vg)
         else:
+            k_true[l] = O.widen(st(synth.layer_cache(w, l, "k", 0, width=w.D))) if w.save_k else None
             inputs[l] = (q, kg, vg,
                          O.widen(st(synth.layer_cache(w, l, "k", 0, width=w.m))),
                          O.widen(st(synth.layer_cache(w, l, "v", 0, width=w.m))),
@@ -382,7 +397,7 @@ def run_reference(args):
             if len(x) == 3:
                 O.full_attention(x[0], x[1], x[2], w.n_kv_heads, rope_theta=rope)
             else:
-                O.decode_attention(*x, n_kv_heads=w.n_kv_heads, rope_theta=rope)
+                O.decode_attention(*x, n_kv_heads=w.n_kv_heads, rope_theta=rope, k_true=k_true[l])
 
     times = []
     for i in range(args.steps + args.warmup):
@@ -499,7 +514,7 @@ def run_ours(args):
     binding.lib()
 
     w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio,
-                         args.retained_dims)
+                         args.retained_dims, args.save_k)
     w = w.replace(seed=rep.seed_for(w.seed))
     full = args.mode == "full"
     resident, step_layers = plan_layers(w, args.mode)
@@ -634,6 +649,8 @@ def run_ours(args):
         ak_ms, ak_n = timing["absorb_k"]
         av_ms, av_n = timing["absorb_v"]
         k_ms = (ak_ms + av_ms) / max(ak_n, 1)
+        if w.save_k:      # the K pass streams the layer's own D key dims instead of [anchor ; retained]
+            bytes_ = w.batch * w.context * float(w.D + w.d_in) * elem
         achieved_gbs = bytes_ / (k_ms * 1e-3) / 1e9
         peak_gbs = float(peaks["hbm_gbs"])
         roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
@@ -645,7 +662,10 @@ def run_ours(args):
                     "peak_source": "%s (STREAM-style copy)" % peaks_kind,
                     "algorithmic_bytes_per_launch": bytes_,
                     "mode": "absorbed predictors: the same outputs as the explicit path, a separate roofline row"}
-        if args.rope:
+        if args.rope and w.save_k:
+            roofline["kernel"] = "key_scores_stored_kernel + absorb_pv_kernel"
+            roofline["mode"] = "keys kept whole and rotated when read: stored-key scores, V side with absorbed predictors"
+        elif args.rope:
             # rotated keys: the K side is explicit (Eq. 3 for the keys on the tensor cores, rotation, scores), only
             # the V side is absorbed; the K pass is the dominant kernel and tensor-bound
             tokens = float(w.batch) * w.context
@@ -754,6 +774,8 @@ def main():
                                                  "paper's setting); default none, as the benchmark configs state")
     ap.add_argument("--rope", type=float, default=0.0, help="theta of a rotary embedding applied when the cache is "
                     "read (the cache then holds un-rotated keys); 0 = none, as in the paper's configurations")
+    ap.add_argument("--save-k", action="store_true", help="compressed layers keep their keys whole, only the values "
+                    "are predicted (the paper's \"save K\" ablation); needs --decode-mode absorbed")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")

@@ -84,11 +84,17 @@ typedef struct {
                                 retained head is served by the absorbed mode only: echokv_create succeeds
                                 where that mode is available (EUNSUPPORTED otherwise) and
                                 echokv_decode_attention returns EUNSUPPORTED until echokv_enable_absorbed */
+  int32_t save_k;            /* non-zero: the "save K" setting of Section 5.2 -- compressed layers keep their keys
+                                whole (K pools of width D, nothing of K is predicted, Wk may be NULL) and only the
+                                values are evicted and predicted.  Served by the absorbed mode only (as above);
+                                not combined with echokv_set_full_precision_window or echokv_compress_layer
+                                (EUNSUPPORTED) */
 } echokv_config;
 
 typedef struct {
   uint64_t anchor_pool_bytes;     /* one K (or V) pool of an anchor layer                  */
-  uint64_t compressed_pool_bytes; /* one K (or V) pool of a compressed layer (0 if m = 0)  */
+  uint64_t compressed_pool_bytes; /* one K (or V) pool of a compressed layer (0 if m = 0); with
+                                     save_k the K pools of compressed layers have anchor_pool_bytes */
   uint64_t block_table_bytes;
   uint64_t workspace_bytes;       /* minimum size of echokv_buffers.workspace              */
   int32_t max_partials;           /* split-K partial results kept per (sequence, head)     */
@@ -197,7 +203,7 @@ int echokv_decode_path(const echokv_ctx* ctx);
  * the fastest family their shape allows.  Meant for tests that check all against the oracle. */
 int echokv_set_decode_path(echokv_ctx* ctx, int path);
 
-/* Sink and recent-window tokens at full precision (Section 5.1, "Implement details": the paper keeps
+/* Sink and recent-window tokens at full precision (Section 4.1, "Implement details": the paper keeps
  * 4 sink tokens and a local window of 128 tokens uncompressed).  With (n_sink, n_window) set, the first
  * n_sink and the last n_window tokens of every sequence are never predicted: the dims m .. D-1 of those
  * tokens are kept in per-layer side buffers and Eq. 7 uses them as stored; every other token is

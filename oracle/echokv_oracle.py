@@ -27,7 +27,7 @@ Readings of points the paper leaves open (all listed in the design notes):
   * flattening is head-major: flat index = head * d + feature.
   * query head h attends KV head floor(h / (H_q / H_kv)) (contiguous groups).
   * every cached token, the newest included, is reconstructed alike, unless a
-    sink / recent window is asked for (Section 5.1): those tokens keep all dims.
+    sink / recent window is asked for (Section 4.1): those tokens keep all dims.
   * the predictors see keys BEFORE the rotary position embedding (Section 3.2), so a
     cache of such keys must be rotated when it is read: with rope_theta given, every
     row t of K_tilde (retained, predicted or full-precision alike) is rotated to
@@ -248,7 +248,7 @@ def decode_attention(q: np.ndarray,
                      Wk: np.ndarray, Wv: np.ndarray,
                      n_kv_heads: int, scale: float | None = None,
                      bk: np.ndarray | None = None, bv: np.ndarray | None = None,
-                     rope_theta: float | None = None) -> np.ndarray:
+                     rope_theta: float | None = None, k_true: np.ndarray | None = None) -> np.ndarray:
     """One decode step of a compressed layer for one sequence.
 
     k_global, v_global [L, D]  full cache of the group's anchor layer   (Eq. 1)
@@ -257,13 +257,19 @@ def decode_attention(q: np.ndarray,
     q [H_q, d]                 the new token's queries
     Steps: predict the dropped dims (Eq. 3), rebuild K_tilde, V_tilde (Eq. 6),
     (rotate K_tilde by position if rope_theta is given), attend (Eq. 7).  Returns [H_q, d].
+    k_true [L, D]: the "save K" setting of Section 5.2 -- the layer's keys are kept whole and
+    used as they are (k_local, Wk, bk are ignored); reconstruction applies to the values only.
     """
     k_global = np.asarray(k_global, dtype=np.float64)
     D = k_global.shape[1]
     d = D // n_kv_heads
-    k_hat = reconstruct_dropped(Wk, k_global, k_local, bk)
     v_hat = reconstruct_dropped(Wv, v_global, v_local, bv)
-    K_t = assemble_cache(k_local, k_hat, n_kv_heads, d)
+    if k_true is not None:
+        K_t = np.asarray(k_true, dtype=np.float64).reshape(-1, n_kv_heads, d)
+        if K_t.shape[0] != k_global.shape[0]:
+            raise ValueError("token counts differ")
+    else:
+        K_t = assemble_cache(k_local, reconstruct_dropped(Wk, k_global, k_local, bk), n_kv_heads, d)
     V_t = assemble_cache(v_local, v_hat, n_kv_heads, d)
     return attention(q, K_t, V_t, scale, rope_theta)
 
@@ -319,7 +325,7 @@ def decode_attention_query_heads(q: np.ndarray,
 
 
 # ----------------------------------------------------------------------------
-# Sink and recent-window tokens kept at full precision (Section 5.1, "Implement
+# Sink and recent-window tokens kept at full precision (Section 4.1, "Implement
 # details": 4 sink tokens and a local window of 128 tokens)
 # ----------------------------------------------------------------------------
 

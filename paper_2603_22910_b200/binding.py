@@ -26,7 +26,7 @@ class echokv_config(C.Structure):
                 ("head_dim", C.c_int32), ("group_size", C.c_int32), ("n_retained_heads", C.c_int32),
                 ("page_tokens", C.c_int32), ("max_batch", C.c_int32), ("max_pages_per_seq", C.c_int32),
                 ("dtype", C.c_int32), ("n_pages", C.c_int64), ("softmax_scale", C.c_float),
-                ("device", C.c_int32), ("n_retained_dims", C.c_int32)]
+                ("device", C.c_int32), ("n_retained_dims", C.c_int32), ("save_k", C.c_int32)]
 
 
 class echokv_sizes(C.Structure):
@@ -129,10 +129,10 @@ def _stream_handle(stream) -> int | None:
 
 def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_retained_heads,
                 page_tokens, max_batch, max_pages_per_seq, n_pages, dtype, softmax_scale=0.0,
-                device=0, n_retained_dims=0) -> echokv_config:
+                device=0, n_retained_dims=0, save_k=0) -> echokv_config:
     return echokv_config(n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_retained_heads,
                          page_tokens, max_batch, max_pages_per_seq, dtype, n_pages, softmax_scale, device,
-                         n_retained_dims)
+                         n_retained_dims, save_k)
 
 
 def echokv_query_sizes(cfg: echokv_config) -> echokv_sizes:
@@ -159,15 +159,14 @@ class Context:
         self.D, self.m = D, m
         alloc = torch.zeros if zero_pools else torch.empty
         self.k_pools, self.v_pools = [], []
+        self.mk = D if (cfg.save_k and m < D) else m      # K dims a compressed layer stores ("save K": all of them)
         for l in range(cfg.n_layers):
-            width = D if l % cfg.group_size == 0 else m
-            if width == 0:
-                self.k_pools.append(None)
-                self.v_pools.append(None)
-            else:
-                shape = (cfg.n_pages, cfg.page_tokens, width)
-                self.k_pools.append(alloc(shape, dtype=self.tdtype, device=self.device))
-                self.v_pools.append(alloc(shape, dtype=self.tdtype, device=self.device))
+            for pools, width in ((self.k_pools, D if l % cfg.group_size == 0 else self.mk),
+                                 (self.v_pools, D if l % cfg.group_size == 0 else m)):
+                if width == 0:
+                    pools.append(None)
+                else:
+                    pools.append(alloc((cfg.n_pages, cfg.page_tokens, width), dtype=self.tdtype, device=self.device))
         self.workspace = torch.empty(self.sizes.workspace_bytes, dtype=torch.uint8, device=self.device)
         self.block_table = torch.zeros((cfg.max_batch, cfg.max_pages_per_seq), dtype=torch.int32,
                                        device=self.device)
@@ -347,4 +346,4 @@ def config_for(w, n_pages: int | None = None, device: int = 0, max_batch: int | 
                        n_pages=n_pages or w.batch * pages,
                        dtype=ECHOKV_BF16 if w.dtype == "bf16" else ECHOKV_FP32,
                        softmax_scale=1.0 / math.sqrt(w.head_dim), device=device,
-                       n_retained_dims=w.n_retained_dims)
+                       n_retained_dims=w.n_retained_dims, save_k=1 if w.save_k else 0)

@@ -919,7 +919,11 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   cudaError_t e;
 
   const bool rotated = a.rope.cs != nullptr;
-  if (rotated && (r.m % 128 != 0 || !layer.weights_ready)) return cudaErrorInvalidValue;
+  if (rotated && !r.save_k && (r.m % 128 != 0 || !layer.weights_ready)) return cudaErrorInvalidValue;
+  if (r.save_k && (r.n_sink > 0 || r.n_window > 0)) return cudaErrorInvalidValue;
+  // K side: features [anchor dims ; retained dims] and Wk^T q -- or, where the layer keeps its keys whole, the
+  // layer's own D key dims with every query placed at its head's dims
+  const int k_m = r.save_k ? r.D : r.m, k_anchor_dims = r.save_k ? 0 : r.D;
 
   // 1. absorbed queries
   if (!rotated) {
@@ -933,7 +937,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
       return e;
     absorb_query_kernel<<<grid, 256, kQuerySmemBytes, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q),
                                                   reinterpret_cast<const __nv_bfloat16*>(r.Wk), q2, a.batch,
-                                                  a.n_q_heads, g, r.m, r.D, d_in, a.scale_log2e);
+                                                  a.n_q_heads, g, k_m, k_anchor_dims, d_in, a.scale_log2e);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
 
@@ -975,11 +979,20 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     ra.capacity_tokens = capacity;
     ra.n_sink = r.n_sink; ra.n_window = r.n_window;
     if (ev) cudaEventRecord(ev[0], stream);
-    if ((e = launch_recon_pair_key_scores(a, ra, anchor, layer, S, lay.l_cap, sm_count, stream)) != cudaSuccess) return e;
-    if ((e = launch_key_scores_stored(a, r.k_local, r.m, n_ret, S, lay.l_cap, r.n_sink, r.n_window, stream)) != cudaSuccess)
-      return e;
+    if (r.save_k) {
+      if ((e = launch_key_scores_stored(a, r.k_local, r.D, a.n_kv_heads, S, lay.l_cap, 0, 0, stream)) != cudaSuccess) return e;
+    } else {
+      if ((e = launch_recon_pair_key_scores(a, ra, anchor, layer, S, lay.l_cap, sm_count, stream)) != cudaSuccess) return e;
+      if ((e = launch_key_scores_stored(a, r.k_local, r.m, n_ret, S, lay.l_cap, r.n_sink, r.n_window, stream)) != cudaSuccess)
+        return e;
+    }
     if (ev) cudaEventRecord(ev[1], stream);
   } else {
+    const TcLayerMaps& k_loc = r.save_k ? layer : loc;
+    if (r.save_k) {         // the K pass streams the layer's own keys only
+      p.kc_anchor = 0;
+      p.kc_total = r.D / kChunk;
+    }
     p.stage_bytes = 2u * (kScoreXBytes + (uint32_t)lay.nh2 * kRowBytes);
     p.n_stages = (int)(kSmemBudget / p.stage_bytes);
     if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;
@@ -992,10 +1005,13 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     const long long max_items = (long long)a.batch * ((capacity + kScoreTokens - 1) / kScoreTokens);
     const int grid = (int)(max_items < sm_count ? max_items : sm_count);
     if (ev) cudaEventRecord(ev[0], stream);
-    absorb_scores_kernel<<<grid, kThreads, smem, stream>>>(anchor.k_pool, loc.k_pool, anchor.k_pool_run, loc.k_pool_run,
-                                                           anchor.k_pool_run128, loc.k_pool_run128, maps.q2, p);
+    absorb_scores_kernel<<<grid, kThreads, smem, stream>>>(anchor.k_pool, k_loc.k_pool, anchor.k_pool_run,
+                                                           k_loc.k_pool_run, anchor.k_pool_run128, k_loc.k_pool_run128,
+                                                           maps.q2, p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (ev) cudaEventRecord(ev[1], stream);
+    p.kc_anchor = r.D / kChunk;      // (the V pass streams [anchor dims ; retained dims] in any case)
+    p.kc_total = d_in / kChunk;
   }
 
   // the V pass splits every sequence into token ranges; the softmax works range by range as well
@@ -1055,7 +1071,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
                                                  a.n_q_heads, g, r.m, r.D, d_in);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  // 6. sink and recent-window tokens (Section 5.1): attended at full precision by the side kernel, then
+  // 6. sink and recent-window tokens (Section 4.1): attended at full precision by the side kernel, then
   //    combined with the result over the predicted tokens
   if (r.n_sink > 0 || r.n_window > 0) {
     SideArgs side;

@@ -48,6 +48,8 @@ struct AbsorbArgs {
   const void* bk = nullptr;     // K bias or null; read only when the keys are rotated (a.rope set): it cancels otherwise
   int D, m;
   int capacity_tokens;
+  bool save_k = false;          // the layer keeps its keys whole (k_local: pool of width D): no K predictor, every head's
+                                // scores come from its stored keys; only the V side is predicted
   int n_sink = 0, n_window = 0; // sink / recent-window tokens kept at full precision (0, 0 = none) ...
   void* k_side = nullptr; void* v_side = nullptr;            // ... their dropped dims (side buffers of the layer)
   const void* k_local = nullptr; const void* v_local = nullptr;   // ... and the layer's pools (retained dims); also

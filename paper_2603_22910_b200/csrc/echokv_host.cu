@@ -20,6 +20,8 @@ inline uint64_t align_up(uint64_t v) { return (v + kAlign - 1) / kAlign * kAlign
 
 struct Derived {
   int D, m, d_in, d_drop, g, elem, part_tokens, capacity, max_parts;
+  int mk;              // K dims a compressed layer stores: m, or D in the "save K" setting
+  bool save_k;
   bool head_aligned;   // m ends on a head boundary (the explicit kernels need it; the absorbed mode does not)
   uint64_t off_status, off_ml, off_o, off_q, off_k, off_v, off_out, off_lens, off_pos, total;
 };
@@ -49,6 +51,8 @@ int derive(const echokv_config* c, Derived* d) {
     d->m = c->n_retained_dims;
   }
   d->head_aligned = d->m % c->head_dim == 0;
+  d->save_k = c->save_k != 0 && d->m < d->D;
+  d->mk = d->save_k ? d->D : d->m;
   d->d_in = d->D + d->m;
   d->d_drop = d->D - d->m;
   d->elem = c->dtype == ECHOKV_BF16 ? 2 : 4;
@@ -303,10 +307,10 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
   if (reinterpret_cast<uintptr_t>(buf->workspace) % kAlign != 0) return ECHOKV_EINVAL;
   for (int l = 0; l < cfg->n_layers; ++l) {
     const bool anchor = l % cfg->group_size == 0;
-    const bool needs_pool = anchor || d.m > 0;
-    if (needs_pool && (!buf->k_pools[l] || !buf->v_pools[l])) return ECHOKV_EINVAL;
-    if (needs_pool && (reinterpret_cast<uintptr_t>(buf->k_pools[l]) % 16 != 0 ||
-                       reinterpret_cast<uintptr_t>(buf->v_pools[l]) % 16 != 0))
+    const bool needs_k = anchor || d.mk > 0, needs_v = anchor || d.m > 0;
+    if ((needs_k && !buf->k_pools[l]) || (needs_v && !buf->v_pools[l])) return ECHOKV_EINVAL;
+    if ((needs_k && reinterpret_cast<uintptr_t>(buf->k_pools[l]) % 16 != 0) ||
+        (needs_v && reinterpret_cast<uintptr_t>(buf->v_pools[l]) % 16 != 0))
       return ECHOKV_EINVAL;
   }
   echokv_ctx* c = new (std::nothrow) echokv_ctx();
@@ -331,8 +335,8 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
   if (cudaMemset(c->ws + d.off_status, 0, kAlign) != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
   c->tc_capable = tc_shape_supported(cfg->dtype, cfg->head_dim, cfg->page_tokens, d.D, d.m);
   if (!any_compressed || d.d_drop == 0) c->path = 0;
-  else if (!d.head_aligned) {
-    // a partly retained head: served by the absorbed mode only
+  else if (!d.head_aligned || d.save_k) {
+    // a partly retained head, or keys kept whole: served by the absorbed mode only
     if (!absorbed_supported(cfg->dtype, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, d.m, cfg->page_tokens)) {
       delete c;
       return ECHOKV_EUNSUPPORTED;
@@ -351,9 +355,9 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
     // tensor maps of every pool (the predictors' maps follow in echokv_set_weights)
     for (int l = 0; l < cfg->n_layers; ++l) {
       Layer& L = c->layers[l];
-      const int width = L.anchor ? d.D : d.m;
-      if (width == 0) continue;
-      const cudaError_t e = tc_encode_pool_maps(&L.tc, L.k_pool, L.v_pool, width,
+      const int k_width = L.anchor ? d.D : d.mk, v_width = L.anchor ? d.D : d.m;
+      if (k_width == 0 && v_width == 0) continue;
+      const cudaError_t e = tc_encode_pool_maps(&L.tc, L.k_pool, k_width, L.v_pool, v_width,
                                                 (uint64_t)cfg->n_pages * cfg->page_tokens,
                                                 cfg->page_tokens);
       if (e != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
@@ -365,7 +369,7 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
     for (int l = 0; l < cfg->n_layers; ++l) {
       Layer& L = c->layers[l];
       const int width = L.anchor ? d.D : d.m;
-      if (width == 0) continue;
+      if (width == 0 || (!L.anchor && d.save_k)) continue;   // (keys kept whole: no stored-head call on that layer)
       const uint64_t rows = (uint64_t)cfg->n_pages * cfg->page_tokens;
       if (encode_pool_box_map(&L.stored_k, L.k_pool, width, rows, box_rows) != cudaSuccess ||
           encode_pool_box_map(&L.stored_v, L.v_pool, width, rows, box_rows) != cudaSuccess ||
@@ -388,7 +392,7 @@ int echokv_set_weights(echokv_ctx* c, int layer, const void* Wk, const void* Wv,
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return ECHOKV_EINVAL;
   Layer& L = c->layers[layer];
   if (L.anchor) return ECHOKV_ENOTCOMPRESSED;
-  if (c->d.d_drop > 0 && (!Wk || !Wv)) return ECHOKV_EINVAL;
+  if (c->d.d_drop > 0 && (!Wv || (!Wk && !c->d.save_k))) return ECHOKV_EINVAL;   // (keys kept whole: no K predictor)
   if ((reinterpret_cast<uintptr_t>(Wk) | reinterpret_cast<uintptr_t>(Wv)) % 16 != 0) return ECHOKV_EINVAL;
   L.Wk = Wk; L.Wv = Wv; L.bk = bk; L.bv = bv;
   if (c->tc_capable && c->d.d_drop > 0) {
@@ -429,7 +433,8 @@ int echokv_set_full_precision_window(echokv_ctx* c, int n_sink, int n_window, vo
                                      void* const* v_side) {
   if (!c || n_sink < 0 || n_window < 0) return ECHOKV_EINVAL;
   if (n_sink + n_window > 4096) return ECHOKV_EUNSUPPORTED;
-  if (!c->d.head_aligned && (n_sink > 0 || n_window > 0)) return ECHOKV_EUNSUPPORTED;   // (side buffers are per head)
+  if ((!c->d.head_aligned || c->d.save_k) && (n_sink > 0 || n_window > 0))
+    return ECHOKV_EUNSUPPORTED;   // (side buffers are per head, and hold K and V alike)
   const bool on = (n_sink > 0 || n_window > 0) && c->d.d_drop > 0;
   if (on) {
     if (!k_side || !v_side) return ECHOKV_EINVAL;
@@ -467,8 +472,8 @@ int echokv_set_rope(echokv_ctx* c, double theta, void* table, uint64_t table_byt
   }
   if (!std::isfinite(theta) || theta < 1.0) return ECHOKV_EINVAL;
   // a rotation that depends on the token cannot be folded into the queries: the K side stays explicit, which
-  // needs whole heads
-  if (!c->d.head_aligned) return ECHOKV_EUNSUPPORTED;
+  // needs whole heads (unless the keys are kept whole anyway)
+  if (!c->d.head_aligned && !c->d.save_k) return ECHOKV_EUNSUPPORTED;
   uint64_t need = 0;
   const int rc = echokv_rope_table_bytes(&c->cfg, &need);
   if (rc != ECHOKV_OK) return rc;
@@ -540,10 +545,10 @@ int echokv_append_kv(echokv_ctx* c, int layer, const void* k_new, const void* v_
   if (B > c->cfg.max_batch) return ECHOKV_ECAPACITY;
   if (!c->table) return ECHOKV_ENOTABLE;
   const Layer& L = c->layers[layer];
-  const int width = L.anchor ? c->d.D : c->d.m;
-  if (width == 0)                     // nothing of this layer is kept in the pools (m = 0)
+  const int k_width = L.anchor ? c->d.D : c->d.mk, v_width = L.anchor ? c->d.D : c->d.m;
+  if (k_width == 0 && v_width == 0)   // nothing of this layer is kept in the pools (m = 0)
     return append_side(c, L, k_new, v_new, dev_seq_slots, dev_positions, B, static_cast<cudaStream_t>(stream));
-  const cudaError_t e = launch_append(c->cfg.dtype, L.k_pool, L.v_pool, width, c->d.D, k_new, v_new,
+  const cudaError_t e = launch_append(c->cfg.dtype, L.k_pool, L.v_pool, k_width, v_width, c->d.D, k_new, v_new,
                                       dev_seq_slots, dev_positions, B, geom_of(c), status_ptr(c),
                                       static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return ECHOKV_ECUDA;
@@ -561,6 +566,7 @@ int echokv_compress_layer(echokv_ctx* c, int layer, const void* k_full, const vo
   if (!c->table) return ECHOKV_ENOTABLE;
   const Layer& L = c->layers[layer];
   if (L.anchor) return ECHOKV_ENOTCOMPRESSED;
+  if (c->d.save_k) return ECHOKV_EUNSUPPORTED;
   const bool side = side_active(c, L);
   if (c->d.m == 0 && !side) return ECHOKV_OK;          // nothing of this layer is kept
   const SideArgs sa = side_args(c, L);
@@ -592,7 +598,7 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (L.anchor || c->d.d_drop == 0)
     return attend_stored_layer(c, L, q, out, dev_seq_slots, dev_seq_lens, B, s);
-  if (!L.Wk || !L.Wv) return ECHOKV_ENOWEIGHTS;
+  if (!L.Wv || (!L.Wk && !c->d.save_k)) return ECHOKV_ENOWEIGHTS;
   const Layer& A = c->layers[layer - layer % c->cfg.group_size];
   AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
   const bool side = side_active(c, L);
@@ -605,6 +611,7 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     aa.Wk = L.Wk; aa.Wv = L.Wv; aa.bv = L.bv;
     aa.bk = c->rope.cs != nullptr ? L.bk : nullptr;
     aa.k_local = L.k_pool; aa.v_local = L.v_pool;
+    aa.save_k = c->d.save_k;
     aa.D = c->d.D; aa.m = c->d.m;
     aa.capacity_tokens = c->d.capacity;
     aa.kernel_ms = nullptr;
@@ -612,16 +619,18 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
       aa.n_sink = c->n_sink; aa.n_window = c->n_window;
       aa.k_side = L.k_side; aa.v_side = L.v_side;
       aa.k_local = L.k_pool; aa.v_local = L.v_pool;
+    aa.save_k = c->d.save_k;
     }
     cudaEvent_t ev[4];
     const bool timed = timed_pair(c, ECHOKV_TIMED_ABSORB_K, &ev[0], &ev[1]) &&
                        timed_pair(c, ECHOKV_TIMED_ABSORB_V, &ev[2], &ev[3]);
     if (launch_absorbed(a, aa, c->amaps, A.tc, L.tc, out, c->sm_count, s, timed ? ev : nullptr) != cudaSuccess)
       return ECHOKV_ECUDA;
-    c->launches += (c->rope.cs != nullptr ? 5 + (c->d.m > 0 ? 1 : 0) : 6) + (side ? 2 : 0);
+    c->launches += (c->rope.cs != nullptr ? (c->d.save_k ? 5 : 5 + (c->d.m > 0 ? 1 : 0)) : 6) + (side ? 2 : 0);
     return ECHOKV_OK;
   }
-  if (!c->d.head_aligned) return ECHOKV_EUNSUPPORTED;   // explicit reconstruction needs whole heads: use the absorbed mode
+  if (!c->d.head_aligned || c->d.save_k)
+    return ECHOKV_EUNSUPPORTED;   // explicit reconstruction needs whole heads and predicts K as well: use the absorbed mode
   const int r = c->d.m / c->cfg.head_dim;
   // retained heads: Eq. 7 on what is stored (Eq. 6 keeps them as they are)
   const int n_splits = stored_splits(c, B, r);

@@ -26,8 +26,8 @@ size_t rope_table_pairs(int stride, int head_dim);
 RopeTable rope_table_view(const float2* buffer, int stride, int head_dim);
 cudaError_t launch_rope_table(float2* buffer, int stride, int head_dim, double theta, cudaStream_t stream);
 
-// Append one token per sequence: writes the first `width` flat dims of k_new / v_new.
-cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int width, int D, const void* k_new,
+// Append one token per sequence: writes the first k_width flat dims of k_new and the first v_width of v_new.
+cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int k_width, int v_width, int D, const void* k_new,
                           const void* v_new, const int32_t* slots, const int32_t* positions, int B,
                           const PageGeom& geom, int32_t* status, cudaStream_t stream);
 
@@ -56,7 +56,7 @@ struct ReconArgs {
                                                 // attended from the side buffers, see launch_attn_side)
 };
 
-// Tokens of a sequence of `len` tokens that are predicted: [lo, hi) (Section 5.1: sink and recent-window
+// Tokens of a sequence of `len` tokens that are predicted: [lo, hi) (Section 4.1: sink and recent-window
 // tokens keep all their dims).
 __host__ __device__ inline int predicted_lo(int len, int n_sink) { return n_sink < len ? n_sink : len; }
 __host__ __device__ inline int predicted_hi(int len, int n_sink, int n_window) {

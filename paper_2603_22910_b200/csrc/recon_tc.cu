@@ -598,43 +598,47 @@ cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, u
   return encode_2d(map, pool, rows, width, box_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
-cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const void* v_pool, int width,
+cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, int k_width, const void* v_pool, int v_width,
                                 uint64_t rows, int page_tokens) {
-  cudaError_t e = encode_2d(&maps->k_pool, k_pool, rows, width, page_tokens, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-  if (e != cudaSuccess) return e;
-  e = encode_2d(&maps->v_pool, v_pool, rows, width, page_tokens, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-  if (e != cudaSuccess) return e;
-  // boxes of 64 token rows: runs of consecutive pages, or part of a page that is taller
-  const int run_rows = kRunTokens;
-  e = encode_2d(&maps->k_pool_run, k_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-  if (e != cudaSuccess) return e;
-  e = encode_2d(&maps->v_pool_run, v_pool, rows, width, run_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-  if (e != cudaSuccess) return e;
-  // CTA-pair kernel: 128 consecutive token rows x two 64-feature chunks in one copy
-  if (width >= 128) {     // (a pool one chunk wide is never read two chunks at a time)
-    e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-    if (e != cudaSuccess) return e;
-    e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, width, 128, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-    if (e != cudaSuccess) return e;
-  } else {
-    maps->k_pool_run128 = maps->k_pool_run;
-    maps->v_pool_run128 = maps->v_pool_run;
+  cudaError_t e;
+  const CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
+  if (k_width > 0) {
+    if ((e = encode_2d(&maps->k_pool, k_pool, rows, k_width, page_tokens, promo)) != cudaSuccess) return e;
+    // boxes of 64 token rows: runs of consecutive pages, or part of a page that is taller
+    if ((e = encode_2d(&maps->k_pool_run, k_pool, rows, k_width, kRunTokens, promo)) != cudaSuccess) return e;
+    // CTA-pair kernel: 128 consecutive token rows x two 64-feature chunks in one copy
+    if (k_width >= 128) {     // (a pool one chunk wide is never read two chunks at a time)
+      if ((e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, k_width, 128, 2, promo)) != cudaSuccess) return e;
+    } else {
+      maps->k_pool_run128 = maps->k_pool_run;
+    }
   }
-  // absorbed mode, V side: 64 consecutive token rows x four 64-feature chunks in one copy
-  if (width >= 256) {
-    e = encode_3d_chunks(&maps->v_pool_tok64x4, v_pool, rows, width, 64, 4, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-    if (e != cudaSuccess) return e;
+  if (v_width > 0) {
+    if ((e = encode_2d(&maps->v_pool, v_pool, rows, v_width, page_tokens, promo)) != cudaSuccess) return e;
+    if ((e = encode_2d(&maps->v_pool_run, v_pool, rows, v_width, kRunTokens, promo)) != cudaSuccess) return e;
+    if (v_width >= 128) {
+      if ((e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, v_width, 128, 2, promo)) != cudaSuccess) return e;
+    } else {
+      maps->v_pool_run128 = maps->v_pool_run;
+    }
+    // absorbed mode, V side: 64 consecutive token rows x four 64-feature chunks in one copy
+    if (v_width >= 256) {
+      if ((e = encode_3d_chunks(&maps->v_pool_tok64x4, v_pool, rows, v_width, 64, 4, promo)) != cudaSuccess) return e;
+    }
   }
   maps->pools_ready = true;
   return cudaSuccess;
 }
 
 cudaError_t tc_encode_weight_maps(TcLayerMaps* maps, const void* Wk, const void* Wv, int d_drop, int d_in) {
-  cudaError_t e = encode_2d(&maps->wk, Wk, d_drop, d_in, kWRows, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
+  if (Wk != nullptr) {      // (no K predictor where the keys are kept whole)
+    e = encode_2d(&maps->wk, Wk, d_drop, d_in, kWRows, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+    if (e != cudaSuccess) return e;
+    e = encode_3d_chunks(&maps->wk_half, Wk, d_drop, d_in, kWRows / 2, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+    if (e != cudaSuccess) return e;
+  }
   e = encode_2d(&maps->wv, Wv, d_drop, d_in, kWRows, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
-  if (e != cudaSuccess) return e;
-  e = encode_3d_chunks(&maps->wk_half, Wk, d_drop, d_in, kWRows / 2, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
   if (e != cudaSuccess) return e;
   e = encode_3d_chunks(&maps->wv_half, Wv, d_drop, d_in, kWRows / 2, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
   if (e != cudaSuccess) return e;

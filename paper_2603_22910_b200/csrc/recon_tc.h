@@ -31,7 +31,8 @@ cudaError_t encode_chunked_3d_map(CUtensorMap* map, const void* base, uint64_t r
 
 bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m);
 
-cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, const void* v_pool, int width,
+// k_width / v_width: row widths of the two pools (they differ where a layer keeps its keys whole); 0 = no pool
+cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, int k_width, const void* v_pool, int v_width,
                                 uint64_t rows, int page_tokens);
 
 cudaError_t tc_encode_weight_maps(TcLayerMaps* maps, const void* Wk, const void* Wv, int d_drop,

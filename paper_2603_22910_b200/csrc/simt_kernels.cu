@@ -61,7 +61,7 @@ cudaError_t launch_rope_table(float2* buffer, int stride, int head_dim, double t
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(128) append_kernel(T* __restrict__ k_pool, T* __restrict__ v_pool,
-                                                     int width, int D, const T* __restrict__ k_new,
+                                                     int k_width, int v_width, int D, const T* __restrict__ k_new,
                                                      const T* __restrict__ v_new,
                                                      const int32_t* __restrict__ slots,
                                                      const int32_t* __restrict__ positions,
@@ -78,28 +78,25 @@ __global__ void __launch_bounds__(128) append_kernel(T* __restrict__ k_pool, T* 
     if (threadIdx.x == 0) report(status, ECHOKV_EBADPAGE);
     return;
   }
-  const size_t row = ((size_t)page * g.page_tokens + pos % g.page_tokens) * (size_t)width;
+  const size_t row = (size_t)page * g.page_tokens + pos % g.page_tokens;
   constexpr int kVec = 16 / sizeof(T);
-  const int n_vec = width / kVec;
   const uint4* ks = reinterpret_cast<const uint4*>(k_new + (size_t)b * D);
   const uint4* vs = reinterpret_cast<const uint4*>(v_new + (size_t)b * D);
-  uint4* kd = reinterpret_cast<uint4*>(k_pool + row);
-  uint4* vd = reinterpret_cast<uint4*>(v_pool + row);
-  for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
-    kd[i] = ks[i];
-    vd[i] = vs[i];
-  }
+  uint4* kd = reinterpret_cast<uint4*>(k_pool + row * (size_t)k_width);
+  uint4* vd = reinterpret_cast<uint4*>(v_pool + row * (size_t)v_width);
+  for (int i = threadIdx.x; i < k_width / kVec; i += blockDim.x) kd[i] = ks[i];
+  for (int i = threadIdx.x; i < v_width / kVec; i += blockDim.x) vd[i] = vs[i];
 }
 
-cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int width, int D, const void* k_new,
+cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int k_width, int v_width, int D, const void* k_new,
                           const void* v_new, const int32_t* slots, const int32_t* positions, int B,
                           const PageGeom& geom, int32_t* status, cudaStream_t stream) {
   if (dtype == ECHOKV_BF16) {
     append_kernel<__nv_bfloat16><<<B, 128, 0, stream>>>(
-        (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, width, D, (const __nv_bfloat16*)k_new,
+        (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, k_width, v_width, D, (const __nv_bfloat16*)k_new,
         (const __nv_bfloat16*)v_new, slots, positions, geom, status);
   } else {
-    append_kernel<float><<<B, 128, 0, stream>>>((float*)k_pool, (float*)v_pool, width, D,
+    append_kernel<float><<<B, 128, 0, stream>>>((float*)k_pool, (float*)v_pool, k_width, v_width, D,
                                                 (const float*)k_new, (const float*)v_new, slots,
                                                 positions, geom, status);
   }
@@ -844,7 +841,7 @@ cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Sink and recent-window tokens at full precision (Section 5.1): their dropped dims live in small
+// Sink and recent-window tokens at full precision (Section 4.1): their dropped dims live in small
 // side buffers; these two kernels write and attend them.
 // ---------------------------------------------------------------------------------------------
 template <typename T>

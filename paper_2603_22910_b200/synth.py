@@ -45,6 +45,7 @@ class Workload:
     random_pages: bool = False
     seed: int = 1000
     n_retained_dims: int = 0   # if non-zero: m itself, in flat dims (need not end on a head boundary)
+    save_k: bool = False       # compressed layers keep their keys whole; only the values are evicted and predicted
 
     @property
     def D(self) -> int:
@@ -53,6 +54,11 @@ class Workload:
     @property
     def m(self) -> int:
         return self.n_retained_dims if self.n_retained_dims else self.n_retained_heads * self.head_dim
+
+    @property
+    def mk(self) -> int:
+        """K dims a compressed layer stores."""
+        return self.D if (self.save_k and self.m < self.D) else self.m
 
     @property
     def d_in(self) -> int:

@@ -17,7 +17,7 @@ class Case:
 
     def __init__(self, w: synth.Workload, lens=None, n_pages=None, layers=None, keep_host=True,
                  biases=False, window=None, rope=None):
-        """window = (n_sink, n_window): those tokens of every sequence keep all their dims (Section 5.1).
+        """window = (n_sink, n_window): those tokens of every sequence keep all their dims (Section 4.1).
         rope = theta: the cache holds un-rotated keys that are rotated to their positions when read."""
         self.w = w
         self.lens = list(lens) if lens is not None else [w.context] * w.batch
@@ -41,8 +41,9 @@ class Case:
         dev = self.ctx.device
         needed = set(self.layers) | {w.anchor_of(l) for l in self.layers}
         for l in sorted(needed):
-            width = w.D if w.is_anchor(l) else w.m
             for kind in ("k", "v"):
+                # a compressed layer stores m dims of K and V -- or all of K in the "save K" setting
+                width = w.D if w.is_anchor(l) else (w.mk if kind == "k" else w.m)
                 side_only = width == 0 and bool(window) and not w.is_anchor(l)
                 if width == 0 and not side_only:
                     continue
@@ -86,14 +87,18 @@ class Case:
                     bv = (synth.normal((w.d_drop,), w.seed, 91, l) * 0.1).to(synth.torch_dtype(w))
                 self.host_w[l] = (Wk, Wv, bk, bv)
                 devw = tuple(None if t is None else t.to(dev) for t in (Wk, Wv, bk, bv))
+                if w.save_k:
+                    devw = (None, devw[1], None, devw[3])     # keys kept whole: the library takes no K predictor
                 self.weights[l] = devw
                 self.ctx.set_weights(l, *devw)
         self.seq_lens = torch.tensor(self.lens, dtype=torch.int32, device=dev)
         self.positions = self.seq_lens - 1
         for l in sorted(needed):
             if (l, "k", "new") in self.host:
-                self.ctx.append_kv(l, self.host[(l, "k", "new")].to(dev), self.host[(l, "v", "new")].to(dev),
-                                   self.positions)
+                v_new = self.host.get((l, "v", "new"))
+                if v_new is None:        # nothing of V is stored on this layer: whatever is passed must be ignored
+                    v_new = torch.full((w.batch, w.D), 777.0, dtype=synth.torch_dtype(w))
+                self.ctx.append_kv(l, self.host[(l, "k", "new")].to(dev), v_new.to(dev), self.positions)
         self.q = {l: synth.queries(w, l) for l in self.layers}
 
     def run(self, layer, full=False):
@@ -125,7 +130,8 @@ class Case:
             a = w.anchor_of(layer)
             kg, vg = self._stored(a, "k", b), self._stored(a, "v", b)
             L = kg.shape[0]
-            kl = self._stored(layer, "k", b) if w.m else np.zeros((L, 0))
+            k_true = self._stored(layer, "k", b) if w.save_k else None      # keys kept whole
+            kl = (k_true[:, :w.m] if w.save_k else self._stored(layer, "k", b)) if w.m else np.zeros((L, 0))
             vl = self._stored(layer, "v", b) if w.m else np.zeros((L, 0))
             Wk, Wv, bk, bv = (None if t is None else O.widen(synth.to_numpy_stored(t))
                               for t in self.host_w[layer])
@@ -138,7 +144,7 @@ class Case:
                                                      rope_theta=self.rope)
             elif query_heads is None:
                 res[b] = O.decode_attention(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv,
-                                            rope_theta=self.rope)
+                                            rope_theta=self.rope, k_true=k_true)
             else:
                 per = O.decode_attention_query_heads(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, query_heads,
                                                      rope_theta=self.rope)

@@ -1,4 +1,4 @@
-"""GPU parity with sink and recent-window tokens kept at full precision (Section 5.1 of the paper:
+"""GPU parity with sink and recent-window tokens kept at full precision (Section 4.1 of the paper:
 4 sink tokens and a local window of 128 tokens): those tokens' dropped dims come from the side buffers,
 every other token is predicted."""
 import ctypes as C

@@ -85,6 +85,37 @@ def test_eviction_eq2_eq4_matches_the_printed_shapes():
         O.retained_dims(np.zeros((2, 8)), 9)
 
 
+def test_save_k_setting_uses_the_true_keys():
+    # "save K" (Section 5.2): keys whole, values predicted.  Pins: with a selector W^V it is standard attention on
+    # the true cache (library routine); with a selector W^K the ordinary path gives the same as handing over the
+    # true keys; the K predictor and the retained key dims are not read at all
+    c = rand_case(41, L=19, H_q=8, H_kv=4, d=8, r=1)
+    g = rng(41)
+    D, m, L = c["D"], c["m"], c["L"]
+    k_true = np.concatenate([c["kl"], g.standard_normal((L, D - m))], axis=1)
+    v_true_drop = g.standard_normal((L, D - m))
+    # the anchor's V carries this layer's dropped V dims, and W^V selects them
+    vg = c["vg"].copy()
+    vg[:, m:] = v_true_drop
+    Wv_sel = np.zeros((D - m, D + m))
+    Wv_sel[np.arange(D - m), m + np.arange(D - m)] = 1.0
+    got = O.decode_attention(c["q"], c["kg"], vg, c["kl"], c["vl"], None, Wv_sel, c["H_kv"], k_true=k_true)
+    V_true = np.concatenate([c["vl"], v_true_drop], axis=1).reshape(L, c["H_kv"], c["d"])
+    np.testing.assert_allclose(got, sdpa(c["q"], k_true.reshape(L, c["H_kv"], c["d"]), V_true), rtol=1e-12, atol=1e-13)
+    # selector W^K on an anchor that carries the true dropped key dims: the ordinary path equals the save-K path
+    kg = c["kg"].copy()
+    kg[:, m:] = k_true[:, m:]
+    ordinary = O.decode_attention(c["q"], kg, c["vg"], c["kl"], c["vl"], Wv_sel, c["Wv"], c["H_kv"])
+    saved = O.decode_attention(c["q"], kg, c["vg"], np.full_like(c["kl"], np.nan), c["vl"], None, c["Wv"], c["H_kv"],
+                               k_true=k_true)
+    np.testing.assert_allclose(saved, ordinary, rtol=1e-12, atol=1e-13)
+    # and it differs from predicting the keys with a random predictor
+    assert np.abs(run(c) - O.decode_attention(c["q"], c["kg"], c["vg"], c["kl"], c["vl"], None, c["Wv"], c["H_kv"],
+                                              k_true=k_true)).max() > 1e-3
+    with pytest.raises(ValueError):
+        O.decode_attention(c["q"], c["kg"], c["vg"], c["kl"], c["vl"], None, c["Wv"], c["H_kv"], k_true=k_true[:-1])
+
+
 def test_anchor_assignment_eq1():
     S = 4
     assert [O.is_anchor_layer(l, S) for l in range(9)] == [True, False, False, False, True, False, False, False, True]
@@ -433,7 +464,7 @@ def test_planted_mistakes_are_caught(monkeypatch):
 
 
 # --------------------------------------------------------------------------
-# Sink and recent-window tokens at full precision (Section 5.1)
+# Sink and recent-window tokens at full precision (Section 4.1)
 # --------------------------------------------------------------------------
 def true_dropped(c, seed):
     """A layer's own dims m..D-1 (what the predictor stands in for), unrelated to W on purpose."""
