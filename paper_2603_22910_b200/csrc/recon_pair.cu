@@ -19,8 +19,11 @@
 //   result     : one split-K partial per 128 tokens and query head.
 //
 // acc0 and acc1 are separate halves of tensor memory, so the K epilogue runs under the V-phase
-// MMAs and the V epilogue under the next item's K-phase MMAs.  Warp roles per CTA: warp 0 TMA,
-// warp 1 MMA issue (only in the pair's first CTA) and tensor-memory allocation, warps 2..9 epilogue.
+// MMAs and the V epilogue under the next item's K-phase MMAs.  Warp roles per CTA: warps 0 and 10 TMA
+// (alternate stages: with 16-token pages in no particular order a stage is up to 17 copies per CTA, and one
+// warp does not issue them as fast as the tensor cores consume a stage; measured 6 % on such pools, nothing
+// on consecutive pages), warp 1 MMA issue (only in the pair's first CTA) and tensor-memory allocation,
+// warps 2..9 epilogue.
 // Every wait is bounded; when one runs out the kernel raises the status word and winds down.
 #include "recon_tc.h"
 
@@ -43,7 +46,7 @@ constexpr int kWRows = 128;                          // predictor rows per CTA: 
 constexpr int kWBytes = kWRows * kRowBytes;          // 16 KiB: predictor rows of one chunk
 constexpr int kStageXBytes = kStageChunks * kXBytes;  // token rows: chunk 0, chunk 1
 constexpr int kStageBytes = kStageChunks * (kXBytes + kWBytes);   // then predictor rows: chunk 0, chunk 1
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;                        // warps 0 and 10: TMA, 1: MMA, 2..9: epilogue
 constexpr int kEpilogueThreads = 256;
 constexpr int kMaxBatchPerLaunch = 256;
 constexpr int kRunTokens = 64;                       // token rows of a tall box over consecutive pages
@@ -216,8 +219,9 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
   const int n_steps = p.kc_total / kStageChunks;            // stages per phase (kc_total is even)
   bool gave_up = false;
 
-  if (warp == 0) {
-    // =============================== TMA producer ===============================================
+  if (warp == 0 || warp == 10) {
+    // =============================== TMA producers (alternate stages) ============================
+    const uint32_t mine = warp == 0 ? 0u : 1u;
     uint32_t it = 0;
     bool alive = true;
     for (int item = pair_id; item < n_items && alive; item += n_clusters) {
@@ -264,6 +268,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
         const CUtensorMap* m_local_128 = phase == 0 ? &tm_local_k_128 : &tm_local_v_128;
         const CUtensorMap* m_w = phase == 0 ? &tm_wk : &tm_wv;
         for (int step = 0; step < n_steps; ++step, ++it) {
+          if ((it & 1u) != mine) continue;
           const uint32_t s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           // both CTAs' copies of a stage complete on the first CTA's barrier, where the MMAs are issued
