@@ -40,7 +40,7 @@ UNIT = "tokens/s"
 # the ncu captures summarised under profiles/; None until a capture of that workload exists.
 NCU_TRAFFIC_BYTES = {
     "c1": 4 * 619.0e6,        # recon_tc_kernel: B = 2 capture x 4 (tokens)
-    "c2": 8 * 348.1e6,        # recon_pair_kernel: B = 2 capture x 8
+    "c2": 8 * 348.2e6,        # recon_pair_kernel: B = 2 capture x 8
     "c1_full": 4 * 272.9e6,   # attn_stored_mma_kernel: B = 2 capture x 4
     "c2_full": 8 * 274.5e6,   # attn_stored_mma_kernel: B = 2 capture x 8
     "c1_absorbed": 4 * 418.8e6,   # absorb_scores_kernel + absorb_pv_kernel (one launch each): B = 2 capture x 4
