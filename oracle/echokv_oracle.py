@@ -368,6 +368,41 @@ def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n
 
 
 # ----------------------------------------------------------------------------
+# Prefill-shaped use: the last n_q tokens of a sequence are queries at once (Section 5.4: the
+# dropped parts of the cache can be evicted already during the pre-filling phase)
+# ----------------------------------------------------------------------------
+
+
+def prefill_attention(q: np.ndarray, k_global, v_global, k_local, v_local, Wk, Wv, n_kv_heads: int,
+                      scale: float | None = None, bk=None, bv=None, rope_theta: float | None = None) -> np.ndarray:
+    """q [n_q, H_q, d]: queries of the last n_q of the L cached tokens; query i sits at position
+    L - n_q + i and attends the tokens up to and including its own (causal).  The cache of a
+    compressed layer is rebuilt once (Eq. 3, Eq. 6) and each query evaluates Eq. 7 over its prefix.
+    With Wk = Wv = None the layer holds its full cache (k_global, v_global are used as they are:
+    an anchor layer).  Returns [n_q, H_q, d]."""
+    q = np.asarray(q, dtype=np.float64)
+    n_q, H_q, d = q.shape
+    k_global = np.asarray(k_global, dtype=np.float64)
+    v_global = np.asarray(v_global, dtype=np.float64)
+    L = k_global.shape[0]
+    if n_q < 1 or n_q > L:
+        raise ValueError("need 1 <= n_q <= L")
+    if Wk is None and Wv is None:
+        K_t = k_global.reshape(L, n_kv_heads, d)
+        V_t = v_global.reshape(L, n_kv_heads, d)
+    else:
+        K_t = assemble_cache(k_local, reconstruct_dropped(Wk, k_global, k_local, bk), n_kv_heads, d)
+        V_t = assemble_cache(v_local, reconstruct_dropped(Wv, v_global, v_local, bv), n_kv_heads, d)
+    if rope_theta is not None:
+        K_t = rotate_keys(K_t, rope_theta)
+    out = np.empty((n_q, H_q, d), dtype=np.float64)
+    for i in range(n_q):
+        n_seen = L - n_q + i + 1
+        out[i] = attention(q[i], K_t[:n_seen], V_t[:n_seen], scale)
+    return out
+
+
+# ----------------------------------------------------------------------------
 # Multi-layer step (Eq. 1): which cache each layer attends over
 # ----------------------------------------------------------------------------
 

@@ -116,6 +116,42 @@ def test_save_k_setting_uses_the_true_keys():
         O.decode_attention(c["q"], c["kg"], c["vg"], c["kl"], c["vl"], None, c["Wv"], c["H_kv"], k_true=k_true[:-1])
 
 
+def test_prefill_shaped_attention():
+    c = rand_case(51, L=21, H_q=8, H_kv=4, d=8, r=1)
+    g = rng(51)
+    n_q = 6
+    q = g.standard_normal((n_q, c["H_q"], c["d"]))
+    args = (c["kg"], c["vg"], c["kl"], c["vl"], c["Wk"], c["Wv"], c["H_kv"])
+    got = O.prefill_attention(q, *args)
+    # the last query sees the whole cache: the decode step; every other query: the decode step on its prefix
+    np.testing.assert_allclose(got[-1], O.decode_attention(q[-1], *args), rtol=1e-12, atol=1e-14)
+    for i in (0, 3):
+        n = c["L"] - n_q + i + 1
+        want = O.decode_attention(q[i], c["kg"][:n], c["vg"][:n], c["kl"][:n], c["vl"][:n], c["Wk"], c["Wv"], c["H_kv"])
+        np.testing.assert_allclose(got[i], want, rtol=1e-12, atol=1e-14)
+    # causal: what comes after a query's own token does not matter to it
+    kg2, vg2 = c["kg"].copy(), c["vg"].copy()
+    kg2[-2:] = 7.0
+    vg2[-2:] = -3.0
+    got2 = O.prefill_attention(q, kg2, vg2, c["kl"], c["vl"], c["Wk"], c["Wv"], c["H_kv"])
+    np.testing.assert_array_equal(got2[: n_q - 2], got[: n_q - 2])
+    assert np.abs(got2[-1] - got[-1]).max() > 1e-3
+    # a full (anchor) cache with all tokens as queries: causal scaled-dot-product attention (library routine)
+    L, H, d = c["L"], c["H_kv"], c["d"]
+    qa = g.standard_normal((L, c["H_q"], d))
+    full = O.prefill_attention(qa, c["kg"], c["vg"], None, None, None, None, H)
+    tq = torch.from_numpy(qa).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(c["kg"].reshape(L, H, d)).permute(1, 0, 2)[None]
+    tv = torch.from_numpy(c["vg"].reshape(L, H, d)).permute(1, 0, 2)[None]
+    ref = F.scaled_dot_product_attention(tq, tk, tv, is_causal=True, enable_gqa=True)[0].permute(1, 0, 2).numpy()
+    np.testing.assert_allclose(full, ref, rtol=1e-12, atol=1e-13)
+    # rotation: position of key t is t whatever the query
+    rot = O.prefill_attention(q, *args, rope_theta=10000.0)
+    np.testing.assert_allclose(rot[-1], O.decode_attention(q[-1], *args, rope_theta=10000.0), rtol=1e-12, atol=1e-14)
+    with pytest.raises(ValueError):
+        O.prefill_attention(g.standard_normal((c["L"] + 1, c["H_q"], c["d"])), *args)
+
+
 def test_anchor_assignment_eq1():
     S = 4
     assert [O.is_anchor_layer(l, S) for l in range(9)] == [True, False, False, False, True, False, False, False, True]
