@@ -168,6 +168,25 @@ int echokv_decode_attention(echokv_ctx* ctx, int layer, const void* q, float* ou
                             const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
                             void* stream);
 
+/* Prefill-shaped attention: the last n_q cached tokens of every sequence are queries at once (a later chunk of
+ * a prompt whose earlier chunks were already evicted down to the compressed cache: Section 5.4, "drop unnecessary
+ * cache entries during the pre-filling phase").  Query i of sequence b sits at position dev_seq_lens[b] - n_q + i
+ * and attends the tokens up to and including its own (causal); its own K / V must already be in the cache.
+ * q: device pointer [B][n_q][n_q_heads][head_dim]; out: device pointer to fp32 of the same shape.
+ * With many queries the cache is rebuilt once per call rather than once per query: the stored dims are gathered
+ * and the dropped dims predicted (Eq. 3, on the tensor cores; K bias and rotary table applied if set) into
+ * `scratch`, a caller-owned device buffer of echokv_prefill_scratch_bytes() bytes (16-byte aligned) that holds K~
+ * and V~ as bf16 rows [B][max_pages_per_seq * page_tokens][D] each, and a causal attention kernel runs over those
+ * rows.  Unlike the decode calls this one does round the predicted K and V to bf16 (as the paper's own
+ * materialise-then-attend implementation does).  Works on anchor layers too (nothing is predicted there).
+ * bf16, head_dim 128 and head-aligned m only; not with sink / window tokens or save_k: EUNSUPPORTED.
+ * A sequence with fewer than n_q cached tokens, or an unusable slot / length: zeros and the device status.
+ * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (batch, scratch too small), ENOWEIGHTS, ENOTABLE, ECUDA. */
+int echokv_prefill_scratch_bytes(const echokv_config* cfg, uint64_t* out);
+int echokv_prefill_attention(echokv_ctx* ctx, int layer, const void* q, float* out, int n_q,
+                             const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                             void* scratch, uint64_t scratch_bytes, void* stream);
+
 /* Attention over a layer that holds its full cache (anchor layers; the uncompressed
  * short-context mode the paper switches from, Section 5.4): Eq. 7 on the stored K, V.
  * Same arguments as echokv_decode_attention.  Errors: as above plus ENOTANCHOR. */

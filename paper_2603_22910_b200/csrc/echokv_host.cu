@@ -10,6 +10,7 @@
 #include "recon_tc.h"
 #include "stored_mma.h"
 #include "absorbed.h"
+#include "prefill.h"
 
 using namespace echokv;
 
@@ -574,6 +575,63 @@ int echokv_compress_layer(echokv_ctx* c, int layer, const void* k_full, const vo
                       dev_seq_slots, dev_seq_begins, dev_seq_lens, B, geom_of(c), status_ptr(c),
                       static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return ECHOKV_ECUDA;
+  c->launches += 1;
+  return ECHOKV_OK;
+}
+
+int echokv_prefill_scratch_bytes(const echokv_config* cfg, uint64_t* out) {
+  if (!out) return ECHOKV_EINVAL;
+  Derived d;
+  const int rc = derive(cfg, &d);
+  if (rc != ECHOKV_OK) return rc;
+  if (cfg->dtype != ECHOKV_BF16 || cfg->head_dim != 128) return ECHOKV_EUNSUPPORTED;
+  *out = 2ull * (uint64_t)cfg->max_batch * (uint64_t)d.capacity * (uint64_t)d.D * 2ull;
+  return ECHOKV_OK;
+}
+
+int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out, int n_q,
+                             const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                             void* scratch, uint64_t scratch_bytes, void* stream) {
+  const int rc = check_call(c, layer, q, out, dev_seq_lens, B);
+  if (rc != ECHOKV_OK) return rc;
+  if (!scratch || n_q < 1 || reinterpret_cast<uintptr_t>(scratch) % 16 != 0) return ECHOKV_EINVAL;
+  const Layer& L = c->layers[layer];
+  const bool compressed = !L.anchor && c->d.d_drop > 0;
+  if (c->cfg.dtype != ECHOKV_BF16 || c->cfg.head_dim != 128) return ECHOKV_EUNSUPPORTED;
+  if (compressed && (!c->tc_capable || !c->d.head_aligned || c->d.save_k || side_active(c, L))) return ECHOKV_EUNSUPPORTED;
+  if (n_q > c->d.capacity) return ECHOKV_ECAPACITY;
+  const uint64_t rows_bytes = (uint64_t)B * c->d.capacity * c->d.D * 2ull;     // one of K~, V~
+  if (scratch_bytes < 2 * rows_bytes) return ECHOKV_ECAPACITY;
+  if (compressed && (!L.Wk || !L.Wv)) return ECHOKV_ENOWEIGHTS;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
+  __nv_bfloat16* k_rows = static_cast<__nv_bfloat16*>(scratch);
+  __nv_bfloat16* v_rows = k_rows + rows_bytes / 2;
+  const int width = compressed ? c->d.m : c->d.D;
+  // stored dims as they are (keys rotated to their positions), then the predicted ones beside them
+  if (launch_gather_rows(a, L.k_pool, width, k_rows, c->d.capacity, c->d.D, true, s) != cudaSuccess ||
+      launch_gather_rows(a, L.v_pool, width, v_rows, c->d.capacity, c->d.D, false, s) != cudaSuccess)
+    return ECHOKV_ECUDA;
+  c->launches += width > 0 ? 2 : 0;
+  if (compressed) {
+    const Layer& A = c->layers[layer - layer % c->cfg.group_size];
+    ReconArgs ra;
+    ra.k_anchor = A.k_pool; ra.v_anchor = A.v_pool;
+    ra.k_local = L.k_pool; ra.v_local = L.v_pool;
+    ra.Wk = L.Wk; ra.Wv = L.Wv;
+    ra.D = c->d.D; ra.m = c->d.m;
+    ra.part_tokens = c->d.part_tokens;
+    ra.capacity_tokens = c->d.capacity;
+    ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
+    ra.bk = L.bk;
+    if (launch_recon_pair_store(a, ra, A.tc, L.tc, false, k_rows, c->d.capacity, c->d.D, c->sm_count, s) != cudaSuccess)
+      return ECHOKV_ECUDA;
+    ra.bk = L.bv;
+    if (launch_recon_pair_store(a, ra, A.tc, L.tc, true, v_rows, c->d.capacity, c->d.D, c->sm_count, s) != cudaSuccess)
+      return ECHOKV_ECUDA;
+    c->launches += 2;
+  }
+  if (launch_prefill_attn(a, k_rows, v_rows, c->d.capacity, c->d.D, n_q, out, s) != cudaSuccess) return ECHOKV_ECUDA;
   c->launches += 1;
   return ECHOKV_OK;
 }

@@ -1,0 +1,276 @@
+// Prefill-shaped attention: the last n_q tokens of every sequence are queries at once (the paper's
+// Section 5.4 notes that the dropped parts of the cache can be evicted already during the pre-filling
+// phase; later chunks of a prompt then attend a compressed cache with many queries).
+//
+// With many queries per sequence the cache is rebuilt ONCE per call instead of once per query:
+//   1. the stored dims of every cached token are gathered from the paged pool into contiguous rows
+//      (gather_rows_kernel; keys rotated to their positions if a rotary table is set),
+//   2. the dropped dims are predicted on the tensor cores and written beside them (Eq. 3; the
+//      row-storing mode of the CTA-pair kernel),
+//   3. prefill_attn_kernel evaluates Eq. 7 causally over those rows: 64 query rows per CTA, keys and
+//      values in 64-token tiles, S = Q K^T and O += P V as mma.sync m16n8k16, online softmax in fp32.
+// The rebuilt rows are bf16 in a caller-owned scratch, as in the paper's own materialise-then-attend
+// design; the decode path never writes them.
+#include "prefill.h"
+
+#include "ptx_sm100.cuh"
+
+namespace echokv {
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// 1. stored dims of a paged pool -> out[b][t][out_width] at flat dims 0 .. width-1 (whole heads of 128)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* __restrict__ pool, int width,
+                                                          __nv_bfloat16* __restrict__ out, int out_tokens,
+                                                          int out_width, const int32_t* __restrict__ slots,
+                                                          const int32_t* __restrict__ lens, PageGeom g, RopeTable rope,
+                                                          int32_t* status) {
+  const int b = blockIdx.y, t0 = blockIdx.x * 32;
+  const int slot = slots ? slots[b] : b;
+  const int len = lens[b];
+  if (slot < 0 || slot >= g.max_batch || len < 1 || len > g.max_pages_per_seq * g.page_tokens) return;
+  if (t0 >= len) return;
+  const int n_heads = width / 128;
+  // item = (token of the tile, head, 8-dim piece c of the head's first half, with its partner piece 64 dims on)
+  const int n_items = 32 * n_heads * 8;
+  for (int it = threadIdx.x; it < n_items; it += blockDim.x) {
+    const int c = it & 7, hd = (it >> 3) % n_heads, tt = it / (8 * n_heads);
+    const int t = t0 + tt;
+    if (t >= len) continue;
+    const int page = g.table[(size_t)slot * g.max_pages_per_seq + t / g.page_tokens];
+    if (page < 0 || page >= g.n_pages) {
+      report(status, ECHOKV_EBADPAGE);
+      continue;
+    }
+    const __nv_bfloat16* src = pool + ((size_t)page * g.page_tokens + t % g.page_tokens) * (size_t)width + hd * 128 + c * 8;
+    __nv_bfloat16* dst = out + ((size_t)b * out_tokens + t) * (size_t)out_width + hd * 128 + c * 8;
+    uint4 lo = *reinterpret_cast<const uint4*>(src), hi = *reinterpret_cast<const uint4*>(src + 64);
+    if (rope.cs != nullptr) {
+      uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
+      const float2* cs = rope.cs + min(t, rope.stride - 1);
+#pragma unroll
+      for (int e2 = 0; e2 < 4; ++e2) {
+        float r_lo[2], r_hi[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float k_lo = h ? __uint_as_float(lw[e2] & 0xffff0000u) : __uint_as_float(lw[e2] << 16);
+          const float k_hi = h ? __uint_as_float(hw[e2] & 0xffff0000u) : __uint_as_float(hw[e2] << 16);
+          const float2 w = cs[(size_t)(c * 8 + 2 * e2 + h) * rope.stride];
+          r_lo[h] = k_lo * w.x - k_hi * w.y;
+          r_hi[h] = k_hi * w.x + k_lo * w.y;
+        }
+        const __nv_bfloat162 a = __floats2bfloat162_rn(r_lo[0], r_lo[1]), bb = __floats2bfloat162_rn(r_hi[0], r_hi[1]);
+        lw[e2] = *reinterpret_cast<const uint32_t*>(&a);
+        hw[e2] = *reinterpret_cast<const uint32_t*>(&bb);
+      }
+      lo = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+      hi = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+    }
+    *reinterpret_cast<uint4*>(dst) = lo;
+    *reinterpret_cast<uint4*>(dst + 64) = hi;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 3. causal attention of n_q query rows over contiguous bf16 rows
+// ---------------------------------------------------------------------------------------------
+constexpr int kPfRows = 64;      // query rows per CTA: 4 warps x 16
+constexpr int kPfKeys = 64;      // keys per tile
+constexpr int kPfRowBytes = 256; // 128 bf16
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(128) prefill_attn_kernel(const __nv_bfloat16* __restrict__ q,
+                                                           const __nv_bfloat16* __restrict__ ks,
+                                                           const __nv_bfloat16* __restrict__ vs,
+                                                           float* __restrict__ out, int n_q, int n_q_heads,
+                                                           int n_kv_heads, int kv_tokens, int kv_width,
+                                                           const int32_t* __restrict__ slots,
+                                                           const int32_t* __restrict__ lens, int max_batch,
+                                                           int capacity, float scale_log2e, int32_t* status) {
+  __shared__ __align__(128) unsigned char k_tile[kPfKeys * kPfRowBytes];
+  __shared__ __align__(128) unsigned char v_tile[kPfKeys * kPfRowBytes];
+  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qd = (lane & 3) * 2;
+  const int kvh = h / (n_q_heads / n_kv_heads);
+  const int slot = slots ? slots[b] : b;
+  const int len = lens[b];
+  const int i0 = qt * kPfRows + warp * 16 + (lane >> 2), i1 = i0 + 8;      // this thread's two query rows
+  float* out0 = out + (((size_t)b * n_q + i0) * n_q_heads + h) * 128;
+  float* out1 = out + (((size_t)b * n_q + i1) * n_q_heads + h) * 128;
+  if (slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
+    // unusable sequence (or fewer cached tokens than queries): zeros and a status
+    if (tid == 0 && qt == 0 && h == 0) report(status, slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
+    for (int nt = 0; nt < 16; ++nt) {
+      if (i0 < n_q) *reinterpret_cast<float2*>(out0 + nt * 8 + qd) = make_float2(0.f, 0.f);
+      if (i1 < n_q) *reinterpret_cast<float2*>(out1 + nt * 8 + qd) = make_float2(0.f, 0.f);
+    }
+    return;
+  }
+  const int pos0 = len - n_q + i0, pos1 = len - n_q + i1;               // the rows' own positions
+  // A fragments of Q (rows past n_q are zero)
+  uint32_t qa[8][4];
+  {
+    const __nv_bfloat16* q0 = q + (((size_t)b * n_q + i0) * n_q_heads + h) * 128 + qd;
+    const __nv_bfloat16* q1 = q + (((size_t)b * n_q + i1) * n_q_heads + h) * 128 + qd;
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      qa[kk][0] = i0 < n_q ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16) : 0u;
+      qa[kk][1] = i1 < n_q ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16) : 0u;
+      qa[kk][2] = i0 < n_q ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16 + 8) : 0u;
+      qa[kk][3] = i1 < n_q ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16 + 8) : 0u;
+    }
+  }
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  float o[16][4];
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
+
+  // keys this CTA's rows may see: up to the position of its last row
+  const int last_row = min(n_q, (qt + 1) * kPfRows) - 1;
+  const int kv_end = len - n_q + last_row + 1;
+  const uint32_t k_base = smem_u32(k_tile), v_base = smem_u32(v_tile);
+  const __nv_bfloat16* k_seq = ks + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
+  const __nv_bfloat16* v_seq = vs + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
+
+  for (int kv0 = 0; kv0 < kv_end; kv0 += kPfKeys) {
+    // ---- stage 64 key rows and 64 value rows (16-byte pieces swizzled by row so that ldmatrix is conflict-free)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int idx = tid + 128 * i, r = idx >> 4, c = idx & 15;
+      uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
+      if (kv0 + r < kv_end) {
+        kk = *reinterpret_cast<const uint4*>(k_seq + (size_t)(kv0 + r) * kv_width + c * 8);
+        vv = *reinterpret_cast<const uint4*>(v_seq + (size_t)(kv0 + r) * kv_width + c * 8);
+      }
+      const int off = r * kPfRowBytes + ((c ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4*>(k_tile + off) = kk;
+      *reinterpret_cast<uint4*>(v_tile + off) = vv;
+    }
+    __syncthreads();
+
+    // ---- S = Q K^T for this warp's 16 rows x 64 keys
+    float sc[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sc[nt][e] = 0.f;
+#pragma unroll
+    for (int np = 0; np < 4; ++np) {
+      const int tok = np * 16 + (lane >> 4) * 8 + (lane & 7);
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        const int c = 2 * kk + ((lane >> 3) & 1);
+        uint32_t r0, r1, r2, r3;
+        ldsm_x4(k_base + tok * kPfRowBytes + ((c ^ (tok & 7)) << 4), r0, r1, r2, r3);
+        mma_m16n8k16_bf16(sc[2 * np], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], r0, r1);
+        mma_m16n8k16_bf16(sc[2 * np + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], r2, r3);
+      }
+    }
+
+    // ---- causal mask, online softmax (rows i0: elements 0, 1; rows i1: elements 2, 3)
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int key = kv0 + nt * 8 + qd + (e & 1);
+        const int row_pos = e < 2 ? pos0 : pos1;
+        const bool row_ok = e < 2 ? i0 < n_q : i1 < n_q;
+        const float v = (row_ok && key <= row_pos) ? sc[nt][e] * scale_log2e : -INFINITY;
+        sc[nt][e] = v;
+        mx[e >> 1] = fmaxf(mx[e >> 1], v);
+      }
+    float alpha[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+      const float m_new = fmaxf(m_run[r], mx[r]);
+      // (a row that has seen no key yet keeps m = -inf: its probabilities are all 0 and alpha is irrelevant)
+      alpha[r] = m_new == -INFINITY ? 1.f : exp2f(m_run[r] - m_new);
+      m_run[r] = m_new;
+    }
+    uint32_t pa[4][4];
+    float psum[2] = {0.f, 0.f};
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      float pv[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        pv[e] = m_run[e >> 1] == -INFINITY ? 0.f : exp2f(sc[nt][e] - m_run[e >> 1]);
+        psum[e >> 1] += pv[e];
+      }
+      // C fragments of key tiles 2j, 2j + 1 are the A fragment of key step j
+      pa[nt >> 1][(nt & 1) * 2 + 0] = pack2(pv[0], pv[1]);
+      pa[nt >> 1][(nt & 1) * 2 + 1] = pack2(pv[2], pv[3]);
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) l_run[r] = l_run[r] * alpha[r] + psum[r];
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) {
+      o[nt][0] *= alpha[0]; o[nt][1] *= alpha[0];
+      o[nt][2] *= alpha[1]; o[nt][3] *= alpha[1];
+    }
+
+    // ---- O += P V
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int tok = j * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+      for (int dp = 0; dp < 8; ++dp) {
+        const int c = 2 * dp + (lane >> 4);
+        uint32_t r0, r1, r2, r3;
+        ldsm_x4_trans(v_base + tok * kPfRowBytes + ((c ^ (tok & 7)) << 4), r0, r1, r2, r3);
+        mma_m16n8k16_bf16(o[2 * dp], pa[j][0], pa[j][1], pa[j][2], pa[j][3], r0, r1);
+        mma_m16n8k16_bf16(o[2 * dp + 1], pa[j][0], pa[j][1], pa[j][2], pa[j][3], r2, r3);
+      }
+    }
+    __syncthreads();       // the tiles are free for the next load
+  }
+
+  // ---- normalise and write
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+  }
+  const float inv0 = l_run[0] > 0.f ? 1.f / l_run[0] : 0.f, inv1 = l_run[1] > 0.f ? 1.f / l_run[1] : 0.f;
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt) {
+    if (i0 < n_q) *reinterpret_cast<float2*>(out0 + nt * 8 + qd) = make_float2(o[nt][0] * inv0, o[nt][1] * inv0);
+    if (i1 < n_q) *reinterpret_cast<float2*>(out1 + nt * 8 + qd) = make_float2(o[nt][2] * inv1, o[nt][3] * inv1);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, __nv_bfloat16* out, int out_tokens,
+                               int out_width, bool rotate, cudaStream_t stream) {
+  if (width == 0) return cudaSuccess;
+  if (width % 128 != 0) return cudaErrorInvalidValue;
+  dim3 grid((out_tokens + 31) / 32, a.batch);
+  gather_rows_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(pool), width, out, out_tokens,
+                                               out_width, a.slots, a.lens, a.geom, rotate ? a.rope : RopeTable(), a.status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
+                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream) {
+  dim3 grid((n_q + kPfRows - 1) / kPfRows, a.n_q_heads, a.batch);
+  prefill_attn_kernel<<<grid, 128, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q), k_rows, v_rows, out, n_q,
+                                                a.n_q_heads, a.n_kv_heads, kv_tokens, kv_width, a.slots, a.lens,
+                                                a.geom.max_batch, a.geom.max_pages_per_seq * a.geom.page_tokens,
+                                                a.scale_log2e, a.status);
+  return cudaGetLastError();
+}
+
+}  // namespace echokv

@@ -1,0 +1,19 @@
+// Prefill-shaped attention (many queries per sequence): host interface of the two CUDA-core / mma.sync kernels.
+#pragma once
+
+#include "kernels.h"
+
+namespace echokv {
+
+// Stored dims 0 .. width-1 (whole heads of 128, bf16) of every cached token, from a paged pool into contiguous rows
+// out[b][token][out_width]; keys are rotated to their positions if `rotate` and a.rope is set.
+cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, __nv_bfloat16* out, int out_tokens,
+                               int out_width, bool rotate, cudaStream_t stream);
+
+// Eq. 7 for n_q queries per sequence (a.q: [B][n_q][H_q][128] bf16), query i at position len - n_q + i attending the
+// keys up to its own, over k_rows / v_rows [B][kv_tokens][kv_width] bf16.  out: fp32 [B][n_q][H_q][128].
+// A sequence with fewer than n_q cached tokens gets zeros and the device status EBADLENGTH.
+cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
+                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream);
+
+}  // namespace echokv

@@ -74,6 +74,10 @@ struct PairParams {
   const __nv_bfloat16* bk;    // bias of the K predictor or null (ROPE instantiations only: otherwise it cancels)
   float* s_out;               // KS instantiations: scores [b][query head][l_cap], base-2 units
   int l_cap;
+  // KS instantiations, when set: no scores at all -- the predicted rows themselves (bias added, rotated if
+  // store_rotate) are written as bf16 to store_out[b][token][store_width] at the head's flat dims
+  __nv_bfloat16* store_out;
+  int store_tokens, store_width, store_rotate;
 };
 
 template <int G>
@@ -368,7 +372,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
       const uint32_t k_par = KS ? ((n >> 1) & 1u) : par;
       const uint32_t k_addr = lane_addr + k_acc * kAccCols;
       // queries of the pair's query heads, pre-scaled (the previous item's K epilogue is long done)
-      for (int idx = et; idx < 2 * G * 128; idx += kEpilogueThreads) {
+      for (int idx = et; idx < (KS && p.store_out != nullptr ? 0 : 2 * G * 128); idx += kEpilogueThreads) {
         const int hh = idx / (G * 128), rem = idx % (G * 128);
         float v = 0.f;
         if (hh == 0 || second)
@@ -389,7 +393,57 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
       float sc[G];
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) sc[gi] = 0.f;
-      if constexpr (ROPE) {
+      bool stored_rows = false;
+      if constexpr (KS && ROPE) {
+        if (p.store_out != nullptr) {
+          // the predicted rows go to memory: (token `row` of this CTA, head `sel`), 128 values as bf16
+          stored_rows = true;
+          const int t_row = w.tile * kTileTokens + (int)rank * kCtaTokens + row;
+          const bool live = t_row < len && (sel == 0 || second);
+          const bool rotate = p.store_rotate != 0 && p.rope.cs != nullptr;
+          const float2* cs_row = rotate ? p.rope.cs + min(t_row, p.rope.stride - 1) : nullptr;
+          __nv_bfloat16* dst = p.store_out + ((size_t)b * p.store_tokens + (live ? t_row : 0)) * p.store_width +
+                               (size_t)(kvh0 + sel) * 128;
+#pragma unroll 1
+          for (int cb = 0; cb < 4; ++cb) {
+            float lo[16], hi[16];
+            tmem_ld16(k_addr + sel * 128 + cb * 16, lo);
+            tmem_ld16(k_addr + sel * 128 + 64 + cb * 16, hi);
+            uint32_t pl[8], ph[8];
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+              float v_lo[2], v_hi[2];
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const float k_lo = lo[j + e] + t.kb[sel][cb * 16 + j + e], k_hi = hi[j + e] + t.kb[sel][64 + cb * 16 + j + e];
+                if (rotate) {
+                  const float2 cw = cs_row[(size_t)(cb * 16 + j + e) * p.rope.stride];
+                  v_lo[e] = k_lo * cw.x - k_hi * cw.y;
+                  v_hi[e] = k_hi * cw.x + k_lo * cw.y;
+                } else {
+                  v_lo[e] = k_lo;
+                  v_hi[e] = k_hi;
+                }
+              }
+              const __nv_bfloat162 a2 = __floats2bfloat162_rn(v_lo[0], v_lo[1]);
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(v_hi[0], v_hi[1]);
+              pl[j / 2] = *reinterpret_cast<const uint32_t*>(&a2);
+              ph[j / 2] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            if (live) {
+              uint4* d_lo = reinterpret_cast<uint4*>(dst + cb * 16);
+              uint4* d_hi = reinterpret_cast<uint4*>(dst + 64 + cb * 16);
+              d_lo[0] = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+              d_lo[1] = make_uint4(pl[4], pl[5], pl[6], pl[7]);
+              d_hi[0] = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+              d_hi[1] = make_uint4(ph[4], ph[5], ph[6], ph[7]);
+            }
+          }
+        }
+      }
+      if (stored_rows) {
+        // (nothing to score)
+      } else if constexpr (ROPE) {
         // this thread's row is token t_rot: features j and j + 64 of the head turn by t_rot * theta^(-2j/128)
         const int t_rot = min(w.tile * kTileTokens + (int)rank * kCtaTokens + row, p.rope.stride - 1);
         const float2* cs_row = p.rope.cs + t_rot;
@@ -441,7 +495,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
         epilogue_sync();       // every warp is done reading the accumulator (and the staged queries)
         if (et == 0) mbar_arrive_cluster(k_acc ? acc_empty1 : acc_empty0);
         // scores of every token slot of the tile; slots without a predicted token read as -inf downstream
-        if (t_seq < p.l_cap && (sel == 0 || second)) {
+        if (p.store_out == nullptr && t_seq < p.l_cap && (sel == 0 || second)) {
           float* dst = p.s_out + ((size_t)b * p.n_q_heads + (size_t)(kvh0 + sel) * G) * p.l_cap + t_seq;
 #pragma unroll
           for (int gi = 0; gi < G; ++gi) dst[(size_t)gi * p.l_cap] = tok_valid ? sc[gi] : -INFINITY;
@@ -607,15 +661,21 @@ cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUt
     if (p.rope.cs == nullptr) return cudaErrorInvalidValue;     // (only built for rotated keys)
     return launch_g<G, true, true>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
   }
+  if (p.store_out != nullptr) return cudaErrorInvalidValue;     // (rows are stored by the G = 1 instantiation, below)
   if (p.rope.cs != nullptr) return launch_g<G, true, false>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
   return launch_g<G, false, false>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
 }
 
 }  // namespace
 
+struct StoreRows {
+  __nv_bfloat16* out = nullptr;
+  int tokens = 0, width = 0, rotate = 0;
+};
+
 static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
                                     const TcLayerMaps& layer, int sm_count, cudaStream_t stream, float* s_out,
-                                    int l_cap) {
+                                    int l_cap, const StoreRows& store = StoreRows()) {
   if (!anchor.pools_ready || !layer.weights_ready) return cudaErrorInvalidValue;
   if (r.m > 0 && !layer.pools_ready) return cudaErrorInvalidValue;
   const int g = a.n_q_heads / a.n_kv_heads;
@@ -645,6 +705,10 @@ static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const
   p.bk = reinterpret_cast<const __nv_bfloat16*>(r.bk);
   p.s_out = s_out;
   p.l_cap = l_cap;
+  p.store_out = store.out;
+  p.store_tokens = store.tokens;
+  p.store_width = store.width;
+  p.store_rotate = store.rotate;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;
@@ -661,6 +725,11 @@ static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const
     const long long max_items = (long long)p.nb * tiles_cap * p.n_pairs;
     const int n_clusters = (int)(max_items < sm_count / 2 ? max_items : sm_count / 2);
     cudaError_t e;
+    if (store.out != nullptr) {      // rows to memory: no queries involved, one instantiation serves every group size
+      e = launch_g<1, true, true>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream);
+      if (e != cudaSuccess) return e;
+      continue;
+    }
     switch (g) {
       case 1: e = launch_g<1>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream); break;
       case 2: e = launch_g<2>(anchor, lk, lv, lkr, lvr, lk8, lv8, layer, p, n_clusters, stream); break;
@@ -683,6 +752,27 @@ cudaError_t launch_recon_pair_key_scores(const AttnArgs& a, const ReconArgs& r, 
                                          cudaStream_t stream) {
   if (scores == nullptr) return cudaErrorInvalidValue;
   return launch_pair_impl(a, r, anchor, layer, sm_count, stream, scores, l_cap);
+}
+
+cudaError_t launch_recon_pair_store(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                                    const TcLayerMaps& layer, bool values, __nv_bfloat16* out, int out_tokens,
+                                    int out_width, int sm_count, cudaStream_t stream) {
+  if (out == nullptr) return cudaErrorInvalidValue;
+  StoreRows store;
+  store.out = out;
+  store.tokens = out_tokens;
+  store.width = out_width;
+  store.rotate = values ? 0 : 1;                 // (keys are rotated only if a.rope is set; values never)
+  if (!values) return launch_pair_impl(a, r, anchor, layer, sm_count, stream, nullptr, 0, store);
+  // the V predictor over the V pools: the same kernel with the V maps in the K places
+  auto as_keys = [](const TcLayerMaps& m) {
+    TcLayerMaps t = m;
+    t.k_pool = m.v_pool; t.k_pool_run = m.v_pool_run; t.k_pool_run128 = m.v_pool_run128;
+    t.wk = m.wv; t.wk_half = m.wv_half;
+    return t;
+  };
+  const TcLayerMaps av = as_keys(anchor), lv = as_keys(layer);
+  return launch_pair_impl(a, r, av, lv, sm_count, stream, nullptr, 0, store);
 }
 
 }  // namespace echokv

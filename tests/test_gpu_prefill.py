@@ -1,0 +1,119 @@
+"""GPU parity of the prefill-shaped call: the last n_q cached tokens of every sequence as causal queries over the
+rebuilt cache (rebuilt once per call into a bf16 scratch, then a causal attention kernel)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import echokv_oracle as O
+from paper_2603_22910_b200 import binding, build, synth
+from tests.harness import Case, errors
+
+pytestmark = pytest.mark.gpu
+
+THETA = 10000.0
+
+# This call materialises the rebuilt K~ / V~ rows in bf16 (the decode calls keep them in fp32): a query that attends a
+# handful of tokens returns nearly a single V~ row, so the bf16 rounding of that row (|v| 2^-9, |v| up to ~5 here) and
+# of the keys behind its few probabilities shows unaveraged in the maximum error.  rel-L2 as for the decode calls.
+TOL_PREFILL = dict(max_abs=4e-2, rel_l2=5e-3)
+
+
+def assert_parity(out, ref, dtype, what=""):
+    max_abs, rel_l2 = errors(out, ref)
+    assert np.all(np.isfinite(out)), "non-finite output " + what
+    assert max_abs <= TOL_PREFILL["max_abs"] and rel_l2 <= TOL_PREFILL["rel_l2"], \
+        "%s: max_abs %.3e, rel_l2 %.3e" % (what, max_abs, rel_l2)
+    return max_abs, rel_l2
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.lib()
+
+
+def queries(w, n_q, seed):
+    return (synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, seed)).to(synth.torch_dtype(w))
+
+
+def oracle_prefill(case, layer, q, b, rope):
+    w = case.w
+    qn = O.widen(synth.to_numpy_stored(q))[b]
+    a = w.anchor_of(layer)
+    kg, vg = case._stored(a, "k", b), case._stored(a, "v", b)
+    if w.is_anchor(layer):
+        return O.prefill_attention(qn, kg, vg, None, None, None, None, w.n_kv_heads, rope_theta=rope)
+    L = kg.shape[0]
+    kl = case._stored(layer, "k", b) if w.m else np.zeros((L, 0))
+    vl = case._stored(layer, "v", b) if w.m else np.zeros((L, 0))
+    Wk, Wv, bk, bv = (None if t is None else O.widen(synth.to_numpy_stored(t)) for t in case.host_w[layer])
+    return O.prefill_attention(qn, kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv, rope_theta=rope)
+
+
+CASES = [
+    # name, base, overrides, lens, n_q, biases, rope
+    ("gqa_one_tile", synth.C2, dict(batch=2, context=700), [700, 333], 37, False, None),
+    ("gqa_three_tiles", synth.C2, dict(batch=2, context=600, random_pages=True), [600, 200], 150, True, None),
+    ("mha", synth.C1, dict(batch=2, context=500), [500, 257], 64, False, None),
+    ("gqa_rope", synth.C2, dict(batch=2, context=700, page_tokens=64, random_pages=True), [700, 130], 65, True, THETA),
+    ("one_query_is_the_decode_step", synth.C2, dict(batch=2, context=300), [300, 17], 1, False, None),
+    ("every_token_a_query", synth.C2, dict(batch=1, context=200, n_retained_heads=6), [200], 200, False, THETA),
+    ("nothing_retained", synth.C2, dict(batch=2, context=400, n_retained_heads=0), [400, 129], 70, False, None),
+]
+
+
+@pytest.mark.parametrize("name,base,over,lens,n_q,biases,rope", CASES, ids=[c[0] for c in CASES])
+def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope):
+    w = base.replace(**over)
+    case = Case(w, lens=lens, layers=[0, 1], biases=biases, rope=rope)
+    ctx = case.ctx
+    for layer in (1, 0):
+        q = queries(w, n_q, layer)
+        out = ctx.prefill_attention(layer, q.to(ctx.device), case.seq_lens)
+        torch.cuda.synchronize()
+        out = out.cpu().numpy().astype(np.float64)
+        for b in range(w.batch):
+            ref = oracle_prefill(case, layer, q, b, rope)
+            assert_parity(out[b], ref, w.dtype, "%s layer %d seq %d" % (name, layer, b))
+    if n_q == 1:     # a single query per sequence: the same function as the decode call
+        q = queries(w, 1, 1)
+        dec = ctx.decode_attention(1, q[:, 0].contiguous().to(ctx.device), case.seq_lens).cpu().numpy()
+        pre = ctx.prefill_attention(1, q.to(ctx.device), case.seq_lens).cpu().numpy()[:, 0]
+        assert_parity(pre, dec.astype(np.float64), w.dtype, name + " vs decode")
+    assert ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+def test_prefill_short_sequences_and_argument_checks():
+    w = synth.C2.replace(batch=3, context=300)
+    case = Case(w, lens=[300, 20, 64], layers=[0, 1])
+    ctx, dev = case.ctx, case.ctx.device
+    n_q = 64
+    q = queries(w, n_q, 3)
+    out = ctx.prefill_attention(1, q.to(dev), case.seq_lens).cpu().numpy().astype(np.float64)
+    assert ctx.device_status() == binding.ECHOKV_EBADLENGTH       # sequence 1 holds fewer tokens than queries
+    assert not out[1].any()
+    for b in (0, 2):
+        assert_parity(out[b], oracle_prefill(case, 1, q, b, None), w.dtype, "seq %d" % b)
+    lib, h = binding.lib(), ctx.handle
+    o = torch.empty(q.shape, dtype=torch.float32, device=dev)
+    qd = q.to(dev)
+    scratch = ctx.prefill_scratch
+    args = (qd.data_ptr(), o.data_ptr())
+    assert lib.echokv_prefill_attention(h, 1, *args, 0, None, case.seq_lens.data_ptr(), 3, scratch.data_ptr(),
+                                        scratch.numel(), None) == binding.ECHOKV_EINVAL
+    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, scratch.data_ptr(), 1024,
+                                        None) == binding.ECHOKV_ECAPACITY
+    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, None, 0,
+                                        None) == binding.ECHOKV_EINVAL
+    ctx.set_full_precision_window(4, 128)
+    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, scratch.data_ptr(),
+                                        scratch.numel(), None) == binding.ECHOKV_EUNSUPPORTED
+    case.close()
+    small = Case(synth.C0, layers=[1])
+    n = torch.zeros(1, dtype=torch.int64)
+    import ctypes as C
+    nbytes = C.c_uint64(0)
+    assert lib.echokv_prefill_scratch_bytes(C.byref(small.cfg), C.byref(nbytes)) == binding.ECHOKV_EUNSUPPORTED
+    small.close()
