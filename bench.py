@@ -426,6 +426,72 @@ def run_reference(args):
     return 0
 
 
+def run_prefill(args):
+    """--prefill-queries N: the prefill-shaped call on the compressed layer (N causal queries per sequence at the end
+    of the cached context), timed on the device; an extra measurement beside the decode benchmark, one JSON line."""
+    import numpy as np
+    import torch
+    from paper_2603_22910_b200 import binding, synth
+    from oracle import echokv_oracle as O
+    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio)
+    n_q = args.prefill_queries
+    st = State(w, 0, [0, 1])
+    ctx, dev = st.ctx, st.dev
+    if args.rope:
+        ctx.set_rope(args.rope)
+    st.rope = args.rope
+    q = synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, 1, device=dev).to(torch.bfloat16)
+    out = torch.empty(q.shape, dtype=torch.float32, device=dev)
+    for _ in range(max(3, args.warmup)):
+        ctx.prefill_attention(1, q, st.lens, out=out)
+    torch.cuda.synchronize()
+    ctx.set_kernel_timing(True)
+    ctx.read_kernel_timing_by_kind()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ctx.prefill_attention(1, q, st.lens, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    recon_ms, recon_n = ctx.read_kernel_timing_by_kind()["recon"]
+    assert ctx.device_status() == binding.ECHOKV_OK
+    peaks, peaks_kind = load_peaks()
+    tokens = float(w.batch) * w.context
+    recon_flops = tokens * 4.0 * w.d_in * w.d_drop
+    k_ms = recon_ms / max(recon_n, 1)
+    peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+    # causal attention: query i sees L - n_q + i + 1 keys; 4 d FLOP per (query, key, head)
+    seen = n_q * (w.context - n_q) + n_q * (n_q + 1) / 2.0
+    attn_flops = w.batch * w.n_q_heads * seen * 4.0 * w.head_dim
+    # parity on the last 16 queries of sequence 0 (they see the whole cache)
+    n_chk = min(16, n_q)
+    inputs = st.oracle_inputs(1, 0)
+    q_chk = O.widen(synth.to_numpy_stored(q[0, -n_chk:].cpu()))
+    ref = O.prefill_attention(q_chk, *inputs[1:], n_kv_heads=w.n_kv_heads, rope_theta=args.rope or None)
+    got = out[0, -n_chk:].cpu().numpy().astype(np.float64)
+    line = {
+        "metric": "prefill_query_tokens_per_s", "value": w.batch * n_q / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "%s, prefill-shaped: %d causal queries per sequence over B=%d L=%d" %
+                               (w.name, n_q, w.batch, w.context), "parallelism": "one GPU"},
+        "roofline": {"bound": "tensor", "achieved": recon_flops / (k_ms * 1e-3) / 1e12, "peak": peak_tf,
+                     "unit": "TFLOP/s", "frac": recon_flops / (k_ms * 1e-3) / 1e12 / peak_tf, "traffic": None,
+                     "kernel": "recon_pair_kernel (rows to memory), K pass + V pass", "kernel_ms": k_ms,
+                     "share_of_step": k_ms / ms, "peak_source": "%s (cuBLAS bf16 GEMM, sustained)" % peaks_kind},
+        "attention": {"kernel": "prefill_attn_kernel (mma.sync) + gather_rows_kernel x 2", "ms": ms - k_ms,
+                      "tflops": attn_flops / ((ms - k_ms) * 1e-3) / 1e12},
+        "parity_vs_oracle": {"rows": "last %d queries of sequence 0" % n_chk,
+                             "max_abs": float(np.max(np.abs(got - ref))),
+                             "rel_l2": float(np.linalg.norm(got - ref) / np.linalg.norm(ref))},
+        "rope_theta": args.rope or None,
+    }
+    print(json.dumps(line))
+    ctx.close()
+    return 0
+
+
 def workload_config(w, full=False):
     elem = 2 if w.dtype == "bf16" else 4
     pages = "%d-token pages%s" % (w.page_tokens, " in a random order" if w.random_pages else "")
@@ -776,6 +842,8 @@ def main():
                     "read (the cache then holds un-rotated keys); 0 = none, as in the paper's configurations")
     ap.add_argument("--save-k", action="store_true", help="compressed layers keep their keys whole, only the values "
                     "are predicted (the paper's \"save K\" ablation); needs --decode-mode absorbed")
+    ap.add_argument("--prefill-queries", type=int, default=0, help="time the prefill-shaped call instead: this many "
+                    "causal queries per sequence on the compressed layer (an extra measurement, its own JSON line)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")
@@ -794,6 +862,8 @@ def main():
         args.steps = 10      # a 32-layer step is ~25x a single layer-step
     if args.impl == "reference":
         return run_reference(args)
+    if args.prefill_queries:
+        return run_prefill(args)
     return run_ours(args)
 
 
