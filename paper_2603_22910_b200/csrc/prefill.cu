@@ -80,6 +80,14 @@ constexpr int kPfRows = 64;      // query rows per CTA: 4 warps x 16
 constexpr int kPfKeys = 64;      // keys per tile
 constexpr int kPfRowBytes = 256; // 128 bf16
 
+// 16-byte asynchronous copy global -> shared; n_bytes = 0 writes zeros without reading
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t n_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -93,8 +101,9 @@ __global__ void __launch_bounds__(128) prefill_attn_kernel(const __nv_bfloat16* 
                                                            const int32_t* __restrict__ slots,
                                                            const int32_t* __restrict__ lens, int max_batch,
                                                            int capacity, float scale_log2e, int32_t* status) {
-  __shared__ __align__(128) unsigned char k_tile[kPfKeys * kPfRowBytes];
-  __shared__ __align__(128) unsigned char v_tile[kPfKeys * kPfRowBytes];
+  // two buffers of a key tile and a value tile each: the next tile is copied while this one is multiplied
+  extern __shared__ __align__(128) unsigned char pf_smem[];
+  constexpr int kTileBytes = kPfKeys * kPfRowBytes;
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int qd = (lane & 3) * 2;
@@ -137,25 +146,34 @@ __global__ void __launch_bounds__(128) prefill_attn_kernel(const __nv_bfloat16* 
   // keys this CTA's rows may see: up to the position of its last row
   const int last_row = min(n_q, (qt + 1) * kPfRows) - 1;
   const int kv_end = len - n_q + last_row + 1;
-  const uint32_t k_base = smem_u32(k_tile), v_base = smem_u32(v_tile);
+  const uint32_t smem_base = smem_u32(pf_smem);
   const __nv_bfloat16* k_seq = ks + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
   const __nv_bfloat16* v_seq = vs + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
-
-  for (int kv0 = 0; kv0 < kv_end; kv0 += kPfKeys) {
-    // ---- stage 64 key rows and 64 value rows (16-byte pieces swizzled by row so that ldmatrix is conflict-free)
+  // stage 64 key rows and 64 value rows into buffer `buf` (16-byte pieces swizzled by row so that ldmatrix is
+  // conflict-free; rows past the last key the CTA may see are zero-filled)
+  auto stage = [&](int kv0, int buf) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int idx = tid + 128 * i, r = idx >> 4, c = idx & 15;
-      uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
-      if (kv0 + r < kv_end) {
-        kk = *reinterpret_cast<const uint4*>(k_seq + (size_t)(kv0 + r) * kv_width + c * 8);
-        vv = *reinterpret_cast<const uint4*>(v_seq + (size_t)(kv0 + r) * kv_width + c * 8);
-      }
-      const int off = r * kPfRowBytes + ((c ^ (r & 7)) << 4);
-      *reinterpret_cast<uint4*>(k_tile + off) = kk;
-      *reinterpret_cast<uint4*>(v_tile + off) = vv;
+      const bool in = kv0 + r < kv_end;
+      const size_t src = (size_t)(in ? kv0 + r : 0) * kv_width + c * 8;
+      const uint32_t off = smem_base + buf * 2 * kTileBytes + r * kPfRowBytes + ((c ^ (r & 7)) << 4);
+      cp_async16(off, k_seq + src, in ? 16u : 0u);
+      cp_async16(off + kTileBytes, v_seq + src, in ? 16u : 0u);
+    }
+    cp_async_commit();
+  };
+  stage(0, 0);
+
+  for (int kv0 = 0, tile = 0; kv0 < kv_end; kv0 += kPfKeys, ++tile) {
+    if (kv0 + kPfKeys < kv_end) {
+      stage(kv0 + kPfKeys, (tile + 1) & 1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
     }
     __syncthreads();
+    const uint32_t k_base = smem_base + (tile & 1) * 2 * kTileBytes, v_base = k_base + kTileBytes;
 
     // ---- S = Q K^T for this warp's 16 rows x 64 keys
     float sc[8][4];
@@ -266,7 +284,13 @@ cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, _
 cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
                                 int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream) {
   dim3 grid((n_q + kPfRows - 1) / kPfRows, a.n_q_heads, a.batch);
-  prefill_attn_kernel<<<grid, 128, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q), k_rows, v_rows, out, n_q,
+  const size_t smem = 4 * (size_t)kPfKeys * kPfRowBytes;
+  cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared);
+  if (e != cudaSuccess) return e;
+  prefill_attn_kernel<<<grid, 128, smem, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q), k_rows, v_rows, out, n_q,
                                                 a.n_q_heads, a.n_kv_heads, kv_tokens, kv_width, a.slots, a.lens,
                                                 a.geom.max_batch, a.geom.max_pages_per_seq * a.geom.page_tokens,
                                                 a.scale_log2e, a.status);
