@@ -141,6 +141,15 @@ int echokv_set_block_table(echokv_ctx* ctx, const int32_t* dev_block_table);
 int echokv_append_kv(echokv_ctx* ctx, int layer, const void* k_new, const void* v_new,
                      const int32_t* dev_seq_slots, const int32_t* dev_positions, int B, void* stream);
 
+/* The same for n_tokens consecutive new tokens per sequence (a chunk of a prompt during prefill): k_new, v_new are
+ * device pointers [B][n_tokens][n_kv_heads][head_dim], dev_first_positions[b] = position of the first of them.  With
+ * a sink / window set, of the chunk's tokens only the last n_window enter the window ring (the others would be
+ * overwritten by them anyway).  echokv_append_kv is this call with n_tokens = 1.
+ * Errors: as echokv_append_kv; ECAPACITY also if n_tokens exceeds 65535 or the sequence capacity. */
+int echokv_append_kv_chunk(echokv_ctx* ctx, int layer, const void* k_new, const void* v_new,
+                           const int32_t* dev_seq_slots, const int32_t* dev_first_positions, int n_tokens, int B,
+                           void* stream);
+
 /* The switch from full-cache generation to compressed inference (Section 3.1: compression is evicting part
  * of each token's K / V, at the moment memory runs short; Section 5.4: or already during prefill).  The caller
  * has cached layer `layer` at full width in pools of its own, k_full / v_full: device pointers

@@ -49,6 +49,8 @@ EXPORTS = {
     "echokv_set_block_table": (C.c_int, [C.c_void_p, C.c_void_p]),
     "echokv_append_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_int, C.c_void_p]),
+    "echokv_append_kv_chunk": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_int, C.c_int, C.c_void_p]),
     "echokv_compress_layer": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_int, C.c_void_p]),
     "echokv_decode_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -208,6 +210,12 @@ class Context:
         _check(lib().echokv_append_kv(self.handle, layer, _ptr(k_new), _ptr(v_new), _ptr(seq_slots),
                                       _ptr(positions), k_new.shape[0], _stream_handle(stream)),
                "echokv_append_kv")
+
+    def append_kv_chunk(self, layer: int, k_new, v_new, first_positions, seq_slots=None, stream=None) -> None:
+        """k_new, v_new [B][n_tokens][H_kv][d]: n_tokens consecutive new tokens per sequence."""
+        _check(lib().echokv_append_kv_chunk(self.handle, layer, _ptr(k_new), _ptr(v_new), _ptr(seq_slots),
+                                            _ptr(first_positions), k_new.shape[1], k_new.shape[0],
+                                            _stream_handle(stream)), "echokv_append_kv_chunk")
 
     def compress_layer(self, layer: int, k_full, v_full, seq_lens, seq_begins=None, seq_slots=None, stream=None) -> None:
         """Evict a layer cached at full width ([n_pages][page_tokens][D] pools) down to its retained dims."""

@@ -228,9 +228,9 @@ SideArgs side_args(const echokv_ctx* c, const Layer& L) {
 
 // The new token's dropped dims of a compressed layer go to the side buffers while a sink / window is set.
 int append_side(echokv_ctx* c, const Layer& L, const void* k_new, const void* v_new, const int32_t* slots,
-                const int32_t* positions, int B, cudaStream_t s) {
+                const int32_t* positions, int B, int n_tokens, cudaStream_t s) {
   if (!side_active(c, L)) return ECHOKV_OK;
-  if (launch_append_side(c->cfg.dtype, side_args(c, L), c->d.m, c->d.D, k_new, v_new, slots, positions, B,
+  if (launch_append_side(c->cfg.dtype, side_args(c, L), c->d.m, c->d.D, k_new, v_new, slots, positions, B, n_tokens,
                          c->cfg.max_batch, status_ptr(c), s) != cudaSuccess)
     return ECHOKV_ECUDA;
   c->launches += 1;
@@ -539,22 +539,28 @@ int echokv_set_stored_path(echokv_ctx* c, int path) {
   return ECHOKV_OK;
 }
 
-int echokv_append_kv(echokv_ctx* c, int layer, const void* k_new, const void* v_new,
-                     const int32_t* dev_seq_slots, const int32_t* dev_positions, int B, void* stream) {
-  if (!c || !k_new || !v_new || !dev_positions) return ECHOKV_EINVAL;
-  if (layer < 0 || layer >= c->cfg.n_layers || B < 1) return ECHOKV_EINVAL;
-  if (B > c->cfg.max_batch) return ECHOKV_ECAPACITY;
+int echokv_append_kv_chunk(echokv_ctx* c, int layer, const void* k_new, const void* v_new,
+                           const int32_t* dev_seq_slots, const int32_t* dev_first_positions, int n_tokens, int B,
+                           void* stream) {
+  if (!c || !k_new || !v_new || !dev_first_positions) return ECHOKV_EINVAL;
+  if (layer < 0 || layer >= c->cfg.n_layers || B < 1 || n_tokens < 1) return ECHOKV_EINVAL;
+  if (B > c->cfg.max_batch || n_tokens > c->d.capacity || n_tokens > 65535) return ECHOKV_ECAPACITY;
   if (!c->table) return ECHOKV_ENOTABLE;
   const Layer& L = c->layers[layer];
   const int k_width = L.anchor ? c->d.D : c->d.mk, v_width = L.anchor ? c->d.D : c->d.m;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (k_width == 0 && v_width == 0)   // nothing of this layer is kept in the pools (m = 0)
-    return append_side(c, L, k_new, v_new, dev_seq_slots, dev_positions, B, static_cast<cudaStream_t>(stream));
+    return append_side(c, L, k_new, v_new, dev_seq_slots, dev_first_positions, B, n_tokens, s);
   const cudaError_t e = launch_append(c->cfg.dtype, L.k_pool, L.v_pool, k_width, v_width, c->d.D, k_new, v_new,
-                                      dev_seq_slots, dev_positions, B, geom_of(c), status_ptr(c),
-                                      static_cast<cudaStream_t>(stream));
+                                      dev_seq_slots, dev_first_positions, B, n_tokens, geom_of(c), status_ptr(c), s);
   if (e != cudaSuccess) return ECHOKV_ECUDA;
   c->launches += 1;
-  return append_side(c, L, k_new, v_new, dev_seq_slots, dev_positions, B, static_cast<cudaStream_t>(stream));
+  return append_side(c, L, k_new, v_new, dev_seq_slots, dev_first_positions, B, n_tokens, s);
+}
+
+int echokv_append_kv(echokv_ctx* c, int layer, const void* k_new, const void* v_new,
+                     const int32_t* dev_seq_slots, const int32_t* dev_positions, int B, void* stream) {
+  return echokv_append_kv_chunk(c, layer, k_new, v_new, dev_seq_slots, dev_positions, 1, B, stream);
 }
 
 int echokv_compress_layer(echokv_ctx* c, int layer, const void* k_full, const void* v_full,

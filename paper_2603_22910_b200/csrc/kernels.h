@@ -26,9 +26,10 @@ size_t rope_table_pairs(int stride, int head_dim);
 RopeTable rope_table_view(const float2* buffer, int stride, int head_dim);
 cudaError_t launch_rope_table(float2* buffer, int stride, int head_dim, double theta, cudaStream_t stream);
 
-// Append one token per sequence: writes the first k_width flat dims of k_new and the first v_width of v_new.
+// Append n_tokens consecutive tokens per sequence (k_new / v_new: [B][n_tokens][D]; positions[b] = where the first
+// one goes): writes the first k_width flat dims of every new K row and the first v_width of every new V row.
 cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int k_width, int v_width, int D, const void* k_new,
-                          const void* v_new, const int32_t* slots, const int32_t* positions, int B,
+                          const void* v_new, const int32_t* slots, const int32_t* positions, int B, int n_tokens,
                           const PageGeom& geom, int32_t* status, cudaStream_t stream);
 
 // Attention of query heads whose KV head is stored (heads 0..n_heads-1 of a pool of row width
@@ -73,9 +74,9 @@ struct SideArgs {
   int n_sink, n_window, d_drop;
 };
 
-// Append: the new token's dropped dims go to its side slots.
+// Append: the new tokens' dropped dims go to their side slots.
 cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, const void* k_new, const void* v_new,
-                               const int32_t* slots, const int32_t* positions, int B, int max_batch,
+                               const int32_t* slots, const int32_t* positions, int B, int n_tokens, int max_batch,
                                int32_t* status, cudaStream_t stream);
 
 // Evict a full-width cache ([n_pages][page_tokens][D], same block table) down to what a compressed layer keeps:

@@ -66,10 +66,11 @@ __global__ void __launch_bounds__(128) append_kernel(T* __restrict__ k_pool, T* 
                                                      const int32_t* __restrict__ slots,
                                                      const int32_t* __restrict__ positions,
                                                      PageGeom g, int32_t* status) {
-  const int b = blockIdx.x;
+  // block (b, i): token i of the gridDim.y new tokens of sequence b, written at position positions[b] + i
+  const int b = blockIdx.x, i_tok = blockIdx.y, n_tok = gridDim.y;
   const int slot = slots ? slots[b] : b;
-  const int pos = positions[b];
-  if (slot < 0 || slot >= g.max_batch || pos < 0 || pos >= g.max_pages_per_seq * g.page_tokens) {
+  const int pos = positions[b] + i_tok;
+  if (slot < 0 || slot >= g.max_batch || positions[b] < 0 || pos >= g.max_pages_per_seq * g.page_tokens) {
     if (threadIdx.x == 0) report(status, ECHOKV_EBADPAGE);
     return;
   }
@@ -80,8 +81,8 @@ __global__ void __launch_bounds__(128) append_kernel(T* __restrict__ k_pool, T* 
   }
   const size_t row = (size_t)page * g.page_tokens + pos % g.page_tokens;
   constexpr int kVec = 16 / sizeof(T);
-  const uint4* ks = reinterpret_cast<const uint4*>(k_new + (size_t)b * D);
-  const uint4* vs = reinterpret_cast<const uint4*>(v_new + (size_t)b * D);
+  const uint4* ks = reinterpret_cast<const uint4*>(k_new + ((size_t)b * n_tok + i_tok) * D);
+  const uint4* vs = reinterpret_cast<const uint4*>(v_new + ((size_t)b * n_tok + i_tok) * D);
   uint4* kd = reinterpret_cast<uint4*>(k_pool + row * (size_t)k_width);
   uint4* vd = reinterpret_cast<uint4*>(v_pool + row * (size_t)v_width);
   for (int i = threadIdx.x; i < k_width / kVec; i += blockDim.x) kd[i] = ks[i];
@@ -89,14 +90,15 @@ __global__ void __launch_bounds__(128) append_kernel(T* __restrict__ k_pool, T* 
 }
 
 cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int k_width, int v_width, int D, const void* k_new,
-                          const void* v_new, const int32_t* slots, const int32_t* positions, int B,
+                          const void* v_new, const int32_t* slots, const int32_t* positions, int B, int n_tokens,
                           const PageGeom& geom, int32_t* status, cudaStream_t stream) {
+  const dim3 grid(B, n_tokens);
   if (dtype == ECHOKV_BF16) {
-    append_kernel<__nv_bfloat16><<<B, 128, 0, stream>>>(
+    append_kernel<__nv_bfloat16><<<grid, 128, 0, stream>>>(
         (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, k_width, v_width, D, (const __nv_bfloat16*)k_new,
         (const __nv_bfloat16*)v_new, slots, positions, geom, status);
   } else {
-    append_kernel<float><<<B, 128, 0, stream>>>((float*)k_pool, (float*)v_pool, k_width, v_width, D,
+    append_kernel<float><<<grid, 128, 0, stream>>>((float*)k_pool, (float*)v_pool, k_width, v_width, D,
                                                 (const float*)k_new, (const float*)v_new, slots,
                                                 positions, geom, status);
   }
@@ -851,23 +853,25 @@ __global__ void __launch_bounds__(128) append_side_kernel(T* __restrict__ k_side
                                                           const int32_t* __restrict__ slots,
                                                           const int32_t* __restrict__ positions, int max_batch,
                                                           int32_t* status) {
-  const int b = blockIdx.x;
+  // block (b, i): token i of the gridDim.y new tokens of sequence b, at position positions[b] + i
+  const int b = blockIdx.x, i_tok = blockIdx.y, n_tok = gridDim.y;
   const int slot = slots ? slots[b] : b;
-  const int pos = positions[b];
-  if (slot < 0 || slot >= max_batch || pos < 0) {
+  const int pos = positions[b] + i_tok;
+  if (slot < 0 || slot >= max_batch || positions[b] < 0) {
     if (threadIdx.x == 0) report(status, ECHOKV_EBADPAGE);
     return;
   }
   constexpr int kVec = 16 / sizeof(T);
   const int n_vec = d_drop / kVec;
-  const uint4* ks = reinterpret_cast<const uint4*>(k_new + (size_t)b * D + m);
-  const uint4* vs = reinterpret_cast<const uint4*>(v_new + (size_t)b * D + m);
+  const uint4* ks = reinterpret_cast<const uint4*>(k_new + ((size_t)b * n_tok + i_tok) * D + m);
+  const uint4* vs = reinterpret_cast<const uint4*>(v_new + ((size_t)b * n_tok + i_tok) * D + m);
   const size_t seq_base = (size_t)slot * (n_sink + n_window);
-  // a token inside the sink is written there; every token also enters the window ring
+  // a token inside the sink is written there; every token also enters the window ring -- of a chunk only the
+  // last n_window tokens, which are the ones that remain in it (and no two of them share a ring slot)
   for (int which = 0; which < 2; ++which) {
     int idx;
     if (which == 0) { if (pos >= n_sink) continue; idx = pos; }
-    else { if (n_window == 0) continue; idx = n_sink + pos % n_window; }
+    else { if (n_window == 0 || i_tok < n_tok - n_window) continue; idx = n_sink + pos % n_window; }
     uint4* kd = reinterpret_cast<uint4*>(k_side + (seq_base + idx) * d_drop);
     uint4* vd = reinterpret_cast<uint4*>(v_side + (seq_base + idx) * d_drop);
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
@@ -878,14 +882,15 @@ __global__ void __launch_bounds__(128) append_side_kernel(T* __restrict__ k_side
 }
 
 cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, const void* k_new, const void* v_new,
-                               const int32_t* slots, const int32_t* positions, int B, int max_batch,
+                               const int32_t* slots, const int32_t* positions, int B, int n_tokens, int max_batch,
                                int32_t* status, cudaStream_t stream) {
+  const dim3 grid(B, n_tokens);
   if (dtype == ECHOKV_BF16) {
-    append_side_kernel<__nv_bfloat16><<<B, 128, 0, stream>>>(
+    append_side_kernel<__nv_bfloat16><<<grid, 128, 0, stream>>>(
         (__nv_bfloat16*)side.k_side, (__nv_bfloat16*)side.v_side, side.n_sink, side.n_window, side.d_drop, m, D,
         (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, slots, positions, max_batch, status);
   } else {
-    append_side_kernel<float><<<B, 128, 0, stream>>>((float*)side.k_side, (float*)side.v_side, side.n_sink,
+    append_side_kernel<float><<<grid, 128, 0, stream>>>((float*)side.k_side, (float*)side.v_side, side.n_sink,
                                                      side.n_window, side.d_drop, m, D, (const float*)k_new,
                                                      (const float*)v_new, slots, positions, max_batch, status);
   }

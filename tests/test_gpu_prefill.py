@@ -117,3 +117,45 @@ def test_prefill_short_sequences_and_argument_checks():
     nbytes = C.c_uint64(0)
     assert lib.echokv_prefill_scratch_bytes(C.byref(small.cfg), C.byref(nbytes)) == binding.ECHOKV_EUNSUPPORTED
     small.close()
+
+
+@pytest.mark.parametrize("window", [None, (4, 128), (3, 20)], ids=["plain", "window_4_128", "window_3_20"])
+def test_chunk_append_equals_token_by_token(window):
+    # a chunk of n new tokens per sequence appended in one call: the cache (pools and side buffers) and the decode
+    # result are those of a context that held the longer sequences from the start
+    w = synth.C2.replace(batch=3, context=700, random_pages=True)
+    n = 150
+    long_lens = [700, 333, 151]
+    ref = Case(w, lens=long_lens, layers=[0, 1], window=window)
+    short = Case(w, lens=[L - n for L in long_lens], layers=[0, 1], window=window)
+    dev = short.ctx.device
+    first = torch.tensor([L - n for L in long_lens], dtype=torch.int32, device=dev)
+    for layer in (0, 1):
+        rows = {}
+        for kind in "kv":
+            full = torch.stack([synth.layer_cache(w, layer, kind, b, width=w.D)[long_lens[b] - n: long_lens[b]]
+                                for b in range(w.batch)])                      # [B][n][D]
+            if not w.is_anchor(layer) and not window:
+                full[:, :, w.m:] = 777.0                                         # must never reach the cache
+            rows[kind] = full.to(dev)
+        short.ctx.append_kv_chunk(layer, rows["k"], rows["v"], first)
+    torch.cuda.synchronize()
+    assert short.ctx.device_status() == binding.ECHOKV_OK
+    short.seq_lens = ref.seq_lens.clone()
+    for layer in (0, 1):
+        for b, L in enumerate(long_lens):
+            for t in (0, L - n - 1, L - n, L - 75, L - 1):
+                page, r = int(ref.table[b, t // w.page_tokens]), t % w.page_tokens
+                for pa, pb in ((ref.ctx.k_pools, short.ctx.k_pools), (ref.ctx.v_pools, short.ctx.v_pools)):
+                    assert torch.equal(pa[layer][page, r], pb[layer][page, r]), (layer, b, t)
+    if window:
+        n_sink, n_window = window
+        for b, L in enumerate(long_lens):
+            live = [t for t in range(L) if t < n_sink or t >= L - n_window]
+            slots = [t if t < n_sink else n_sink + t % n_window for t in live]
+            assert torch.equal(ref.ctx.k_side[1][b, slots], short.ctx.k_side[1][b, slots])
+            assert torch.equal(ref.ctx.v_side[1][b, slots], short.ctx.v_side[1][b, slots])
+    np.testing.assert_array_equal(short.run(1), ref.run(1))
+    np.testing.assert_array_equal(short.run(0), ref.run(0))
+    ref.close()
+    short.close()
