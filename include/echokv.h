@@ -191,6 +191,10 @@ int echokv_decode_attention(echokv_ctx* ctx, int layer, const void* q, float* ou
  * bf16, head_dim 128 and head-aligned m only; not with sink / window tokens or save_k: EUNSUPPORTED.
  * A sequence with fewer than n_q cached tokens, or an unusable slot / length: zeros and the device status.
  * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (batch, scratch too small), ENOWEIGHTS, ENOTABLE, ECUDA. */
+/* Which attention kernel the prefill-shaped call runs over the rebuilt rows: 0 = mma.sync kernel, 1 = tcgen05 kernel
+ * (accumulators in tensor memory; the default).  Meant for tests that check both against the oracle. */
+int echokv_prefill_path(const echokv_ctx* ctx);
+int echokv_set_prefill_path(echokv_ctx* ctx, int path);
 int echokv_prefill_scratch_bytes(const echokv_config* cfg, uint64_t* out);
 int echokv_prefill_attention(echokv_ctx* ctx, int layer, const void* q, float* out, int n_q,
                              const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,

@@ -57,6 +57,8 @@ EXPORTS = {
                                           C.c_void_p, C.c_int, C.c_void_p]),
     "echokv_full_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_int, C.c_void_p]),
+    "echokv_prefill_path": (C.c_int, [C.c_void_p]),
+    "echokv_set_prefill_path": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_prefill_scratch_bytes": (C.c_int, [C.POINTER(echokv_config), C.POINTER(C.c_uint64)]),
     "echokv_prefill_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                            C.c_void_p, C.c_int, C.c_void_p, C.c_uint64, C.c_void_p]),
@@ -243,6 +245,9 @@ class Context:
                                               self.prefill_scratch.numel(), _stream_handle(stream)),
                "echokv_prefill_attention")
         return out
+
+    def set_prefill_path(self, path: int) -> None:
+        _check(lib().echokv_set_prefill_path(self.handle, path), "echokv_set_prefill_path")
 
     def full_attention(self, layer: int, q, seq_lens, out=None, seq_slots=None, stream=None):
         out = self._out(q) if out is None else out

@@ -112,6 +112,7 @@ struct echokv_ctx {
   AbsorbMaps amaps;
   bool stored_capable = false;   // shape served by the TMA + mma.sync stored-head kernel
   int stored_path = 0;           // 0 = CUDA-core kernel, 1 = TMA + mma.sync kernel
+  int prefill_path = 1;          // attention kernel of the prefill-shaped call: 0 = mma.sync, 1 = tcgen05
   int64_t launches = 0;
   float scale = 0.f;
   std::vector<int32_t> pos_scratch;
@@ -530,6 +531,14 @@ int echokv_set_decode_mode(echokv_ctx* c, int mode) {
   return ECHOKV_OK;
 }
 
+int echokv_prefill_path(const echokv_ctx* c) { return c ? c->prefill_path : 0; }
+
+int echokv_set_prefill_path(echokv_ctx* c, int path) {
+  if (!c || (path != 0 && path != 1)) return ECHOKV_EINVAL;
+  c->prefill_path = path;
+  return ECHOKV_OK;
+}
+
 int echokv_stored_path(const echokv_ctx* c) { return c ? c->stored_path : 0; }
 
 int echokv_set_stored_path(echokv_ctx* c, int path) {
@@ -637,7 +646,8 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
       return ECHOKV_ECUDA;
     c->launches += 2;
   }
-  if (launch_prefill_attn(a, k_rows, v_rows, c->d.capacity, c->d.D, n_q, out, s) != cudaSuccess) return ECHOKV_ECUDA;
+  if (launch_prefill_attn(a, k_rows, v_rows, c->d.capacity, c->d.D, n_q, out, s, c->prefill_path) != cudaSuccess)
+    return ECHOKV_ECUDA;
   c->launches += 1;
   return ECHOKV_OK;
 }

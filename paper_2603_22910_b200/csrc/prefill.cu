@@ -269,6 +269,260 @@ __global__ void __launch_bounds__(128) prefill_attn_kernel(const __nv_bfloat16* 
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// 3b. the same on the 5th-generation tensor cores (tcgen05, accumulators in tensor memory)
+// ---------------------------------------------------------------------------------------------
+// One CTA of 256 threads per (128 query rows, query head, sequence); keys in tiles of 128.
+//   S   [128 rows x 128 keys]  = Q K^T        A = Q tile, B = key tile, both K-major       -> TMEM columns 0..127
+//   O^T [128 dims x 128 rows]  = V^T P^T      A = value tile used M-major (it is stored [key][dim]), B = P K-major
+//                                              -> TMEM columns 128..255, fresh for every key tile
+// Two threads share S row r (query row r), 64 keys each: mask, running max / sum, probabilities as bf16 into a
+// shared-memory tile in the MMA's swizzled layout.  The same two share O^T row d (output dim d), 64 query rows each:
+// o[row] = o[row] * alpha[row] + O^T tile, in registers, so nothing is rescaled in tensor memory.  Key / value tiles are double-buffered with cp.async; the
+// waits on the two MMA-completion barriers are bounded.
+constexpr int kTcTile = 128;                     // query rows per CTA, keys per tile
+constexpr int kTcChunkBytes = kTcTile * 128;     // [128 rows x 64 dims] bf16, 128-byte swizzle
+constexpr int kTcTileBytes = 2 * kTcChunkBytes;  // 128 dims
+constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescO = kIdescS | (1u << 15);                  // A operand M-major
+
+struct PfTcTail {
+  float alpha[kTcTile];
+  float mx[2][kTcTile];          // partial row maxima of the two column halves
+  float l[2][kTcTile];
+  unsigned long long bar_s, bar_o;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint64_t pf_desc_kmajor(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// M-major operand made of [K rows][64 M-elements] tiles in the 128-byte swizzle: 8-row groups along K are 1024 bytes
+// apart, successive 64-element blocks along M are block_bytes apart
+__device__ __forceinline__ uint64_t pf_desc_mmajor(uint32_t smem_addr, uint32_t block_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
+  d |= static_cast<uint64_t>(block_bytes >> 4) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// byte offset of 16-byte piece `piece` (0..15) of row `row` inside a [128 rows x 128 dims] swizzled tile
+__device__ __forceinline__ uint32_t pf_sw(int row, int piece) {
+  return (uint32_t)((piece >> 3) * kTcChunkBytes + row * 128 + (((piece & 7) ^ (row & 7)) << 4));
+}
+
+// 256 threads: thread (lane row r = tid % 128, half = tid / 128) owns columns [64 half, 64 half + 64) of TMEM lane r
+// in both accumulators: half of S row r (keys) and half of O^T row r (query rows of output dim r).  Two warps per
+// scheduler instead of one hide the tensor-memory and special-function latencies of the epilogue.
+__global__ void __launch_bounds__(256, 1)
+prefill_attn_tc_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ ks,
+                       const __nv_bfloat16* __restrict__ vs, float* __restrict__ out, int n_q, int n_q_heads,
+                       int n_kv_heads, int kv_tokens, int kv_width, const int32_t* __restrict__ slots,
+                       const int32_t* __restrict__ lens, int max_batch, int capacity, float scale_log2e,
+                       int32_t* status) {
+  extern __shared__ unsigned char pf_tc_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_tc_raw) + 1023) &
+                                                         ~static_cast<uintptr_t>(1023));
+  // Q | K buffer 0, 1 | V buffer 0, 1 | P
+  const uint32_t q_addr = smem_u32(smem), k_addr = q_addr + kTcTileBytes, v_addr = k_addr + 2 * kTcTileBytes,
+                 p_addr = v_addr + 2 * kTcTileBytes;
+  unsigned char* p_tile = smem + 5 * kTcTileBytes;
+  PfTcTail& t = *reinterpret_cast<PfTcTail*>(smem + 6 * kTcTileBytes);
+  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int r = tid & 127, half = tid >> 7;                 // TMEM lane / row, and which 64 columns
+  const int kvh = h / (n_q_heads / n_kv_heads);
+  const int slot = slots ? slots[b] : b;
+  const int len = lens[b];
+  const int i_row = qt * kTcTile + r;                       // the query row of S row r
+  if (slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
+    if (tid == 0 && qt == 0 && h == 0) report(status, slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
+    for (int c = half * 64; c < half * 64 + 64; ++c) {
+      const int i = qt * kTcTile + c;
+      if (i < n_q) out[(((size_t)b * n_q + i) * n_q_heads + h) * 128 + r] = 0.f;
+    }
+    return;
+  }
+  volatile int* abort_flag = &t.abort_flag;
+  if (tid == 0) {
+    t.abort_flag = 0;
+    mbar_init(smem_u32(&t.bar_s), 1);
+    mbar_init(smem_u32(&t.bar_o), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&t.tmem_base), 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = t.tmem_base;
+  const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + half * 64;
+
+  const int last_row = min(n_q, (qt + 1) * kTcTile) - 1;
+  const int kv_end = len - n_q + last_row + 1;              // keys this CTA's rows may see
+  const int n_tiles = (kv_end + kTcTile - 1) / kTcTile;
+  const __nv_bfloat16* k_seq = ks + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
+  const __nv_bfloat16* v_seq = vs + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
+  auto stage = [&](int tile, int buf) {          // 128 key rows and 128 value rows, zero-filled past kv_end
+    const int kv0 = tile * kTcTile;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int idx = tid + 256 * i, row = idx >> 4, piece = idx & 15;
+      const bool in = kv0 + row < kv_end;
+      const size_t src = (size_t)(in ? kv0 + row : 0) * kv_width + piece * 8;
+      const uint32_t off = buf * kTcTileBytes + pf_sw(row, piece);
+      cp_async16(k_addr + off, k_seq + src, in ? 16u : 0u);
+      cp_async16(v_addr + off, v_seq + src, in ? 16u : 0u);
+    }
+  };
+  // the query rows (rows past n_q are zero), with the first key / value tile
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int idx = tid + 256 * i, row = idx >> 4, piece = idx & 15;
+    const int iq = qt * kTcTile + row;
+    const bool in = iq < n_q;
+    cp_async16(q_addr + pf_sw(row, piece), q + (((size_t)b * n_q + (in ? iq : 0)) * n_q_heads + h) * 128 + piece * 8,
+               in ? 16u : 0u);
+  }
+  stage(0, 0);
+  cp_async_commit();
+
+  const int pos = len - n_q + i_row;                        // position of query row r
+  const bool row_ok = i_row < n_q;
+  float m_run = -INFINITY, l_run = 0.f;                     // (m_run is the same in both halves; l_run is this half's)
+  float o[64];                                              // output dim r, query rows 64 half .. 64 half + 63
+#pragma unroll
+  for (int c = 0; c < 64; ++c) o[c] = 0.f;
+  bool alive = true;
+
+  for (int tile = 0; tile < n_tiles; ++tile) {
+    const int buf = tile & 1;
+    if (tile + 1 < n_tiles) {
+      stage(tile + 1, buf ^ 1);
+      cp_async_commit();
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    fence_proxy_async_smem();        // the copied tiles, before the tensor cores read them
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        const uint64_t a = pf_desc_kmajor(q_addr + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
+        const uint64_t bd = pf_desc_kmajor(k_addr + buf * kTcTileBytes + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
+        tc_mma_bf16(tmem, a, bd, kIdescS, kk > 0 ? 1u : 0u);
+      }
+      tc_commit(smem_u32(&t.bar_s));
+    }
+    if (!__syncthreads_and(mbar_wait(smem_u32(&t.bar_s), tile & 1, abort_flag, status) ? 1 : 0)) { alive = false; break; }
+    tc_fence_after();
+
+    // ---- this thread's 64 keys of S row r: partial maximum, exchanged with the other half
+    const int key0 = tile * kTcTile + half * 64;
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c2 = 0; c2 < 2; ++c2) {
+      float v[32];
+      tmem_ld32(lane_addr + c2 * 32, v);
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (row_ok && key0 + c2 * 32 + j <= pos) mx = fmaxf(mx, v[j]);
+    }
+    t.mx[half][r] = mx * scale_log2e;       // (scale > 0: the maximum commutes with it; -inf stays -inf)
+    __syncthreads();
+    const float m_new = fmaxf(m_run, fmaxf(t.mx[0][r], t.mx[1][r]));
+    const float alpha = m_new == -INFINITY ? 1.f : exp2f(m_run - m_new);
+    m_run = m_new;
+    float psum = 0.f;
+#pragma unroll
+    for (int c2 = 0; c2 < 2; ++c2) {
+      float v[32];
+      tmem_ld32(lane_addr + c2 * 32, v);
+      uint32_t packed[16];
+#pragma unroll
+      for (int j = 0; j < 32; j += 2) {
+        const float p0 = (row_ok && key0 + c2 * 32 + j <= pos) ? exp2f(v[j] * scale_log2e - m_new) : 0.f;
+        const float p1 = (row_ok && key0 + c2 * 32 + j + 1 <= pos) ? exp2f(v[j + 1] * scale_log2e - m_new) : 0.f;
+        psum += p0 + p1;
+        packed[j >> 1] = pack2(p0, p1);
+      }
+#pragma unroll
+      for (int pc = 0; pc < 4; ++pc)    // four 16-byte pieces of 8 keys
+        *reinterpret_cast<uint4*>(p_tile + pf_sw(r, half * 8 + c2 * 4 + pc)) =
+            make_uint4(packed[4 * pc], packed[4 * pc + 1], packed[4 * pc + 2], packed[4 * pc + 3]);
+    }
+    l_run = l_run * alpha + psum;
+    if (half == 0) t.alpha[r] = alpha;
+    tc_fence_before();
+    fence_proxy_async_smem();        // the probabilities, before the tensor cores read them
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      const uint64_t a0 = pf_desc_mmajor(v_addr + buf * kTcTileBytes, kTcChunkBytes);
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {   // 16 keys per MMA: 2048 bytes of value rows, 32 bytes along P's keys
+        const uint64_t bd = pf_desc_kmajor(p_addr + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
+        tc_mma_bf16(tmem + 128, a0 + 128 * kk, bd, kIdescO, kk > 0 ? 1u : 0u);
+      }
+      tc_commit(smem_u32(&t.bar_o));
+    }
+    if (!__syncthreads_and(mbar_wait(smem_u32(&t.bar_o), tile & 1, abort_flag, status) ? 1 : 0)) { alive = false; break; }
+    tc_fence_after();
+
+    // ---- O^T row r (output dim r), this thread's 64 query rows: fold this tile in
+#pragma unroll
+    for (int c2 = 0; c2 < 2; ++c2) {
+      float v[32];
+      tmem_ld32(lane_addr + 128 + c2 * 32, v);
+      const float4* al = reinterpret_cast<const float4*>(&t.alpha[half * 64 + c2 * 32]);
+#pragma unroll
+      for (int j4 = 0; j4 < 8; ++j4) {
+        const float4 a4 = al[j4];
+        o[c2 * 32 + 4 * j4 + 0] = fmaf(o[c2 * 32 + 4 * j4 + 0], a4.x, v[4 * j4 + 0]);
+        o[c2 * 32 + 4 * j4 + 1] = fmaf(o[c2 * 32 + 4 * j4 + 1], a4.y, v[4 * j4 + 1]);
+        o[c2 * 32 + 4 * j4 + 2] = fmaf(o[c2 * 32 + 4 * j4 + 2], a4.z, v[4 * j4 + 2]);
+        o[c2 * 32 + 4 * j4 + 3] = fmaf(o[c2 * 32 + 4 * j4 + 3], a4.w, v[4 * j4 + 3]);
+      }
+    }
+    tc_fence_before();
+    __syncthreads();                 // S, P and alpha are free for the next tile
+  }
+
+  if (alive) {
+    t.l[half][r] = l_run;
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < 64; ++c) {
+      const int row = half * 64 + c, i = qt * kTcTile + row;
+      const float l = t.l[0][row] + t.l[1][row];
+      if (i < n_q) out[(((size_t)b * n_q + i) * n_q_heads + h) * 128 + r] = l > 0.f ? o[c] / l : 0.f;
+    }
+  } else {
+    cp_async_wait<0>();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 256);
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, __nv_bfloat16* out, int out_tokens,
@@ -282,7 +536,20 @@ cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, _
 }
 
 cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
-                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream) {
+                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream, int path) {
+  if (path == 1) {
+    dim3 grid((n_q + kTcTile - 1) / kTcTile, a.n_q_heads, a.batch);
+    const size_t smem = 1024 + 6 * (size_t)kTcTileBytes + sizeof(PfTcTail);
+    const cudaError_t e = cudaFuncSetAttribute(prefill_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)smem);
+    if (e != cudaSuccess) return e;
+    prefill_attn_tc_kernel<<<grid, 256, smem, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q), k_rows, v_rows, out,
+                                                        n_q, a.n_q_heads, a.n_kv_heads, kv_tokens, kv_width, a.slots,
+                                                        a.lens, a.geom.max_batch,
+                                                        a.geom.max_pages_per_seq * a.geom.page_tokens, a.scale_log2e,
+                                                        a.status);
+    return cudaGetLastError();
+  }
   dim3 grid((n_q + kPfRows - 1) / kPfRows, a.n_q_heads, a.batch);
   const size_t smem = 4 * (size_t)kPfKeys * kPfRowBytes;
   cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -13,7 +13,8 @@ cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, _
 // Eq. 7 for n_q queries per sequence (a.q: [B][n_q][H_q][128] bf16), query i at position len - n_q + i attending the
 // keys up to its own, over k_rows / v_rows [B][kv_tokens][kv_width] bf16.  out: fp32 [B][n_q][H_q][128].
 // A sequence with fewer than n_q cached tokens gets zeros and the device status EBADLENGTH.
+// path: 0 = mma.sync kernel, 1 = tcgen05 kernel.
 cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
-                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream);
+                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream, int path);
 
 }  // namespace echokv

@@ -64,10 +64,13 @@ CASES = [
 
 
 @pytest.mark.parametrize("name,base,over,lens,n_q,biases,rope", CASES, ids=[c[0] for c in CASES])
-def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope):
+@pytest.mark.parametrize("path", [0, 1], ids=["mma_sync", "tcgen05"])
+def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope, path):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], biases=biases, rope=rope)
     ctx = case.ctx
+    assert binding.lib().echokv_prefill_path(ctx.handle) == 1
+    ctx.set_prefill_path(path)
     for layer in (1, 0):
         q = queries(w, n_q, layer)
         out = ctx.prefill_attention(layer, q.to(ctx.device), case.seq_lens)
