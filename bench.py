@@ -440,6 +440,11 @@ def run_prefill(args):
     if args.rope:
         ctx.set_rope(args.rope)
     st.rope = args.rope
+    if args.prefill_path is not None:
+        ctx.set_prefill_path(args.prefill_path)
+    attn_kernel = {0: "prefill_attn_kernel (mma.sync)", 1: "prefill_attn_tc_kernel (tcgen05)",
+                   2: "prefill_attn_ws_kernel (tcgen05, warp-specialised)"}[
+                       binding.lib().echokv_prefill_path(ctx.handle)]
     q = synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, 1, device=dev).to(torch.bfloat16)
     out = torch.empty(q.shape, dtype=torch.float32, device=dev)
     for _ in range(max(3, args.warmup)):
@@ -480,7 +485,7 @@ def run_prefill(args):
                      "unit": "TFLOP/s", "frac": recon_flops / (k_ms * 1e-3) / 1e12 / peak_tf, "traffic": None,
                      "kernel": "recon_pair_kernel (rows to memory), K pass + V pass", "kernel_ms": k_ms,
                      "share_of_step": k_ms / ms, "peak_source": "%s (cuBLAS bf16 GEMM, sustained)" % peaks_kind},
-        "attention": {"kernel": "prefill_attn_kernel (mma.sync) + gather_rows_kernel x 2", "ms": ms - k_ms,
+        "attention": {"kernel": attn_kernel + " + gather_rows_kernel x 2", "ms": ms - k_ms,
                       "tflops": attn_flops / ((ms - k_ms) * 1e-3) / 1e12},
         "parity_vs_oracle": {"rows": "last %d queries of sequence 0" % n_chk,
                              "max_abs": float(np.max(np.abs(got - ref))),
@@ -842,6 +847,8 @@ def main():
                     "read (the cache then holds un-rotated keys); 0 = none, as in the paper's configurations")
     ap.add_argument("--save-k", action="store_true", help="compressed layers keep their keys whole, only the values "
                     "are predicted (the paper's \"save K\" ablation); needs --decode-mode absorbed")
+    ap.add_argument("--prefill-path", type=int, default=None, choices=[0, 1, 2],
+                    help="attention kernel of the prefill-shaped call (default: the library's)")
     ap.add_argument("--prefill-queries", type=int, default=0, help="time the prefill-shaped call instead: this many "
                     "causal queries per sequence on the compressed layer (an extra measurement, its own JSON line)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

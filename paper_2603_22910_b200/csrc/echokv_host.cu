@@ -534,7 +534,7 @@ int echokv_set_decode_mode(echokv_ctx* c, int mode) {
 int echokv_prefill_path(const echokv_ctx* c) { return c ? c->prefill_path : 0; }
 
 int echokv_set_prefill_path(echokv_ctx* c, int path) {
-  if (!c || (path != 0 && path != 1)) return ECHOKV_EINVAL;
+  if (!c || path < 0 || path > 2) return ECHOKV_EINVAL;
   c->prefill_path = path;
   return ECHOKV_OK;
 }
@@ -624,10 +624,10 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
   __nv_bfloat16* v_rows = k_rows + rows_bytes / 2;
   const int width = compressed ? c->d.m : c->d.D;
   // stored dims as they are (keys rotated to their positions), then the predicted ones beside them
-  if (launch_gather_rows(a, L.k_pool, width, k_rows, c->d.capacity, c->d.D, true, s) != cudaSuccess ||
-      launch_gather_rows(a, L.v_pool, width, v_rows, c->d.capacity, c->d.D, false, s) != cudaSuccess)
+  if (launch_gather_rows(a, L.k_pool, width, k_rows, c->d.capacity, c->d.D, true, 0, s) != cudaSuccess ||
+      launch_gather_rows(a, L.v_pool, width, v_rows, c->d.capacity, c->d.D, false, 128, s) != cudaSuccess)
     return ECHOKV_ECUDA;
-  c->launches += width > 0 ? 2 : 0;
+  c->launches += width > 0 ? 2 : 1;
   if (compressed) {
     const Layer& A = c->layers[layer - layer % c->cfg.group_size];
     ReconArgs ra;

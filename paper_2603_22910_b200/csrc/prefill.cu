@@ -14,6 +14,7 @@
 #include "prefill.h"
 
 #include "ptx_sm100.cuh"
+#include "recon_tc.h"
 
 namespace echokv {
 
@@ -26,11 +27,23 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
                                                           __nv_bfloat16* __restrict__ out, int out_tokens,
                                                           int out_width, const int32_t* __restrict__ slots,
                                                           const int32_t* __restrict__ lens, PageGeom g, RopeTable rope,
-                                                          int32_t* status) {
+                                                          int zero_tail, int32_t* status) {
   const int b = blockIdx.y, t0 = blockIdx.x * 32;
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
   if (slot < 0 || slot >= g.max_batch || len < 1 || len > g.max_pages_per_seq * g.page_tokens) return;
+  if (zero_tail > 0) {
+    // rows len .. (next multiple of zero_tail) - 1 become zeros over the whole row: a consumer that reads whole
+    // tiles of rows multiplies them by zero weights, which garbage (a NaN pattern) would not survive
+    const int end = min(out_tokens, (len + zero_tail - 1) / zero_tail * zero_tail);
+    const int pieces = out_width / 8;
+    for (int it = threadIdx.x; it < 32 * pieces; it += blockDim.x) {
+      const int t = t0 + it / pieces;
+      if (t >= len && t < end)
+        *reinterpret_cast<uint4*>(out + ((size_t)b * out_tokens + t) * (size_t)out_width + (it % pieces) * 8) =
+            make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
   if (t0 >= len) return;
   const int n_heads = width / 128;
   // item = (token of the tile, head, 8-dim piece c of the head's first half, with its partner piece 64 dims on)
@@ -523,20 +536,354 @@ prefill_attn_tc_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// 3c. tcgen05 again, with the steps given to different warps so that they overlap
+// ---------------------------------------------------------------------------------------------
+// One CTA per (256 query rows, query head, sequence): two query tiles X = 0, 1 of 128 rows share every key / value tile,
+// and while the tensor cores work for one of them the other one's softmax runs.
+//   warps 0-3 / 4-7  softmax of tile 0 / 1: thread = one query row.  Reads its S row (128 keys) from tensor memory,
+//                    keeps a reference maximum that only moves when the row's maximum has grown by more than 2^8
+//                    (then it rescales its O row in tensor memory itself), writes the probabilities as bf16 over the
+//                    first 64 columns of S, and at the end normalises and writes its O row.
+//   warp 8           one thread issues every MMA:  S_X = Q_X K^T (A, B from shared memory, K-major) and
+//                    O_X += P_X V (A = P_X from tensor memory, B = the value tile as stored [key][dim]: N-major).
+//   warp 9           one thread issues the TMA loads: Q once, then key tiles (3 stages) and value tiles (2 stages).
+// Tensor memory: S_0 | S_1 | O_0 | O_1, 128 columns each.  MMAs of one thread run in the order issued, so S_X(t + 1),
+// issued right after O_X += P_X(t) V(t), overwrites P_X(t) only after it was read, and its completion tells the
+// softmax warps that O_X is at rest as well.  Every wait is bounded.
+constexpr int kWsKStages = 3, kWsVStages = 2;
+constexpr int kWsThreads = 320;
+constexpr uint32_t kIdescPV = kIdescS | (1u << 16);                 // B operand N-major
+constexpr float kWsGrowLog2 = 8.f;
+
+struct PfWsTail {
+  unsigned long long q_full;
+  unsigned long long k_full[kWsKStages], k_empty[kWsKStages];
+  unsigned long long v_full[kWsVStages], v_empty[kWsVStages];
+  unsigned long long s_full[2], p_ready[2], o_done[2], drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(kWsThreads, 1)
+prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, float* __restrict__ out, int n_q, int n_q_heads,
+                       int n_kv_heads, const int32_t* __restrict__ slots, const int32_t* __restrict__ lens,
+                       int max_batch, int capacity, float scale_log2e, int32_t* status) {
+  extern __shared__ unsigned char pf_ws_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_ws_raw) + 1023) &
+                                                         ~static_cast<uintptr_t>(1023));
+  // Q tile 0, 1 | K stages | V stages
+  const uint32_t q_addr = smem_u32(smem), k_addr = q_addr + 2 * kTcTileBytes,
+                 v_addr = k_addr + kWsKStages * kTcTileBytes;
+  PfWsTail& t = *reinterpret_cast<PfWsTail*>(smem + (2 + kWsKStages + kWsVStages) * kTcTileBytes);
+  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kvh = h / (n_q_heads / n_kv_heads);
+  const int slot = slots ? slots[b] : b;
+  const int len = lens[b];
+  if (slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
+    if (tid == 0 && qt == 0 && h == 0) report(status, slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
+    if (tid < 256) {
+      const int i = qt * 2 * kTcTile + tid;
+      if (i < n_q) {
+        float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + i) * n_q_heads + h) * 128);
+        for (int c = 0; c < 32; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    return;
+  }
+  volatile int* abort_flag = &t.abort_flag;
+  if (tid == 0) {
+    t.abort_flag = 0;
+    mbar_init(smem_u32(&t.q_full), 1);
+    for (int s = 0; s < kWsKStages; ++s) {
+      mbar_init(smem_u32(&t.k_full[s]), 1);
+      mbar_init(smem_u32(&t.k_empty[s]), 1);
+    }
+    for (int s = 0; s < kWsVStages; ++s) {
+      mbar_init(smem_u32(&t.v_full[s]), 1);
+      mbar_init(smem_u32(&t.v_empty[s]), 1);
+    }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(smem_u32(&t.s_full[x]), 1);
+      mbar_init(smem_u32(&t.p_ready[x]), 128);
+      mbar_init(smem_u32(&t.o_done[x]), 1);
+    }
+    mbar_init(smem_u32(&t.drain), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (warp == 8) {
+    tmem_alloc(smem_u32(&t.tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = t.tmem_base;
+
+  const int row0 = qt * 2 * kTcTile;                        // first query row of the CTA
+  const int last_row = min(n_q, row0 + 2 * kTcTile) - 1;
+  const int kv_end = len - n_q + last_row + 1;              // keys this CTA's rows may see
+  const int n_tiles = (kv_end + kTcTile - 1) / kTcTile;
+
+  if (warp == 9) {
+    // =============================== TMA producer ===============================================
+    if (lane == 0) {
+      const uint32_t qb = smem_u32(&t.q_full);
+      mbar_arrive_expect_tx(qb, 2 * kTcTileBytes);
+      tma_load_5d(q_addr, &tm_q, 0, row0, 0, h, b, qb);
+      tma_load_5d(q_addr + kTcTileBytes, &tm_q, 0, row0 + kTcTile, 0, h, b, qb);
+      bool alive = true;
+      int k_issued = 0, v_issued = 0;
+      for (int tile = 0; tile < n_tiles && alive; ++tile) {
+        {
+          const int s = tile % kWsKStages, use = tile / kWsKStages;
+          if (!mbar_wait(smem_u32(&t.k_empty[s]), (use & 1) ^ 1, abort_flag, status)) { alive = false; break; }
+          const uint32_t full = smem_u32(&t.k_full[s]);
+          mbar_arrive_expect_tx(full, kTcTileBytes);
+          tma_load_4d(k_addr + s * kTcTileBytes, &tm_k, 0, tile * kTcTile, 2 * kvh, b, full);
+          k_issued = tile + 1;
+        }
+        {
+          const int s = tile % kWsVStages, use = tile / kWsVStages;
+          if (!mbar_wait(smem_u32(&t.v_empty[s]), (use & 1) ^ 1, abort_flag, status)) { alive = false; break; }
+          const uint32_t full = smem_u32(&t.v_full[s]);
+          mbar_arrive_expect_tx(full, kTcTileBytes);
+          tma_load_4d(v_addr + s * kTcTileBytes, &tm_v, 0, tile * kTcTile, 2 * kvh, b, full);
+          v_issued = tile + 1;
+        }
+      }
+      if (!alive) {
+        // let every copy that was started land before the CTA leaves
+        mbar_drain(qb, 0);
+        for (int i = max(0, k_issued - kWsKStages); i < k_issued; ++i)
+          mbar_drain(smem_u32(&t.k_full[i % kWsKStages]), (i / kWsKStages) & 1);
+        for (int i = max(0, v_issued - kWsVStages); i < v_issued; ++i)
+          mbar_drain(smem_u32(&t.v_full[i % kWsVStages]), (i / kWsVStages) & 1);
+      }
+    }
+  } else if (warp == 8) {
+    // =============================== MMA issuer ================================================
+    if (lane == 0) {
+      bool alive = mbar_wait(smem_u32(&t.q_full), 0, abort_flag, status);
+      auto issue_s = [&](int x, int tile) {          // S_x = Q_x K(tile)^T
+        const int s = tile % kWsKStages;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t a = pf_desc_kmajor(q_addr + x * kTcTileBytes + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
+          const uint64_t bd = pf_desc_kmajor(k_addr + s * kTcTileBytes + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
+          tc_mma_bf16(tmem + x * 128, a, bd, kIdescS, kk > 0 ? 1u : 0u);
+        }
+        tc_commit(smem_u32(&t.s_full[x]));
+        if (x == 1) tc_commit(smem_u32(&t.k_empty[s]));
+      };
+      if (alive) alive = mbar_wait(smem_u32(&t.k_full[0]), 0, abort_flag, status);
+      if (alive) {
+        tc_fence_after();
+        issue_s(0, 0);
+        issue_s(1, 0);
+      }
+      for (int tile = 0; tile < n_tiles && alive; ++tile) {
+        const int sv = tile % kWsVStages;
+        if (!mbar_wait(smem_u32(&t.v_full[sv]), (tile / kWsVStages) & 1, abort_flag, status)) { alive = false; break; }
+        const uint64_t b0 = pf_desc_mmajor(v_addr + sv * kTcTileBytes, kTcChunkBytes);
+        for (int x = 0; x < 2 && alive; ++x) {
+          if (!mbar_wait(smem_u32(&t.p_ready[x]), tile & 1, abort_flag, status)) { alive = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)     // 16 keys per MMA: 8 columns of packed probabilities, 2048 bytes of value rows
+            tc_mma_bf16_tmem_a(tmem + 256 + x * 128, tmem + x * 128 + 8 * kk, b0 + 128 * kk, kIdescPV,
+                               (tile > 0 || kk > 0) ? 1u : 0u);
+          if (tile + 1 == n_tiles) tc_commit(smem_u32(&t.o_done[x]));
+          if (x == 1) tc_commit(smem_u32(&t.v_empty[sv]));
+          if (tile + 1 < n_tiles) {
+            if (x == 0) {
+              const int sk = (tile + 1) % kWsKStages;
+              if (!mbar_wait(smem_u32(&t.k_full[sk]), ((tile + 1) / kWsKStages) & 1, abort_flag, status)) { alive = false; break; }
+              tc_fence_after();
+            }
+            issue_s(x, tile + 1);
+          }
+        }
+      }
+      if (!alive) {
+        // every MMA issued so far retires before the tensor memory is given back
+        tc_commit(smem_u32(&t.drain));
+        mbar_drain(smem_u32(&t.drain), 0);
+      }
+    }
+  } else {
+    // =============================== softmax, one thread per query row ===========================
+    const int x = warp >> 2, wl = tid & 127;
+    const int i_row = row0 + x * kTcTile + wl;
+    const bool row_ok = i_row < n_q;
+    const int pos = len - n_q + i_row;                      // position of this query row
+    const uint32_t lane_base = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const uint32_t s_addr = lane_base + x * 128, o_addr = lane_base + 256 + x * 128;
+    float m_ref = -INFINITY, l_run = 0.f;
+    bool alive = true;
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      if (!mbar_wait(smem_u32(&t.s_full[x]), tile & 1, abort_flag, status)) { alive = false; break; }
+      tc_fence_after();
+      uint32_t sr[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32_issue(s_addr + 32 * c, sr[c]);
+      tmem_ld_wait();
+      // keys of this tile the row sees: the first n_vis
+      const int n_vis = row_ok ? max(0, min(kTcTile, pos - tile * kTcTile + 1)) : 0;
+      float mx = -INFINITY;
+      if (n_vis == kTcTile) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(sr[c][j]));
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (32 * c + j < n_vis) mx = fmaxf(mx, __uint_as_float(sr[c][j]));
+      }
+      mx *= scale_log2e;                     // (scale > 0: the maximum commutes with it; -inf stays -inf)
+      const bool grow = mx > m_ref + kWsGrowLog2;
+      float alpha = 1.f;
+      if (grow) {
+        alpha = ex2_approx(m_ref - mx);      // 0 on the first tile
+        m_ref = mx;
+        l_run *= alpha;
+      }
+      if (tile > 0 && __any_sync(0xffffffffu, grow)) {
+        // O_x is at rest (the MMA that wrote S came after every earlier one): rescale this thread's row
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t orow[32];
+          tmem_ld32_issue(o_addr + 32 * c, orow);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * alpha);
+          tmem_st32(o_addr + 32 * c, orow);
+        }
+      }
+      float psum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        // 32 keys -> 16 columns of packed bf16 pairs; sr[c] is dead afterwards, so the pairs overwrite its first half
+        if (n_vis == kTcTile) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c][j]), scale_log2e, -m_ref));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c][j + 1]), scale_log2e, -m_ref));
+            psum += p0 + p1;
+            sr[c][j >> 1] = pack2(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = 32 * c + j < n_vis ? ex2_approx(fmaf(__uint_as_float(sr[c][j]), scale_log2e, -m_ref)) : 0.f;
+            const float p1 = 32 * c + j + 1 < n_vis ? ex2_approx(fmaf(__uint_as_float(sr[c][j + 1]), scale_log2e, -m_ref)) : 0.f;
+            psum += p0 + p1;
+            sr[c][j >> 1] = pack2(p0, p1);
+          }
+        }
+      }
+      l_run += psum;
+      {
+        uint32_t pk[32];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          pk[j] = sr[0][j];
+          pk[16 + j] = sr[1][j];
+        }
+        tmem_st32(s_addr, pk);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          pk[j] = sr[2][j];
+          pk[16 + j] = sr[3][j];
+        }
+        tmem_st32(s_addr + 32, pk);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&t.p_ready[x]));
+    }
+    if (alive && mbar_wait(smem_u32(&t.o_done[x]), 0, abort_flag, status)) {
+      tc_fence_after();
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + (row_ok ? i_row : 0)) * n_q_heads + h) * 128);
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(o_addr + 32 * c, v);
+        if (row_ok) {
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4)
+            dst[8 * c + j4] = make_float4(v[4 * j4] * inv, v[4 * j4 + 1] * inv, v[4 * j4 + 2] * inv, v[4 * j4 + 3] * inv);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, __nv_bfloat16* out, int out_tokens,
-                               int out_width, bool rotate, cudaStream_t stream) {
-  if (width == 0) return cudaSuccess;
-  if (width % 128 != 0) return cudaErrorInvalidValue;
+                               int out_width, bool rotate, int zero_tail, cudaStream_t stream) {
+  if (width == 0 && zero_tail == 0) return cudaSuccess;
+  if (width % 128 != 0 || out_width % 8 != 0) return cudaErrorInvalidValue;
   dim3 grid((out_tokens + 31) / 32, a.batch);
   gather_rows_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(pool), width, out, out_tokens,
-                                               out_width, a.slots, a.lens, a.geom, rotate ? a.rope : RopeTable(), a.status);
+                                               out_width, a.slots, a.lens, a.geom, rotate ? a.rope : RopeTable(), zero_tail,
+                                               a.status);
   return cudaGetLastError();
 }
 
 cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
                                 int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream, int path) {
+  if (path == 2) {
+    if (kv_width % 64 != 0 || reinterpret_cast<uintptr_t>(a.q) % 16 != 0) return cudaErrorInvalidValue;
+    CUtensorMap tm_q, tm_k, tm_v;
+    {
+      // q [B][n_q][H_q][128] seen as [B][H_q][2 chunks][n_q][64]: a box is the two 64-dim chunks of 128 query rows
+      const uint64_t dims[5] = {64, (uint64_t)n_q, 2, (uint64_t)a.n_q_heads, (uint64_t)a.batch};
+      const uint64_t strides[4] = {(uint64_t)a.n_q_heads * 256, 128, 256, (uint64_t)n_q * a.n_q_heads * 256};
+      const uint32_t box[5] = {64, (uint32_t)kTcTile, 2, 1, 1};
+      const cudaError_t e = encode_tiled_bf16(&tm_q, a.q, 5, dims, strides, box);
+      if (e != cudaSuccess) return e;
+    }
+    for (int kind = 0; kind < 2; ++kind) {
+      // rows [B][kv_tokens][kv_width] seen as [B][kv_width / 64][kv_tokens][64]: a box is one head (two chunks) of 128 rows
+      const uint64_t dims[4] = {64, (uint64_t)kv_tokens, (uint64_t)kv_width / 64, (uint64_t)a.batch};
+      const uint64_t strides[3] = {(uint64_t)kv_width * 2, 128, (uint64_t)kv_tokens * kv_width * 2};
+      const uint32_t box[4] = {64, (uint32_t)kTcTile, 2, 1};
+      const cudaError_t e = encode_tiled_bf16(kind ? &tm_v : &tm_k, kind ? v_rows : k_rows, 4, dims, strides, box);
+      if (e != cudaSuccess) return e;
+    }
+    dim3 grid((n_q + 2 * kTcTile - 1) / (2 * kTcTile), a.n_q_heads, a.batch);
+    const size_t smem = 1024 + (size_t)(2 + kWsKStages + kWsVStages) * kTcTileBytes + sizeof(PfWsTail);
+    const cudaError_t e = cudaFuncSetAttribute(prefill_attn_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)smem);
+    if (e != cudaSuccess) return e;
+    prefill_attn_ws_kernel<<<grid, kWsThreads, smem, stream>>>(tm_q, tm_k, tm_v, out, n_q, a.n_q_heads, a.n_kv_heads,
+                                                               a.slots, a.lens, a.geom.max_batch,
+                                                               a.geom.max_pages_per_seq * a.geom.page_tokens,
+                                                               a.scale_log2e, a.status);
+    return cudaGetLastError();
+  }
   if (path == 1) {
     dim3 grid((n_q + kTcTile - 1) / kTcTile, a.n_q_heads, a.batch);
     const size_t smem = 1024 + 6 * (size_t)kTcTileBytes + sizeof(PfTcTail);

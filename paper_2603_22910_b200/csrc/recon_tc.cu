@@ -594,6 +594,27 @@ cudaError_t encode_chunked_3d_map(CUtensorMap* map, const void* base, uint64_t r
   return encode_3d_chunks(map, base, rows, cols, box_rows, box_chunks, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
+// General form: bf16 tensor of `rank` dims (innermost first; strides in bytes for dims 1 .. rank-1), boxes in the
+// 128-byte swizzle (the innermost box extent is 64 elements), out-of-range elements read as zero.
+cudaError_t encode_tiled_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                              const uint64_t* strides, const uint32_t* box) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return cudaErrorNotSupported;
+  if (rank < 2 || rank > 5) return cudaErrorInvalidValue;
+  cuuint64_t d[5], st[4];
+  cuuint32_t bx[5], estr[5];
+  for (int i = 0; i < rank; ++i) {
+    d[i] = dims[i];
+    bx[i] = box[i];
+    estr[i] = 1;
+    if (i + 1 < rank) st[i] = strides[i];
+  }
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), d, st, bx, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows) {
   return encode_2d(map, pool, rows, width, box_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }

@@ -29,6 +29,11 @@ cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, u
 cudaError_t encode_chunked_3d_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int box_rows,
                                   int box_chunks);
 
+// General form: a bf16 tensor of `rank` dims (2..5, innermost first; strides in bytes for dims 1 .. rank-1), boxes in
+// the 128-byte swizzle (innermost box extent 64 elements); elements outside the tensor read as zero.
+cudaError_t encode_tiled_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                              const uint64_t* strides, const uint32_t* box);
+
 bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m);
 
 // k_width / v_width: row widths of the two pools (they differ where a layer keeps its keys whole); 0 = no pool

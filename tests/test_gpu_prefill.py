@@ -64,7 +64,7 @@ CASES = [
 
 
 @pytest.mark.parametrize("name,base,over,lens,n_q,biases,rope", CASES, ids=[c[0] for c in CASES])
-@pytest.mark.parametrize("path", [0, 1], ids=["mma_sync", "tcgen05"])
+@pytest.mark.parametrize("path", [0, 1, 2], ids=["mma_sync", "tcgen05", "tcgen05_ws"])
 def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope, path):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], biases=biases, rope=rope)
@@ -73,6 +73,9 @@ def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope, path)
     ctx.set_prefill_path(path)
     for layer in (1, 0):
         q = queries(w, n_q, layer)
+        # the scratch starts as NaN patterns: rows past a sequence's end must never reach a result
+        ctx.prefill_attention(layer, q.to(ctx.device), case.seq_lens)
+        ctx.prefill_scratch.fill_(0xFF)
         out = ctx.prefill_attention(layer, q.to(ctx.device), case.seq_lens)
         torch.cuda.synchronize()
         out = out.cpu().numpy().astype(np.float64)
