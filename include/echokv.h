@@ -192,7 +192,8 @@ int echokv_decode_attention(echokv_ctx* ctx, int layer, const void* q, float* ou
  * A sequence with fewer than n_q cached tokens, or an unusable slot / length: zeros and the device status.
  * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (batch, scratch too small), ENOWEIGHTS, ENOTABLE, ECUDA. */
 /* Which attention kernel the prefill-shaped call runs over the rebuilt rows: 0 = mma.sync kernel, 1 = tcgen05 kernel
- * (accumulators in tensor memory; the default).  Meant for tests that check both against the oracle. */
+ * (accumulators in tensor memory, one thread group doing every step in turn), 2 = warp-specialised tcgen05 kernel
+ * (softmax, MMA and TMA warps; the default).  Meant for tests that check all of them against the oracle. */
 int echokv_prefill_path(const echokv_ctx* ctx);
 int echokv_set_prefill_path(echokv_ctx* ctx, int path);
 int echokv_prefill_scratch_bytes(const echokv_config* cfg, uint64_t* out);

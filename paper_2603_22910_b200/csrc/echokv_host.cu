@@ -112,7 +112,7 @@ struct echokv_ctx {
   AbsorbMaps amaps;
   bool stored_capable = false;   // shape served by the TMA + mma.sync stored-head kernel
   int stored_path = 0;           // 0 = CUDA-core kernel, 1 = TMA + mma.sync kernel
-  int prefill_path = 1;          // attention kernel of the prefill-shaped call: 0 = mma.sync, 1 = tcgen05
+  int prefill_path = 2;          // attention kernel of the prefill-shaped call: 0 = mma.sync, 1 = tcgen05, 2 = tcgen05 warp-specialised
   int64_t launches = 0;
   float scale = 0.f;
   std::vector<int32_t> pos_scratch;

@@ -571,6 +571,57 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
+// two fp32 values in one 64-bit register, for the two-wide fp32 instructions of sm_100
+__device__ __forceinline__ uint64_t pack_u2(uint32_t lo, uint32_t hi) {
+  uint64_t v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(lo), "r"(hi));
+  return v;
+}
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi) { return pack_u2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void unpack_u2(uint64_t v, uint32_t& lo, uint32_t& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& lo, float& hi) {
+  uint32_t a, b;
+  unpack_u2(v, a, b);
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x for a pair, x <= ~8, without the special-function unit: n = round(x) by the add-a-large-constant trick,
+// f = x - n in [-0.5, 0.5], a cubic for 2^f (relative error 7.5e-5, far below the bf16 rounding that follows),
+// then n added into the exponent field.  x is clamped at -125 so that the exponent cannot wrap.
+constexpr int kPolyPer = 5, kPolyOf = 2;         // 2 of every 5 pairs
+__device__ __forceinline__ uint64_t ex2_poly_f2(uint64_t x2) {
+  float x0, x1;
+  unpack_f2(x2, x0, x1);
+  x2 = pack_f2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+  const float kMagic = 12582912.f;               // 1.5 * 2^23
+  const uint64_t t2 = add_f2(x2, pack_f2(kMagic, kMagic));
+  const uint64_t n2 = add_f2(t2, pack_f2(-kMagic, -kMagic));
+  const uint64_t f2 = fma_f2(n2, pack_f2(-1.f, -1.f), x2);
+  uint64_t p2 = fma_f2(pack_f2(0.0551716685295105f, 0.0551716685295105f), f2, pack_f2(0.2426111251115799f, 0.2426111251115799f));
+  p2 = fma_f2(p2, f2, pack_f2(0.6932609677314758f, 0.6932609677314758f));
+  p2 = fma_f2(p2, f2, pack_f2(0.9999280571937561f, 0.9999280571937561f));
+  uint32_t p0, p1, t0, t1;
+  unpack_u2(p2, p0, p1);
+  unpack_u2(t2, t0, t1);
+  return pack_u2(p0 + (t0 << 23), p1 + (t1 << 23));
+}
 
 __global__ void __launch_bounds__(kWsThreads, 1)
 prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -742,10 +793,20 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const int n_vis = row_ok ? max(0, min(kTcTile, pos - tile * kTcTile + 1)) : 0;
       float mx = -INFINITY;
       if (n_vis == kTcTile) {
+        // eight independent chains of three-input maxima instead of one chain of 128
+        float m8[8];
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(sr[c][j]));
+          for (int u = 0; u < 2; ++u) {
+            float a = fmaxf(__uint_as_float(sr[c][16 * u]), __uint_as_float(sr[c][16 * u + 1]));
+#pragma unroll
+            for (int j = 2; j < 16; j += 2)
+              a = max3(a, __uint_as_float(sr[c][16 * u + j]), __uint_as_float(sr[c][16 * u + j + 1]));
+            m8[2 * c + u] = a;
+          }
+        mx = fmaxf(max3(m8[0], m8[1], m8[2]), max3(m8[3], m8[4], m8[5]));
+        mx = max3(mx, m8[6], m8[7]);
       } else {
 #pragma unroll
         for (int c = 0; c < 4; ++c)
@@ -774,18 +835,39 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
       }
       float psum = 0.f;
+      if (n_vis == kTcTile) {
+        // Two scores per instruction where the pipe has a two-wide form (scale-and-shift, the polynomial, the row
+        // sum); kPolyOf of every kPolyPer pairs take 2^x from the polynomial instead of the special-function unit,
+        // whose 16 results per clock would otherwise set the pace of the whole kernel.
+        const uint64_t sc2 = pack_f2(scale_log2e, scale_log2e), nm2 = pack_f2(-m_ref, -m_ref);
+        uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        // 32 keys -> 16 columns of packed bf16 pairs; sr[c] is dead afterwards, so the pairs overwrite its first half
-        if (n_vis == kTcTile) {
+        for (int c = 0; c < 4; ++c) {
+          // 32 keys -> 16 columns of packed bf16 pairs; sr[c] is dead afterwards, so the pairs overwrite its first half
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
-            const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c][j]), scale_log2e, -m_ref));
-            const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c][j + 1]), scale_log2e, -m_ref));
-            psum += p0 + p1;
+            const uint64_t x2 = fma_f2(pack_u2(sr[c][j], sr[c][j + 1]), sc2, nm2);
+            uint64_t p2;
+            if (((j >> 1) % kPolyPer) < kPolyOf) {
+              p2 = ex2_poly_f2(x2);
+            } else {
+              float x0, x1;
+              unpack_f2(x2, x0, x1);
+              p2 = pack_f2(ex2_approx(x0), ex2_approx(x1));
+            }
+            sum2[(j >> 1) & 1] = add_f2(sum2[(j >> 1) & 1], p2);
+            float p0, p1;
+            unpack_f2(p2, p0, p1);
             sr[c][j >> 1] = pack2(p0, p1);
           }
-        } else {
+        }
+        float a0, a1, b0, b1;
+        unpack_f2(sum2[0], a0, a1);
+        unpack_f2(sum2[1], b0, b1);
+        psum = (a0 + a1) + (b0 + b1);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             const float p0 = 32 * c + j < n_vis ? ex2_approx(fmaf(__uint_as_float(sr[c][j]), scale_log2e, -m_ref)) : 0.f;

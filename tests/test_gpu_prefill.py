@@ -69,7 +69,7 @@ def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope, path)
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], biases=biases, rope=rope)
     ctx = case.ctx
-    assert binding.lib().echokv_prefill_path(ctx.handle) == 1
+    assert binding.lib().echokv_prefill_path(ctx.handle) == 2
     ctx.set_prefill_path(path)
     for layer in (1, 0):
         q = queries(w, n_q, layer)
