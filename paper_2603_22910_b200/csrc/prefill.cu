@@ -540,24 +540,30 @@ prefill_attn_tc_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
 // ---------------------------------------------------------------------------------------------
 // 3c. tcgen05 again, with the steps given to different warps so that they overlap
 // ---------------------------------------------------------------------------------------------
-// One CTA per (256 query rows, query head, sequence): two query tiles X = 0, 1 of 128 rows share every key / value tile,
+// One CTA per (256 query rows, query head, sequence): two query tiles x = 0, 1 of 128 rows share every key / value tile,
 // and while the tensor cores work for one of them the other one's softmax runs.
-//   warps 0-3 / 4-7  softmax of tile 0 / 1: thread = one query row.  Reads its S row (128 keys) from tensor memory,
-//                    keeps a reference maximum that only moves when the row's maximum has grown by more than 2^8
-//                    (then it rescales its O row in tensor memory itself), writes the probabilities as bf16 over the
-//                    first 64 columns of S, and at the end normalises and writes its O row.
-//   warp 8           one thread issues every MMA:  S_X = Q_X K^T (A, B from shared memory, K-major) and
-//                    O_X += P_X V (A = P_X from tensor memory, B = the value tile as stored [key][dim]: N-major).
-//   warp 9           one thread issues the TMA loads: Q once, then key tiles (3 stages) and value tiles (2 stages).
-// Tensor memory: S_0 | S_1 | O_0 | O_1, 128 columns each.  MMAs of one thread run in the order issued, so S_X(t + 1),
-// issued right after O_X += P_X(t) V(t), overwrites P_X(t) only after it was read, and its completion tells the
-// softmax warps that O_X is at rest as well.  Every wait is bounded.
+//   warps 0-7 / 8-15 softmax of tile 0 / 1, two threads per query row (64 keys of the tile each; four warps per
+//                    scheduler, so that their special-function, ALU and FMA work overlaps).  A row keeps a reference
+//                    maximum that only moves when the row's maximum has grown by more than 2^8.  The common case is
+//                    taken speculatively: the probabilities are computed against the old reference while the maximum
+//                    is found, and one vote of the row's two warps confirms that nothing moved; otherwise the tile is
+//                    redone the careful way (masks, maxima exchanged through shared memory, O rescaled in tensor
+//                    memory).  Probabilities go back as bf16 over the first 32 of the thread's own 64 columns of S.
+//   warp 16          one thread issues every MMA:  S_x = Q_x K^T (A, B from shared memory, K-major) and
+//                    O_x += P_x V (A = P_x from tensor memory, B = the value tile as stored [key][dim]: N-major).
+//   warp 17          one thread issues the TMA loads: Q once, then key tiles (3 stages) and value tiles (2 stages).
+// Tensor memory: S_0 | S_1 | O_0 | O_1, 128 columns each.  MMAs of one thread run in the order issued, so S_x(t + 1),
+// issued right after O_x += P_x(t) V(t), overwrites P_x(t) only after it was read, and its completion tells the
+// softmax warps that O_x is at rest as well.  Every wait is bounded.
 constexpr int kWsKStages = 3, kWsVStages = 2;
-constexpr int kWsThreads = 320;
+constexpr int kWsSoftmaxWarps = 16;
+constexpr int kWsThreads = (kWsSoftmaxWarps + 2) * 32;
+constexpr int kWsTailBytes = 3072;                                   // the tail sits in front of the tiles
 constexpr uint32_t kIdescPV = kIdescS | (1u << 16);                 // B operand N-major
 constexpr float kWsGrowLog2 = 8.f;
 
 struct PfWsTail {
+  float ex[2][2][kTcTile];         // [query tile][half][row]: row maxima, at the end row sums
   unsigned long long q_full;
   unsigned long long k_full[kWsKStages], k_empty[kWsKStages];
   unsigned long long v_full[kWsVStages], v_empty[kWsVStages];
@@ -565,6 +571,7 @@ struct PfWsTail {
   uint32_t tmem_base;
   int abort_flag;
 };
+static_assert(sizeof(PfWsTail) <= kWsTailBytes, "tail does not fit in front of the tiles");
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -602,46 +609,41 @@ __device__ __forceinline__ uint64_t add_f2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-// 2^x for a pair, x <= ~8, without the special-function unit: n = round(x) by the add-a-large-constant trick,
-// f = x - n in [-0.5, 0.5], a cubic for 2^f (relative error 7.5e-5, far below the bf16 rounding that follows),
-// then n added into the exponent field.  x is clamped at -125 so that the exponent cannot wrap.
-constexpr int kPolyPer = 5, kPolyOf = 2;         // 2 of every 5 pairs
-__device__ __forceinline__ uint64_t ex2_poly_f2(uint64_t x2) {
-  float x0, x1;
-  unpack_f2(x2, x0, x1);
-  x2 = pack_f2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-  const float kMagic = 12582912.f;               // 1.5 * 2^23
-  const uint64_t t2 = add_f2(x2, pack_f2(kMagic, kMagic));
-  const uint64_t n2 = add_f2(t2, pack_f2(-kMagic, -kMagic));
-  const uint64_t f2 = fma_f2(n2, pack_f2(-1.f, -1.f), x2);
-  uint64_t p2 = fma_f2(pack_f2(0.0551716685295105f, 0.0551716685295105f), f2, pack_f2(0.2426111251115799f, 0.2426111251115799f));
-  p2 = fma_f2(p2, f2, pack_f2(0.6932609677314758f, 0.6932609677314758f));
-  p2 = fma_f2(p2, f2, pack_f2(0.9999280571937561f, 0.9999280571937561f));
-  uint32_t p0, p1, t0, t1;
-  unpack_u2(p2, p0, p1);
-  unpack_u2(t2, t0, t1);
-  return pack_u2(p0 + (t0 << 23), p1 + (t1 << 23));
+// barrier `id` over the 64 threads of a row pair's two warps; returns whether any of them passed a set flag
+__device__ __forceinline__ bool pair_any(int id, bool flag) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %2, 0;\n\t"
+      "bar.red.or.pred p, %1, 64, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(flag ? 1u : 0u)
+      : "memory");
+  return r != 0;
 }
+__device__ __forceinline__ void pair_sync(int id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
 
 __global__ void __launch_bounds__(kWsThreads, 1)
 prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, float* __restrict__ out, int n_q, int n_q_heads,
                        int n_kv_heads, const int32_t* __restrict__ slots, const int32_t* __restrict__ lens,
                        int max_batch, int capacity, float scale_log2e, int32_t* status) {
-  extern __shared__ unsigned char pf_ws_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_ws_raw) + 1023) &
-                                                         ~static_cast<uintptr_t>(1023));
-  // Q tile 0, 1 | K stages | V stages
-  const uint32_t q_addr = smem_u32(smem), k_addr = q_addr + 2 * kTcTileBytes,
+  // tail | Q tile 0, 1 | K stages | V stages; the tiles need 1024-byte alignment, and with all of the shared memory in
+  // use there is no room to round the start up
+  extern __shared__ __align__(1024) unsigned char pf_ws_raw[];
+  PfWsTail& t = *reinterpret_cast<PfWsTail*>(pf_ws_raw);
+  const uint32_t q_addr = smem_u32(pf_ws_raw) + kWsTailBytes, k_addr = q_addr + 2 * kTcTileBytes,
                  v_addr = k_addr + kWsKStages * kTcTileBytes;
-  PfWsTail& t = *reinterpret_cast<PfWsTail*>(smem + (2 + kWsKStages + kWsVStages) * kTcTileBytes);
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kvh = h / (n_q_heads / n_kv_heads);
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
-  if (slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
-    if (tid == 0 && qt == 0 && h == 0) report(status, slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
+  const bool misaligned = (q_addr & 1023u) != 0;
+  if (misaligned || slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
+    if (tid == 0 && qt == 0 && h == 0)
+      report(status, misaligned ? ECHOKV_ECUDA : slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
     if (tid < 256) {
       const int i = qt * 2 * kTcTile + tid;
       if (i < n_q) {
@@ -665,14 +667,14 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(smem_u32(&t.s_full[x]), 1);
-      mbar_init(smem_u32(&t.p_ready[x]), 128);
+      mbar_init(smem_u32(&t.p_ready[x]), 256);
       mbar_init(smem_u32(&t.o_done[x]), 1);
     }
     mbar_init(smem_u32(&t.drain), 1);
     mbar_fence_init();
   }
   __syncthreads();
-  if (warp == 8) {
+  if (warp == kWsSoftmaxWarps) {
     tmem_alloc(smem_u32(&t.tmem_base), 512);
     tmem_relinquish();
   }
@@ -686,7 +688,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int kv_end = len - n_q + last_row + 1;              // keys this CTA's rows may see
   const int n_tiles = (kv_end + kTcTile - 1) / kTcTile;
 
-  if (warp == 9) {
+  if (warp == kWsSoftmaxWarps + 1) {
     // =============================== TMA producer ===============================================
     if (lane == 0) {
       const uint32_t qb = smem_u32(&t.q_full);
@@ -722,7 +724,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           mbar_drain(smem_u32(&t.v_full[i % kWsVStages]), (i / kWsVStages) & 1);
       }
     }
-  } else if (warp == 8) {
+  } else if (warp == kWsSoftmaxWarps) {
     // =============================== MMA issuer ================================================
     if (lane == 0) {
       bool alive = mbar_wait(smem_u32(&t.q_full), 0, abort_flag, status);
@@ -751,9 +753,10 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (!mbar_wait(smem_u32(&t.p_ready[x]), tile & 1, abort_flag, status)) { alive = false; break; }
           tc_fence_after();
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)     // 16 keys per MMA: 8 columns of packed probabilities, 2048 bytes of value rows
-            tc_mma_bf16_tmem_a(tmem + 256 + x * 128, tmem + x * 128 + 8 * kk, b0 + 128 * kk, kIdescPV,
-                               (tile > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < 8; ++kk)     // 16 keys per MMA: 8 columns of packed probabilities (each half of the keys
+                                             // at the start of its own 64 columns), 2048 bytes of value rows
+            tc_mma_bf16_tmem_a(tmem + 256 + x * 128, tmem + x * 128 + 64 * (kk >> 2) + 8 * (kk & 3), b0 + 128 * kk,
+                               kIdescPV, (tile > 0 || kk > 0) ? 1u : 0u);
           if (tile + 1 == n_tiles) tc_commit(smem_u32(&t.o_done[x]));
           if (x == 1) tc_commit(smem_u32(&t.v_empty[sv]));
           if (tile + 1 < n_tiles) {
@@ -773,101 +776,100 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
     }
   } else {
-    // =============================== softmax, one thread per query row ===========================
-    const int x = warp >> 2, wl = tid & 127;
-    const int i_row = row0 + x * kTcTile + wl;
+    // =============================== softmax: two threads per query row, 64 keys each ===================
+    const int x = warp >> 3, hf = (warp >> 2) & 1, row = (warp & 3) * 32 + lane;
+    const int pair_id = 1 + x * 4 + (warp & 3);             // named barrier of this row's two warps
+    const int i_row = row0 + x * kTcTile + row;
     const bool row_ok = i_row < n_q;
     const int pos = len - n_q + i_row;                      // position of this query row
     const uint32_t lane_base = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    const uint32_t s_addr = lane_base + x * 128, o_addr = lane_base + 256 + x * 128;
-    float m_ref = -INFINITY, l_run = 0.f;
+    const uint32_t s_addr = lane_base + x * 128 + hf * 64, o_addr = lane_base + 256 + x * 128 + hf * 64;
+    float m_ref = -INFINITY, l_run = 0.f;                   // m_ref is the same in both threads of a row
     bool alive = true;
     for (int tile = 0; tile < n_tiles; ++tile) {
-      if (!mbar_wait(smem_u32(&t.s_full[x]), tile & 1, abort_flag, status)) { alive = false; break; }
-      tc_fence_after();
-      uint32_t sr[4][32];
+      const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&t.s_full[x]), tile & 1, abort_flag, status) ? 1 : 0) != 0;
+      // keys of this thread's half the row sees: the first n_vis
+      const int n_vis = row_ok ? max(0, min(64, pos - (tile * kTcTile + hf * 64) + 1)) : 0;
+      uint32_t sr[2][32];
+      float mx = -INFINITY, psum = 0.f;
+      if (ok) {
+        tc_fence_after();
+        tmem_ld32_issue(s_addr, sr[0]);
+        tmem_ld32_issue(s_addr + 32, sr[1]);
+        tmem_ld_wait();
+        // Speculation: every key visible and the reference maximum unchanged.  Two scores per instruction where the
+        // pipe has a two-wide form (scale-and-shift, row sum); the maximum is found beside it (independent chains of
+        // three-input maxima).  (Taking part of the 2^x from a cubic on the FMA pipe instead of the special-function
+        // unit was measured too: with four softmax warps per scheduler it only cost issue slots.)
+        const uint64_t sc2 = pack_f2(scale_log2e, scale_log2e), nm2 = pack_f2(-m_ref, -m_ref);
+        uint64_t sum2[2] = {0ull, 0ull};
+        float m4[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32_issue(s_addr + 32 * c, sr[c]);
-      tmem_ld_wait();
-      // keys of this tile the row sees: the first n_vis
-      const int n_vis = row_ok ? max(0, min(kTcTile, pos - tile * kTcTile + 1)) : 0;
-      float mx = -INFINITY;
-      if (n_vis == kTcTile) {
-        // eight independent chains of three-input maxima instead of one chain of 128
-        float m8[8];
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < 2; ++c) {
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
             float a = fmaxf(__uint_as_float(sr[c][16 * u]), __uint_as_float(sr[c][16 * u + 1]));
 #pragma unroll
             for (int j = 2; j < 16; j += 2)
               a = max3(a, __uint_as_float(sr[c][16 * u + j]), __uint_as_float(sr[c][16 * u + j + 1]));
-            m8[2 * c + u] = a;
+            m4[2 * c + u] = a;
           }
-        mx = fmaxf(max3(m8[0], m8[1], m8[2]), max3(m8[3], m8[4], m8[5]));
-        mx = max3(mx, m8[6], m8[7]);
-      } else {
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (32 * c + j < n_vis) mx = fmaxf(mx, __uint_as_float(sr[c][j]));
-      }
-      mx *= scale_log2e;                     // (scale > 0: the maximum commutes with it; -inf stays -inf)
-      const bool grow = mx > m_ref + kWsGrowLog2;
-      float alpha = 1.f;
-      if (grow) {
-        alpha = ex2_approx(m_ref - mx);      // 0 on the first tile
-        m_ref = mx;
-        l_run *= alpha;
-      }
-      if (tile > 0 && __any_sync(0xffffffffu, grow)) {
-        // O_x is at rest (the MMA that wrote S came after every earlier one): rescale this thread's row
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t orow[32];
-          tmem_ld32_issue(o_addr + 32 * c, orow);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * alpha);
-          tmem_st32(o_addr + 32 * c, orow);
-        }
-      }
-      float psum = 0.f;
-      if (n_vis == kTcTile) {
-        // Two scores per instruction where the pipe has a two-wide form (scale-and-shift, the polynomial, the row
-        // sum); kPolyOf of every kPolyPer pairs take 2^x from the polynomial instead of the special-function unit,
-        // whose 16 results per clock would otherwise set the pace of the whole kernel.
-        const uint64_t sc2 = pack_f2(scale_log2e, scale_log2e), nm2 = pack_f2(-m_ref, -m_ref);
-        uint64_t sum2[2] = {0ull, 0ull};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
           // 32 keys -> 16 columns of packed bf16 pairs; sr[c] is dead afterwards, so the pairs overwrite its first half
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             const uint64_t x2 = fma_f2(pack_u2(sr[c][j], sr[c][j + 1]), sc2, nm2);
-            uint64_t p2;
-            if (((j >> 1) % kPolyPer) < kPolyOf) {
-              p2 = ex2_poly_f2(x2);
-            } else {
-              float x0, x1;
-              unpack_f2(x2, x0, x1);
-              p2 = pack_f2(ex2_approx(x0), ex2_approx(x1));
-            }
-            sum2[(j >> 1) & 1] = add_f2(sum2[(j >> 1) & 1], p2);
-            float p0, p1;
-            unpack_f2(p2, p0, p1);
+            float x0, x1;
+            unpack_f2(x2, x0, x1);
+            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+            sum2[(j >> 1) & 1] = add_f2(sum2[(j >> 1) & 1], pack_f2(p0, p1));
             sr[c][j >> 1] = pack2(p0, p1);
           }
         }
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * scale_log2e;   // (scale > 0; -inf stays -inf)
         float a0, a1, b0, b1;
         unpack_f2(sum2[0], a0, a1);
         unpack_f2(sum2[1], b0, b1);
         psum = (a0 + a1) + (b0 + b1);
-      } else {
+      }
+      const bool careful = !ok || tile == 0 || n_vis != 64 || !(mx <= m_ref + kWsGrowLog2);
+      if (pair_any(pair_id, careful)) {
+        if (pair_any(pair_id, !ok)) { alive = false; break; }     // both warps of the row leave together
+        // ---- the careful way: masks, the row maximum over both halves, O rescaled if the reference moves
+        tmem_ld32_issue(s_addr, sr[0]);
+        tmem_ld32_issue(s_addr + 32, sr[1]);
+        tmem_ld_wait();
+        mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (32 * c + j < n_vis) mx = fmaxf(mx, __uint_as_float(sr[c][j]));
+        mx *= scale_log2e;
+        t.ex[x][hf][row] = mx;
+        pair_sync(pair_id);
+        mx = fmaxf(mx, t.ex[x][hf ^ 1][row]);
+        const bool grow = mx > m_ref + kWsGrowLog2;
+        float alpha = 1.f;
+        if (grow) {
+          alpha = ex2_approx(m_ref - mx);      // 0 on the first tile
+          m_ref = mx;
+          l_run *= alpha;
+        }
+        if (tile > 0 && __any_sync(0xffffffffu, grow)) {
+          // O_x is at rest (the MMA that wrote S came after every earlier one): rescale this thread's half of its row
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {
+            uint32_t orow[32];
+            tmem_ld32_issue(o_addr + 32 * c, orow);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * alpha);
+            tmem_st32(o_addr + 32 * c, orow);
+          }
+        }
+        psum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             const float p0 = 32 * c + j < n_vis ? ex2_approx(fmaf(__uint_as_float(sr[c][j]), scale_log2e, -m_ref)) : 0.f;
@@ -875,7 +877,6 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             psum += p0 + p1;
             sr[c][j >> 1] = pack2(p0, p1);
           }
-        }
       }
       l_run += psum;
       {
@@ -886,36 +887,36 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           pk[16 + j] = sr[1][j];
         }
         tmem_st32(s_addr, pk);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          pk[j] = sr[2][j];
-          pk[16 + j] = sr[3][j];
-        }
-        tmem_st32(s_addr + 32, pk);
       }
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(smem_u32(&t.p_ready[x]));
     }
-    if (alive && mbar_wait(smem_u32(&t.o_done[x]), 0, abort_flag, status)) {
-      tc_fence_after();
-      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + (row_ok ? i_row : 0)) * n_q_heads + h) * 128);
+    if (alive) {
+      // the row's sum over both halves; every wait from here on is on the same barrier for both warps of a row
+      t.ex[x][hf][row] = l_run;
+      pair_sync(pair_id);
+      l_run += t.ex[x][hf ^ 1][row];
+      if (mbar_wait(smem_u32(&t.o_done[x]), 0, abort_flag, status)) {
+        tc_fence_after();
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + (row_ok ? i_row : 0)) * n_q_heads + h) * 128 + hf * 64);
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float v[32];
-        tmem_ld32(o_addr + 32 * c, v);
-        if (row_ok) {
+        for (int c = 0; c < 2; ++c) {
+          float v[32];
+          tmem_ld32(o_addr + 32 * c, v);
+          if (row_ok) {
 #pragma unroll
-          for (int j4 = 0; j4 < 8; ++j4)
-            dst[8 * c + j4] = make_float4(v[4 * j4] * inv, v[4 * j4 + 1] * inv, v[4 * j4 + 2] * inv, v[4 * j4 + 3] * inv);
+            for (int j4 = 0; j4 < 8; ++j4)
+              dst[8 * c + j4] = make_float4(v[4 * j4] * inv, v[4 * j4 + 1] * inv, v[4 * j4 + 2] * inv, v[4 * j4 + 3] * inv);
+          }
         }
       }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == kWsSoftmaxWarps) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
@@ -956,7 +957,7 @@ cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, 
       if (e != cudaSuccess) return e;
     }
     dim3 grid((n_q + 2 * kTcTile - 1) / (2 * kTcTile), a.n_q_heads, a.batch);
-    const size_t smem = 1024 + (size_t)(2 + kWsKStages + kWsVStages) * kTcTileBytes + sizeof(PfWsTail);
+    const size_t smem = kWsTailBytes + (size_t)(2 + kWsKStages + kWsVStages) * kTcTileBytes;
     const cudaError_t e = cudaFuncSetAttribute(prefill_attn_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                (int)smem);
     if (e != cudaSuccess) return e;
