@@ -7,8 +7,10 @@
 //      (gather_rows_kernel; keys rotated to their positions if a rotary table is set),
 //   2. the dropped dims are predicted on the tensor cores and written beside them (Eq. 3; the
 //      row-storing mode of the CTA-pair kernel),
-//   3. prefill_attn_kernel evaluates Eq. 7 causally over those rows: 64 query rows per CTA, keys and
-//      values in 64-token tiles, S = Q K^T and O += P V as mma.sync m16n8k16, online softmax in fp32.
+//   3. a causal attention kernel evaluates Eq. 7 over those rows, online softmax in fp32.  Three versions,
+//      selectable for tests: prefill_attn_ws_kernel (tcgen05, warp-specialised; the default),
+//      prefill_attn_tc_kernel (tcgen05, one thread group doing every step in turn) and prefill_attn_kernel
+//      (mma.sync m16n8k16, 64 query rows per CTA, 64-token tiles).
 // The rebuilt rows are bf16 in a caller-owned scratch, as in the paper's own materialise-then-attend
 // design; the decode path never writes them.
 #include "prefill.h"

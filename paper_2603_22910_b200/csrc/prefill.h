@@ -1,4 +1,4 @@
-// Prefill-shaped attention (many queries per sequence): host interface of the two CUDA-core / mma.sync kernels.
+// Prefill-shaped attention (many queries per sequence): host interface of the row gather and the attention kernels.
 #pragma once
 
 #include "kernels.h"
