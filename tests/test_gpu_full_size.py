@@ -92,3 +92,38 @@ def test_config4_sweep_points_sampled():
 def test_uncompressed_path_full_size_sampled():
     sampled_check(synth.C1, "full", samples=4, absorbed=False)
     sampled_check(synth.C2, "full", samples=4, absorbed=False)
+
+
+def test_prefill_call_config2_full_size_sampled():
+    """The prefill-shaped call at the C2 shape with 512 causal queries per sequence (the configuration
+    `bench.py --prefill-queries 512` times): query i of the chunk attends the cached prefix up to its own
+    position, which is the decode step of a sequence cut off there, so sampled (sequence, query, head)
+    outputs are recomputed with the single-head decode oracle on the truncated cache."""
+    w, n_q, layer = synth.C2, 512, 1
+    st = bench.State(w, 0, [0, 1])
+    ctx = st.ctx
+    q = synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, 1, device=st.dev).to(torch.bfloat16)
+    out = ctx.prefill_attention(layer, q, st.lens)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.ECHOKV_OK
+    rng = np.random.default_rng(11)
+    picks = [(0, 0, 0), (w.batch - 1, n_q - 1, w.n_q_heads - 1)]           # first and last query of the chunk
+    picks += [(int(rng.integers(w.batch)), int(rng.integers(n_q)), int(rng.integers(w.n_q_heads))) for _ in range(4)]
+    worst = num = den = 0.0
+    for b, i, h in picks:
+        _, kg, vg, kl, vl, Wk, Wv = st.oracle_inputs(layer, b)
+        n_seen = w.context - n_q + i + 1
+        qi = O.widen(synth.to_numpy_stored(q[b, i].cpu()))
+        ref = O.decode_attention_query_heads(qi, kg[:n_seen], vg[:n_seen], kl[:n_seen], vl[:n_seen], Wk, Wv,
+                                             n_kv_heads=w.n_kv_heads, query_heads=[h])[h]
+        got = out[b, i, h].cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got))
+        worst = max(worst, float(np.max(np.abs(got - ref))))
+        num += float(np.sum((got - ref) ** 2))
+        den += float(np.sum(ref ** 2))
+    rel = (num / max(den, 1e-300)) ** 0.5
+    ctx.close()
+    del st
+    torch.cuda.empty_cache()
+    # the tolerance of the prefill-shaped call (it rounds the rebuilt rows to bf16): tests/test_gpu_prefill.py
+    assert worst <= 4e-2 and rel <= 5e-3, (worst, rel)
