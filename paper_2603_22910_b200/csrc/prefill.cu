@@ -869,6 +869,10 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tmem_st32(o_addr + 32 * c, orow);
           }
         }
+        // (the scores are read once more rather than kept in registers across the rescaling)
+        tmem_ld32_issue(s_addr, sr[0]);
+        tmem_ld32_issue(s_addr + 32, sr[1]);
+        tmem_ld_wait();
         psum = 0.f;
 #pragma unroll
         for (int c = 0; c < 2; ++c)
@@ -881,15 +885,8 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           }
       }
       l_run += psum;
-      {
-        uint32_t pk[32];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          pk[j] = sr[0][j];
-          pk[16 + j] = sr[1][j];
-        }
-        tmem_st32(s_addr, pk);
-      }
+      tmem_st16(s_addr, sr[0]);            // the packed pairs sit in the first 16 registers of each block of 32
+      tmem_st16(s_addr + 16, sr[1]);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(smem_u32(&t.p_ready[x]));
