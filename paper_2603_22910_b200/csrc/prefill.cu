@@ -556,7 +556,9 @@ prefill_attn_tc_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
 //   warp 17          one thread issues the TMA loads: Q once, then key tiles (3 stages) and value tiles (2 stages).
 // Tensor memory: S_0 | S_1 | O_0 | O_1, 128 columns each.  MMAs of one thread run in the order issued, so S_x(t + 1),
 // issued right after O_x += P_x(t) V(t), overwrites P_x(t) only after it was read, and its completion tells the
-// softmax warps that O_x is at rest as well.  Every wait is bounded.
+// softmax warps that O_x is at rest as well.  Every wait on an mbarrier is bounded; the named barriers only join the
+// two warps of a row pair, which take the same path through every tile (their votes also make them leave together
+// when a wait ran out).
 constexpr int kWsKStages = 3, kWsVStages = 2;
 constexpr int kWsSoftmaxWarps = 16;
 constexpr int kWsThreads = (kWsSoftmaxWarps + 2) * 32;
