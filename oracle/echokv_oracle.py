@@ -374,12 +374,14 @@ def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n
 
 
 def prefill_attention(q: np.ndarray, k_global, v_global, k_local, v_local, Wk, Wv, n_kv_heads: int,
-                      scale: float | None = None, bk=None, bv=None, rope_theta: float | None = None) -> np.ndarray:
+                      scale: float | None = None, bk=None, bv=None, rope_theta: float | None = None,
+                      k_true=None) -> np.ndarray:
     """q [n_q, H_q, d]: queries of the last n_q of the L cached tokens; query i sits at position
     L - n_q + i and attends the tokens up to and including its own (causal).  The cache of a
     compressed layer is rebuilt once (Eq. 3, Eq. 6) and each query evaluates Eq. 7 over its prefix.
     With Wk = Wv = None the layer holds its full cache (k_global, v_global are used as they are:
-    an anchor layer).  Returns [n_q, H_q, d]."""
+    an anchor layer).  k_true [L, D]: the "save K" setting of Section 5.2, as in decode_attention
+    (keys whole and used as they are; only the values are predicted).  Returns [n_q, H_q, d]."""
     q = np.asarray(q, dtype=np.float64)
     n_q, H_q, d = q.shape
     k_global = np.asarray(k_global, dtype=np.float64)
@@ -391,7 +393,12 @@ def prefill_attention(q: np.ndarray, k_global, v_global, k_local, v_local, Wk, W
         K_t = k_global.reshape(L, n_kv_heads, d)
         V_t = v_global.reshape(L, n_kv_heads, d)
     else:
-        K_t = assemble_cache(k_local, reconstruct_dropped(Wk, k_global, k_local, bk), n_kv_heads, d)
+        if k_true is not None:
+            K_t = np.asarray(k_true, dtype=np.float64).reshape(-1, n_kv_heads, d)
+            if K_t.shape[0] != L:
+                raise ValueError("token counts differ")
+        else:
+            K_t = assemble_cache(k_local, reconstruct_dropped(Wk, k_global, k_local, bk), n_kv_heads, d)
         V_t = assemble_cache(v_local, reconstruct_dropped(Wv, v_global, v_local, bv), n_kv_heads, d)
     if rope_theta is not None:
         K_t = rotate_keys(K_t, rope_theta)

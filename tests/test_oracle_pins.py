@@ -150,6 +150,18 @@ def test_prefill_shaped_attention():
     np.testing.assert_allclose(rot[-1], O.decode_attention(q[-1], *args, rope_theta=10000.0), rtol=1e-12, atol=1e-14)
     with pytest.raises(ValueError):
         O.prefill_attention(g.standard_normal((c["L"] + 1, c["H_q"], c["d"])), *args)
+    # "save K" (Section 5.2): whole keys as they are; a query's row is the save-K decode step on its prefix, and with
+    # the keys of a selector-predictor cache it is plain causal attention over those keys and the rebuilt values
+    k_true = g.standard_normal((c["L"], c["H_kv"] * c["d"]))
+    sk = O.prefill_attention(q, *args, k_true=k_true)
+    for i in (0, n_q - 1):
+        n = c["L"] - n_q + i + 1
+        want = O.decode_attention(q[i], c["kg"][:n], c["vg"][:n], c["kl"][:n], c["vl"][:n], c["Wk"], c["Wv"], c["H_kv"],
+                                  k_true=k_true[:n])
+        np.testing.assert_allclose(sk[i], want, rtol=1e-12, atol=1e-14)
+    assert np.abs(sk - got).max() > 1e-3            # the predicted keys are not used
+    np.testing.assert_array_equal(O.prefill_attention(q, c["kg"], c["vg"], None, c["vl"], None, c["Wv"], c["H_kv"],
+                                                      k_true=k_true), sk)       # k_local, Wk ignored
 
 
 def test_anchor_assignment_eq1():
