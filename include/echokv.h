@@ -188,7 +188,8 @@ int echokv_decode_attention(echokv_ctx* ctx, int layer, const void* q, float* ou
  * and V~ as bf16 rows [B][max_pages_per_seq * page_tokens][D] each, and a causal attention kernel runs over those
  * rows.  Unlike the decode calls this one does round the predicted K and V to bf16 (as the paper's own
  * materialise-then-attend implementation does).  Works on anchor layers too (nothing is predicted there).
- * bf16, head_dim 128 and head-aligned m only; not with sink / window tokens or save_k: EUNSUPPORTED.
+ * bf16, head_dim 128 and head-aligned m only; not with sink / window tokens: EUNSUPPORTED.  With save_k the keys
+ * are gathered whole and only the values are predicted.
  * A sequence with fewer than n_q cached tokens, or an unusable slot / length: zeros and the device status.
  * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (batch, scratch too small), ENOWEIGHTS, ENOTABLE, ECUDA. */
 /* Which attention kernel the prefill-shaped call runs over the rebuilt rows: 0 = mma.sync kernel, 1 = tcgen05 kernel

@@ -613,21 +613,22 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
   const Layer& L = c->layers[layer];
   const bool compressed = !L.anchor && c->d.d_drop > 0;
   if (c->cfg.dtype != ECHOKV_BF16 || c->cfg.head_dim != 128) return ECHOKV_EUNSUPPORTED;
-  if (compressed && (!c->tc_capable || !c->d.head_aligned || c->d.save_k || side_active(c, L))) return ECHOKV_EUNSUPPORTED;
+  if (compressed && (!c->tc_capable || !c->d.head_aligned || side_active(c, L))) return ECHOKV_EUNSUPPORTED;
+  const bool keys_whole = compressed && c->d.save_k;      // Section 5.2: nothing to predict on the K side
   if (n_q > c->d.capacity) return ECHOKV_ECAPACITY;
   const uint64_t rows_bytes = (uint64_t)B * c->d.capacity * c->d.D * 2ull;     // one of K~, V~
   if (scratch_bytes < 2 * rows_bytes) return ECHOKV_ECAPACITY;
-  if (compressed && (!L.Wk || !L.Wv)) return ECHOKV_ENOWEIGHTS;
+  if (compressed && (!L.Wv || (!L.Wk && !keys_whole))) return ECHOKV_ENOWEIGHTS;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
   __nv_bfloat16* k_rows = static_cast<__nv_bfloat16*>(scratch);
   __nv_bfloat16* v_rows = k_rows + rows_bytes / 2;
-  const int width = compressed ? c->d.m : c->d.D;
+  const int k_width = compressed ? c->d.mk : c->d.D, v_width = compressed ? c->d.m : c->d.D;
   // stored dims as they are (keys rotated to their positions), then the predicted ones beside them
-  if (launch_gather_rows(a, L.k_pool, width, k_rows, c->d.capacity, c->d.D, true, 0, s) != cudaSuccess ||
-      launch_gather_rows(a, L.v_pool, width, v_rows, c->d.capacity, c->d.D, false, 128, s) != cudaSuccess)
+  if (launch_gather_rows(a, L.k_pool, k_width, k_rows, c->d.capacity, c->d.D, true, 0, s) != cudaSuccess ||
+      launch_gather_rows(a, L.v_pool, v_width, v_rows, c->d.capacity, c->d.D, false, 128, s) != cudaSuccess)
     return ECHOKV_ECUDA;
-  c->launches += width > 0 ? 2 : 1;
+  c->launches += (k_width > 0 ? 1 : 0) + 1;
   if (compressed) {
     const Layer& A = c->layers[layer - layer % c->cfg.group_size];
     ReconArgs ra;
@@ -638,13 +639,15 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
     ra.part_tokens = c->d.part_tokens;
     ra.capacity_tokens = c->d.capacity;
     ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
-    ra.bk = L.bk;
-    if (launch_recon_pair_store(a, ra, A.tc, L.tc, false, k_rows, c->d.capacity, c->d.D, c->sm_count, s) != cudaSuccess)
-      return ECHOKV_ECUDA;
+    if (!keys_whole) {
+      ra.bk = L.bk;
+      if (launch_recon_pair_store(a, ra, A.tc, L.tc, false, k_rows, c->d.capacity, c->d.D, c->sm_count, s) != cudaSuccess)
+        return ECHOKV_ECUDA;
+    }
     ra.bk = L.bv;
     if (launch_recon_pair_store(a, ra, A.tc, L.tc, true, v_rows, c->d.capacity, c->d.D, c->sm_count, s) != cudaSuccess)
       return ECHOKV_ECUDA;
-    c->launches += 2;
+    c->launches += keys_whole ? 1 : 2;
   }
   if (launch_prefill_attn(a, k_rows, v_rows, c->d.capacity, c->d.D, n_q, out, s, c->prefill_path) != cudaSuccess)
     return ECHOKV_ECUDA;

@@ -48,7 +48,11 @@ def oracle_prefill(case, layer, q, b, rope):
     kl = case._stored(layer, "k", b) if w.m else np.zeros((L, 0))
     vl = case._stored(layer, "v", b) if w.m else np.zeros((L, 0))
     Wk, Wv, bk, bv = (None if t is None else O.widen(synth.to_numpy_stored(t)) for t in case.host_w[layer])
-    return O.prefill_attention(qn, kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv, rope_theta=rope)
+    k_true = None
+    if w.save_k:                 # keys kept whole (Section 5.2): the stored K rows are the whole keys
+        k_true = case._stored(layer, "k", b)
+        kl = k_true[:, :w.m]
+    return O.prefill_attention(qn, kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv, rope_theta=rope, k_true=k_true)
 
 
 CASES = [
@@ -60,6 +64,8 @@ CASES = [
     ("one_query_is_the_decode_step", synth.C2, dict(batch=2, context=300), [300, 17], 1, False, None),
     ("every_token_a_query", synth.C2, dict(batch=1, context=200, n_retained_heads=6), [200], 200, False, THETA),
     ("nothing_retained", synth.C2, dict(batch=2, context=400, n_retained_heads=0), [400, 129], 70, False, None),
+    ("keys_whole", synth.C2, dict(batch=2, context=500, save_k=True), [500, 260], 130, True, None),
+    ("keys_whole_rope", synth.C1, dict(batch=2, context=300, save_k=True), [300, 77], 40, False, THETA),
 ]
 
 
