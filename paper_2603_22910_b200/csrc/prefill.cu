@@ -543,7 +543,8 @@ prefill_attn_tc_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
 // 3c. tcgen05 again, with the steps given to different warps so that they overlap
 // ---------------------------------------------------------------------------------------------
 // One CTA per (256 query rows, query head, sequence): two query tiles x = 0, 1 of 128 rows share every key / value tile,
-// and while the tensor cores work for one of them the other one's softmax runs.
+// and while the tensor cores work for one of them the other one's softmax runs.  (With few queries per sequence the
+// 256 rows are all the rows of 2, 4 or 8 query heads of one KV head instead.)
 //   warps 0-7 / 8-15 softmax of tile 0 / 1, two threads per query row (64 keys of the tile each; four warps per
 //                    scheduler, so that their special-function, ALU and FMA work overlaps).  A row keeps a reference
 //                    maximum that only moves when the row's maximum has grown by more than 2^8.  The common case is
@@ -606,26 +607,35 @@ __global__ void __launch_bounds__(kWsThreads, 1)
 prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, float* __restrict__ out, int n_q, int n_q_heads,
                        int n_kv_heads, const int32_t* __restrict__ slots, const int32_t* __restrict__ lens,
-                       int max_batch, int capacity, float scale_log2e, int32_t* status) {
+                       int max_batch, int capacity, float scale_log2e, int rows_per_head, int32_t* status) {
   // tail | Q tile 0, 1 | K stages | V stages; the tiles need 1024-byte alignment, and with all of the shared memory in
   // use there is no room to round the start up
   extern __shared__ __align__(1024) unsigned char pf_ws_raw[];
   PfWsTail& t = *reinterpret_cast<PfWsTail*>(pf_ws_raw);
   const uint32_t q_addr = smem_u32(pf_ws_raw) + kWsTailBytes, k_addr = q_addr + 2 * kTcTileBytes,
                  v_addr = k_addr + kWsKStages * kTcTileBytes;
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int kvh = h / (n_q_heads / n_kv_heads);
+  // The CTA's 256 query rows: rows 256 qt .. + 255 of one query head (rows_per_head = 0), or -- with few queries per
+  // sequence -- rows 0 .. rows_per_head - 1 of 256 / rows_per_head query heads that share their KV head
+  // (rows_per_head = 128, 64 or 32, at least n_q).  A tile whose rows all lie past n_q is not worked on at all.
+  const int by = blockIdx.y, row_base = (int)blockIdx.x * 2 * kTcTile;
+  const int heads_per_cta = rows_per_head ? 2 * kTcTile / rows_per_head : 1;
+  // (tile x, row r of the tile) -> query head and query row
+  auto head_of = [&](int x, int r) { return rows_per_head ? by * heads_per_cta + (x * kTcTile + r) / rows_per_head : by; };
+  auto query_of = [&](int x, int r) { return rows_per_head ? r % rows_per_head : row_base + x * kTcTile + r; };
+  const int n_act = (rows_per_head || row_base + kTcTile < n_q) ? 2 : 1;      // (tile 0 always holds a query)
+  const int kvh = head_of(0, 0) / (n_q_heads / n_kv_heads);
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
   const bool misaligned = (q_addr & 1023u) != 0;
   if (misaligned || slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
-    if (tid == 0 && qt == 0 && h == 0)
+    if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0)
       report(status, misaligned ? ECHOKV_ECUDA : slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
     if (tid < 256) {
-      const int i = qt * 2 * kTcTile + tid;
+      const int x = tid >> 7, i = query_of(x, tid & 127);
       if (i < n_q) {
-        float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + i) * n_q_heads + h) * 128);
+        float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + i) * n_q_heads + head_of(x, tid & 127)) * 128);
         for (int c = 0; c < 32; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
@@ -661,8 +671,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_after();
   const uint32_t tmem = t.tmem_base;
 
-  const int row0 = qt * 2 * kTcTile;                        // first query row of the CTA
-  const int last_row = min(n_q, row0 + 2 * kTcTile) - 1;
+  const int last_row = rows_per_head ? n_q - 1 : min(n_q, row_base + n_act * kTcTile) - 1;
   const int kv_end = len - n_q + last_row + 1;              // keys this CTA's rows may see
   const int n_tiles = (kv_end + kTcTile - 1) / kTcTile;
 
@@ -670,9 +679,18 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // =============================== TMA producer ===============================================
     if (lane == 0) {
       const uint32_t qb = smem_u32(&t.q_full);
-      mbar_arrive_expect_tx(qb, 2 * kTcTileBytes);
-      tma_load_5d(q_addr, &tm_q, 0, row0, 0, h, b, qb);
-      tma_load_5d(q_addr + kTcTileBytes, &tm_q, 0, row0 + kTcTile, 0, h, b, qb);
+      mbar_arrive_expect_tx(qb, n_act * kTcTileBytes);
+      if (rows_per_head) {
+        // one box per (head, 64-dim chunk): rows_per_head query rows (tm_q's box is that high and one chunk deep)
+        for (int j = 0; j < heads_per_cta; ++j)
+          for (int c = 0; c < 2; ++c)
+            tma_load_5d(q_addr + (j * rows_per_head / kTcTile) * kTcTileBytes + c * kTcChunkBytes +
+                            (j * rows_per_head % kTcTile) * 128,
+                        &tm_q, 0, 0, c, by * heads_per_cta + j, b, qb);
+      } else {
+        for (int x = 0; x < n_act; ++x)
+          tma_load_5d(q_addr + x * kTcTileBytes, &tm_q, 0, row_base + x * kTcTile, 0, by, b, qb);
+      }
       bool alive = true;
       int k_issued = 0, v_issued = 0;
       for (int tile = 0; tile < n_tiles && alive; ++tile) {
@@ -715,19 +733,18 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           tc_mma_bf16(tmem + x * 128, a, bd, kIdescS, kk > 0 ? 1u : 0u);
         }
         tc_commit(smem_u32(&t.s_full[x]));
-        if (x == 1) tc_commit(smem_u32(&t.k_empty[s]));
+        if (x == n_act - 1) tc_commit(smem_u32(&t.k_empty[s]));
       };
       if (alive) alive = mbar_wait(smem_u32(&t.k_full[0]), 0, abort_flag, status);
       if (alive) {
         tc_fence_after();
-        issue_s(0, 0);
-        issue_s(1, 0);
+        for (int x = 0; x < n_act; ++x) issue_s(x, 0);
       }
       for (int tile = 0; tile < n_tiles && alive; ++tile) {
         const int sv = tile % kWsVStages;
         if (!mbar_wait(smem_u32(&t.v_full[sv]), (tile / kWsVStages) & 1, abort_flag, status)) { alive = false; break; }
         const uint64_t b0 = pf_desc_mmajor(v_addr + sv * kTcTileBytes, kTcChunkBytes);
-        for (int x = 0; x < 2 && alive; ++x) {
+        for (int x = 0; x < n_act && alive; ++x) {
           if (!mbar_wait(smem_u32(&t.p_ready[x]), tile & 1, abort_flag, status)) { alive = false; break; }
           tc_fence_after();
 #pragma unroll
@@ -736,7 +753,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc_mma_bf16_tmem_a(tmem + 256 + x * 128, tmem + x * 128 + 64 * (kk >> 2) + 8 * (kk & 3), b0 + 128 * kk,
                                kIdescPV, (tile > 0 || kk > 0) ? 1u : 0u);
           if (tile + 1 == n_tiles) tc_commit(smem_u32(&t.o_done[x]));
-          if (x == 1) tc_commit(smem_u32(&t.v_empty[sv]));
+          if (x == n_act - 1) tc_commit(smem_u32(&t.v_empty[sv]));
           if (tile + 1 < n_tiles) {
             if (x == 0) {
               const int sk = (tile + 1) % kWsKStages;
@@ -753,11 +770,12 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         mbar_drain(smem_u32(&t.drain), 0);
       }
     }
-  } else {
+  } else if ((warp >> 3) < n_act) {
     // =============================== softmax: two threads per query row, 64 keys each ===================
     const int x = warp >> 3, hf = (warp >> 2) & 1, row = (warp & 3) * 32 + lane;
     const int pair_id = 1 + x * 4 + (warp & 3);             // named barrier of this row's two warps
-    const int i_row = row0 + x * kTcTile + row;
+    const int h = head_of(x, row);
+    const int i_row = query_of(x, row);
     const bool row_ok = i_row < n_q;
     const int pos = len - n_q + i_row;                      // position of this query row
     const uint32_t lane_base = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
@@ -915,11 +933,17 @@ cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, 
   if (path == 2) {
     if (kv_width % 64 != 0 || reinterpret_cast<uintptr_t>(a.q) % 16 != 0) return cudaErrorInvalidValue;
     CUtensorMap tm_q, tm_k, tm_v;
+    // few queries per sequence: the CTA's 256 rows are 2, 4 or 8 query heads of one KV head, rows_per_head rows each
+    const int group = a.n_q_heads / a.n_kv_heads;
+    int rows_per_head = 0;
+    for (int r = 32; r <= kTcTile; r *= 2)
+      if (rows_per_head == 0 && n_q <= r && group % (2 * kTcTile / r) == 0) rows_per_head = r;
     {
-      // q [B][n_q][H_q][128] seen as [B][H_q][2 chunks][n_q][64]: a box is the two 64-dim chunks of 128 query rows
+      // q [B][n_q][H_q][128] seen as [B][H_q][2 chunks][n_q][64]: a box is the two 64-dim chunks of 128 query rows,
+      // or one chunk of rows_per_head rows
       const uint64_t dims[5] = {64, (uint64_t)n_q, 2, (uint64_t)a.n_q_heads, (uint64_t)a.batch};
       const uint64_t strides[4] = {(uint64_t)a.n_q_heads * 256, 128, 256, (uint64_t)n_q * a.n_q_heads * 256};
-      const uint32_t box[5] = {64, (uint32_t)kTcTile, 2, 1, 1};
+      const uint32_t box[5] = {64, (uint32_t)(rows_per_head ? rows_per_head : kTcTile), rows_per_head ? 1u : 2u, 1, 1};
       const cudaError_t e = encode_tiled_bf16(&tm_q, a.q, 5, dims, strides, box);
       if (e != cudaSuccess) return e;
     }
@@ -931,7 +955,8 @@ cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, 
       const cudaError_t e = encode_tiled_bf16(kind ? &tm_v : &tm_k, kind ? v_rows : k_rows, 4, dims, strides, box);
       if (e != cudaSuccess) return e;
     }
-    dim3 grid((n_q + 2 * kTcTile - 1) / (2 * kTcTile), a.n_q_heads, a.batch);
+    dim3 grid(rows_per_head ? 1 : (n_q + 2 * kTcTile - 1) / (2 * kTcTile),
+              rows_per_head ? a.n_q_heads / (2 * kTcTile / rows_per_head) : a.n_q_heads, a.batch);
     const size_t smem = kWsTailBytes + (size_t)(2 + kWsKStages + kWsVStages) * kTcTileBytes;
     const cudaError_t e = cudaFuncSetAttribute(prefill_attn_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                (int)smem);
@@ -939,7 +964,7 @@ cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, 
     prefill_attn_ws_kernel<<<grid, kWsThreads, smem, stream>>>(tm_q, tm_k, tm_v, out, n_q, a.n_q_heads, a.n_kv_heads,
                                                                a.slots, a.lens, a.geom.max_batch,
                                                                a.geom.max_pages_per_seq * a.geom.page_tokens,
-                                                               a.scale_log2e, a.status);
+                                                               a.scale_log2e, rows_per_head, a.status);
     return cudaGetLastError();
   }
   if (path == 1) {

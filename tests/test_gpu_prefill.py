@@ -64,6 +64,9 @@ CASES = [
     ("one_query_is_the_decode_step", synth.C2, dict(batch=2, context=300), [300, 17], 1, False, None),
     ("every_token_a_query", synth.C2, dict(batch=1, context=200, n_retained_heads=6), [200], 200, False, THETA),
     ("nothing_retained", synth.C2, dict(batch=2, context=400, n_retained_heads=0), [400, 129], 70, False, None),
+    ("two_heads_per_cta_128_queries", synth.C2, dict(batch=2, context=400, random_pages=True), [400, 128], 128, False, THETA),
+    ("eight_heads_per_cta", synth.C2, dict(batch=2, context=300, n_q_heads=64), [300, 33], 20, False, None),
+    ("second_cta_half_empty", synth.C2, dict(batch=2, context=700), [700, 300], 300, False, None),
     ("keys_whole", synth.C2, dict(batch=2, context=500, save_k=True), [500, 260], 130, True, None),
     ("keys_whole_rope", synth.C1, dict(batch=2, context=300, save_k=True), [300, 77], 40, False, THETA),
 ]
