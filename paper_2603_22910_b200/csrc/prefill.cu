@@ -546,12 +546,15 @@ prefill_attn_tc_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16*
 // and while the tensor cores work for one of them the other one's softmax runs.  (With few queries per sequence the
 // 256 rows are all the rows of 2, 4 or 8 query heads of one KV head instead.)
 //   warps 0-7 / 8-15 softmax of tile 0 / 1, two threads per query row (64 keys of the tile each; four warps per
-//                    scheduler, so that their special-function, ALU and FMA work overlaps).  A row keeps a reference
-//                    maximum that only moves when the row's maximum has grown by more than 2^8.  The common case is
-//                    taken speculatively: the probabilities are computed against the old reference while the maximum
-//                    is found, and one vote of the row's two warps confirms that nothing moved; otherwise the tile is
-//                    redone the careful way (masks, maxima exchanged through shared memory, O rescaled in tensor
-//                    memory).  Probabilities go back as bf16 over the first 32 of the thread's own 64 columns of S.
+//                    scheduler, so that their special-function, ALU and FMA work overlaps).  Probabilities are taken
+//                    against a reference maximum per row, 2^(s - ref): o / l does not depend on the reference, and
+//                    bf16 and fp32 hold large values as precisely as small ones, so the reference only has to move
+//                    before anything could overflow.  The common case is therefore taken speculatively, without
+//                    looking for the maximum at all: if a thread's 64 probabilities sum to less than 2^40, nothing
+//                    moves; one vote of the row's two warps confirms it.  Otherwise, and on the first and the
+//                    diagonal tiles, the tile is redone the careful way (masks, maxima exchanged through shared
+//                    memory, reference moved to the new maximum, O rescaled in tensor memory).  Probabilities go
+//                    back as bf16 over the first 32 of the thread's own 64 columns of S.
 //   warp 16          one thread issues every MMA:  S_x = Q_x K^T (A, B from shared memory, K-major) and
 //                    O_x += P_x V (A = P_x from tensor memory, B = the value tile as stored [key][dim]: N-major).
 //   warp 17          one thread issues the TMA loads: Q once, then key tiles (3 stages) and value tiles (2 stages).
@@ -565,7 +568,8 @@ constexpr int kWsSoftmaxWarps = 16;
 constexpr int kWsThreads = (kWsSoftmaxWarps + 2) * 32;
 constexpr int kWsTailBytes = 3072;                                   // the tail sits in front of the tiles
 constexpr uint32_t kIdescPV = kIdescS | (1u << 16);                 // B operand N-major
-constexpr float kWsGrowLog2 = 8.f;
+constexpr float kWsGrowLog2 = 8.f;                // the careful path moves the reference if the maximum is this far above it
+constexpr float kWsSumLimit = 1099511627776.f;    // 2^40: a half-row's probabilities summing to less leave the reference alone
 
 struct PfWsTail {
   float ex[2][2][kTcTile];         // [query tile][half][row]: row maxima, at the end row sums
@@ -581,11 +585,6 @@ static_assert(sizeof(PfWsTail) <= kWsTailBytes, "tail does not fit in front of t
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float y;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
 // barrier `id` over the 64 threads of a row pair's two warps; returns whether any of them passed a set flag
@@ -793,23 +792,13 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tmem_ld32_issue(s_addr, sr[0]);
         tmem_ld32_issue(s_addr + 32, sr[1]);
         tmem_ld_wait();
-        // Speculation: every key visible and the reference maximum unchanged.  Two scores per instruction where the
-        // pipe has a two-wide form (scale-and-shift, row sum); the maximum is found beside it (independent chains of
-        // three-input maxima).  (Taking part of the 2^x from a cubic on the FMA pipe instead of the special-function
-        // unit was measured too: with four softmax warps per scheduler it only cost issue slots.)
+        // Speculation: every key visible and the reference where it is.  Two scores per instruction where the pipe
+        // has a two-wide form (scale-and-shift, row sum).  (Measured and dropped: a cubic on the FMA pipe for part of
+        // the 2^x, +10 % time at a quarter of them; looking for the row maximum beside the 2^x, +5 %.)
         const uint64_t sc2 = pack_f2(scale_log2e, scale_log2e), nm2 = pack_f2(-m_ref, -m_ref);
         uint64_t sum2[2] = {0ull, 0ull};
-        float m4[4];
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            float a = fmaxf(__uint_as_float(sr[c][16 * u]), __uint_as_float(sr[c][16 * u + 1]));
-#pragma unroll
-            for (int j = 2; j < 16; j += 2)
-              a = max3(a, __uint_as_float(sr[c][16 * u + j]), __uint_as_float(sr[c][16 * u + j + 1]));
-            m4[2 * c + u] = a;
-          }
           // 32 keys -> 16 columns of packed bf16 pairs; sr[c] is dead afterwards, so the pairs overwrite its first half
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
@@ -821,13 +810,12 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             sr[c][j >> 1] = pack2(p0, p1);
           }
         }
-        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * scale_log2e;   // (scale > 0; -inf stays -inf)
         float a0, a1, b0, b1;
         unpack_f2(sum2[0], a0, a1);
         unpack_f2(sum2[1], b0, b1);
         psum = (a0 + a1) + (b0 + b1);
       }
-      const bool careful = !ok || tile == 0 || n_vis != 64 || !(mx <= m_ref + kWsGrowLog2);
+      const bool careful = !ok || tile == 0 || n_vis != 64 || !(psum < kWsSumLimit);
       if (pair_any(pair_id, careful)) {
         if (pair_any(pair_id, !ok)) { alive = false; break; }     // both warps of the row leave together
         // ---- the careful way: masks, the row maximum over both halves, O rescaled if the reference moves

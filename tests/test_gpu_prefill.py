@@ -174,3 +174,25 @@ def test_chunk_append_equals_token_by_token(window):
     np.testing.assert_array_equal(short.run(0), ref.run(0))
     ref.close()
     short.close()
+
+
+@pytest.mark.parametrize("path", [1, 2], ids=["tcgen05", "tcgen05_ws"])
+def test_prefill_scores_that_jump_mid_sequence(path):
+    """A few keys in the middle of the cache score far above everything before them (2^46 and more above the running
+    reference, some beyond what 2^x can hold in fp32): the kernels that keep a lazy reference maximum must notice,
+    move it and rescale what they have accumulated."""
+    w = synth.C2.replace(batch=1, context=1000)
+    case = Case(w, lens=[1000], layers=[0])
+    ctx = case.ctx
+    ctx.set_prefill_path(path)
+    hot = slice(400, 421)
+    rows = case.host[(0, "k", 0)]
+    rows[hot] = rows[hot] * 32                       # (a power of two: exact in bf16)
+    ctx.k_pools[0].view(-1, w.D)[hot] = rows[hot].to(ctx.device)       # identity page order: pool row = token
+    n_q = 300
+    q = queries(w, n_q, 5)
+    out = ctx.prefill_attention(0, q.to(ctx.device), case.seq_lens).cpu().numpy().astype(np.float64)
+    assert ctx.device_status() == binding.ECHOKV_OK
+    ref = oracle_prefill(case, 0, q, 0, None)
+    assert_parity(out[0], ref, w.dtype, "jumping scores")
+    case.close()
