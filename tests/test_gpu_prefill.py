@@ -66,6 +66,7 @@ CASES = [
     ("nothing_retained", synth.C2, dict(batch=2, context=400, n_retained_heads=0), [400, 129], 70, False, None),
     ("two_heads_per_cta_128_queries", synth.C2, dict(batch=2, context=400, random_pages=True), [400, 128], 128, False, THETA),
     ("eight_heads_per_cta", synth.C2, dict(batch=2, context=300, n_q_heads=64), [300, 33], 20, False, None),
+    ("mha_two_ctas_per_head", synth.C1, dict(batch=1, context=600), [600], 300, False, None),
     ("second_cta_half_empty", synth.C2, dict(batch=2, context=700), [700, 300], 300, False, None),
     ("keys_whole", synth.C2, dict(batch=2, context=500, save_k=True), [500, 260], 130, True, None),
     ("keys_whole_rope", synth.C1, dict(batch=2, context=300, save_k=True), [300, 77], 40, False, THETA),
@@ -195,4 +196,20 @@ def test_prefill_scores_that_jump_mid_sequence(path):
     assert ctx.device_status() == binding.ECHOKV_OK
     ref = oracle_prefill(case, 0, q, 0, None)
     assert_parity(out[0], ref, w.dtype, "jumping scores")
+    case.close()
+
+
+def test_prefill_sequence_slots_select_block_table_rows():
+    w = synth.C2.replace(batch=3, context=300)
+    case = Case(w, lens=[300, 150, 99], layers=[0, 1])
+    ctx, dev = case.ctx, case.ctx.device
+    n_q = 70
+    q = queries(w, n_q, 9).to(dev)
+    base = ctx.prefill_attention(1, q, case.seq_lens).cpu().numpy()
+    order = [2, 0, 1]
+    slots = torch.tensor(order, dtype=torch.int32, device=dev)
+    out = ctx.prefill_attention(1, q[order].contiguous(), case.seq_lens[order].contiguous(), seq_slots=slots)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out.cpu().numpy(), base[order])
+    assert ctx.device_status() == binding.ECHOKV_OK
     case.close()
