@@ -29,8 +29,8 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
                                                           __nv_bfloat16* __restrict__ out, int out_tokens,
                                                           int out_width, const int32_t* __restrict__ slots,
                                                           const int32_t* __restrict__ lens, PageGeom g, RopeTable rope,
-                                                          int zero_tail, int32_t* status) {
-  const int b = blockIdx.y, t0 = blockIdx.x * 32;
+                                                          int zero_tail, int block_tokens, int32_t* status) {
+  const int b = blockIdx.y, t0 = blockIdx.x * block_tokens;
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
   if (slot < 0 || slot >= g.max_batch || len < 1 || len > g.max_pages_per_seq * g.page_tokens) return;
@@ -39,7 +39,8 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
     // tiles of rows multiplies them by zero weights, which garbage (a NaN pattern) would not survive
     const int end = min(out_tokens, (len + zero_tail - 1) / zero_tail * zero_tail);
     const int pieces = out_width / 8;
-    for (int it = threadIdx.x; it < 32 * pieces; it += blockDim.x) {
+    const bool any = t0 < end && t0 + block_tokens > len;        // (most blocks hold no such row)
+    for (int it = threadIdx.x; any && it < block_tokens * pieces; it += blockDim.x) {
       const int t = t0 + it / pieces;
       if (t >= len && t < end)
         *reinterpret_cast<uint4*>(out + ((size_t)b * out_tokens + t) * (size_t)out_width + (it % pieces) * 8) =
@@ -48,43 +49,63 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
   }
   if (t0 >= len) return;
   const int n_heads = width / 128;
-  // item = (token of the tile, head, 8-dim piece c of the head's first half, with its partner piece 64 dims on)
-  const int n_items = 32 * n_heads * 8;
-  for (int it = threadIdx.x; it < n_items; it += blockDim.x) {
-    const int c = it & 7, hd = (it >> 3) % n_heads, tt = it / (8 * n_heads);
-    const int t = t0 + tt;
-    if (t >= len) continue;
-    const int page = g.table[(size_t)slot * g.max_pages_per_seq + t / g.page_tokens];
-    if (page < 0 || page >= g.n_pages) {
-      report(status, ECHOKV_EBADPAGE);
-      continue;
+  // item = (token of the tile, head, 8-dim piece c of the head's first half, with its partner piece 64 dims on);
+  // a thread takes four items at a time: four page look-ups, then eight loads, then the stores, so that they overlap
+  constexpr int kBatch = 4;
+  const int n_items = block_tokens * n_heads * 8;
+  const int c = threadIdx.x & 7;                   // (the block size is a multiple of 8: the same for all its items)
+  for (int it0 = threadIdx.x; it0 < n_items; it0 += blockDim.x * kBatch) {
+    int tok[kBatch], head[kBatch], page[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int it = it0 + u * blockDim.x;
+      head[u] = (it >> 3) % n_heads;
+      tok[u] = it < n_items ? t0 + it / (8 * n_heads) : len;       // (len: nothing to do)
+      page[u] = tok[u] < len ? g.table[(size_t)slot * g.max_pages_per_seq + tok[u] / g.page_tokens] : 0;
     }
-    const __nv_bfloat16* src = pool + ((size_t)page * g.page_tokens + t % g.page_tokens) * (size_t)width + hd * 128 + c * 8;
-    __nv_bfloat16* dst = out + ((size_t)b * out_tokens + t) * (size_t)out_width + hd * 128 + c * 8;
-    uint4 lo = *reinterpret_cast<const uint4*>(src), hi = *reinterpret_cast<const uint4*>(src + 64);
-    if (rope.cs != nullptr) {
-      uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
-      const float2* cs = rope.cs + min(t, rope.stride - 1);
+    uint4 lo[kBatch], hi[kBatch];
 #pragma unroll
-      for (int e2 = 0; e2 < 4; ++e2) {
-        float r_lo[2], r_hi[2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float k_lo = h ? __uint_as_float(lw[e2] & 0xffff0000u) : __uint_as_float(lw[e2] << 16);
-          const float k_hi = h ? __uint_as_float(hw[e2] & 0xffff0000u) : __uint_as_float(hw[e2] << 16);
-          const float2 w = cs[(size_t)(c * 8 + 2 * e2 + h) * rope.stride];
-          r_lo[h] = k_lo * w.x - k_hi * w.y;
-          r_hi[h] = k_hi * w.x + k_lo * w.y;
-        }
-        const __nv_bfloat162 a = __floats2bfloat162_rn(r_lo[0], r_lo[1]), bb = __floats2bfloat162_rn(r_hi[0], r_hi[1]);
-        lw[e2] = *reinterpret_cast<const uint32_t*>(&a);
-        hw[e2] = *reinterpret_cast<const uint32_t*>(&bb);
+    for (int u = 0; u < kBatch; ++u) {
+      if (tok[u] < len && (page[u] < 0 || page[u] >= g.n_pages)) {
+        report(status, ECHOKV_EBADPAGE);
+        tok[u] = len;
       }
-      lo = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-      hi = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      if (tok[u] < len) {
+        const __nv_bfloat16* src = pool + ((size_t)page[u] * g.page_tokens + tok[u] % g.page_tokens) * (size_t)width +
+                                   head[u] * 128 + c * 8;
+        lo[u] = *reinterpret_cast<const uint4*>(src);
+        hi[u] = *reinterpret_cast<const uint4*>(src + 64);
+      }
     }
-    *reinterpret_cast<uint4*>(dst) = lo;
-    *reinterpret_cast<uint4*>(dst + 64) = hi;
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      if (tok[u] >= len) continue;
+      const int t = tok[u];
+      if (rope.cs != nullptr) {
+        uint32_t lw[4] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w}, hw[4] = {hi[u].x, hi[u].y, hi[u].z, hi[u].w};
+        const float2* cs = rope.cs + min(t, rope.stride - 1);
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) {
+          float r_lo[2], r_hi[2];
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const float k_lo = h ? __uint_as_float(lw[e2] & 0xffff0000u) : __uint_as_float(lw[e2] << 16);
+            const float k_hi = h ? __uint_as_float(hw[e2] & 0xffff0000u) : __uint_as_float(hw[e2] << 16);
+            const float2 w = cs[(size_t)(c * 8 + 2 * e2 + h) * rope.stride];
+            r_lo[h] = k_lo * w.x - k_hi * w.y;
+            r_hi[h] = k_hi * w.x + k_lo * w.y;
+          }
+          const __nv_bfloat162 a = __floats2bfloat162_rn(r_lo[0], r_lo[1]), bb = __floats2bfloat162_rn(r_hi[0], r_hi[1]);
+          lw[e2] = *reinterpret_cast<const uint32_t*>(&a);
+          hw[e2] = *reinterpret_cast<const uint32_t*>(&bb);
+        }
+        lo[u] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+        hi[u] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      }
+      __nv_bfloat16* dst = out + ((size_t)b * out_tokens + t) * (size_t)out_width + head[u] * 128 + c * 8;
+      *reinterpret_cast<uint4*>(dst) = lo[u];
+      *reinterpret_cast<uint4*>(dst + 64) = hi[u];
+    }
   }
 }
 
@@ -909,10 +930,12 @@ cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, _
                                int out_width, bool rotate, int zero_tail, cudaStream_t stream) {
   if (width == 0 && zero_tail == 0) return cudaSuccess;
   if (width % 128 != 0 || out_width % 8 != 0) return cudaErrorInvalidValue;
-  dim3 grid((out_tokens + 31) / 32, a.batch);
+  // enough tokens per block that every thread has four items to overlap
+  const int block_tokens = width <= 256 ? 64 : 32;
+  dim3 grid((out_tokens + block_tokens - 1) / block_tokens, a.batch);
   gather_rows_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(pool), width, out, out_tokens,
                                                out_width, a.slots, a.lens, a.geom, rotate ? a.rope : RopeTable(), zero_tail,
-                                               a.status);
+                                               block_tokens, a.status);
   return cudaGetLastError();
 }
 
