@@ -848,11 +848,24 @@ absorb_out_kernel(const float* __restrict__ ysum, const __nv_bfloat16* __restric
 
 // out[b][h][:] holds the normalised result over the predicted tokens, ml[b][h] its (max, sum); parts hold the
 // partial over the sink / window tokens at index 0.  Combine the two by log-sum-exp.
+// bk_shift (may be null): the K predictor's bias, which the absorbed queries leave out; it shifts the scores of a
+// predicted head's predicted tokens by q . b_k against the sink / window tokens' true keys.
 __global__ void __launch_bounds__(128)
-absorb_combine_kernel(float* __restrict__ out, const float2* __restrict__ ml, Partials parts, int n_q_heads) {
+absorb_combine_kernel(float* __restrict__ out, const float2* __restrict__ ml, Partials parts, int n_q_heads,
+                      const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ bk_shift, int g, int m,
+                      float scale_log2e) {
   const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
   const size_t bh = (size_t)b * n_q_heads + h;
-  const float2 mid = ml[bh];
+  float2 mid = ml[bh];
+  const int flat = (h / g) * 128 + j;              // this thread's flat dim of the head
+  if (bk_shift != nullptr && (h / g) * 128 + 127 >= m) {
+    __shared__ float s_dot[4];
+    float d = flat >= m ? __bfloat162float(q[bh * 128 + j]) * __bfloat162float(bk_shift[flat - m]) : 0.f;
+    d = warp_sum(d);
+    if ((j & 31) == 0) s_dot[j >> 5] = d;
+    __syncthreads();
+    mid.x += ((s_dot[0] + s_dot[1]) + (s_dot[2] + s_dot[3])) * scale_log2e;
+  }
   const float2 side = parts.ml[bh * parts.max_parts];
   const float M = fmaxf(mid.x, side.x);
   if (M == -INFINITY) return;      // (an unusable sequence: zeros were written already)
@@ -1081,7 +1094,10 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     pool.k_pool = r.k_local; pool.v_pool = r.v_local; pool.width = r.m; pool.part = 0;
     if ((e = launch_attn_side(a, side, n_ret, 1, stream, &pool)) != cudaSuccess) return e;
     dim3 grid(a.n_q_heads, a.batch);
-    absorb_combine_kernel<<<grid, 128, 0, stream>>>(out, ml, a.parts, a.n_q_heads);
+    absorb_combine_kernel<<<grid, 128, 0, stream>>>(out, ml, a.parts, a.n_q_heads,
+                                                    reinterpret_cast<const __nv_bfloat16*>(a.q),
+                                                    reinterpret_cast<const __nv_bfloat16*>(r.bk_shift), g, r.m,
+                                                    a.scale_log2e);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;

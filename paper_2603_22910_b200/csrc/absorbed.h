@@ -46,6 +46,8 @@ struct AbsorbArgs {
   AbsorbLayout lay;
   const void* Wk; const void* Wv; const void* bv;     // predictors of the layer ([D - m][D + m]), V bias or null
   const void* bk = nullptr;     // K bias or null; read only when the keys are rotated (a.rope set): it cancels otherwise
+  const void* bk_shift = nullptr;   // K bias or null: un-rotated keys with sink / window tokens, against whose true keys
+                                    // the predicted tokens' scores are shifted by q . b_k
   int D, m;
   int capacity_tokens;
   bool save_k = false;          // the layer keeps its keys whole (k_local: pool of width D): no K predictor, every head's

@@ -687,6 +687,7 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     aa.lay = c->alay;
     aa.Wk = L.Wk; aa.Wv = L.Wv; aa.bv = L.bv;
     aa.bk = c->rope.cs != nullptr ? L.bk : nullptr;
+    aa.bk_shift = side && c->rope.cs == nullptr ? L.bk : nullptr;
     aa.k_local = L.k_pool; aa.v_local = L.v_pool;
     aa.save_k = c->d.save_k;
     aa.D = c->d.D; aa.m = c->d.m;
@@ -742,8 +743,10 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     if (launch_attn_side(a, side_args(c, L), r, recon_part_tokens, s) != cudaSuccess) return ECHOKV_ECUDA;
     c->launches += 1;
   }
+  // (a K bias is inside the scores already where the keys are rotated; otherwise it only matters against the
+  // sink / window tokens, and the merge accounts for it)
   if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, recon_part_tokens, L.bv, s,
-                   side ? 1 : 0) != cudaSuccess)
+                   side ? 1 : 0, side && c->rope.cs == nullptr ? L.bk : nullptr) != cudaSuccess)
     return ECHOKV_ECUDA;
   c->launches += 2;
   return ECHOKV_OK;

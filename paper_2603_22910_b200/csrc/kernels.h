@@ -106,9 +106,13 @@ cudaError_t launch_recon_simt(const AttnArgs& a, const ReconArgs& r, cudaStream_
 // n_stored_parts partials or, when stored_item_tokens is given (device; one entry per
 // stored_batch_per_slot sequences, written by the stored-head kernel), ceil(len / that entry);
 // the others ceil(len / part_tokens).  bv (may be null): bias of the V predictor, fp32-converted
-// on the fly, added to dropped heads ([D - m] in storage dtype).
+// on the fly, added to dropped heads ([D - m] in storage dtype) with the predicted tokens' share of the probability.
+// extra_recon_part = 1: the dropped heads have one more partial, their last, over the sink / window tokens.
+// bk_shift (may be null): bias of the K predictor where the kernels left it out of the scores; it then moves the
+// predicted partials of a head by q . b_k against that sink / window partial (without one it cancels).
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
                          const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-                         const void* bv, cudaStream_t stream, int extra_recon_part = 0);
+                         const void* bv, cudaStream_t stream, int extra_recon_part = 0,
+                         const void* bk_shift = nullptr);
 
 }  // namespace echokv

@@ -815,7 +815,7 @@ template <typename T>
 __global__ void __launch_bounds__(128 * kMergeGroups)
 merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stored_parts,
              const int32_t* __restrict__ stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-             const T* __restrict__ bv, int extra_recon_part) {
+             const T* __restrict__ bv, const T* __restrict__ bk_shift, int extra_recon_part) {
   const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x, grp = threadIdx.y;
   const int DH = a.head_dim;                      // == blockDim.x
   const int tid = grp * DH + j, n_threads = DH * kMergeGroups;
@@ -842,55 +842,79 @@ merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stor
   const size_t base = ((size_t)b * a.n_q_heads + h) * a.parts.max_parts;
   __shared__ float s_max[16];
   __shared__ float s_l[kMergeGroups];
+  __shared__ float s_l_side[kMergeGroups];
   __shared__ float s_acc[kMergeGroups][128];
+  // (the sink / window partial of a predicted head is its last one: those tokens' keys and values are the true ones)
+  const int side_part = (!stored && extra_recon_part) ? n - 1 : -1;
+  // A bias on the K predictor shifts the scores of a head's predicted tokens by q . b_k: it cancels in the softmax
+  // unless sink / window tokens, whose keys are not predicted, take part; then the predicted partials move by it.
+  // (bk_shift is null when nothing has to move, and when the kernels added the bias themselves: rotated keys.)
+  float shift = 0.f;
+  if (bk_shift != nullptr && side_part >= 0) {
+    __shared__ float s_dot[4];
+    const T* qrow = reinterpret_cast<const T*>(a.q) + ((size_t)b * a.n_q_heads + h) * DH;
+    float d = grp == 0 ? to_f32(qrow[j]) * to_f32(bk_shift[(kvh - n_stored_heads) * DH + j]) : 0.f;
+    d = warp_sum(d);
+    if (grp == 0 && (j & 31) == 0) s_dot[j >> 5] = d;
+    __syncthreads();
+    for (int w = 0; w < DH / 32; ++w) shift += s_dot[w];
+    shift *= a.scale_log2e;
+  }
   // pass 1: the largest partial maximum, all threads of the block together
   float m = -INFINITY;
-  for (int p = tid; p < n; p += n_threads) m = fmaxf(m, a.parts.ml[base + p].x);
+  for (int p = tid; p < n; p += n_threads) m = fmaxf(m, a.parts.ml[base + p].x + (p == side_part ? 0.f : shift));
   m = warp_max(m);
   if ((tid & 31) == 0) s_max[tid >> 5] = m;
   __syncthreads();
   float M = -INFINITY;
   for (int w = 0; w < n_threads / 32; ++w) M = fmaxf(M, s_max[w]);
   // pass 2: each group sums every kMergeGroups-th partial
-  float L = 0.f, acc = 0.f;
+  float L = 0.f, L_side = 0.f, acc = 0.f;
   if (M > -INFINITY) {
 #pragma unroll 4
     for (int p = grp; p < n; p += kMergeGroups) {
       const float2 ml = a.parts.ml[base + p];
-      const float w = exp2f(ml.x - M);
+      const float w = exp2f(ml.x + (p == side_part ? 0.f : shift) - M);
       L = fmaf(w, ml.y, L);
+      if (p == side_part) L_side = w * ml.y;
       acc = fmaf(w, a.parts.o[(base + p) * DH + j], acc);
     }
   }
   s_acc[grp][j] = acc;
-  if (j == 0) s_l[grp] = L;
+  if (j == 0) {
+    s_l[grp] = L;
+    s_l_side[grp] = L_side;
+  }
   __syncthreads();
   if (grp != 0) return;
 #pragma unroll
   for (int k = 1; k < kMergeGroups; ++k) {
     acc += s_acc[k][j];
     L += s_l[k];
+    L_side += s_l_side[k];
   }
   float res = L > 0.f ? acc / L : 0.f;
-  // a bias on the V predictor shifts every predicted V row alike, so (sum_t p_t = 1) it adds
-  // to the output unchanged; a bias on the K predictor shifts all scores of a head by the
-  // same amount and cancels in the softmax.
-  if (bv != nullptr && !stored) res += to_f32(bv[(kvh - n_stored_heads) * DH + j]);
+  // A bias on the V predictor shifts every predicted V row alike, so it adds to the output weighted by the
+  // probability of the predicted tokens: all of it (sum_t p_t = 1) unless sink / window tokens, whose values are not
+  // predicted, take their share.  A bias on the K predictor shifts all scores of a head by the same amount and
+  // cancels in the softmax (without a rotation).
+  if (bv != nullptr && !stored && L > 0.f) res += to_f32(bv[(kvh - n_stored_heads) * DH + j]) * ((L - L_side) / L);
   out[oidx] = res;
 }
 
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
                          const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-                         const void* bv, cudaStream_t stream, int extra_recon_part) {
+                         const void* bv, cudaStream_t stream, int extra_recon_part, const void* bk_shift) {
   dim3 grid(a.n_q_heads, a.batch);
   if (a.dtype == ECHOKV_BF16) {
     merge_kernel<__nv_bfloat16><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(
         a, out, n_stored_heads, n_stored_parts, stored_item_tokens, stored_batch_per_slot, part_tokens,
-        (const __nv_bfloat16*)bv, extra_recon_part);
+        (const __nv_bfloat16*)bv, (const __nv_bfloat16*)bk_shift, extra_recon_part);
   } else {
     merge_kernel<float><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(a, out, n_stored_heads, n_stored_parts,
                                                          stored_item_tokens, stored_batch_per_slot,
-                                                         part_tokens, (const float*)bv, extra_recon_part);
+                                                         part_tokens, (const float*)bv, (const float*)bk_shift,
+                                                         extra_recon_part);
   }
   return cudaGetLastError();
 }

@@ -63,14 +63,17 @@ def test_rope_against_oracle(name, base, over, lens, window):
     case.close()
 
 
-@pytest.mark.parametrize("base,over,lens", [
-    (synth.C2, dict(batch=2, context=600), [600, 131]),
-    (synth.C0, dict(batch=2, context=200), [200, 50]),
-], ids=["bf16_gqa", "fp32_d64"])
-def test_rope_with_predictor_biases(base, over, lens):
+@pytest.mark.parametrize("base,over,lens,window", [
+    (synth.C2, dict(batch=2, context=600), [600, 131], None),
+    (synth.C0, dict(batch=2, context=200), [200, 50], None),
+    (synth.C2, dict(batch=2, context=600, n_q_heads=16, n_retained_heads=5, page_tokens=64), [600, 107], (0, 16)),
+    (synth.C0, dict(batch=2, context=200), [200, 50], (2, 16)),
+], ids=["bf16_gqa", "fp32_d64", "bf16_gqa2_window", "fp32_d64_window"])
+def test_rope_with_predictor_biases(base, over, lens, window):
     # a bias on the K predictor is rotated with the predicted keys: it does not cancel in the softmax any more
+    # (with sink / window tokens a V bias reaches the output only with the predicted tokens' share of the probability)
     w = base.replace(**over)
-    case = Case(w, lens=lens, layers=[0, 1], biases=True, rope=THETA)
+    case = Case(w, lens=lens, layers=[0, 1], biases=True, rope=THETA, window=window)
     ref = case.oracle(1)
     for path in ([1, 2, 3] if case.ctx.decode_path() >= 2 else [1]):
         case.ctx.set_decode_path(path)
@@ -89,6 +92,7 @@ MIXED = [
     ("pages64_random", synth.C2, dict(batch=2, context=600, page_tokens=64, random_pages=True), [600, 65], None, False),
     ("ragged_many_tiles", synth.C2, dict(batch=5, context=2000, random_pages=True), [2000, 129, 128, 1153, 1], None, True),
     ("window", synth.C2, dict(batch=3, context=1000, random_pages=True), [1000, 517, 100], (4, 128), False),
+    ("window_biases", synth.C2, dict(batch=2, context=700), [700, 150], (4, 128), True),
     ("nothing_retained", synth.C2, dict(batch=2, context=700, n_retained_heads=0), [700, 300], None, True),
     ("one_dropped_head", synth.C2, dict(batch=2, context=400, n_retained_heads=7), [400, 258], (2, 40), False),
 ]

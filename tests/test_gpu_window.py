@@ -32,10 +32,14 @@ CASES = [
 ]
 
 
+# biases: Eq. 3 with the optional bias vectors.  With sink / window tokens a K bias no longer cancels in the softmax
+# (it shifts the scores of the predicted tokens only) and a V bias reaches the output only with the predicted
+# tokens' share of the probability.
+@pytest.mark.parametrize("biases", [False, True], ids=["no_bias", "biases"])
 @pytest.mark.parametrize("name,base,over,lens,window", CASES, ids=[c[0] for c in CASES])
-def test_window_against_oracle(name, base, over, lens, window):
+def test_window_against_oracle(name, base, over, lens, window, biases):
     w = base.replace(**over)
-    case = Case(w, lens=lens, layers=[0, 1], window=window)
+    case = Case(w, lens=lens, layers=[0, 1], window=window, biases=biases)
     paths = [1, 2, 3] if case.ctx.decode_path() >= 2 else [1]
     for path in paths:
         case.ctx.set_decode_path(path)
