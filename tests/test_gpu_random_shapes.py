@@ -1,0 +1,121 @@
+"""GPU parity on drawn configurations: shapes, lengths, page sizes and orders, group sizes, retained heads and the
+option combinations (sink / window tokens, rotation, biases, absorbed predictors, keys kept whole, a retained-dim count
+that ends inside a head, fp32) are drawn from a seeded generator, so that combinations nobody listed by hand are
+compared with the oracle too.  (A run of this kind found the bias x sink / window cases.)"""
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_22910_b200 import binding, build, synth
+from tests.harness import TOL, Case, errors
+from tests.test_gpu_prefill import TOL_PREFILL, oracle_prefill, queries
+
+pytestmark = pytest.mark.gpu
+
+THETA = 10000.0
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.lib()
+
+
+def draw_heads(rnd):
+    """(group size, KV heads) with 16, 32 or 64 query heads."""
+    while True:
+        g = rnd.choice([1, 2, 4, 8])
+        n_kv = rnd.choice([4, 8]) if g > 1 else rnd.choice([8, 16, 32])
+        if n_kv * g in (16, 32, 64):
+            return g, n_kv
+
+
+@pytest.mark.parametrize("seed", [101, 102, 103])
+def test_decode_drawn_configurations(seed):
+    rnd = random.Random(seed)
+    checked = 0
+    for k in range(14):
+        g, n_kv = draw_heads(rnd)
+        r = rnd.randrange(0, n_kv + 1)
+        B = rnd.choice([1, 2, 4])
+        context = rnd.randrange(20, 1200)
+        lens = [context] + [rnd.randrange(1, context + 1) for _ in range(B - 1)]
+        pt = rnd.choice([16, 16, 32, 64, 128])
+        rope = THETA if rnd.random() < 0.35 else None
+        window = rnd.choice([(4, 128), (0, 16), (3, 0)]) if rnd.random() < 0.35 else None
+        absorbed = rnd.random() < 0.4
+        save_k = rnd.random() < 0.15 and 0 < r < n_kv and not window
+        absorbed = absorbed or save_k
+        ragged = 0
+        if absorbed and not save_k and not rope and not window and rnd.random() < 0.3:
+            ragged = 64 * rnd.randrange(1, n_kv * 2)
+        fp32 = rnd.random() < 0.12 and not absorbed
+        biases = rnd.random() < 0.4
+        w = (synth.C2 if g > 1 else synth.C1).replace(
+            batch=B, context=context, n_q_heads=n_kv * g, n_kv_heads=n_kv, n_retained_heads=r, page_tokens=pt,
+            random_pages=rnd.random() < 0.5, save_k=save_k, seed=seed * 100 + k, n_layers=3,
+            group_size=rnd.choice([2, 3]), n_retained_dims=ragged)
+        if fp32:
+            lens = [min(l, 300) for l in lens]
+            w = w.replace(dtype="fp32", head_dim=rnd.choice([64, 128]), context=max(lens), page_tokens=16)
+        what = dict(seed=seed, k=k, g=g, n_kv=n_kv, r=r, lens=lens, pt=w.page_tokens, rope=bool(rope), window=window,
+                    absorbed=absorbed, save_k=save_k, ragged=ragged, fp32=fp32, biases=biases)
+        try:
+            case = Case(w, lens=lens, layers=[0, 1, 2], biases=biases, window=window, rope=rope)
+            if absorbed and w.m < w.D:
+                case.ctx.enable_absorbed()
+        except binding.EchoKVError as e:      # a combination the library declines when the context is made
+            assert e.status == binding.ECHOKV_EUNSUPPORTED, what
+            continue
+        tol = TOL[w.dtype]
+        for layer in (0, 1, 2):
+            out = case.run(layer, full=w.is_anchor(layer))
+            assert np.all(np.isfinite(out)), what
+            max_abs, rel_l2 = errors(out, case.oracle(layer))
+            assert max_abs <= tol["max_abs"] and rel_l2 <= tol["rel_l2"], (what, layer, max_abs, rel_l2)
+        assert case.ctx.device_status() == binding.ECHOKV_OK, what
+        case.close()
+        checked += 1
+    assert checked >= 8
+
+
+@pytest.mark.parametrize("seed", [201, 202])
+def test_prefill_drawn_configurations(seed):
+    rnd = random.Random(seed)
+    checked = 0
+    for k in range(12):
+        g, n_kv = draw_heads(rnd)
+        r = rnd.randrange(0, n_kv)
+        B = rnd.choice([1, 2, 3])
+        context = rnd.randrange(40, 700)
+        lens = [context] + [rnd.randrange(1, context + 1) for _ in range(B - 1)]
+        n_q = rnd.randrange(1, min(lens) + 1)
+        if rnd.random() < 0.5:
+            n_q = min(n_q, rnd.choice([1, 7, 32, 33, 64, 65, 128, 129]))
+        rope = THETA if rnd.random() < 0.4 else None
+        save_k = rnd.random() < 0.2 and r > 0
+        w = (synth.C2 if g > 1 else synth.C1).replace(
+            batch=B, context=context, n_q_heads=n_kv * g, n_kv_heads=n_kv, n_retained_heads=r,
+            page_tokens=rnd.choice([16, 16, 32, 64]), random_pages=rnd.random() < 0.5, save_k=save_k, seed=seed * 100 + k)
+        what = dict(seed=seed, k=k, g=g, n_kv=n_kv, r=r, lens=lens, n_q=n_q, pt=w.page_tokens, rope=bool(rope), save_k=save_k)
+        try:
+            case = Case(w, lens=lens, layers=[0, 1], biases=rnd.random() < 0.3, rope=rope)
+        except binding.EchoKVError as e:
+            assert e.status == binding.ECHOKV_EUNSUPPORTED, what
+            continue
+        for layer in (1, 0):
+            q = queries(w, n_q, layer)
+            out = case.ctx.prefill_attention(layer, q.to(case.ctx.device), case.seq_lens)
+            torch.cuda.synchronize()
+            out = out.cpu().numpy().astype(np.float64)
+            assert np.all(np.isfinite(out)), what
+            for b in range(B):
+                max_abs, rel_l2 = errors(out[b], oracle_prefill(case, layer, q, b, rope))
+                assert max_abs <= TOL_PREFILL["max_abs"] and rel_l2 <= TOL_PREFILL["rel_l2"], (what, layer, b, max_abs, rel_l2)
+        assert case.ctx.device_status() == binding.ECHOKV_OK, what
+        case.close()
+        checked += 1
+    assert checked >= 8
