@@ -119,3 +119,54 @@ def test_prefill_drawn_configurations(seed):
         case.close()
         checked += 1
     assert checked >= 8
+
+
+@pytest.mark.parametrize("seed", [301, 302])
+def test_many_decode_steps_with_a_turning_window(seed):
+    """Tokens are appended through the library for tens of steps (the recent-window ring turns over several times, the
+    sink fills up) and the result is compared with the oracle every few steps."""
+    rnd = random.Random(seed)
+    for k in range(5):
+        g, n_kv = rnd.choice([2, 4]), 8
+        r = rnd.randrange(0, n_kv)
+        B = rnd.choice([1, 2, 3])
+        steps = rnd.randrange(20, 60)
+        lens = [rnd.randrange(1, 200) for _ in range(B)]
+        window = rnd.choice([(4, 128), (2, 5), (0, 16), (3, 0), (1, 33)])
+        rope = THETA if rnd.random() < 0.4 else None
+        absorbed = rnd.random() < 0.5
+        biases = rnd.random() < 0.5
+        w = synth.C2.replace(batch=B, context=max(lens) + steps, n_q_heads=n_kv * g, n_kv_heads=n_kv, n_retained_heads=r,
+                             page_tokens=rnd.choice([16, 32, 64]), random_pages=rnd.random() < 0.5, seed=seed * 100 + k)
+        what = dict(seed=seed, k=k, g=g, r=r, lens=lens, steps=steps, window=window, rope=bool(rope), absorbed=absorbed,
+                    biases=biases, pt=w.page_tokens)
+        case = Case(w, lens=lens, layers=[0, 1], biases=biases, window=window, rope=rope)
+        if absorbed:
+            case.ctx.enable_absorbed()
+        dev = case.ctx.device
+        full = {(l, kind, b): synth.layer_cache(w, l, kind, b, width=w.D)
+                for l in (0, 1) for kind in "kv" for b in range(B)}
+        tol = TOL[w.dtype]
+        for t in range(steps):
+            for l in (0, 1):
+                k_new = torch.stack([full[(l, "k", b)][lens[b]] for b in range(B)]).to(dev)
+                v_new = torch.stack([full[(l, "v", b)][lens[b]] for b in range(B)]).to(dev)
+                case.ctx.append_kv(l, k_new, v_new, torch.tensor(lens, dtype=torch.int32, device=dev))
+            lens = [n + 1 for n in lens]
+            if t % 7 != 3 and t != steps - 1:
+                continue
+            case.lens = list(lens)
+            case.seq_lens = torch.tensor(lens, dtype=torch.int32, device=dev)
+            for l in (0, 1):
+                width = w.D if w.is_anchor(l) else w.m
+                for kind in "kv":
+                    for b in range(B):
+                        if width:
+                            case.host[(l, kind, b)] = full[(l, kind, b)][:lens[b], :width]
+                        if l == 1:
+                            case.true_drop[(l, kind, b)] = full[(l, kind, b)][:lens[b], w.m:]
+            for l in (0, 1):
+                max_abs, rel_l2 = errors(case.run(l, full=w.is_anchor(l)), case.oracle(l))
+                assert max_abs <= tol["max_abs"] and rel_l2 <= tol["rel_l2"], (what, t, l, max_abs, rel_l2)
+            assert case.ctx.device_status() == binding.ECHOKV_OK, what
+        case.close()
