@@ -20,6 +20,9 @@
  *    the caller (e.g. by PyTorch); the library BORROWS it: it must stay valid until
  *    echokv_destroy().  "host pointer" = ordinary host memory, read during the call
  *    only, unless stated otherwise.  The library itself allocates no device memory.
+ *  - Alignment: pools, predictors, queries (q), new K / V rows (k_new, v_new), side buffers, scratch and
+ *    result buffers (out) must be 16-byte aligned -- the kernels move them 16 bytes at a time; workspaces
+ *    256-byte aligned.  A pointer aligned to less is refused with ECHOKV_EINVAL on the host, before any launch.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
  *    that take a stream only enqueue work on it and return; the *_host calls and
  *    echokv_get_device_status() synchronise.
@@ -347,7 +350,8 @@ int echokv_read_kernel_timing_by_kind(echokv_ctx* ctx, double* total_ms, int64_t
  *  - cfg describes the geometry (heads, head_dim, page_tokens, max_batch, max_pages_per_seq,
  *    n_pages, dtype, softmax_scale, device); n_layers, group_size, n_retained_heads are ignored.
  *    k_pool / v_pool: device pointers [n_pages][page_tokens][n_kv_heads * head_dim]; the other
- *    pointers as in echokv_full_attention.  dev_status_out: optional device int32 that receives
+ *    pointers as in echokv_full_attention (k_pool, v_pool, q and out 16-byte aligned, else EINVAL;
+ *    max_pages_per_seq * page_tokens at most 2^30).  dev_status_out: optional device int32 that receives
  *    the device status of this call (ECHOKV_OK, EBADPAGE, EBADLENGTH), stream-ordered.
  *  - It calls no cudaMalloc / cudaFree and no routine that allocates.  Makes cfg->device current.
  *  - The FIRST call on each device looks up the device address of the array; make that first

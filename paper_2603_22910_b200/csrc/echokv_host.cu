@@ -238,8 +238,12 @@ int append_side(echokv_ctx* c, const Layer& L, const void* k_new, const void* v_
   return ECHOKV_OK;
 }
 
+// The kernels read queries and new K / V rows with 16-byte loads and may store results 16 bytes at a time.
+inline bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
 int check_call(echokv_ctx* c, int layer, const void* q, const float* out, const int32_t* lens, int B) {
   if (!c || !q || !out || !lens) return ECHOKV_EINVAL;
+  if (!aligned16(q) || !aligned16(out)) return ECHOKV_EINVAL;
   if (layer < 0 || layer >= c->cfg.n_layers || B < 1) return ECHOKV_EINVAL;
   if (B > c->cfg.max_batch) return ECHOKV_ECAPACITY;
   if (!c->table) return ECHOKV_ENOTABLE;
@@ -552,6 +556,7 @@ int echokv_append_kv_chunk(echokv_ctx* c, int layer, const void* k_new, const vo
                            const int32_t* dev_seq_slots, const int32_t* dev_first_positions, int n_tokens, int B,
                            void* stream) {
   if (!c || !k_new || !v_new || !dev_first_positions) return ECHOKV_EINVAL;
+  if (!aligned16(k_new) || !aligned16(v_new)) return ECHOKV_EINVAL;
   if (layer < 0 || layer >= c->cfg.n_layers || B < 1 || n_tokens < 1) return ECHOKV_EINVAL;
   if (B > c->cfg.max_batch || n_tokens > c->d.capacity || n_tokens > 65535) return ECHOKV_ECAPACITY;
   if (!c->table) return ECHOKV_ENOTABLE;
@@ -696,8 +701,6 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     if (side) {
       aa.n_sink = c->n_sink; aa.n_window = c->n_window;
       aa.k_side = L.k_side; aa.v_side = L.v_side;
-      aa.k_local = L.k_pool; aa.v_local = L.v_pool;
-    aa.save_k = c->d.save_k;
     }
     cudaEvent_t ev[4];
     const bool timed = timed_pair(c, ECHOKV_TIMED_ABSORB_K, &ev[0], &ev[1]) &&

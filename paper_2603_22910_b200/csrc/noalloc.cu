@@ -5,6 +5,7 @@
 // execution callback where device allocation is forbidden, or a host thread that is only handed
 // raw pointers to an arena sized long ago.  For them this file keeps the scratch in a fixed
 // device array that is part of the library image.  The paper has no counterpart to this.
+#include <cmath>
 #include <mutex>
 
 #include "kernels.h"
@@ -63,7 +64,14 @@ extern "C" int echokv_full_attention_noalloc(const echokv_config* cfg, const voi
   if (cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads != 0) return ECHOKV_EINVAL;
   if (cfg->max_batch < 1 || cfg->max_pages_per_seq < 1 || cfg->n_pages < 1 || B < 1) return ECHOKV_EINVAL;
   if (cfg->dtype != ECHOKV_BF16 && cfg->dtype != ECHOKV_FP32) return ECHOKV_EINVAL;
-  if (!(cfg->softmax_scale >= 0.f)) return ECHOKV_EINVAL;
+  if (!(cfg->softmax_scale >= 0.f) || !std::isfinite(cfg->softmax_scale)) return ECHOKV_EINVAL;
+  // a capacity beyond 2^30 tokens would overflow the kernels' int arithmetic on lengths
+  if ((long long)cfg->max_pages_per_seq * cfg->page_tokens > (1ll << 30)) return ECHOKV_EINVAL;
+  // the kernel reads the pools and the queries with 16-byte loads: a pointer aligned to less would fault on
+  // the device instead of returning a status
+  if ((reinterpret_cast<uintptr_t>(k_pool) | reinterpret_cast<uintptr_t>(v_pool) | reinterpret_cast<uintptr_t>(q) |
+       reinterpret_cast<uintptr_t>(out)) % 16 != 0)
+    return ECHOKV_EINVAL;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return ECHOKV_EUNSUPPORTED;
   if (cfg->page_tokens != 16 && cfg->page_tokens != 32 && cfg->page_tokens != 64 && cfg->page_tokens != 128)
     return ECHOKV_EUNSUPPORTED;

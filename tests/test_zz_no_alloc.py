@@ -71,3 +71,72 @@ def test_noalloc_rejects_what_does_not_fit_the_fixed_scratch():
                                              None) == binding.ECHOKV_EINVAL
     assert lib.echokv_full_attention_noalloc(C.byref(cfg), 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, None, 0x1000,
                                              2048, None, None) == binding.ECHOKV_ECAPACITY
+
+
+def test_noalloc_rejects_misaligned_pointers_and_overflowing_geometry_on_the_host():
+    """Fake pointers only: every one of these must be refused before any CUDA call is made."""
+    build.build()
+    lib = binding.lib()
+    cfg = binding.config_for(synth.C2.replace(batch=2, context=64))
+    ok = [0x1000, 0x1000, 0x1000, 0x1000, 0x1000]          # k_pool, v_pool, table, q, out
+    for i in (0, 1, 3, 4):                                 # a pointer aligned to 4 bytes only
+        args = list(ok)
+        args[i] = 0x1004
+        rc = lib.echokv_full_attention_noalloc(C.byref(cfg), *args, None, 0x1000, 1, None, None)
+        assert rc == binding.ECHOKV_EINVAL, i
+    big = binding.config_for(synth.C2.replace(batch=2, context=64))
+    big.max_pages_per_seq = (1 << 30) // big.page_tokens + 1       # capacity beyond 2^30 tokens
+    assert lib.echokv_full_attention_noalloc(C.byref(big), *ok, None, 0x1000, 1, None, None) == binding.ECHOKV_EINVAL
+    inf = binding.config_for(synth.C2.replace(batch=2, context=64))
+    inf.softmax_scale = float("inf")
+    assert lib.echokv_full_attention_noalloc(C.byref(inf), *ok, None, 0x1000, 1, None, None) == binding.ECHOKV_EINVAL
+
+
+@pytest.mark.gpu
+def test_noalloc_with_fewer_splits_than_it_would_like():
+    """Many short sequences: 4 * SMs / (B * H_kv) splits do not fit the 8 MiB, so the split count is cut."""
+    build.build()
+    w = synth.C2.replace(batch=400, context=64)
+    lens = [1 + (7 * i) % 64 for i in range(w.batch)]
+    case = Case(w, lens=lens, layers=[0])
+    ctx, dev = case.ctx, case.ctx.device
+    tol = TOL["bf16"]
+    q = case.q[0].to(dev)
+    ref = ctx.full_attention(0, q, case.seq_lens)
+    status = torch.full((1,), 99, dtype=torch.int32, device=dev)
+    for _ in range(2):
+        out = torch.full_like(ref, float("nan"))
+        binding.echokv_full_attention_noalloc(case.cfg, ctx.k_pools[0], ctx.v_pools[0], ctx.block_table,
+                                              q, out, case.seq_lens, status_out=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == binding.ECHOKV_OK
+        max_abs, rel_l2 = errors(out.cpu().numpy(), ref.cpu().numpy())
+        assert max_abs <= tol["max_abs"] and rel_l2 <= tol["rel_l2"], (max_abs, rel_l2)
+    max_abs, rel_l2 = errors(out.cpu().numpy(), case.oracle(0))
+    assert max_abs <= tol["max_abs"] and rel_l2 <= tol["rel_l2"], (max_abs, rel_l2)
+    case.close()
+
+
+@pytest.mark.gpu
+def test_noalloc_fp32_head_dim_64_with_sequence_slots():
+    build.build()
+    w = synth.C0.replace(batch=3, context=200)
+    case = Case(w, lens=[200, 77, 130], layers=[0])
+    ctx, dev = case.ctx, case.ctx.device
+    tol = TOL["fp32"]
+    # rows of the block table taken in another order: sequence i of the call lives in slot slots[i]
+    slots = torch.tensor([2, 0, 1], dtype=torch.int32, device=dev)
+    q = case.q[0].to(dev)[slots.long()].contiguous()
+    lens = case.seq_lens[slots.long()].contiguous()
+    ref = ctx.full_attention(0, q, lens, seq_slots=slots)
+    for _ in range(2):
+        out = torch.full_like(ref, float("nan"))
+        binding.echokv_full_attention_noalloc(case.cfg, ctx.k_pools[0], ctx.v_pools[0], ctx.block_table,
+                                              q, out, lens, seq_slots=slots)
+        torch.cuda.synchronize()
+        max_abs, rel_l2 = errors(out.cpu().numpy(), ref.cpu().numpy())
+        assert max_abs <= tol["max_abs"] and rel_l2 <= tol["rel_l2"], (max_abs, rel_l2)
+    want = case.oracle(0)[slots.cpu().numpy()]
+    max_abs, rel_l2 = errors(out.cpu().numpy(), want)
+    assert max_abs <= tol["max_abs"] and rel_l2 <= tol["rel_l2"], (max_abs, rel_l2)
+    case.close()
