@@ -40,7 +40,10 @@ force, torch scaled_dot_product_attention (library routine) for the m = D and
 selector-weight cases, zero-weight closed forms, linearity, softmax shift /
 permutation / log-sum-exp merge invariants, the paper's printed predictor
 shapes, ratios and parameter totals; for the rotation: hand values, the complex-
-number form, a library rotary routine, and the relative-position property.  What stays "parity unpinned": nothing in
+number form, a library rotary routine, and the relative-position property; for an m that splits a
+head, whole keys with a window, and the prefill-shaped call with a sink / window: index-by-index brute
+force, the windowed decode step on every prefix, causal library attention in the all-true limit, and a
+planted mistake.  What stays "parity unpinned": nothing in
 the paper prints a numeric attention output, and how well a *trained* W
 approximates the dropped cache cannot be checked without trained weights (it is
 not part of what the kernels compute).
@@ -280,13 +283,17 @@ def decode_attention_query_heads(q: np.ndarray,
                                  Wk: np.ndarray, Wv: np.ndarray,
                                  n_kv_heads: int, query_heads, scale: float | None = None,
                                  k_true_drop=None, v_true_drop=None, n_sink: int = 0, n_window: int = 0,
-                                 rope_theta: float | None = None) -> dict[int, np.ndarray]:
-    """The same quantity as decode_attention, for a chosen few query heads only.
+                                 rope_theta: float | None = None, k_true=None,
+                                 bk=None, bv=None) -> dict[int, np.ndarray]:
+    """The same quantity as decode_attention (or decode_attention_windowed, when a sink / window
+    is given), for a chosen few query heads only.
 
     Heads are independent in Eq. 7 and each dropped flat dim is one row of W in
-    Eq. 3, so for query head h only the d rows of W that produce KV head kv(h)
-    are evaluated.  Used to check sampled outputs of workloads too large to run
-    in full.  Returns {h: out[h] as [d]}.
+    Eq. 3, so for query head h only the rows of W that produce dims of KV head kv(h)
+    are evaluated.  Eq. 6 concatenates at the flat index m, wherever that falls: of a
+    head that m splits, the dims below m are the stored ones and the rest are predicted.
+    k_true [L, D]: the "save K" setting (keys whole, used as they are).
+    Used to check sampled outputs of workloads too large to run in full.  Returns {h: out[h] as [d]}.
     """
     q = np.asarray(q, dtype=np.float64)
     k_global = np.asarray(k_global, dtype=np.float64)
@@ -295,27 +302,36 @@ def decode_attention_query_heads(q: np.ndarray,
     v_local = np.asarray(v_local, dtype=np.float64)
     H_q, d = q.shape
     D = k_global.shape[1]
-    m = k_local.shape[1]
+    m = v_local.shape[1]
+    L = k_global.shape[0]
     g = H_q // n_kv_heads
     if scale is None:
         scale = 1.0 / math.sqrt(d)
+    keep = full_precision_tokens(L, n_sink, n_window) if (n_sink or n_window) else None
+
+    def head_dims(c_global, c_local, W, bias, c_true_drop, lo):
+        """Flat dims [lo, lo + d) of the rebuilt cache: [L, d]."""
+        n_stored = min(max(m - lo, 0), d)             # dims of this head below m: stored
+        parts = [c_local[:, lo:lo + n_stored]]
+        if n_stored < d:                              # the rest: rows of W (Eq. 3)
+            rows = slice(lo + n_stored - m, lo + d - m)
+            pred = predictor_input(c_global, c_local) @ np.asarray(W, dtype=np.float64)[rows].T
+            if bias is not None:
+                pred = pred + np.asarray(bias, dtype=np.float64)[rows]
+            if keep is not None:                      # sink / window tokens keep their true dims
+                pred = overlay_true_dims(pred, np.asarray(c_true_drop, dtype=np.float64)[:, rows], keep)
+            parts.append(pred)
+        return np.concatenate(parts, axis=1)
+
     out = {}
     for h in query_heads:
         kv = h // g
         lo = kv * d                                   # flat dims [lo, lo + d) of K_tilde
-        if lo + d <= m:                               # a retained head: stored values
-            K_h = k_local[:, lo:lo + d]
-            V_h = v_local[:, lo:lo + d]
-        elif lo >= m:                                 # a dropped head: rows lo-m .. of W
-            rows = slice(lo - m, lo - m + d)
-            K_h = predictor_input(k_global, k_local) @ np.asarray(Wk, dtype=np.float64)[rows].T
-            V_h = predictor_input(v_global, v_local) @ np.asarray(Wv, dtype=np.float64)[rows].T
-            if n_sink or n_window:       # sink / window tokens keep their true dims
-                keep = full_precision_tokens(K_h.shape[0], n_sink, n_window)
-                K_h = overlay_true_dims(K_h, np.asarray(k_true_drop, dtype=np.float64)[:, rows], keep)
-                V_h = overlay_true_dims(V_h, np.asarray(v_true_drop, dtype=np.float64)[:, rows], keep)
+        if k_true is not None:
+            K_h = np.asarray(k_true, dtype=np.float64)[:, lo:lo + d]
         else:
-            raise ValueError("m must be head-aligned for per-head evaluation")
+            K_h = head_dims(k_global, k_local, Wk, bk, k_true_drop, lo)
+        V_h = head_dims(v_global, v_local, Wv, bv, v_true_drop, lo)
         if rope_theta is not None:
             K_h = rotate_keys(K_h[:, None, :], rope_theta)[:, 0, :]
         s = (K_h @ q[h]) * scale
@@ -351,20 +367,28 @@ def overlay_true_dims(c_hat_drop: np.ndarray, c_true_drop: np.ndarray, keep: np.
 def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n_kv_heads: int,
                               k_true_drop, v_true_drop, n_sink: int, n_window: int,
                               scale: float | None = None, bk=None, bv=None,
-                              rope_theta: float | None = None) -> np.ndarray:
+                              rope_theta: float | None = None, k_true=None) -> np.ndarray:
     """decode_attention with the sink and recent-window tokens at full precision:
     for those tokens the dropped dims come from k_true_drop / v_true_drop ([L, D - m],
-    the layer's own dims m..D-1), for all others from Eq. 3.  Returns [H_q, d]."""
+    the layer's own dims m..D-1), for all others from Eq. 3.  With k_true [L, D] (the
+    "save K" setting of Section 5.2) the keys are whole anyway and used as they are
+    (k_local, Wk, bk, k_true_drop are ignored); the window then matters to the values only.
+    Returns [H_q, d]."""
     q = np.asarray(q, dtype=np.float64)
     d = q.shape[1]
     L = np.asarray(k_global).shape[0]
     if L < 1:
         raise ValueError("empty cache: softmax over no token is undefined")
     keep = full_precision_tokens(L, n_sink, n_window)
-    k_drop = overlay_true_dims(reconstruct_dropped(Wk, k_global, k_local, bk), k_true_drop, keep)
+    if k_true is not None:
+        K_t = np.asarray(k_true, dtype=np.float64).reshape(-1, n_kv_heads, d)
+        if K_t.shape[0] != L:
+            raise ValueError("token counts differ")
+    else:
+        k_drop = overlay_true_dims(reconstruct_dropped(Wk, k_global, k_local, bk), k_true_drop, keep)
+        K_t = assemble_cache(k_local, k_drop, n_kv_heads, d)
     v_drop = overlay_true_dims(reconstruct_dropped(Wv, v_global, v_local, bv), v_true_drop, keep)
-    return attention(q, assemble_cache(k_local, k_drop, n_kv_heads, d),
-                     assemble_cache(v_local, v_drop, n_kv_heads, d), scale, rope_theta)
+    return attention(q, K_t, assemble_cache(v_local, v_drop, n_kv_heads, d), scale, rope_theta)
 
 
 # ----------------------------------------------------------------------------
@@ -375,13 +399,19 @@ def decode_attention_windowed(q, k_global, v_global, k_local, v_local, Wk, Wv, n
 
 def prefill_attention(q: np.ndarray, k_global, v_global, k_local, v_local, Wk, Wv, n_kv_heads: int,
                       scale: float | None = None, bk=None, bv=None, rope_theta: float | None = None,
-                      k_true=None) -> np.ndarray:
+                      k_true=None, k_true_drop=None, v_true_drop=None, n_sink: int = 0,
+                      n_window: int = 0) -> np.ndarray:
     """q [n_q, H_q, d]: queries of the last n_q of the L cached tokens; query i sits at position
     L - n_q + i and attends the tokens up to and including its own (causal).  The cache of a
     compressed layer is rebuilt once (Eq. 3, Eq. 6) and each query evaluates Eq. 7 over its prefix.
     With Wk = Wv = None the layer holds its full cache (k_global, v_global are used as they are:
     an anchor layer).  k_true [L, D]: the "save K" setting of Section 5.2, as in decode_attention
-    (keys whole and used as they are; only the values are predicted).  Returns [n_q, H_q, d]."""
+    (keys whole and used as they are; only the values are predicted).
+    With a sink / window (Section 4.1) every query is the decode step of the sequence cut off at its
+    own position: of ITS prefix the first n_sink and the last n_window tokens are at full precision
+    (k_true_drop, v_true_drop [L, D - m] as in decode_attention_windowed), so a token is read at full
+    precision by the queries at most n_window - 1 positions after it and as predicted by the later ones.
+    Returns [n_q, H_q, d]."""
     q = np.asarray(q, dtype=np.float64)
     n_q, H_q, d = q.shape
     k_global = np.asarray(k_global, dtype=np.float64)
@@ -389,23 +419,42 @@ def prefill_attention(q: np.ndarray, k_global, v_global, k_local, v_local, Wk, W
     L = k_global.shape[0]
     if n_q < 1 or n_q > L:
         raise ValueError("need 1 <= n_q <= L")
+    windowed = (n_sink > 0 or n_window > 0) and not (Wk is None and Wv is None)
+    if windowed:
+        k_local = np.asarray(k_local, dtype=np.float64)
+        v_local = np.asarray(v_local, dtype=np.float64)
     if Wk is None and Wv is None:
         K_t = k_global.reshape(L, n_kv_heads, d)
         V_t = v_global.reshape(L, n_kv_heads, d)
     else:
+        v_hat = reconstruct_dropped(Wv, v_global, v_local, bv)
         if k_true is not None:
             K_t = np.asarray(k_true, dtype=np.float64).reshape(-1, n_kv_heads, d)
             if K_t.shape[0] != L:
                 raise ValueError("token counts differ")
+            k_hat = None
         else:
-            K_t = assemble_cache(k_local, reconstruct_dropped(Wk, k_global, k_local, bk), n_kv_heads, d)
-        V_t = assemble_cache(v_local, reconstruct_dropped(Wv, v_global, v_local, bv), n_kv_heads, d)
-    if rope_theta is not None:
+            k_hat = reconstruct_dropped(Wk, k_global, k_local, bk)
+            K_t = assemble_cache(k_local, k_hat, n_kv_heads, d)
+        V_t = assemble_cache(v_local, v_hat, n_kv_heads, d)
+    if rope_theta is not None and not windowed:
         K_t = rotate_keys(K_t, rope_theta)
     out = np.empty((n_q, H_q, d), dtype=np.float64)
     for i in range(n_q):
         n_seen = L - n_q + i + 1
-        out[i] = attention(q[i], K_t[:n_seen], V_t[:n_seen], scale)
+        if windowed:
+            # this query's own sink and window, on its own prefix
+            keep = full_precision_tokens(n_seen, n_sink, n_window)
+            V_i = assemble_cache(v_local[:n_seen], overlay_true_dims(v_hat[:n_seen], np.asarray(v_true_drop)[:n_seen], keep),
+                                 n_kv_heads, d)
+            if k_hat is None:
+                K_i = K_t[:n_seen]
+            else:
+                K_i = assemble_cache(k_local[:n_seen],
+                                     overlay_true_dims(k_hat[:n_seen], np.asarray(k_true_drop)[:n_seen], keep), n_kv_heads, d)
+            out[i] = attention(q[i], K_i, V_i, scale, rope_theta)
+        else:
+            out[i] = attention(q[i], K_t[:n_seen], V_t[:n_seen], scale)
     return out
 
 

@@ -18,9 +18,11 @@ def rng(seed):
     return np.random.default_rng(seed)
 
 
-def rand_case(seed, L=37, H_q=8, H_kv=4, d=8, r=1):
+def rand_case(seed, L=37, H_q=8, H_kv=4, d=8, r=1, m=None):
+    """m, when given, is the retained width in flat dims and need not end on a head boundary."""
     g = rng(seed)
-    D, m = H_kv * d, r * d
+    D = H_kv * d
+    m = r * d if m is None else m
     return dict(
         q=g.standard_normal((H_q, d)),
         kg=g.standard_normal((L, D)), vg=g.standard_normal((L, D)),
@@ -525,24 +527,25 @@ def run_windowed(c, kt, vt, n_sink, n_window, scale=None):
                                        kt, vt, n_sink, n_window, scale)
 
 
-def brute_force_windowed(c, kt, vt, n_sink, n_window):
-    """Index by index: a sink / window token reads its stored dims, any other token the predicted ones."""
+def brute_force_windowed(c, kt, vt, n_sink, n_window, all_keys_true=False):
+    """Index by index: a sink / window token reads its stored dims, any other token the predicted ones.
+    all_keys_true: every token's key dims m..D-1 are read from kt (keys kept whole)."""
     q, kg, vg, kl, vl, Wk, Wv = (c[k].tolist() for k in ("q", "kg", "vg", "kl", "vl", "Wk", "Wv"))
     H_q, H_kv, d, m, D, L = c["H_q"], c["H_kv"], c["d"], c["m"], c["D"], c["L"]
     grp = H_q // H_kv
 
-    def value(glob, loc, W, true, t, flat):
+    def value(glob, loc, W, true, t, flat, always_true=False):
         if flat < m:
             return loc[t][flat]
-        if t < n_sink or t > L - 1 - n_window:
+        if always_true or t < n_sink or t > L - 1 - n_window:
             return true[t][flat - m]
         row = W[flat - m]
         return math.fsum([row[i] * glob[t][i] for i in range(D)] + [row[D + i] * loc[t][i] for i in range(m)])
     out = []
     for h in range(H_q):
         kv = h // grp
-        s = [math.fsum(q[h][j] * value(kg, kl, Wk, kt.tolist(), t, kv * d + j) for j in range(d)) / math.sqrt(d)
-             for t in range(L)]
+        s = [math.fsum(q[h][j] * value(kg, kl, Wk, kt.tolist(), t, kv * d + j, all_keys_true) for j in range(d))
+             / math.sqrt(d) for t in range(L)]
         mx = max(s)
         e = [math.exp(v - mx) for v in s]
         z = math.fsum(e)
@@ -601,3 +604,152 @@ def test_windowed_planted_mistakes_are_caught(monkeypatch):
             lambda: test_windowed_brute_force_tiny(13, 8, 6, 3, 2, 2, 0, 2)]
     for bad in (window_at_the_front, off_by_one, sink_forgotten):
         _expect_caught(monkeypatch, "full_precision_tokens", bad, pins)
+
+
+# --------------------------------------------------------------------------
+# m that splits a head (the paper's m = 64 and m = 384 with d = 128: Appendix
+# "Compression-Ratio Configurations"): Eq. 6 concatenates at the flat index
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,L,H_q,H_kv,d,m", [(31, 5, 4, 2, 4, 2), (32, 6, 4, 2, 4, 6), (33, 4, 6, 3, 4, 5),
+                                                   (34, 7, 2, 2, 8, 12)])
+def test_brute_force_with_a_split_head(seed, L, H_q, H_kv, d, m):
+    c = rand_case(seed, L, H_q, H_kv, d, m=m)
+    assert c["m"] % d != 0 and c["Wk"].shape == (c["D"] - m, c["D"] + m)
+    bf = brute_force(c)
+    np.testing.assert_allclose(run(c), bf, rtol=1e-12, atol=1e-13)
+    # the per-head evaluation takes the stored dims of the split head from the cache and the rest from W
+    per = O.decode_attention_query_heads(c["q"], c["kg"], c["vg"], c["kl"], c["vl"], c["Wk"], c["Wv"], c["H_kv"],
+                                         query_heads=range(H_q))
+    for h in range(H_q):
+        np.testing.assert_allclose(per[h], bf[h], rtol=1e-12, atol=1e-13)
+    # a selector predictor makes the split head exact: standard attention on the true cache (library routine)
+    g = rng(seed + 100)
+    D = c["D"]
+    k_true = np.concatenate([c["kl"], g.standard_normal((L, D - m))], axis=1)
+    v_true = np.concatenate([c["vl"], g.standard_normal((L, D - m))], axis=1)
+    sel = np.zeros((D - m, D + m))
+    sel[np.arange(D - m), m + np.arange(D - m)] = 1.0
+    kg, vg = c["kg"].copy(), c["vg"].copy()
+    kg[:, m:], vg[:, m:] = k_true[:, m:], v_true[:, m:]
+    got = O.decode_attention(c["q"], kg, vg, c["kl"], c["vl"], sel, sel, c["H_kv"])
+    np.testing.assert_allclose(got, sdpa(c["q"], k_true.reshape(L, H_kv, d), v_true.reshape(L, H_kv, d)),
+                               rtol=1e-12, atol=1e-13)
+
+
+def test_per_head_evaluation_with_biases_whole_keys_and_a_window():
+    for m in (8, 12):                           # head-aligned and head-splitting (d = 8)
+        c = rand_case(90 + m, L=23, H_q=8, H_kv=4, d=8, m=m)
+        g = rng(90 + m)
+        bk, bv = g.standard_normal(c["D"] - m), g.standard_normal(c["D"] - m)
+        args = (c["q"], c["kg"], c["vg"], c["kl"], c["vl"], c["Wk"], c["Wv"], c["H_kv"])
+        heads = range(c["H_q"])
+        full = O.decode_attention(*args, bk=bk, bv=bv)
+        per = O.decode_attention_query_heads(*args, query_heads=heads, bk=bk, bv=bv)
+        k_true = g.standard_normal((c["L"], c["D"]))
+        full_sk = O.decode_attention(*args, bv=bv, k_true=k_true, rope_theta=500.0)
+        per_sk = O.decode_attention_query_heads(*args, query_heads=heads, bv=bv, k_true=k_true, rope_theta=500.0)
+        kt, vt = true_dropped(c, m)
+        full_w = O.decode_attention_windowed(*args, kt, vt, 2, 5, bk=bk, bv=bv, rope_theta=500.0)
+        per_w = O.decode_attention_query_heads(*args, query_heads=heads, k_true_drop=kt, v_true_drop=vt, n_sink=2,
+                                               n_window=5, bk=bk, bv=bv, rope_theta=500.0)
+        full_wsk = O.decode_attention_windowed(*args, None, vt, 2, 5, bv=bv, k_true=k_true)
+        per_wsk = O.decode_attention_query_heads(*args, query_heads=heads, v_true_drop=vt, n_sink=2, n_window=5, bv=bv,
+                                                 k_true=k_true)
+        for h in heads:
+            np.testing.assert_allclose(per[h], full[h], rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(per_sk[h], full_sk[h], rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(per_w[h], full_w[h], rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(per_wsk[h], full_wsk[h], rtol=1e-12, atol=1e-13)
+        # the bias is a plain shift of the predicted dims: the same as one more input feature that is always 1
+        ones = np.ones((c["L"], 1))
+        kl1, vl1 = np.concatenate([c["kl"], ones], axis=1), np.concatenate([c["vl"], ones], axis=1)
+        Wk1 = np.concatenate([c["Wk"], bk[:, None]], axis=1)
+        Wv1 = np.concatenate([c["Wv"], bv[:, None]], axis=1)
+        K1 = O.reconstruct_dropped(Wk1, c["kg"], kl1)
+        np.testing.assert_allclose(K1, O.reconstruct_dropped(c["Wk"], c["kg"], c["kl"], bk), rtol=1e-12, atol=1e-13)
+        V1 = O.reconstruct_dropped(Wv1, c["vg"], vl1)
+        np.testing.assert_allclose(V1, O.reconstruct_dropped(c["Wv"], c["vg"], c["vl"], bv), rtol=1e-12, atol=1e-13)
+
+
+def test_window_with_whole_keys():
+    """"Save K" with a sink / window: the keys are whole, so the window changes the values only."""
+    c = rand_case(61, L=11, H_q=4, H_kv=2, d=4, m=4)
+    g = rng(61)
+    L, D, m, H, d = c["L"], c["D"], c["m"], c["H_kv"], c["d"]
+    k_true = g.standard_normal((L, D))
+    kt, vt = true_dropped(c, 61)
+    args = (c["q"], c["kg"], c["vg"], c["kl"], c["vl"], c["Wk"], c["Wv"], H)
+    got = O.decode_attention_windowed(*args, kt, vt, 2, 3, k_true=k_true)
+    # brute force: the keys of a cache whose K predictor is never consulted = every token's keys "true"
+    c2 = dict(c)
+    c2["kl"] = k_true[:, :m]
+    bf = brute_force_windowed(c2, k_true[:, m:], vt, 2, 3, all_keys_true=True)
+    np.testing.assert_allclose(got, bf, rtol=1e-12, atol=1e-13)
+    # no window: the plain save-K step; everything inside the window: standard attention on the true cache
+    np.testing.assert_array_equal(O.decode_attention_windowed(*args, kt, vt, 0, 0, k_true=k_true),
+                                  O.decode_attention(*args, k_true=k_true))
+    V = np.concatenate([c["vl"], vt], axis=1).reshape(L, H, d)
+    np.testing.assert_allclose(O.decode_attention_windowed(*args, kt, vt, 0, L, k_true=k_true),
+                               sdpa(c["q"], k_true.reshape(L, H, d), V), rtol=1e-12, atol=1e-13)
+    # k_local, Wk and k_true_drop are not read
+    bad = (c["q"], c["kg"], c["vg"], np.full_like(c["kl"], np.nan), c["vl"], None, c["Wv"], H)
+    np.testing.assert_array_equal(O.decode_attention_windowed(*bad, None, vt, 2, 3, k_true=k_true), got)
+
+
+def test_prefill_shaped_attention_with_sink_and_window():
+    """Every query is the windowed decode step of the sequence cut off at its own position."""
+    for m, rope in ((8, None), (12, 700.0)):
+        c = rand_case(71 + m, L=19, H_q=8, H_kv=4, d=8, m=m)
+        g = rng(71 + m)
+        n_q, n_sink, n_window = 9, 2, 4
+        L, H, d = c["L"], c["H_kv"], c["d"]
+        q = g.standard_normal((n_q, c["H_q"], d))
+        kt, vt = true_dropped(c, m)
+        args = (c["kg"], c["vg"], c["kl"], c["vl"], c["Wk"], c["Wv"], H)
+        got = O.prefill_attention(q, *args, k_true_drop=kt, v_true_drop=vt, n_sink=n_sink, n_window=n_window,
+                                  rope_theta=rope)
+        for i in range(n_q):
+            n = L - n_q + i + 1
+            want = O.decode_attention_windowed(q[i], c["kg"][:n], c["vg"][:n], c["kl"][:n], c["vl"][:n], c["Wk"],
+                                               c["Wv"], H, kt[:n], vt[:n], n_sink, n_window, rope_theta=rope)
+            np.testing.assert_allclose(got[i], want, rtol=1e-12, atol=1e-13)
+        if rope is None:
+            # index by index, for a query in the middle of the chunk: ITS last n_window tokens are the true ones
+            i = 4
+            n = L - n_q + i + 1
+            cut = dict(c, q=q[i], kg=c["kg"][:n], vg=c["vg"][:n], kl=c["kl"][:n], vl=c["vl"][:n], L=n)
+            np.testing.assert_allclose(got[i], brute_force_windowed(cut, kt[:n], vt[:n], n_sink, n_window),
+                                       rtol=1e-12, atol=1e-13)
+        # a token is read as stored by the queries close behind it and as predicted by the later ones: what is
+        # stored for token L - n_q (the first query's own) reaches the queries 0 .. n_window - 1 only
+        kt2, vt2 = kt.copy(), vt.copy()
+        kt2[L - n_q] += 1.0
+        vt2[L - n_q] -= 1.0
+        got2 = O.prefill_attention(q, *args, k_true_drop=kt2, v_true_drop=vt2, n_sink=n_sink, n_window=n_window,
+                                   rope_theta=rope)
+        assert all(np.abs(got2[i] - got[i]).max() > 1e-6 for i in range(n_window))
+        np.testing.assert_array_equal(got2[n_window:], got[n_window:])
+        # no sink, no window: the plain prefill-shaped call; a window as long as the cache: causal attention on
+        # the true cache (library routine)
+        np.testing.assert_array_equal(O.prefill_attention(q, *args, k_true_drop=kt, v_true_drop=vt, rope_theta=rope),
+                                      O.prefill_attention(q, *args, rope_theta=rope))
+        if rope is None:
+            allq = g.standard_normal((L, c["H_q"], d))
+            full = O.prefill_attention(allq, *args, k_true_drop=kt, v_true_drop=vt, n_sink=0, n_window=L)
+            K = np.concatenate([c["kl"], kt], axis=1).reshape(L, H, d)
+            V = np.concatenate([c["vl"], vt], axis=1).reshape(L, H, d)
+            tq = torch.from_numpy(allq).permute(1, 0, 2)[None]
+            tk = torch.from_numpy(K).permute(1, 0, 2)[None]
+            tv = torch.from_numpy(V).permute(1, 0, 2)[None]
+            ref = F.scaled_dot_product_attention(tq, tk, tv, is_causal=True, enable_gqa=True)[0].permute(1, 0, 2).numpy()
+            np.testing.assert_allclose(full, ref, rtol=1e-12, atol=1e-13)
+
+
+def test_prefill_window_planted_mistake_is_caught(monkeypatch):
+    good = O.full_precision_tokens
+
+    def window_of_the_whole_cache(L, n_sink, n_window):          # one window for all queries, at the end of the cache
+        return good(19, n_sink, n_window)[:L]
+
+    _expect_caught(monkeypatch, "full_precision_tokens", window_of_the_whole_cache,
+                   [test_prefill_shaped_attention_with_sink_and_window])
