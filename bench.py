@@ -1,17 +1,25 @@
 #!/usr/bin/env python
 """Benchmark of the EchoKV decode path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4] [--mode compressed|full]
-                    [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload c1|c2|c3|c4] [--mode compressed|full] [--sweep] ...
 
 One "step" = one pass of the whole hot path over one batch of synthetic input.  For the
-single-layer workloads (c1, the default and the headline; c2; a point of the c4 sweep) that is:
-append the new token to the anchor layer and to the compressed layer (which keeps only the
-retained heads), then decode attention on the compressed layer -- retained heads from the
-cache, dropped heads reconstructed on chip -- including the split-K merge.  For c3 it is the
-whole 32-layer decode step: per layer an append and the layer's attention (full-cache on the
-8 anchor layers, reconstruct-then-attend on the 24 compressed ones).  --mode full times the
-uncompressed path instead (full-cache attention on the anchor layer).
+single-layer workloads (c1; c2; a point of the c4 sweep) that is: append the new token to the
+anchor layer and to the compressed layer (which keeps only the retained dims), then decode
+attention on the compressed layer -- retained heads from the cache, dropped heads reconstructed
+on chip -- including the split-K merge.  For c3 it is the whole 32-layer decode step: per layer an
+append and the layer's attention (full-cache on the 8 anchor layers, reconstruct-then-attend on the
+24 compressed ones).  --mode full times the uncompressed path instead.
+
+Without --workload the run is the whole record: the headline is the largest single-GPU
+configuration (c3: 32 layers, 16-token pages in a random order), followed by a `sustained` leg
+(the same step repeated for at least two seconds, with the clocks sampled throughout) and a
+`configs` object with one sub-record per benchmark configuration (c1, c2, c3 and three points of
+the c4 sweep), each with its step time, its end-to-end time, the dominant kernel's time and its
+fraction of both measured tensor peaks, a parity sample against the CPU oracle and the
+uncompressed step at the same shape.  With --workload only that workload is measured.
+`--workload c4 --sweep` walks the whole sweep (ratio x context x batch), one sub-record per point.
 
 `value` is decode tokens per second (sequences advanced per second) with the caches resident
 in HBM; `e2e` is the same step driven from pinned host buffers through
@@ -24,6 +32,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -35,6 +44,17 @@ if ROOT not in sys.path:
 
 METRIC = "decode_attention_tokens_per_s"
 UNIT = "tokens/s"
+
+HEADLINE = "c3"
+# the sub-records of the default run: every benchmark configuration that fits a short run
+SUITE = [
+    ("c1", dict(workload="c1")),
+    ("c2", dict(workload="c2")),
+    ("c3", dict(workload="c3")),
+    ("c4_75pct_B8_L65536", dict(workload="c4", ratio=75, batch=8, context=65536)),
+    ("c4_75pct_B2_L131072", dict(workload="c4", ratio=75, batch=2, context=131072)),
+    ("c4_25pct_B8_L16384", dict(workload="c4", ratio=25, batch=8, context=16384)),
+]
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu captures summarised under profiles/; None until a capture of that workload exists.
@@ -51,7 +71,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 def traffic_of(args, key):
-    """The stored ncu figure, only for the exact workload it was scaled to."""
+    """The stored ncu figure, only for the exact workload and kernel it was taken on."""
     if args.batch or args.context or args.page_tokens or args.random_pages:
         return None
     if (args.rope or args.window or args.retained_dims or args.save_k or args.decode_path is not None
@@ -76,9 +96,13 @@ def workload_by_name(name, batch=0, context=0, page_tokens=0, random_pages=False
         return w.replace(save_k=True, name=w.name + "_saveK")
     if name == "c4":
         w = synth.c4_point(ratio, context or 16384, batch or 8)
-        if retained_dims:   # the paper's own settings, e.g. m = 64: half of the first head (absorbed mode only)
+        if retained_dims:   # the paper's own settings, e.g. m = 64: half of the first head
             w = w.replace(n_retained_dims=retained_dims, n_retained_heads=retained_dims // w.head_dim,
                           name="c4_m%d_L%d_B%d" % (retained_dims, w.context, w.batch))
+        if page_tokens:
+            w = w.replace(page_tokens=page_tokens, name=w.name + "_P%d" % page_tokens)
+        if random_pages:
+            w = w.replace(random_pages=True, name=w.name + "_randpages")
         return w
     w = {"c1": synth.C1, "c2": synth.C2, "c3": synth.C3}[name]
     if page_tokens:
@@ -90,6 +114,11 @@ def workload_by_name(name, batch=0, context=0, page_tokens=0, random_pages=False
     if context:
         w = w.replace(context=context, name=w.name + "_L%d" % context)
     return w
+
+
+def workload_of_args(args):
+    return workload_by_name(args.workload or HEADLINE, args.batch, args.context, args.page_tokens, args.random_pages,
+                            args.ratio, args.retained_dims, args.save_k)
 
 
 def algorithmic_work(w):
@@ -106,12 +135,13 @@ def algorithmic_work(w):
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+    """Samples SM clock, power and throttle reasons through NVML (read-only) while a timed region runs."""
 
-    def __init__(self, index):
+    def __init__(self, index, period_s=0.002):
         super().__init__(daemon=True)
         self.index = index
-        self.samples, self.reasons = [], set()
+        self.period_s = period_s
+        self.samples, self.power, self.reasons = [], [], set()
         self.max_mhz = None
         self._stop_evt = threading.Event()
         self.error = None
@@ -135,13 +165,17 @@ class ClockSampler(threading.Thread):
             while not self._stop_evt.is_set():
                 self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
                 try:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
+                except Exception:
+                    pass
+                try:
                     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
                 except Exception:
                     mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
                 for bit, name in names.items():
                     if mask & bit and name != "gpu_idle":
                         self.reasons.add(name)
-                time.sleep(0.004)
+                time.sleep(self.period_s)
         except Exception as e:  # NVML missing: report it rather than guess
             self.error = repr(e)
 
@@ -151,6 +185,10 @@ class ClockSampler(threading.Thread):
         s = sorted(self.samples)
         med = s[len(s) // 2] if s else None
         out = {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s)}
+        if s:
+            out["sm_mhz_min"] = s[0]
+        if self.power:
+            out["power_w_max"] = max(self.power)
         if self.error:
             out["error"] = self.error
         return out
@@ -178,6 +216,7 @@ class State:
         from paper_2603_22910_b200 import binding, synth
         self.w, self.layers = w, layers
         self.window = window if (window and w.D > w.m) else None
+        self.rope = None
         self.dev = dev = torch.device("cuda", local_rank)
         self.ctx = ctx = binding.Context(binding.config_for(w, device=local_rank))
         if self.window:
@@ -192,32 +231,34 @@ class State:
         for l in needed:
             for kind, pools in (("k", ctx.k_pools), ("v", ctx.v_pools)):
                 width = w.D if w.is_anchor(l) else (w.mk if kind == "k" else w.m)
+                side = self.window and not w.is_anchor(l) and not (w.save_k and kind == "k")
                 newest = torch.zeros((w.batch, w.D), dtype=tdt, device=dev)
                 for b in range(w.batch):
-                    if width == 0:
+                    if width == 0 and not side:
                         continue
                     ids = self.table[b].long().to(dev)
-                    x = synth.layer_cache(w, l, kind, b, width=w.D if self.window else width, device=dev)
-                    if self.window and not w.is_anchor(l):
+                    x = synth.layer_cache(w, l, kind, b, width=w.D if side else width, device=dev)
+                    if side:
                         # sink and recent-window tokens keep their dims m..D-1 in the side buffers
                         n_sink, n_window = self.window
                         L = w.context
                         toks = [t for t in range(L) if t < n_sink or t >= L - n_window]
                         tt = torch.tensor(toks, device=dev)
                         rows = x[tt, w.m:]
-                        side = (ctx.k_side if kind == "k" else ctx.v_side)[l]
+                        buf = (ctx.k_side if kind == "k" else ctx.v_side)[l]
                         slots = torch.tensor([t if t < n_sink else n_sink + t % n_window for t in toks], device=dev)
-                        side[b, slots] = rows          # (a sink token inside the window: same values twice)
+                        buf[b, slots] = rows          # (a sink token inside the window: same values twice)
                         self.true_rows[(l, kind, b)] = (toks, rows.cpu())
                         newest_full = x[w.context - 1].clone()
                         x = x[:, :width].contiguous()
                     else:
                         newest_full = None
-                    pad = w.pages_per_seq * w.page_tokens - w.context
-                    if pad:
-                        x = torch.cat([x, torch.zeros((pad, width), dtype=tdt, device=dev)])
-                    pools[l][ids] = x.reshape(w.pages_per_seq, w.page_tokens, width)
-                    newest[b, :width] = x[w.context - 1]
+                    if width:
+                        pad = w.pages_per_seq * w.page_tokens - w.context
+                        if pad:
+                            x = torch.cat([x, torch.zeros((pad, width), dtype=tdt, device=dev)])
+                        pools[l][ids] = x.reshape(w.pages_per_seq, w.page_tokens, width)
+                        newest[b, :width] = x[w.context - 1]
                     if newest_full is not None:
                         newest[b] = newest_full        # the step re-appends the newest token, all its dims
                     del x
@@ -278,9 +319,10 @@ class State:
         import numpy as np
         from oracle import echokv_oracle as O
         from paper_2603_22910_b200 import synth
-        toks, rows = self.true_rows[(layer, kind, b)]
         out = np.full((self.w.context, self.w.D - self.w.m), np.nan)
-        out[toks] = O.widen(synth.to_numpy_stored(rows))
+        if (layer, kind, b) in self.true_rows:
+            toks, rows = self.true_rows[(layer, kind, b)]
+            out[toks] = O.widen(synth.to_numpy_stored(rows))
         return out
 
 
@@ -315,12 +357,93 @@ def oracle_layer(inputs, w, state=None, layer=None, b=None):
     rope = getattr(state, "rope", None) or None
     if len(inputs) == 3:
         return O.full_attention(inputs[0], inputs[1], inputs[2], w.n_kv_heads, rope_theta=rope)
+    k_true = state.true_keys(layer, b) if state is not None else None
     if state is not None and state.window:
         return O.decode_attention_windowed(*inputs, w.n_kv_heads, state.true_dropped(layer, "k", b),
                                            state.true_dropped(layer, "v", b), state.window[0], state.window[1],
-                                           rope_theta=rope)
-    k_true = state.true_keys(layer, b) if state is not None else None
+                                           rope_theta=rope, k_true=k_true)
     return O.decode_attention(*inputs, n_kv_heads=w.n_kv_heads, rope_theta=rope, k_true=k_true)
+
+
+def oracle_heads(state, layer, b, heads, inputs=None):
+    """Oracle outputs {h: [d]} of a few query heads of (layer, sequence b): heads are independent in Eq. 7
+    and a predicted head needs only its own rows of W in Eq. 3."""
+    from oracle import echokv_oracle as O
+    w = state.w
+    rope = state.rope or None
+    inputs = state.oracle_inputs(layer, b) if inputs is None else inputs
+    if len(inputs) == 3:                # a stored (anchor / uncompressed) layer: only the head's own dims
+        q, kg, vg = inputs
+        d, g = w.head_dim, w.n_q_heads // w.n_kv_heads
+        out = {}
+        for h in heads:
+            kv = h // g
+            out[h] = O.attention(q[h:h + 1], kg[:, None, kv * d:(kv + 1) * d], vg[:, None, kv * d:(kv + 1) * d],
+                                 rope_theta=rope)[0]
+        return out
+    kw = {}
+    if state.window:
+        kw = dict(k_true_drop=state.true_dropped(layer, "k", b), v_true_drop=state.true_dropped(layer, "v", b),
+                  n_sink=state.window[0], n_window=state.window[1])
+    k_true = state.true_keys(layer, b)
+    if k_true is not None:
+        kw["k_true"] = k_true
+    return O.decode_attention_query_heads(*inputs, n_kv_heads=w.n_kv_heads, query_heads=list(heads), rope_theta=rope,
+                                          **kw)
+
+
+def stratified_picks(w, attend_layers, n_outputs, seed=7, max_combos=16):
+    """[(layer, sequence, [query heads])] covering, between them: every sequence of the batch, the first, a
+    middle and the last compressed layer and the first and last anchor layer of the step, and every KV head
+    (dropped heads first, so every pair of dropped heads a fused-kernel work item handles is met)."""
+    import numpy as np
+    rng = np.random.default_rng(seed)
+    g = w.n_q_heads // w.n_kv_heads
+    comp = [l for l in attend_layers if not w.is_anchor(l) and w.d_drop > 0]
+    anch = [l for l in attend_layers if l not in comp]
+    layers = []
+    if comp:
+        layers += sorted({comp[0], comp[len(comp) // 2], comp[-1]})
+    if anch:
+        layers += sorted({anch[0], anch[-1]})
+    n_combos = min(max(w.batch, len(layers)), max_combos, n_outputs)
+    per = int(math.ceil(n_outputs / float(n_combos)))
+    first_drop = w.m // w.head_dim            # (a partly retained head is predicted in part: counts as dropped)
+    picks, walk = [], 0
+    for k in range(n_combos):
+        l, b = layers[k % len(layers)], k % w.batch
+        if w.is_anchor(l) or w.d_drop == 0:
+            kv_order = list(range(w.n_kv_heads))
+        else:
+            kv_order = list(range(first_drop, w.n_kv_heads)) + list(range(first_drop))
+        heads = []
+        for _ in range(per):
+            kv = kv_order[walk % len(kv_order)]
+            walk += 1
+            h = kv * g + int(rng.integers(g))
+            if h not in heads:
+                heads.append(h)
+        picks.append((l, b, heads))
+    return picks
+
+
+def parity_sample(state, picks):
+    """Element-wise comparison of sampled GPU outputs (state.out, as the last step left them) with the oracle."""
+    import numpy as np
+    worst = num = den = 0.0
+    n = 0
+    for l, b, heads in picks:
+        ref = oracle_heads(state, l, b, heads)
+        for h in heads:
+            got = state.out[l][b, h].cpu().numpy().astype(np.float64)
+            if not np.all(np.isfinite(got)):
+                return {"outputs": n, "max_abs": float("inf"), "rel_l2": float("inf")}
+            worst = max(worst, float(np.max(np.abs(got - ref[h]))))
+            num += float(np.sum((got - ref[h]) ** 2))
+            den += float(np.sum(ref[h] ** 2))
+            n += 1
+    return {"outputs": n, "combos": [(l, b, len(hs)) for l, b, hs in picks], "max_abs": worst,
+            "rel_l2": (num / max(den, 1e-300)) ** 0.5}
 
 
 def time_oracle(state, step_layers, budget_s):
@@ -342,20 +465,28 @@ def time_oracle(state, step_layers, budget_s):
         n_seq = len(outs)
         return n_seq / elapsed, ("%d of %d sequences of the batch, all heads, all %d tokens (%.1f s)"
                                  % (n_seq, w.batch, w.context, elapsed)), outs
-    # multi-layer step: one group of S consecutive layers (an anchor and the layers that lean on
-    # it) for one sequence; every group costs the same, so the step takes n_groups times as long
-    S = w.group_size
-    group = [l for l in attend if l < S]
-    b = 0
-    for l in group:
-        inputs = state.oracle_inputs(l, b)
-        t0 = time.perf_counter()
-        outs[(l, b)] = oracle_layer(inputs, w, state, l, b)
-        elapsed += time.perf_counter() - t0
-    scale = len(attend) / float(len(group))
-    return 1.0 / (elapsed * scale), ("sequence 0 of %d, layers 0..%d (one group of S = %d), all heads, all %d "
-                                     "tokens (%.1f s); extrapolated x%.0f to the %d layers"
-                                     % (w.batch, S - 1, S, w.context, elapsed, scale, len(attend))), outs
+    # multi-layer step: whole sequences through the first anchor layer and the first compressed layer (every
+    # anchor layer costs the same, every compressed layer costs the same), scaled to the layer counts
+    anchors = [l for l in attend if w.is_anchor(l)]
+    comps = [l for l in attend if not w.is_anchor(l)]
+    t_kind = {"a": 0.0, "c": 0.0}
+    n_seq = 0
+    for b in range(w.batch):
+        for kind, ls in (("a", anchors), ("c", comps)):
+            if not ls:
+                continue
+            inputs = state.oracle_inputs(ls[0], b)
+            t0 = time.perf_counter()
+            outs[(ls[0], b)] = oracle_layer(inputs, w, state, ls[0], b)
+            t_kind[kind] += time.perf_counter() - t0
+        n_seq += 1
+        if t_kind["a"] + t_kind["c"] >= budget_s:
+            break
+    t_seq = (t_kind["a"] * len(anchors) + t_kind["c"] * len(comps)) / n_seq     # one sequence, all layers
+    return 1.0 / t_seq, ("%d of %d sequences through layer %d (anchor) and layer %d (compressed), all heads, all %d "
+                         "tokens (%.1f s); scaled to %d anchor + %d compressed layers"
+                         % (n_seq, w.batch, anchors[0] if anchors else -1, comps[0] if comps else -1, w.context,
+                            t_kind["a"] + t_kind["c"], len(anchors), len(comps))), outs
 
 
 def run_reference(args):
@@ -365,16 +496,16 @@ def run_reference(args):
         return 0
     from oracle import echokv_oracle as O
     from paper_2603_22910_b200 import synth
-    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio,
-                         args.retained_dims, args.save_k)
+    w = workload_of_args(args)
     st = synth.to_numpy_stored
     full = args.mode == "full"
     rope = args.rope or None
-    # The same sampling as the cpu_baseline leg: whole sequences, all heads, all tokens.  A step evaluates
-    # sequence 0 of the batch for one layer (single-layer workloads) or for one group of S consecutive layers
-    # (the 32-layer workload: every group costs the same); the result is scaled to the batch and the layers.
+    # One step evaluates sequence 0 of the batch, all heads, all tokens, for one layer (single-layer workloads)
+    # or for the first anchor layer and the first compressed layer (the 32-layer workload: every anchor layer
+    # costs the same and every compressed layer costs the same).  ms_per_step is the time of that sample as
+    # measured; only `value` is scaled to the batch and the layer counts.
     multi = w.n_layers > 2 and not full
-    layers = list(range(w.group_size)) if multi else [0 if full else 1]
+    layers = [0, 1] if multi else [0 if full else 1]
     inputs, k_true = {}, {}
     for l in layers:
         a = w.anchor_of(l)
@@ -392,30 +523,40 @@ def run_reference(args):
                          O.widen(st(synth.predictor_weights(w, l, "v"))))
 
     def run():
+        per_layer = {}
         for l in layers:
             x = inputs[l]
+            t0 = time.perf_counter()
             if len(x) == 3:
                 O.full_attention(x[0], x[1], x[2], w.n_kv_heads, rope_theta=rope)
             else:
                 O.decode_attention(*x, n_kv_heads=w.n_kv_heads, rope_theta=rope, k_true=k_true[l])
+            per_layer[l] = time.perf_counter() - t0
+        return per_layer
 
-    times = []
+    times, per = [], {l: [] for l in layers}
     for i in range(args.steps + args.warmup):
         t0 = time.perf_counter()
-        run()
+        pl = run()
         dt = time.perf_counter() - t0
         if i >= args.warmup:
             times.append(dt)
+            for l in layers:
+                per[l].append(pl[l])
     t_step = sum(times) / len(times)
-    n_attend = w.n_layers if multi else 1
-    t_batch = t_step * w.batch * (n_attend / float(len(layers)))
-    value = w.batch / t_batch
-    sample = ("sequence 0 of %d per step, %s, all heads, all %d tokens; scaled to the full batch%s"
-              % (w.batch, "layers 0..%d (one group of S = %d)" % (w.group_size - 1, w.group_size) if multi
-                 else "one layer", w.context, " and to %d layers" % n_attend if multi else ""))
+    if multi:
+        n_anchor = (w.n_layers + w.group_size - 1) // w.group_size
+        t_seq = (sum(per[0]) / len(per[0])) * n_anchor + (sum(per[1]) / len(per[1])) * (w.n_layers - n_anchor)
+        scaled = "value scaled to %d anchor + %d compressed layers" % (n_anchor, w.n_layers - n_anchor)
+    else:
+        t_seq = t_step
+        scaled = "value = sequences per second of this sample"
+    value = 1.0 / t_seq                  # sequences advanced per second = decode tokens per second
+    sample = ("each step: sequence 0 of %d, %s, all heads, all %d tokens; ms_per_step is that sample as measured; %s"
+              % (w.batch, "layer 0 (anchor) and layer 1 (compressed)" if multi else "one layer", w.context, scaled))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_batch * 1e3,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": workload_config(w, full),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
@@ -433,18 +574,14 @@ def run_prefill(args):
     import torch
     from paper_2603_22910_b200 import binding, synth
     from oracle import echokv_oracle as O
-    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio)
+    w = workload_of_args(args)
     n_q = args.prefill_queries
-    st = State(w, 0, [0, 1])
+    window = parse_window(args)
+    st = State(w, 0, [0, 1], window)
     ctx, dev = st.ctx, st.dev
     if args.rope:
         ctx.set_rope(args.rope)
     st.rope = args.rope
-    if args.prefill_path is not None:
-        ctx.set_prefill_path(args.prefill_path)
-    attn_kernel = {0: "prefill_attn_kernel (mma.sync)", 1: "prefill_attn_tc_kernel (tcgen05)",
-                   2: "prefill_attn_ws_kernel (tcgen05, warp-specialised)"}[
-                       binding.lib().echokv_prefill_path(ctx.handle)]
     q = synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, 1, device=dev).to(torch.bfloat16)
     out = torch.empty(q.shape, dtype=torch.float32, device=dev)
     for _ in range(max(3, args.warmup)):
@@ -465,7 +602,7 @@ def run_prefill(args):
     tokens = float(w.batch) * w.context
     recon_flops = tokens * 4.0 * w.d_in * w.d_drop
     k_ms = recon_ms / max(recon_n, 1)
-    peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+    peak_tf = float(peaks["bf16_tflops"])
     # causal attention: query i sees L - n_q + i + 1 keys; 4 d FLOP per (query, key, head)
     seen = n_q * (w.context - n_q) + n_q * (n_q + 1) / 2.0
     attn_flops = w.batch * w.n_q_heads * seen * 4.0 * w.head_dim
@@ -473,7 +610,11 @@ def run_prefill(args):
     n_chk = min(16, n_q)
     inputs = st.oracle_inputs(1, 0)
     q_chk = O.widen(synth.to_numpy_stored(q[0, -n_chk:].cpu()))
-    ref = O.prefill_attention(q_chk, *inputs[1:], n_kv_heads=w.n_kv_heads, rope_theta=args.rope or None)
+    kw = {}
+    if st.window:
+        kw = dict(k_true_drop=st.true_dropped(1, "k", 0), v_true_drop=st.true_dropped(1, "v", 0),
+                  n_sink=st.window[0], n_window=st.window[1])
+    ref = O.prefill_attention(q_chk, *inputs[1:], n_kv_heads=w.n_kv_heads, rope_theta=args.rope or None, **kw)
     got = out[0, -n_chk:].cpu().numpy().astype(np.float64)
     line = {
         "metric": "prefill_query_tokens_per_s", "value": w.batch * n_q / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
@@ -484,13 +625,14 @@ def run_prefill(args):
         "roofline": {"bound": "tensor", "achieved": recon_flops / (k_ms * 1e-3) / 1e12, "peak": peak_tf,
                      "unit": "TFLOP/s", "frac": recon_flops / (k_ms * 1e-3) / 1e12 / peak_tf, "traffic": None,
                      "kernel": "recon_pair_kernel (rows to memory), K pass + V pass", "kernel_ms": k_ms,
-                     "share_of_step": k_ms / ms, "peak_source": "%s (cuBLAS bf16 GEMM, sustained)" % peaks_kind},
-        "attention": {"kernel": attn_kernel + " + gather_rows_kernel x 2", "ms": ms - k_ms,
-                      "tflops": attn_flops / ((ms - k_ms) * 1e-3) / 1e12},
+                     "share_of_step": k_ms / ms, "peak_source": "%s (cuBLAS bf16 GEMM, burst)" % peaks_kind},
+        "attention": {"kernel": "prefill_attn_ws_kernel (tcgen05, warp-specialised) + gather_rows_kernel x 2",
+                      "ms": ms - k_ms, "tflops": attn_flops / ((ms - k_ms) * 1e-3) / 1e12},
         "parity_vs_oracle": {"rows": "last %d queries of sequence 0" % n_chk,
                              "max_abs": float(np.max(np.abs(got - ref))),
                              "rel_l2": float(np.linalg.norm(got - ref) / np.linalg.norm(ref))},
         "rope_theta": args.rope or None,
+        "full_precision_tokens": {"sink": window[0], "window": window[1]} if window else None,
     }
     print(json.dumps(line))
     ctx.close()
@@ -506,15 +648,15 @@ def workload_config(w, full=False):
         gb = w.batch * w.context * 2 * w.D * elem / 1e9
     elif w.n_layers > 2:
         n_anchor = (w.n_layers + w.group_size - 1) // w.group_size
-        what = ("%s: %d layers (S=%d: %d anchor + %d compressed), B=%d L=%d H_q=%d H_kv=%d d=%d retained=%d "
+        what = ("%s: %d layers (S=%d: %d anchor + %d compressed), B=%d L=%d H_q=%d H_kv=%d d=%d m=%d "
                 "(D_in=%d -> D_drop=%d), %s, %s" % (w.name, w.n_layers, w.group_size, n_anchor, w.n_layers - n_anchor,
                                                    w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim,
-                                                   w.n_retained_heads, w.d_in, w.d_drop, w.dtype, pages))
+                                                   w.m, w.d_in, w.d_drop, w.dtype, pages))
         gb = w.batch * w.context * 2 * elem * (n_anchor * w.D + (w.n_layers - n_anchor) * w.d_in) / 1e9
     else:
-        what = ("%s: B=%d L=%d H_q=%d H_kv=%d d=%d retained=%d (D_in=%d -> D_drop=%d), %s, %s, "
+        what = ("%s: B=%d L=%d H_q=%d H_kv=%d d=%d m=%d (D_in=%d -> D_drop=%d), %s, %s, "
                 "anchor + compressed layer" % (w.name, w.batch, w.context, w.n_q_heads, w.n_kv_heads, w.head_dim,
-                                               w.n_retained_heads, w.d_in, w.d_drop, w.dtype, pages))
+                                               w.m, w.d_in, w.d_drop, w.dtype, pages))
         gb = w.batch * w.context * 2 * w.d_in * elem / 1e9
     return {"workload": what, "global_batch": w.batch, "context": w.context,
             "l2": "inputs (%.2f GB of cache read per step) exceed the 126 MB L2; no flush needed" % gb,
@@ -568,145 +710,115 @@ class Replicas:
 # --------------------------------------------------------------------------------------------
 # GPU arm
 # --------------------------------------------------------------------------------------------
-def run_ours(args):
-    import numpy as np
-    import torch
-    from paper_2603_22910_b200 import binding, build
+def parse_window(args):
+    if not args.window or args.mode == "full":
+        return None
+    window = tuple(int(v) for v in args.window.split(","))
+    return window if sum(window) else None
 
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    rep = Replicas("nccl", torch.device("cuda", local_rank))
-    rank, world, dist = rep.rank, rep.world, rep.dist
-    if rank == 0:
-        build.build()
-    rep.barrier()
-    binding.lib()
 
-    w = workload_by_name(args.workload, args.batch, args.context, args.page_tokens, args.random_pages, args.ratio,
-                         args.retained_dims, args.save_k)
-    w = w.replace(seed=rep.seed_for(w.seed))
-    full = args.mode == "full"
-    resident, step_layers = plan_layers(w, args.mode)
-    window = None
-    if args.window and not full:
-        window = tuple(int(v) for v in args.window.split(","))
-        if sum(window) == 0:
-            window = None
-    st = State(w, local_rank, resident, window)
-    ctx, dev = st.ctx, st.dev
-    if args.stored_path is not None:
-        ctx.set_stored_path(args.stored_path)
-    if args.decode_path is not None and not full:
-        ctx.set_decode_path(args.decode_path)
-    absorbed = args.decode_mode == "absorbed" and not full
-    if absorbed:
-        ctx.enable_absorbed()
-    st.rope = args.rope
-    if args.rope:
-        ctx.set_rope(args.rope)      # (the library refuses it together with the absorbed mode)
-    last = [l for l, a in step_layers if a][-1]
+class Run:
+    """One workload on one GPU with the options of the command line applied, and the steps that are timed."""
 
-    def attend(l):
-        if full or w.is_anchor(l):   # the uncompressed mode / an anchor layer: Eq. 7 on the stored full cache
+    def __init__(self, w, args, local_rank):
+        import torch
+        self.torch = torch
+        self.w, self.args = w, args
+        self.full = args.mode == "full"
+        resident, self.step_layers = plan_layers(w, args.mode)
+        self.window = parse_window(args)
+        self.st = st = State(w, local_rank, resident, self.window)
+        self.ctx = ctx = st.ctx
+        if args.stored_path is not None:
+            ctx.set_stored_path(args.stored_path)
+        if args.decode_path is not None and not self.full:
+            ctx.set_decode_path(args.decode_path)
+        self.absorbed = args.decode_mode == "absorbed" and not self.full
+        if self.absorbed:
+            ctx.enable_absorbed()
+        st.rope = args.rope
+        if args.rope:
+            ctx.set_rope(args.rope)
+        self.n_attend = sum(1 for _, a in self.step_layers if a)
+        self.last = [l for l, a in self.step_layers if a][-1]
+        # the uncompressed step at the same shape: every layer attends a full cache.  The layers that hold one
+        # here are the anchors; a 32-layer step walks them n_layers / n_anchors times.
+        anchors = [l for l in resident if w.is_anchor(l)]
+        n_layers_step = w.n_layers if w.n_layers > 2 else 1
+        self.full_layers = [anchors[i % len(anchors)] for i in range(n_layers_step)]
+
+    def attend(self, l):
+        st, ctx = self.st, self.ctx
+        if self.full or self.w.is_anchor(l):   # the uncompressed mode / an anchor layer: Eq. 7 on the stored full cache
             ctx.full_attention(l, st.q_dev[l], st.lens, out=st.out[l])
         else:
             ctx.decode_attention(l, st.q_dev[l], st.lens, out=st.out[l])
 
-    def step():
-        for l, a in step_layers:
+    def step(self):
+        st, ctx = self.st, self.ctx
+        for l, a in self.step_layers:
             ctx.append_kv(l, st.new_dev[(l, "k")], st.new_dev[(l, "v")], st.positions)
             if a:
-                attend(l)
+                self.attend(l)
 
-    def step_host():
-        for l, a in step_layers:
+    def step_host(self):
+        st, ctx = self.st, self.ctx
+        for l, a in self.step_layers:
             ctx.layer_step_host(l, st.q_host[l] if a else None, st.new_host[(l, "k")], st.new_host[(l, "v")],
                                 st.out_host[l] if a else None, st.lens_host, attend=a)
 
+    def step_uncompressed(self):
+        st, ctx = self.st, self.ctx
+        for l in self.full_layers:
+            ctx.append_kv(l, st.new_dev[(l, "k")], st.new_dev[(l, "v")], st.positions)
+            ctx.full_attention(l, st.q_dev[l], st.lens, out=self.full_out)
+
+    def close(self):
+        self.ctx.close()
+
+
+def timed(run, rep, fn, steps, kernel_timing=True):
+    """`steps` calls of fn between two events on torch's current stream (the one every launch goes to), a
+    barrier + synchronize on both sides, max over ranks.  Returns (ms total, per-kind kernel times, launches)."""
+    torch = run.torch
+    ctx = run.ctx
+
     def sync_all():
         torch.cuda.synchronize()
-        if dist:
+        if rep.dist:
             rep.barrier()
             torch.cuda.synchronize()
 
-    max_over_ranks = rep.max_over_ranks
-
-    for _ in range(args.warmup):
-        step()
-    sync_all()
-    assert ctx.device_status() == binding.ECHOKV_OK, "device status after warm-up"
-
-    # ---- device-resident timed region -------------------------------------------------------
-    sampler = ClockSampler(physical_gpu_index(local_rank))
-    sampler.start()
-    ctx.set_kernel_timing(True)
-    ctx.read_kernel_timing()
+    if kernel_timing:
+        ctx.set_kernel_timing(True)
+        ctx.read_kernel_timing()
     launches0 = ctx.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
     e0.record()
-    for _ in range(args.steps):
-        step()
+    for _ in range(steps):
+        fn()
     e1.record()
     sync_all()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_total = rep.max_over_ranks(e0.elapsed_time(e1))
     launches = ctx.launch_count() - launches0
-    timing = ctx.read_kernel_timing_by_kind()
+    timing = ctx.read_kernel_timing_by_kind() if kernel_timing else None
     ctx.set_kernel_timing(False)
-    ms_eager = ms_total
-    if args.graph:
-        # the same step captured once in a CUDA graph and replayed: what the launch gaps cost; the per-kernel
-        # times above come from the eager pass (events cannot be read out of a captured region)
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            step()                                   # (first-use set-up of every kernel stays outside the capture)
-            side.synchronize()
-            with torch.cuda.graph(graph, stream=side):
-                step()
-        torch.cuda.current_stream().wait_stream(side)
-        for _ in range(3):
-            graph.replay()
-        sync_all()
-        e0.record()
-        for _ in range(args.steps):
-            graph.replay()
-        e1.record()
-        sync_all()
-        ms_total = max_over_ranks(e0.elapsed_time(e1))
-    clocks = sampler.stop()
-    status = ctx.device_status()
-    assert status == binding.ECHOKV_OK, "device status %d after the timed region" % status
+    return ms_total, timing, launches
 
-    # ---- end to end from pinned host memory -----------------------------------------------
-    for _ in range(min(3, args.warmup)):
-        step_host()
-    sync_all()
-    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2.record()
-    for _ in range(args.steps):
-        step_host()
-    e3.record()
-    sync_all()
-    ms_e2e = max_over_ranks(e2.elapsed_time(e3))
+
+def roofline_of(run, args, timing, ms_region, peaks, peaks_kind):
+    """The roofline record of the dominant kernel from the per-kind kernel times of a timed region."""
+    w, ctx = run.w, run.ctx
     elem = 2 if w.dtype == "bf16" else 4
-    n_attend = sum(1 for _, a in step_layers if a)
-    h2d = (len(step_layers) * (2 * w.batch * w.D * elem + 2 * w.batch * 4)
-           + n_attend * w.batch * w.n_q_heads * w.head_dim * elem)
-    d2h = n_attend * w.batch * w.n_q_heads * w.head_dim * 4
-    same = bool(torch.equal(st.out_host[last], st.out[last].cpu()))
-
-    ms_step = ms_total / args.steps
-    value = rep.job_value(w.batch, ms_step)
-    e2e_value = rep.job_value(w.batch, ms_e2e / args.steps)
-
-    peaks, peaks_kind = load_peaks()
     flops, bytes_ = algorithmic_work(w)
     stored_ms, stored_n = timing["stored"]
     recon_ms, recon_n = timing["recon"]
+    burst_tf = float(peaks["bf16_tflops"])
+    sustained_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+    tensor_source = ("%s cuBLAS bf16 GEMM, burst figure: the ceiling (a GEMM loop under the power cap -- the "
+                     "sustained figure, %.0f TFLOP/s -- is below what this kernel reaches, so it is listed as "
+                     "frac_of_sustained_peak only)" % (peaks_kind, sustained_tf))
     full_bytes = w.batch * w.context * 2.0 * w.D * elem   # a stored layer: every K and V row once
     stored_info = None
     if stored_n:
@@ -714,7 +826,7 @@ def run_ours(args):
         stored_info = {"kernel": "attn_stored_mma_kernel" if ctx.stored_path() == 1 else "attn_stored_kernel",
                        "kernel_ms": k_ms, "kernel_launches": stored_n, "achieved_gbs": full_bytes / (k_ms * 1e-3) / 1e9,
                        "frac_of_%s_hbm" % peaks_kind: full_bytes / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"])}
-    if absorbed:
+    if run.absorbed:
         # the absorbed mode streams [anchor dims ; retained dims] of K once and of V once: HBM-bound; its two
         # streaming kernels are reported together (each moves half of the bytes)
         ak_ms, ak_n = timing["absorb_k"]
@@ -726,10 +838,10 @@ def run_ours(args):
         peak_gbs = float(peaks["hbm_gbs"])
         roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
                     "frac": achieved_gbs / peak_gbs,
-                    "traffic": traffic_of(args, args.workload + "_absorbed"),
+                    "traffic": traffic_of(args, (args.workload or HEADLINE) + "_absorbed"),
                     "kernel": "absorb_scores_kernel + absorb_pv_kernel", "kernel_ms": k_ms,
                     "kernel_ms_k_pass": ak_ms / max(ak_n, 1), "kernel_ms_v_pass": av_ms / max(av_n, 1),
-                    "kernel_launches": ak_n + av_n, "share_of_step": (ak_ms + av_ms) / ms_eager,
+                    "kernel_launches": ak_n + av_n, "share_of_step": (ak_ms + av_ms) / ms_region,
                     "peak_source": "%s (STREAM-style copy)" % peaks_kind,
                     "algorithmic_bytes_per_launch": bytes_,
                     "mode": "absorbed predictors: the same outputs as the explicit path, a separate roofline row"}
@@ -743,13 +855,13 @@ def run_ours(args):
             k_flops = tokens * 2.0 * w.d_in * w.d_drop
             k_pass_ms = ak_ms / max(ak_n, 1)
             achieved_tf = k_flops / (k_pass_ms * 1e-3) / 1e12
-            peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
-            roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                        "frac": achieved_tf / peak_tf, "traffic": None,
+            roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": burst_tf, "unit": "TFLOP/s",
+                        "frac": achieved_tf / burst_tf, "frac_of_sustained_peak": achieved_tf / sustained_tf,
+                        "traffic": None,
                         "kernel": "recon_pair_kernel (key scores) + key_scores_stored_kernel", "kernel_ms": k_pass_ms,
                         "kernel_ms_k_pass": k_pass_ms, "kernel_ms_v_pass": av_ms / max(av_n, 1),
-                        "kernel_launches": ak_n, "share_of_step": ak_ms / ms_eager,
-                        "peak_source": "%s (cuBLAS bf16 GEMM, sustained)" % peaks_kind,
+                        "kernel_launches": ak_n, "share_of_step": ak_ms / ms_region,
+                        "peak_source": tensor_source,
                         "algorithmic_flops_per_launch": k_flops,
                         "v_pass_frac_of_hbm": (bytes_ / 2) / (av_ms / max(av_n, 1) * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
                         "mode": "rotated keys: K side explicit, V side with absorbed predictors"}
@@ -758,16 +870,16 @@ def run_ours(args):
     elif recon_n:
         k_ms = recon_ms / recon_n
         achieved_tf = flops / (k_ms * 1e-3) / 1e12
-        peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
-        roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                    "frac": achieved_tf / peak_tf, "traffic": traffic_of(args, args.workload),
+        roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": burst_tf, "unit": "TFLOP/s",
+                    "frac": achieved_tf / burst_tf, "frac_of_burst_peak": achieved_tf / burst_tf,
+                    "frac_of_sustained_peak": achieved_tf / sustained_tf, "peak_sustained": sustained_tf,
+                    "traffic": traffic_of(args, args.workload or HEADLINE),
                     "kernel": {3: "recon_pair_kernel", 2: "recon_tc_kernel"}.get(ctx.decode_path(), "recon_simt_kernel"),
                     "kernel_ms": k_ms, "kernel_launches": recon_n,
-                    "share_of_step": recon_ms / ms_eager,
-                    "peak_source": "%s (bf16 sustained; kernel timed inside a long step)" % peaks_kind,
+                    "share_of_step": recon_ms / ms_region,
+                    "peak_source": tensor_source,
                     "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": bytes_,
-                    "hbm_frac_of_%s" % peaks_kind: bytes_ / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
-                    "frac_of_burst_peak": achieved_tf / float(peaks["bf16_tflops"])}
+                    "hbm_frac_of_%s" % peaks_kind: bytes_ / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"])}
         if stored_info:
             roofline["anchor_layers"] = stored_info
     else:
@@ -775,47 +887,328 @@ def run_ours(args):
         achieved_gbs = full_bytes / (k_ms * 1e-3) / 1e9
         peak_gbs = float(peaks["hbm_gbs"])
         roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": peak_gbs, "unit": "GB/s",
-                    "frac": achieved_gbs / peak_gbs, "traffic": traffic_of(args, args.workload + "_full"),
+                    "frac": achieved_gbs / peak_gbs, "traffic": traffic_of(args, (args.workload or HEADLINE) + "_full"),
                     "kernel": stored_info["kernel"] if stored_info else None,
-                    "kernel_ms": k_ms, "kernel_launches": stored_n, "share_of_step": stored_ms / ms_eager,
+                    "kernel_ms": k_ms, "kernel_launches": stored_n, "share_of_step": stored_ms / ms_region,
                     "peak_source": "%s (STREAM-style copy)" % peaks_kind,
                     "algorithmic_bytes_per_launch": full_bytes}
+    return roofline
 
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": workload_config(w, full),
-        "us_per_layer_step": ms_step * 1e3 / n_attend,
-        "kv_tokens_scanned_per_s": world * w.batch * w.context * n_attend / (ms_step * 1e-3),
+
+def measure(run, rep, args, steps, warmup, peaks, peaks_kind, with_e2e=True):
+    """Warm-up, the device-resident timed region, and the end-to-end region of one workload."""
+    torch = run.torch
+    w, ctx, st = run.w, run.ctx, run.st
+    from paper_2603_22910_b200 import binding
+    for _ in range(warmup):
+        run.step()
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.ECHOKV_OK, "device status after warm-up"
+    sampler = ClockSampler(physical_gpu_index(rep.local_rank))
+    sampler.start()
+    ms_total, timing, launches = timed(run, rep, run.step, steps)
+    ms_eager = ms_total
+    if args.graph:
+        # the same step captured once in a CUDA graph and replayed: what the launch gaps cost; the per-kernel
+        # times above come from the eager pass (events cannot be read out of a captured region)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            run.step()                                   # (first-use set-up of every kernel stays outside the capture)
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                run.step()
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            graph.replay()
+        ms_total, _, _ = timed(run, rep, graph.replay, steps, kernel_timing=False)
+    clocks = sampler.stop()
+    status = ctx.device_status()
+    assert status == binding.ECHOKV_OK, "device status %d after the timed region" % status
+    ms_step = ms_total / steps
+    rec = {
+        "ms_per_step": ms_step,
+        "value": rep.job_value(w.batch, ms_step),
+        "us_per_layer_step": ms_step * 1e3 / run.n_attend,
+        "kv_tokens_scanned_per_s": rep.world * w.batch * w.context * run.n_attend / (ms_step * 1e-3),
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": ms_e2e / args.steps, "matches_device_path": same},
         "gpu_launches": int(launches),
-        "roofline": roofline,
-        "decode_path": ctx.decode_path(), "stored_path": ctx.stored_path(),
-        "decode_mode": "absorbed" if absorbed else "explicit",
-        "cuda_graph": {"ms_per_step_eager": ms_eager / args.steps} if args.graph else None,
-        "full_precision_tokens": {"sink": window[0], "window": window[1]} if window else None,
-        "rope_theta": args.rope or None,
-        "input_generation_s": st.gen_s,
+        "roofline": roofline_of(run, args, timing, ms_eager, peaks, peaks_kind),
+        "cuda_graph": {"ms_per_step_eager": ms_eager / steps} if args.graph else None,
     }
+    if with_e2e:
+        # ---- end to end from pinned host memory ----
+        for _ in range(min(3, warmup)):
+            run.step_host()
+        ms_e2e, _, _ = timed(run, rep, run.step_host, steps, kernel_timing=False)
+        elem = 2 if w.dtype == "bf16" else 4
+        h2d = (len(run.step_layers) * (2 * w.batch * w.D * elem + 2 * w.batch * 4)
+               + run.n_attend * w.batch * w.n_q_heads * w.head_dim * elem)
+        d2h = run.n_attend * w.batch * w.n_q_heads * w.head_dim * 4
+        same = bool(torch.equal(st.out_host[run.last], st.out[run.last].cpu()))
+        rec["e2e"] = {"value": rep.job_value(w.batch, ms_e2e / steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps, "matches_device_path": same}
+    return rec
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_value, sample, outs = time_oracle(st, step_layers, budget_s=12.0)
+
+def measure_uncompressed(run, rep, steps, peaks, peaks_kind):
+    """The uncompressed step at the same shape (every layer attends a full cache), beside the compressed one."""
+    torch = run.torch
+    w = run.w
+    if run.full:
+        return None
+    run.full_out = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=run.st.dev)
+    for _ in range(3):
+        run.step_uncompressed()
+    ms_total, timing, _ = timed(run, rep, run.step_uncompressed, steps)
+    stored_ms, stored_n = timing["stored"]
+    elem = 2 if w.dtype == "bf16" else 4
+    full_bytes = w.batch * w.context * 2.0 * w.D * elem
+    k_ms = stored_ms / max(stored_n, 1)
+    gbs = full_bytes / (k_ms * 1e-3) / 1e9
+    return {"ms_per_step": ms_total / steps, "layers_per_step": len(run.full_layers),
+            "kernel": "attn_stored_mma_kernel" if run.ctx.stored_path() == 1 else "attn_stored_kernel",
+            "kernel_ms": k_ms, "achieved_gbs": gbs, "frac_of_%s_hbm" % peaks_kind: gbs / float(peaks["hbm_gbs"]),
+            "what": "full-cache attention on every layer of the step (the layers that hold a full cache here, "
+                    "walked %d time(s))" % (len(run.full_layers) // max(1, len(set(run.full_layers))))}
+
+
+def sustained_leg(run, rep, ms_step, seconds, peaks, peaks_kind, args):
+    """The step repeated for at least `seconds`, with its own kernel times and clock samples."""
+    steps = max(3, int(math.ceil(seconds * 1e3 / ms_step)))
+    sampler = ClockSampler(physical_gpu_index(rep.local_rank))
+    sampler.start()
+    ms_total, timing, _ = timed(run, rep, run.step, steps)
+    clocks = sampler.stop()
+    roof = roofline_of(run, args, timing, ms_total, peaks, peaks_kind)
+    out = {"seconds": ms_total * 1e-3, "steps": steps, "ms_per_step": ms_total / steps,
+           "value": rep.job_value(run.w.batch, ms_total / steps), "kernel": roof.get("kernel"),
+           "kernel_ms": roof.get("kernel_ms"), "frac": roof.get("frac"), "unit": roof.get("unit"),
+           "achieved": roof.get("achieved"), "clocks": clocks}
+    for k in ("frac_of_burst_peak", "frac_of_sustained_peak", "anchor_layers"):
+        if k in roof:
+            out[k] = roof[k]
+    if clocks.get("sm_mhz") and roof.get("kernel_ms"):
+        # time x clock: compares kernels measured at different clocks (NVML's reading of the SM clock)
+        out["kernel_ms_x_sm_mhz"] = roof["kernel_ms"] * clocks["sm_mhz"]
+    return out
+
+
+def sub_args(args, **kw):
+    a = argparse.Namespace(**vars(args))
+    a.batch = a.context = a.page_tokens = 0
+    a.random_pages = False
+    a.ratio = 75
+    for k, v in kw.items():
+        setattr(a, k, v)
+    return a
+
+
+def run_suite(args, rep, peaks, peaks_kind):
+    """The default run: headline + sustained leg + one sub-record per benchmark configuration."""
+    import torch
+    from paper_2603_22910_b200 import binding
+    line, configs = None, {}
+    order = [HEADLINE] + [k for k, _ in SUITE if k != HEADLINE]
+    specs = dict(SUITE)
+    single_gpu = rep.world == 1
+    for key in order:
+        if key != HEADLINE and not single_gpu:
+            break                                  # the sub-records are a one-GPU matter
+        a = sub_args(args, **specs[key])
+        w = workload_of_args(a)
+        w = w.replace(seed=rep.seed_for(w.seed))
+        run = Run(w, a, rep.local_rank)
+        steps = args.steps if key == HEADLINE else max(10, min(args.steps, 30))
+        if w.n_layers > 2 and key != HEADLINE:
+            steps = min(steps, 10)
+        rec = measure(run, rep, a, steps, args.warmup, peaks, peaks_kind)
+        rec["steps"] = steps
+        rec["config"] = workload_config(w)
+        rec["decode_path"] = run.ctx.decode_path()
+        if key == HEADLINE:
+            rec["sustained"] = sustained_leg(run, rep, rec["ms_per_step"], args.sustained_s, peaks, peaks_kind, a)
+        if single_gpu and rep.rank == 0:
+            run.step()
+            torch.cuda.synchronize()
+            picks = stratified_picks(w, [l for l, at in run.step_layers if at], 8, seed=11, max_combos=2)
+            rec["parity_vs_oracle"] = parity_sample(run.st, picks)
+            if key == HEADLINE and not args.no_cpu_baseline:
+                cpu_value, sample, _ = time_oracle(run.st, run.step_layers, budget_s=10.0)
+                rec["cpu_baseline"] = {"value": cpu_value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                                       "sample": sample}
+            rec["uncompressed"] = measure_uncompressed(run, rep, steps, peaks, peaks_kind)
+        assert run.ctx.device_status() == binding.ECHOKV_OK
+        rec["input_generation_s"] = run.st.gen_s
+        configs[key] = rec
+        if key == HEADLINE:
+            line = headline_line(rec, w, a, rep, args, run)
+        run.close()
+        del run
+        torch.cuda.empty_cache()
+    if single_gpu:
+        line["configs"] = {k: summary_of(v) for k, v in configs.items()}
+    return line
+
+
+def summary_of(rec):
+    r = rec["roofline"]
+    out = {"workload": rec["config"]["workload"], "steps": rec["steps"], "ms_per_step": rec["ms_per_step"],
+           "tokens_per_s": rec["value"], "e2e_ms_per_step": rec["e2e"]["ms_per_step"],
+           "e2e_tokens_per_s": rec["e2e"]["value"], "kernel": r.get("kernel"), "kernel_ms": r.get("kernel_ms"),
+           "bound": r.get("bound"), "achieved": r.get("achieved"), "unit": r.get("unit"),
+           "frac_of_burst_peak": r.get("frac_of_burst_peak"), "frac_of_sustained_peak": r.get("frac_of_sustained_peak"),
+           "algorithmic_flops_per_launch": r.get("algorithmic_flops_per_launch"),
+           "clocks": rec["clocks"], "parity_vs_oracle": rec.get("parity_vs_oracle"),
+           "uncompressed": rec.get("uncompressed")}
+    if "anchor_layers" in r:
+        out["anchor_layers"] = r["anchor_layers"]
+    return out
+
+
+def headline_line(rec, w, a, rep, args, run):
+    line = {
+        "metric": METRIC, "value": rec["value"], "unit": UNIT, "n_gpus": rep.world, "steps": rec.get("steps", args.steps),
+        "warmup": args.warmup, "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": workload_config(w, run.full),
+        "us_per_layer_step": rec["us_per_layer_step"],
+        "kv_tokens_scanned_per_s": rec["kv_tokens_scanned_per_s"],
+        "clocks": rec["clocks"],
+        "e2e": rec["e2e"],
+        "gpu_launches": rec["gpu_launches"],
+        "roofline": rec["roofline"],
+        "decode_path": run.ctx.decode_path(), "stored_path": run.ctx.stored_path(),
+        "decode_mode": "absorbed" if run.absorbed else "explicit",
+        "cuda_graph": rec["cuda_graph"],
+        "full_precision_tokens": {"sink": run.window[0], "window": run.window[1]} if run.window else None,
+        "rope_theta": a.rope or None,
+        "input_generation_s": run.st.gen_s,
+    }
+    for k in ("sustained", "cpu_baseline", "parity_vs_oracle"):
+        if k in rec:
+            line[k] = rec[k]
+    return line
+
+
+def run_single(args, rep, peaks, peaks_kind):
+    """--workload given: that workload alone, with the command line's options."""
+    import numpy as np
+    import torch
+    w = workload_of_args(args)
+    w = w.replace(seed=rep.seed_for(w.seed))
+    run = Run(w, args, rep.local_rank)
+    rec = measure(run, rep, args, args.steps, args.warmup, peaks, peaks_kind)
+    rec["steps"] = args.steps
+    if args.sustained_s > 0:
+        rec["sustained"] = sustained_leg(run, rep, rec["ms_per_step"], args.sustained_s, peaks, peaks_kind, args)
+    if rep.rank == 0 and rep.world == 1 and not args.no_cpu_baseline:
+        st = run.st
+        cpu_value, sample, outs = time_oracle(st, run.step_layers, budget_s=12.0)
         worst_abs, num, den = 0.0, 0.0, 0.0
         for (l, b), ref in outs.items():
             gpu = st.out[l][b].cpu().numpy().astype(np.float64)
             worst_abs = max(worst_abs, float(np.max(np.abs(gpu - ref))))
             num += float(np.sum((gpu - ref) ** 2))
             den += float(np.sum(ref ** 2))
-        line["cpu_baseline"] = {"value": cpu_value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                                "sample": sample}
-        line["parity_vs_oracle"] = {"outputs": sorted(outs.keys()), "max_abs": worst_abs,
-                                    "rel_l2": (num / max(den, 1e-300)) ** 0.5}
-    if rank == 0:
+        rec["cpu_baseline"] = {"value": cpu_value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                               "sample": sample}
+        rec["parity_vs_oracle"] = {"outputs": sorted(outs.keys()), "max_abs": worst_abs,
+                                   "rel_l2": (num / max(den, 1e-300)) ** 0.5}
+    line = headline_line(rec, w, args, rep, args, run)
+    run.close()
+    return line
+
+
+def run_sweep(args, rep, peaks, peaks_kind):
+    """--workload c4 --sweep: every point of the sweep that fits the device, explicit, absorbed and uncompressed
+    steps side by side, each against its own roofline."""
+    import torch
+    points = []
+    burst = float(peaks["bf16_tflops"])
+    sustained = float(peaks.get("bf16_tflops_sustained") or burst)
+    hbm = float(peaks["hbm_gbs"])
+    ratios = [int(v) for v in args.sweep_ratios.split(",")]
+    contexts = [int(v) for v in args.sweep_contexts.split(",")]
+    batches = [int(v) for v in args.sweep_batches.split(",")]
+    for ratio in ratios:
+        for L in contexts:
+            for B in batches:
+                a = sub_args(args, workload="c4", ratio=ratio, context=L, batch=B)
+                w = workload_of_args(a)
+                cache_gb = B * L * 2 * (w.D + w.d_in) * 2 / 1e9      # anchor + compressed layer pools
+                if cache_gb > 120:
+                    points.append({"ratio": ratio, "context": L, "batch": B, "skipped": "%.0f GB of cache" % cache_gb})
+                    continue
+                run = Run(w, a, rep.local_rank)
+                steps = 20 if B * L <= 2 ** 20 else 8
+                for _ in range(3):
+                    run.step()
+                ms_exp, timing, _ = timed(run, rep, run.step, steps)
+                ref = run.st.out[1].clone()
+                run.full_out = torch.empty_like(ref)
+                for _ in range(3):
+                    run.step_uncompressed()
+                ms_full, timing_full, _ = timed(run, rep, run.step_uncompressed, steps)
+                run.ctx.enable_absorbed()
+                for _ in range(3):
+                    run.step()
+                ms_abs, _, _ = timed(run, rep, run.step, steps)
+                diff = float((run.st.out[1] - ref).norm() / ref.norm())
+                status = run.ctx.device_status()
+                flops, bytes_ = algorithmic_work(w)
+                recon_ms, recon_n = timing["recon"]
+                k_ms = recon_ms / max(recon_n, 1)
+                full_bytes = B * L * 2.0 * w.D * 2
+                points.append({
+                    "ratio": ratio, "context": L, "batch": B, "decode_path": run.ctx.decode_path(),
+                    "ms_explicit": ms_exp / steps, "kernel_ms": k_ms,
+                    "kernel_frac_of_burst_peak": flops / (k_ms * 1e-3) / 1e12 / burst,
+                    "step_frac_of_burst_peak": flops / (ms_exp / steps * 1e-3) / 1e12 / burst,
+                    "step_frac_of_sustained_peak": flops / (ms_exp / steps * 1e-3) / 1e12 / sustained,
+                    "ms_absorbed": ms_abs / steps, "absorbed_step_frac_of_hbm": bytes_ / (ms_abs / steps * 1e-3) / 1e9 / hbm,
+                    "ms_uncompressed": ms_full / steps,
+                    "uncompressed_step_frac_of_hbm": full_bytes / (ms_full / steps * 1e-3) / 1e9 / hbm,
+                    "rel_l2_absorbed_vs_explicit": diff, "device_status": status})
+                run.close()
+                del run, ref
+                torch.cuda.empty_cache()
+    done = [p for p in points if "ms_explicit" in p]
+    last = done[-1]
+    return {"metric": METRIC, "value": last["batch"] / (last["ms_explicit"] * 1e-3), "unit": UNIT, "n_gpus": rep.world,
+            "steps": 20, "warmup": 3, "ms_per_step": last["ms_explicit"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "c4 sweep on the Llama-3-8B layer shape: ratios %s x contexts %s x batches %s; "
+                                   "value / ms_per_step are the last point's" % (ratios, contexts, batches),
+                       "parallelism": "one GPU"},
+            "peaks": {"bf16_tflops_burst": burst, "bf16_tflops_sustained": sustained, "hbm_gbs": hbm,
+                      "source": peaks_kind},
+            "sweep": points}
+
+
+def run_ours(args):
+    import torch
+    from paper_2603_22910_b200 import binding, build
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    rep = Replicas("nccl", torch.device("cuda", local_rank))
+    if rep.rank == 0:
+        build.build()
+    rep.barrier()
+    binding.lib()
+    peaks, peaks_kind = load_peaks()
+    if args.sweep:
+        line = run_sweep(args, rep, peaks, peaks_kind)
+    elif args.workload is None:
+        line = run_suite(args, rep, peaks, peaks_kind)
+    else:
+        line = run_single(args, rep, peaks, peaks_kind)
+    if rep.rank == 0:
         print(json.dumps(line))
-    ctx.close()
     rep.close()
     return 0
 
@@ -823,15 +1216,22 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c1", choices=["c1", "c2", "c3", "c4"],
-                    help="c1 (default, the headline): Llama-2-7B-shaped layer; c2: Llama-3-8B-shaped GQA layer; "
-                         "c3: 32-layer Llama-2-7B-shaped decode step; c4: one point of the GQA sweep "
-                         "(--ratio, --context, --batch)")
+    ap.add_argument("--workload", default=None, choices=["c1", "c2", "c3", "c4"],
+                    help="default: the whole record (headline c3, the 32-layer decode step, plus one sub-record per "
+                         "configuration).  c1: Llama-2-7B-shaped layer; c2: Llama-3-8B-shaped GQA layer; c3: 32-layer "
+                         "Llama-2-7B-shaped decode step; c4: one point of the GQA sweep (--ratio, --context, --batch)")
     ap.add_argument("--mode", default="compressed", choices=["compressed", "full"],
                     help="compressed: decode attention of a compressed layer (the headline); full: the "
                          "uncompressed path, full-cache attention on the anchor layer")
+    ap.add_argument("--sweep", action="store_true", help="with --workload c4: the whole sweep, one sub-record per point")
+    ap.add_argument("--sweep-ratios", default="25,50,75")
+    ap.add_argument("--sweep-contexts", default="4096,16384,65536,131072")
+    ap.add_argument("--sweep-batches", default="1,8,32,64")
+    ap.add_argument("--sustained-s", type=float, default=None,
+                    help="repeat the step for at least this many seconds after the timed steps, with the clocks "
+                         "sampled (default 2 for the whole record, 0 with --workload)")
     ap.add_argument("--stored-path", type=int, default=None, choices=[0, 1],
                     help="kernel for stored heads: 0 CUDA-core, 1 TMA + tensor-core (default: the library's choice)")
     ap.add_argument("--decode-path", type=int, default=None, choices=[1, 2, 3],
@@ -846,9 +1246,7 @@ def main():
     ap.add_argument("--rope", type=float, default=0.0, help="theta of a rotary embedding applied when the cache is "
                     "read (the cache then holds un-rotated keys); 0 = none, as in the paper's configurations")
     ap.add_argument("--save-k", action="store_true", help="compressed layers keep their keys whole, only the values "
-                    "are predicted (the paper's \"save K\" ablation); needs --decode-mode absorbed")
-    ap.add_argument("--prefill-path", type=int, default=None, choices=[0, 1, 2],
-                    help="attention kernel of the prefill-shaped call (default: the library's)")
+                    "are predicted (the paper's \"save K\" ablation)")
     ap.add_argument("--prefill-queries", type=int, default=0, help="time the prefill-shaped call instead: this many "
                     "causal queries per sequence on the compressed layer (an extra measurement, its own JSON line)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -858,18 +1256,19 @@ def main():
     ap.add_argument("--ratio", type=int, default=75, choices=[25, 50, 75],
                     help="c4 only: percent of the layer's KV heads discarded")
     ap.add_argument("--retained-dims", type=int, default=0,
-                    help="c4 only: m in flat dims instead of --ratio, e.g. 64 or 384 (the paper's settings); a value "
-                         "that splits a head needs --decode-mode absorbed")
+                    help="c4 only: m in flat dims instead of --ratio, e.g. 64 or 384 (the paper's settings)")
     ap.add_argument("--page-tokens", type=int, default=0, choices=[0, 16, 32, 64, 128],
                     help="override the tokens per cache page (default 16)")
     ap.add_argument("--random-pages", action="store_true", help="pages of the pool in a seeded random order")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.workload == "c3" and args.steps == 50 and args.impl == "ours":
-        args.steps = 10      # a 32-layer step is ~25x a single layer-step
+    if args.sustained_s is None:
+        args.sustained_s = 2.0 if args.workload is None else 0.0
     if args.impl == "reference":
         return run_reference(args)
     if args.prefill_queries:
+        if args.workload is None:
+            args.workload = "c2"
         return run_prefill(args)
     return run_ours(args)
 
