@@ -920,7 +920,8 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   if (a.batch > kMaxBatchPerLaunch) return cudaErrorInvalidValue;
   const int g = a.n_q_heads / a.n_kv_heads;
   const int d_in = r.D + r.m;
-  const int n_ret = r.m / 128;           // (whole retained heads; used by the sink / window side kernel only)
+  const int m_heads = r.m_heads >= 0 ? r.m_heads : r.m / 128 * 128;
+  const int n_ret = m_heads / 128;       // whole retained heads: scored from the pool when the keys are rotated
   const AbsorbLayout& lay = r.lay;
   __nv_bfloat16* q2 = reinterpret_cast<__nv_bfloat16*>(r.ws + lay.off_q2);
   float* S = reinterpret_cast<float*>(r.ws + lay.off_s);
@@ -932,8 +933,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
   cudaError_t e;
 
   const bool rotated = a.rope.cs != nullptr;
-  if (rotated && !r.save_k && (r.m % 128 != 0 || !layer.weights_ready)) return cudaErrorInvalidValue;
-  if (r.save_k && (r.n_sink > 0 || r.n_window > 0)) return cudaErrorInvalidValue;
+  if (rotated && !r.save_k && !layer.weights_ready) return cudaErrorInvalidValue;
   // K side: features [anchor dims ; retained dims] and Wk^T q -- or, where the layer keeps its keys whole, the
   // layer's own D key dims with every query placed at its head's dims
   const int k_m = r.save_k ? r.D : r.m, k_anchor_dims = r.save_k ? 0 : r.D;
@@ -986,14 +986,17 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     // the layer's pool; both write the score rows the softmax below reads
     ReconArgs ra;
     ra.k_anchor = nullptr; ra.v_anchor = nullptr; ra.k_local = r.k_local; ra.v_local = r.v_local;
-    ra.Wk = r.Wk; ra.Wv = r.Wv; ra.bk = r.bk;
-    ra.D = r.D; ra.m = r.m;
+    ra.Wk = r.Wk_x != nullptr ? r.Wk_x : r.Wk; ra.Wv = r.Wv;
+    ra.bk = r.bk != nullptr ? (r.Wk_x != nullptr ? r.bk_x : r.bk) : nullptr;
+    ra.D = r.D; ra.m = r.m; ra.m_heads = m_heads;
     ra.part_tokens = 0;
     ra.capacity_tokens = capacity;
     ra.n_sink = r.n_sink; ra.n_window = r.n_window;
     if (ev) cudaEventRecord(ev[0], stream);
     if (r.save_k) {
-      if ((e = launch_key_scores_stored(a, r.k_local, r.D, a.n_kv_heads, S, lay.l_cap, 0, 0, stream)) != cudaSuccess) return e;
+      if ((e = launch_key_scores_stored(a, r.k_local, r.D, a.n_kv_heads, S, lay.l_cap, r.n_sink, r.n_window, stream)) !=
+          cudaSuccess)
+        return e;
     } else {
       if ((e = launch_recon_pair_key_scores(a, ra, anchor, layer, S, lay.l_cap, sm_count, stream)) != cudaSuccess) return e;
       if ((e = launch_key_scores_stored(a, r.k_local, r.m, n_ret, S, lay.l_cap, r.n_sink, r.n_window, stream)) != cudaSuccess)
@@ -1092,7 +1095,8 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     side.n_sink = r.n_sink; side.n_window = r.n_window; side.d_drop = r.D - r.m;
     SidePool pool;
     pool.k_pool = r.k_local; pool.v_pool = r.v_local; pool.width = r.m; pool.part = 0;
-    if ((e = launch_attn_side(a, side, n_ret, 1, stream, &pool)) != cudaSuccess) return e;
+    pool.k_width = r.save_k ? r.D : 0;
+    if ((e = launch_attn_side(a, side, 0, 1, stream, pool)) != cudaSuccess) return e;
     dim3 grid(a.n_q_heads, a.batch);
     absorb_combine_kernel<<<grid, 128, 0, stream>>>(out, ml, a.parts, a.n_q_heads,
                                                     reinterpret_cast<const __nv_bfloat16*>(a.q),

@@ -45,6 +45,11 @@ struct AbsorbArgs {
   unsigned char* ws;            // the absorbed-mode workspace
   AbsorbLayout lay;
   const void* Wk; const void* Wv; const void* bv;     // predictors of the layer ([D - m][D + m]), V bias or null
+  // rotated keys (a.rope set), where the K side is explicit: the K predictor and bias the tensor-core kernel reads
+  // -- where m splits a head, extended by the rows that pass the split head's stored dims through (kernels.h,
+  // ReconArgs::m_heads) -- and the flat dims of the whole retained heads (-1: m)
+  const void* Wk_x = nullptr; const void* bk_x = nullptr;
+  int m_heads = -1;
   const void* bk = nullptr;     // K bias or null; read only when the keys are rotated (a.rope set): it cancels otherwise
   const void* bk_shift = nullptr;   // K bias or null: un-rotated keys with sink / window tokens, against whose true keys
                                     // the predicted tokens' scores are shifted by q . b_k
@@ -61,8 +66,8 @@ struct AbsorbArgs {
 
 // One compressed layer, all query heads: out[B][H_q][d].  With a.rope set (keys cached before the rotary embedding) a
 // rotation that depends on the token sits between Eq. 3 and q . k, so W_k cannot be folded into the queries: the K
-// side is then explicit (predicted keys on the tensor cores, rotated, scored; stored heads scored from the pool; m
-// must be head-aligned) and only the V side uses the absorbed form.
+// side is then explicit (predicted keys on the tensor cores, rotated, scored; stored heads scored from the pool)
+// and only the V side uses the absorbed form.
 cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const AbsorbMaps& maps, const TcLayerMaps& anchor,
                             const TcLayerMaps& layer, float* out, int sm_count, cudaStream_t stream,
                             cudaEvent_t* timing_events /* 4 events or null: around the K pass and the V pass */);

@@ -23,8 +23,13 @@ struct Derived {
   int D, m, d_in, d_drop, g, elem, part_tokens, capacity, max_parts;
   int mk;              // K dims a compressed layer stores: m, or D in the "save K" setting
   bool save_k;
-  bool head_aligned;   // m ends on a head boundary (the explicit kernels need it; the absorbed mode does not)
-  uint64_t off_status, off_ml, off_o, off_q, off_k, off_v, off_out, off_lens, off_pos, total;
+  bool head_aligned;   // m ends on a head boundary
+  // Where m splits a head the explicit kernels treat that head as predicted: m_heads = flat dims of the whole
+  // retained heads, split = m - m_heads stored dims of the split head, which predictors extended by `split`
+  // one-hot rows pass through.  The extended predictors (and biases) of every compressed layer live in the workspace.
+  int m_heads, split;
+  uint64_t wx_bytes, bx_bytes;   // one extended predictor / bias (256-byte multiples), 0 when m is head-aligned
+  uint64_t off_status, off_ml, off_o, off_q, off_k, off_v, off_out, off_lens, off_pos, off_wx, total;
 };
 
 int derive(const echokv_config* c, Derived* d) {
@@ -52,6 +57,8 @@ int derive(const echokv_config* c, Derived* d) {
     d->m = c->n_retained_dims;
   }
   d->head_aligned = d->m % c->head_dim == 0;
+  d->m_heads = d->m / c->head_dim * c->head_dim;
+  d->split = d->m - d->m_heads;
   d->save_k = c->save_k != 0 && d->m < d->D;
   d->mk = d->save_k ? d->D : d->m;
   d->d_in = d->D + d->m;
@@ -73,6 +80,13 @@ int derive(const echokv_config* c, Derived* d) {
   d->off_out = off; off = align_up(off + (uint64_t)c->max_batch * c->n_q_heads * c->head_dim * 4);
   d->off_lens = off; off = align_up(off + (uint64_t)c->max_batch * 4);
   d->off_pos = off; off = align_up(off + (uint64_t)c->max_batch * 4);
+  d->off_wx = off;
+  d->wx_bytes = d->bx_bytes = 0;
+  if (d->split > 0) {
+    d->wx_bytes = align_up((uint64_t)(d->D - d->m_heads) * d->d_in * d->elem);
+    d->bx_bytes = align_up((uint64_t)(d->D - d->m_heads) * d->elem);
+    off += (uint64_t)c->n_layers * 2 * (d->wx_bytes + d->bx_bytes);     // K and V of every layer
+  }
   d->total = off;
   return ECHOKV_OK;
 }
@@ -84,6 +98,11 @@ struct Layer {
   const void* Wv = nullptr;
   const void* bk = nullptr;
   const void* bv = nullptr;
+  // what the explicit kernels read: the predictors as given, or (m splits a head) their extended copies
+  const void* Wk_x = nullptr;
+  const void* Wv_x = nullptr;
+  const void* bk_x = nullptr;
+  const void* bv_x = nullptr;
   bool anchor = false;
   void* k_side = nullptr;   // dropped dims of the sink and recent-window tokens (compressed layers)
   void* v_side = nullptr;
@@ -341,8 +360,8 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
   if (cudaMemset(c->ws + d.off_status, 0, kAlign) != cudaSuccess) { delete c; return ECHOKV_ECUDA; }
   c->tc_capable = tc_shape_supported(cfg->dtype, cfg->head_dim, cfg->page_tokens, d.D, d.m);
   if (!any_compressed || d.d_drop == 0) c->path = 0;
-  else if (!d.head_aligned || d.save_k) {
-    // a partly retained head, or keys kept whole: served by the absorbed mode only
+  else if (d.save_k) {
+    // keys kept whole: served by the absorbed mode only
     if (!absorbed_supported(cfg->dtype, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, d.m, cfg->page_tokens)) {
       delete c;
       return ECHOKV_EUNSUPPORTED;
@@ -401,8 +420,28 @@ int echokv_set_weights(echokv_ctx* c, int layer, const void* Wk, const void* Wv,
   if (c->d.d_drop > 0 && (!Wv || (!Wk && !c->d.save_k))) return ECHOKV_EINVAL;   // (keys kept whole: no K predictor)
   if ((reinterpret_cast<uintptr_t>(Wk) | reinterpret_cast<uintptr_t>(Wv)) % 16 != 0) return ECHOKV_EINVAL;
   L.Wk = Wk; L.Wv = Wv; L.bk = bk; L.bv = bv;
-  if (c->tc_capable && c->d.d_drop > 0) {
-    if (tc_encode_weight_maps(&L.tc, Wk, Wv, c->d.d_drop, c->d.d_in) != cudaSuccess) return ECHOKV_ECUDA;
+  L.Wk_x = Wk; L.Wv_x = Wv; L.bk_x = bk; L.bv_x = bv;
+  const Derived& d = c->d;
+  if (d.split > 0 && d.d_drop > 0) {
+    // m splits a head: build the extended predictors in the workspace (device work on the default stream, waited for)
+    if (cudaSetDevice(c->cfg.device) != cudaSuccess) return ECHOKV_ECUDA;
+    unsigned char* base = c->ws + d.off_wx + (uint64_t)layer * 2 * (d.wx_bytes + d.bx_bytes);
+    void* wkx = base; void* wvx = base + d.wx_bytes;
+    void* bkx = base + 2 * d.wx_bytes; void* bvx = base + 2 * d.wx_bytes + d.bx_bytes;
+    const int pass_col0 = d.D + d.m_heads;            // input column of local dim m_heads
+    if (Wk && launch_extend_predictor(c->cfg.dtype, Wk, bk, wkx, bkx, d.d_drop, d.d_in, d.split, pass_col0, nullptr) !=
+                  cudaSuccess)
+      return ECHOKV_ECUDA;
+    if (launch_extend_predictor(c->cfg.dtype, Wv, bv, wvx, bvx, d.d_drop, d.d_in, d.split, pass_col0, nullptr) !=
+        cudaSuccess)
+      return ECHOKV_ECUDA;
+    if (cudaStreamSynchronize(nullptr) != cudaSuccess) return ECHOKV_ECUDA;
+    c->launches += Wk ? 2 : 1;
+    L.Wk_x = Wk ? wkx : nullptr; L.Wv_x = wvx;
+    L.bk_x = (Wk && bk) ? bkx : nullptr; L.bv_x = bv ? bvx : nullptr;
+  }
+  if (c->tc_capable && d.d_drop > 0) {
+    if (tc_encode_weight_maps(&L.tc, L.Wk_x, L.Wv_x, d.D - d.m_heads, d.d_in) != cudaSuccess) return ECHOKV_ECUDA;
   }
   return ECHOKV_OK;
 }
@@ -439,19 +478,18 @@ int echokv_set_full_precision_window(echokv_ctx* c, int n_sink, int n_window, vo
                                      void* const* v_side) {
   if (!c || n_sink < 0 || n_window < 0) return ECHOKV_EINVAL;
   if (n_sink + n_window > 4096) return ECHOKV_EUNSUPPORTED;
-  if ((!c->d.head_aligned || c->d.save_k) && (n_sink > 0 || n_window > 0))
-    return ECHOKV_EUNSUPPORTED;   // (side buffers are per head, and hold K and V alike)
   const bool on = (n_sink > 0 || n_window > 0) && c->d.d_drop > 0;
+  const bool need_k = !c->d.save_k;     // (keys kept whole are in the pool already: no K side buffer is read or written)
   if (on) {
-    if (!k_side || !v_side) return ECHOKV_EINVAL;
+    if (!v_side || (need_k && !k_side)) return ECHOKV_EINVAL;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
       if (c->layers[l].anchor) continue;
-      if (!k_side[l] || !v_side[l]) return ECHOKV_EINVAL;
-      if ((reinterpret_cast<uintptr_t>(k_side[l]) | reinterpret_cast<uintptr_t>(v_side[l])) % 16 != 0)
+      if (!v_side[l] || (need_k && !k_side[l])) return ECHOKV_EINVAL;
+      if ((reinterpret_cast<uintptr_t>(need_k ? k_side[l] : nullptr) | reinterpret_cast<uintptr_t>(v_side[l])) % 16 != 0)
         return ECHOKV_EINVAL;
     }
     for (int l = 0; l < c->cfg.n_layers; ++l) {
-      c->layers[l].k_side = c->layers[l].anchor ? nullptr : k_side[l];
+      c->layers[l].k_side = (c->layers[l].anchor || !need_k) ? nullptr : k_side[l];
       c->layers[l].v_side = c->layers[l].anchor ? nullptr : v_side[l];
     }
   }
@@ -477,9 +515,9 @@ int echokv_set_rope(echokv_ctx* c, double theta, void* table, uint64_t table_byt
     return ECHOKV_OK;
   }
   if (!std::isfinite(theta) || theta < 1.0) return ECHOKV_EINVAL;
-  // a rotation that depends on the token cannot be folded into the queries: the K side stays explicit, which
-  // needs whole heads (unless the keys are kept whole anyway)
-  if (!c->d.head_aligned && !c->d.save_k) return ECHOKV_EUNSUPPORTED;
+  // (a rotation that depends on the token cannot be folded into the queries: the K side is then explicit, the
+  // tensor-core kernels for the predicted heads and the stored-head kernels for the rest)
+  if (!c->d.head_aligned && !c->d.save_k && !c->tc_capable) return ECHOKV_EUNSUPPORTED;
   uint64_t need = 0;
   const int rc = echokv_rope_table_bytes(&c->cfg, &need);
   if (rc != ECHOKV_OK) return rc;
@@ -587,11 +625,10 @@ int echokv_compress_layer(echokv_ctx* c, int layer, const void* k_full, const vo
   if (!c->table) return ECHOKV_ENOTABLE;
   const Layer& L = c->layers[layer];
   if (L.anchor) return ECHOKV_ENOTCOMPRESSED;
-  if (c->d.save_k) return ECHOKV_EUNSUPPORTED;
   const bool side = side_active(c, L);
-  if (c->d.m == 0 && !side) return ECHOKV_OK;          // nothing of this layer is kept
+  if (c->d.mk == 0 && !side) return ECHOKV_OK;         // nothing of this layer is kept
   const SideArgs sa = side_args(c, L);
-  if (launch_compress(c->d.elem, k_full, v_full, L.k_pool, L.v_pool, side ? &sa : nullptr, c->d.D, c->d.m,
+  if (launch_compress(c->d.elem, k_full, v_full, L.k_pool, L.v_pool, side ? &sa : nullptr, c->d.D, c->d.mk, c->d.m,
                       dev_seq_slots, dev_seq_begins, dev_seq_lens, B, geom_of(c), status_ptr(c),
                       static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return ECHOKV_ECUDA;
@@ -618,7 +655,7 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
   const Layer& L = c->layers[layer];
   const bool compressed = !L.anchor && c->d.d_drop > 0;
   if (c->cfg.dtype != ECHOKV_BF16 || c->cfg.head_dim != 128) return ECHOKV_EUNSUPPORTED;
-  if (compressed && (!c->tc_capable || !c->d.head_aligned || side_active(c, L))) return ECHOKV_EUNSUPPORTED;
+  if (compressed && (!c->tc_capable || side_active(c, L))) return ECHOKV_EUNSUPPORTED;
   const bool keys_whole = compressed && c->d.save_k;      // Section 5.2: nothing to predict on the K side
   if (n_q > c->d.capacity) return ECHOKV_ECAPACITY;
   const uint64_t rows_bytes = (uint64_t)B * c->d.capacity * c->d.D * 2ull;     // one of K~, V~
@@ -629,27 +666,30 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
   __nv_bfloat16* k_rows = static_cast<__nv_bfloat16*>(scratch);
   __nv_bfloat16* v_rows = k_rows + rows_bytes / 2;
   const int k_width = compressed ? c->d.mk : c->d.D, v_width = compressed ? c->d.m : c->d.D;
-  // stored dims as they are (keys rotated to their positions), then the predicted ones beside them
-  if (launch_gather_rows(a, L.k_pool, k_width, k_rows, c->d.capacity, c->d.D, true, 0, s) != cudaSuccess ||
-      launch_gather_rows(a, L.v_pool, v_width, v_rows, c->d.capacity, c->d.D, false, 128, s) != cudaSuccess)
+  // stored dims as they are (keys rotated to their positions), then the predicted ones beside them; of a head that m
+  // splits nothing is copied here: the extended predictor writes it whole (a rotation needs both halves of a head)
+  const int k_copy = (compressed && !keys_whole) ? c->d.m_heads : k_width;
+  const int v_copy = compressed ? c->d.m_heads : v_width;
+  if (launch_gather_rows(a, L.k_pool, k_width, k_copy, k_rows, c->d.capacity, c->d.D, true, 0, s) != cudaSuccess ||
+      launch_gather_rows(a, L.v_pool, v_width, v_copy, v_rows, c->d.capacity, c->d.D, false, 128, s) != cudaSuccess)
     return ECHOKV_ECUDA;
-  c->launches += (k_width > 0 ? 1 : 0) + 1;
+  c->launches += (k_copy > 0 ? 1 : 0) + 1;
   if (compressed) {
     const Layer& A = c->layers[layer - layer % c->cfg.group_size];
     ReconArgs ra;
     ra.k_anchor = A.k_pool; ra.v_anchor = A.v_pool;
     ra.k_local = L.k_pool; ra.v_local = L.v_pool;
-    ra.Wk = L.Wk; ra.Wv = L.Wv;
-    ra.D = c->d.D; ra.m = c->d.m;
+    ra.Wk = L.Wk_x; ra.Wv = L.Wv_x;
+    ra.D = c->d.D; ra.m = c->d.m; ra.m_heads = c->d.m_heads;
     ra.part_tokens = c->d.part_tokens;
     ra.capacity_tokens = c->d.capacity;
     ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
     if (!keys_whole) {
-      ra.bk = L.bk;
+      ra.bk = L.bk_x;
       if (launch_recon_pair_store(a, ra, A.tc, L.tc, false, k_rows, c->d.capacity, c->d.D, c->sm_count, s) != cudaSuccess)
         return ECHOKV_ECUDA;
     }
-    ra.bk = L.bv;
+    ra.bk = L.bv_x;
     if (launch_recon_pair_store(a, ra, A.tc, L.tc, true, v_rows, c->d.capacity, c->d.D, c->sm_count, s) != cudaSuccess)
       return ECHOKV_ECUDA;
     c->launches += keys_whole ? 1 : 2;
@@ -691,8 +731,9 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     aa.ws = c->ws_absorbed;
     aa.lay = c->alay;
     aa.Wk = L.Wk; aa.Wv = L.Wv; aa.bv = L.bv;
+    aa.Wk_x = L.Wk_x; aa.bk_x = L.bk_x; aa.m_heads = c->d.m_heads;     // rotated keys: the explicit K pass
     aa.bk = c->rope.cs != nullptr ? L.bk : nullptr;
-    aa.bk_shift = side && c->rope.cs == nullptr ? L.bk : nullptr;
+    aa.bk_shift = side && c->rope.cs == nullptr && !c->d.save_k ? L.bk : nullptr;
     aa.k_local = L.k_pool; aa.v_local = L.v_pool;
     aa.save_k = c->d.save_k;
     aa.D = c->d.D; aa.m = c->d.m;
@@ -710,9 +751,9 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     c->launches += (c->rope.cs != nullptr ? (c->d.save_k ? 5 : 5 + (c->d.m > 0 ? 1 : 0)) : 6) + (side ? 2 : 0);
     return ECHOKV_OK;
   }
-  if (!c->d.head_aligned || c->d.save_k)
-    return ECHOKV_EUNSUPPORTED;   // explicit reconstruction needs whole heads and predicts K as well: use the absorbed mode
-  const int r = c->d.m / c->cfg.head_dim;
+  if (c->d.save_k) return ECHOKV_EUNSUPPORTED;   // explicit reconstruction predicts K as well: use the absorbed mode
+  // whole retained heads; a head that m splits is predicted whole (its stored dims pass through the extended predictor)
+  const int r = c->d.m_heads / c->cfg.head_dim;
   // retained heads: Eq. 7 on what is stored (Eq. 6 keeps them as they are)
   const int n_splits = stored_splits(c, B, r);
   const int32_t* item_tokens = nullptr;
@@ -721,9 +762,9 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   ReconArgs ra;
   ra.k_anchor = A.k_pool; ra.v_anchor = A.v_pool;
   ra.k_local = L.k_pool; ra.v_local = L.v_pool;
-  ra.Wk = L.Wk; ra.Wv = L.Wv;
-  ra.bk = c->rope.cs != nullptr ? L.bk : nullptr;
-  ra.D = c->d.D; ra.m = c->d.m;
+  ra.Wk = L.Wk_x; ra.Wv = L.Wv_x;
+  ra.bk = c->rope.cs != nullptr ? L.bk_x : nullptr;
+  ra.D = c->d.D; ra.m = c->d.m; ra.m_heads = c->d.m_heads;
   ra.part_tokens = c->d.part_tokens;
   ra.capacity_tokens = c->d.capacity;
   ra.n_sink = side ? c->n_sink : 0;
@@ -743,13 +784,15 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   const int recon_part_tokens = c->path == 2 ? kTcPartTokens : c->d.part_tokens;
   if (side) {
     // sink and recent-window tokens: Eq. 7 on their stored dims, one more partial per query head
-    if (launch_attn_side(a, side_args(c, L), r, recon_part_tokens, s) != cudaSuccess) return ECHOKV_ECUDA;
+    SidePool pool;
+    pool.k_pool = L.k_pool; pool.v_pool = L.v_pool; pool.width = c->d.m; pool.part = -1;
+    if (launch_attn_side(a, side_args(c, L), r, recon_part_tokens, s, pool) != cudaSuccess) return ECHOKV_ECUDA;
     c->launches += 1;
   }
   // (a K bias is inside the scores already where the keys are rotated; otherwise it only matters against the
   // sink / window tokens, and the merge accounts for it)
-  if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, recon_part_tokens, L.bv, s,
-                   side ? 1 : 0, side && c->rope.cs == nullptr ? L.bk : nullptr) != cudaSuccess)
+  if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, recon_part_tokens, L.bv_x, s,
+                   side ? 1 : 0, side && c->rope.cs == nullptr ? L.bk_x : nullptr) != cudaSuccess)
     return ECHOKV_ECUDA;
   c->launches += 2;
   return ECHOKV_OK;

@@ -50,12 +50,24 @@ struct ReconArgs {
                                                 // are rotated after prediction: without a rotation it shifts every
                                                 // score of a head alike and cancels in the softmax
   int D, m;
+  int m_heads = -1;                             // flat dims of the WHOLE retained heads (a multiple of head_dim, <= m);
+                                                // -1: m.  Where m splits a head, the split head counts as predicted:
+                                                // Wk, Wv, bk then have D - m_heads rows, the first m - m_heads of
+                                                // them passing the head's stored dims through (one-hot rows)
   int part_tokens;                              // tokens per partial
   int capacity_tokens;                          // max_pages_per_seq * page_tokens
   int n_sink = 0, n_window = 0;                 // tokens kept at full precision: the first n_sink and the last
                                                 // n_window of a sequence are NOT predicted here (they are
                                                 // attended from the side buffers, see launch_attn_side)
 };
+
+// Whole retained heads of a compressed layer (the kernels' first predicted head).
+__host__ __device__ inline int retained_heads(const ReconArgs& r, int head_dim) { return (r.m_heads >= 0 ? r.m_heads : r.m) / head_dim; }
+
+// Predictor [d_drop][d_in] (+ bias [d_drop] or null) -> Wx [split + d_drop][d_in] (+ bx, may be null): `split`
+// one-hot rows in front that pass input columns pass_col0 .. pass_col0 + split - 1 through unchanged.
+cudaError_t launch_extend_predictor(int dtype, const void* W, const void* bias, void* Wx, void* bx, int d_drop,
+                                    int d_in, int split, int pass_col0, cudaStream_t stream);
 
 // Tokens of a sequence of `len` tokens that are predicted: [lo, hi) (Section 4.1: sink and recent-window
 // tokens keep all their dims).
@@ -80,23 +92,26 @@ cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, co
                                int32_t* status, cudaStream_t stream);
 
 // Evict a full-width cache ([n_pages][page_tokens][D], same block table) down to what a compressed layer keeps:
-// dims 0 .. m-1 of tokens [begins[b], lens[b]) into k_local / v_local (skipped when m == 0), dims m .. D-1 of the
-// sink / window tokens (window relative to lens[b]) into the side buffers (side may be null).  Bit-exact copies.
+// dims 0 .. mk-1 of the keys and 0 .. m-1 of the values of tokens [begins[b], lens[b]) into k_local / v_local
+// (skipped when 0), dims m .. D-1 of the sink / window tokens (window relative to lens[b]) into the side buffers
+// (side may be null; side->k_side may be null: keys kept whole).  Bit-exact copies.
 cudaError_t launch_compress(int elem_bytes, const void* k_full, const void* v_full, void* k_local, void* v_local,
-                            const SideArgs* side, int D, int m, const int32_t* slots, const int32_t* begins,
+                            const SideArgs* side, int D, int mk, int m, const int32_t* slots, const int32_t* begins,
                             const int32_t* lens, int B, const PageGeom& geom, int32_t* status, cudaStream_t stream);
 
-// Eq. 7 over the sink and window tokens of the dropped heads, from the side buffers: one split-K partial per
-// (sequence, query head of a dropped KV head), written at partial index ceil(len / part_tokens).
-// With `pool` given (the absorbed mode), the retained heads are covered too, from their stored dims in the
-// layer's pool, and every partial goes to index pool->part.
+// Eq. 7 over the sink and window tokens, at full precision, for the KV heads first_head .. n_kv_heads-1: one
+// split-K partial per (sequence, query head), written at partial index pool.part, or ceil(len / part_tokens)
+// when that is < 0.  Of every head the dims below pool.width (= m) come from the layer's pools and the rest from
+// the side buffers, so the call serves dropped heads, a head that m splits, and (the absorbed mode, first_head = 0)
+// retained heads alike.
 struct SidePool {
-  const void* k_pool; const void* v_pool;   // the layer's pools (row width `width` = m)
+  const void* k_pool; const void* v_pool;   // the layer's pools (row width `width` = m; may be null when m == 0)
   int width;
   int part;
+  int k_width = 0;                          // row width of the K pool where it differs (keys kept whole: D); 0: width
 };
-cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int n_ret_heads, int part_tokens,
-                             cudaStream_t stream, const SidePool* pool = nullptr);
+cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int first_head, int part_tokens,
+                             cudaStream_t stream, const SidePool& pool);
 
 // CUDA-core reconstruct-then-attend (fp32 or bf16 storage, fp32 FFMA): Eq. 3, 6, 7 for the
 // dropped KV heads; one partial per part_tokens tokens.

@@ -23,10 +23,11 @@ namespace echokv {
 namespace {
 
 // ---------------------------------------------------------------------------------------------
-// 1. stored dims of a paged pool -> out[b][t][out_width] at flat dims 0 .. width-1 (whole heads of 128)
+// 1. stored dims of a paged pool (rows of `width` dims) -> out[b][t][out_width] at flat dims 0 .. copy_width-1
+//    (whole heads of 128)
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* __restrict__ pool, int width,
-                                                          __nv_bfloat16* __restrict__ out, int out_tokens,
+                                                          int copy_width, __nv_bfloat16* __restrict__ out, int out_tokens,
                                                           int out_width, const int32_t* __restrict__ slots,
                                                           const int32_t* __restrict__ lens, PageGeom g, RopeTable rope,
                                                           int zero_tail, int block_tokens, int32_t* status) {
@@ -47,8 +48,8 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
             make_uint4(0u, 0u, 0u, 0u);
     }
   }
-  if (t0 >= len) return;
-  const int n_heads = width / 128;
+  if (t0 >= len || copy_width == 0) return;
+  const int n_heads = copy_width / 128;
   // item = (token of the tile, head, 8-dim piece c of the head's first half, with its partner piece 64 dims on);
   // a thread takes four items at a time: four page look-ups, then eight loads, then the stores, so that they overlap
   constexpr int kBatch = 4;
@@ -926,14 +927,14 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
 }  // namespace
 
-cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, __nv_bfloat16* out, int out_tokens,
-                               int out_width, bool rotate, int zero_tail, cudaStream_t stream) {
-  if (width == 0 && zero_tail == 0) return cudaSuccess;
-  if (width % 128 != 0 || out_width % 8 != 0) return cudaErrorInvalidValue;
+cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, int copy_width, __nv_bfloat16* out,
+                               int out_tokens, int out_width, bool rotate, int zero_tail, cudaStream_t stream) {
+  if (copy_width == 0 && zero_tail == 0) return cudaSuccess;
+  if (copy_width % 128 != 0 || copy_width > width || out_width % 8 != 0) return cudaErrorInvalidValue;
   // enough tokens per block that every thread has four items to overlap
-  const int block_tokens = width <= 256 ? 64 : 32;
+  const int block_tokens = copy_width <= 256 ? 64 : 32;
   dim3 grid((out_tokens + block_tokens - 1) / block_tokens, a.batch);
-  gather_rows_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(pool), width, out, out_tokens,
+  gather_rows_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(pool), width, copy_width, out, out_tokens,
                                                out_width, a.slots, a.lens, a.geom, rotate ? a.rope : RopeTable(), zero_tail,
                                                block_tokens, a.status);
   return cudaGetLastError();

@@ -5,11 +5,12 @@
 
 namespace echokv {
 
-// Stored dims 0 .. width-1 (whole heads of 128, bf16) of every cached token, from a paged pool into contiguous rows
-// out[b][token][out_width]; keys are rotated to their positions if `rotate` and a.rope is set.  zero_tail > 0 also
-// writes zeros over the whole rows len .. (next multiple of zero_tail) - 1 (launched even when width is 0).
-cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, __nv_bfloat16* out, int out_tokens,
-                               int out_width, bool rotate, int zero_tail, cudaStream_t stream);
+// Stored dims 0 .. copy_width-1 (whole heads of 128, bf16) of every cached token, from a paged pool whose rows hold
+// `width` dims into contiguous rows out[b][token][out_width]; keys are rotated to their positions if `rotate` and
+// a.rope is set.  zero_tail > 0 also writes zeros over the whole rows len .. (next multiple of zero_tail) - 1
+// (launched even when copy_width is 0).
+cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, int copy_width, __nv_bfloat16* out,
+                               int out_tokens, int out_width, bool rotate, int zero_tail, cudaStream_t stream);
 
 // Eq. 7 for n_q queries per sequence (a.q: [B][n_q][H_q][128] bf16), query i at position len - n_q + i attending the
 // keys up to its own, over k_rows / v_rows [B][kv_tokens][kv_width] bf16.  out: fp32 [B][n_q][H_q][128].

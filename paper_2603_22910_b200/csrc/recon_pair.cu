@@ -220,7 +220,10 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
   const int boxes = kCtaTokens / p.page_tokens;             // TMA boxes (pages) of this CTA's tokens
   const uint32_t page_bytes = p.page_tokens * kRowBytes;
   const uint32_t peer_abort = mapa_u32(smem_u32(&t.abort_flag), rank ^ 1u);
-  const int n_steps = p.kc_total / kStageChunks;            // stages per phase (kc_total is even)
+  // stages per phase: two chunks each.  With an odd number of chunks (a retained width that is an odd multiple
+  // of 64) the last stage's second chunk lies past the end of the pool rows and of the predictor rows: TMA fills
+  // both with zeros, which add nothing to the accumulators
+  const int n_steps = (p.kc_total + kStageChunks - 1) / kStageChunks;
   bool gave_up = false;
 
   if (warp == 0 || warp == 10) {
@@ -693,7 +696,7 @@ static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const
   p.max_parts = a.parts.max_parts;
   p.status = a.status;
   p.n_q_heads = a.n_q_heads;
-  p.n_ret_heads = r.m / 128;
+  p.n_ret_heads = retained_heads(r, 128);
   p.n_drop_heads = a.n_kv_heads - p.n_ret_heads;
   p.n_pairs = (p.n_drop_heads + 1) / 2;
   p.kc_anchor = r.D / kChunk;
@@ -717,7 +720,7 @@ static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const
   const CUtensorMap& lvr = r.m > 0 ? layer.v_pool_run : anchor.v_pool_run;
   const CUtensorMap& lk8 = r.m > 0 ? layer.k_pool_run128 : anchor.k_pool_run128;
   const CUtensorMap& lv8 = r.m > 0 ? layer.v_pool_run128 : anchor.v_pool_run128;
-  if (p.kc_total % kStageChunks != 0 || p.kc_anchor % kStageChunks != 0) return cudaErrorInvalidValue;
+  if (p.kc_anchor % kStageChunks != 0) return cudaErrorInvalidValue;   // (a stage never straddles the two pools)
   const int tiles_cap = (r.capacity_tokens + kTileTokens - 1) / kTileTokens;
   for (int b0 = 0; b0 < a.batch; b0 += kMaxBatchPerLaunch) {
     p.b0 = b0;

@@ -628,20 +628,13 @@ cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, int k_wid
     // boxes of 64 token rows: runs of consecutive pages, or part of a page that is taller
     if ((e = encode_2d(&maps->k_pool_run, k_pool, rows, k_width, kRunTokens, promo)) != cudaSuccess) return e;
     // CTA-pair kernel: 128 consecutive token rows x two 64-feature chunks in one copy
-    if (k_width >= 128) {     // (a pool one chunk wide is never read two chunks at a time)
-      if ((e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, k_width, 128, 2, promo)) != cudaSuccess) return e;
-    } else {
-      maps->k_pool_run128 = maps->k_pool_run;
-    }
+    // (of a pool one chunk wide the box's second chunk lies outside the tensor and reads as zeros)
+    if ((e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, k_width, 128, 2, promo)) != cudaSuccess) return e;
   }
   if (v_width > 0) {
     if ((e = encode_2d(&maps->v_pool, v_pool, rows, v_width, page_tokens, promo)) != cudaSuccess) return e;
     if ((e = encode_2d(&maps->v_pool_run, v_pool, rows, v_width, kRunTokens, promo)) != cudaSuccess) return e;
-    if (v_width >= 128) {
-      if ((e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, v_width, 128, 2, promo)) != cudaSuccess) return e;
-    } else {
-      maps->v_pool_run128 = maps->v_pool_run;
-    }
+    if ((e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, v_width, 128, 2, promo)) != cudaSuccess) return e;
     // absorbed mode, V side: 64 consecutive token rows x four 64-feature chunks in one copy
     if (v_width >= 256) {
       if ((e = encode_3d_chunks(&maps->v_pool_tok64x4, v_pool, rows, v_width, 64, 4, promo)) != cudaSuccess) return e;
@@ -686,7 +679,7 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
   p.max_parts = a.parts.max_parts;
   p.status = a.status;
   p.n_q_heads = a.n_q_heads;
-  p.n_ret_heads = r.m / 128;
+  p.n_ret_heads = retained_heads(r, 128);
   p.n_drop_heads = a.n_kv_heads - p.n_ret_heads;
   p.n_pairs = (p.n_drop_heads + 1) / 2;
   p.kc_anchor = r.D / kChunk;

@@ -109,13 +109,14 @@ cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int k_width, in
 // The switch from full-cache generation to compressed inference (Section 3.1: compression is evicting
 // part of each token's K / V; Section 5.4: done only once memory runs short, or during prefill): rows of a
 // full-width cache are cut down to what a compressed layer keeps.  One block per (page of a sequence):
-// dims 0 .. m-1 of every token go to the layer's pools (Eq. 2), dims m .. D-1 of sink / window tokens to the
-// side buffers.  Plain 16-byte copies: bit-exact.
+// dims 0 .. m-1 of every token go to the layer's pools (Eq. 2; the keys' first mk dims, mk = D where a layer keeps
+// its keys whole), dims m .. D-1 of sink / window tokens to the side buffers (values only where the keys are
+// whole).  Plain 16-byte copies: bit-exact.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) compress_kernel(const uint4* __restrict__ k_full, const uint4* __restrict__ v_full,
                                                        uint4* __restrict__ k_local, uint4* __restrict__ v_local,
                                                        uint4* __restrict__ k_side, uint4* __restrict__ v_side,
-                                                       int d_vec, int m_vec, int n_sink, int n_window,
+                                                       int d_vec, int mk_vec, int m_vec, int n_sink, int n_window,
                                                        const int32_t* __restrict__ slots,
                                                        const int32_t* __restrict__ begins,
                                                        const int32_t* __restrict__ lens, PageGeom g, int32_t* status) {
@@ -140,15 +141,20 @@ __global__ void __launch_bounds__(256) compress_kernel(const uint4* __restrict__
     return;
   }
   const size_t row0 = (size_t)page * P;
+  if (mk_vec > 0) {
+    for (int idx = r_lo * mk_vec + threadIdx.x; idx < r_hi * mk_vec; idx += blockDim.x) {
+      const int r = idx / mk_vec, v = idx - r * mk_vec;
+      k_local[(row0 + r) * mk_vec + v] = k_full[(row0 + r) * d_vec + v];
+    }
+  }
   if (m_vec > 0) {
     for (int idx = r_lo * m_vec + threadIdx.x; idx < r_hi * m_vec; idx += blockDim.x) {
       const int r = idx / m_vec, v = idx - r * m_vec;
-      k_local[(row0 + r) * m_vec + v] = k_full[(row0 + r) * d_vec + v];
       v_local[(row0 + r) * m_vec + v] = v_full[(row0 + r) * d_vec + v];
     }
   }
   const int drop_vec = d_vec - m_vec;
-  if (k_side != nullptr && drop_vec > 0 && (t0 + r_lo < n_sink || t0 + r_hi > len - n_window)) {
+  if (v_side != nullptr && drop_vec > 0 && (t0 + r_lo < n_sink || t0 + r_hi > len - n_window)) {
     const size_t seq_base = (size_t)slot * (n_sink + n_window);
     for (int idx = r_lo * drop_vec + threadIdx.x; idx < r_hi * drop_vec; idx += blockDim.x) {
       const int r = idx / drop_vec, v = idx - r * drop_vec;
@@ -156,11 +162,11 @@ __global__ void __launch_bounds__(256) compress_kernel(const uint4* __restrict__
       const uint4 kv = k_full[(row0 + r) * d_vec + m_vec + v];
       const uint4 vv = v_full[(row0 + r) * d_vec + m_vec + v];
       if (t < n_sink) {
-        k_side[(seq_base + t) * drop_vec + v] = kv;
+        if (k_side != nullptr) k_side[(seq_base + t) * drop_vec + v] = kv;
         v_side[(seq_base + t) * drop_vec + v] = vv;
       }
       if (n_window > 0 && t >= len - n_window) {
-        k_side[(seq_base + n_sink + t % n_window) * drop_vec + v] = kv;
+        if (k_side != nullptr) k_side[(seq_base + n_sink + t % n_window) * drop_vec + v] = kv;
         v_side[(seq_base + n_sink + t % n_window) * drop_vec + v] = vv;
       }
     }
@@ -168,13 +174,13 @@ __global__ void __launch_bounds__(256) compress_kernel(const uint4* __restrict__
 }
 
 cudaError_t launch_compress(int elem_bytes, const void* k_full, const void* v_full, void* k_local, void* v_local,
-                            const SideArgs* side, int D, int m, const int32_t* slots, const int32_t* begins,
+                            const SideArgs* side, int D, int mk, int m, const int32_t* slots, const int32_t* begins,
                             const int32_t* lens, int B, const PageGeom& geom, int32_t* status, cudaStream_t stream) {
-  const int d_vec = D * elem_bytes / 16, m_vec = m * elem_bytes / 16;
+  const int d_vec = D * elem_bytes / 16, mk_vec = mk * elem_bytes / 16, m_vec = m * elem_bytes / 16;
   dim3 grid(geom.max_pages_per_seq, B);
   compress_kernel<<<grid, 256, 0, stream>>>(
       (const uint4*)k_full, (const uint4*)v_full, (uint4*)k_local, (uint4*)v_local,
-      side ? (uint4*)side->k_side : nullptr, side ? (uint4*)side->v_side : nullptr, d_vec, m_vec,
+      side ? (uint4*)side->k_side : nullptr, side ? (uint4*)side->v_side : nullptr, d_vec, mk_vec, m_vec,
       side ? side->n_sink : 0, side ? side->n_window : 0, slots, begins, lens, geom, status);
   return cudaGetLastError();
 }
@@ -669,7 +675,7 @@ __global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r
   extern __shared__ __align__(16) unsigned char smem_raw[];
   ReconSmem<DH>& sm = *reinterpret_cast<ReconSmem<DH>*>(smem_raw);
   const int part = blockIdx.x, b = blockIdx.z;
-  const int n_ret = r.m / DH;
+  const int n_ret = retained_heads(r, DH);
   const int kvh = n_ret + blockIdx.y;                 // dropped KV head
   const int g = a.n_q_heads / a.n_kv_heads;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -785,7 +791,7 @@ __global__ void __launch_bounds__(128) recon_simt_kernel(AttnArgs a, ReconArgs r
 
 template <typename T, int DH>
 static cudaError_t launch_recon_simt_t(const AttnArgs& a, const ReconArgs& r, cudaStream_t stream) {
-  const int n_drop = a.n_kv_heads - r.m / DH;
+  const int n_drop = a.n_kv_heads - retained_heads(r, DH);
   const int n_parts = (r.capacity_tokens + r.part_tokens - 1) / r.part_tokens;
   const size_t smem = sizeof(ReconSmem<DH>);
   cudaError_t e = cudaFuncSetAttribute(recon_simt_kernel<T, DH>,
@@ -920,6 +926,41 @@ cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int 
 }
 
 // ---------------------------------------------------------------------------------------------
+// A retained width m that splits a head (Eq. 6 concatenates at the flat index m, wherever it falls): the
+// explicit kernels work on whole heads, so the split head is treated as predicted and its stored dims are
+// passed through the predictor by `split` one-hot rows put in front of W -- row i < split copies local dim
+// m_heads + i (input column D + m_heads + i); multiplying a stored bf16 / fp32 value by 1 and adding zeros
+// is exact, so the rebuilt head holds the stored dims bit for bit.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) extend_predictor_kernel(const T* __restrict__ W, const T* __restrict__ bias,
+                                                               T* __restrict__ Wx, T* __restrict__ bx, int d_in,
+                                                               int split, int pass_col0) {
+  const int row = blockIdx.x;                       // row of the extended matrix
+  T* dst = Wx + (size_t)row * d_in;
+  if (row < split) {
+    for (int c = threadIdx.x; c < d_in; c += blockDim.x) dst[c] = c == pass_col0 + row ? T(1.0f) : T(0.0f);
+  } else {
+    const T* src = W + (size_t)(row - split) * d_in;
+    for (int c = threadIdx.x; c < d_in; c += blockDim.x) dst[c] = src[c];
+  }
+  if (threadIdx.x == 0 && bx != nullptr) bx[row] = (row < split || bias == nullptr) ? T(0.0f) : bias[row - split];
+}
+
+cudaError_t launch_extend_predictor(int dtype, const void* W, const void* bias, void* Wx, void* bx, int d_drop,
+                                    int d_in, int split, int pass_col0, cudaStream_t stream) {
+  const int rows = d_drop + split;
+  if (dtype == ECHOKV_BF16)
+    extend_predictor_kernel<__nv_bfloat16><<<rows, 256, 0, stream>>>((const __nv_bfloat16*)W, (const __nv_bfloat16*)bias,
+                                                                  (__nv_bfloat16*)Wx, (__nv_bfloat16*)bx, d_in, split,
+                                                                  pass_col0);
+  else
+    extend_predictor_kernel<float><<<rows, 256, 0, stream>>>((const float*)W, (const float*)bias, (float*)Wx, (float*)bx,
+                                                          d_in, split, pass_col0);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Sink and recent-window tokens at full precision (Section 4.1): their dropped dims live in small
 // side buffers; these two kernels write and attend them.
 // ---------------------------------------------------------------------------------------------
@@ -949,10 +990,10 @@ __global__ void __launch_bounds__(128) append_side_kernel(T* __restrict__ k_side
     int idx;
     if (which == 0) { if (pos >= n_sink) continue; idx = pos; }
     else { if (n_window == 0 || i_tok < n_tok - n_window) continue; idx = n_sink + pos % n_window; }
-    uint4* kd = reinterpret_cast<uint4*>(k_side + (seq_base + idx) * d_drop);
+    uint4* kd = k_side != nullptr ? reinterpret_cast<uint4*>(k_side + (seq_base + idx) * d_drop) : nullptr;
     uint4* vd = reinterpret_cast<uint4*>(v_side + (seq_base + idx) * d_drop);
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
-      kd[i] = ks[i];
+      if (kd != nullptr) kd[i] = ks[i];        // (no K side buffer where the keys are kept whole)
       vd[i] = vs[i];
     }
   }
@@ -975,24 +1016,30 @@ cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, co
 }
 
 // One block per (KV head, sequence): scores of the <= n_sink + n_window full-precision tokens against the
-// group's query heads, softmax, weighted V; one partial per query head.  A dropped head reads the side
-// buffers; a retained head (only asked for by the absorbed mode, first_head = 0) reads its stored dims
-// from the layer's pool.  The partial goes to index fixed_part, or ceil(len / part_tokens) if that is < 0.
+// group's query heads, softmax, weighted V; one partial per query head.  Of a head's DH dims the first
+// n_stored = clamp(m - head * DH, 0, DH) are read from the layer's pool (row width m) and the rest from the side
+// buffers (dims m .. D-1): a dropped head reads the side buffers only, a head that m splits reads half and half, a
+// retained head (only asked for by the absorbed mode, first_head = 0) reads the pool only.  The K pool may be wider
+// than the V pool (mk > m: keys kept whole); the keys' side buffer is then not read at all.
+// The partial goes to index fixed_part, or ceil(len / part_tokens) if that is < 0.
 template <typename T, int DH>
 __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __restrict__ k_side,
                                                         const T* __restrict__ v_side, int n_sink, int n_window,
-                                                        int d_drop, int n_ret, int part_tokens, int first_head,
+                                                        int d_drop, int mk, int m, int part_tokens, int first_head,
                                                         int fixed_part, const T* __restrict__ k_pool,
-                                                        const T* __restrict__ v_pool, int pool_width) {
+                                                        const T* __restrict__ v_pool) {
   extern __shared__ float side_smem[];
   const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = a.n_q_heads / a.n_kv_heads;
   const int kvh = first_head + blockIdx.x;
-  const int dh = kvh - n_ret;                  // index among the dropped heads (< 0: a retained head)
+  const int n_stored_k = min(max(mk - kvh * DH, 0), DH);  // 0, DH / 2 or DH (m is a multiple of 64)
+  const int n_stored = min(max(m - kvh * DH, 0), DH);     // the same for the values
   const int n_side = n_sink + n_window;
   float* qs = side_smem;                      // [g][DH]
   float* sc = qs + kMaxGroup * DH;            // [g][n_side]
-  unsigned long long* rows = reinterpret_cast<unsigned long long*>(sc + kMaxGroup * n_side);   // [n_side]
+  // element offsets of every full-precision token's row: [0] in the K pool, [1] in the V pool (the head's dim 0),
+  // [2] in the side buffers (dim m)
+  unsigned long long* rows = reinterpret_cast<unsigned long long*>(sc + kMaxGroup * n_side);   // [3][n_side]
   __shared__ float red[4][kMaxGroup];
   __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
   const int slot = a.slots ? a.slots[b] : b;
@@ -1007,25 +1054,30 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     qs[idx] = to_f32(q[((size_t)b * a.n_q_heads + kvh * g) * DH + idx]) * a.scale_log2e;
   __syncthreads();
   const size_t seq_base = (size_t)slot * n_side;
-  const T* k_src = dh >= 0 ? k_side : k_pool;
-  const T* v_src = dh >= 0 ? v_side : v_pool;
   const int32_t* table = a.geom.table + (size_t)slot * a.geom.max_pages_per_seq;
-  auto side_row = [&](int i) -> size_t {       // i-th full-precision token -> offset of its head's dims
-    const int t = i < lo ? i : hi + (i - lo);
-    if (dh >= 0) return (seq_base + (t < lo ? t : n_sink + t % n_window)) * (size_t)d_drop + (size_t)dh * DH;
-    int page = table[t / a.geom.page_tokens];
-    if (page < 0 || page >= a.geom.n_pages) {
-      report(a.status, ECHOKV_EBADPAGE);
-      page = 0;
-    }
-    return ((size_t)page * a.geom.page_tokens + t % a.geom.page_tokens) * (size_t)pool_width + (size_t)kvh * DH;
-  };
   // where each full-precision token lives (looked up once: the loops below must not chase the block table)
-  for (int i = tid; i < n_tok; i += 128) rows[i] = side_row(i);
+  for (int i = tid; i < n_tok; i += 128) {
+    const int t = i < lo ? i : hi + (i - lo);
+    if (n_stored_k > 0) {
+      int page = table[t / a.geom.page_tokens];
+      if (page < 0 || page >= a.geom.n_pages) {
+        report(a.status, ECHOKV_EBADPAGE);
+        page = 0;
+      }
+      const size_t r = (size_t)page * a.geom.page_tokens + t % a.geom.page_tokens;
+      rows[i] = r * (size_t)mk + (size_t)kvh * DH;
+      rows[n_side + i] = r * (size_t)m + (size_t)kvh * DH;
+    }
+    // (offset of flat dim m; a head's first dim that is not stored is added where it is read)
+    rows[2 * n_side + i] = (seq_base + (t < lo ? t : n_sink + t % n_window)) * (size_t)d_drop;
+  }
   __syncthreads();
+  // address of dims [j, j + vector) of token i's key / value row (a vector never straddles n_stored)
+  auto k_at = [&](int i, int j) -> const T* {
+    return j < n_stored_k ? k_pool + rows[i] + j : k_side + rows[2 * n_side + i] + (kvh * DH + j - mk);
+  };
   // scores: one token per thread
   for (int i = tid; i < n_tok; i += 128) {
-    const T* kr = k_src + rows[i];
     float acc[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
@@ -1034,8 +1086,8 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
       const float2* cs = a.rope.cs + (i < lo ? i : hi + (i - lo));
       for (int j = 0; j < DH / 2; j += Vec16<T>::N) {
         float k_lo[Vec16<T>::N], k_hi[Vec16<T>::N];
-        Vec16<T>::load(kr + j, k_lo);
-        Vec16<T>::load(kr + DH / 2 + j, k_hi);
+        Vec16<T>::load(k_at(i, j), k_lo);
+        Vec16<T>::load(k_at(i, DH / 2 + j), k_hi);
 #pragma unroll
         for (int e = 0; e < Vec16<T>::N; ++e) {
           const float2 w = cs[(size_t)(j + e) * a.rope.stride];
@@ -1048,7 +1100,7 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     } else {
       for (int j = 0; j < DH; j += Vec16<T>::N) {
         float kv[Vec16<T>::N];
-        Vec16<T>::load(kr + j, kv);
+        Vec16<T>::load(k_at(i, j), kv);
 #pragma unroll
         for (int gi = 0; gi < kMaxGroup; ++gi)
           if (gi < g) {
@@ -1064,10 +1116,10 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
   __syncthreads();
   // max and sum per query head
   for (int gi = 0; gi < g; ++gi) {
-    float m = -INFINITY;
-    for (int i = tid; i < n_tok; i += 128) m = fmaxf(m, sc[gi * n_side + i]);
-    m = warp_max(m);
-    if (lane == 0) red[warp][gi] = m;
+    float mx = -INFINITY;
+    for (int i = tid; i < n_tok; i += 128) mx = fmaxf(mx, sc[gi * n_side + i]);
+    mx = warp_max(mx);
+    if (lane == 0) red[warp][gi] = mx;
   }
   __syncthreads();
   if (tid < g) s_m[tid] = fmaxf(fmaxf(red[0][tid], red[1][tid]), fmaxf(red[2][tid], red[3][tid]));
@@ -1089,12 +1141,15 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
   // weighted V: one output feature per thread
   const int part = fixed_part >= 0 ? fixed_part : (len + part_tokens - 1) / part_tokens;
   if (tid < DH) {
+    const bool from_pool = tid < n_stored;
+    const T* v_src = from_pool ? v_pool + tid : v_side + (kvh * DH + tid - m);
+    const unsigned long long* v_rows = from_pool ? rows + n_side : rows + 2 * n_side;
     float o[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
 #pragma unroll 4
     for (int i = 0; i < n_tok; ++i) {
-      const float vv = to_f32(v_src[rows[i] + tid]);
+      const float vv = to_f32(v_src[v_rows[i]]);
 #pragma unroll
       for (int gi = 0; gi < kMaxGroup; ++gi)
         if (gi < g) o[gi] = fmaf(sc[gi * n_side + i], vv, o[gi]);
@@ -1108,31 +1163,31 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
 }
 
 template <typename T, int DH>
-static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, int n_ret, int part_tokens,
-                                      cudaStream_t stream, const SidePool* pool) {
-  const int first_head = pool ? 0 : n_ret;
+static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, int first_head, int part_tokens,
+                                      cudaStream_t stream, const SidePool& pool) {
   const int n_heads = a.n_kv_heads - first_head;
   const int n_side = side.n_sink + side.n_window;
-  const size_t smem = (size_t)(kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float) + (size_t)n_side * 8 + 8;
+  const size_t smem = (size_t)(kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float) + (size_t)n_side * 24 + 8;
   cudaError_t e = cudaFuncSetAttribute(attn_side_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
+  if (n_heads <= 0) return cudaSuccess;
   dim3 grid(n_heads, a.batch);
   attn_side_kernel<T, DH><<<grid, 128, smem, stream>>>(
-      a, (const T*)side.k_side, (const T*)side.v_side, side.n_sink, side.n_window, side.d_drop, n_ret, part_tokens,
-      first_head, pool ? pool->part : -1, pool ? (const T*)pool->k_pool : nullptr,
-      pool ? (const T*)pool->v_pool : nullptr, pool ? pool->width : 0);
+      a, (const T*)side.k_side, (const T*)side.v_side, side.n_sink, side.n_window, side.d_drop,
+      pool.k_width > 0 ? pool.k_width : pool.width, pool.width, part_tokens, first_head, pool.part,
+      (const T*)pool.k_pool, (const T*)pool.v_pool);
   return cudaGetLastError();
 }
 
-cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int n_ret_heads, int part_tokens,
-                             cudaStream_t stream, const SidePool* pool) {
+cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int first_head, int part_tokens,
+                             cudaStream_t stream, const SidePool& pool) {
   if (a.dtype == ECHOKV_BF16) {
     if (a.head_dim == 128)
-      return launch_attn_side_t<__nv_bfloat16, 128>(a, side, n_ret_heads, part_tokens, stream, pool);
-    return launch_attn_side_t<__nv_bfloat16, 64>(a, side, n_ret_heads, part_tokens, stream, pool);
+      return launch_attn_side_t<__nv_bfloat16, 128>(a, side, first_head, part_tokens, stream, pool);
+    return launch_attn_side_t<__nv_bfloat16, 64>(a, side, first_head, part_tokens, stream, pool);
   }
-  if (a.head_dim == 128) return launch_attn_side_t<float, 128>(a, side, n_ret_heads, part_tokens, stream, pool);
-  return launch_attn_side_t<float, 64>(a, side, n_ret_heads, part_tokens, stream, pool);
+  if (a.head_dim == 128) return launch_attn_side_t<float, 128>(a, side, first_head, part_tokens, stream, pool);
+  return launch_attn_side_t<float, 64>(a, side, first_head, part_tokens, stream, pool);
 }
 
 }  // namespace echokv

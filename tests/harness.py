@@ -141,7 +141,7 @@ class Case:
                 assert query_heads is None
                 res[b] = O.decode_attention_windowed(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, kt, vt,
                                                      self.window[0], self.window[1], bk=bk, bv=bv,
-                                                     rope_theta=self.rope)
+                                                     rope_theta=self.rope, k_true=k_true)
             elif query_heads is None:
                 res[b] = O.decode_attention(qn[b], kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv,
                                             rope_theta=self.rope, k_true=k_true)
@@ -151,6 +151,22 @@ class Case:
                 for h, v in per.items():
                     res[(b, h)] = v
         return res
+
+    def recent_rows(self, layer, n_q):
+        """Full-width K and V rows of the last n_q + n_window - 1 tokens of every sequence, [B][n][D] on the
+        device (rows of positions before the sequence's start are zero): what the prefill-shaped call takes
+        when a window is set."""
+        w = self.w
+        n = n_q + self.window[1] - 1
+        outs = []
+        for kind in ("k", "v"):
+            rows = torch.zeros((w.batch, n, w.D), dtype=synth.torch_dtype(w))
+            for b in range(w.batch):
+                full = synth.layer_cache(w, layer, kind, b, width=w.D)[: self.lens[b]]
+                take = min(n, full.shape[0])
+                rows[b, n - take:] = full[full.shape[0] - take:]
+            outs.append(rows.to(self.ctx.device))
+        return outs
 
     def close(self):
         self.ctx.close()
