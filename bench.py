@@ -584,15 +584,23 @@ def run_prefill(args):
     st.rope = args.rope
     q = synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, 1, device=dev).to(torch.bfloat16)
     out = torch.empty(q.shape, dtype=torch.float32, device=dev)
+    recent = {}
+    if st.window:
+        # whole K / V rows of the chunk and the n_window - 1 tokens before it (what a caller has at hand while it
+        # prefills in chunks): the call reads every query's own window from them
+        n_rows = n_q + st.window[1] - 1
+        for kind in ("k", "v"):
+            recent[kind + "_recent"] = torch.stack([synth.layer_cache(w, 1, kind, b, width=w.D, device=dev)[-n_rows:]
+                                                    for b in range(w.batch)]).contiguous()
     for _ in range(max(3, args.warmup)):
-        ctx.prefill_attention(1, q, st.lens, out=out)
+        ctx.prefill_attention(1, q, st.lens, out=out, **recent)
     torch.cuda.synchronize()
     ctx.set_kernel_timing(True)
     ctx.read_kernel_timing_by_kind()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        ctx.prefill_attention(1, q, st.lens, out=out)
+        ctx.prefill_attention(1, q, st.lens, out=out, **recent)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / args.steps

@@ -83,15 +83,17 @@ typedef struct {
   int32_t device;            /* CUDA device ordinal                                        */
   int32_t n_retained_dims;   /* 0: m = n_retained_heads * head_dim.  Otherwise m itself, in flat dims: a
                                 multiple of 64 in [0, D] that need not end on a head boundary (the paper's
-                                m = 64 keeps half of head 0); n_retained_heads is then ignored.  A partly
-                                retained head is served by the absorbed mode only: echokv_create succeeds
-                                where that mode is available (EUNSUPPORTED otherwise) and
-                                echokv_decode_attention returns EUNSUPPORTED until echokv_enable_absorbed */
+                                m = 64 keeps half of head 0, its m = 384 three heads); n_retained_heads is then
+                                ignored.  Eq. 6 concatenates at the flat index m: of a head that m splits the
+                                dims below m are the stored ones and the rest are predicted.  The kernels that
+                                work on whole heads predict such a head whole, with `m mod head_dim` one-hot rows
+                                in front of the predictors that pass its stored dims through unchanged (exact);
+                                the extended predictors live in the workspace (echokv_query_sizes accounts for
+                                them) and echokv_set_weights builds them */
   int32_t save_k;            /* non-zero: the "save K" setting of Section 5.2 -- compressed layers keep their keys
                                 whole (K pools of width D, nothing of K is predicted, Wk may be NULL) and only the
-                                values are evicted and predicted.  Served by the absorbed mode only (as above);
-                                not combined with echokv_set_full_precision_window or echokv_compress_layer
-                                (EUNSUPPORTED) */
+                                values are evicted and predicted.  Decode calls are served by the absorbed mode
+                                only (EUNSUPPORTED until echokv_enable_absorbed) */
 } echokv_config;
 
 typedef struct {
@@ -160,7 +162,8 @@ int echokv_append_kv_chunk(echokv_ctx* ctx, int layer, const void* k_new, const 
  * dev_seq_begins[b] .. dev_seq_lens[b]-1 of each of the B sequences the call copies dims 0 .. m-1 of K and V
  * into the layer's own pools (Eq. 2) and, while a sink / window is set, dims m .. D-1 of the sink tokens and of
  * the last n_window tokens before dev_seq_lens[b] into the side buffers; afterwards echokv_decode_attention
- * serves the layer and the caller may release the full-width pools.  dev_seq_begins = NULL means 0; with a
+ * serves the layer and the caller may release the full-width pools.  With save_k the keys are copied whole and the
+ * side buffers receive values only.  dev_seq_begins = NULL means 0; with a
  * prefill done in chunks, call it once per chunk with the chunk's range.  The copies are bit-exact.
  * Bad slot / page -> device status EBADPAGE, bad length or begin -> EBADLENGTH; that sequence is skipped.
  * Errors: EINVAL, ENOTCOMPRESSED (anchor layers keep everything), ECAPACITY, ENOTABLE, ECUDA. */
@@ -188,21 +191,24 @@ int echokv_decode_attention(echokv_ctx* ctx, int layer, const void* q, float* ou
  * With many queries the cache is rebuilt once per call rather than once per query: the stored dims are gathered
  * and the dropped dims predicted (Eq. 3, on the tensor cores; K bias and rotary table applied if set) into
  * `scratch`, a caller-owned device buffer of echokv_prefill_scratch_bytes() bytes (16-byte aligned) that holds K~
- * and V~ as bf16 rows [B][max_pages_per_seq * page_tokens][D] each, and a causal attention kernel runs over those
- * rows.  Unlike the decode calls this one does round the predicted K and V to bf16 (as the paper's own
- * materialise-then-attend implementation does).  Works on anchor layers too (nothing is predicted there).
- * bf16, head_dim 128 and head-aligned m only; not with sink / window tokens: EUNSUPPORTED.  With save_k the keys
- * are gathered whole and only the values are predicted.
+ * and V~ as bf16 rows [B][max_pages_per_seq * page_tokens][D] each (plus one float per sequence, query and query
+ * head), and a causal attention kernel runs over those rows.  Unlike the decode calls this one does round the
+ * predicted K and V to bf16 (as the paper's own materialise-then-attend implementation does).  Works on anchor
+ * layers too (nothing is predicted there).  bf16, head_dim 128 only (EUNSUPPORTED otherwise); m may split a head.
+ * With save_k the keys are gathered whole and only the values are predicted.
+ * With sink / window tokens set (Section 4.1) every query is the decode step of the sequence cut off at its own
+ * position: it reads the first n_sink tokens and ITS OWN last n_window tokens at full precision and every other
+ * token as predicted.  The side buffers hold the window of the end of the sequence only, so the call then takes the
+ * recent tokens' rows from the caller: k_recent, v_recent are device pointers (16-byte aligned, EINVAL if NULL) to
+ * [B][n_q + n_window - 1][n_kv_heads][head_dim], the whole K and V rows of positions dev_seq_lens[b] - n_q -
+ * n_window + 1 .. dev_seq_lens[b] - 1 -- the chunk itself preceded by the n_window - 1 tokens before it; rows of
+ * positions below 0 are not read.  Without a window (and on anchor layers) both are ignored and may be NULL.
  * A sequence with fewer than n_q cached tokens, or an unusable slot / length: zeros and the device status.
  * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (batch, scratch too small), ENOWEIGHTS, ENOTABLE, ECUDA. */
-/* Which attention kernel the prefill-shaped call runs over the rebuilt rows: 0 = mma.sync kernel, 1 = tcgen05 kernel
- * (accumulators in tensor memory, one thread group doing every step in turn), 2 = warp-specialised tcgen05 kernel
- * (softmax, MMA and TMA warps; the default).  Meant for tests that check all of them against the oracle. */
-int echokv_prefill_path(const echokv_ctx* ctx);
-int echokv_set_prefill_path(echokv_ctx* ctx, int path);
 int echokv_prefill_scratch_bytes(const echokv_config* cfg, uint64_t* out);
 int echokv_prefill_attention(echokv_ctx* ctx, int layer, const void* q, float* out, int n_q,
                              const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                             const void* k_recent, const void* v_recent,
                              void* scratch, uint64_t scratch_bytes, void* stream);
 
 /* Attention over a layer that holds its full cache (anchor layers; the uncompressed
@@ -248,7 +254,8 @@ int echokv_set_decode_path(echokv_ctx* ctx, int path);
  *  - echokv_side_buffer_bytes: size of ONE side buffer: [max_batch][n_sink + n_window][D - m] elements
  *    of the storage dtype.  EUNSUPPORTED if n_sink + n_window > 4096.
  *  - echokv_set_full_precision_window: k_side / v_side are host arrays [n_layers] of device pointers
- *    (16-byte aligned, borrowed; entries of anchor layers are ignored and may be NULL).  From then on
+ *    (16-byte aligned, borrowed; entries of anchor layers are ignored and may be NULL; with save_k the keys
+ *    are whole in the pools already and k_side itself may be NULL).  From then on
  *    echokv_append_kv on a compressed layer also writes the new token's dims m .. D-1 to the side buffers
  *    (slot `position` while position < n_sink, and ring slot n_sink + position % n_window), and
  *    echokv_decode_attention attends the sink / window tokens from there.  Set it before the first
@@ -272,8 +279,7 @@ int echokv_set_full_precision_window(echokv_ctx* ctx, int n_sink, int n_window, 
  *  - echokv_set_rope: `table` is a device pointer of at least that size (16-byte aligned, borrowed until
  *    echokv_destroy or until rope is switched off); the call enqueues one kernel on `stream` that fills it
  *    (angles and sin / cos in fp64, rounded to fp32 once) and switches rotation on for later calls.
- *    theta = 0 with table = NULL switches it off.  Not available with n_retained_dims that split a head
- *    (EUNSUPPORTED).  In the absorbed mode a rotation that depends on the token cannot be folded into the
+ *    theta = 0 with table = NULL switches it off.  In the absorbed mode a rotation that depends on the token cannot be folded into the
  *    queries: with a table set that mode evaluates the K side explicitly (predicted keys on the tensor cores,
  *    rotated, scored) and keeps the absorbed form for the V side only -- about half the tensor work of the
  *    explicit mode.  Errors: EINVAL (theta < 1, misaligned), ECAPACITY, EUNSUPPORTED, ECUDA. */

@@ -57,11 +57,10 @@ EXPORTS = {
                                           C.c_void_p, C.c_int, C.c_void_p]),
     "echokv_full_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_int, C.c_void_p]),
-    "echokv_prefill_path": (C.c_int, [C.c_void_p]),
-    "echokv_set_prefill_path": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_prefill_scratch_bytes": (C.c_int, [C.POINTER(echokv_config), C.POINTER(C.c_uint64)]),
     "echokv_prefill_attention": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
-                                           C.c_void_p, C.c_int, C.c_void_p, C.c_uint64, C.c_void_p]),
+                                           C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
+                                           C.c_void_p]),
     "echokv_layer_step_host": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "echokv_get_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
@@ -232,22 +231,22 @@ class Context:
                "echokv_decode_attention")
         return out
 
-    def prefill_attention(self, layer: int, q, seq_lens, out=None, seq_slots=None, stream=None):
+    def prefill_attention(self, layer: int, q, seq_lens, out=None, seq_slots=None, stream=None, k_recent=None,
+                          v_recent=None):
         """q [B][n_q][H_q][d]: the last n_q cached tokens of every sequence as causal queries.  The scratch
-        for the rebuilt cache rows is allocated on first use and kept."""
+        for the rebuilt cache rows is allocated on first use and kept.  k_recent, v_recent [B][n_q + n_window - 1][D]:
+        whole K / V rows of the chunk and the n_window - 1 tokens before it (needed while a window is set)."""
         if getattr(self, "prefill_scratch", None) is None:
             n = C.c_uint64(0)
             _check(lib().echokv_prefill_scratch_bytes(C.byref(self.cfg), C.byref(n)), "echokv_prefill_scratch_bytes")
             self.prefill_scratch = self.torch.empty(n.value, dtype=self.torch.uint8, device=self.device)
         out = self._out(q) if out is None else out
         _check(lib().echokv_prefill_attention(self.handle, layer, _ptr(q), _ptr(out), q.shape[1], _ptr(seq_slots),
-                                              _ptr(seq_lens), q.shape[0], self.prefill_scratch.data_ptr(),
+                                              _ptr(seq_lens), q.shape[0], _ptr(k_recent), _ptr(v_recent),
+                                              self.prefill_scratch.data_ptr(),
                                               self.prefill_scratch.numel(), _stream_handle(stream)),
                "echokv_prefill_attention")
         return out
-
-    def set_prefill_path(self, path: int) -> None:
-        _check(lib().echokv_set_prefill_path(self.handle, path), "echokv_set_prefill_path")
 
     def full_attention(self, layer: int, q, seq_lens, out=None, seq_slots=None, stream=None):
         out = self._out(q) if out is None else out

@@ -131,7 +131,6 @@ struct echokv_ctx {
   AbsorbMaps amaps;
   bool stored_capable = false;   // shape served by the TMA + mma.sync stored-head kernel
   int stored_path = 0;           // 0 = CUDA-core kernel, 1 = TMA + mma.sync kernel
-  int prefill_path = 2;          // attention kernel of the prefill-shaped call: 0 = mma.sync, 1 = tcgen05, 2 = tcgen05 warp-specialised
   int64_t launches = 0;
   float scale = 0.f;
   std::vector<int32_t> pos_scratch;
@@ -573,14 +572,6 @@ int echokv_set_decode_mode(echokv_ctx* c, int mode) {
   return ECHOKV_OK;
 }
 
-int echokv_prefill_path(const echokv_ctx* c) { return c ? c->prefill_path : 0; }
-
-int echokv_set_prefill_path(echokv_ctx* c, int path) {
-  if (!c || path < 0 || path > 2) return ECHOKV_EINVAL;
-  c->prefill_path = path;
-  return ECHOKV_OK;
-}
-
 int echokv_stored_path(const echokv_ctx* c) { return c ? c->stored_path : 0; }
 
 int echokv_set_stored_path(echokv_ctx* c, int path) {
@@ -642,12 +633,15 @@ int echokv_prefill_scratch_bytes(const echokv_config* cfg, uint64_t* out) {
   const int rc = derive(cfg, &d);
   if (rc != ECHOKV_OK) return rc;
   if (cfg->dtype != ECHOKV_BF16 || cfg->head_dim != 128) return ECHOKV_EUNSUPPORTED;
-  *out = 2ull * (uint64_t)cfg->max_batch * (uint64_t)d.capacity * (uint64_t)d.D * 2ull;
+  // K~ rows, V~ rows, and one fp32 per (sequence, query, query head) for the sink / window combination
+  *out = 2ull * (uint64_t)cfg->max_batch * (uint64_t)d.capacity * (uint64_t)d.D * 2ull +
+         (uint64_t)cfg->max_batch * (uint64_t)d.capacity * (uint64_t)cfg->n_q_heads * 4ull;
   return ECHOKV_OK;
 }
 
 int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out, int n_q,
                              const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
+                             const void* k_recent, const void* v_recent,
                              void* scratch, uint64_t scratch_bytes, void* stream) {
   const int rc = check_call(c, layer, q, out, dev_seq_lens, B);
   if (rc != ECHOKV_OK) return rc;
@@ -655,11 +649,14 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
   const Layer& L = c->layers[layer];
   const bool compressed = !L.anchor && c->d.d_drop > 0;
   if (c->cfg.dtype != ECHOKV_BF16 || c->cfg.head_dim != 128) return ECHOKV_EUNSUPPORTED;
-  if (compressed && (!c->tc_capable || side_active(c, L))) return ECHOKV_EUNSUPPORTED;
+  if (compressed && !c->tc_capable) return ECHOKV_EUNSUPPORTED;
+  const bool windowed = compressed && side_active(c, L);
+  if (windowed && (!k_recent || !v_recent || !aligned16(k_recent) || !aligned16(v_recent))) return ECHOKV_EINVAL;
   const bool keys_whole = compressed && c->d.save_k;      // Section 5.2: nothing to predict on the K side
   if (n_q > c->d.capacity) return ECHOKV_ECAPACITY;
   const uint64_t rows_bytes = (uint64_t)B * c->d.capacity * c->d.D * 2ull;     // one of K~, V~
-  if (scratch_bytes < 2 * rows_bytes) return ECHOKV_ECAPACITY;
+  const uint64_t lse_bytes = (uint64_t)B * n_q * c->cfg.n_q_heads * 4ull;
+  if (scratch_bytes < 2 * rows_bytes + (windowed ? lse_bytes : 0)) return ECHOKV_ECAPACITY;
   if (compressed && (!L.Wv || (!L.Wk && !keys_whole))) return ECHOKV_ENOWEIGHTS;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   AttnArgs a = attn_args(c, q, dev_seq_slots, dev_seq_lens, B);
@@ -694,9 +691,25 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
       return ECHOKV_ECUDA;
     c->launches += keys_whole ? 1 : 2;
   }
-  if (launch_prefill_attn(a, k_rows, v_rows, c->d.capacity, c->d.D, n_q, out, s, c->prefill_path) != cudaSuccess)
+  if (!windowed) {
+    if (launch_prefill_attn(a, k_rows, v_rows, c->d.capacity, c->d.D, n_q, out, s) != cudaSuccess) return ECHOKV_ECUDA;
+    c->launches += 1;
+    return ECHOKV_OK;
+  }
+  // Section 4.1: every query's own sink and window at full precision.  The attention kernel covers what the query
+  // sees as predicted (the sink left out, nothing closer than n_window positions); the band kernel adds the rest.
+  float* lse = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + 2 * rows_bytes);
+  if (launch_prefill_attn(a, k_rows, v_rows, c->d.capacity, c->d.D, n_q, out, s, c->n_window, c->n_sink, lse) !=
+      cudaSuccess)
     return ECHOKV_ECUDA;
-  c->launches += 1;
+  PrefillBand band;
+  band.k_recent = k_recent; band.v_recent = v_recent;
+  band.k_pool = L.k_pool; band.v_pool = L.v_pool;
+  band.k_side = L.k_side; band.v_side = L.v_side;
+  band.D = c->d.D; band.mk = c->d.mk; band.m = c->d.m; band.d_drop = c->d.d_drop;
+  band.n_sink = c->n_sink; band.n_window = c->n_window;
+  if (launch_prefill_band(a, band, n_q, out, lse, s) != cudaSuccess) return ECHOKV_ECUDA;
+  c->launches += 2;
   return ECHOKV_OK;
 }
 

@@ -7,10 +7,12 @@
 //      (gather_rows_kernel; keys rotated to their positions if a rotary table is set),
 //   2. the dropped dims are predicted on the tensor cores and written beside them (Eq. 3; the
 //      row-storing mode of the CTA-pair kernel),
-//   3. a causal attention kernel evaluates Eq. 7 over those rows, online softmax in fp32.  Three versions,
-//      selectable for tests: prefill_attn_ws_kernel (tcgen05, warp-specialised; the default),
-//      prefill_attn_tc_kernel (tcgen05, one thread group doing every step in turn) and prefill_attn_kernel
-//      (mma.sync m16n8k16, 64 query rows per CTA, 64-token tiles).
+//   3. a causal attention kernel (prefill_attn_ws_kernel: tcgen05, warp-specialised) evaluates Eq. 7 over those
+//      rows, online softmax in fp32,
+//   4. with sink / recent-window tokens at full precision (Section 4.1) every query is the decode step of the
+//      sequence cut off at its own position: step 3 then covers the tokens the query sees as predicted (those more
+//      than n_window - 1 positions before it, the sink left out), and prefill_band_kernel adds the query's own sink
+//      and window tokens from their stored values and combines the two by log-sum-exp.
 // The rebuilt rows are bf16 in a caller-owned scratch, as in the paper's own materialise-then-attend
 // design; the decode path never writes them.
 #include "prefill.h"
@@ -111,227 +113,18 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
 }
 
 // ---------------------------------------------------------------------------------------------
-// 3. causal attention of n_q query rows over contiguous bf16 rows
+// 3. causal attention of n_q query rows over contiguous bf16 rows, on the 5th-generation tensor cores
+//    (tcgen05, accumulators in tensor memory), the steps given to different warps so that they overlap
 // ---------------------------------------------------------------------------------------------
-constexpr int kPfRows = 64;      // query rows per CTA: 4 warps x 16
-constexpr int kPfKeys = 64;      // keys per tile
-constexpr int kPfRowBytes = 256; // 128 bf16
-
-// 16-byte asynchronous copy global -> shared; n_bytes = 0 writes zeros without reading
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t n_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+constexpr int kTcTile = 128;                     // query rows per tile, keys per tile
+constexpr int kTcChunkBytes = kTcTile * 128;     // [128 rows x 64 dims] bf16, 128-byte swizzle
+constexpr int kTcTileBytes = 2 * kTcChunkBytes;  // 128 dims
+constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
 }
-
-__global__ void __launch_bounds__(128) prefill_attn_kernel(const __nv_bfloat16* __restrict__ q,
-                                                           const __nv_bfloat16* __restrict__ ks,
-                                                           const __nv_bfloat16* __restrict__ vs,
-                                                           float* __restrict__ out, int n_q, int n_q_heads,
-                                                           int n_kv_heads, int kv_tokens, int kv_width,
-                                                           const int32_t* __restrict__ slots,
-                                                           const int32_t* __restrict__ lens, int max_batch,
-                                                           int capacity, float scale_log2e, int32_t* status) {
-  // two buffers of a key tile and a value tile each: the next tile is copied while this one is multiplied
-  extern __shared__ __align__(128) unsigned char pf_smem[];
-  constexpr int kTileBytes = kPfKeys * kPfRowBytes;
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qd = (lane & 3) * 2;
-  const int kvh = h / (n_q_heads / n_kv_heads);
-  const int slot = slots ? slots[b] : b;
-  const int len = lens[b];
-  const int i0 = qt * kPfRows + warp * 16 + (lane >> 2), i1 = i0 + 8;      // this thread's two query rows
-  float* out0 = out + (((size_t)b * n_q + i0) * n_q_heads + h) * 128;
-  float* out1 = out + (((size_t)b * n_q + i1) * n_q_heads + h) * 128;
-  if (slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
-    // unusable sequence (or fewer cached tokens than queries): zeros and a status
-    if (tid == 0 && qt == 0 && h == 0) report(status, slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
-    for (int nt = 0; nt < 16; ++nt) {
-      if (i0 < n_q) *reinterpret_cast<float2*>(out0 + nt * 8 + qd) = make_float2(0.f, 0.f);
-      if (i1 < n_q) *reinterpret_cast<float2*>(out1 + nt * 8 + qd) = make_float2(0.f, 0.f);
-    }
-    return;
-  }
-  const int pos0 = len - n_q + i0, pos1 = len - n_q + i1;               // the rows' own positions
-  // A fragments of Q (rows past n_q are zero)
-  uint32_t qa[8][4];
-  {
-    const __nv_bfloat16* q0 = q + (((size_t)b * n_q + i0) * n_q_heads + h) * 128 + qd;
-    const __nv_bfloat16* q1 = q + (((size_t)b * n_q + i1) * n_q_heads + h) * 128 + qd;
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      qa[kk][0] = i0 < n_q ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16) : 0u;
-      qa[kk][1] = i1 < n_q ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16) : 0u;
-      qa[kk][2] = i0 < n_q ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16 + 8) : 0u;
-      qa[kk][3] = i1 < n_q ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16 + 8) : 0u;
-    }
-  }
-  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-  float o[16][4];
-#pragma unroll
-  for (int nt = 0; nt < 16; ++nt)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
-
-  // keys this CTA's rows may see: up to the position of its last row
-  const int last_row = min(n_q, (qt + 1) * kPfRows) - 1;
-  const int kv_end = len - n_q + last_row + 1;
-  const uint32_t smem_base = smem_u32(pf_smem);
-  const __nv_bfloat16* k_seq = ks + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
-  const __nv_bfloat16* v_seq = vs + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
-  // stage 64 key rows and 64 value rows into buffer `buf` (16-byte pieces swizzled by row so that ldmatrix is
-  // conflict-free; rows past the last key the CTA may see are zero-filled)
-  auto stage = [&](int kv0, int buf) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int idx = tid + 128 * i, r = idx >> 4, c = idx & 15;
-      const bool in = kv0 + r < kv_end;
-      const size_t src = (size_t)(in ? kv0 + r : 0) * kv_width + c * 8;
-      const uint32_t off = smem_base + buf * 2 * kTileBytes + r * kPfRowBytes + ((c ^ (r & 7)) << 4);
-      cp_async16(off, k_seq + src, in ? 16u : 0u);
-      cp_async16(off + kTileBytes, v_seq + src, in ? 16u : 0u);
-    }
-    cp_async_commit();
-  };
-  stage(0, 0);
-
-  for (int kv0 = 0, tile = 0; kv0 < kv_end; kv0 += kPfKeys, ++tile) {
-    if (kv0 + kPfKeys < kv_end) {
-      stage(kv0 + kPfKeys, (tile + 1) & 1);
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
-    __syncthreads();
-    const uint32_t k_base = smem_base + (tile & 1) * 2 * kTileBytes, v_base = k_base + kTileBytes;
-
-    // ---- S = Q K^T for this warp's 16 rows x 64 keys
-    float sc[8][4];
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) sc[nt][e] = 0.f;
-#pragma unroll
-    for (int np = 0; np < 4; ++np) {
-      const int tok = np * 16 + (lane >> 4) * 8 + (lane & 7);
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        const int c = 2 * kk + ((lane >> 3) & 1);
-        uint32_t r0, r1, r2, r3;
-        ldsm_x4(k_base + tok * kPfRowBytes + ((c ^ (tok & 7)) << 4), r0, r1, r2, r3);
-        mma_m16n8k16_bf16(sc[2 * np], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], r0, r1);
-        mma_m16n8k16_bf16(sc[2 * np + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], r2, r3);
-      }
-    }
-
-    // ---- causal mask, online softmax (rows i0: elements 0, 1; rows i1: elements 2, 3)
-    float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = kv0 + nt * 8 + qd + (e & 1);
-        const int row_pos = e < 2 ? pos0 : pos1;
-        const bool row_ok = e < 2 ? i0 < n_q : i1 < n_q;
-        const float v = (row_ok && key <= row_pos) ? sc[nt][e] * scale_log2e : -INFINITY;
-        sc[nt][e] = v;
-        mx[e >> 1] = fmaxf(mx[e >> 1], v);
-      }
-    float alpha[2];
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-      const float m_new = fmaxf(m_run[r], mx[r]);
-      // (a row that has seen no key yet keeps m = -inf: its probabilities are all 0 and alpha is irrelevant)
-      alpha[r] = m_new == -INFINITY ? 1.f : exp2f(m_run[r] - m_new);
-      m_run[r] = m_new;
-    }
-    uint32_t pa[4][4];
-    float psum[2] = {0.f, 0.f};
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      float pv[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        pv[e] = m_run[e >> 1] == -INFINITY ? 0.f : exp2f(sc[nt][e] - m_run[e >> 1]);
-        psum[e >> 1] += pv[e];
-      }
-      // C fragments of key tiles 2j, 2j + 1 are the A fragment of key step j
-      pa[nt >> 1][(nt & 1) * 2 + 0] = pack2(pv[0], pv[1]);
-      pa[nt >> 1][(nt & 1) * 2 + 1] = pack2(pv[2], pv[3]);
-    }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) l_run[r] = l_run[r] * alpha[r] + psum[r];
-#pragma unroll
-    for (int nt = 0; nt < 16; ++nt) {
-      o[nt][0] *= alpha[0]; o[nt][1] *= alpha[0];
-      o[nt][2] *= alpha[1]; o[nt][3] *= alpha[1];
-    }
-
-    // ---- O += P V
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int tok = j * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
-#pragma unroll
-      for (int dp = 0; dp < 8; ++dp) {
-        const int c = 2 * dp + (lane >> 4);
-        uint32_t r0, r1, r2, r3;
-        ldsm_x4_trans(v_base + tok * kPfRowBytes + ((c ^ (tok & 7)) << 4), r0, r1, r2, r3);
-        mma_m16n8k16_bf16(o[2 * dp], pa[j][0], pa[j][1], pa[j][2], pa[j][3], r0, r1);
-        mma_m16n8k16_bf16(o[2 * dp + 1], pa[j][0], pa[j][1], pa[j][2], pa[j][3], r2, r3);
-      }
-    }
-    __syncthreads();       // the tiles are free for the next load
-  }
-
-  // ---- normalise and write
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-  }
-  const float inv0 = l_run[0] > 0.f ? 1.f / l_run[0] : 0.f, inv1 = l_run[1] > 0.f ? 1.f / l_run[1] : 0.f;
-#pragma unroll
-  for (int nt = 0; nt < 16; ++nt) {
-    if (i0 < n_q) *reinterpret_cast<float2*>(out0 + nt * 8 + qd) = make_float2(o[nt][0] * inv0, o[nt][1] * inv0);
-    if (i1 < n_q) *reinterpret_cast<float2*>(out1 + nt * 8 + qd) = make_float2(o[nt][2] * inv1, o[nt][3] * inv1);
-  }
-}
-
-
-// ---------------------------------------------------------------------------------------------
-// 3b. the same on the 5th-generation tensor cores (tcgen05, accumulators in tensor memory)
-// ---------------------------------------------------------------------------------------------
-// One CTA of 256 threads per (128 query rows, query head, sequence); keys in tiles of 128.
-//   S   [128 rows x 128 keys]  = Q K^T        A = Q tile, B = key tile, both K-major       -> TMEM columns 0..127
-//   O^T [128 dims x 128 rows]  = V^T P^T      A = value tile used M-major (it is stored [key][dim]), B = P K-major
-//                                              -> TMEM columns 128..255, fresh for every key tile
-// Two threads share S row r (query row r), 64 keys each: mask, running max / sum, probabilities as bf16 into a
-// shared-memory tile in the MMA's swizzled layout.  The same two share O^T row d (output dim d), 64 query rows each:
-// o[row] = o[row] * alpha[row] + O^T tile, in registers, so nothing is rescaled in tensor memory.  Key / value tiles are double-buffered with cp.async; the
-// waits on the two MMA-completion barriers are bounded.
-constexpr int kTcTile = 128;                     // query rows per CTA, keys per tile
-constexpr int kTcChunkBytes = kTcTile * 128;     // [128 rows x 64 dims] bf16, 128-byte swizzle
-constexpr int kTcTileBytes = 2 * kTcChunkBytes;  // 128 dims
-constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescO = kIdescS | (1u << 15);                  // A operand M-major
-
-struct PfTcTail {
-  float alpha[kTcTile];
-  float mx[2][kTcTile];          // partial row maxima of the two column halves
-  float l[2][kTcTile];
-  unsigned long long bar_s, bar_o;
-  uint32_t tmem_base;
-  int abort_flag;
-};
 
 __device__ __forceinline__ uint64_t pf_desc_kmajor(uint32_t smem_addr) {
   uint64_t d = 0;
@@ -353,217 +146,7 @@ __device__ __forceinline__ uint64_t pf_desc_mmajor(uint32_t smem_addr, uint32_t 
   d |= static_cast<uint64_t>(2) << 61;
   return d;
 }
-// byte offset of 16-byte piece `piece` (0..15) of row `row` inside a [128 rows x 128 dims] swizzled tile
-__device__ __forceinline__ uint32_t pf_sw(int row, int piece) {
-  return (uint32_t)((piece >> 3) * kTcChunkBytes + row * 128 + (((piece & 7) ^ (row & 7)) << 4));
-}
 
-// 256 threads: thread (lane row r = tid % 128, half = tid / 128) owns columns [64 half, 64 half + 64) of TMEM lane r
-// in both accumulators: half of S row r (keys) and half of O^T row r (query rows of output dim r).  Two warps per
-// scheduler instead of one hide the tensor-memory and special-function latencies of the epilogue.
-__global__ void __launch_bounds__(256, 1)
-prefill_attn_tc_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ ks,
-                       const __nv_bfloat16* __restrict__ vs, float* __restrict__ out, int n_q, int n_q_heads,
-                       int n_kv_heads, int kv_tokens, int kv_width, const int32_t* __restrict__ slots,
-                       const int32_t* __restrict__ lens, int max_batch, int capacity, float scale_log2e,
-                       int32_t* status) {
-  extern __shared__ unsigned char pf_tc_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_tc_raw) + 1023) &
-                                                         ~static_cast<uintptr_t>(1023));
-  // Q | K buffer 0, 1 | V buffer 0, 1 | P
-  const uint32_t q_addr = smem_u32(smem), k_addr = q_addr + kTcTileBytes, v_addr = k_addr + 2 * kTcTileBytes,
-                 p_addr = v_addr + 2 * kTcTileBytes;
-  unsigned char* p_tile = smem + 5 * kTcTileBytes;
-  PfTcTail& t = *reinterpret_cast<PfTcTail*>(smem + 6 * kTcTileBytes);
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int r = tid & 127, half = tid >> 7;                 // TMEM lane / row, and which 64 columns
-  const int kvh = h / (n_q_heads / n_kv_heads);
-  const int slot = slots ? slots[b] : b;
-  const int len = lens[b];
-  const int i_row = qt * kTcTile + r;                       // the query row of S row r
-  if (slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
-    if (tid == 0 && qt == 0 && h == 0) report(status, slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
-    for (int c = half * 64; c < half * 64 + 64; ++c) {
-      const int i = qt * kTcTile + c;
-      if (i < n_q) out[(((size_t)b * n_q + i) * n_q_heads + h) * 128 + r] = 0.f;
-    }
-    return;
-  }
-  volatile int* abort_flag = &t.abort_flag;
-  if (tid == 0) {
-    t.abort_flag = 0;
-    mbar_init(smem_u32(&t.bar_s), 1);
-    mbar_init(smem_u32(&t.bar_o), 1);
-    mbar_fence_init();
-  }
-  __syncthreads();
-  if (warp == 0) {
-    tmem_alloc(smem_u32(&t.tmem_base), 256);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = t.tmem_base;
-  const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + half * 64;
-
-  const int last_row = min(n_q, (qt + 1) * kTcTile) - 1;
-  const int kv_end = len - n_q + last_row + 1;              // keys this CTA's rows may see
-  const int n_tiles = (kv_end + kTcTile - 1) / kTcTile;
-  const __nv_bfloat16* k_seq = ks + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
-  const __nv_bfloat16* v_seq = vs + (size_t)b * kv_tokens * kv_width + (size_t)kvh * 128;
-  auto stage = [&](int tile, int buf) {          // 128 key rows and 128 value rows, zero-filled past kv_end
-    const int kv0 = tile * kTcTile;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int idx = tid + 256 * i, row = idx >> 4, piece = idx & 15;
-      const bool in = kv0 + row < kv_end;
-      const size_t src = (size_t)(in ? kv0 + row : 0) * kv_width + piece * 8;
-      const uint32_t off = buf * kTcTileBytes + pf_sw(row, piece);
-      cp_async16(k_addr + off, k_seq + src, in ? 16u : 0u);
-      cp_async16(v_addr + off, v_seq + src, in ? 16u : 0u);
-    }
-  };
-  // the query rows (rows past n_q are zero), with the first key / value tile
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int idx = tid + 256 * i, row = idx >> 4, piece = idx & 15;
-    const int iq = qt * kTcTile + row;
-    const bool in = iq < n_q;
-    cp_async16(q_addr + pf_sw(row, piece), q + (((size_t)b * n_q + (in ? iq : 0)) * n_q_heads + h) * 128 + piece * 8,
-               in ? 16u : 0u);
-  }
-  stage(0, 0);
-  cp_async_commit();
-
-  const int pos = len - n_q + i_row;                        // position of query row r
-  const bool row_ok = i_row < n_q;
-  float m_run = -INFINITY, l_run = 0.f;                     // (m_run is the same in both halves; l_run is this half's)
-  float o[64];                                              // output dim r, query rows 64 half .. 64 half + 63
-#pragma unroll
-  for (int c = 0; c < 64; ++c) o[c] = 0.f;
-  bool alive = true;
-
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    const int buf = tile & 1;
-    if (tile + 1 < n_tiles) {
-      stage(tile + 1, buf ^ 1);
-      cp_async_commit();
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
-    fence_proxy_async_smem();        // the copied tiles, before the tensor cores read them
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        const uint64_t a = pf_desc_kmajor(q_addr + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
-        const uint64_t bd = pf_desc_kmajor(k_addr + buf * kTcTileBytes + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
-        tc_mma_bf16(tmem, a, bd, kIdescS, kk > 0 ? 1u : 0u);
-      }
-      tc_commit(smem_u32(&t.bar_s));
-    }
-    if (!__syncthreads_and(mbar_wait(smem_u32(&t.bar_s), tile & 1, abort_flag, status) ? 1 : 0)) { alive = false; break; }
-    tc_fence_after();
-
-    // ---- this thread's 64 keys of S row r: partial maximum, exchanged with the other half
-    const int key0 = tile * kTcTile + half * 64;
-    float mx = -INFINITY;
-#pragma unroll
-    for (int c2 = 0; c2 < 2; ++c2) {
-      float v[32];
-      tmem_ld32(lane_addr + c2 * 32, v);
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (row_ok && key0 + c2 * 32 + j <= pos) mx = fmaxf(mx, v[j]);
-    }
-    t.mx[half][r] = mx * scale_log2e;       // (scale > 0: the maximum commutes with it; -inf stays -inf)
-    __syncthreads();
-    const float m_new = fmaxf(m_run, fmaxf(t.mx[0][r], t.mx[1][r]));
-    const float alpha = m_new == -INFINITY ? 1.f : exp2f(m_run - m_new);
-    m_run = m_new;
-    float psum = 0.f;
-#pragma unroll
-    for (int c2 = 0; c2 < 2; ++c2) {
-      float v[32];
-      tmem_ld32(lane_addr + c2 * 32, v);
-      uint32_t packed[16];
-#pragma unroll
-      for (int j = 0; j < 32; j += 2) {
-        const float p0 = (row_ok && key0 + c2 * 32 + j <= pos) ? exp2f(v[j] * scale_log2e - m_new) : 0.f;
-        const float p1 = (row_ok && key0 + c2 * 32 + j + 1 <= pos) ? exp2f(v[j + 1] * scale_log2e - m_new) : 0.f;
-        psum += p0 + p1;
-        packed[j >> 1] = pack2(p0, p1);
-      }
-#pragma unroll
-      for (int pc = 0; pc < 4; ++pc)    // four 16-byte pieces of 8 keys
-        *reinterpret_cast<uint4*>(p_tile + pf_sw(r, half * 8 + c2 * 4 + pc)) =
-            make_uint4(packed[4 * pc], packed[4 * pc + 1], packed[4 * pc + 2], packed[4 * pc + 3]);
-    }
-    l_run = l_run * alpha + psum;
-    if (half == 0) t.alpha[r] = alpha;
-    tc_fence_before();
-    fence_proxy_async_smem();        // the probabilities, before the tensor cores read them
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-      const uint64_t a0 = pf_desc_mmajor(v_addr + buf * kTcTileBytes, kTcChunkBytes);
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {   // 16 keys per MMA: 2048 bytes of value rows, 32 bytes along P's keys
-        const uint64_t bd = pf_desc_kmajor(p_addr + (kk >> 2) * kTcChunkBytes) + 2 * (kk & 3);
-        tc_mma_bf16(tmem + 128, a0 + 128 * kk, bd, kIdescO, kk > 0 ? 1u : 0u);
-      }
-      tc_commit(smem_u32(&t.bar_o));
-    }
-    if (!__syncthreads_and(mbar_wait(smem_u32(&t.bar_o), tile & 1, abort_flag, status) ? 1 : 0)) { alive = false; break; }
-    tc_fence_after();
-
-    // ---- O^T row r (output dim r), this thread's 64 query rows: fold this tile in
-#pragma unroll
-    for (int c2 = 0; c2 < 2; ++c2) {
-      float v[32];
-      tmem_ld32(lane_addr + 128 + c2 * 32, v);
-      const float4* al = reinterpret_cast<const float4*>(&t.alpha[half * 64 + c2 * 32]);
-#pragma unroll
-      for (int j4 = 0; j4 < 8; ++j4) {
-        const float4 a4 = al[j4];
-        o[c2 * 32 + 4 * j4 + 0] = fmaf(o[c2 * 32 + 4 * j4 + 0], a4.x, v[4 * j4 + 0]);
-        o[c2 * 32 + 4 * j4 + 1] = fmaf(o[c2 * 32 + 4 * j4 + 1], a4.y, v[4 * j4 + 1]);
-        o[c2 * 32 + 4 * j4 + 2] = fmaf(o[c2 * 32 + 4 * j4 + 2], a4.z, v[4 * j4 + 2]);
-        o[c2 * 32 + 4 * j4 + 3] = fmaf(o[c2 * 32 + 4 * j4 + 3], a4.w, v[4 * j4 + 3]);
-      }
-    }
-    tc_fence_before();
-    __syncthreads();                 // S, P and alpha are free for the next tile
-  }
-
-  if (alive) {
-    t.l[half][r] = l_run;
-    __syncthreads();
-#pragma unroll
-    for (int c = 0; c < 64; ++c) {
-      const int row = half * 64 + c, i = qt * kTcTile + row;
-      const float l = t.l[0][row] + t.l[1][row];
-      if (i < n_q) out[(((size_t)b * n_q + i) * n_q_heads + h) * 128 + r] = l > 0.f ? o[c] / l : 0.f;
-    }
-  } else {
-    cp_async_wait<0>();
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0) {
-    tc_fence_after();
-    tmem_dealloc(tmem, 256);
-  }
-}
-
-
-// ---------------------------------------------------------------------------------------------
-// 3c. tcgen05 again, with the steps given to different warps so that they overlap
-// ---------------------------------------------------------------------------------------------
 // One CTA per (256 query rows, query head, sequence): two query tiles x = 0, 1 of 128 rows share every key / value tile,
 // and while the tensor cores work for one of them the other one's softmax runs.  (With few queries per sequence the
 // 256 rows are all the rows of 2, 4 or 8 query heads of one KV head instead.)
@@ -628,7 +211,11 @@ __global__ void __launch_bounds__(kWsThreads, 1)
 prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, float* __restrict__ out, int n_q, int n_q_heads,
                        int n_kv_heads, const int32_t* __restrict__ slots, const int32_t* __restrict__ lens,
-                       int max_batch, int capacity, float scale_log2e, int rows_per_head, int32_t* status) {
+                       int max_batch, int capacity, float scale_log2e, int rows_per_head, int32_t* status,
+                       int shift, int n_skip, float* __restrict__ lse_out) {
+  // shift, n_skip: query row at position pos attends keys n_skip <= t <= pos - shift (plain causal attention: 0, 0);
+  // lse_out (may be null): [B][n_q][H_q] log2 of the row's softmax denominator in the kernel's base-2 units
+  // (-inf for a row that attends nothing; its output row is zero)
   // tail | Q tile 0, 1 | K stages | V stages; the tiles need 1024-byte alignment, and with all of the shared memory in
   // use there is no room to round the start up
   extern __shared__ __align__(1024) unsigned char pf_ws_raw[];
@@ -650,14 +237,19 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
   const bool misaligned = (q_addr & 1023u) != 0;
-  if (misaligned || slot < 0 || slot >= max_batch || len < n_q || len > capacity) {
-    if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0)
+  const bool unusable = misaligned || slot < 0 || slot >= max_batch || len < n_q || len > capacity;
+  const int last_row = rows_per_head ? n_q - 1 : min(n_q, row_base + n_act * kTcTile) - 1;
+  const int kv_end = len - n_q + last_row + 1 - shift;      // keys this CTA's rows may see
+  if (unusable || kv_end <= n_skip) {                       // (the latter: none of the rows attends anything here)
+    if (unusable && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0)
       report(status, misaligned ? ECHOKV_ECUDA : slot < 0 || slot >= max_batch ? ECHOKV_EBADPAGE : ECHOKV_EBADLENGTH);
     if (tid < 256) {
       const int x = tid >> 7, i = query_of(x, tid & 127);
-      if (i < n_q) {
-        float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + i) * n_q_heads + head_of(x, tid & 127)) * 128);
+      if (i < n_q && x < n_act) {
+        const size_t row = ((size_t)b * n_q + i) * n_q_heads + head_of(x, tid & 127);
+        float4* dst = reinterpret_cast<float4*>(out + row * 128);
         for (int c = 0; c < 32; ++c) dst[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (lse_out != nullptr) lse_out[row] = -INFINITY;
       }
     }
     return;
@@ -692,8 +284,6 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_after();
   const uint32_t tmem = t.tmem_base;
 
-  const int last_row = rows_per_head ? n_q - 1 : min(n_q, row_base + n_act * kTcTile) - 1;
-  const int kv_end = len - n_q + last_row + 1;              // keys this CTA's rows may see
   const int n_tiles = (kv_end + kTcTile - 1) / kTcTile;
 
   if (warp == kWsSoftmaxWarps + 1) {
@@ -798,7 +388,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int h = head_of(x, row);
     const int i_row = query_of(x, row);
     const bool row_ok = i_row < n_q;
-    const int pos = len - n_q + i_row;                      // position of this query row
+    const int pos = len - n_q + i_row - shift;              // last key this query row attends here
     const uint32_t lane_base = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const uint32_t s_addr = lane_base + x * 128 + hf * 64, o_addr = lane_base + 256 + x * 128 + hf * 64;
     float m_ref = -INFINITY, l_run = 0.f;                   // m_ref is the same in both threads of a row
@@ -807,6 +397,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&t.s_full[x]), tile & 1, abort_flag, status) ? 1 : 0) != 0;
       // keys of this thread's half the row sees: the first n_vis
       const int n_vis = row_ok ? max(0, min(64, pos - (tile * kTcTile + hf * 64) + 1)) : 0;
+      const int n_lo = max(0, min(64, n_skip - (tile * kTcTile + hf * 64)));    // ... but not the first n_lo
       uint32_t sr[2][32];
       float mx = -INFINITY, psum = 0.f;
       if (ok) {
@@ -837,7 +428,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         unpack_f2(sum2[1], b0, b1);
         psum = (a0 + a1) + (b0 + b1);
       }
-      const bool careful = !ok || tile == 0 || n_vis != 64 || !(psum < kWsSumLimit);
+      const bool careful = !ok || tile == 0 || n_vis != 64 || n_lo != 0 || !(psum < kWsSumLimit);
       if (pair_any(pair_id, careful)) {
         if (pair_any(pair_id, !ok)) { alive = false; break; }     // both warps of the row leave together
         // ---- the careful way: masks, the row maximum over both halves, O rescaled if the reference moves
@@ -849,7 +440,7 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int c = 0; c < 2; ++c)
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (32 * c + j < n_vis) mx = fmaxf(mx, __uint_as_float(sr[c][j]));
+            if (32 * c + j < n_vis && 32 * c + j >= n_lo) mx = fmaxf(mx, __uint_as_float(sr[c][j]));
         mx *= scale_log2e;
         t.ex[x][hf][row] = mx;
         pair_sync(pair_id);
@@ -882,8 +473,9 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int c = 0; c < 2; ++c)
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
-            const float p0 = 32 * c + j < n_vis ? ex2_approx(fmaf(__uint_as_float(sr[c][j]), scale_log2e, -m_ref)) : 0.f;
-            const float p1 = 32 * c + j + 1 < n_vis ? ex2_approx(fmaf(__uint_as_float(sr[c][j + 1]), scale_log2e, -m_ref)) : 0.f;
+            const bool v0 = 32 * c + j < n_vis && 32 * c + j >= n_lo, v1 = 32 * c + j + 1 < n_vis && 32 * c + j + 1 >= n_lo;
+            const float p0 = v0 ? ex2_approx(fmaf(__uint_as_float(sr[c][j]), scale_log2e, -m_ref)) : 0.f;
+            const float p1 = v1 ? ex2_approx(fmaf(__uint_as_float(sr[c][j + 1]), scale_log2e, -m_ref)) : 0.f;
             psum += p0 + p1;
             sr[c][j >> 1] = pack2(p0, p1);
           }
@@ -903,6 +495,8 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (mbar_wait(smem_u32(&t.o_done[x]), 0, abort_flag, status)) {
         tc_fence_after();
         const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        if (lse_out != nullptr && row_ok && hf == 0)
+          lse_out[((size_t)b * n_q + i_row) * n_q_heads + h] = l_run > 0.f ? m_ref + log2f(l_run) : -INFINITY;
         float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * n_q + (row_ok ? i_row : 0)) * n_q_heads + h) * 128 + hf * 64);
 #pragma unroll 1
         for (int c = 0; c < 2; ++c) {
@@ -925,6 +519,161 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// 4. the sink and window tokens of every query, at full precision (Section 4.1), combined with step 3
+// ---------------------------------------------------------------------------------------------
+// One block per (query i, KV head, sequence).  The query at position p reads as stored: the sink tokens
+// t < min(n_sink, p + 1) -- their retained dims from the layer's pools, the rest from the side buffers -- and the
+// window tokens max(n_sink, p - n_window + 1) .. p, whole rows of k_recent / v_recent.  Scores (keys rotated to
+// their positions if a table is set), softmax over these tokens, weighted values; then the log-sum-exp combination
+// with what step 3 left in out / lse for the tokens the query sees as predicted.  Thread per token for the scores,
+// thread per output dim for the values.
+__global__ void __launch_bounds__(128) prefill_band_kernel(AttnArgs a, PrefillBand w, int n_q, float* __restrict__ out,
+                                                           const float* __restrict__ lse) {
+  extern __shared__ float band_smem[];
+  constexpr int DH = 128;
+  using T = __nv_bfloat16;
+  const int i = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = a.n_q_heads / a.n_kv_heads;
+  const int n_list = w.n_sink + w.n_window;
+  float* qs = band_smem;                       // [g][DH], scaled
+  float* sc = qs + kMaxGroup * DH;             // [g][n_list]
+  __shared__ float red[4][kMaxGroup];
+  __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
+  const int slot = a.slots ? a.slots[b] : b;
+  const int len = a.lens[b];
+  if (slot < 0 || slot >= a.geom.max_batch || len < n_q || len > a.geom.max_pages_per_seq * a.geom.page_tokens)
+    return;                                    // (reported, and zeros written, by step 3)
+  const int p = len - n_q + i;                 // this query's position
+  const int n_sink_tok = min(w.n_sink, p + 1);
+  const int win_lo = max(w.n_sink, p - w.n_window + 1);
+  const int n_tok = n_sink_tok + max(0, p - win_lo + 1);
+  const int n_stored_k = min(max(w.mk - kvh * DH, 0), DH), n_stored_v = min(max(w.m - kvh * DH, 0), DH);
+  const int n_rows = n_q + w.n_window - 1;     // rows of k_recent / v_recent per sequence; row 0 is position t_base
+  const int t_base = len - n_rows;
+  const T* q = reinterpret_cast<const T*>(a.q) + (((size_t)b * n_q + i) * a.n_q_heads + (size_t)kvh * g) * DH;
+  for (int idx = tid; idx < g * DH; idx += 128) qs[idx] = __bfloat162float(q[idx]) * a.scale_log2e;
+  __syncthreads();
+  const T* k_pool = reinterpret_cast<const T*>(w.k_pool);
+  const T* v_pool = reinterpret_cast<const T*>(w.v_pool);
+  const T* k_side = reinterpret_cast<const T*>(w.k_side);
+  const T* v_side = reinterpret_cast<const T*>(w.v_side);
+  const T* k_recent = reinterpret_cast<const T*>(w.k_recent);
+  const T* v_recent = reinterpret_cast<const T*>(w.v_recent);
+  const int32_t* table = a.geom.table + (size_t)slot * a.geom.max_pages_per_seq;
+  // pool row (in token rows) of sink token t
+  auto pool_row = [&](int t) -> size_t {
+    int page = table[t / a.geom.page_tokens];
+    if (page < 0 || page >= a.geom.n_pages) {
+      report(a.status, ECHOKV_EBADPAGE);
+      page = 0;
+    }
+    return (size_t)page * a.geom.page_tokens + t % a.geom.page_tokens;
+  };
+  const size_t side_base = (size_t)slot * n_list;
+  // scores: one token per thread
+  for (int idx = tid; idx < n_tok; idx += 128) {
+    const bool sink = idx < n_sink_tok;
+    const int t = sink ? idx : win_lo + (idx - n_sink_tok);
+    const T* a_ptr;      // dims [0, n_a) of the head
+    const T* b_ptr;      // the rest
+    int n_a;
+    if (sink) {
+      const size_t r = n_stored_k > 0 ? pool_row(t) : 0;
+      a_ptr = k_pool + r * (size_t)w.mk + (size_t)kvh * DH;
+      n_a = n_stored_k;
+      b_ptr = k_side + (side_base + t) * (size_t)w.d_drop + (kvh * DH + n_stored_k - w.mk);
+    } else {
+      a_ptr = k_recent + ((size_t)b * n_rows + (t - t_base)) * (size_t)w.D + (size_t)kvh * DH;
+      n_a = DH;
+      b_ptr = a_ptr;
+    }
+    auto k_at = [&](int j) -> const T* { return j < n_a ? a_ptr + j : b_ptr + (j - n_a); };
+    float acc[kMaxGroup];
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
+    if (a.rope.cs != nullptr) {
+      const float2* cs = a.rope.cs + min(t, a.rope.stride - 1);
+      for (int j = 0; j < DH / 2; j += 8) {
+        float k_lo[8], k_hi[8];
+        Vec16<T>::load(k_at(j), k_lo);
+        Vec16<T>::load(k_at(DH / 2 + j), k_hi);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float2 cw = cs[(size_t)(j + e) * a.rope.stride];
+          const float r_lo = k_lo[e] * cw.x - k_hi[e] * cw.y, r_hi = k_hi[e] * cw.x + k_lo[e] * cw.y;
+#pragma unroll
+          for (int gi = 0; gi < kMaxGroup; ++gi)
+            if (gi < g) acc[gi] = fmaf(r_hi, qs[gi * DH + DH / 2 + j + e], fmaf(r_lo, qs[gi * DH + j + e], acc[gi]));
+        }
+      }
+    } else {
+      for (int j = 0; j < DH; j += 8) {
+        float kv[8];
+        Vec16<T>::load(k_at(j), kv);
+#pragma unroll
+        for (int gi = 0; gi < kMaxGroup; ++gi)
+          if (gi < g) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[gi] = fmaf(kv[e], qs[gi * DH + j + e], acc[gi]);
+          }
+      }
+    }
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi)
+      if (gi < g) sc[gi * n_list + idx] = acc[gi];
+  }
+  __syncthreads();
+  for (int gi = 0; gi < g; ++gi) {
+    float mx = -INFINITY;
+    for (int idx = tid; idx < n_tok; idx += 128) mx = fmaxf(mx, sc[gi * n_list + idx]);
+    mx = warp_max(mx);
+    if (lane == 0) red[warp][gi] = mx;
+  }
+  __syncthreads();
+  if (tid < g) s_m[tid] = fmaxf(fmaxf(red[0][tid], red[1][tid]), fmaxf(red[2][tid], red[3][tid]));
+  __syncthreads();
+  for (int gi = 0; gi < g; ++gi) {
+    const float M = s_m[gi];
+    float l = 0.f;
+    for (int idx = tid; idx < n_tok; idx += 128) {
+      const float pv = exp2f(sc[gi * n_list + idx] - M);
+      sc[gi * n_list + idx] = pv;
+      l += pv;
+    }
+    l = warp_sum(l);
+    if (lane == 0) red[warp][gi] = l;
+  }
+  __syncthreads();
+  if (tid < g) s_l[tid] = (red[0][tid] + red[1][tid]) + (red[2][tid] + red[3][tid]);
+  __syncthreads();
+  // weighted values: output dim tid of the head; then the combination with the predicted tokens' result
+  float o[kMaxGroup];
+#pragma unroll
+  for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
+  const bool from_pool = tid < n_stored_v;
+  for (int idx = 0; idx < n_tok; ++idx) {
+    const bool sink = idx < n_sink_tok;
+    const int t = sink ? idx : win_lo + (idx - n_sink_tok);
+    float vv;
+    if (!sink) vv = __bfloat162float(v_recent[((size_t)b * n_rows + (t - t_base)) * (size_t)w.D + (size_t)kvh * DH + tid]);
+    else if (from_pool) vv = __bfloat162float(v_pool[pool_row(t) * (size_t)w.m + (size_t)kvh * DH + tid]);
+    else vv = __bfloat162float(v_side[(side_base + t) * (size_t)w.d_drop + (kvh * DH + tid - w.m)]);
+#pragma unroll
+    for (int gi = 0; gi < kMaxGroup; ++gi)
+      if (gi < g) o[gi] = fmaf(sc[gi * n_list + idx], vv, o[gi]);
+  }
+  for (int gi = 0; gi < g; ++gi) {
+    const size_t row = ((size_t)b * n_q + i) * a.n_q_heads + (size_t)kvh * g + gi;
+    const float lse_a = lse[row];                        // -inf: the query sees no token as predicted
+    const float M = fmaxf(lse_a, s_m[gi]);
+    const float w_a = lse_a > -INFINITY ? exp2f(lse_a - M) : 0.f;
+    const float w_b = exp2f(s_m[gi] - M);
+    const float denom = w_a + w_b * s_l[gi];
+    out[row * DH + tid] = (w_a * out[row * DH + tid] + w_b * o[gi]) / denom;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, int copy_width, __nv_bfloat16* out,
@@ -941,68 +690,54 @@ cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, i
 }
 
 cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
-                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream, int path) {
-  if (path == 2) {
-    if (kv_width % 64 != 0 || reinterpret_cast<uintptr_t>(a.q) % 16 != 0) return cudaErrorInvalidValue;
-    CUtensorMap tm_q, tm_k, tm_v;
-    // few queries per sequence: the CTA's 256 rows are 2, 4 or 8 query heads of one KV head, rows_per_head rows each
-    const int group = a.n_q_heads / a.n_kv_heads;
-    int rows_per_head = 0;
-    for (int r = 32; r <= kTcTile; r *= 2)
-      if (rows_per_head == 0 && n_q <= r && group % (2 * kTcTile / r) == 0) rows_per_head = r;
-    {
-      // q [B][n_q][H_q][128] seen as [B][H_q][2 chunks][n_q][64]: a box is the two 64-dim chunks of 128 query rows,
-      // or one chunk of rows_per_head rows
-      const uint64_t dims[5] = {64, (uint64_t)n_q, 2, (uint64_t)a.n_q_heads, (uint64_t)a.batch};
-      const uint64_t strides[4] = {(uint64_t)a.n_q_heads * 256, 128, 256, (uint64_t)n_q * a.n_q_heads * 256};
-      const uint32_t box[5] = {64, (uint32_t)(rows_per_head ? rows_per_head : kTcTile), rows_per_head ? 1u : 2u, 1, 1};
-      const cudaError_t e = encode_tiled_bf16(&tm_q, a.q, 5, dims, strides, box);
-      if (e != cudaSuccess) return e;
-    }
-    for (int kind = 0; kind < 2; ++kind) {
-      // rows [B][kv_tokens][kv_width] seen as [B][kv_width / 64][kv_tokens][64]: a box is one head (two chunks) of 128 rows
-      const uint64_t dims[4] = {64, (uint64_t)kv_tokens, (uint64_t)kv_width / 64, (uint64_t)a.batch};
-      const uint64_t strides[3] = {(uint64_t)kv_width * 2, 128, (uint64_t)kv_tokens * kv_width * 2};
-      const uint32_t box[4] = {64, (uint32_t)kTcTile, 2, 1};
-      const cudaError_t e = encode_tiled_bf16(kind ? &tm_v : &tm_k, kind ? v_rows : k_rows, 4, dims, strides, box);
-      if (e != cudaSuccess) return e;
-    }
-    dim3 grid(rows_per_head ? 1 : (n_q + 2 * kTcTile - 1) / (2 * kTcTile),
-              rows_per_head ? a.n_q_heads / (2 * kTcTile / rows_per_head) : a.n_q_heads, a.batch);
-    const size_t smem = kWsTailBytes + (size_t)(2 + kWsKStages + kWsVStages) * kTcTileBytes;
-    const cudaError_t e = cudaFuncSetAttribute(prefill_attn_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)smem);
+                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream, int shift,
+                                int n_skip, float* lse_out) {
+  if (kv_width % 64 != 0 || reinterpret_cast<uintptr_t>(a.q) % 16 != 0) return cudaErrorInvalidValue;
+  CUtensorMap tm_q, tm_k, tm_v;
+  // few queries per sequence: the CTA's 256 rows are 2, 4 or 8 query heads of one KV head, rows_per_head rows each
+  const int group = a.n_q_heads / a.n_kv_heads;
+  int rows_per_head = 0;
+  for (int r = 32; r <= kTcTile; r *= 2)
+    if (rows_per_head == 0 && n_q <= r && group % (2 * kTcTile / r) == 0) rows_per_head = r;
+  {
+    // q [B][n_q][H_q][128] seen as [B][H_q][2 chunks][n_q][64]: a box is the two 64-dim chunks of 128 query rows,
+    // or one chunk of rows_per_head rows
+    const uint64_t dims[5] = {64, (uint64_t)n_q, 2, (uint64_t)a.n_q_heads, (uint64_t)a.batch};
+    const uint64_t strides[4] = {(uint64_t)a.n_q_heads * 256, 128, 256, (uint64_t)n_q * a.n_q_heads * 256};
+    const uint32_t box[5] = {64, (uint32_t)(rows_per_head ? rows_per_head : kTcTile), rows_per_head ? 1u : 2u, 1, 1};
+    const cudaError_t e = encode_tiled_bf16(&tm_q, a.q, 5, dims, strides, box);
     if (e != cudaSuccess) return e;
-    prefill_attn_ws_kernel<<<grid, kWsThreads, smem, stream>>>(tm_q, tm_k, tm_v, out, n_q, a.n_q_heads, a.n_kv_heads,
-                                                               a.slots, a.lens, a.geom.max_batch,
-                                                               a.geom.max_pages_per_seq * a.geom.page_tokens,
-                                                               a.scale_log2e, rows_per_head, a.status);
-    return cudaGetLastError();
   }
-  if (path == 1) {
-    dim3 grid((n_q + kTcTile - 1) / kTcTile, a.n_q_heads, a.batch);
-    const size_t smem = 1024 + 6 * (size_t)kTcTileBytes + sizeof(PfTcTail);
-    const cudaError_t e = cudaFuncSetAttribute(prefill_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)smem);
+  for (int kind = 0; kind < 2; ++kind) {
+    // rows [B][kv_tokens][kv_width] seen as [B][kv_width / 64][kv_tokens][64]: a box is one head (two chunks) of 128 rows
+    const uint64_t dims[4] = {64, (uint64_t)kv_tokens, (uint64_t)kv_width / 64, (uint64_t)a.batch};
+    const uint64_t strides[3] = {(uint64_t)kv_width * 2, 128, (uint64_t)kv_tokens * kv_width * 2};
+    const uint32_t box[4] = {64, (uint32_t)kTcTile, 2, 1};
+    const cudaError_t e = encode_tiled_bf16(kind ? &tm_v : &tm_k, kind ? v_rows : k_rows, 4, dims, strides, box);
     if (e != cudaSuccess) return e;
-    prefill_attn_tc_kernel<<<grid, 256, smem, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q), k_rows, v_rows, out,
-                                                        n_q, a.n_q_heads, a.n_kv_heads, kv_tokens, kv_width, a.slots,
-                                                        a.lens, a.geom.max_batch,
-                                                        a.geom.max_pages_per_seq * a.geom.page_tokens, a.scale_log2e,
-                                                        a.status);
-    return cudaGetLastError();
   }
-  dim3 grid((n_q + kPfRows - 1) / kPfRows, a.n_q_heads, a.batch);
-  const size_t smem = 4 * (size_t)kPfKeys * kPfRowBytes;
-  cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  dim3 grid(rows_per_head ? 1 : (n_q + 2 * kTcTile - 1) / (2 * kTcTile),
+            rows_per_head ? a.n_q_heads / (2 * kTcTile / rows_per_head) : a.n_q_heads, a.batch);
+  const size_t smem = kWsTailBytes + (size_t)(2 + kWsKStages + kWsVStages) * kTcTileBytes;
+  const cudaError_t e = cudaFuncSetAttribute(prefill_attn_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                           cudaSharedmemCarveoutMaxShared);
+  prefill_attn_ws_kernel<<<grid, kWsThreads, smem, stream>>>(tm_q, tm_k, tm_v, out, n_q, a.n_q_heads, a.n_kv_heads,
+                                                             a.slots, a.lens, a.geom.max_batch,
+                                                             a.geom.max_pages_per_seq * a.geom.page_tokens,
+                                                             a.scale_log2e, rows_per_head, a.status, shift, n_skip,
+                                                             lse_out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_band(const AttnArgs& a, const PrefillBand& band, int n_q, float* out, const float* lse,
+                                cudaStream_t stream) {
+  const int n_list = band.n_sink + band.n_window;
+  const size_t smem = (size_t)(kMaxGroup * 128 + kMaxGroup * n_list) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(prefill_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  prefill_attn_kernel<<<grid, 128, smem, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.q), k_rows, v_rows, out, n_q,
-                                                a.n_q_heads, a.n_kv_heads, kv_tokens, kv_width, a.slots, a.lens,
-                                                a.geom.max_batch, a.geom.max_pages_per_seq * a.geom.page_tokens,
-                                                a.scale_log2e, a.status);
+  dim3 grid(n_q, a.n_kv_heads, a.batch);
+  prefill_band_kernel<<<grid, 128, smem, stream>>>(a, band, n_q, out, lse);
   return cudaGetLastError();
 }
 

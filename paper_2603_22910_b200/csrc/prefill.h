@@ -13,11 +13,27 @@ cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, i
                                int out_tokens, int out_width, bool rotate, int zero_tail, cudaStream_t stream);
 
 // Eq. 7 for n_q queries per sequence (a.q: [B][n_q][H_q][128] bf16), query i at position len - n_q + i attending the
-// keys up to its own, over k_rows / v_rows [B][kv_tokens][kv_width] bf16.  out: fp32 [B][n_q][H_q][128].
+// keys n_skip .. its own position - shift (plain causal attention: shift = n_skip = 0), over k_rows / v_rows
+// [B][kv_tokens][kv_width] bf16 (v_rows zeroed from each sequence's length to the next multiple of 128 rows).
+// out: fp32 [B][n_q][H_q][128]; lse_out (may be null): fp32 [B][n_q][H_q], log2 of every row's softmax denominator in
+// base-2 score units, -inf for a row that attends nothing (its output is zero).
 // A sequence with fewer than n_q cached tokens gets zeros and the device status EBADLENGTH.
-// path: 0 = mma.sync kernel, 1 = tcgen05 kernel (one thread group does every step in turn), 2 = warp-specialised
-// tcgen05 kernel (needs v_rows zeroed from each sequence's length to the next multiple of 128 rows).
 cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, const __nv_bfloat16* v_rows,
-                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream, int path);
+                                int kv_tokens, int kv_width, int n_q, float* out, cudaStream_t stream, int shift = 0,
+                                int n_skip = 0, float* lse_out = nullptr);
+
+// The sink and recent-window tokens of every query at full precision (Section 4.1), added to what launch_prefill_attn
+// (shift = n_window, n_skip = n_sink) left in out / lse: query i at position p reads the sink tokens t < min(n_sink,
+// p + 1) from the layer's pools (dims below mk / m) and side buffers (the rest), and the window tokens
+// max(n_sink, p - n_window + 1) .. p from k_recent / v_recent: [B][n_q + n_window - 1][D] bf16, whole K / V rows of
+// the positions len - n_q - n_window + 1 .. len - 1 (rows of negative positions are never read).
+struct PrefillBand {
+  const void* k_recent; const void* v_recent;
+  const void* k_pool; const void* v_pool;    // the layer's pools, row widths mk and m (null when 0)
+  const void* k_side; const void* v_side;    // [max_batch][n_sink + n_window][D - m]; k_side null when mk == D
+  int D, mk, m, d_drop, n_sink, n_window;
+};
+cudaError_t launch_prefill_band(const AttnArgs& a, const PrefillBand& band, int n_q, float* out, const float* lse,
+                                cudaStream_t stream);
 
 }  // namespace echokv

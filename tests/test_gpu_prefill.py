@@ -74,13 +74,10 @@ CASES = [
 
 
 @pytest.mark.parametrize("name,base,over,lens,n_q,biases,rope", CASES, ids=[c[0] for c in CASES])
-@pytest.mark.parametrize("path", [0, 1, 2], ids=["mma_sync", "tcgen05", "tcgen05_ws"])
-def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope, path):
+def test_prefill_against_oracle(name, base, over, lens, n_q, biases, rope):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], biases=biases, rope=rope)
     ctx = case.ctx
-    assert binding.lib().echokv_prefill_path(ctx.handle) == 2
-    ctx.set_prefill_path(path)
     for layer in (1, 0):
         q = queries(w, n_q, layer)
         # the scratch starts as NaN patterns: rows past a sequence's end must never reach a result
@@ -117,15 +114,16 @@ def test_prefill_short_sequences_and_argument_checks():
     qd = q.to(dev)
     scratch = ctx.prefill_scratch
     args = (qd.data_ptr(), o.data_ptr())
-    assert lib.echokv_prefill_attention(h, 1, *args, 0, None, case.seq_lens.data_ptr(), 3, scratch.data_ptr(),
-                                        scratch.numel(), None) == binding.ECHOKV_EINVAL
-    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, scratch.data_ptr(), 1024,
-                                        None) == binding.ECHOKV_ECAPACITY
-    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, None, 0,
+    assert lib.echokv_prefill_attention(h, 1, *args, 0, None, case.seq_lens.data_ptr(), 3, None, None,
+                                        scratch.data_ptr(), scratch.numel(), None) == binding.ECHOKV_EINVAL
+    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, None, None,
+                                        scratch.data_ptr(), 1024, None) == binding.ECHOKV_ECAPACITY
+    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, None, None, None, 0,
                                         None) == binding.ECHOKV_EINVAL
+    # with a window set the call needs the recent tokens' rows from the caller
     ctx.set_full_precision_window(4, 128)
-    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, scratch.data_ptr(),
-                                        scratch.numel(), None) == binding.ECHOKV_EUNSUPPORTED
+    assert lib.echokv_prefill_attention(h, 1, *args, n_q, None, case.seq_lens.data_ptr(), 3, None, None,
+                                        scratch.data_ptr(), scratch.numel(), None) == binding.ECHOKV_EINVAL
     case.close()
     small = Case(synth.C0, layers=[1])
     n = torch.zeros(1, dtype=torch.int64)
@@ -177,15 +175,13 @@ def test_chunk_append_equals_token_by_token(window):
     short.close()
 
 
-@pytest.mark.parametrize("path", [1, 2], ids=["tcgen05", "tcgen05_ws"])
-def test_prefill_scores_that_jump_mid_sequence(path):
+def test_prefill_scores_that_jump_mid_sequence():
     """A few keys in the middle of the cache score far above everything before them (2^46 and more above the running
-    reference, some beyond what 2^x can hold in fp32): the kernels that keep a lazy reference maximum must notice,
-    move it and rescale what they have accumulated."""
+    reference, some beyond what 2^x can hold in fp32): the kernel, which keeps a lazy reference maximum, must notice,
+    move it and rescale what it has accumulated."""
     w = synth.C2.replace(batch=1, context=1000)
     case = Case(w, lens=[1000], layers=[0])
     ctx = case.ctx
-    ctx.set_prefill_path(path)
     hot = slice(400, 421)
     rows = case.host[(0, "k", 0)]
     rows[hot] = rows[hot] * 32                       # (a power of two: exact in bf16)
