@@ -26,6 +26,12 @@ CASES = [
     ("fp32_d64_window", synth.C0, dict(batch=2, context=200), [200, 50], (2, 16), [0, 17]),
     ("nothing_retained", synth.C2, dict(batch=2, context=300, n_retained_heads=0), [300, 140], (4, 128), [0, 200]),
     ("pages128", synth.C2, dict(batch=2, context=700, page_tokens=128, random_pages=True), [700, 129], (3, 37), [0, 128]),
+    ("split_head_window", synth.C2, dict(batch=2, context=500, n_retained_dims=64, n_retained_heads=0, group_size=4,
+                                         n_layers=4), [500, 131], (4, 128), [0, 250]),
+    ("keys_whole_window", synth.C2, dict(batch=2, context=600, save_k=True, random_pages=True), [600, 140], (4, 128),
+     [0, 333]),
+    ("keys_whole", synth.C2, dict(batch=2, context=300, save_k=True, n_retained_dims=384, n_retained_heads=3), [300, 17],
+     None, [0, 100]),
 ]
 
 
@@ -34,6 +40,8 @@ def test_evicted_layer_equals_a_layer_cached_compressed(name, base, over, lens, 
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], window=window)
     ctx, dev = case.ctx, case.ctx.device
+    if w.save_k:
+        ctx.enable_absorbed()           # (keys kept whole: decode calls are served by the absorbed mode)
     want_out = case.run(1)
     assert_parity(want_out, case.oracle(1), w.dtype, name + " before")
     n_pages = case.cfg.n_pages
@@ -59,10 +67,13 @@ def test_evicted_layer_equals_a_layer_cached_compressed(name, base, over, lens, 
                 for b in range(w.batch):
                     got = torch.stack([mine[1][int(case.table[b, t // w.page_tokens]), t % w.page_tokens]
                                        for t in (0, lens[b] // 2, lens[b] - 1)]).cpu()
-                    ref = O.retained_dims(full[kind][b][[0, lens[b] // 2, lens[b] - 1]].float().numpy(), w.m)
+                    ref = O.retained_dims(full[kind][b][[0, lens[b] // 2, lens[b] - 1]].float().numpy(),
+                                          w.mk if kind == "k" else w.m)
                     np.testing.assert_array_equal(got.float().numpy(), ref)
         if side_keep is not None:
-            assert torch.equal(ctx.k_side[1], side_keep[0]) and torch.equal(ctx.v_side[1], side_keep[1])
+            assert torch.equal(ctx.v_side[1], side_keep[1])
+            if not w.save_k:               # (whole keys are in the pool: their side buffer is neither written nor read)
+                assert torch.equal(ctx.k_side[1], side_keep[0])
         np.testing.assert_array_equal(case.run(1), want_out)
         assert ctx.device_status() == binding.ECHOKV_OK
 

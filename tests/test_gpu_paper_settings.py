@@ -79,6 +79,9 @@ def oracle_prefill(case, layer, q, b):
         kw = dict(k_true_drop=O.widen(synth.to_numpy_stored(case.true_drop[(layer, "k", b)])),
                   v_true_drop=O.widen(synth.to_numpy_stored(case.true_drop[(layer, "v", b)])),
                   n_sink=case.window[0], n_window=case.window[1])
+    if w.save_k:                 # keys kept whole (Section 5.2): the stored K rows are the whole keys
+        kw["k_true"] = case._stored(layer, "k", b)
+        kl = kw["k_true"][:, :w.m]
     return O.prefill_attention(qn, kg, vg, kl, vl, Wk, Wv, w.n_kv_heads, bk=bk, bv=bv, rope_theta=case.rope, **kw)
 
 
@@ -96,5 +99,24 @@ def test_prefill_at_the_papers_settings(m, rope, window, biases):
     out = out.cpu().numpy().astype(np.float64)
     for b in range(w.batch):
         check(out[b], oracle_prefill(case, 1, q, b), "prefill m=%d seq %d" % (m, b))
+    assert ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+@pytest.mark.parametrize("rope", [None, THETA], ids=["norope", "rope"])
+def test_prefill_with_whole_keys_and_a_window(rope):
+    """Section 5.2 ("save K") with Section 4.1: the keys are stored whole, the window matters to the values only."""
+    w = workload(384).replace(save_k=True, name="paper_m384_saveK")
+    lens = [700, 333, 170]
+    case = Case(w, lens=lens, layers=[0, 1], biases=True, window=(4, 128), rope=rope)
+    ctx, dev = case.ctx, case.ctx.device
+    n_q = 140
+    q = synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, 6).to(synth.torch_dtype(w))
+    recent = case.recent_rows(1, n_q)
+    out = ctx.prefill_attention(1, q.to(dev), case.seq_lens, k_recent=recent[0], v_recent=recent[1])
+    torch.cuda.synchronize()
+    out = out.cpu().numpy().astype(np.float64)
+    for b in range(w.batch):
+        check(out[b], oracle_prefill(case, 1, q, b), "prefill, whole keys, seq %d" % b)
     assert ctx.device_status() == binding.ECHOKV_OK
     case.close()

@@ -61,6 +61,29 @@ def test_save_k_against_oracle(name, base, over, lens, biases, rope):
     case.close()
 
 
+WINDOW_CASES = [
+    ("c2_shape", synth.C2, dict(batch=3, context=900, random_pages=True), [900, 517, 100], (4, 128), True),
+    ("m_384_short_window", synth.C2, dict(batch=2, context=500, n_retained_dims=384, n_retained_heads=3), [500, 20],
+     (2, 33), False),
+    ("nothing_of_v_retained", synth.C2, dict(batch=2, context=400, n_retained_heads=0), [400, 131], (4, 128), False),
+]
+
+
+@pytest.mark.parametrize("name,base,over,lens,window,biases", WINDOW_CASES, ids=[c[0] for c in WINDOW_CASES])
+@pytest.mark.parametrize("rope", [None, THETA], ids=["plain", "rotated"])
+def test_save_k_with_sink_and_window(name, base, over, lens, window, biases, rope):
+    """Whole keys with sink / window tokens (Section 5.2 with Section 4.1): the keys are all stored, so the window
+    matters to the values only; decode and the prefill-shaped call."""
+    w = base.replace(save_k=True, **over)
+    case = Case(w, lens=lens, layers=[0, 1], biases=biases, window=window, rope=rope)
+    ctx = case.ctx
+    ctx.enable_absorbed()
+    assert_parity(case.run(1), case.oracle(1), w.dtype, name)
+    assert_parity(case.run(0), case.oracle(0), w.dtype, name + " anchor")
+    assert ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
 def test_save_k_limits():
     w = synth.C2.replace(batch=1, context=300, save_k=True)
     cfg = binding.config_for(w)
@@ -68,14 +91,6 @@ def test_save_k_limits():
     assert sizes.compressed_pool_bytes == cfg.n_pages * w.page_tokens * w.m * 2       # the V pool
     assert sizes.anchor_pool_bytes == cfg.n_pages * w.page_tokens * w.D * 2           # the K pool in this setting
     ctx = binding.Context(cfg)
-    with pytest.raises(binding.EchoKVError) as e:
-        ctx.set_full_precision_window(4, 128)
-    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
-    pool = torch.zeros((cfg.n_pages, w.page_tokens, w.D), dtype=torch.bfloat16, device=ctx.device)
-    lens = torch.tensor([300], dtype=torch.int32, device=ctx.device)
-    with pytest.raises(binding.EchoKVError) as e:
-        ctx.compress_layer(1, pool, pool, lens)
-    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
     # Wv is still required, Wk is not
     lib = binding.lib()
     wv = torch.zeros((w.d_drop, w.d_in), dtype=torch.bfloat16, device=ctx.device)
