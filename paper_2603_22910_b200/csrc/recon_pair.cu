@@ -8,8 +8,13 @@
 //   stage      = per CTA 128 token rows and the 128 predictor rows of its head, two 64-feature chunks
 //                of each (64 KiB, 3 deep); every MMA reads the token rows of both CTAs and the predictor
 //                rows of both CTAs, so each operand byte is fetched into shared memory once per pair.
-//                When the CTA's 128 tokens lie consecutively in the pool a stage is two TMA copies
-//                (tokens, predictor); otherwise 64-row runs or single pages are copied chunk by chunk
+//                The token rows sit as 1 KiB swizzle atoms (8 rows x 64 features) in the order (8-row group,
+//                chunk): one TMA box then brings BOTH chunks of a page (the pools are described to TMA as
+//                [group][chunk][row][64]), and the groups of one chunk are a uniform 2 KiB apart for the
+//                operand descriptor.  A stage is one copy per page -- 8 + 1 with 16-token pages in any order
+//                (an SM starts only about one copy per 80 cycles whatever its size, and a stage is ~1000
+//                cycles of tensor work) -- one per run of 64 consecutive rows, or one when the CTA's 128
+//                tokens lie consecutively in the pool
 //   K phase    : acc0[tok, feat] (M = tokens: 128 per CTA, N = 256 features of both heads)
 //                -> a thread owns (token, head): scores of the head's G query heads, tile max / exp2 /
 //                   sum over the CTA's 128 tokens; the probabilities go to the CTA that owns the
@@ -42,6 +47,8 @@ constexpr int kRowBytes = kChunk * 2;
 constexpr int kStageChunks = 2;                      // 64-feature chunks per stage
 constexpr int kStages = 3;
 constexpr int kXBytes = kCtaTokens * kRowBytes;      // 16 KiB: token rows of one chunk
+constexpr int kAtomBytes = 8 * kRowBytes;            // 1 KiB: 8 token rows of one chunk
+constexpr int kGroupBytes = kStageChunks * kAtomBytes;   // 2 KiB: an 8-row group, chunk after chunk
 constexpr int kWRows = 128;                          // predictor rows per CTA: one head
 constexpr int kWBytes = kWRows * kRowBytes;          // 16 KiB: predictor rows of one chunk
 constexpr int kStageXBytes = kStageChunks * kXBytes;  // token rows: chunk 0, chunk 1
@@ -113,12 +120,12 @@ __device__ __forceinline__ bool epilogue_all(bool ok) {
   return r != 0;
 }
 
-// K-major bf16 operand, 128-byte rows in the 128-byte swizzle, 8-row groups 1024 bytes apart
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+// K-major bf16 operand, 128-byte rows in the 128-byte swizzle, 8-row groups group_bytes apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t group_bytes = 1024) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
   d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(group_bytes >> 4) << 32;
   d |= static_cast<uint64_t>(1) << 46;
   d |= static_cast<uint64_t>(2) << 61;
   return d;
@@ -218,7 +225,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
   const uint32_t tmem = t.tmem_base;
   const int n_items = t.cum_tiles[p.nb] * p.n_pairs;
   const int boxes = kCtaTokens / p.page_tokens;             // TMA boxes (pages) of this CTA's tokens
-  const uint32_t page_bytes = p.page_tokens * kRowBytes;
+  const uint32_t page_bytes = p.page_tokens * kRowBytes;    // of one chunk
   const uint32_t peer_abort = mapa_u32(smem_u32(&t.abort_flag), rank ^ 1u);
   // stages per phase: two chunks each.  With an odd number of chunks (a retained width that is an odd multiple
   // of 64) the last stage's second chunk lies past the end of the pool rows and of the predictor rows: TMA fills
@@ -290,16 +297,14 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
           if (lane == 0) mbar_arrive_expect_tx_cluster(full, stage_tx);
           __syncwarp();
           const uint32_t x_dst = stage_base + s * kStageBytes;
+          // one box = both chunks of the rows it covers, as (group, chunk) atoms
           if (run128) {
             if (lane == 0)
-              tma_load_3d_pair(x_dst, from_anchor ? m_anchor_128 : m_local_128, 0, page * p.page_tokens, kx0, full);
+              tma_load_4d_pair(x_dst, from_anchor ? m_anchor_128 : m_local_128, 0, 0, kx0, page * p.page_tokens / 8, full);
           } else if (page >= 0 && !run_member) {
             const CUtensorMap* m = run_lead ? (from_anchor ? m_anchor_run : m_local_run)
                                             : (from_anchor ? m_anchor : m_local);
-#pragma unroll
-            for (int j = 0; j < kStageChunks; ++j)
-              tma_load_2d_pair(x_dst + j * kXBytes + lane * page_bytes, m, (kx0 + j) * kChunk, page * p.page_tokens,
-                               full);
+            tma_load_4d_pair(x_dst + lane * kStageChunks * page_bytes, m, 0, 0, kx0, page * p.page_tokens / 8, full);
           }
           if (lane == 16)
             tma_load_3d_pair(x_dst + kStageXBytes, m_w, 0, w.pair * 2 * kWRows + (int)rank * kWRows, kc0, full);
@@ -330,12 +335,13 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
             tc_fence_after();
 #pragma unroll
             for (int j = 0; j < kStageChunks; ++j) {
-              const uint32_t x_addr = stage_base + s * kStageBytes + j * kXBytes;
+              const uint32_t x_addr = stage_base + s * kStageBytes + j * kAtomBytes;
               const uint32_t w_addr = stage_base + s * kStageBytes + kStageXBytes + j * kWBytes;
               // K phase: A = token rows (128 per CTA), B = predictor rows (128 per CTA: 256 features).
               // V phase: A = predictor rows (head r on CTA r), B = token rows (128 per CTA: 256 tokens).
-              const uint64_t a_desc = umma_desc(phase == 0 ? x_addr : w_addr);
-              const uint64_t b_desc = umma_desc(phase == 0 ? w_addr : x_addr);
+              const uint64_t x_desc = umma_desc(x_addr, kGroupBytes), w_desc = umma_desc(w_addr);
+              const uint64_t a_desc = phase == 0 ? x_desc : w_desc;
+              const uint64_t b_desc = phase == 0 ? w_desc : x_desc;
 #pragma unroll
               for (int k16 = 0; k16 < kChunk / 16; ++k16)   // +32 bytes along K = +2 in the address field
                 tc_mma_bf16_pair(d_tmem, a_desc + 2 * k16, b_desc + 2 * k16, kIdescPair,
@@ -651,8 +657,8 @@ cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUt
   }
   if (n_clusters > resident_pairs) n_clusters = resident_pairs;
   cfg.gridDim = dim3(2 * n_clusters, 1, 1);
-  return cudaLaunchKernelEx(&cfg, recon_pair_kernel<G, ROPE, KS>, anchor.k_pool, anchor.v_pool, lk, lv, anchor.k_pool_run,
-                            anchor.v_pool_run, lkr, lvr, anchor.k_pool_run128, anchor.v_pool_run128, lk8, lv8,
+  return cudaLaunchKernelEx(&cfg, recon_pair_kernel<G, ROPE, KS>, anchor.k_grp_page, anchor.v_grp_page, lk, lv,
+                            anchor.k_grp_64, anchor.v_grp_64, lkr, lvr, anchor.k_grp_128, anchor.v_grp_128, lk8, lv8,
                             layer.wk_half, layer.wv_half, p);
 }
 
@@ -714,12 +720,12 @@ static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const
   p.store_rotate = store.rotate;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
-  const CUtensorMap& lk = r.m > 0 ? layer.k_pool : anchor.k_pool;
-  const CUtensorMap& lv = r.m > 0 ? layer.v_pool : anchor.v_pool;
-  const CUtensorMap& lkr = r.m > 0 ? layer.k_pool_run : anchor.k_pool_run;
-  const CUtensorMap& lvr = r.m > 0 ? layer.v_pool_run : anchor.v_pool_run;
-  const CUtensorMap& lk8 = r.m > 0 ? layer.k_pool_run128 : anchor.k_pool_run128;
-  const CUtensorMap& lv8 = r.m > 0 ? layer.v_pool_run128 : anchor.v_pool_run128;
+  const CUtensorMap& lk = r.m > 0 ? layer.k_grp_page : anchor.k_grp_page;
+  const CUtensorMap& lv = r.m > 0 ? layer.v_grp_page : anchor.v_grp_page;
+  const CUtensorMap& lkr = r.m > 0 ? layer.k_grp_64 : anchor.k_grp_64;
+  const CUtensorMap& lvr = r.m > 0 ? layer.v_grp_64 : anchor.v_grp_64;
+  const CUtensorMap& lk8 = r.m > 0 ? layer.k_grp_128 : anchor.k_grp_128;
+  const CUtensorMap& lv8 = r.m > 0 ? layer.v_grp_128 : anchor.v_grp_128;
   if (p.kc_anchor % kStageChunks != 0) return cudaErrorInvalidValue;   // (a stage never straddles the two pools)
   const int tiles_cap = (r.capacity_tokens + kTileTokens - 1) / kTileTokens;
   for (int b0 = 0; b0 < a.batch; b0 += kMaxBatchPerLaunch) {
@@ -771,6 +777,7 @@ cudaError_t launch_recon_pair_store(const AttnArgs& a, const ReconArgs& r, const
   auto as_keys = [](const TcLayerMaps& m) {
     TcLayerMaps t = m;
     t.k_pool = m.v_pool; t.k_pool_run = m.v_pool_run; t.k_pool_run128 = m.v_pool_run128;
+    t.k_grp_page = m.v_grp_page; t.k_grp_64 = m.v_grp_64; t.k_grp_128 = m.v_grp_128;
     t.wk = m.wv; t.wk_half = m.wv_half;
     return t;
   };

@@ -589,6 +589,24 @@ cudaError_t encode_3d_chunks(CUtensorMap* map, const void* base, uint64_t rows, 
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// The same matrix seen as [rows / 8][cols / 64][8][64] (8-row groups outermost): a box of box_rows rows x 2 chunks
+// lands in shared memory as 1 KiB swizzle atoms (8 rows x 64 columns) in the order (group, chunk).  A chunk past
+// the last column reads as zeros.
+cudaError_t encode_4d_groups(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                             CUtensorMapL2promotion promo) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return cudaErrorNotSupported;
+  if (rows % 8 != 0 || box_rows % 8 != 0) return cudaErrorInvalidValue;
+  cuuint64_t dims[4] = {kChunk, 8, cols / kChunk, rows / 8};
+  cuuint64_t strides[3] = {cols * 2, kChunk * 2, 8 * cols * 2};
+  cuuint32_t box[4] = {kChunk, 8, 2, box_rows / 8};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 cudaError_t encode_chunked_3d_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int box_rows,
                                   int box_chunks) {
   return encode_3d_chunks(map, base, rows, cols, box_rows, box_chunks, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
@@ -630,11 +648,17 @@ cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, int k_wid
     // CTA-pair kernel: 128 consecutive token rows x two 64-feature chunks in one copy
     // (of a pool one chunk wide the box's second chunk lies outside the tensor and reads as zeros)
     if ((e = encode_3d_chunks(&maps->k_pool_run128, k_pool, rows, k_width, 128, 2, promo)) != cudaSuccess) return e;
+    if ((e = encode_4d_groups(&maps->k_grp_page, k_pool, rows, k_width, page_tokens, promo)) != cudaSuccess) return e;
+    if ((e = encode_4d_groups(&maps->k_grp_64, k_pool, rows, k_width, 64, promo)) != cudaSuccess) return e;
+    if ((e = encode_4d_groups(&maps->k_grp_128, k_pool, rows, k_width, 128, promo)) != cudaSuccess) return e;
   }
   if (v_width > 0) {
     if ((e = encode_2d(&maps->v_pool, v_pool, rows, v_width, page_tokens, promo)) != cudaSuccess) return e;
     if ((e = encode_2d(&maps->v_pool_run, v_pool, rows, v_width, kRunTokens, promo)) != cudaSuccess) return e;
     if ((e = encode_3d_chunks(&maps->v_pool_run128, v_pool, rows, v_width, 128, 2, promo)) != cudaSuccess) return e;
+    if ((e = encode_4d_groups(&maps->v_grp_page, v_pool, rows, v_width, page_tokens, promo)) != cudaSuccess) return e;
+    if ((e = encode_4d_groups(&maps->v_grp_64, v_pool, rows, v_width, 64, promo)) != cudaSuccess) return e;
+    if ((e = encode_4d_groups(&maps->v_grp_128, v_pool, rows, v_width, 128, promo)) != cudaSuccess) return e;
     // absorbed mode, V side: 64 consecutive token rows x four 64-feature chunks in one copy
     if (v_width >= 256) {
       if ((e = encode_3d_chunks(&maps->v_pool_tok64x4, v_pool, rows, v_width, 64, 4, promo)) != cudaSuccess) return e;

@@ -16,6 +16,12 @@ struct TcLayerMaps {
   // 128 rows each: of the pools (128 consecutive token rows) and of the predictors (one head)
   CUtensorMap k_pool_run128, v_pool_run128;
   CUtensorMap wk_half, wv_half;
+  // CTA-pair kernel: the pools seen as [8-row group][64-column chunk][row of the group][64], so that ONE box holds
+  // two 64-feature chunks of a page (or of a run of 64 / 128 consecutive token rows) and lands in shared memory as
+  // 8-row swizzle atoms in the order (group, chunk): the groups of one chunk are then a uniform 2 KiB apart, which a
+  // tensor-core operand descriptor can walk.  Boxes of one page, of 64 rows and of 128 rows
+  CUtensorMap k_grp_page, k_grp_64, k_grp_128;
+  CUtensorMap v_grp_page, v_grp_64, v_grp_128;
   CUtensorMap v_pool_tok64x4;           // [chunk][row][64] view of the V pool, boxes of 4 chunks x 64 rows
   bool pools_ready = false;
   bool weights_ready = false;

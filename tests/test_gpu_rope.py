@@ -122,14 +122,14 @@ def test_rotated_keys_with_the_absorbed_value_side(name, base, over, lens, windo
     case.close()
 
 
-def test_rope_needs_whole_heads():
-    w = synth.C2.replace(batch=1, context=300, n_retained_dims=64)
-    cfg = binding.config_for(w)
-    ctx = binding.Context(cfg)
-    with pytest.raises(binding.EchoKVError) as e:
-        ctx.set_rope(THETA)
-    assert e.value.status == binding.ECHOKV_EUNSUPPORTED
-    ctx.close()
+def test_rope_with_a_retained_width_that_splits_a_head():
+    # the paper's m = 64 keeps half of head 0: the split head is predicted whole (its stored dims passed through),
+    # so the rotation, which pairs feature j with j + 64 of a head, finds both halves in one place
+    w = synth.C2.replace(batch=2, context=300, n_retained_dims=64, n_retained_heads=0)
+    case = Case(w, lens=[300, 77], layers=[0, 1], rope=THETA)
+    assert_parity(case.run(1), case.oracle(1), w.dtype, "m = 64, rotated")
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
 
 
 def test_rope_argument_checks():
