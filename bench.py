@@ -620,8 +620,15 @@ def run_prefill(args):
     q_chk = O.widen(synth.to_numpy_stored(q[0, -n_chk:].cpu()))
     kw = {}
     if st.window:
-        kw = dict(k_true_drop=st.true_dropped(1, "k", 0), v_true_drop=st.true_dropped(1, "v", 0),
-                  n_sink=st.window[0], n_window=st.window[1])
+        # the queries' own windows reach back n_window - 1 tokens before the chunk: their true dims come from the rows
+        # handed to the call (the sink tokens' from what the side buffers hold)
+        true = {}
+        for kind in ("k", "v"):
+            t = st.true_dropped(1, kind, 0)
+            rows = recent[kind + "_recent"][0].cpu()
+            t[w.context - rows.shape[0]:] = O.widen(synth.to_numpy_stored(rows))[:, w.m:]
+            true[kind] = t
+        kw = dict(k_true_drop=true["k"], v_true_drop=true["v"], n_sink=st.window[0], n_window=st.window[1])
     ref = O.prefill_attention(q_chk, *inputs[1:], n_kv_heads=w.n_kv_heads, rope_theta=args.rope or None, **kw)
     got = out[0, -n_chk:].cpu().numpy().astype(np.float64)
     line = {

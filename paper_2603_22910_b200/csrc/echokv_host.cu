@@ -668,7 +668,7 @@ int echokv_prefill_attention(echokv_ctx* c, int layer, const void* q, float* out
   const int k_copy = (compressed && !keys_whole) ? c->d.m_heads : k_width;
   const int v_copy = compressed ? c->d.m_heads : v_width;
   if (launch_gather_rows(a, L.k_pool, k_width, k_copy, k_rows, c->d.capacity, c->d.D, true, 0, s) != cudaSuccess ||
-      launch_gather_rows(a, L.v_pool, v_width, v_copy, v_rows, c->d.capacity, c->d.D, false, 128, s) != cudaSuccess)
+      launch_gather_rows(a, L.v_pool, v_width, v_copy, v_rows, c->d.capacity, c->d.D, false, 128, s, true) != cudaSuccess)
     return ECHOKV_ECUDA;
   c->launches += (k_copy > 0 ? 1 : 0) + 1;
   if (compressed) {

@@ -13,9 +13,14 @@
 //      sequence cut off at its own position: step 3 then covers the tokens the query sees as predicted (those more
 //      than n_window - 1 positions before it, the sink left out), and prefill_band_kernel adds the query's own sink
 //      and window tokens from their stored values and combines the two by log-sum-exp.
-// The rebuilt rows are bf16 in a caller-owned scratch, as in the paper's own materialise-then-attend
-// design; the decode path never writes them.
+// The rebuilt rows are 16-bit in a caller-owned scratch, as in the paper's own materialise-then-attend
+// design; the decode path never writes them.  K~ rows are bf16 (the S = Q K^T MMA takes bf16 queries).  V~ rows
+// are fp16, and so are the probabilities of the P V MMA: a query that sees a handful of tokens returns nearly one
+// V~ row, so the rounding of that row shows unaveraged in the output -- 2^-9 |v| in bf16, 2^-12 |v| in fp16
+// (stored bf16 values are exact in fp16 between 6e-5 and 65504; probabilities stay below 2^15).
 #include "prefill.h"
+
+#include <cuda_fp16.h>
 
 #include "ptx_sm100.cuh"
 #include "recon_tc.h"
@@ -32,7 +37,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
                                                           int copy_width, __nv_bfloat16* __restrict__ out, int out_tokens,
                                                           int out_width, const int32_t* __restrict__ slots,
                                                           const int32_t* __restrict__ lens, PageGeom g, RopeTable rope,
-                                                          int zero_tail, int block_tokens, int32_t* status) {
+                                                          int zero_tail, int block_tokens, int32_t* status, int to_half) {
   const int b = blockIdx.y, t0 = blockIdx.x * block_tokens;
   const int slot = slots ? slots[b] : b;
   const int len = lens[b];
@@ -104,6 +109,18 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
         }
         lo[u] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
         hi[u] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      } else if (to_half) {
+        // the same values as fp16 (value rows; exact for every stored value a cache holds in practice)
+        uint32_t lw[4] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w}, hw[4] = {hi[u].x, hi[u].y, hi[u].z, hi[u].w};
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) {
+          const __half2 a = __floats2half2_rn(__uint_as_float(lw[e2] << 16), __uint_as_float(lw[e2] & 0xffff0000u));
+          const __half2 bb = __floats2half2_rn(__uint_as_float(hw[e2] << 16), __uint_as_float(hw[e2] & 0xffff0000u));
+          lw[e2] = *reinterpret_cast<const uint32_t*>(&a);
+          hw[e2] = *reinterpret_cast<const uint32_t*>(&bb);
+        }
+        lo[u] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+        hi[u] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
       }
       __nv_bfloat16* dst = out + ((size_t)b * out_tokens + t) * (size_t)out_width + head[u] * 128 + c * 8;
       *reinterpret_cast<uint4*>(dst) = lo[u];
@@ -121,8 +138,9 @@ constexpr int kTcChunkBytes = kTcTile * 128;     // [128 rows x 64 dims] bf16, 1
 constexpr int kTcTileBytes = 2 * kTcChunkBytes;  // 128 dims
 constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
+// two probabilities as an fp16 pair (the A operand of the P V MMA)
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  const __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
@@ -172,9 +190,11 @@ constexpr int kWsKStages = 3, kWsVStages = 2;
 constexpr int kWsSoftmaxWarps = 16;
 constexpr int kWsThreads = (kWsSoftmaxWarps + 2) * 32;
 constexpr int kWsTailBytes = 3072;                                   // the tail sits in front of the tiles
-constexpr uint32_t kIdescPV = kIdescS | (1u << 16);                 // B operand N-major
+// P V: fp16 x fp16 -> fp32 (formats 0), M = 128, N = 128, B operand N-major
+constexpr uint32_t kIdescPV = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24) | (1u << 16);
 constexpr float kWsGrowLog2 = 8.f;                // the careful path moves the reference if the maximum is this far above it
-constexpr float kWsSumLimit = 1099511627776.f;    // 2^40: a half-row's probabilities summing to less leave the reference alone
+constexpr float kWsSumLimit = 32768.f;            // 2^15: a half-row's probabilities summing to less leave the reference
+                                                  // alone (and every one of them fits fp16)
 
 struct PfWsTail {
   float ex[2][2][kTcTile];         // [query tile][half][row]: row maxima, at the end row sums
@@ -677,7 +697,8 @@ __global__ void __launch_bounds__(128) prefill_band_kernel(AttnArgs a, PrefillBa
 }  // namespace
 
 cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, int copy_width, __nv_bfloat16* out,
-                               int out_tokens, int out_width, bool rotate, int zero_tail, cudaStream_t stream) {
+                               int out_tokens, int out_width, bool rotate, int zero_tail, cudaStream_t stream,
+                               bool to_half) {
   if (copy_width == 0 && zero_tail == 0) return cudaSuccess;
   if (copy_width % 128 != 0 || copy_width > width || out_width % 8 != 0) return cudaErrorInvalidValue;
   // enough tokens per block that every thread has four items to overlap
@@ -685,7 +706,7 @@ cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, i
   dim3 grid((out_tokens + block_tokens - 1) / block_tokens, a.batch);
   gather_rows_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(pool), width, copy_width, out, out_tokens,
                                                out_width, a.slots, a.lens, a.geom, rotate ? a.rope : RopeTable(), zero_tail,
-                                               block_tokens, a.status);
+                                               block_tokens, a.status, to_half ? 1 : 0);
   return cudaGetLastError();
 }
 

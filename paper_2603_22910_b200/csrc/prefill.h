@@ -9,12 +9,14 @@ namespace echokv {
 // `width` dims into contiguous rows out[b][token][out_width]; keys are rotated to their positions if `rotate` and
 // a.rope is set.  zero_tail > 0 also writes zeros over the whole rows len .. (next multiple of zero_tail) - 1
 // (launched even when copy_width is 0).
+// to_half: the rows are written as fp16 instead (the value rows of the attention kernel below).
 cudaError_t launch_gather_rows(const AttnArgs& a, const void* pool, int width, int copy_width, __nv_bfloat16* out,
-                               int out_tokens, int out_width, bool rotate, int zero_tail, cudaStream_t stream);
+                               int out_tokens, int out_width, bool rotate, int zero_tail, cudaStream_t stream,
+                               bool to_half = false);
 
 // Eq. 7 for n_q queries per sequence (a.q: [B][n_q][H_q][128] bf16), query i at position len - n_q + i attending the
-// keys n_skip .. its own position - shift (plain causal attention: shift = n_skip = 0), over k_rows / v_rows
-// [B][kv_tokens][kv_width] bf16 (v_rows zeroed from each sequence's length to the next multiple of 128 rows).
+// keys n_skip .. its own position - shift (plain causal attention: shift = n_skip = 0), over k_rows (bf16) and v_rows
+// (fp16), [B][kv_tokens][kv_width] each (v_rows zeroed from each sequence's length to the next multiple of 128 rows).
 // out: fp32 [B][n_q][H_q][128]; lse_out (may be null): fp32 [B][n_q][H_q], log2 of every row's softmax denominator in
 // base-2 score units, -inf for a row that attends nothing (its output is zero).
 // A sequence with fewer than n_q cached tokens gets zeros and the device status EBADLENGTH.

@@ -33,6 +33,7 @@
 #include "recon_tc.h"
 
 #include <cudaTypedefs.h>
+#include <cuda_fp16.h>
 
 #include "ptx_sm100.cuh"
 
@@ -85,6 +86,7 @@ struct PairParams {
   // store_rotate) are written as bf16 to store_out[b][token][store_width] at the head's flat dims
   __nv_bfloat16* store_out;
   int store_tokens, store_width, store_rotate;
+  int store_half;             // the rows are written as fp16 instead of bf16 (value rows of the prefill-shaped call)
 };
 
 template <int G>
@@ -434,10 +436,16 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
                   v_hi[e] = k_hi;
                 }
               }
-              const __nv_bfloat162 a2 = __floats2bfloat162_rn(v_lo[0], v_lo[1]);
-              const __nv_bfloat162 b2 = __floats2bfloat162_rn(v_hi[0], v_hi[1]);
-              pl[j / 2] = *reinterpret_cast<const uint32_t*>(&a2);
-              ph[j / 2] = *reinterpret_cast<const uint32_t*>(&b2);
+              if (p.store_half) {
+                const __half2 a2 = __floats2half2_rn(v_lo[0], v_lo[1]), b2 = __floats2half2_rn(v_hi[0], v_hi[1]);
+                pl[j / 2] = *reinterpret_cast<const uint32_t*>(&a2);
+                ph[j / 2] = *reinterpret_cast<const uint32_t*>(&b2);
+              } else {
+                const __nv_bfloat162 a2 = __floats2bfloat162_rn(v_lo[0], v_lo[1]);
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(v_hi[0], v_hi[1]);
+                pl[j / 2] = *reinterpret_cast<const uint32_t*>(&a2);
+                ph[j / 2] = *reinterpret_cast<const uint32_t*>(&b2);
+              }
             }
             if (live) {
               uint4* d_lo = reinterpret_cast<uint4*>(dst + cb * 16);
@@ -679,7 +687,7 @@ cudaError_t launch_g(const TcLayerMaps& anchor, const CUtensorMap& lk, const CUt
 
 struct StoreRows {
   __nv_bfloat16* out = nullptr;
-  int tokens = 0, width = 0, rotate = 0;
+  int tokens = 0, width = 0, rotate = 0, half = 0;
 };
 
 static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
@@ -718,6 +726,7 @@ static cudaError_t launch_pair_impl(const AttnArgs& a, const ReconArgs& r, const
   p.store_tokens = store.tokens;
   p.store_width = store.width;
   p.store_rotate = store.rotate;
+  p.store_half = store.half;
   p.run_pages = a.geom.page_tokens < kRunTokens ? kRunTokens / a.geom.page_tokens : 1;
   // with m == 0 the local maps are never used; pass the anchor's so the parameters stay valid
   const CUtensorMap& lk = r.m > 0 ? layer.k_grp_page : anchor.k_grp_page;
@@ -772,6 +781,7 @@ cudaError_t launch_recon_pair_store(const AttnArgs& a, const ReconArgs& r, const
   store.tokens = out_tokens;
   store.width = out_width;
   store.rotate = values ? 0 : 1;                 // (keys are rotated only if a.rope is set; values never)
+  store.half = values ? 1 : 0;                   // (value rows are fp16: see the attention kernel that reads them)
   if (!values) return launch_pair_impl(a, r, anchor, layer, sm_count, stream, nullptr, 0, store);
   // the V predictor over the V pools: the same kernel with the V maps in the K places
   auto as_keys = [](const TcLayerMaps& m) {

@@ -65,9 +65,9 @@ cudaError_t launch_recon_pair_key_scores(const AttnArgs& a, const ReconArgs& r, 
                                          const TcLayerMaps& layer, float* scores, int l_cap, int sm_count,
                                          cudaStream_t stream);
 
-// Eq. 3 alone: the predicted dims of every cached token written out as bf16 rows, out[b][token][out_width] at flat
-// dims m .. D-1 (keys: + bias r.bk, rotated to the token's position if a.rope is set; values: the V predictor over
-// the V pools; r.bk is then the V bias or null).  For uses with many queries per sequence, where rebuilding the
+// Eq. 3 alone: the predicted dims of every cached token written out as 16-bit rows, out[b][token][out_width] at flat
+// dims m .. D-1 (keys: bf16, + bias r.bk, rotated to the token's position if a.rope is set; values: fp16, the V
+// predictor over the V pools; r.bk is then the V bias or null).  For uses with many queries per sequence, where rebuilding the
 // cache once and attending it with a standard kernel is cheaper than rebuilding it per query.
 cudaError_t launch_recon_pair_store(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
                                     const TcLayerMaps& layer, bool values, __nv_bfloat16* out, int out_tokens,

@@ -112,5 +112,5 @@ def test_prefill_call_config2_full_size_sampled():
     ctx.close()
     del st
     torch.cuda.empty_cache()
-    # the tolerance of the prefill-shaped call (it rounds the rebuilt rows to bf16): tests/test_gpu_prefill.py
-    assert worst <= 4e-2 and rel <= 5e-3, (worst, rel)
+    # (the tolerance of the decode calls)
+    assert worst <= 2e-2 and rel <= 5e-3, (worst, rel)

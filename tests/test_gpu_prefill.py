@@ -12,10 +12,10 @@ pytestmark = pytest.mark.gpu
 
 THETA = 10000.0
 
-# This call materialises the rebuilt K~ / V~ rows in bf16 (the decode calls keep them in fp32): a query that attends a
-# handful of tokens returns nearly a single V~ row, so the bf16 rounding of that row (|v| 2^-9, |v| up to ~5 here) and
-# of the keys behind its few probabilities shows unaveraged in the maximum error.  rel-L2 as for the decode calls.
-TOL_PREFILL = dict(max_abs=4e-2, rel_l2=5e-3)
+# This call materialises the rebuilt K~ / V~ rows in 16 bits (the decode calls keep them in fp32).  A query that attends
+# a handful of tokens returns nearly a single V~ row, so the value rows (and the probabilities) are fp16, whose rounding
+# of |v| up to ~5 stays near 1e-3; the tolerance is that of the decode calls.
+TOL_PREFILL = dict(max_abs=2e-2, rel_l2=5e-3)
 
 
 def assert_parity(out, ref, dtype, what=""):
