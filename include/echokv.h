@@ -178,7 +178,11 @@ int echokv_compress_layer(echokv_ctx* ctx, int layer, const void* k_full, const 
  * layer's retained dims.  Called on an anchor layer it is the same as echokv_full_attention.
  * Uses the workspace; calls on one context must not overlap on the device.
  * A length < 1 or beyond max_pages_per_seq * page_tokens -> device status EBADLENGTH and
- * zeros for that sequence.  Errors: EINVAL, ECAPACITY, ENOWEIGHTS, ENOTABLE, ECUDA. */
+ * zeros for that sequence.  A page id outside the pool (a caller's error) -> device status EBADPAGE; nothing is
+ * read through it and every other sequence of the call is unaffected, but the output of the sequence it belongs
+ * to is unspecified: the stored-head kernels leave the page's tokens out, the tensor-core kernels find whatever
+ * rows their staging memory held in their place.
+ * Errors: EINVAL, ECAPACITY, ENOWEIGHTS, ENOTABLE, ECUDA. */
 int echokv_decode_attention(echokv_ctx* ctx, int layer, const void* q, float* out,
                             const int32_t* dev_seq_slots, const int32_t* dev_seq_lens, int B,
                             void* stream);
@@ -231,20 +235,6 @@ int echokv_layer_step_host(echokv_ctx* ctx, int layer, const void* q_host, const
 /* Read and clear the device status word (synchronises the device).  *host_out receives
  * ECHOKV_OK or the first device-side error (ETIMEOUT, EBADPAGE, EBADLENGTH). */
 int echokv_get_device_status(echokv_ctx* ctx, int32_t* host_out);
-
-/* Number of kernels the library has launched on this context since creation. */
-int64_t echokv_launch_count(const echokv_ctx* ctx);
-
-/* Which kernel family serves compressed layers of this context:
- * 0 = none (no layer is compressed or nothing is dropped), 1 = fp32/bf16 CUDA-core kernel,
- * 2 = bf16 tcgen05 tensor-core kernel, one CTA per SM, 3 = the same on CTA pairs
- * (cta_group::2: two SMs share every operand tile and the accumulators are double-buffered). */
-int echokv_decode_path(const echokv_ctx* ctx);
-
-/* Choose the kernel family for compressed layers: 1 = CUDA-core kernel (always possible),
- * 2 or 3 = tcgen05 kernels (EUNSUPPORTED unless dtype is bf16, head_dim 128).  Contexts start on
- * the fastest family their shape allows.  Meant for tests that check all against the oracle. */
-int echokv_set_decode_path(echokv_ctx* ctx, int path);
 
 /* Sink and recent-window tokens at full precision (Section 4.1, "Implement details": the paper keeps
  * 4 sink tokens and a local window of 128 tokens uncompressed).  With (n_sink, n_window) set, the first
@@ -306,40 +296,11 @@ int echokv_rope_enabled(const echokv_ctx* ctx);
  *    Errors: EINVAL, EUNSUPPORTED, ECAPACITY (workspace too small), ECUDA.
  *  - echokv_set_decode_mode: 0 = explicit reconstruction, 1 = absorbed (EUNSUPPORTED before
  *    echokv_enable_absorbed).  Anchor layers and echokv_full_attention are not affected.
- *  In this mode a page id outside the pool is still reported (EBADPAGE) but the output of that
- *  sequence is unspecified. */
+ *  A page id outside the pool: as for echokv_decode_attention. */
 int echokv_absorbed_workspace_bytes(const echokv_config* cfg, uint64_t* out);
 int echokv_enable_absorbed(echokv_ctx* ctx, void* workspace, uint64_t workspace_bytes);
 int echokv_decode_mode(const echokv_ctx* ctx);
 int echokv_set_decode_mode(echokv_ctx* ctx, int mode);
-
-/* Which kernel serves attention over stored heads (anchor layers, retained heads, the
- * uncompressed mode): 0 = CUDA-core kernel (any supported shape), 1 = TMA + tensor-core kernel
- * (bf16, head_dim 128).  Contexts start on 1 when their shape allows it.
- * echokv_set_stored_path: EINVAL (not 0 or 1), EUNSUPPORTED (1 on a shape it does not take).
- * Meant for tests that check both against the oracle. */
-int echokv_stored_path(const echokv_ctx* ctx);
-int echokv_set_stored_path(echokv_ctx* ctx, int path);
-
-/* Device timing of the dominant kernel of each attention call (the fused reconstruct-attend
- * kernel on compressed layers, the stored-head attention kernel on anchor layers): when enabled,
- * the library records a CUDA event pair around that kernel on the call's stream.
- * echokv_read_kernel_timing synchronises the device, returns the summed duration and the number
- * of timed launches since the last read, and starts over.  Errors: EINVAL, ECUDA. */
-int echokv_set_kernel_timing(echokv_ctx* ctx, int enable);
-int echokv_read_kernel_timing(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
-
-/* The same reading split by kernel: total_ms and n_launches are host arrays of
- * ECHOKV_TIMED_KINDS entries, indexed by ECHOKV_TIMED_STORED (stored-head attention of an
- * anchor / uncompressed layer), ECHOKV_TIMED_RECON (fused reconstruct-attend kernel) and the two
- * streaming kernels of the absorbed mode. */
-enum {
-  ECHOKV_TIMED_STORED = 0, ECHOKV_TIMED_RECON = 1,
-  ECHOKV_TIMED_ABSORB_K = 2,   /* absorbed mode: the pass over the K features (scores)          */
-  ECHOKV_TIMED_ABSORB_V = 3,   /* absorbed mode: the pass over the V features (weighted sums)   */
-  ECHOKV_TIMED_KINDS = 4
-};
-int echokv_read_kernel_timing_by_kind(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
 
 /* Full-cache attention for callers that cannot allocate device memory (the paper has no
  * counterpart to this entry point; it exists for the library's users).
@@ -376,6 +337,62 @@ int echokv_full_attention_noalloc(const echokv_config* cfg, const void* k_pool, 
 
 /* Size in bytes of the fixed scratch array behind echokv_full_attention_noalloc. */
 uint64_t echokv_noalloc_scratch_bytes(void);
+
+/* =====================================================================================================
+ * Diagnostics: switches, counters and probes for tests and benchmarks.  No product call depends on them;
+ * contexts start on the fastest kernels their shape allows.
+ * ===================================================================================================== */
+
+/* Number of kernels the library has launched on this context since creation. */
+int64_t echokv_launch_count(const echokv_ctx* ctx);
+
+/* Which kernel family serves compressed layers of this context:
+ * 0 = none (no layer is compressed or nothing is dropped), 1 = fp32/bf16 CUDA-core kernel,
+ * 2 = bf16 tcgen05 tensor-core kernel, one CTA per SM, 3 = the same on CTA pairs
+ * (cta_group::2: two SMs share every operand tile and the accumulators are double-buffered). */
+int echokv_decode_path(const echokv_ctx* ctx);
+
+/* Choose the kernel family for compressed layers: 1 = CUDA-core kernel (always possible),
+ * 2 or 3 = tcgen05 kernels (EUNSUPPORTED unless dtype is bf16, head_dim 128).  Contexts start on
+ * the fastest family their shape allows.  Meant for tests that check all against the oracle. */
+int echokv_set_decode_path(echokv_ctx* ctx, int path);
+
+/* Which kernel serves attention over stored heads (anchor layers, retained heads, the
+ * uncompressed mode): 0 = CUDA-core kernel (any supported shape), 1 = TMA + tensor-core kernel
+ * (bf16, head_dim 128).  Contexts start on 1 when their shape allows it.
+ * echokv_set_stored_path: EINVAL (not 0 or 1), EUNSUPPORTED (1 on a shape it does not take).
+ * Meant for tests that check both against the oracle. */
+int echokv_stored_path(const echokv_ctx* ctx);
+int echokv_set_stored_path(echokv_ctx* ctx, int path);
+
+/* Device timing of the dominant kernel of each attention call (the fused reconstruct-attend
+ * kernel on compressed layers, the stored-head attention kernel on anchor layers): when enabled,
+ * the library records a CUDA event pair around that kernel on the call's stream.
+ * echokv_read_kernel_timing synchronises the device, returns the summed duration and the number
+ * of timed launches since the last read, and starts over.  Errors: EINVAL, ECUDA. */
+int echokv_set_kernel_timing(echokv_ctx* ctx, int enable);
+int echokv_read_kernel_timing(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
+
+/* The same reading split by kernel: total_ms and n_launches are host arrays of
+ * ECHOKV_TIMED_KINDS entries, indexed by ECHOKV_TIMED_STORED (stored-head attention of an
+ * anchor / uncompressed layer), ECHOKV_TIMED_RECON (fused reconstruct-attend kernel) and the two
+ * streaming kernels of the absorbed mode. */
+enum {
+  ECHOKV_TIMED_STORED = 0, ECHOKV_TIMED_RECON = 1,
+  ECHOKV_TIMED_ABSORB_K = 2,   /* absorbed mode: the pass over the K features (scores)          */
+  ECHOKV_TIMED_ABSORB_V = 3,   /* absorbed mode: the pass over the V features (weighted sums)   */
+  ECHOKV_TIMED_KINDS = 4
+};
+int echokv_read_kernel_timing_by_kind(echokv_ctx* ctx, double* total_ms, int64_t* n_launches);
+
+/* The give-up path of the kernels' bounded waits, exercised without a fault: enqueues one small block that waits,
+ * with the same routine the kernels use and a limit of limit_cycles SM cycles (1 .. 2e9), on a barrier nothing ever
+ * arrives on.  The waiting warp raises ECHOKV_ETIMEOUT in the device status word (read it with
+ * echokv_get_device_status) and a flag that releases the block's other waiting warp, as a kernel's other roles are
+ * released; the block issues no copy and allocates no tensor memory, so nothing is pending when it returns and the
+ * context stays usable.  dev_left_by: device pointer to int32[2], how each of the two warps left (1 = gave up or was
+ * released by the flag, 0 = its barrier completed, which cannot happen).  Errors: EINVAL, ECUDA. */
+int echokv_diag_bounded_wait(echokv_ctx* ctx, int64_t limit_cycles, int32_t* dev_left_by, void* stream);
 
 /* Static, human-readable name of a status code. */
 const char* echokv_strerror(int status);

@@ -82,6 +82,7 @@ EXPORTS = {
     "echokv_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "echokv_read_kernel_timing": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "echokv_read_kernel_timing_by_kind": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "echokv_diag_bounded_wait": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "echokv_full_attention_noalloc": (C.c_int, [C.POINTER(echokv_config), C.c_void_p, C.c_void_p, C.c_void_p,
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                                 C.c_void_p, C.c_void_p]),
@@ -348,6 +349,13 @@ class Context:
         ms, n = (C.c_double * 4)(), (C.c_int64 * 4)()
         _check(lib().echokv_read_kernel_timing_by_kind(self.handle, ms, n), "echokv_read_kernel_timing_by_kind")
         return {"stored": (ms[0], n[0]), "recon": (ms[1], n[1]), "absorb_k": (ms[2], n[2]), "absorb_v": (ms[3], n[3])}
+
+    def diag_bounded_wait(self, limit_cycles: int, stream=None):
+        """Run the bounded-wait probe; returns the device tensor int32[2] saying how its two warps left."""
+        left = self.torch.zeros(2, dtype=self.torch.int32, device=self.device)
+        _check(lib().echokv_diag_bounded_wait(self.handle, int(limit_cycles), left.data_ptr(), _stream_handle(stream)),
+               "echokv_diag_bounded_wait")
+        return left
 
     def _out(self, q):
         return self.torch.empty(q.shape, dtype=self.torch.float32, device=self.device)

@@ -899,6 +899,15 @@ int echokv_read_kernel_timing(echokv_ctx* c, double* total_ms, int64_t* n_launch
   return ECHOKV_OK;
 }
 
+int echokv_diag_bounded_wait(echokv_ctx* c, int64_t limit_cycles, int32_t* dev_left_by, void* stream) {
+  if (!c || !dev_left_by || limit_cycles < 1 || limit_cycles > 2000000000ll) return ECHOKV_EINVAL;
+  if (launch_bounded_wait_probe(status_ptr(c), limit_cycles, dev_left_by, static_cast<cudaStream_t>(stream)) !=
+      cudaSuccess)
+    return ECHOKV_ECUDA;
+  c->launches += 1;
+  return ECHOKV_OK;
+}
+
 int64_t echokv_launch_count(const echokv_ctx* c) { return c ? c->launches : 0; }
 
 int echokv_decode_path(const echokv_ctx* c) { return c ? c->path : 0; }

@@ -35,7 +35,7 @@
 #include <cudaTypedefs.h>
 #include <cuda_fp16.h>
 
-#include "ptx_sm100.cuh"
+#include "recon_common.cuh"
 
 namespace echokv {
 
@@ -106,53 +106,10 @@ struct PairSmemTail {
   int abort_flag;
 };
 
-__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-// Barrier over the 256 epilogue threads that also ANDs a flag, so that all of them take the same
-// decision after a bounded wait.
-__device__ __forceinline__ bool epilogue_all(bool ok) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.b32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, 256, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r)
-      : "r"(ok ? 1u : 0u)
-      : "memory");
-  return r != 0;
-}
 
-// K-major bf16 operand, 128-byte rows in the 128-byte swizzle, 8-row groups group_bytes apart
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t group_bytes = 1024) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
-  d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>(group_bytes >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
 // kind::f16: bf16 x bf16 -> fp32, both operands K-major, M = 256 over the pair, N = 256
 constexpr uint32_t kIdescPair = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
 
-struct Item {
-  int b, tile, pair;
-};
-
-template <int G>
-__device__ __forceinline__ Item decode_item(const PairSmemTail<G>& t, int item, int n_pairs, int nb) {
-  Item it;
-  const int tg = item / n_pairs;
-  it.pair = item - tg * n_pairs;
-  int lo = 0, hi = nb;   // largest b with cum_tiles[b] <= tg
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (t.cum_tiles[mid] <= tg) lo = mid; else hi = mid;
-  }
-  it.b = lo;
-  it.tile = tg - t.cum_tiles[lo];
-  return it;
-}
 
 // ROPE: the predicted key rows are rotated to their positions before q . k (Section 3.2: the predictors
 // produce keys prior to the rotary embedding).
@@ -241,7 +198,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
     uint32_t it = 0;
     bool alive = true;
     for (int item = pair_id; item < n_items && alive; item += n_clusters) {
-      const Item w = decode_item<G>(t, item, p.n_pairs, p.nb);
+      const ReconItem w = decode_recon_item(t.cum_tiles, item, p.n_pairs, p.nb);
       const int b = p.b0 + w.b;
       const int slot = p.slots ? p.slots[b] : b;
       const int len = p.lens[b];
@@ -372,7 +329,7 @@ recon_pair_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
     uint32_t n = 0;
     bool alive = true;
     for (int item = pair_id; item < n_items && alive; item += n_clusters, ++n) {
-      const Item w = decode_item<G>(t, item, p.n_pairs, p.nb);
+      const ReconItem w = decode_recon_item(t.cum_tiles, item, p.n_pairs, p.nb);
       const int b = p.b0 + w.b;
       const int len = p.lens[b];
       const int n_valid = min(kTileTokens, len - w.tile * kTileTokens);   // cached tokens in the tile

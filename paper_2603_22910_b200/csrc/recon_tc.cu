@@ -27,7 +27,7 @@
 
 #include <cudaTypedefs.h>
 
-#include "ptx_sm100.cuh"
+#include "recon_common.cuh"
 
 namespace echokv {
 
@@ -85,55 +85,10 @@ struct TcSmemTail {
   int abort_flag;
 };
 
-__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-// Barrier over the 256 epilogue threads that also ANDs a flag, so that all of them take the same
-// decision after a bounded wait (a warp that left alone would strand the others at a barrier).
-__device__ __forceinline__ bool epilogue_all(bool ok) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.b32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, 256, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r)
-      : "r"(ok ? 1u : 0u)
-      : "memory");
-  return r != 0;
-}
 
-// Shared-memory matrix descriptor of a K-major bf16 operand whose rows are 128 bytes (64
-// features) in the 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);          // start address
-  d |= static_cast<uint64_t>(1) << 16;                              // leading byte offset (unused here)
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;                      // stride between 8-row groups
-  d |= static_cast<uint64_t>(1) << 46;                              // descriptor version of sm_100
-  d |= static_cast<uint64_t>(2) << 61;                              // 128-byte swizzle
-  return d;
-}
 // kind::f16 instruction: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
 
-struct Item {
-  int b, tile, pair;
-};
-
-// item -> (sequence, token tile, head pair); tiles of all sequences are numbered consecutively
-template <int G>
-__device__ __forceinline__ Item decode_item(const TcSmemTail<G>& t, int item, int n_pairs, int nb) {
-  Item it;
-  const int tg = item / n_pairs;
-  it.pair = item - tg * n_pairs;
-  int lo = 0, hi = nb;   // largest b with cum_tiles[b] <= tg
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (t.cum_tiles[mid] <= tg) lo = mid; else hi = mid;
-  }
-  it.b = lo;
-  it.tile = tg - t.cum_tiles[lo];
-  return it;
-}
 
 // ROPE: the predicted key rows are rotated to their positions before q . k (Section 3.2: the predictors
 // produce keys prior to the rotary embedding).
@@ -208,7 +163,7 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
     for (int s = 0; s < kStages; ++s) issued[s] = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
-      const Item w = decode_item<G>(t, item, p.n_pairs, p.nb);
+      const ReconItem w = decode_recon_item(t.cum_tiles, item, p.n_pairs, p.nb);
       const int b = p.b0 + w.b;
       const int slot = p.slots ? p.slots[b] : b;
       const int len = p.lens[b];
@@ -334,7 +289,7 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
     uint32_t round = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
-      const Item w = decode_item<G>(t, item, p.n_pairs, p.nb);
+      const ReconItem w = decode_recon_item(t.cum_tiles, item, p.n_pairs, p.nb);
       const int b = p.b0 + w.b;
       const int len = p.lens[b];
       const int n_valid = min(kTileTokens, len - w.tile * kTileTokens);
@@ -566,6 +521,36 @@ cudaError_t launch_g(const CUtensorMap& ak, const CUtensorMap& av, const CUtenso
 }
 
 }  // namespace
+
+// Exercises the give-up path of the kernels' bounded waits without putting anything in flight: one warp waits, with
+// the same routine and a short limit, on a barrier that nothing ever arrives on; a second warp, as the kernels'
+// other roles do, waits on a barrier of its own and must leave through the abort flag the first one raises.  No TMA
+// copy is issued and no tensor memory is allocated, so nothing is pending when the block returns.
+__global__ void __launch_bounds__(64) bounded_wait_probe_kernel(int32_t* status, long long limit_cycles, int* left_by) {
+  __shared__ unsigned long long bars[2];
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bars[0]), 1);
+    mbar_init(smem_u32(&bars[1]), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  volatile int* flag = &abort_flag;
+  const int warp = threadIdx.x >> 5;
+  bool ok = true;
+  if ((threadIdx.x & 31) == 0) {
+    // warp 0 runs out of time; warp 1 has a limit a thousand times longer and must be released by the flag
+    ok = mbar_wait(smem_u32(&bars[warp]), 0, flag, status, warp == 0 ? limit_cycles : limit_cycles * 1000);
+    left_by[warp] = ok ? 0 : (abort_flag ? 1 : 2);
+  }
+  __syncthreads();
+}
+
+cudaError_t launch_bounded_wait_probe(int32_t* status, long long limit_cycles, int* left_by, cudaStream_t stream) {
+  bounded_wait_probe_kernel<<<1, 64, 0, stream>>>(status, limit_cycles, left_by);
+  return cudaGetLastError();
+}
 
 bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m) {
   if (dtype != ECHOKV_BF16 || head_dim != 128) return false;

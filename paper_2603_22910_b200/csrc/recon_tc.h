@@ -42,6 +42,11 @@ cudaError_t encode_tiled_bf16(CUtensorMap* map, const void* base, int rank, cons
 
 bool tc_shape_supported(int dtype, int head_dim, int page_tokens, int D, int m);
 
+// One small block that waits, with the kernels' own bounded-wait routine and a limit of limit_cycles, on a barrier
+// nothing arrives on: raises ECHOKV_ETIMEOUT in *status and returns.  left_by[2] (device): how its two waiting warps
+// left (1 = gave up / was released by the abort flag).
+cudaError_t launch_bounded_wait_probe(int32_t* status, long long limit_cycles, int* left_by, cudaStream_t stream);
+
 // k_width / v_width: row widths of the two pools (they differ where a layer keeps its keys whole); 0 = no pool
 cudaError_t tc_encode_pool_maps(TcLayerMaps* maps, const void* k_pool, int k_width, const void* v_pool, int v_width,
                                 uint64_t rows, int page_tokens);

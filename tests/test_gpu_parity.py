@@ -207,7 +207,7 @@ def test_bad_length_and_bad_page_are_reported_not_fatal():
     too_long = torch.tensor([100, 10 ** 6], dtype=torch.int32, device=dev)
     case.ctx.decode_attention(1, q, too_long)
     assert case.ctx.device_status() == binding.ECHOKV_EBADLENGTH
-    # a page id outside the pool: reported, the tokens of that page are skipped, no fault
+    # a page id outside the pool: reported, no fault
     saved = case.ctx.block_table.clone()
     case.ctx.block_table[1, 1] = 10 ** 6
     out = case.ctx.decode_attention(1, q, case.seq_lens)
@@ -320,4 +320,48 @@ def test_every_sequence_unusable_gives_zeros_and_a_status():
         out = case.ctx.decode_attention(l, case.q[l].to(dev), bad)
         assert case.ctx.device_status() == binding.ECHOKV_EBADLENGTH
         assert np.all(out.cpu().numpy() == 0.0)
+    case.close()
+
+
+def test_a_bounded_wait_that_runs_out_reports_a_timeout_and_leaves_the_context_usable():
+    """The give-up path of the kernels' waits (a limit, a status, an abort flag that releases the other roles),
+    driven by a probe that waits on a barrier nothing arrives on: no fault, no hang, nothing left in flight."""
+    import time
+    w = synth.C2.replace(batch=2, context=300)
+    case = Case(w, lens=[300, 77], layers=[0, 1])
+    ctx = case.ctx
+    before = case.run(1)
+    assert ctx.device_status() == binding.ECHOKV_OK
+    t0 = time.perf_counter()
+    left = ctx.diag_bounded_wait(200000)            # ~0.1 ms of SM cycles
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0
+    assert left.cpu().tolist() == [1, 1]            # the waiting warp gave up; the other one was released by its flag
+    assert ctx.device_status() == binding.ECHOKV_ETIMEOUT
+    assert ctx.device_status() == binding.ECHOKV_OK          # read and cleared
+    np.testing.assert_array_equal(case.run(1), before)       # the context works as before
+    assert ctx.device_status() == binding.ECHOKV_OK
+    assert binding.lib().echokv_diag_bounded_wait(ctx.handle, 0, left.data_ptr(), None) == binding.ECHOKV_EINVAL
+    case.close()
+
+
+@pytest.mark.parametrize("mode", ["explicit", "absorbed"])
+def test_a_page_outside_the_pool_is_reported_and_harms_no_other_sequence(mode):
+    """A page id outside the pool is a caller's error: it is reported, nothing is read through it (no fault), and
+    the other sequences of the call come out bit for bit as without it."""
+    w = synth.C2.replace(batch=3, context=200)
+    case = Case(w, lens=[200, 100, 77], layers=[0, 1])
+    ctx = case.ctx
+    if mode == "absorbed":
+        ctx.enable_absorbed()
+    good = case.run(1)
+    saved = ctx.block_table.clone()
+    ctx.block_table[1, 2] = 10 ** 6                     # tokens 32 .. 47 of sequence 1
+    out = case.run(1)
+    assert ctx.device_status() == binding.ECHOKV_EBADPAGE
+    np.testing.assert_array_equal(out[0], good[0])
+    np.testing.assert_array_equal(out[2], good[2])
+    ctx.block_table.copy_(saved)
+    np.testing.assert_array_equal(case.run(1), good)
+    assert ctx.device_status() == binding.ECHOKV_OK
     case.close()
