@@ -395,10 +395,10 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
       const int width = L.anchor ? d.D : d.m;
       if (width == 0 || (!L.anchor && d.save_k)) continue;   // (keys kept whole: no stored-head call on that layer)
       const uint64_t rows = (uint64_t)cfg->n_pages * cfg->page_tokens;
-      if (encode_pool_box_map(&L.stored_k, L.k_pool, width, rows, box_rows) != cudaSuccess ||
-          encode_pool_box_map(&L.stored_v, L.v_pool, width, rows, box_rows) != cudaSuccess ||
-          encode_pool_box_map(&L.stored_k_run, L.k_pool, width, rows, 64) != cudaSuccess ||
-          encode_pool_box_map(&L.stored_v_run, L.v_pool, width, rows, 64) != cudaSuccess) {
+      if (encode_pool_group_map(&L.stored_k, L.k_pool, width, rows, box_rows) != cudaSuccess ||
+          encode_pool_group_map(&L.stored_v, L.v_pool, width, rows, box_rows) != cudaSuccess ||
+          encode_pool_group_map(&L.stored_k_run, L.k_pool, width, rows, 64) != cudaSuccess ||
+          encode_pool_group_map(&L.stored_v_run, L.v_pool, width, rows, 64) != cudaSuccess) {
         delete c;
         return ECHOKV_ECUDA;
       }

@@ -618,6 +618,10 @@ cudaError_t encode_tiled_bf16(CUtensorMap* map, const void* base, int rank, cons
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+cudaError_t encode_pool_group_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows) {
+  return encode_4d_groups(map, pool, rows, width, box_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+}
+
 cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows) {
   return encode_2d(map, pool, rows, width, box_rows, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }

@@ -30,6 +30,11 @@ struct TcLayerMaps {
 // TMA descriptor of a bf16 pool [rows][width]: boxes of box_rows token rows x 64 features, 128-byte swizzle.
 cudaError_t encode_pool_box_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows);
 
+// A bf16 pool [rows][width] seen as [rows / 8][width / 64][8][64] (8-row groups outermost): a box of box_rows rows x
+// two 64-column chunks lands in shared memory as 1 KiB swizzle atoms (8 rows x 64 columns) in the order (group,
+// chunk) -- one copy per page for both chunks of a head or of a stage.  A chunk past the last column reads as zeros.
+cudaError_t encode_pool_group_map(CUtensorMap* map, const void* pool, int width, uint64_t rows, int box_rows);
+
 // The matrix [rows][cols] seen as [cols / 64][rows][64]: boxes of box_chunks x box_rows x 64 land in shared
 // memory as box_chunks consecutive swizzled sub-tiles of box_rows rows.
 cudaError_t encode_chunked_3d_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int box_rows,

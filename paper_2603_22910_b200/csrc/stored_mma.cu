@@ -37,7 +37,14 @@ template <int G, bool ROPE>
 struct StoredStages { static constexpr int value = (ROPE && G >= 4) ? 2 : 3; };
 constexpr int kStageTokens = 64;
 constexpr int kBlockBytes = kStageTokens * 128;      // 64 token rows x 64 features (128 bytes)
-constexpr int kStageBytes = 4 * kBlockBytes;         // K lo, K hi, V lo, V hi
+constexpr int kStageBytes = 4 * kBlockBytes;         // K (both 64-feature halves of the head), then V
+// Inside the K (or V) half of a stage the rows sit as 1 KiB swizzle atoms (8 rows x 64 features) in the order
+// (8-row group, feature half): one TMA box brings both halves of a page's rows (the pools are described to TMA as
+// [group][chunk][row of the group][64]).  Byte offset of 16-byte piece `piece` (0..15 over the head's 128 features)
+// of token row `tok` of the stage:
+__device__ __forceinline__ uint32_t stage_off(int tok, int piece) {
+  return (uint32_t)((tok >> 3) * 2048 + (piece >> 3) * 1024 + (tok & 7) * 128 + (((piece & 7) ^ (tok & 7)) << 4));
+}
 constexpr int kConsumers = 4;
 constexpr int kWarpTokens = kStageTokens / kConsumers;   // every consumer warp takes 16 tokens of each stage
 constexpr int kThreads = 32 * (1 + kConsumers);
@@ -274,13 +281,14 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
           mbar_arrive_expect_tx(full, __popc(ok_mask) * (uint32_t)rpb * 128u);
         }
         __syncwarp();
+        // (lanes of kinds 0 and 2 copy: one box holds both feature halves, K or V)
         if (run) {
-          if (lane < 4)
-            tma_load_2d(stage_base + s * kStageBytes + kind * kBlockBytes, kind < 2 ? &tm_k_run : &tm_v_run,
-                        w.kvh * 128 + (kind & 1) * 64, (int)row, full);
-        } else if (row >= 0) {
-          tma_load_2d(stage_base + s * kStageBytes + kind * kBlockBytes + sub * rpb * 128,
-                      kind < 2 ? &tm_k : &tm_v, w.kvh * 128 + (kind & 1) * 64, (int)row, full);
+          if (lane < 4 && (kind & 1) == 0)
+            tma_load_4d(stage_base + s * kStageBytes + kind * kBlockBytes, kind < 2 ? &tm_k_run : &tm_v_run, 0, 0,
+                        w.kvh * 2, (int)(row >> 3), full);
+        } else if (row >= 0 && (kind & 1) == 0) {
+          tma_load_4d(stage_base + s * kStageBytes + kind * kBlockBytes + sub * rpb * 256,
+                      kind < 2 ? &tm_k : &tm_v, 0, 0, w.kvh * 2, (int)(row >> 3), full);
         }
         issued[s] = it + 1;
       }
@@ -368,7 +376,8 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
             for (int idx = lane; idx < kWarpTokens * 16; idx += 32) {
               const int r = idx >> 4, piece = idx & 15;
               if (!((vmask >> r) & 1u)) {
-                const uint32_t a = sb + (2 + (piece >> 3)) * kBlockBytes + (cw * kWarpTokens + r) * 128 + (piece & 7) * 16;
+                // (every piece of the row is zeroed, so the swizzle does not matter: any order of its 16 pieces)
+                const uint32_t a = sb + 2 * kBlockBytes + stage_off(cw * kWarpTokens + r, piece);
                 asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
               }
             }
@@ -389,10 +398,9 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
               const int c0 = ks * 2 + ((lane >> 3) & 1);
-              const uint32_t off = tok_k * 128 + ((c0 ^ (tok_k & 7)) << 4);
               uint32_t a[4], b[4];
-              ldsm_x4(sb + off, a[0], a[1], a[2], a[3]);
-              ldsm_x4(sb + kBlockBytes + off, b[0], b[1], b[2], b[3]);
+              ldsm_x4(sb + stage_off(tok_k, c0), a[0], a[1], a[2], a[3]);
+              ldsm_x4(sb + stage_off(tok_k, 8 + c0), b[0], b[1], b[2], b[3]);
               uint32_t lo_h[4], lo_r[4], hi_h[4], hi_r[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
@@ -419,7 +427,7 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
           for (int ks = 0; ks < 8; ++ks) {
             const int c0 = (ks & 3) * 2 + ((lane >> 3) & 1);
             uint32_t r0, r1, r2, r3;
-            ldsm_x4(sb + (ks >> 2) * kBlockBytes + tok_k * 128 + ((c0 ^ (tok_k & 7)) << 4), r0, r1, r2, r3);
+            ldsm_x4(sb + stage_off(tok_k, (ks >> 2) * 8 + c0), r0, r1, r2, r3);
             mma_m16n8k16_bf16(sc[0], qa0[ks], 0u, qa2[ks], 0u, r0, r1);
             mma_m16n8k16_bf16(sc[1], qa0[ks], 0u, qa2[ks], 0u, r2, r3);
           }
@@ -467,8 +475,7 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
           for (int dp = 0; dp < 8; ++dp) {
             const int chunk = 2 * dp + (lane >> 4);
             uint32_t r0, r1, r2, r3;
-            ldsm_x4_trans(sb + (2 + (chunk >> 3)) * kBlockBytes + tok_v * 128 + (((chunk & 7) ^ (tok_v & 7)) << 4),
-                          r0, r1, r2, r3);
+            ldsm_x4_trans(sb + 2 * kBlockBytes + stage_off(tok_v, chunk), r0, r1, r2, r3);
             mma_m16n8k16_bf16(o[2 * dp], p_hi[0], p_lo[0], p_hi[1], p_lo[1], r0, r1);
             mma_m16n8k16_bf16(o[2 * dp + 1], p_hi[0], p_lo[0], p_hi[1], p_lo[1], r2, r3);
           }
