@@ -51,24 +51,24 @@ __device__ __forceinline__ bool epi_all(bool ok) {
   return r != 0;
 }
 
-// K-major bf16 operand: 128-byte rows in the 128-byte swizzle, 8-row groups 1024 bytes apart
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t smem_addr) {
+// K-major bf16 operand: 128-byte rows in the 128-byte swizzle, 8-row groups group_bytes apart
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t smem_addr, uint32_t group_bytes = 1024) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
   d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(group_bytes >> 4) << 32;
   d |= static_cast<uint64_t>(1) << 46;
   d |= static_cast<uint64_t>(2) << 61;
   return d;
 }
 // M-major bf16 operand made of [K rows][64 M-elements] tiles in the 128-byte swizzle (what a TMA box
 // of token rows x 64 features is when tokens are the contraction index): 8-row groups along K are
-// 1024 bytes apart, successive 64-element blocks along M are `block_bytes` apart
-__device__ __forceinline__ uint64_t desc_mmajor(uint32_t smem_addr, uint32_t block_bytes) {
+// group_bytes apart, successive 64-element blocks along M are `block_bytes` apart
+__device__ __forceinline__ uint64_t desc_mmajor(uint32_t smem_addr, uint32_t block_bytes, uint32_t group_bytes = 1024) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
   d |= static_cast<uint64_t>(block_bytes >> 4) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(group_bytes >> 4) << 32;
   d |= static_cast<uint64_t>(1) << 46;
   d |= static_cast<uint64_t>(2) << 61;
   return d;
@@ -190,7 +190,6 @@ struct StreamParams {
   int d_in;
   int range_tokens;             // pv kernel: tokens per range
   int n_slices;                 // pv kernel: 256-feature slices
-  int v_tile_ok;                // pv kernel: the 4-chunk V maps exist (bit 0: anchor pool, bit 1: local pool)
   int n_sink, n_window;         // scores kernel: sink / recent-window tokens are left to the side kernel
 };
 
@@ -364,18 +363,18 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
         const int n_chunks = min(2, p.kc_total - kc0);
         const bool from_anchor = kc0 < p.kc_anchor;
         const int kx0 = from_anchor ? kc0 : kc0 - p.kc_anchor;
-        // (the absorbed-query box always brings two chunks: past the last one it is filled with zeros)
-        if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)n_chunks * ps.n_valid * page_bytes + 2u * q_chunk_bytes);
+        // (every box brings two chunks -- of the token rows as (8-row group, chunk) swizzle atoms, one copy per page
+        // for both -- and so does the absorbed-query box: past the last chunk they are filled with zeros)
+        if (lane == 0) mbar_arrive_expect_tx(full, 2u * ps.n_valid * page_bytes + 2u * q_chunk_bytes);
         __syncwarp();
         const uint32_t x_dst = stage_base + s * p.stage_bytes;
-        if (ps.all_run && n_chunks == 2) {
+        if (ps.all_run) {
           if (lane == 0)
-            tma_load_3d(x_dst, from_anchor ? &tm_anchor_128 : &tm_local_128, 0, ps.row, kx0, full);
+            tma_load_4d(x_dst, from_anchor ? &tm_anchor_128 : &tm_local_128, 0, 0, kx0, ps.row >> 3, full);
         } else if (ps.row >= 0 && !ps.run_member) {
           const CUtensorMap* m = ps.run_lead ? (from_anchor ? &tm_anchor_run : &tm_local_run)
                                              : (from_anchor ? &tm_anchor : &tm_local);
-          for (int j = 0; j < n_chunks; ++j)
-            tma_load_2d(x_dst + j * kScoreXBytes + lane * page_bytes, m, (kx0 + j) * kChunk, ps.row, full);
+          tma_load_4d(x_dst + lane * 2 * page_bytes, m, 0, 0, kx0, ps.row >> 3, full);
         }
         if (lane == 16) tma_load_3d(x_dst + 2 * kScoreXBytes, &tm_q2, 0, b * p.nh2, kc0, full);
       }
@@ -398,7 +397,7 @@ absorb_scores_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid
           const uint32_t x_addr = stage_base + s * p.stage_bytes;
           const int n_chunks = min(2, p.kc_total - step * 2);
           for (int j = 0; j < n_chunks; ++j) {
-            const uint64_t a_desc = desc_kmajor(x_addr + j * kScoreXBytes);
+            const uint64_t a_desc = desc_kmajor(x_addr + j * 1024, 2048);     // groups of one chunk: 2 KiB apart
             const uint64_t b_desc = desc_kmajor(x_addr + 2 * kScoreXBytes + j * q_chunk_bytes);
 #pragma unroll
             for (int k16 = 0; k16 < 4; ++k16)
@@ -527,7 +526,6 @@ constexpr int kPvVBytes = 4 * kPvTileBytes;          // four chunks
 __global__ void __launch_bounds__(kThreads, 1)
 absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_constant__ CUtensorMap tm_local,
                  const __grid_constant__ CUtensorMap tm_anchor_run, const __grid_constant__ CUtensorMap tm_local_run,
-                 const __grid_constant__ CUtensorMap tm_anchor_4, const __grid_constant__ CUtensorMap tm_local_4,
                  const __grid_constant__ CUtensorMap tm_p2, const StreamParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
@@ -576,7 +574,6 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
     bool alive = true;
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       const Work w = decode(item);
-      const bool one_pool = w.kc0 + w.n_chunks <= p.kc_anchor || w.kc0 >= p.kc_anchor;
       // block-table entries are requested one own stage (two stages) ahead of their use
       const int first = ((it & 1u) == mine) ? 0 : 1;
       int raw_next = first < w.n_steps
@@ -595,22 +592,24 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
         if (!ok) { alive = false; break; }
         const int t0 = w.t_begin + step * kPvTokens;
         const PageSet ps = make_page_set(p, raw, w.len, t0, boxes, box_tokens, lane);
-        if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)w.n_chunks * ps.n_valid * page_bytes + p_tile_bytes);
+        // The value rows of a stage are two 16 KiB halves (features 0-127 and 128-255 of the slice), each laid out
+        // as (8-token group, chunk) swizzle atoms: one copy per page brings both chunks of a half (a chunk past the
+        // end of the pool rows reads as zeros)
+        const int n_mt = (w.n_chunks + 1) / 2;
+        if (lane == 0) mbar_arrive_expect_tx(full, 2u * (uint32_t)n_mt * ps.n_valid * page_bytes + p_tile_bytes);
         __syncwarp();
         const uint32_t v_dst = stage_base + s * p.stage_bytes;
-        if (ps.all_run && w.n_chunks == 4 && one_pool && (p.v_tile_ok & (w.from_anchor ? 1 : 2))) {
-          if (lane == 0)
-            tma_load_3d(v_dst, w.from_anchor ? &tm_anchor_4 : &tm_local_4, 0, ps.row,
-                        w.from_anchor ? w.kc0 : w.kc0 - p.kc_anchor, full);
-        } else if (ps.row >= 0 && !ps.run_member) {
-          for (int c = 0; c < w.n_chunks; ++c) {
-            const int kc = w.kc0 + c;
-            const bool fa = kc < p.kc_anchor;
+        for (int mt = 0; mt < n_mt; ++mt) {
+          const int kc = w.kc0 + 2 * mt;                 // (a pair of chunks never straddles the two pools: D / 64 is even)
+          const bool fa = kc < p.kc_anchor;
+          const int kx = fa ? kc : kc - p.kc_anchor;
+          if (ps.all_run) {
+            if (lane == 0) tma_load_4d(v_dst + mt * 2 * kPvTileBytes, fa ? &tm_anchor_run : &tm_local_run, 0, 0, kx, ps.row >> 3, full);
+          } else if (ps.row >= 0 && !ps.run_member) {
             // (pages of 64 tokens or more: the 64-row maps are the box of one stage)
             const bool tall = ps.run_lead || p.page_tokens >= kPvTokens;
             const CUtensorMap* m = tall ? (fa ? &tm_anchor_run : &tm_local_run) : (fa ? &tm_anchor : &tm_local);
-            tma_load_2d(v_dst + c * kPvTileBytes + lane * page_bytes, m, (fa ? kc : kc - p.kc_anchor) * kChunk, ps.row,
-                        full);
+            tma_load_4d(v_dst + mt * 2 * kPvTileBytes + lane * 2 * page_bytes, m, 0, 0, kx, ps.row >> 3, full);
           }
         }
         if (lane == 16) tma_load_2d(v_dst + kPvVBytes, &tm_p2, t0, w.b * p.nh2, full);
@@ -643,12 +642,12 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
           const uint32_t v_addr = stage_base + s * p.stage_bytes;
           const uint64_t b_desc = desc_kmajor(v_addr + kPvVBytes);
           for (int mt = 0; mt < n_mtiles; ++mt) {
-            // A: 128 features (two 64-feature tiles, kPvTileBytes apart) x 16 tokens per MMA, M-major
-            const uint64_t a_desc = desc_mmajor(v_addr + mt * 2 * kPvTileBytes, kPvTileBytes);
+            // A: 128 features (two 64-feature atoms, 1 KiB apart) x 16 tokens per MMA, M-major; 8-token groups 2 KiB apart
+            const uint64_t a_desc = desc_mmajor(v_addr + mt * 2 * kPvTileBytes, 1024, 2048);
             const uint32_t d_tmem = tmem + buf * 256u + mt * (uint32_t)p.nh2;
 #pragma unroll
-            for (int k16 = 0; k16 < 4; ++k16)   // 16 tokens = 2048 bytes of A rows, 32 bytes along B's K
-              tc_mma_bf16(d_tmem, a_desc + 128 * k16, b_desc + 2 * k16, p.idesc, (step > 0 || k16 > 0) ? 1u : 0u);
+            for (int k16 = 0; k16 < 4; ++k16)   // 16 tokens = two groups = 4096 bytes of A, 32 bytes along B's K
+              tc_mma_bf16(d_tmem, a_desc + 256 * k16, b_desc + 2 * k16, p.idesc, (step > 0 || k16 > 0) ? 1u : 0u);
           }
           tc_commit(smem_u32(&t.empty_bar[s]));
         }
@@ -673,7 +672,9 @@ absorb_pv_kernel(const __grid_constant__ CUtensorMap tm_anchor, const __grid_con
         const int n_rows = kPvTokens - n_tok;                 // rows n_tok .. 63 of every chunk tile
         for (int idx = lane; idx < w.n_chunks * n_rows * 8; idx += 32) {
           const int piece = idx & 7, rr = (idx >> 3) % n_rows, c = (idx >> 3) / n_rows;
-          const uint32_t a = v_addr + c * kPvTileBytes + (n_tok + rr) * kRowBytes + piece * 16;
+          const int tr = n_tok + rr;            // (all eight pieces of the row are zeroed: the swizzle does not matter)
+          const uint32_t a = v_addr + (c >> 1) * 2 * kPvTileBytes + (tr >> 3) * 2048 + (c & 1) * 1024 + (tr & 7) * kRowBytes +
+                             piece * 16;
           asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
         }
         fence_proxy_async_smem();
@@ -1013,7 +1014,7 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     p.n_stages = (int)(kSmemBudget / p.stage_bytes);
     if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;
     p.idesc = make_idesc(lay.nh2, false);
-    p.range_tokens = 0; p.n_slices = 0; p.v_tile_ok = 0;
+    p.range_tokens = 0; p.n_slices = 0;
     const size_t smem = 1024 + (size_t)p.n_stages * p.stage_bytes + sizeof(StreamSmemTail);
     if ((e = cudaFuncSetAttribute(absorb_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
         cudaSuccess)
@@ -1021,8 +1022,8 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     const long long max_items = (long long)a.batch * ((capacity + kScoreTokens - 1) / kScoreTokens);
     const int grid = (int)(max_items < sm_count ? max_items : sm_count);
     if (ev) cudaEventRecord(ev[0], stream);
-    absorb_scores_kernel<<<grid, kThreads, smem, stream>>>(anchor.k_pool, k_loc.k_pool, anchor.k_pool_run,
-                                                           k_loc.k_pool_run, anchor.k_pool_run128, k_loc.k_pool_run128,
+    absorb_scores_kernel<<<grid, kThreads, smem, stream>>>(anchor.k_grp_page, k_loc.k_grp_page, anchor.k_grp_64,
+                                                           k_loc.k_grp_64, anchor.k_grp_128, k_loc.k_grp_128,
                                                            maps.q2, p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (ev) cudaEventRecord(ev[1], stream);
@@ -1058,19 +1059,15 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     p.n_stages = (int)(kSmemBudget / p.stage_bytes);
     if (p.n_stages > kMaxStages) p.n_stages = kMaxStages;
     p.idesc = make_idesc(lay.nh2, true);
-    // the 4-chunk maps exist for pools at least 256 dims wide (bit 0: anchor pool, bit 1: this layer's pool)
-    p.v_tile_ok = (r.D >= 256 ? 1 : 0) | (r.m >= 256 ? 2 : 0);
     const size_t smem = 1024 + (size_t)p.n_stages * p.stage_bytes + sizeof(StreamSmemTail);
     if ((e = cudaFuncSetAttribute(absorb_pv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
         cudaSuccess)
       return e;
     const long long max_items = (long long)a.batch * ((capacity + range_tokens - 1) / range_tokens) * p.n_slices;
     const int grid = (int)(max_items < sm_count ? max_items : sm_count);
-    const CUtensorMap& a4 = (p.v_tile_ok & 1) ? anchor.v_pool_tok64x4 : anchor.v_pool_run;
-    const CUtensorMap& l4 = (p.v_tile_ok & 2) ? loc.v_pool_tok64x4 : a4;
     if (ev) cudaEventRecord(ev[2], stream);
-    absorb_pv_kernel<<<grid, kThreads, smem, stream>>>(anchor.v_pool, loc.v_pool, anchor.v_pool_run, loc.v_pool_run, a4,
-                                                       l4, maps.p2, p);
+    absorb_pv_kernel<<<grid, kThreads, smem, stream>>>(anchor.v_grp_page, loc.v_grp_page, anchor.v_grp_64, loc.v_grp_64,
+                                                       maps.p2, p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (ev) cudaEventRecord(ev[3], stream);
   }
