@@ -889,7 +889,7 @@ def roofline_of(run, args, timing, ms_region, peaks, peaks_kind):
                     "frac": achieved_tf / burst_tf, "frac_of_burst_peak": achieved_tf / burst_tf,
                     "frac_of_sustained_peak": achieved_tf / sustained_tf, "peak_sustained": sustained_tf,
                     "traffic": traffic_of(args, args.workload or HEADLINE),
-                    "kernel": {3: "recon_pair_kernel", 2: "recon_tc_kernel"}.get(ctx.decode_path(), "recon_simt_kernel"),
+                    "kernel": {4: "recon_quad_kernel", 3: "recon_pair_kernel", 2: "recon_tc_kernel"}.get(ctx.decode_path(), "recon_simt_kernel"),
                     "kernel_ms": k_ms, "kernel_launches": recon_n,
                     "share_of_step": recon_ms / ms_region,
                     "peak_source": tensor_source,
@@ -1249,7 +1249,7 @@ def main():
                          "sampled (default 2 for the whole record, 0 with --workload)")
     ap.add_argument("--stored-path", type=int, default=None, choices=[0, 1],
                     help="kernel for stored heads: 0 CUDA-core, 1 TMA + tensor-core (default: the library's choice)")
-    ap.add_argument("--decode-path", type=int, default=None, choices=[1, 2, 3],
+    ap.add_argument("--decode-path", type=int, default=None, choices=[1, 2, 3, 4],
                     help="kernel family for compressed layers (default: the library's choice)")
     ap.add_argument("--decode-mode", default="explicit", choices=["explicit", "absorbed"],
                     help="explicit: reconstruct-then-attend as the paper states it (the headline); absorbed: the "

@@ -349,12 +349,14 @@ int64_t echokv_launch_count(const echokv_ctx* ctx);
 /* Which kernel family serves compressed layers of this context:
  * 0 = none (no layer is compressed or nothing is dropped), 1 = fp32/bf16 CUDA-core kernel,
  * 2 = bf16 tcgen05 tensor-core kernel, one CTA per SM, 3 = the same on CTA pairs
- * (cta_group::2: two SMs share every operand tile and the accumulators are double-buffered). */
+ * (cta_group::2: two SMs share every operand tile and the accumulators are double-buffered),
+ * 4 = CTA pairs with four dropped heads per work item (a token tile staged once per four heads). */
 int echokv_decode_path(const echokv_ctx* ctx);
 
 /* Choose the kernel family for compressed layers: 1 = CUDA-core kernel (always possible),
- * 2 or 3 = tcgen05 kernels (EUNSUPPORTED unless dtype is bf16, head_dim 128).  Contexts start on
- * the fastest family their shape allows.  Meant for tests that check all against the oracle. */
+ * 2, 3 or 4 = tcgen05 kernels (EUNSUPPORTED unless dtype is bf16, head_dim 128; 4 also needs at most two query
+ * heads per KV head).  Contexts start on the fastest family their shape allows.  Meant for tests that check all
+ * against the oracle. */
 int echokv_set_decode_path(echokv_ctx* ctx, int path);
 
 /* Which kernel serves attention over stored heads (anchor layers, retained heads, the

@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libechokv.so")
-SOURCES = ["echokv_host.cu", "simt_kernels.cu", "stored_mma.cu", "recon_tc.cu", "recon_pair.cu", "absorbed.cu", "prefill.cu", "noalloc.cu"]
+SOURCES = ["echokv_host.cu", "simt_kernels.cu", "stored_mma.cu", "recon_tc.cu", "recon_pair.cu", "recon_quad.cu", "absorbed.cu", "prefill.cu", "noalloc.cu"]
 HEADERS = ["common.cuh", "kernels.h", "recon_tc.h", "recon_common.cuh", "stored_mma.h", "absorbed.h", "prefill.h", "ptx_sm100.cuh", os.path.join("..", "..", "include", "echokv.h")]
 
 

@@ -370,10 +370,16 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
   else if (!c->tc_capable) c->path = 1;
   else {
     // Long contractions (many 64-feature chunks per phase, few query heads per KV head) hide the
-    // epilogue by themselves and run best one CTA per SM; short ones need the CTA-pair kernel's
-    // double-buffered accumulators.
+    // epilogue by themselves and run best with all of tensor memory given to one phase; short ones need the
+    // CTA-pair kernel's double-buffered accumulators.  Of the two kernels for long contractions the one-CTA kernel
+    // is the faster while the pages of a tile follow one another in the pool (fewer, taller TMA boxes), but with
+    // small pages in no particular order -- what a paged pool becomes in service -- it is bound by the number of
+    // copies per stage; the four-heads-per-pair kernel needs half as many and is indifferent to the order
+    // (measured at the 7B layer shape, 16-token pages: in order 2.08 against 2.28 ms, random order 2.34-2.42
+    // against 2.28 ms).  So small pages go to the latter.
     const int chunks = d.d_in / 64;
-    c->path = chunks <= 12 * d.g ? 3 : 2;
+    if (chunks <= 12 * d.g) c->path = 3;
+    else c->path = (recon_quad_supported(d.g) && cfg->page_tokens <= 32) ? 4 : 2;
   }
   if (c->tc_capable) {
     // tensor maps of every pool (the predictors' maps follow in echokv_set_weights)
@@ -455,8 +461,8 @@ int echokv_set_decode_path(echokv_ctx* c, int path) {
   if (!c) return ECHOKV_EINVAL;
   if (c->path == 0) return path == 0 ? ECHOKV_OK : ECHOKV_EINVAL;
   if (path == 1) { c->path = 1; return ECHOKV_OK; }
-  if (path == 2 || path == 3) {
-    if (!c->tc_capable) return ECHOKV_EUNSUPPORTED;
+  if (path == 2 || path == 3 || path == 4) {
+    if (!c->tc_capable || (path == 4 && !recon_quad_supported(c->d.g))) return ECHOKV_EUNSUPPORTED;
     c->path = path;
     return ECHOKV_OK;
   }
@@ -785,7 +791,9 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   cudaError_t e;
   {
     ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
-    if (c->path == 3) {
+    if (c->path == 4) {
+      e = launch_recon_quad(a, ra, A.tc, L.tc, c->sm_count, s);
+    } else if (c->path == 3) {
       e = launch_recon_pair(a, ra, A.tc, L.tc, c->sm_count, s);
     } else if (c->path == 2) {
       e = launch_recon_tc(a, ra, A.tc, L.tc, c->sm_count, s);

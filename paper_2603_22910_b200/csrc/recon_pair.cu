@@ -745,7 +745,7 @@ cudaError_t launch_recon_pair_store(const AttnArgs& a, const ReconArgs& r, const
     TcLayerMaps t = m;
     t.k_pool = m.v_pool; t.k_pool_run = m.v_pool_run; t.k_pool_run128 = m.v_pool_run128;
     t.k_grp_page = m.v_grp_page; t.k_grp_64 = m.v_grp_64; t.k_grp_128 = m.v_grp_128;
-    t.wk = m.wv; t.wk_half = m.wv_half;
+    t.wk = m.wv; t.wk_half = m.wv_half; t.wk_head = m.wv_head;
     return t;
   };
   const TcLayerMaps av = as_keys(anchor), lv = as_keys(layer);

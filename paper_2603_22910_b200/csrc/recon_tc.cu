@@ -664,10 +664,14 @@ cudaError_t tc_encode_weight_maps(TcLayerMaps* maps, const void* Wk, const void*
     if (e != cudaSuccess) return e;
     e = encode_3d_chunks(&maps->wk_half, Wk, d_drop, d_in, kWRows / 2, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     if (e != cudaSuccess) return e;
+    e = encode_2d(&maps->wk_head, Wk, d_drop, d_in, kWRows / 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+    if (e != cudaSuccess) return e;
   }
   e = encode_2d(&maps->wv, Wv, d_drop, d_in, kWRows, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
   if (e != cudaSuccess) return e;
   e = encode_3d_chunks(&maps->wv_half, Wv, d_drop, d_in, kWRows / 2, 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+  if (e != cudaSuccess) return e;
+  e = encode_2d(&maps->wv_head, Wv, d_drop, d_in, kWRows / 2, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
   if (e != cudaSuccess) return e;
   maps->weights_ready = true;
   return cudaSuccess;

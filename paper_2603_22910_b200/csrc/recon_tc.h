@@ -16,6 +16,7 @@ struct TcLayerMaps {
   // 128 rows each: of the pools (128 consecutive token rows) and of the predictors (one head)
   CUtensorMap k_pool_run128, v_pool_run128;
   CUtensorMap wk_half, wv_half;
+  CUtensorMap wk_head, wv_head;         // the predictors in boxes of one head (128 rows) x 64 input features
   // CTA-pair kernel: the pools seen as [8-row group][64-column chunk][row of the group][64], so that ONE box holds
   // two 64-feature chunks of a page (or of a run of 64 / 128 consecutive token rows) and lands in shared memory as
   // 8-row swizzle atoms in the order (group, chunk): the groups of one chunk are then a uniform 2 KiB apart, which a
@@ -65,6 +66,12 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
 
 // The same on pairs of CTAs (cta_group::2, M = 256): one split-K partial per kPairPartTokens tokens.
 cudaError_t launch_recon_pair(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
+                              const TcLayerMaps& layer, int sm_count, cudaStream_t stream);
+
+// The same with four dropped heads per work item (a token tile is staged once per four heads; all of tensor memory
+// belongs to the running phase): for long contractions with one or two query heads per KV head.
+bool recon_quad_supported(int group);
+cudaError_t launch_recon_quad(const AttnArgs& a, const ReconArgs& r, const TcLayerMaps& anchor,
                               const TcLayerMaps& layer, int sm_count, cudaStream_t stream);
 
 // The K half of the same kernel for rotated keys (a.rope must be set): Eq. 3 for the dropped heads' keys, the

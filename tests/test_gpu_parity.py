@@ -54,18 +54,24 @@ SMALL = [
     ("many_tiles_ragged", synth.C2, dict(batch=5, context=2000, random_pages=True), [2000, 129, 128, 1153, 1]),
     ("mha_three_dropped", synth.C1.replace(n_q_heads=4, n_kv_heads=4), dict(n_retained_heads=1, batch=2, context=600),
      [600, 385]),
+    ("gqa2_six_dropped", synth.C2, dict(n_q_heads=16, batch=3, context=900, random_pages=True), [900, 257, 130]),
+    ("mha_m64", synth.C1.replace(n_q_heads=8, n_kv_heads=8), dict(n_retained_heads=0, n_retained_dims=64, batch=2,
+                                                                 context=400, random_pages=True), [400, 33]),
 ]
 
 
 @pytest.mark.parametrize("name,base,over,lens", SMALL, ids=[s[0] for s in SMALL])
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 4])
 def test_small_shapes_against_oracle(name, base, over, lens, path):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1])
     if path >= 2 and case.ctx.decode_path() < 2:
         case.close()
         pytest.skip("shape is served by the CUDA-core kernel only")
-    assert case.ctx.decode_path() in (1, 2, 3)  # a context starts on the family its shape runs fastest on
+    if path == 4 and w.n_q_heads // w.n_kv_heads > 2:
+        case.close()
+        pytest.skip("the four-heads-per-item kernel takes at most two query heads per KV head")
+    assert case.ctx.decode_path() in (1, 2, 3, 4)  # a context starts on the family its shape runs fastest on
     case.ctx.set_decode_path(path)
     check_layers(case, name)
     case.close()
@@ -306,6 +312,12 @@ def test_more_sequences_than_one_launch_indexes():
     for path in (2, 3):
         case.ctx.set_decode_path(path)
         assert_parity(case.run(1), case.oracle(1), w.dtype, "batch 600, path %d" % path)
+    wide = synth.C1.replace(batch=300, context=40, n_kv_heads=8, n_q_heads=8, n_retained_heads=2)
+    lens_w = [int(v) for v in rng.integers(1, 41, size=wide.batch)]
+    case_w = Case(wide, lens=lens_w, layers=[0, 1])
+    case_w.ctx.set_decode_path(4)
+    assert_parity(case_w.run(1), case_w.oracle(1), wide.dtype, "batch 300, path 4")
+    case_w.close()
     assert_parity(case.run(0), case.oracle(0), w.dtype, "batch 600, anchor")
     assert case.ctx.device_status() == binding.ECHOKV_OK
     case.close()
