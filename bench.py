@@ -59,12 +59,15 @@ SUITE = [
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu captures summarised under profiles/; None until a capture of that workload exists.
 NCU_TRAFFIC_BYTES = {
-    "c1": 4 * 619.0e6,        # recon_tc_kernel: B = 2 capture x 4 (tokens)
-    "c2": 8 * 348.2e6,        # recon_pair_kernel: B = 2 capture x 8
-    "c1_full": 4 * 272.9e6,   # attn_stored_mma_kernel: B = 2 capture x 4
-    "c2_full": 8 * 274.5e6,   # attn_stored_mma_kernel: B = 2 capture x 8
-    "c1_absorbed": 4 * 418.8e6,   # absorb_scores_kernel + absorb_pv_kernel (one launch each): B = 2 capture x 4
-    "c2_absorbed": 8 * 354.3e6,   # the same: B = 2 capture x 8
+    # B = 2 captures of the same layer shape, scaled by the tokens of a full launch (traffic grows with the rows read)
+    "c1": 4 * 620.7e6,        # recon_quad_kernel, pages in order: B = 2 capture x 4
+    "c3": 4 * 620.5e6,        # recon_quad_kernel per launch (one compressed layer; 65 536 tokens as C1), 16-token
+                              # pages in a random order: B = 2, L = 8192 capture x 4
+    "c2": 8 * 348.6e6,        # recon_pair_kernel: B = 2 capture x 8
+    "c1_full": 4 * 272.1e6,   # attn_stored_mma_kernel: B = 2 capture x 4
+    "c2_full": 8 * 273.9e6,   # attn_stored_mma_kernel: B = 2 capture x 8
+    "c1_absorbed": 4 * 418.7e6,   # absorb_scores_kernel + absorb_pv_kernel (one launch each): B = 2 capture x 4
+    "c2_absorbed": 8 * 354.7e6,   # the same: B = 2 capture x 8
 }
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
