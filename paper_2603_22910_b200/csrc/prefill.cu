@@ -672,16 +672,30 @@ __global__ void __launch_bounds__(128) prefill_band_kernel(AttnArgs a, PrefillBa
 #pragma unroll
   for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
   const bool from_pool = tid < n_stored_v;
-  for (int idx = 0; idx < n_tok; ++idx) {
-    const bool sink = idx < n_sink_tok;
-    const int t = sink ? idx : win_lo + (idx - n_sink_tok);
+  for (int idx = 0; idx < n_sink_tok; ++idx) {           // sink tokens: pool + side buffers
     float vv;
-    if (!sink) vv = __bfloat162float(v_recent[((size_t)b * n_rows + (t - t_base)) * (size_t)w.D + (size_t)kvh * DH + tid]);
-    else if (from_pool) vv = __bfloat162float(v_pool[pool_row(t) * (size_t)w.m + (size_t)kvh * DH + tid]);
-    else vv = __bfloat162float(v_side[(side_base + t) * (size_t)w.d_drop + (kvh * DH + tid - w.m)]);
+    if (from_pool) vv = __bfloat162float(v_pool[pool_row(idx) * (size_t)w.m + (size_t)kvh * DH + tid]);
+    else vv = __bfloat162float(v_side[(side_base + idx) * (size_t)w.d_drop + (kvh * DH + tid - w.m)]);
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi)
       if (gi < g) o[gi] = fmaf(sc[gi * n_list + idx], vv, o[gi]);
+  }
+  {
+    // window tokens: consecutive rows of v_recent, eight loads in flight at a time
+    const int n_win = n_tok - n_sink_tok;
+    const T* v_row = v_recent + ((size_t)b * n_rows + (win_lo - t_base)) * (size_t)w.D + (size_t)kvh * DH + tid;
+    for (int i0 = 0; i0 < n_win; i0 += 8) {
+      float vv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) vv[u] = i0 + u < n_win ? __bfloat162float(v_row[(size_t)(i0 + u) * w.D]) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int idx = min(n_sink_tok + i0 + u, n_tok - 1);      // (vv is zero past the end)
+#pragma unroll
+        for (int gi = 0; gi < kMaxGroup; ++gi)
+          if (gi < g) o[gi] = fmaf(sc[gi * n_list + idx], vv[u], o[gi]);
+      }
+    }
   }
   for (int gi = 0; gi < g; ++gi) {
     const size_t row = ((size_t)b * n_q + i) * a.n_q_heads + (size_t)kvh * g + gi;
