@@ -841,7 +841,7 @@ def roofline_of(run, args, timing, ms_region, peaks, peaks_kind):
     stored_info = None
     if stored_n:
         k_ms = stored_ms / stored_n
-        stored_info = {"kernel": "attn_stored_mma_kernel" if ctx.stored_path() == 1 else "attn_stored_kernel",
+        stored_info = {"kernel": stored_kernel_name(ctx),
                        "kernel_ms": k_ms, "kernel_launches": stored_n, "achieved_gbs": full_bytes / (k_ms * 1e-3) / 1e9,
                        "frac_of_%s_hbm" % peaks_kind: full_bytes / (k_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"])}
     if run.absorbed:
@@ -986,10 +986,17 @@ def measure_uncompressed(run, rep, steps, peaks, peaks_kind):
     k_ms = stored_ms / max(stored_n, 1)
     gbs = full_bytes / (k_ms * 1e-3) / 1e9
     return {"ms_per_step": ms_total / steps, "layers_per_step": len(run.full_layers),
-            "kernel": "attn_stored_mma_kernel" if run.ctx.stored_path() == 1 else "attn_stored_kernel",
+            "kernel": stored_kernel_name(run.ctx),
             "kernel_ms": k_ms, "achieved_gbs": gbs, "frac_of_%s_hbm" % peaks_kind: gbs / float(peaks["hbm_gbs"]),
             "what": "full-cache attention on every layer of the step (the layers that hold a full cache here, "
                     "walked %d time(s))" % (len(run.full_layers) // max(1, len(set(run.full_layers))))}
+
+
+def stored_kernel_name(ctx):
+    """The kernel that serves stored heads in this context (csrc/stored_mma.cu, csrc/simt_kernels.cu)."""
+    if ctx.stored_path() != 1:
+        return "attn_stored_kernel"
+    return "attn_stored_rope_kernel" if ctx.rope_enabled() else "attn_stored_mma_kernel"
 
 
 def sustained_leg(run, rep, ms_step, seconds, peaks, peaks_kind, args):

@@ -324,5 +324,16 @@ __device__ __forceinline__ void mma_m16n8k16_bf16(float (&c)[4], uint32_t a0, ui
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// tf32 x tf32 -> fp32: a0 = A[lane / 4][lane % 4], a1 = A[lane / 4 + 8][lane % 4], a2 / a3 the same rows at column
+// lane % 4 + 4; b0 = B[k = lane % 4][n = lane / 4], b1 = B[k = lane % 4 + 4][n = lane / 4].  The operands are fp32
+// bit patterns; the tensor core reads their upper 19 bits.
+__device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 
 }  // namespace echokv
