@@ -164,3 +164,80 @@ def test_rope_argument_checks():
         np.testing.assert_allclose(coarse[:, j, 1], np.sin(t[::16] * wj), atol=1e-7)
         np.testing.assert_allclose(fine[:, j, 1], np.sin(t[:16] * wj), atol=1e-7)
     case.close()
+
+
+# ---- the rotating stored-head kernel (anchor layer 0 and the retained heads of layer 1) on its own edge cases ----
+STORED_ROPE = [
+    # name, base, overrides, lens
+    ("mha_many_items", synth.C1, dict(batch=3, context=2100), [2100, 1025, 64]),
+    ("gqa4_one_token", synth.C2, dict(batch=3, context=1500, n_retained_heads=3, random_pages=True), [1500, 257, 1]),
+    ("gqa2_pages32", synth.C2, dict(n_q_heads=16, batch=2, context=900, page_tokens=32, random_pages=True), [900, 33]),
+    ("gqa8_pages64", synth.C2, dict(n_q_heads=32, n_kv_heads=4, n_retained_heads=2, batch=2, context=700,
+                                    page_tokens=64), [700, 65]),
+    ("gqa8_long", synth.C2, dict(n_q_heads=32, n_kv_heads=4, n_retained_heads=1, batch=2, context=5000,
+                                 random_pages=True), [5000, 4097]),
+    ("gqa4_pages128", synth.C2, dict(batch=2, context=1000, page_tokens=128, n_retained_heads=5,
+                                     random_pages=True), [1000, 129]),
+]
+
+
+@pytest.mark.parametrize("name,base,over,lens", STORED_ROPE, ids=[s[0] for s in STORED_ROPE])
+def test_rotating_stored_head_kernel_against_oracle(name, base, over, lens):
+    w = base.replace(**over)
+    case = Case(w, lens=lens, layers=[0, 1], rope=THETA)
+    assert case.ctx.stored_path() == 1 and case.ctx.rope_enabled()
+    for layer in (0, 1):
+        out = case.run(layer)
+        assert_parity(out, case.oracle(layer), w.dtype, "%s layer %d" % (name, layer))
+        np.testing.assert_array_equal(case.run(layer), out)            # repeatable bit for bit
+    np.testing.assert_array_equal(case.run(0, full=True), case.run(0))
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+def test_rotating_stored_head_kernel_more_sequences_than_one_launch_indexes():
+    w = synth.C2.replace(batch=600, context=48, n_kv_heads=2, n_q_heads=8, n_retained_heads=1)
+    rng = np.random.default_rng(5)
+    lens = [int(v) for v in rng.integers(1, 49, size=w.batch)]
+    case = Case(w, lens=lens, layers=[0, 1], rope=THETA)
+    assert_parity(case.run(0), case.oracle(0), w.dtype, "batch 600, anchor, rotated")
+    assert_parity(case.run(1), case.oracle(1), w.dtype, "batch 600, compressed, rotated")
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+def test_rotating_stored_head_kernel_ignores_what_unused_slots_hold_and_reports_bad_input():
+    w = synth.C2.replace(batch=2, context=600, n_retained_heads=3, random_pages=True)
+    lens = [600, 70]
+    n_pages = 2 * w.pages_per_seq + 9
+    case = Case(w, lens=lens, layers=[0, 1], n_pages=n_pages, rope=THETA)
+    clean = {l: case.run(l) for l in (0, 1)}
+    used = torch.zeros((n_pages, w.page_tokens), dtype=torch.bool)
+    for b, L in enumerate(lens):
+        for t in range(L):
+            used[int(case.table[b, t // w.page_tokens]), t % w.page_tokens] = True
+    junk = torch.tensor([float("nan"), float("inf"), -3.0e38, 1.0e30], dtype=torch.float32)
+    for l in (0, 1):
+        for pool in (case.ctx.k_pools[l], case.ctx.v_pools[l]):
+            fill = junk[torch.arange(pool.shape[-1]) % 4].to(pool.dtype).to(pool.device)
+            pool[(~used).to(pool.device)] = fill
+    for l in (0, 1):
+        np.testing.assert_array_equal(case.run(l), clean[l])
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    # a length of zero and a page id outside the pool: reported, the other sequence untouched, nothing faults
+    dev = case.ctx.device
+    q = case.q[0].to(dev)
+    out = case.ctx.decode_attention(0, q, torch.tensor([600, 0], dtype=torch.int32, device=dev)).cpu().numpy()
+    assert case.ctx.device_status() == binding.ECHOKV_EBADLENGTH
+    np.testing.assert_array_equal(out[0], clean[0][0])
+    assert np.all(out[1] == 0.0)
+    saved = case.ctx.block_table.clone()
+    case.ctx.block_table[1, 1] = 10 ** 6
+    out = case.ctx.decode_attention(0, q, case.seq_lens).cpu().numpy()
+    assert case.ctx.device_status() == binding.ECHOKV_EBADPAGE
+    np.testing.assert_array_equal(out[0], clean[0][0])
+    assert np.all(np.isfinite(out))
+    case.ctx.block_table.copy_(saved)
+    np.testing.assert_array_equal(case.run(0), clean[0])
+    assert case.ctx.device_status() == binding.ECHOKV_OK
+    case.close()
