@@ -542,37 +542,51 @@ prefill_attn_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 // ---------------------------------------------------------------------------------------------
 // 4. the sink and window tokens of every query, at full precision (Section 4.1), combined with step 3
 // ---------------------------------------------------------------------------------------------
-// One block per (query i, KV head, sequence).  The query at position p reads as stored: the sink tokens
-// t < min(n_sink, p + 1) -- their retained dims from the layer's pools, the rest from the side buffers -- and the
-// window tokens max(n_sink, p - n_window + 1) .. p, whole rows of k_recent / v_recent.  Scores (keys rotated to
-// their positions if a table is set), softmax over these tokens, weighted values; then the log-sum-exp combination
-// with what step 3 left in out / lse for the tokens the query sees as predicted.  Thread per token for the scores,
-// thread per output dim for the values.
-__global__ void __launch_bounds__(128) prefill_band_kernel(AttnArgs a, PrefillBand w, int n_q, float* __restrict__ out,
-                                                           const float* __restrict__ lse) {
-  extern __shared__ float band_smem[];
+// One block per (QB consecutive queries, KV head, sequence).  The query at position p reads as stored: the sink
+// tokens t < min(n_sink, p + 1) -- their retained dims from the layer's pools, the rest from the side buffers -- and
+// the window tokens max(n_sink, p - n_window + 1) .. p, whole rows of k_recent / v_recent.  Consecutive queries share
+// all but one of these tokens, so the block reads the union once (n_sink + n_window + QB - 1 rows) and masks per
+// query.  Scores: thread per token, the key row (rotated to its position if a table is set) against the QB x G query
+// rows held in shared memory.  Softmax: warp per (query, head).  Values: 32 threads x 4 output dims per token, the
+// block's five warps on every fifth token, summed through shared memory; then the log-sum-exp combination with what
+// step 3 left in out / lse for the tokens the query sees as predicted.
+constexpr int kBandThreads = 160;
+constexpr int kBandSlices = kBandThreads / 32;
+
+template <int G, int QB>
+__global__ void __launch_bounds__(kBandThreads) prefill_band_kernel(AttnArgs a, PrefillBand w, int n_q,
+                                                                    float* __restrict__ out,
+                                                                    const float* __restrict__ lse) {
+  extern __shared__ __align__(16) float band_smem[];
   constexpr int DH = 128;
+  constexpr int R = QB * G;                    // (query, head) rows of the block
   using T = __nv_bfloat16;
-  const int i = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = a.n_q_heads / a.n_kv_heads;
+  const int i0 = blockIdx.x * QB, kvh = blockIdx.y, b = blockIdx.z, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nq_blk = min(QB, n_q - i0);        // queries of this block
   const int n_list = w.n_sink + w.n_window;
-  float* qs = band_smem;                       // [g][DH], scaled
-  float* sc = qs + kMaxGroup * DH;             // [g][n_list]
-  __shared__ float red[4][kMaxGroup];
-  __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
+  const int NT = n_list + QB - 1;              // most tokens the block can see
+  float* qs = band_smem;                       // [R][DH], scaled
+  float* sc = qs + R * DH;                     // [R][NT]: scores, then probabilities
+  float* osum = sc + R * NT;                   // [R][DH]: weighted values, summed over the slices
+  __shared__ float s_m[R], s_l[R];
   const int slot = a.slots ? a.slots[b] : b;
   const int len = a.lens[b];
   if (slot < 0 || slot >= a.geom.max_batch || len < n_q || len > a.geom.max_pages_per_seq * a.geom.page_tokens)
     return;                                    // (reported, and zeros written, by step 3)
-  const int p = len - n_q + i;                 // this query's position
-  const int n_sink_tok = min(w.n_sink, p + 1);
-  const int win_lo = max(w.n_sink, p - w.n_window + 1);
-  const int n_tok = n_sink_tok + max(0, p - win_lo + 1);
+  const int p_first = len - n_q + i0, p_last = p_first + nq_blk - 1;      // positions of the block's queries
+  const int n_sink_u = min(w.n_sink, p_last + 1);
+  const int wlo = max(w.n_sink, p_first - w.n_window + 1);
+  const int n_tok = n_sink_u + max(0, p_last - wlo + 1);
   const int n_stored_k = min(max(w.mk - kvh * DH, 0), DH), n_stored_v = min(max(w.m - kvh * DH, 0), DH);
   const int n_rows = n_q + w.n_window - 1;     // rows of k_recent / v_recent per sequence; row 0 is position t_base
   const int t_base = len - n_rows;
-  const T* q = reinterpret_cast<const T*>(a.q) + (((size_t)b * n_q + i) * a.n_q_heads + (size_t)kvh * g) * DH;
-  for (int idx = tid; idx < g * DH; idx += 128) qs[idx] = __bfloat162float(q[idx]) * a.scale_log2e;
+  {
+    const T* q = reinterpret_cast<const T*>(a.q) + (((size_t)b * n_q + i0) * a.n_q_heads + (size_t)kvh * G) * DH;
+    for (int idx = tid; idx < R * DH; idx += kBandThreads) {
+      const int qi = idx / (G * DH), rest = idx - qi * G * DH;
+      qs[idx] = qi < nq_blk ? __bfloat162float(q[(size_t)qi * a.n_q_heads * DH + rest]) * a.scale_log2e : 0.f;
+    }
+  }
   __syncthreads();
   const T* k_pool = reinterpret_cast<const T*>(w.k_pool);
   const T* v_pool = reinterpret_cast<const T*>(w.v_pool);
@@ -591,10 +605,10 @@ __global__ void __launch_bounds__(128) prefill_band_kernel(AttnArgs a, PrefillBa
     return (size_t)page * a.geom.page_tokens + t % a.geom.page_tokens;
   };
   const size_t side_base = (size_t)slot * n_list;
-  // scores: one token per thread
-  for (int idx = tid; idx < n_tok; idx += 128) {
-    const bool sink = idx < n_sink_tok;
-    const int t = sink ? idx : win_lo + (idx - n_sink_tok);
+  // ---- scores: one token per thread, against all R query rows ----
+  for (int idx = tid; idx < n_tok; idx += kBandThreads) {
+    const bool sink = idx < n_sink_u;
+    const int t = sink ? idx : wlo + (idx - n_sink_u);
     const T* a_ptr;      // dims [0, n_a) of the head
     const T* b_ptr;      // the rest
     int n_a;
@@ -609,102 +623,142 @@ __global__ void __launch_bounds__(128) prefill_band_kernel(AttnArgs a, PrefillBa
       b_ptr = a_ptr;
     }
     auto k_at = [&](int j) -> const T* { return j < n_a ? a_ptr + j : b_ptr + (j - n_a); };
-    float acc[kMaxGroup];
+    float acc[R];
 #pragma unroll
-    for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
+    for (int r = 0; r < R; ++r) acc[r] = 0.f;
+    // eight dims of the key (kv) against the same dims of every query row
+    auto dot8 = [&](const float (&kv)[8], int j) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float4 q0 = *reinterpret_cast<const float4*>(qs + r * DH + j);
+        const float4 q1 = *reinterpret_cast<const float4*>(qs + r * DH + j + 4);
+        acc[r] = fmaf(kv[0], q0.x, fmaf(kv[1], q0.y, fmaf(kv[2], q0.z, fmaf(kv[3], q0.w, acc[r]))));
+        acc[r] = fmaf(kv[4], q1.x, fmaf(kv[5], q1.y, fmaf(kv[6], q1.z, fmaf(kv[7], q1.w, acc[r]))));
+      }
+    };
     if (a.rope.cs != nullptr) {
       const float2* cs = a.rope.cs + min(t, a.rope.stride - 1);
       for (int j = 0; j < DH / 2; j += 8) {
-        float k_lo[8], k_hi[8];
+        float k_lo[8], k_hi[8], r_lo[8], r_hi[8];
         Vec16<T>::load(k_at(j), k_lo);
         Vec16<T>::load(k_at(DH / 2 + j), k_hi);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const float2 cw = cs[(size_t)(j + e) * a.rope.stride];
-          const float r_lo = k_lo[e] * cw.x - k_hi[e] * cw.y, r_hi = k_hi[e] * cw.x + k_lo[e] * cw.y;
-#pragma unroll
-          for (int gi = 0; gi < kMaxGroup; ++gi)
-            if (gi < g) acc[gi] = fmaf(r_hi, qs[gi * DH + DH / 2 + j + e], fmaf(r_lo, qs[gi * DH + j + e], acc[gi]));
+          r_lo[e] = k_lo[e] * cw.x - k_hi[e] * cw.y;
+          r_hi[e] = k_hi[e] * cw.x + k_lo[e] * cw.y;
         }
+        dot8(r_lo, j);
+        dot8(r_hi, DH / 2 + j);
       }
     } else {
       for (int j = 0; j < DH; j += 8) {
         float kv[8];
         Vec16<T>::load(k_at(j), kv);
-#pragma unroll
-        for (int gi = 0; gi < kMaxGroup; ++gi)
-          if (gi < g) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[gi] = fmaf(kv[e], qs[gi * DH + j + e], acc[gi]);
-          }
+        dot8(kv, j);
       }
     }
 #pragma unroll
-    for (int gi = 0; gi < kMaxGroup; ++gi)
-      if (gi < g) sc[gi * n_list + idx] = acc[gi];
+    for (int qi = 0; qi < QB; ++qi) {
+      // does query qi see token t as stored?  (its sink tokens, its window)
+      const int pq = p_first + qi;
+      const bool seen = qi < nq_blk && (sink ? t < min(w.n_sink, pq + 1) : (t <= pq && t > pq - w.n_window));
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) sc[(qi * G + gi) * NT + idx] = seen ? acc[qi * G + gi] : -INFINITY;
+    }
   }
   __syncthreads();
-  for (int gi = 0; gi < g; ++gi) {
+  // ---- softmax: a warp per (query, head) row ----
+  for (int r = warp; r < R; r += kBandSlices) {
+    float* row = sc + r * NT;
     float mx = -INFINITY;
-    for (int idx = tid; idx < n_tok; idx += 128) mx = fmaxf(mx, sc[gi * n_list + idx]);
+    for (int idx = lane; idx < n_tok; idx += 32) mx = fmaxf(mx, row[idx]);
     mx = warp_max(mx);
-    if (lane == 0) red[warp][gi] = mx;
-  }
-  __syncthreads();
-  if (tid < g) s_m[tid] = fmaxf(fmaxf(red[0][tid], red[1][tid]), fmaxf(red[2][tid], red[3][tid]));
-  __syncthreads();
-  for (int gi = 0; gi < g; ++gi) {
-    const float M = s_m[gi];
     float l = 0.f;
-    for (int idx = tid; idx < n_tok; idx += 128) {
-      const float pv = exp2f(sc[gi * n_list + idx] - M);
-      sc[gi * n_list + idx] = pv;
+    for (int idx = lane; idx < n_tok; idx += 32) {
+      const float pv = mx > -INFINITY ? exp2f(row[idx] - mx) : 0.f;      // (a row of a query past the chunk: nothing)
+      row[idx] = pv;
       l += pv;
     }
     l = warp_sum(l);
-    if (lane == 0) red[warp][gi] = l;
+    if (lane == 0) {
+      s_m[r] = mx;
+      s_l[r] = l;
+    }
   }
+  for (int idx = tid; idx < R * DH; idx += kBandThreads) osum[idx] = 0.f;
   __syncthreads();
-  if (tid < g) s_l[tid] = (red[0][tid] + red[1][tid]) + (red[2][tid] + red[3][tid]);
-  __syncthreads();
-  // weighted values: output dim tid of the head; then the combination with the predicted tokens' result
-  float o[kMaxGroup];
+  // ---- weighted values: output dims 4 lane .. 4 lane + 3 of the head, this warp on every fifth token ----
+  float o[R][4];
 #pragma unroll
-  for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
-  const bool from_pool = tid < n_stored_v;
-  for (int idx = 0; idx < n_sink_tok; ++idx) {           // sink tokens: pool + side buffers
-    float vv;
-    if (from_pool) vv = __bfloat162float(v_pool[pool_row(idx) * (size_t)w.m + (size_t)kvh * DH + tid]);
-    else vv = __bfloat162float(v_side[(side_base + idx) * (size_t)w.d_drop + (kvh * DH + tid - w.m)]);
+  for (int r = 0; r < R; ++r)
 #pragma unroll
-    for (int gi = 0; gi < kMaxGroup; ++gi)
-      if (gi < g) o[gi] = fmaf(sc[gi * n_list + idx], vv, o[gi]);
+    for (int e = 0; e < 4; ++e) o[r][e] = 0.f;
+  auto add_token = [&](int idx, const float (&vv)[4]) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const float pv = sc[r * NT + idx];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[r][e] = fmaf(pv, vv[e], o[r][e]);
+    }
+  };
+  for (int idx = warp; idx < n_sink_u; idx += kBandSlices) {            // sink tokens: pool + side buffers
+    float vv[4];
+    const size_t prow = n_stored_v > 0 ? pool_row(idx) : 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int dim = 4 * lane + e;
+      vv[e] = dim < n_stored_v
+                  ? __bfloat162float(v_pool[prow * (size_t)w.m + (size_t)kvh * DH + dim])
+                  : __bfloat162float(v_side[(side_base + idx) * (size_t)w.d_drop + (kvh * DH + dim - w.m)]);
+    }
+    add_token(idx, vv);
   }
   {
-    // window tokens: consecutive rows of v_recent, eight loads in flight at a time
-    const int n_win = n_tok - n_sink_tok;
-    const T* v_row = v_recent + ((size_t)b * n_rows + (win_lo - t_base)) * (size_t)w.D + (size_t)kvh * DH + tid;
-    for (int i0 = 0; i0 < n_win; i0 += 8) {
-      float vv[8];
+    // window tokens: rows of v_recent, four loads in flight at a time
+    const int n_win = n_tok - n_sink_u;
+    const T* v_col = v_recent + ((size_t)b * n_rows + (wlo - t_base)) * (size_t)w.D + (size_t)kvh * DH + 4 * lane;
+    for (int i = warp; i < n_win; i += 4 * kBandSlices) {
+      uint2 raw[4];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) vv[u] = i0 + u < n_win ? __bfloat162float(v_row[(size_t)(i0 + u) * w.D]) : 0.f;
+      for (int u = 0; u < 4; ++u) {
+        const int iu = i + u * kBandSlices;
+        raw[u] = iu < n_win ? *reinterpret_cast<const uint2*>(v_col + (size_t)iu * w.D) : make_uint2(0u, 0u);
+      }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int idx = min(n_sink_tok + i0 + u, n_tok - 1);      // (vv is zero past the end)
-#pragma unroll
-        for (int gi = 0; gi < kMaxGroup; ++gi)
-          if (gi < g) o[gi] = fmaf(sc[gi * n_list + idx], vv[u], o[gi]);
+      for (int u = 0; u < 4; ++u) {
+        const int iu = i + u * kBandSlices;
+        if (iu < n_win) {
+          const float vv[4] = {__uint_as_float(raw[u].x << 16), __uint_as_float(raw[u].x & 0xffff0000u),
+                               __uint_as_float(raw[u].y << 16), __uint_as_float(raw[u].y & 0xffff0000u)};
+          add_token(n_sink_u + iu, vv);
+        }
       }
     }
   }
-  for (int gi = 0; gi < g; ++gi) {
-    const size_t row = ((size_t)b * n_q + i) * a.n_q_heads + (size_t)kvh * g + gi;
-    const float lse_a = lse[row];                        // -inf: the query sees no token as predicted
-    const float M = fmaxf(lse_a, s_m[gi]);
+  // the slices' sums, one slice after the other
+  for (int s = 0; s < kBandSlices; ++s) {
+    if (warp == s) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        float4* dst = reinterpret_cast<float4*>(osum + r * DH + 4 * lane);
+        float4 v = *dst;
+        v.x += o[r][0]; v.y += o[r][1]; v.z += o[r][2]; v.w += o[r][3];
+        *dst = v;
+      }
+    }
+    __syncthreads();
+  }
+  // ---- the combination with the predicted tokens' result ----
+  for (int idx = tid; idx < nq_blk * G * DH; idx += kBandThreads) {
+    const int r = idx / DH, d = idx - r * DH, qi = r / G, gi = r - qi * G;
+    const size_t orow = ((size_t)b * n_q + i0 + qi) * a.n_q_heads + (size_t)kvh * G + gi;
+    const float lse_a = lse[orow];                       // -inf: the query sees no token as predicted
+    const float M = fmaxf(lse_a, s_m[r]);
     const float w_a = lse_a > -INFINITY ? exp2f(lse_a - M) : 0.f;
-    const float w_b = exp2f(s_m[gi] - M);
-    const float denom = w_a + w_b * s_l[gi];
-    out[row * DH + tid] = (w_a * out[row * DH + tid] + w_b * o[gi]) / denom;
+    const float w_b = exp2f(s_m[r] - M);
+    const float denom = w_a + w_b * s_l[r];
+    out[orow * DH + d] = (w_a * out[orow * DH + d] + w_b * osum[r * DH + d]) / denom;
   }
 }
 
@@ -765,15 +819,41 @@ cudaError_t launch_prefill_attn(const AttnArgs& a, const __nv_bfloat16* k_rows, 
   return cudaGetLastError();
 }
 
+namespace {
+size_t band_smem_bytes(int rows, int n_list, int qb) {
+  return (size_t)(2 * rows * 128 + rows * (n_list + qb - 1)) * sizeof(float);
+}
+template <int G, int QB>
+cudaError_t launch_band_g(const AttnArgs& a, const PrefillBand& band, int n_q, float* out, const float* lse,
+                          cudaStream_t stream) {
+  const size_t smem = band_smem_bytes(G * QB, band.n_sink + band.n_window, QB);
+  cudaError_t e = cudaFuncSetAttribute(prefill_band_kernel<G, QB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid((n_q + QB - 1) / QB, a.n_kv_heads, a.batch);
+  prefill_band_kernel<G, QB><<<grid, kBandThreads, smem, stream>>>(a, band, n_q, out, lse);
+  return cudaGetLastError();
+}
+template <int G>
+cudaError_t launch_band_q(const AttnArgs& a, const PrefillBand& band, int n_q, float* out, const float* lse,
+                          cudaStream_t stream) {
+  // four queries per block share their tokens; a very long window (its probabilities no longer fit in shared
+  // memory four queries at a time) goes one query per block
+  constexpr int kQB = G >= 8 ? 2 : 4;
+  if (band_smem_bytes(G * kQB, band.n_sink + band.n_window, kQB) <= 96 * 1024)
+    return launch_band_g<G, kQB>(a, band, n_q, out, lse, stream);
+  return launch_band_g<G, 1>(a, band, n_q, out, lse, stream);
+}
+}  // namespace
+
 cudaError_t launch_prefill_band(const AttnArgs& a, const PrefillBand& band, int n_q, float* out, const float* lse,
                                 cudaStream_t stream) {
-  const int n_list = band.n_sink + band.n_window;
-  const size_t smem = (size_t)(kMaxGroup * 128 + kMaxGroup * n_list) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(prefill_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  dim3 grid(n_q, a.n_kv_heads, a.batch);
-  prefill_band_kernel<<<grid, 128, smem, stream>>>(a, band, n_q, out, lse);
-  return cudaGetLastError();
+  switch (a.n_q_heads / a.n_kv_heads) {
+    case 1: return launch_band_q<1>(a, band, n_q, out, lse, stream);
+    case 2: return launch_band_q<2>(a, band, n_q, out, lse, stream);
+    case 4: return launch_band_q<4>(a, band, n_q, out, lse, stream);
+    case 8: return launch_band_q<8>(a, band, n_q, out, lse, stream);
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace echokv

@@ -120,3 +120,35 @@ def test_prefill_with_whole_keys_and_a_window(rope):
         check(out[b], oracle_prefill(case, 1, q, b), "prefill, whole keys, seq %d" % b)
     assert ctx.device_status() == binding.ECHOKV_OK
     case.close()
+
+
+BAND = [
+    # name, overrides of the backbone shape, window, queries: the sink / window pass of the prefill-shaped call
+    ("gqa4_no_sink_short_window", dict(), (0, 5), 37),
+    ("gqa4_sink_only", dict(), (6, 0), 9),
+    ("mha_window_longer_than_the_chunk", dict(n_q_heads=8, n_kv_heads=8, n_retained_heads=3, n_retained_dims=384), (2, 70), 33),
+    ("gqa2", dict(n_q_heads=16, n_kv_heads=8, n_retained_heads=3, n_retained_dims=384), (4, 128), 130),
+    ("gqa8", dict(n_q_heads=32, n_kv_heads=4, group_size=2, n_retained_heads=1, n_retained_dims=128), (4, 128), 131),
+    ("gqa4_very_long_window", dict(), (3, 1500), 70),        # (too long for four queries per block)
+]
+
+
+@pytest.mark.parametrize("name,over,window,n_q", BAND, ids=[c[0] for c in BAND])
+@pytest.mark.parametrize("rope", [None, THETA], ids=["norope", "rope"])
+def test_prefill_window_shapes(name, over, window, n_q, rope):
+    """Windows shorter and longer than the chunk of queries, sink only, window only, every group size."""
+    L = max(1700, n_q + 10)
+    w = synth.C2.replace(batch=2, context=L, random_pages=True, name="band_" + name,
+                         **{**SETTINGS[384], **over})
+    lens = [L, max(n_q, L // 2 + 3)]
+    case = Case(w, lens=lens, layers=[0, 1], biases=True, window=window, rope=rope)
+    ctx, dev = case.ctx, case.ctx.device
+    q = synth.normal((w.batch, n_q, w.n_q_heads, w.head_dim), w.seed, 77, 8).to(synth.torch_dtype(w))
+    recent = case.recent_rows(1, n_q)
+    out = ctx.prefill_attention(1, q.to(dev), case.seq_lens, k_recent=recent[0], v_recent=recent[1])
+    torch.cuda.synchronize()
+    out = out.cpu().numpy().astype(np.float64)
+    for b in range(w.batch):
+        check(out[b], oracle_prefill(case, 1, q, b), "prefill %s seq %d" % (name, b))
+    assert ctx.device_status() == binding.ECHOKV_OK
+    case.close()
