@@ -864,7 +864,7 @@ def roofline_of(run, args, timing, ms_region, peaks, peaks_kind):
                     "algorithmic_bytes_per_launch": bytes_,
                     "mode": "absorbed predictors: the same outputs as the explicit path, a separate roofline row"}
         if args.rope and w.save_k:
-            roofline["kernel"] = "key_scores_stored_kernel + absorb_pv_kernel"
+            roofline["kernel"] = "key_scores_rope_kernel + absorb_pv_kernel"
             roofline["mode"] = "keys kept whole and rotated when read: stored-key scores, V side with absorbed predictors"
         elif args.rope:
             # rotated keys: the K side is explicit (Eq. 3 for the keys on the tensor cores, rotation, scores), only
@@ -876,7 +876,7 @@ def roofline_of(run, args, timing, ms_region, peaks, peaks_kind):
             roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": burst_tf, "unit": "TFLOP/s",
                         "frac": achieved_tf / burst_tf, "frac_of_sustained_peak": achieved_tf / sustained_tf,
                         "traffic": None,
-                        "kernel": "recon_pair_kernel (key scores) + key_scores_stored_kernel", "kernel_ms": k_pass_ms,
+                        "kernel": "recon_pair_kernel (key scores) + key_scores_rope_kernel", "kernel_ms": k_pass_ms,
                         "kernel_ms_k_pass": k_pass_ms, "kernel_ms_v_pass": av_ms / max(av_n, 1),
                         "kernel_launches": ak_n, "share_of_step": ak_ms / ms_region,
                         "peak_source": tensor_source,

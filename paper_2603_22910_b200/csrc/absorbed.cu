@@ -21,6 +21,8 @@
 // Every wait is bounded.
 #include "absorbed.h"
 
+#include "stored_mma.h"
+
 #include <cudaTypedefs.h>
 
 #include "ptx_sm100.cuh"
@@ -995,13 +997,18 @@ cudaError_t launch_absorbed(const AttnArgs& a, const AbsorbArgs& r, const Absorb
     ra.n_sink = r.n_sink; ra.n_window = r.n_window;
     if (ev) cudaEventRecord(ev[0], stream);
     if (r.save_k) {
-      if ((e = launch_key_scores_stored(a, r.k_local, r.D, a.n_kv_heads, S, lay.l_cap, r.n_sink, r.n_window, stream)) !=
-          cudaSuccess)
+      if (r.k_stored == nullptr) return cudaErrorInvalidValue;
+      if ((e = launch_key_scores_stored(a, *r.k_stored, *r.k_stored_run, a.n_kv_heads, S, lay.l_cap, r.n_sink,
+                                        r.n_window, sm_count, stream)) != cudaSuccess)
         return e;
     } else {
       if ((e = launch_recon_pair_key_scores(a, ra, anchor, layer, S, lay.l_cap, sm_count, stream)) != cudaSuccess) return e;
-      if ((e = launch_key_scores_stored(a, r.k_local, r.m, n_ret, S, lay.l_cap, r.n_sink, r.n_window, stream)) != cudaSuccess)
-        return e;
+      if (n_ret > 0) {
+        if (r.k_stored == nullptr) return cudaErrorInvalidValue;
+        if ((e = launch_key_scores_stored(a, *r.k_stored, *r.k_stored_run, n_ret, S, lay.l_cap, r.n_sink, r.n_window,
+                                          sm_count, stream)) != cudaSuccess)
+          return e;
+      }
     }
     if (ev) cudaEventRecord(ev[1], stream);
   } else {

@@ -61,6 +61,8 @@ struct AbsorbArgs {
   void* k_side = nullptr; void* v_side = nullptr;            // ... their dropped dims (side buffers of the layer)
   const void* k_local = nullptr; const void* v_local = nullptr;   // ... and the layer's pools (retained dims); also
                                                                  // read when the keys are rotated
+  // rotated keys: the layer's K pool as the stored-head kernels see it (tensor maps in boxes of a page and of 64 rows)
+  const CUtensorMap* k_stored = nullptr; const CUtensorMap* k_stored_run = nullptr;
   double* kernel_ms;            // unused
 };
 

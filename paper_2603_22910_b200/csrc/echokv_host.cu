@@ -399,8 +399,18 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
     for (int l = 0; l < cfg->n_layers; ++l) {
       Layer& L = c->layers[l];
       const int width = L.anchor ? d.D : d.m;
-      if (width == 0 || (!L.anchor && d.save_k)) continue;   // (keys kept whole: no stored-head call on that layer)
       const uint64_t rows = (uint64_t)cfg->n_pages * cfg->page_tokens;
+      if (!L.anchor && d.save_k) {
+        // keys kept whole: no stored-head attention on that layer, but its keys are scored from the pool when a
+        // rotation is set (the K maps only)
+        if (encode_pool_group_map(&L.stored_k, L.k_pool, d.D, rows, box_rows) != cudaSuccess ||
+            encode_pool_group_map(&L.stored_k_run, L.k_pool, d.D, rows, 64) != cudaSuccess) {
+          delete c;
+          return ECHOKV_ECUDA;
+        }
+        continue;
+      }
+      if (width == 0) continue;
       if (encode_pool_group_map(&L.stored_k, L.k_pool, width, rows, box_rows) != cudaSuccess ||
           encode_pool_group_map(&L.stored_v, L.v_pool, width, rows, box_rows) != cudaSuccess ||
           encode_pool_group_map(&L.stored_k_run, L.k_pool, width, rows, 64) != cudaSuccess ||
@@ -758,6 +768,10 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     aa.D = c->d.D; aa.m = c->d.m;
     aa.capacity_tokens = c->d.capacity;
     aa.kernel_ms = nullptr;
+    if (c->stored_capable && (c->d.save_k || c->d.m > 0)) {
+      aa.k_stored = &L.stored_k;
+      aa.k_stored_run = &L.stored_k_run;
+    }
     if (side) {
       aa.n_sink = c->n_sink; aa.n_window = c->n_window;
       aa.k_side = L.k_side; aa.v_side = L.v_side;

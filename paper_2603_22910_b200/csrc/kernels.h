@@ -37,11 +37,6 @@ cudaError_t launch_append(int dtype, void* k_pool, void* v_pool, int k_width, in
 cudaError_t launch_attn_stored(const AttnArgs& a, const void* k_pool, const void* v_pool, int width,
                                int n_heads, int n_splits, cudaStream_t stream);
 
-// Rotated-key scores of stored heads 0 .. n_heads-1 (bf16, head_dim 128, a.rope set): S[b][query head][l_cap] in
-// base-2 units, -inf for token slots without a predicted token; whole 256-token tiles are written.
-cudaError_t launch_key_scores_stored(const AttnArgs& a, const void* k_pool, int width, int n_heads, float* S,
-                                     int l_cap, int n_sink, int n_window, cudaStream_t stream);
-
 struct ReconArgs {
   const void* k_anchor; const void* v_anchor;   // pools of row width D
   const void* k_local; const void* v_local;     // pools of row width m (may be null when m == 0)

@@ -378,207 +378,6 @@ cudaError_t launch_attn_stored(const AttnArgs& a, const void* k_pool, const void
 }
 
 // ---------------------------------------------------------------------------------------------
-// Scores of stored heads whose keys are rotated when read: S[b][h][t] = q_h . R_t k_t (base-2 units) for the
-// query heads of KV heads 0 .. n_heads-1, one thread per token; token slots that hold no predicted token get
-// -inf.  Feeds the softmax of the absorbed V side when the K side has to be explicit (rotated keys).
-// ---------------------------------------------------------------------------------------------
-// The angle of token t = 16 u + r is the sum of a coarse one (u) and a fine one (r):  q . R_t k = (R_coarse(u)^T q) .
-// (R_fine(r) k).  The queries are turned back by the coarse angle once per 16-token group, so a token only turns its
-// key by one of 16 fine angles; that and the products run on the two-wide fp32 instructions.
-//
-// Shared memory of key_scores_stored_kernel: everything the per-token loop reads, so that loop never waits on
-// global memory.  The per-tile part exists twice: the next tile is copied (cp.async) while this one is scored.
-template <int DH, int G>
-struct KeyScoresSmem {
-  static constexpr int kRowPad = DH * 2 + 16;        // staged key rows: 16-byte reads of successive rows hit all banks
-  static constexpr int kFinePad = DH / 2 + 2;        // fine-angle rows: 8-byte reads of successive rows hit all banks
-  static constexpr int kGroups = 128 / kRopeFineRows;
-  struct Stage {
-    float2 coarse[kGroups][DH / 2];                  // (cos, sin) of the tile's eight 16-token groups
-    long long rows[128];                             // pool row of each token, -1 = nothing to read
-    __align__(16) unsigned char ks[128 * kRowPad];   // the tile's 128 key rows of this head
-  };
-  float qs[G][DH];                                   // queries * scale * log2e
-  __align__(16) float qrot[kGroups][G][DH];          // the same, turned back by each group's coarse angle
-  __align__(8) float fine_cos[kRopeFineRows][kFinePad];   // cosines / sines of offsets 0 .. 15
-  __align__(8) float fine_sin[kRopeFineRows][kFinePad];
-  __align__(16) Stage st[2];
-};
-constexpr int kKeyScoresTilesPerBlock = 8;           // consecutive 128-token tiles of one (sequence, head) per block
-
-__device__ __forceinline__ void ks_cp_async16(void* dst_smem, const void* src, bool real) {
-  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(real ? 16u : 0u) : "memory");
-}
-
-template <int DH, int G>
-__global__ void __launch_bounds__(128) key_scores_stored_kernel(AttnArgs a, const __nv_bfloat16* __restrict__ k_pool,
-                                                                int width, float* __restrict__ S, int l_cap,
-                                                                int n_sink, int n_window) {
-  extern __shared__ __align__(16) unsigned char key_scores_smem[];
-  using Smem = KeyScoresSmem<DH, G>;
-  Smem& sm = *reinterpret_cast<Smem*>(key_scores_smem);
-  constexpr int kRowPad = Smem::kRowPad, kGroups = Smem::kGroups;
-  // heads fastest: the blocks that run together read neighbouring pieces of the same cache rows
-  const int b = blockIdx.z, kvh = blockIdx.x, tid = threadIdx.x;
-  const int slot = a.slots ? a.slots[b] : b;
-  const int len = a.lens[b];
-  if (slot < 0 || slot >= a.geom.max_batch || len < 1 || len > a.geom.max_pages_per_seq * a.geom.page_tokens)
-    return;                                    // (reported by the other kernels of the call)
-  // whole 256-token tiles are written, no more
-  const int n_tiles = min(((len + 255) / 256) * 2, (l_cap + 127) / 128);
-  // Block y takes tiles y, y + gridDim.y, ...: the blocks that run together then read neighbouring tiles, a front that
-  // sweeps through the cache, instead of many streams that sit a fixed large stride apart.
-  const int tile_lo = blockIdx.y, tile_step = gridDim.y, tile_hi = n_tiles;
-  if (tile_lo >= tile_hi) return;
-  const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q);
-  for (int idx = tid; idx < G * DH; idx += 128)
-    sm.qs[idx / DH][idx % DH] = __bfloat162float(q[((size_t)b * a.n_q_heads + (size_t)kvh * G) * DH + idx]) * a.scale_log2e;
-  for (int idx = tid; idx < kRopeFineRows * (DH / 2); idx += 128) {
-    const float2 cs = a.rope.fine[idx];
-    sm.fine_cos[idx / (DH / 2)][idx % (DH / 2)] = cs.x;
-    sm.fine_sin[idx / (DH / 2)][idx % (DH / 2)] = cs.y;
-  }
-
-  constexpr int kVecPerRow = DH * 2 / 16;
-  static_assert(kVecPerRow == 16, "one row per 16 lanes");
-  // this thread's token of a tile: its pool row (kept in a register for the scoring, in shared memory for the copy)
-  auto lookup = [&](int tile, int buf) -> long long {
-    const int t = tile * 128 + tid;
-    long long row = -1;
-    if (t < l_cap && t >= predicted_lo(len, n_sink) && t < predicted_hi(len, n_sink, n_window)) {
-      const int page = a.geom.table[(size_t)slot * a.geom.max_pages_per_seq + t / a.geom.page_tokens];
-      if (page < 0 || page >= a.geom.n_pages) report(a.status, ECHOKV_EBADPAGE);
-      else row = (long long)page * a.geom.page_tokens + t % a.geom.page_tokens;
-    }
-    sm.st[buf].rows[tid] = row;
-    return row;
-  };
-  // coalesced copies, 16 lanes x 16 bytes per key row; a row that is not read becomes zeros
-  auto issue = [&](int tile, int buf) {
-    typename Smem::Stage& st = sm.st[buf];
-    const int v = tid % kVecPerRow, r0 = tid / kVecPerRow;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const long long src_row = st.rows[r0 + 8 * i];
-      const __nv_bfloat16* src = k_pool + (size_t)(src_row >= 0 ? src_row : 0) * width + (size_t)kvh * DH + v * 8;
-      ks_cp_async16(st.ks + (r0 + 8 * i) * kRowPad + v * 16, src, src_row >= 0);
-    }
-    constexpr int kCoarseVecs = kGroups * (DH / 2) * 8 / 16;      // 16-byte pieces of the coarse rows
-#pragma unroll
-    for (int i = 0; i < kCoarseVecs / 128; ++i) {
-      const int idx = tid + 128 * i, u_local = idx / (DH / 4), piece = idx % (DH / 4);
-      const int u = min(tile * kGroups + u_local, a.rope.stride / kRopeFineRows - 1);
-      ks_cp_async16(reinterpret_cast<unsigned char*>(st.coarse[u_local]) + piece * 16,
-                    reinterpret_cast<const unsigned char*>(a.rope.coarse + (size_t)u * (DH / 2)) + piece * 16, true);
-    }
-  };
-
-  long long row_cur = lookup(tile_lo, 0);
-  __syncthreads();
-  issue(tile_lo, 0);
-  asm volatile("cp.async.commit_group;" ::: "memory");
-  int buf = 0;
-  for (int tile = tile_lo; tile < tile_hi; tile += tile_step, buf ^= 1) {
-    const int next = tile + tile_step;
-    long long row_next = -1;
-    if (next < tile_hi) row_next = lookup(next, buf ^ 1);
-    __syncthreads();           // the next tile's rows are known; everyone is done scoring out of the other buffer
-    if (next < tile_hi) issue(next, buf ^ 1);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 1;" ::: "memory");
-    __syncthreads();           // this tile's rows and coarse angles (and the queries, the fine table) are in shared memory
-    const typename Smem::Stage& st = sm.st[buf];
-    // queries turned back by the coarse angle of each 16-token group: (q_lo C + q_hi S, q_hi C - q_lo S)
-    for (int idx = tid; idx < kGroups * G * (DH / 2); idx += 128) {
-      const int j = idx % (DH / 2), gi = (idx / (DH / 2)) % G, u = idx / (DH / 2 * G);
-      const float2 cs = st.coarse[u][j];
-      const float q_lo = sm.qs[gi][j], q_hi = sm.qs[gi][DH / 2 + j];
-      sm.qrot[u][gi][j] = q_lo * cs.x + q_hi * cs.y;
-      sm.qrot[u][gi][DH / 2 + j] = q_hi * cs.x - q_lo * cs.y;
-    }
-    __syncthreads();
-    const int t = tile * 128 + tid;
-    uint64_t acc2[G];          // (sum over even pairs, sum over odd pairs)
-#pragma unroll
-    for (int gi = 0; gi < G; ++gi) acc2[gi] = 0ull;
-    if (row_cur >= 0) {
-      const unsigned char* kr = st.ks + tid * kRowPad;
-      const float* fcos = sm.fine_cos[tid % kRopeFineRows];
-      const float* fsin = sm.fine_sin[tid % kRopeFineRows];
-      const float (*qr)[DH] = sm.qrot[tid / kRopeFineRows];
-#pragma unroll 4
-      for (int j = 0; j < DH / 2; j += 8) {
-        const uint4 lo4 = *reinterpret_cast<const uint4*>(kr + j * 2);
-        const uint4 hi4 = *reinterpret_cast<const uint4*>(kr + DH + j * 2);
-        const uint32_t lw[4] = {lo4.x, lo4.y, lo4.z, lo4.w}, hw[4] = {hi4.x, hi4.y, hi4.z, hi4.w};
-        uint64_t r_lo[4], r_hi[4];       // the eight key pairs turned by the fine angle, two per register
-#pragma unroll
-        for (int e2 = 0; e2 < 4; ++e2) {
-          const uint64_t k_lo = pack_u2(lw[e2] << 16, lw[e2] & 0xffff0000u);
-          const uint64_t k_hi = pack_u2(hw[e2] << 16, hw[e2] & 0xffff0000u);
-          const uint64_t c2 = *reinterpret_cast<const uint64_t*>(fcos + j + 2 * e2);
-          const uint64_t s2 = *reinterpret_cast<const uint64_t*>(fsin + j + 2 * e2);
-          const uint64_t ns2 = s2 ^ 0x8000000080000000ull;
-          r_lo[e2] = fma_f2(k_hi, ns2, mul_f2(k_lo, c2));
-          r_hi[e2] = fma_f2(k_lo, s2, mul_f2(k_hi, c2));
-        }
-#pragma unroll
-        for (int gi = 0; gi < G; ++gi) {
-          const ulonglong2* ql = reinterpret_cast<const ulonglong2*>(&qr[gi][j]);
-          const ulonglong2* qh = reinterpret_cast<const ulonglong2*>(&qr[gi][DH / 2 + j]);
-          const ulonglong2 l0 = ql[0], l1 = ql[1], h0 = qh[0], h1 = qh[1];
-          uint64_t v = acc2[gi];
-          v = fma_f2(r_lo[0], l0.x, v); v = fma_f2(r_lo[1], l0.y, v); v = fma_f2(r_lo[2], l1.x, v); v = fma_f2(r_lo[3], l1.y, v);
-          v = fma_f2(r_hi[0], h0.x, v); v = fma_f2(r_hi[1], h0.y, v); v = fma_f2(r_hi[2], h1.x, v); v = fma_f2(r_hi[3], h1.y, v);
-          acc2[gi] = v;
-        }
-      }
-    }
-    if (t < l_cap) {
-#pragma unroll
-      for (int gi = 0; gi < G; ++gi) {
-        float even, odd;
-        unpack_f2(acc2[gi], even, odd);
-        S[((size_t)b * a.n_q_heads + (size_t)kvh * G + gi) * l_cap + t] = row_cur >= 0 ? even + odd : -INFINITY;
-      }
-    }
-    row_cur = row_next;
-  }
-}
-
-template <int G>
-static cudaError_t launch_key_scores_stored_g(const AttnArgs& a, const void* k_pool, int width, int n_heads, float* S,
-                                              int l_cap, int n_sink, int n_window, cudaStream_t stream) {
-  const size_t smem = sizeof(KeyScoresSmem<128, G>);
-  cudaError_t e = cudaFuncSetAttribute(key_scores_stored_kernel<128, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
-  if (e != cudaSuccess) return e;
-  // several blocks per SM: ask for the largest shared-memory carve-out
-  e = cudaFuncSetAttribute(key_scores_stored_kernel<128, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                           cudaSharedmemCarveoutMaxShared);
-  if (e != cudaSuccess) return e;
-  const int n_tiles = (l_cap + 127) / 128;
-  dim3 grid(n_heads, (n_tiles + kKeyScoresTilesPerBlock - 1) / kKeyScoresTilesPerBlock, a.batch);
-  key_scores_stored_kernel<128, G><<<grid, 128, smem, stream>>>(a, reinterpret_cast<const __nv_bfloat16*>(k_pool), width,
-                                                                S, l_cap, n_sink, n_window);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_key_scores_stored(const AttnArgs& a, const void* k_pool, int width, int n_heads, float* S,
-                                     int l_cap, int n_sink, int n_window, cudaStream_t stream) {
-  if (n_heads == 0) return cudaSuccess;
-  if (a.dtype != ECHOKV_BF16 || a.head_dim != 128 || a.rope.cs == nullptr) return cudaErrorInvalidValue;
-  switch (a.n_q_heads / a.n_kv_heads) {
-    case 1: return launch_key_scores_stored_g<1>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
-    case 2: return launch_key_scores_stored_g<2>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
-    case 4: return launch_key_scores_stored_g<4>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
-    case 8: return launch_key_scores_stored_g<8>(a, k_pool, width, n_heads, S, l_cap, n_sink, n_window, stream);
-    default: return cudaErrorInvalidValue;
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
 // CUDA-core reconstruct-then-attend (Eq. 3, 6, 7 for one dropped KV head and one token range)
 // ---------------------------------------------------------------------------------------------
 constexpr int kKc = 32;   // features per staged chunk of the predictor input

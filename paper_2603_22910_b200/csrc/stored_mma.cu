@@ -66,13 +66,16 @@ struct StoredParams {
   float* part_o;
   int max_parts;
   int32_t* status;
-  int32_t* item_tokens_out;   // where this launch publishes its item_tokens
+  int32_t* item_tokens_out;   // where this launch publishes its item_tokens (null: nobody asks)
   int b0, nb;                 // batch entries [b0, b0 + nb) are handled by this launch
   int n_q_heads, n_heads;     // query heads in all; stored KV heads attended (0 .. n_heads - 1)
   int rows_per_box;           // token rows per TMA box: min(page_tokens, 64)
   int page_shift, box_shift;  // log2 of page_tokens and of rows_per_box (both powers of two)
   float scale_log2e;
-  RopeTable rope;             // read by the rotating kernel only
+  RopeTable rope;             // read by the rotating kernels only
+  // key_scores_rope_kernel only: where the scores go, and which tokens count as predicted
+  float* scores;              // [batch][n_q_heads][l_cap]
+  int l_cap, n_sink, n_window;
 };
 
 // What both kernels keep about the work items
@@ -177,7 +180,7 @@ __device__ __forceinline__ int stored_setup(StoredItems& t, const StoredParams& 
     if (per_item < kMinItemTokens) per_item = kMinItemTokens;
     if (per_item > kMaxItemTokens) per_item = kMaxItemTokens;
     t.item_tokens = (int)per_item;
-    if (blockIdx.x == 0) *p.item_tokens_out = (int)per_item;
+    if (blockIdx.x == 0 && p.item_tokens_out != nullptr) *p.item_tokens_out = (int)per_item;
   }
   __syncthreads();
   const int item_tokens = t.item_tokens;
@@ -588,6 +591,67 @@ template <int G> struct RopeVSlots { static constexpr int value = G >= 8 ? 2 : 3
 constexpr int kRingMax = 4;
 constexpr int kSlotBytes = 2 * kBlockBytes;
 
+// The score warps' work on one 16-token slice of a K slot (sb: the slot; tok_k: this lane's ldmatrix row):
+// S^T = K' Q^T as tf32 products m16n8k8 with the 16 tokens on the M rows: the thread's two features of a token (f and
+// f + 1) are the k indices lane % 4 and lane % 4 + 4 of one product, for the key and for the query alike.  The
+// features 64 .. 127 accumulate apart: two shorter chains of products.
+// acc[0], acc[1]: token lane / 4 of the slice, heads qd and qd + 1; acc[2], acc[3]: token lane / 4 + 8 (raw q . k).
+__device__ __forceinline__ void rotated_key_scores(uint32_t sb, int tok_k, const float4* coarse_q,
+                                                   const float4* fine_a, const float4* fine_b,
+                                                   const uint32_t (&qa0)[8], const uint32_t (&qa2)[8], int lane,
+                                                   float (&acc)[4]) {
+  float acc_lo[4] = {0.f, 0.f, 0.f, 0.f}, acc_hi[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int ks = 0; ks < 4; ++ks) {
+    // register i: token tile i >> 1 (slice offsets lane / 4 and lane / 4 + 8), frequency indices
+    // f = 16 ks + 8 (i & 1) + qd and f + 1; ka the features f, kb the features f + 64
+    const int c0 = ks * 2 + ((lane >> 3) & 1);
+    uint32_t ka[4], kb[4];
+    ldsm_x4(sb + stage_off(tok_k, c0), ka[0], ka[1], ka[2], ka[3]);
+    ldsm_x4(sb + stage_off(tok_k, 8 + c0), kb[0], kb[1], kb[2], kb[3]);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float4 bw = coarse_q[ks * 8 + h * 4];                         // (cos f, sin f, cos f+1, sin f+1)
+      const float2 bc = make_float2(bw.x, bw.z), bs = make_float2(bw.y, bw.w);
+      float2 lo[2], hi[2];
+#pragma unroll
+      for (int tile = 0; tile < 2; ++tile) {
+        const int i = tile * 2 + h;
+        const float4 fw = (tile ? fine_b : fine_a)[ks * 8 + h * 4];       // (cos f, cos f+1, sin f, sin f+1)
+        const float2 fc = make_float2(fw.x, fw.y), fs = make_float2(fw.z, fw.w);
+        float2 cw2 = __fmul2_rn(bc, fc);
+        cw2.x = fmaf(-bs.x, fs.x, cw2.x);
+        cw2.y = fmaf(-bs.y, fs.y, cw2.y);
+        const float2 sw2 = __ffma2_rn(bs, fc, __fmul2_rn(bc, fs));
+        const float2 xa = make_float2(bf16_lo(ka[i]), bf16_hi(ka[i]));
+        const float2 xb = make_float2(bf16_lo(kb[i]), bf16_hi(kb[i]));
+        lo[tile] = __fmul2_rn(xa, cw2);
+        lo[tile].x = fmaf(-xb.x, sw2.x, lo[tile].x);
+        lo[tile].y = fmaf(-xb.y, sw2.y, lo[tile].y);
+        hi[tile] = __ffma2_rn(xa, sw2, __fmul2_rn(xb, cw2));
+      }
+      const uint32_t q_lo = h ? qa2[ks] : qa0[ks];
+      const uint32_t q_hi = h ? qa2[ks + 4] : qa0[ks + 4];
+      mma_m16n8k8_tf32(acc_lo, __float_as_uint(lo[0].x), __float_as_uint(lo[1].x), __float_as_uint(lo[0].y),
+                       __float_as_uint(lo[1].y), q_lo << 16, q_lo & 0xffff0000u);
+      mma_m16n8k8_tf32(acc_hi, __float_as_uint(hi[0].x), __float_as_uint(hi[1].x), __float_as_uint(hi[0].y),
+                       __float_as_uint(hi[1].y), q_hi << 16, q_hi & 0xffff0000u);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) acc[e] = acc_lo[e] + acc_hi[e];
+}
+
+// The fine table into shared memory: entry (r, f even) = (cos f, cos f+1, sin f, sin f+1) of offset r.
+__device__ __forceinline__ void load_fine_table(float2* fine, const RopeTable& rope) {
+  for (int i = threadIdx.x; i < kRopeFineRows * 64; i += blockDim.x) {
+    const float2 cs = rope.fine[i];
+    float* entry = reinterpret_cast<float*>(fine + (i >> 6) * kFineRowPairs + (i & 62));
+    entry[i & 1] = cs.x;
+    entry[2 + (i & 1)] = cs.y;
+  }
+}
+
 template <int G>
 struct StoredRopeSmem {
   // entry (r, f even): (cos f, cos f+1, sin f, sin f+1) of offset r; one entry = two float2
@@ -615,12 +679,7 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   const uint32_t k_ring = smem_u32(smem), v_ring = k_ring + NK * kSlotBytes;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &rs.items.abort_flag;
-  for (int i = tid; i < kRopeFineRows * 64; i += kRopeThreads) {
-    const float2 cs = p.rope.fine[i];
-    float* entry = reinterpret_cast<float*>(rs.fine + (i >> 6) * kFineRowPairs + (i & 62));
-    entry[i & 1] = cs.x;
-    entry[2 + (i & 1)] = cs.y;
-  }
+  load_fine_table(rs.fine, p.rope);
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&rs.s_full[i]), kConsumers);
@@ -677,56 +736,17 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
         const uint32_t sb = k_ring + s * kSlotBytes;
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncwarp();            // this slice's coarse row is in the warp's buffer
-        // S^T = K' Q^T as tf32 products m16n8k8 with the 16 tokens on the M rows: the thread's two features of a
-        // token (f and f + 1) are the k indices lane % 4 and lane % 4 + 4 of one product, for the key and for
-        // the query alike.  The features 64 .. 127 accumulate apart: two shorter chains of products.
-        float acc_lo[4] = {0.f, 0.f, 0.f, 0.f}, acc_hi[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          // register i: token tile i >> 1 (slice offsets lane / 4 and lane / 4 + 8), frequency indices
-          // f = 16 ks + 8 (i & 1) + qd and f + 1; ka the features f, kb the features f + 64
-          const int c0 = ks * 2 + ((lane >> 3) & 1);
-          uint32_t ka[4], kb[4];
-          ldsm_x4(sb + stage_off(tok_k, c0), ka[0], ka[1], ka[2], ka[3]);
-          ldsm_x4(sb + stage_off(tok_k, 8 + c0), kb[0], kb[1], kb[2], kb[3]);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const float4 bw = coarse_q[ks * 8 + h * 4];                         // (cos f, sin f, cos f+1, sin f+1)
-            const float2 bc = make_float2(bw.x, bw.z), bs = make_float2(bw.y, bw.w);
-            float2 lo[2], hi[2];
-#pragma unroll
-            for (int tile = 0; tile < 2; ++tile) {
-              const int i = tile * 2 + h;
-              const float4 fw = (tile ? fine_b : fine_a)[ks * 8 + h * 4];       // (cos f, cos f+1, sin f, sin f+1)
-              const float2 fc = make_float2(fw.x, fw.y), fs = make_float2(fw.z, fw.w);
-              float2 cw2 = __fmul2_rn(bc, fc);
-              cw2.x = fmaf(-bs.x, fs.x, cw2.x);
-              cw2.y = fmaf(-bs.y, fs.y, cw2.y);
-              const float2 sw2 = __ffma2_rn(bs, fc, __fmul2_rn(bc, fs));
-              const float2 xa = make_float2(bf16_lo(ka[i]), bf16_hi(ka[i]));
-              const float2 xb = make_float2(bf16_lo(kb[i]), bf16_hi(kb[i]));
-              lo[tile] = __fmul2_rn(xa, cw2);
-              lo[tile].x = fmaf(-xb.x, sw2.x, lo[tile].x);
-              lo[tile].y = fmaf(-xb.y, sw2.y, lo[tile].y);
-              hi[tile] = __ffma2_rn(xa, sw2, __fmul2_rn(xb, cw2));
-            }
-            const uint32_t q_lo = h ? qa2[ks] : qa0[ks];
-            const uint32_t q_hi = h ? qa2[ks + 4] : qa0[ks + 4];
-            mma_m16n8k8_tf32(acc_lo, __float_as_uint(lo[0].x), __float_as_uint(lo[1].x), __float_as_uint(lo[0].y),
-                             __float_as_uint(lo[1].y), q_lo << 16, q_lo & 0xffff0000u);
-            mma_m16n8k8_tf32(acc_hi, __float_as_uint(hi[0].x), __float_as_uint(hi[1].x), __float_as_uint(hi[0].y),
-                             __float_as_uint(hi[1].y), q_hi << 16, q_hi & 0xffff0000u);
-          }
-        }
+        float acc[4];
+        rotated_key_scores(sb, tok_k, coarse_q, fine_a, fine_b, qa0, qa2, lane, acc);
         // acc[0], acc[1]: token lane / 4 of the slice, heads qd and qd + 1; acc[2], acc[3]: token lane / 4 + 8
         float* sbuf = rs.scores[slot] + cw * kWarpTokens + row;
         if (qd < G) {
-          sbuf[qd * kScoreStride] = acc_lo[0] + acc_hi[0];
-          sbuf[qd * kScoreStride + 8] = acc_lo[2] + acc_hi[2];
+          sbuf[qd * kScoreStride] = acc[0];
+          sbuf[qd * kScoreStride + 8] = acc[2];
         }
         if (qd + 1 < G) {
-          sbuf[(qd + 1) * kScoreStride] = acc_lo[1] + acc_hi[1];
-          sbuf[(qd + 1) * kScoreStride + 8] = acc_lo[3] + acc_hi[3];
+          sbuf[(qd + 1) * kScoreStride] = acc[1];
+          sbuf[(qd + 1) * kScoreStride + 8] = acc[3];
         }
         __syncwarp();
         if (lane == 0) {
@@ -882,6 +902,145 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   }
 }
 
+// =================================================================================================================
+// Scores only: S[b][h][t] = q_h . R_t k_t (base-2 units) for the query heads of stored KV heads, written to memory
+// =================================================================================================================
+// What the absorbed V side needs when the K side has to be explicit (rotated keys): the score warps of the kernel
+// above on a K ring alone -- four score warps and a warp that issues the copies.  Token slots of a sequence's whole
+// 256-token tiles that hold no predicted token (sink / window tokens, tokens past the length, a page that could not
+// be read) get -inf.
+constexpr int kScoresThreads = 32 * (kConsumers + 1);
+constexpr int kScoresKSlots = 3;            // three CTAs per SM: the score warps are what this kernel is short of
+
+struct KeyScoresSmem {
+  float2 fine[kRopeFineRows * kFineRowPairs];
+  float2 coarse[kConsumers][64];
+  StoredItems items;
+  unsigned long long k_full[kScoresKSlots], k_empty[kScoresKSlots];
+  uint32_t box_ok[kScoresKSlots];
+};
+
+template <int G>
+__global__ void __launch_bounds__(kScoresThreads, 3)
+key_scores_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_k_run,
+                       const StoredParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  constexpr int NK = kScoresKSlots;
+  KeyScoresSmem& rs = *reinterpret_cast<KeyScoresSmem*>(smem + NK * kSlotBytes);
+  const uint32_t k_ring = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  volatile int* abort_flag = &rs.items.abort_flag;
+  load_fine_table(rs.fine, p.rope);
+  if (tid == 0) {
+    for (int i = 0; i < NK; ++i) {
+      mbar_init(smem_u32(&rs.k_full[i]), 1);
+      mbar_init(smem_u32(&rs.k_empty[i]), kConsumers);
+    }
+  }
+  const int item_tokens = stored_setup(rs.items, p);
+  const int n_items = rs.items.cum_items[p.nb];
+  const int rpb = p.rows_per_box;
+
+  if (warp == kConsumers) {
+    // =============================== the warp that issues the K copies ===========================
+    StoredProducer<NK, 1> pr;
+    pr.init(rs.items, p, item_tokens, n_items, lane);
+    while (pr.step(rs.items, p, &tm_k, &tm_k, &tm_k_run, &tm_k_run, k_ring, rs.k_full, rs.k_empty, rs.box_ok, abort_flag,
+                   item_tokens, n_items, lane)) {
+    }
+    if (pr.gave_up()) pr.drain(rs.k_full, lane);
+  } else {
+    // =============================== score warps =================================================
+    const int cw = warp;
+    const int row = lane >> 2, qd = (lane & 3) * 2;
+    float2* coarse_w = rs.coarse[cw];
+    const float4* coarse_q = reinterpret_cast<const float4*>(coarse_w + qd);
+    const float4* fine_a = reinterpret_cast<const float4*>(rs.fine + row * kFineRowPairs + qd);
+    const float4* fine_b = reinterpret_cast<const float4*>(rs.fine + (row + 8) * kFineRowPairs + qd);
+    const int tok_k = cw * kWarpTokens + (lane >> 4) * 8 + (lane & 7);          // K rows: ldmatrix
+    auto fetch_coarse = [&](int stage_t0) {
+      const int u = min(stage_t0 / kRopeFineRows + cw, p.rope.stride / kRopeFineRows - 1);
+      __syncwarp();          // every lane has read the row that is there now
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_u32(coarse_w + lane * 2)),
+                   "l"(p.rope.coarse + (size_t)u * 64 + lane * 2)
+                   : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    uint32_t it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const Item w = decode_item(rs.items, item, p.n_heads, p.nb);
+      const int b = p.b0 + w.b;
+      const int len = p.lens[b];
+      const int t_begin = w.chunk * item_tokens;
+      const int t_end = min(len, t_begin + item_tokens);
+      const int n_iter = (t_end - t_begin + kStageTokens - 1) / kStageTokens;
+      const int pred_lo = predicted_lo(len, p.n_sink), pred_hi = predicted_hi(len, p.n_sink, p.n_window);
+      const int write_end = min((len + 255) / 256 * 256, p.l_cap);     // whole 256-token tiles are written, no more
+      float* s_rows = p.scores + ((size_t)b * p.n_q_heads + (size_t)w.kvh * G) * p.l_cap;
+      uint32_t qa0[8], qa2[8];
+      load_q_fragments<G>(p, b, w.kvh, lane, qa0, qa2);
+      fetch_coarse(t_begin);
+      for (int j = 0; j < n_iter; ++j, ++it) {
+        const uint32_t s = it % NK;
+        const bool got = mbar_wait(smem_u32(&rs.k_full[s]), (it / NK) & 1u, abort_flag, p.status);
+        if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
+        const uint32_t sb = k_ring + s * kSlotBytes;
+        const int t0 = t_begin + j * kStageTokens;
+        const unsigned long long valid = stage_mask(rs.box_ok[s], rpb, min(kStageTokens, t_end - t0));
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();            // this slice's coarse row is in the warp's buffer
+        float acc[4];
+        rotated_key_scores(sb, tok_k, coarse_q, fine_a, fine_b, qa0, qa2, lane, acc);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&rs.k_empty[s]));
+        if (j + 1 < n_iter) fetch_coarse(t0 + kStageTokens);
+        // acc[0], acc[1]: token `row` of the slice, heads qd and qd + 1; acc[2], acc[3]: token row + 8
+#pragma unroll
+        for (int h8 = 0; h8 < 2; ++h8) {
+          const int ts = cw * kWarpTokens + h8 * 8 + row, t = t0 + ts;
+          const bool keep = ((valid >> ts) & 1ull) && t >= pred_lo && t < pred_hi;
+          if (t < write_end) {
+            if (qd < G) s_rows[(size_t)qd * p.l_cap + t] = keep ? acc[2 * h8] * p.scale_log2e : -INFINITY;
+            if (qd + 1 < G) s_rows[(size_t)(qd + 1) * p.l_cap + t] = keep ? acc[2 * h8 + 1] * p.scale_log2e : -INFINITY;
+          }
+        }
+        if (t0 + kStageTokens >= len) {
+          // the sequence's last stage: the rest of its last 256-token tile holds no token
+          for (int t = t0 + kStageTokens + cw * 32 + lane; t < write_end; t += kConsumers * 32)
+#pragma unroll
+            for (int gi = 0; gi < G; ++gi) s_rows[(size_t)gi * p.l_cap + t] = -INFINITY;
+        }
+      }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");   // (a copy started before a wait gave up)
+  }
+}
+
+template <int G>
+cudaError_t launch_scores_g(const CUtensorMap& k, const CUtensorMap& k_run, const StoredParams& p, int sm_count,
+                            cudaStream_t stream) {
+  const size_t smem = 1024 + (size_t)kScoresKSlots * kSlotBytes + sizeof(KeyScoresSmem);
+  cudaError_t e = cudaFuncSetAttribute(key_scores_rope_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  static int resident = 0;   // per instantiation; the answer depends only on the kernel and the device type
+  if (resident == 0) {
+    int n = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, key_scores_rope_kernel<G>, kScoresThreads, smem);
+    if (e != cudaSuccess) return e;
+    resident = n < 1 ? 1 : n;
+  }
+  const long long cap_items = (long long)p.nb * p.n_heads *
+                              (((long long)p.max_pages_per_seq * p.page_tokens + kMinItemTokens - 1) / kMinItemTokens);
+  long long grid = (long long)resident * sm_count;
+  if (grid > cap_items) grid = cap_items;
+  if (grid < 1) grid = 1;
+  key_scores_rope_kernel<G><<<(int)grid, kScoresThreads, smem, stream>>>(k, k_run, p);
+  return cudaGetLastError();
+}
+
 template <int G, bool ROPE>
 constexpr size_t stored_smem_bytes() {
   return 1024 + (ROPE ? (size_t)(kRopeKSlots + RopeVSlots<G>::value) * kSlotBytes + sizeof(StoredRopeSmem<G>)
@@ -930,9 +1089,8 @@ bool stored_mma_supported(int dtype, int head_dim, int group, int max_batch) {
 
 int stored_rows_per_box(int page_tokens) { return page_tokens < kStageTokens ? page_tokens : kStageTokens; }
 
-cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, const CUtensorMap& v_map,
-                                   const CUtensorMap& k_run_map, const CUtensorMap& v_run_map, int n_heads, int32_t* item_tokens_slots, int sm_count, cudaStream_t stream) {
-  if (n_heads == 0) return cudaSuccess;
+namespace {
+StoredParams stored_params(const AttnArgs& a, int n_heads) {
   StoredParams p;
   p.q = reinterpret_cast<const __nv_bfloat16*>(a.q);
   p.slots = a.slots;
@@ -946,6 +1104,9 @@ cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, 
   p.part_o = a.parts.o;
   p.max_parts = a.parts.max_parts;
   p.status = a.status;
+  p.item_tokens_out = nullptr;
+  p.b0 = 0;
+  p.nb = 0;
   p.n_q_heads = a.n_q_heads;
   p.n_heads = n_heads;
   p.rows_per_box = stored_rows_per_box(a.geom.page_tokens);
@@ -953,9 +1114,19 @@ cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, 
   while ((1 << p.page_shift) < p.page_tokens) ++p.page_shift;
   p.box_shift = 0;
   while ((1 << p.box_shift) < p.rows_per_box) ++p.box_shift;
-  if ((1 << p.page_shift) != p.page_tokens) return cudaErrorInvalidValue;     // (pages of 16, 32, 64 or 128 tokens)
   p.scale_log2e = a.scale_log2e;
   p.rope = a.rope;
+  p.scores = nullptr;
+  p.l_cap = p.n_sink = p.n_window = 0;
+  return p;
+}
+}  // namespace
+
+cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, const CUtensorMap& v_map,
+                                   const CUtensorMap& k_run_map, const CUtensorMap& v_run_map, int n_heads, int32_t* item_tokens_slots, int sm_count, cudaStream_t stream) {
+  if (n_heads == 0) return cudaSuccess;
+  StoredParams p = stored_params(a, n_heads);
+  if ((1 << p.page_shift) != p.page_tokens) return cudaErrorInvalidValue;     // (pages of 16, 32, 64 or 128 tokens)
   const int g = a.n_q_heads / a.n_kv_heads;
   for (int b0 = 0, launch = 0; b0 < a.batch; b0 += kStoredMaxBatchPerLaunch, ++launch) {
     if (launch >= kStoredMaxLaunches) return cudaErrorInvalidValue;
@@ -968,6 +1139,34 @@ cudaError_t launch_attn_stored_mma(const AttnArgs& a, const CUtensorMap& k_map, 
       case 2: e = launch_g<2>(k_map, v_map, k_run_map, v_run_map, p, sm_count, stream); break;
       case 4: e = launch_g<4>(k_map, v_map, k_run_map, v_run_map, p, sm_count, stream); break;
       case 8: e = launch_g<8>(k_map, v_map, k_run_map, v_run_map, p, sm_count, stream); break;
+      default: return cudaErrorInvalidValue;
+    }
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t launch_key_scores_stored(const AttnArgs& a, const CUtensorMap& k_map, const CUtensorMap& k_run_map,
+                                     int n_heads, float* S, int l_cap, int n_sink, int n_window, int sm_count,
+                                     cudaStream_t stream) {
+  if (n_heads == 0) return cudaSuccess;
+  if (a.dtype != ECHOKV_BF16 || a.head_dim != 128 || a.rope.cs == nullptr) return cudaErrorInvalidValue;
+  StoredParams p = stored_params(a, n_heads);
+  if ((1 << p.page_shift) != p.page_tokens) return cudaErrorInvalidValue;
+  p.scores = S;
+  p.l_cap = l_cap;
+  p.n_sink = n_sink;
+  p.n_window = n_window;
+  const int g = a.n_q_heads / a.n_kv_heads;
+  for (int b0 = 0; b0 < a.batch; b0 += kStoredMaxBatchPerLaunch) {
+    p.b0 = b0;
+    p.nb = a.batch - b0 < kStoredMaxBatchPerLaunch ? a.batch - b0 : kStoredMaxBatchPerLaunch;
+    cudaError_t e;
+    switch (g) {
+      case 1: e = launch_scores_g<1>(k_map, k_run_map, p, sm_count, stream); break;
+      case 2: e = launch_scores_g<2>(k_map, k_run_map, p, sm_count, stream); break;
+      case 4: e = launch_scores_g<4>(k_map, k_run_map, p, sm_count, stream); break;
+      case 8: e = launch_scores_g<8>(k_map, k_run_map, p, sm_count, stream); break;
       default: return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;
