@@ -821,8 +821,21 @@ cudaError_t launch_append_side(int dtype, const SideArgs& side, int m, int D, co
 // retained head (only asked for by the absorbed mode, first_head = 0) reads the pool only.  The K pool may be wider
 // than the V pool (mk > m: keys kept whole); the keys' side buffer is then not read at all.
 // The partial goes to index fixed_part, or ceil(len / part_tokens) if that is < 0.
+constexpr int kSideThreads = 160;      // the paper's 4 + 128 full-precision tokens in one pass of a token per thread
+constexpr int kSideWarps = kSideThreads / 32;
+// four consecutive stored elements, widened to fp32
+__device__ __forceinline__ void load4(const float* p, float (&out)[4]) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&out)[4]) {
+  const uint2 v = *reinterpret_cast<const uint2*>(p);
+  out[0] = __uint_as_float(v.x << 16); out[1] = __uint_as_float(v.x & 0xffff0000u);
+  out[2] = __uint_as_float(v.y << 16); out[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+
 template <typename T, int DH>
-__global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __restrict__ k_side,
+__global__ void __launch_bounds__(kSideThreads) attn_side_kernel(AttnArgs a, const T* __restrict__ k_side,
                                                         const T* __restrict__ v_side, int n_sink, int n_window,
                                                         int d_drop, int mk, int m, int part_tokens, int first_head,
                                                         int fixed_part, const T* __restrict__ k_pool,
@@ -839,7 +852,8 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
   // element offsets of every full-precision token's row: [0] in the K pool, [1] in the V pool (the head's dim 0),
   // [2] in the side buffers (dim m)
   unsigned long long* rows = reinterpret_cast<unsigned long long*>(sc + kMaxGroup * n_side);   // [3][n_side]
-  __shared__ float red[4][kMaxGroup];
+  float* osum = reinterpret_cast<float*>(rows + 3 * n_side);                                   // [g][DH]
+  __shared__ float red[kSideWarps][kMaxGroup];
   __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
   const int slot = a.slots ? a.slots[b] : b;
   const int len = a.lens[b];
@@ -849,13 +863,13 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
   const int lo = predicted_lo(len, n_sink), hi = predicted_hi(len, n_sink, n_window);
   const int n_tok = lo + (len - hi);          // sink tokens [0, lo) then window tokens [hi, len)
   const T* q = reinterpret_cast<const T*>(a.q);
-  for (int idx = tid; idx < g * DH; idx += 128)
+  for (int idx = tid; idx < g * DH; idx += kSideThreads)
     qs[idx] = to_f32(q[((size_t)b * a.n_q_heads + kvh * g) * DH + idx]) * a.scale_log2e;
   __syncthreads();
   const size_t seq_base = (size_t)slot * n_side;
   const int32_t* table = a.geom.table + (size_t)slot * a.geom.max_pages_per_seq;
   // where each full-precision token lives (looked up once: the loops below must not chase the block table)
-  for (int i = tid; i < n_tok; i += 128) {
+  for (int i = tid; i < n_tok; i += kSideThreads) {
     const int t = i < lo ? i : hi + (i - lo);
     if (n_stored_k > 0) {
       int page = table[t / a.geom.page_tokens];
@@ -876,7 +890,7 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     return j < n_stored_k ? k_pool + rows[i] + j : k_side + rows[2 * n_side + i] + (kvh * DH + j - mk);
   };
   // scores: one token per thread
-  for (int i = tid; i < n_tok; i += 128) {
+  for (int i = tid; i < n_tok; i += kSideThreads) {
     float acc[kMaxGroup];
 #pragma unroll
     for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
@@ -916,17 +930,21 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
   // max and sum per query head
   for (int gi = 0; gi < g; ++gi) {
     float mx = -INFINITY;
-    for (int i = tid; i < n_tok; i += 128) mx = fmaxf(mx, sc[gi * n_side + i]);
+    for (int i = tid; i < n_tok; i += kSideThreads) mx = fmaxf(mx, sc[gi * n_side + i]);
     mx = warp_max(mx);
     if (lane == 0) red[warp][gi] = mx;
   }
   __syncthreads();
-  if (tid < g) s_m[tid] = fmaxf(fmaxf(red[0][tid], red[1][tid]), fmaxf(red[2][tid], red[3][tid]));
+  if (tid < g) {
+    float mx = red[0][tid];
+    for (int wi = 1; wi < kSideWarps; ++wi) mx = fmaxf(mx, red[wi][tid]);
+    s_m[tid] = mx;
+  }
   __syncthreads();
   for (int gi = 0; gi < g; ++gi) {
     const float M = s_m[gi];
     float l = 0.f;
-    for (int i = tid; i < n_tok; i += 128) {
+    for (int i = tid; i < n_tok; i += kSideThreads) {
       const float pv = exp2f(sc[gi * n_side + i] - M);
       sc[gi * n_side + i] = pv;
       l += pv;
@@ -935,29 +953,65 @@ __global__ void __launch_bounds__(128) attn_side_kernel(AttnArgs a, const T* __r
     if (lane == 0) red[warp][gi] = l;
   }
   __syncthreads();
-  if (tid < g) s_l[tid] = (red[0][tid] + red[1][tid]) + (red[2][tid] + red[3][tid]);
+  if (tid < g) {
+    float l = 0.f;
+    for (int wi = 0; wi < kSideWarps; ++wi) l += red[wi][tid];
+    s_l[tid] = l;
+  }
+  for (int idx = tid; idx < g * DH; idx += kSideThreads) osum[idx] = 0.f;
   __syncthreads();
-  // weighted V: one output feature per thread
+  // weighted V: four output features per lane, warp s on the tokens s, s + 5, ..., four loads in flight; the
+  // warps' sums are added up in shared memory, one warp after the other
   const int part = fixed_part >= 0 ? fixed_part : (len + part_tokens - 1) / part_tokens;
-  if (tid < DH) {
-    const bool from_pool = tid < n_stored;
-    const T* v_src = from_pool ? v_pool + tid : v_side + (kvh * DH + tid - m);
+  {
+    const int d0 = 4 * lane;                     // (a group of four dims never straddles n_stored: a multiple of 64)
+    const bool active = d0 < DH;
+    const bool from_pool = d0 < n_stored;
+    const T* v_src = from_pool ? v_pool + d0 : v_side + (kvh * DH + d0 - m);
     const unsigned long long* v_rows = from_pool ? rows + n_side : rows + 2 * n_side;
-    float o[kMaxGroup];
+    float o[kMaxGroup][4];
 #pragma unroll
-    for (int gi = 0; gi < kMaxGroup; ++gi) o[gi] = 0.f;
-#pragma unroll 4
-    for (int i = 0; i < n_tok; ++i) {
-      const float vv = to_f32(v_src[v_rows[i]]);
+    for (int gi = 0; gi < kMaxGroup; ++gi)
 #pragma unroll
-      for (int gi = 0; gi < kMaxGroup; ++gi)
-        if (gi < g) o[gi] = fmaf(sc[gi * n_side + i], vv, o[gi]);
+      for (int e = 0; e < 4; ++e) o[gi][e] = 0.f;
+    for (int i0 = warp; active && i0 < n_tok; i0 += 4 * kSideWarps) {
+      float vv[4][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * kSideWarps;
+        if (i < n_tok) load4(v_src + v_rows[i], vv[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * kSideWarps;
+        if (i < n_tok) {
+#pragma unroll
+          for (int gi = 0; gi < kMaxGroup; ++gi)
+            if (gi < g) {
+              const float pv = sc[gi * n_side + i];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) o[gi][e] = fmaf(pv, vv[u][e], o[gi][e]);
+            }
+        }
+      }
     }
-    for (int gi = 0; gi < g; ++gi) {
-      const size_t pidx = ((size_t)b * a.n_q_heads + kvh * g + gi) * a.parts.max_parts + part;
-      a.parts.o[pidx * DH + tid] = o[gi];
-      if (tid == 0) a.parts.ml[pidx] = make_float2(s_m[gi], s_l[gi]);
+    for (int sl = 0; sl < kSideWarps; ++sl) {
+      if (warp == sl && active) {
+#pragma unroll
+        for (int gi = 0; gi < kMaxGroup; ++gi)
+          if (gi < g) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) osum[gi * DH + d0 + e] += o[gi][e];
+          }
+      }
+      __syncthreads();
     }
+  }
+  for (int idx = tid; idx < g * DH; idx += kSideThreads) {
+    const int gi = idx / DH, d = idx - gi * DH;
+    const size_t pidx = ((size_t)b * a.n_q_heads + kvh * g + gi) * a.parts.max_parts + part;
+    a.parts.o[pidx * DH + d] = osum[idx];
+    if (d == 0) a.parts.ml[pidx] = make_float2(s_m[gi], s_l[gi]);
   }
 }
 
@@ -966,12 +1020,12 @@ static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, i
                                       cudaStream_t stream, const SidePool& pool) {
   const int n_heads = a.n_kv_heads - first_head;
   const int n_side = side.n_sink + side.n_window;
-  const size_t smem = (size_t)(kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float) + (size_t)n_side * 24 + 8;
+  const size_t smem = (size_t)(2 * kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float) + (size_t)n_side * 24 + 8;
   cudaError_t e = cudaFuncSetAttribute(attn_side_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   if (n_heads <= 0) return cudaSuccess;
   dim3 grid(n_heads, a.batch);
-  attn_side_kernel<T, DH><<<grid, 128, smem, stream>>>(
+  attn_side_kernel<T, DH><<<grid, kSideThreads, smem, stream>>>(
       a, (const T*)side.k_side, (const T*)side.v_side, side.n_sink, side.n_window, side.d_drop,
       pool.k_width > 0 ? pool.k_width : pool.width, pool.width, part_tokens, first_head, pool.part,
       (const T*)pool.k_pool, (const T*)pool.v_pool);
