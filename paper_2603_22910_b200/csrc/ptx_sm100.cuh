@@ -324,6 +324,12 @@ __device__ __forceinline__ void mma_m16n8k16_bf16(float (&c)[4], uint32_t a0, ui
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// fp32 -> tf32, round to nearest (ties away from zero)
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return r;
+}
 // tf32 x tf32 -> fp32: a0 = A[lane / 4][lane % 4], a1 = A[lane / 4 + 8][lane % 4], a2 / a3 the same rows at column
 // lane % 4 + 4; b0 = B[k = lane % 4][n = lane / 4], b1 = B[k = lane % 4 + 4][n = lane / 4].  The operands are fp32
 // bit patterns; the tensor core reads their upper 19 bits.

@@ -49,7 +49,8 @@ __device__ __forceinline__ uint32_t stage_off(int tok, int piece) {
 constexpr int kConsumers = 4;
 constexpr int kWarpTokens = kStageTokens / kConsumers;   // every consumer warp takes 16 tokens of each stage
 constexpr int kThreads = 32 * (1 + kConsumers);          // a warp that issues the copies, four consumer warps
-constexpr int kRopeThreads = 32 * (2 * kConsumers + 2);  // rotating kernel: four score warps, four value warps,
+constexpr int kValueWarps = 2;                            // value warps of the rotating kernel: 64 output features each
+constexpr int kRopeThreads = 32 * (kConsumers + kValueWarps + 2);  // rotating kernel: four score warps, four value warps,
                                                          // a warp that issues the K copies, one for the V copies
 constexpr int kMinItemTokens = 256;
 constexpr int kMaxItemTokens = 16384;
@@ -611,31 +612,36 @@ __device__ __forceinline__ void rotated_key_scores(uint32_t sb, int tok_k, const
     ldsm_x4(sb + stage_off(tok_k, 8 + c0), kb[0], kb[1], kb[2], kb[3]);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
+      // the queries' features f, f + 1 (qa) and f + 64, f + 65 (qb), turned BACK by the slice's coarse angle:
+      // q . R(U + r) k = (R(U)^T q) . (R(r) k), so a key is turned by one of the 16 fine angles only
       const float4 bw = coarse_q[ks * 8 + h * 4];                         // (cos f, sin f, cos f+1, sin f+1)
       const float2 bc = make_float2(bw.x, bw.z), bs = make_float2(bw.y, bw.w);
+      const uint32_t q_lo = h ? qa2[ks] : qa0[ks];
+      const uint32_t q_hi = h ? qa2[ks + 4] : qa0[ks + 4];
+      const float2 qa = make_float2(bf16_lo(q_lo), bf16_hi(q_lo)), qb = make_float2(bf16_lo(q_hi), bf16_hi(q_hi));
+      const float2 ta = __ffma2_rn(bs, qb, __fmul2_rn(bc, qa));
+      float2 tb = __fmul2_rn(bc, qb);
+      tb.x = fmaf(-bs.x, qa.x, tb.x);
+      tb.y = fmaf(-bs.y, qa.y, tb.y);
       float2 lo[2], hi[2];
 #pragma unroll
       for (int tile = 0; tile < 2; ++tile) {
         const int i = tile * 2 + h;
         const float4 fw = (tile ? fine_b : fine_a)[ks * 8 + h * 4];       // (cos f, cos f+1, sin f, sin f+1)
         const float2 fc = make_float2(fw.x, fw.y), fs = make_float2(fw.z, fw.w);
-        float2 cw2 = __fmul2_rn(bc, fc);
-        cw2.x = fmaf(-bs.x, fs.x, cw2.x);
-        cw2.y = fmaf(-bs.y, fs.y, cw2.y);
-        const float2 sw2 = __ffma2_rn(bs, fc, __fmul2_rn(bc, fs));
         const float2 xa = make_float2(bf16_lo(ka[i]), bf16_hi(ka[i]));
         const float2 xb = make_float2(bf16_lo(kb[i]), bf16_hi(kb[i]));
-        lo[tile] = __fmul2_rn(xa, cw2);
-        lo[tile].x = fmaf(-xb.x, sw2.x, lo[tile].x);
-        lo[tile].y = fmaf(-xb.y, sw2.y, lo[tile].y);
-        hi[tile] = __ffma2_rn(xa, sw2, __fmul2_rn(xb, cw2));
+        lo[tile] = __fmul2_rn(xa, fc);
+        lo[tile].x = fmaf(-xb.x, fs.x, lo[tile].x);
+        lo[tile].y = fmaf(-xb.y, fs.y, lo[tile].y);
+        hi[tile] = __ffma2_rn(xa, fs, __fmul2_rn(xb, fc));
       }
-      const uint32_t q_lo = h ? qa2[ks] : qa0[ks];
-      const uint32_t q_hi = h ? qa2[ks + 4] : qa0[ks + 4];
+      // (the tensor core chops its operands to tf32: the turned queries are rounded to nearest first, eight values
+      // per step against the 32 of the keys, which halves the error the chopping leaves in the scores)
       mma_m16n8k8_tf32(acc_lo, __float_as_uint(lo[0].x), __float_as_uint(lo[1].x), __float_as_uint(lo[0].y),
-                       __float_as_uint(lo[1].y), q_lo << 16, q_lo & 0xffff0000u);
+                       __float_as_uint(lo[1].y), to_tf32(ta.x), to_tf32(ta.y));
       mma_m16n8k8_tf32(acc_hi, __float_as_uint(hi[0].x), __float_as_uint(hi[1].x), __float_as_uint(hi[0].y),
-                       __float_as_uint(hi[1].y), q_hi << 16, q_hi & 0xffff0000u);
+                       __float_as_uint(hi[1].y), to_tf32(tb.x), to_tf32(tb.y));
     }
   }
 #pragma unroll
@@ -683,19 +689,19 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&rs.s_full[i]), kConsumers);
-      mbar_init(smem_u32(&rs.s_empty[i]), kConsumers);
+      mbar_init(smem_u32(&rs.s_empty[i]), kValueWarps);
     }
     for (int i = 0; i < kRingMax; ++i) {
       mbar_init(smem_u32(&rs.k_full[i]), 1);
       mbar_init(smem_u32(&rs.k_empty[i]), kConsumers);
       mbar_init(smem_u32(&rs.v_full[i]), 1);
-      mbar_init(smem_u32(&rs.v_empty[i]), kConsumers);
+      mbar_init(smem_u32(&rs.v_empty[i]), kValueWarps);
     }
   }
   const int item_tokens = stored_setup(rs.items, p);
   const int n_items = rs.items.cum_items[p.nb];
   const int rpb = p.rows_per_box;
-  const int cw = warp & 3;
+  const int cw = warp < kConsumers ? warp : warp - kConsumers;      // score warp: its token slice; value warp: its feature slice
   const int row = lane >> 2;                // MMA row / column of this thread: a token (scores) or a query head
   const int qd = (lane & 3) * 2;
 
@@ -757,7 +763,7 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
       }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");   // (a copy started before a wait gave up)
-  } else if (warp == 2 * kConsumers) {
+  } else if (warp == kConsumers + kValueWarps) {
     // =============================== the warp that issues the K copies ===========================
     StoredProducer<NK, 1> pr;
     pr.init(rs.items, p, item_tokens, n_items, lane);
@@ -765,7 +771,7 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                    item_tokens, n_items, lane)) {
     }
     if (pr.gave_up()) pr.drain(rs.k_full, lane);
-  } else if (warp == 2 * kConsumers + 1) {
+  } else if (warp == kConsumers + kValueWarps + 1) {
     // =============================== the warp that issues the V copies ===========================
     StoredProducer<NV, 2> pr;
     pr.init(rs.items, p, item_tokens, n_items, lane);
@@ -775,7 +781,9 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     if (pr.gave_up()) pr.drain(rs.v_full, lane);
   } else {
     // =============================== value warps =================================================
-    const int f0 = cw * 4;                    // first 16-byte piece (8 features) of this warp's slice of V
+    constexpr int kPieces = 16 / kValueWarps;   // 16-byte pieces (8 features) of this warp's slice of V
+    constexpr int kTiles = kPieces;             // 8-feature output tiles of the slice
+    const int f0 = cw * kPieces;
     uint32_t it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
@@ -785,9 +793,9 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
       const int t_end = min(p.lens[b], t_begin + item_tokens);
       const int n_iter = (t_end - t_begin + kStageTokens - 1) / kStageTokens;
       float m_run = -INFINITY, l_run = 0.f;
-      float o[4][4];
+      float o[kTiles][4];
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt)
+      for (int nt = 0; nt < kTiles; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
 
@@ -821,10 +829,10 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
           if (!all_valid) {
             // rows without a cached token may hold anything (never written, or a skipped page): zero this warp's
             // slice of them in V so that 0 * V stays 0; their scores are masked below
-            for (int idx = lane; idx < kStageTokens * 4; idx += 32) {
-              const int r = idx >> 2;
+            for (int idx = lane; idx < kStageTokens * kPieces; idx += 32) {
+              const int r = idx / kPieces;
               if (!((valid >> r) & 1ull)) {
-                const uint32_t a = vb + stage_off(r, f0 + (idx & 3));
+                const uint32_t a = vb + stage_off(r, f0 + idx % kPieces);
                 asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
               }
             }
@@ -864,7 +872,7 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
           l_run = l_run * alpha + psum;
           if (alpha != 1.f) {     // (the quad shares alpha)
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt)
+            for (int nt = 0; nt < kTiles; ++nt)
 #pragma unroll
               for (int e = 0; e < 4; ++e) o[nt][e] *= alpha;
           }
@@ -873,7 +881,7 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
           for (int kk = 0; kk < 4; ++kk) {
             const int tok_v = kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);    // V rows: ldmatrix.trans
 #pragma unroll
-            for (int dp = 0; dp < 2; ++dp) {
+            for (int dp = 0; dp < kTiles / 2; ++dp) {
               uint32_t r0, r1, r2, r3;
               ldsm_x4_trans(vb + stage_off(tok_v, f0 + 2 * dp + (lane >> 4)), r0, r1, r2, r3);
               mma_m16n8k16_bf16(o[2 * dp], p_hi[kk][0], p_lo[kk][0], p_hi[kk][1], p_lo[kk][1], r0, r1);
@@ -893,8 +901,8 @@ attn_stored_rope_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
       if (row < G) {
         const size_t pidx = ((size_t)b * p.n_q_heads + (size_t)w.kvh * G + row) * p.max_parts + w.chunk;
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt)
-          *reinterpret_cast<float2*>(p.part_o + pidx * 128 + cw * 32 + nt * 8 + qd) =
+        for (int nt = 0; nt < kTiles; ++nt)
+          *reinterpret_cast<float2*>(p.part_o + pidx * 128 + cw * (8 * kTiles) + nt * 8 + qd) =
               make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);
         if (cw == 0 && (lane & 3) == 0) p.part_ml[pidx] = make_float2(m_run, l_run);
       }
