@@ -350,12 +350,18 @@ int64_t echokv_launch_count(const echokv_ctx* ctx);
  * 0 = none (no layer is compressed or nothing is dropped), 1 = fp32/bf16 CUDA-core kernel,
  * 2 = bf16 tcgen05 tensor-core kernel, one CTA per SM, 3 = the same on CTA pairs
  * (cta_group::2: two SMs share every operand tile and the accumulators are double-buffered),
- * 4 = CTA pairs with four dropped heads per work item (a token tile staged once per four heads). */
+ * 4 = CTA pairs with four dropped heads per work item (a token tile staged once per four heads),
+ * 5 = 2 or 4, decided on the device at every call by the page order found in the block table (pages handed out in
+ *     order: 2, which fetches four consecutive pages as one copy; otherwise 4, which is indifferent to the order). */
 int echokv_decode_path(const echokv_ctx* ctx);
 
+/* After a decode call on path 5 (synchronises the device): *out = 1 if that call found the pages in order (kernel
+ * family 2 ran), 0 if not (family 4 ran).  EINVAL on another path. */
+int echokv_diag_page_order(echokv_ctx* ctx, int32_t* out);
+
 /* Choose the kernel family for compressed layers: 1 = CUDA-core kernel (always possible),
- * 2, 3 or 4 = tcgen05 kernels (EUNSUPPORTED unless dtype is bf16, head_dim 128; 4 also needs at most two query
- * heads per KV head).  Contexts start on the fastest family their shape allows.  Meant for tests that check all
+ * 2, 3, 4 or 5 = tcgen05 kernels (EUNSUPPORTED unless dtype is bf16, head_dim 128; 4 and 5 also need at most two
+ * query heads per KV head, 5 pages of at most 32 tokens).  Contexts start on the fastest family their shape allows.  Meant for tests that check all
  * against the oracle. */
 int echokv_set_decode_path(echokv_ctx* ctx, int path);
 

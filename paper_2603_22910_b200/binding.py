@@ -83,6 +83,7 @@ EXPORTS = {
     "echokv_read_kernel_timing": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "echokv_read_kernel_timing_by_kind": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "echokv_diag_bounded_wait": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
+    "echokv_diag_page_order": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
     "echokv_full_attention_noalloc": (C.c_int, [C.POINTER(echokv_config), C.c_void_p, C.c_void_p, C.c_void_p,
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                                 C.c_void_p, C.c_void_p]),
@@ -274,6 +275,11 @@ class Context:
 
     def decode_path(self) -> int:
         return lib().echokv_decode_path(self.handle)
+
+    def diag_page_order(self) -> int:
+        out = C.c_int32(-1)
+        _check(lib().echokv_diag_page_order(self.handle, C.byref(out)), "echokv_diag_page_order")
+        return out.value
 
     def set_decode_path(self, path: int) -> None:
         _check(lib().echokv_set_decode_path(self.handle, path), "echokv_set_decode_path")

@@ -152,6 +152,8 @@ int32_t* status_ptr(echokv_ctx* c) { return reinterpret_cast<int32_t*>(c->ws + c
 // item sizes the stored-head kernel publishes for the merge kernel: kStoredMaxLaunches words that
 // share the status word's 256-byte block
 int32_t* item_tokens_ptr(echokv_ctx* c) { return reinterpret_cast<int32_t*>(c->ws + c->d.off_status + 64); }
+// the word the page-order kernel writes (decode path 5)
+int32_t* page_order_ptr(echokv_ctx* c) { return reinterpret_cast<int32_t*>(c->ws + c->d.off_status + 32); }
 
 PageGeom geom_of(const echokv_ctx* c) {
   PageGeom g;
@@ -379,7 +381,7 @@ int echokv_create(const echokv_config* cfg, const echokv_buffers* buf, echokv_ct
     // against 2.28 ms).  So small pages go to the latter.
     const int chunks = d.d_in / 64;
     if (chunks <= 12 * d.g) c->path = 3;
-    else c->path = (recon_quad_supported(d.g) && cfg->page_tokens <= 32) ? 4 : 2;
+    else c->path = (recon_quad_supported(d.g) && cfg->page_tokens <= 32) ? 5 : 2;
   }
   if (c->tc_capable) {
     // tensor maps of every pool (the predictors' maps follow in echokv_set_weights)
@@ -471,8 +473,9 @@ int echokv_set_decode_path(echokv_ctx* c, int path) {
   if (!c) return ECHOKV_EINVAL;
   if (c->path == 0) return path == 0 ? ECHOKV_OK : ECHOKV_EINVAL;
   if (path == 1) { c->path = 1; return ECHOKV_OK; }
-  if (path == 2 || path == 3 || path == 4) {
-    if (!c->tc_capable || (path == 4 && !recon_quad_supported(c->d.g))) return ECHOKV_EUNSUPPORTED;
+  if (path >= 2 && path <= 5) {
+    if (!c->tc_capable || (path >= 4 && !recon_quad_supported(c->d.g))) return ECHOKV_EUNSUPPORTED;
+    if (path == 5 && c->cfg.page_tokens > 32) return ECHOKV_EUNSUPPORTED;
     c->path = path;
     return ECHOKV_OK;
   }
@@ -803,9 +806,23 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
   ra.n_sink = side ? c->n_sink : 0;
   ra.n_window = side ? c->n_window : 0;
   cudaError_t e;
+  const bool by_page_order = c->path == 5;
+  if (by_page_order) {
+    // both kernels are launched and the page order found in the block table says which of them runs
+    if (launch_page_order(a, page_order_ptr(c), s) != cudaSuccess) return ECHOKV_ECUDA;
+    ra.choose = page_order_ptr(c);
+    c->launches += 2;
+  }
   {
     ScopedKernelTimer timer(c, s, ECHOKV_TIMED_RECON);
-    if (c->path == 4) {
+    if (by_page_order) {
+      ra.choose_value = 0;
+      e = launch_recon_quad(a, ra, A.tc, L.tc, c->sm_count, s);
+      if (e == cudaSuccess) {
+        ra.choose_value = 1;
+        e = launch_recon_tc(a, ra, A.tc, L.tc, c->sm_count, s);
+      }
+    } else if (c->path == 4) {
       e = launch_recon_quad(a, ra, A.tc, L.tc, c->sm_count, s);
     } else if (c->path == 3) {
       e = launch_recon_pair(a, ra, A.tc, L.tc, c->sm_count, s);
@@ -821,13 +838,14 @@ int echokv_decode_attention(echokv_ctx* c, int layer, const void* q, float* out,
     // sink and recent-window tokens: Eq. 7 on their stored dims, one more partial per query head
     SidePool pool;
     pool.k_pool = L.k_pool; pool.v_pool = L.v_pool; pool.width = c->d.m; pool.part = -1;
-    if (launch_attn_side(a, side_args(c, L), r, recon_part_tokens, s, pool) != cudaSuccess) return ECHOKV_ECUDA;
+    if (launch_attn_side(a, side_args(c, L), r, recon_part_tokens, s, pool, ra.choose, kTcPartTokens) != cudaSuccess)
+      return ECHOKV_ECUDA;
     c->launches += 1;
   }
   // (a K bias is inside the scores already where the keys are rotated; otherwise it only matters against the
   // sink / window tokens, and the merge accounts for it)
   if (launch_merge(a, out, r, n_splits, item_tokens, kStoredMaxBatchPerLaunch, recon_part_tokens, L.bv_x, s,
-                   side ? 1 : 0, side && c->rope.cs == nullptr ? L.bk_x : nullptr) != cudaSuccess)
+                   side ? 1 : 0, side && c->rope.cs == nullptr ? L.bk_x : nullptr, ra.choose, kTcPartTokens) != cudaSuccess)
     return ECHOKV_ECUDA;
   c->launches += 2;
   return ECHOKV_OK;
@@ -918,6 +936,13 @@ int echokv_read_kernel_timing(echokv_ctx* c, double* total_ms, int64_t* n_launch
     *total_ms += ms[k];
     *n_launches += n[k];
   }
+  return ECHOKV_OK;
+}
+
+int echokv_diag_page_order(echokv_ctx* c, int32_t* out) {
+  if (!c || !out || c->path != 5) return ECHOKV_EINVAL;
+  if (cudaDeviceSynchronize() != cudaSuccess) return ECHOKV_ECUDA;
+  if (cudaMemcpy(out, page_order_ptr(c), sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return ECHOKV_ECUDA;
   return ECHOKV_OK;
 }
 

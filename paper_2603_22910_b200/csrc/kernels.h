@@ -54,7 +54,16 @@ struct ReconArgs {
   int n_sink = 0, n_window = 0;                 // tokens kept at full precision: the first n_sink and the last
                                                 // n_window of a sequence are NOT predicted here (they are
                                                 // attended from the side buffers, see launch_attn_side)
+  // Two kernels launched for the same work, one of which does it: a kernel given `choose` runs only if the device
+  // word holds choose_value (see launch_page_order), else it returns at once.  Null: run.
+  const int32_t* choose = nullptr;
+  int choose_value = 0;
 };
+
+// *flag (device) = 1 if most of the sequences' aligned 64-token groups lie on consecutive pool rows (their pages were
+// handed out in order), else 0: the one-CTA fused kernel fetches such a group as one copy and is the faster one
+// there, the four-head CTA-pair kernel is indifferent to the page order (a sample of the groups is looked at).
+cudaError_t launch_page_order(const AttnArgs& a, int32_t* flag, cudaStream_t stream);
 
 // Whole retained heads of a compressed layer (the kernels' first predicted head).
 __host__ __device__ inline int retained_heads(const ReconArgs& r, int head_dim) { return (r.m_heads >= 0 ? r.m_heads : r.m) / head_dim; }
@@ -105,8 +114,11 @@ struct SidePool {
   int part;
   int k_width = 0;                          // row width of the K pool where it differs (keys kept whole: D); 0: width
 };
+// choose / alt_part_tokens: where two fused kernels with different partial sizes were launched for the same work
+// (ReconArgs::choose), the partials are alt_part_tokens long if *choose == 1, else part_tokens.
 cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int first_head, int part_tokens,
-                             cudaStream_t stream, const SidePool& pool);
+                             cudaStream_t stream, const SidePool& pool, const int32_t* choose = nullptr,
+                             int alt_part_tokens = 0);
 
 // CUDA-core reconstruct-then-attend (fp32 or bf16 storage, fp32 FFMA): Eq. 3, 6, 7 for the
 // dropped KV heads; one partial per part_tokens tokens.
@@ -123,6 +135,6 @@ cudaError_t launch_recon_simt(const AttnArgs& a, const ReconArgs& r, cudaStream_
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
                          const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
                          const void* bv, cudaStream_t stream, int extra_recon_part = 0,
-                         const void* bk_shift = nullptr);
+                         const void* bk_shift = nullptr, const int32_t* choose = nullptr, int alt_part_tokens = 0);
 
 }  // namespace echokv

@@ -65,6 +65,8 @@ struct QuadParams {
   float scale_log2e;
   RopeTable rope;             // read by the ROPE instantiations only
   const __nv_bfloat16* bk;    // bias of the K predictor or null (ROPE instantiations only: otherwise it cancels)
+  const int32_t* choose;      // null, or: run only if this device word holds choose_value (ReconArgs::choose)
+  int choose_value;
 };
 
 template <int G>
@@ -97,6 +99,8 @@ recon_quad_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_
                   const __grid_constant__ CUtensorMap tm_local_k_run, const __grid_constant__ CUtensorMap tm_local_v_run,
                   const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
                   const QuadParams p) {
+  if (p.choose != nullptr && *p.choose != p.choose_value) return;      // (both CTAs of the pair alike: the other
+                                                                       // kernel launched for this work runs)
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -562,6 +566,8 @@ cudaError_t launch_recon_quad(const AttnArgs& a, const ReconArgs& r, const TcLay
   p.part_o = a.parts.o;
   p.max_parts = a.parts.max_parts;
   p.status = a.status;
+  p.choose = r.choose;
+  p.choose_value = r.choose_value;
   p.n_q_heads = a.n_q_heads;
   p.n_ret_heads = retained_heads(r, 128);
   p.n_drop_heads = a.n_kv_heads - p.n_ret_heads;

@@ -66,6 +66,8 @@ struct TcParams {
   float scale_log2e;
   RopeTable rope;             // read by the ROPE instantiations only
   const __nv_bfloat16* bk;    // bias of the K predictor or null (ROPE instantiations only: otherwise it cancels)
+  const int32_t* choose;      // null, or: run only if this device word holds choose_value (ReconArgs::choose)
+  int choose_value;
 };
 
 template <int G>
@@ -100,6 +102,7 @@ recon_tc_kernel(const __grid_constant__ CUtensorMap tm_anchor_k, const __grid_co
                 const __grid_constant__ CUtensorMap tm_local_k_run, const __grid_constant__ CUtensorMap tm_local_v_run,
                 const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
                 const TcParams p) {
+  if (p.choose != nullptr && *p.choose != p.choose_value) return;      // (the other kernel launched for this work runs)
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -695,6 +698,8 @@ cudaError_t launch_recon_tc(const AttnArgs& a, const ReconArgs& r, const TcLayer
   p.part_o = a.parts.o;
   p.max_parts = a.parts.max_parts;
   p.status = a.status;
+  p.choose = r.choose;
+  p.choose_value = r.choose_value;
   p.n_q_heads = a.n_q_heads;
   p.n_ret_heads = retained_heads(r, 128);
   p.n_drop_heads = a.n_kv_heads - p.n_ret_heads;

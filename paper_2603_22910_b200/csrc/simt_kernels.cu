@@ -620,7 +620,9 @@ template <typename T>
 __global__ void __launch_bounds__(128 * kMergeGroups)
 merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stored_parts,
              const int32_t* __restrict__ stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-             const T* __restrict__ bv, const T* __restrict__ bk_shift, int extra_recon_part) {
+             const T* __restrict__ bv, const T* __restrict__ bk_shift, int extra_recon_part,
+             const int32_t* __restrict__ choose, int alt_part_tokens) {
+  if (choose != nullptr && *choose == 1) part_tokens = alt_part_tokens;
   const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x, grp = threadIdx.y;
   const int DH = a.head_dim;                      // == blockDim.x
   const int tid = grp * DH + j, n_threads = DH * kMergeGroups;
@@ -709,17 +711,18 @@ merge_kernel(AttnArgs a, float* __restrict__ out, int n_stored_heads, int n_stor
 
 cudaError_t launch_merge(const AttnArgs& a, float* out, int n_stored_heads, int n_stored_parts,
                          const int32_t* stored_item_tokens, int stored_batch_per_slot, int part_tokens,
-                         const void* bv, cudaStream_t stream, int extra_recon_part, const void* bk_shift) {
+                         const void* bv, cudaStream_t stream, int extra_recon_part, const void* bk_shift,
+                         const int32_t* choose, int alt_part_tokens) {
   dim3 grid(a.n_q_heads, a.batch);
   if (a.dtype == ECHOKV_BF16) {
     merge_kernel<__nv_bfloat16><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(
         a, out, n_stored_heads, n_stored_parts, stored_item_tokens, stored_batch_per_slot, part_tokens,
-        (const __nv_bfloat16*)bv, (const __nv_bfloat16*)bk_shift, extra_recon_part);
+        (const __nv_bfloat16*)bv, (const __nv_bfloat16*)bk_shift, extra_recon_part, choose, alt_part_tokens);
   } else {
     merge_kernel<float><<<grid, dim3(a.head_dim, kMergeGroups), 0, stream>>>(a, out, n_stored_heads, n_stored_parts,
                                                          stored_item_tokens, stored_batch_per_slot,
                                                          part_tokens, (const float*)bv, (const float*)bk_shift,
-                                                         extra_recon_part);
+                                                         extra_recon_part, choose, alt_part_tokens);
   }
   return cudaGetLastError();
 }
@@ -839,7 +842,9 @@ __global__ void __launch_bounds__(kSideThreads) attn_side_kernel(AttnArgs a, con
                                                         const T* __restrict__ v_side, int n_sink, int n_window,
                                                         int d_drop, int mk, int m, int part_tokens, int first_head,
                                                         int fixed_part, const T* __restrict__ k_pool,
-                                                        const T* __restrict__ v_pool) {
+                                                        const T* __restrict__ v_pool,
+                                                        const int32_t* __restrict__ choose, int alt_part_tokens) {
+  if (choose != nullptr && *choose == 1) part_tokens = alt_part_tokens;
   extern __shared__ float side_smem[];
   const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = a.n_q_heads / a.n_kv_heads;
@@ -1017,7 +1022,8 @@ __global__ void __launch_bounds__(kSideThreads) attn_side_kernel(AttnArgs a, con
 
 template <typename T, int DH>
 static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, int first_head, int part_tokens,
-                                      cudaStream_t stream, const SidePool& pool) {
+                                      cudaStream_t stream, const SidePool& pool, const int32_t* choose,
+                                      int alt_part_tokens) {
   const int n_heads = a.n_kv_heads - first_head;
   const int n_side = side.n_sink + side.n_window;
   const size_t smem = (size_t)(2 * kMaxGroup * DH + kMaxGroup * n_side) * sizeof(float) + (size_t)n_side * 24 + 8;
@@ -1028,19 +1034,61 @@ static cudaError_t launch_attn_side_t(const AttnArgs& a, const SideArgs& side, i
   attn_side_kernel<T, DH><<<grid, kSideThreads, smem, stream>>>(
       a, (const T*)side.k_side, (const T*)side.v_side, side.n_sink, side.n_window, side.d_drop,
       pool.k_width > 0 ? pool.k_width : pool.width, pool.width, part_tokens, first_head, pool.part,
-      (const T*)pool.k_pool, (const T*)pool.v_pool);
+      (const T*)pool.k_pool, (const T*)pool.v_pool, choose, alt_part_tokens);
   return cudaGetLastError();
 }
 
 cudaError_t launch_attn_side(const AttnArgs& a, const SideArgs& side, int first_head, int part_tokens,
-                             cudaStream_t stream, const SidePool& pool) {
+                             cudaStream_t stream, const SidePool& pool, const int32_t* choose, int alt_part_tokens) {
   if (a.dtype == ECHOKV_BF16) {
     if (a.head_dim == 128)
-      return launch_attn_side_t<__nv_bfloat16, 128>(a, side, first_head, part_tokens, stream, pool);
-    return launch_attn_side_t<__nv_bfloat16, 64>(a, side, first_head, part_tokens, stream, pool);
+      return launch_attn_side_t<__nv_bfloat16, 128>(a, side, first_head, part_tokens, stream, pool, choose,
+                                                    alt_part_tokens);
+    return launch_attn_side_t<__nv_bfloat16, 64>(a, side, first_head, part_tokens, stream, pool, choose, alt_part_tokens);
   }
-  if (a.head_dim == 128) return launch_attn_side_t<float, 128>(a, side, first_head, part_tokens, stream, pool);
-  return launch_attn_side_t<float, 64>(a, side, first_head, part_tokens, stream, pool);
+  if (a.head_dim == 128)
+    return launch_attn_side_t<float, 128>(a, side, first_head, part_tokens, stream, pool, choose, alt_part_tokens);
+  return launch_attn_side_t<float, 64>(a, side, first_head, part_tokens, stream, pool, choose, alt_part_tokens);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Are the pages of the batch's sequences consecutive in the pool?  (see launch_page_order)
+// ---------------------------------------------------------------------------------------------
+constexpr int kOrderSamplesPerSeq = 256;
+__global__ void __launch_bounds__(256) page_order_kernel(const int32_t* __restrict__ slots,
+                                                         const int32_t* __restrict__ lens, int batch, PageGeom g,
+                                                         int32_t* __restrict__ flag) {
+  __shared__ int s_in_order, s_seen;
+  if (threadIdx.x == 0) s_in_order = s_seen = 0;
+  __syncthreads();
+  const int per_group = 64 / g.page_tokens;          // pages of an aligned 64-token group (page_tokens <= 32)
+  int in_order = 0, seen = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int slot = slots ? slots[b] : b;
+    const int len = lens[b];
+    if (slot < 0 || slot >= g.max_batch || len < 1 || len > g.max_pages_per_seq * g.page_tokens) continue;
+    const int n_groups = len / 64;                    // whole groups only
+    const int n_samples = min(n_groups, kOrderSamplesPerSeq);
+    const int32_t* table = g.table + (size_t)slot * g.max_pages_per_seq;
+    for (int i = threadIdx.x; i < n_samples; i += blockDim.x) {
+      const int grp = (int)((long long)i * n_groups / n_samples);
+      const int p0 = table[grp * per_group];
+      bool ok = true;
+      for (int k = 1; k < per_group; ++k) ok = ok && table[grp * per_group + k] == p0 + k;
+      in_order += ok ? 1 : 0;
+      ++seen;
+    }
+  }
+  atomicAdd(&s_in_order, in_order);
+  atomicAdd(&s_seen, seen);
+  __syncthreads();
+  if (threadIdx.x == 0) *flag = (s_seen > 0 && 2 * s_in_order >= s_seen) ? 1 : 0;
+}
+
+cudaError_t launch_page_order(const AttnArgs& a, int32_t* flag, cudaStream_t stream) {
+  if (a.geom.page_tokens > 32) return cudaErrorInvalidValue;
+  page_order_kernel<<<1, 256, 0, stream>>>(a.slots, a.lens, a.batch, a.geom, flag);
+  return cudaGetLastError();
 }
 
 }  // namespace echokv

@@ -71,7 +71,7 @@ def test_small_shapes_against_oracle(name, base, over, lens, path):
     if path == 4 and w.n_q_heads // w.n_kv_heads > 2:
         case.close()
         pytest.skip("the four-heads-per-item kernel takes at most two query heads per KV head")
-    assert case.ctx.decode_path() in (1, 2, 3, 4)  # a context starts on the family its shape runs fastest on
+    assert case.ctx.decode_path() in (1, 2, 3, 4, 5)  # a context starts on the family its shape runs fastest on
     case.ctx.set_decode_path(path)
     check_layers(case, name)
     case.close()
@@ -376,4 +376,34 @@ def test_a_page_outside_the_pool_is_reported_and_harms_no_other_sequence(mode):
     ctx.block_table.copy_(saved)
     np.testing.assert_array_equal(case.run(1), good)
     assert ctx.device_status() == binding.ECHOKV_OK
+    case.close()
+
+
+def test_the_kernel_family_follows_the_page_order_found_in_the_block_table():
+    """Decode path 5: both fused kernels are launched and a word written on the device (pages of the batch in order
+    or not) says which of them runs; the merge and the sink / window partial follow the partial size of that kernel."""
+    base = synth.C1.replace(batch=3, context=1500)
+    lens = [1500, 700, 64]
+    for window in (None, (4, 128)):
+        flags = {}
+        for random_pages in (False, True):
+            w = base.replace(random_pages=random_pages)
+            case = Case(w, lens=lens, layers=[0, 1], window=window)
+            assert case.ctx.decode_path() == 5            # long contraction, one query head per KV head, 16-token pages
+            out = case.run(1)
+            flags[random_pages] = case.ctx.diag_page_order()
+            assert_parity(out, case.oracle(1), w.dtype, "path 5, random_pages=%s, window=%s" % (random_pages, window))
+            # the same numbers as the kernel family it chose, run on its own
+            case.ctx.set_decode_path(2 if flags[random_pages] == 1 else 4)
+            np.testing.assert_array_equal(case.run(1), out)
+            case.ctx.set_decode_path(5)
+            np.testing.assert_array_equal(case.run(1), out)
+            assert case.ctx.device_status() == binding.ECHOKV_OK
+            case.close()
+        assert flags == {False: 1, True: 0}
+    # pages of 64 tokens: nothing to decide
+    case = Case(synth.C1.replace(batch=2, context=300, page_tokens=64), lens=[300, 100], layers=[0, 1])
+    assert case.ctx.decode_path() == 2
+    with pytest.raises(Exception):
+        case.ctx.set_decode_path(5)
     case.close()

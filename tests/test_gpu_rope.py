@@ -42,7 +42,7 @@ def test_rope_against_oracle(name, base, over, lens, window):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], window=window, rope=THETA)
     assert case.ctx.rope_enabled()
-    paths = ([1, 2, 3] + ([4] if w.n_q_heads // w.n_kv_heads <= 2 else [])) if case.ctx.decode_path() >= 2 else [1]
+    paths = ([1, 2, 3] + (([4, 5] if w.page_tokens <= 32 else [4]) if w.n_q_heads // w.n_kv_heads <= 2 else [])) if case.ctx.decode_path() >= 2 else [1]
     stored_paths = [0, 1] if case.ctx.stored_path() == 1 else [0]
     ref0, ref1 = case.oracle(0), case.oracle(1)
     for stored_path in stored_paths:
@@ -75,7 +75,7 @@ def test_rope_with_predictor_biases(base, over, lens, window):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], biases=True, rope=THETA, window=window)
     ref = case.oracle(1)
-    for path in (([1, 2, 3] + ([4] if w.n_q_heads // w.n_kv_heads <= 2 else [])) if case.ctx.decode_path() >= 2 else [1]):
+    for path in (([1, 2, 3] + (([4, 5] if w.page_tokens <= 32 else [4]) if w.n_q_heads // w.n_kv_heads <= 2 else [])) if case.ctx.decode_path() >= 2 else [1]):
         case.ctx.set_decode_path(path)
         assert_parity(case.run(1), ref, w.dtype, "biases path %d" % path)
     Wk, Wv, bk, bv = case.weights[1]

@@ -40,7 +40,7 @@ CASES = [
 def test_window_against_oracle(name, base, over, lens, window, biases):
     w = base.replace(**over)
     case = Case(w, lens=lens, layers=[0, 1], window=window, biases=biases)
-    paths = ([1, 2, 3] + ([4] if w.n_q_heads // w.n_kv_heads <= 2 else [])) if case.ctx.decode_path() >= 2 else [1]
+    paths = ([1, 2, 3] + (([4, 5] if w.page_tokens <= 32 else [4]) if w.n_q_heads // w.n_kv_heads <= 2 else [])) if case.ctx.decode_path() >= 2 else [1]
     for path in paths:
         case.ctx.set_decode_path(path)
         assert_parity(case.run(1), case.oracle(1), w.dtype, "%s path %d" % (name, path))
