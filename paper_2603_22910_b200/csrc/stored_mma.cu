@@ -25,7 +25,7 @@
 // their positions as they are read.  That is ALU work of several hundred instructions per 16 tokens, too much
 // for the four consumer warps beside their own work, so attn_stored_rope_kernel splits the roles: four score
 // warps turn the keys (fp32, two frequency indices per instruction) and form q . k as tf32 products, hand the
-// scores of a stage through shared memory to four value warps, which run the softmax and P V; two more warps
+// scores of a stage through shared memory to two value warps, which run the softmax and P V; two more warps
 // issue the copies.
 #include "stored_mma.h"
 
@@ -50,8 +50,8 @@ constexpr int kConsumers = 4;
 constexpr int kWarpTokens = kStageTokens / kConsumers;   // every consumer warp takes 16 tokens of each stage
 constexpr int kThreads = 32 * (1 + kConsumers);          // a warp that issues the copies, four consumer warps
 constexpr int kValueWarps = 2;                            // value warps of the rotating kernel: 64 output features each
-constexpr int kRopeThreads = 32 * (kConsumers + kValueWarps + 2);  // rotating kernel: four score warps, four value warps,
-                                                         // a warp that issues the K copies, one for the V copies
+constexpr int kRopeThreads = 32 * (kConsumers + kValueWarps + 2);  // rotating kernel: four score warps, the value
+                                                         // warps, a warp that issues the K copies, one for the V copies
 constexpr int kMinItemTokens = 256;
 constexpr int kMaxItemTokens = 16384;
 constexpr int kItemsPerCta = 6;                      // target number of work items per CTA
@@ -570,14 +570,15 @@ attn_stored_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
 // Keys rotated to their positions as they are read (Section 3.2)
 // =================================================================================================================
 // The angle of token 16 u + r is the sum of a coarse angle (row u of the coarse table) and a fine one (row r of the
-// fine table): (cos, sin) of the sum by the addition formulas.  Frequency index f pairs feature f of the head's
-// first 64 features with feature f + 64.
+// fine table), and q . R(u, r) k = (R(u)^T q) . (R(r) k): the queries are turned back by the coarse angle of the
+// 16-token slice, a key is turned by one of 16 fine angles.  Frequency index f pairs feature f of the head's first
+// 64 features with feature f + 64.
 //
 // Roles.  Score warp w (warps 0..3) takes tokens 16 w .. 16 w + 15 of every stage: keys turned in fp32, q . k as
-// tf32 products, the 16 x G raw scores into a buffer in shared memory.  Value warp w (warps 4..7) takes features
-// 32 w .. 32 w + 31 of the output for all 64 tokens of the stage: every value warp runs the same softmax over the
-// stage's scores (same operations, same results) and multiplies P into its slice of V, so the running output needs
-// 16 registers and nothing is combined across warps at the end of an item.  Warp 8 issues the K copies, warp 9 the
+// tf32 products, the 16 x G raw scores into a buffer in shared memory.  Value warp w (warps 4, 5) takes features
+// 64 w .. 64 w + 63 of the output for all 64 tokens of the stage: both value warps run the same softmax over the
+// stage's scores (same operations, same results) and multiply P into their slice of V, so the running output needs
+// 32 registers and nothing is combined across warps at the end of an item.  Warp 6 issues the K copies, warp 7 the
 // V copies: the per-stage block-table arithmetic is a serial chain of some hundred instructions that must not sit
 // in a warp the others wait for.
 //
@@ -593,9 +594,10 @@ constexpr int kRingMax = 4;
 constexpr int kSlotBytes = 2 * kBlockBytes;
 
 // The score warps' work on one 16-token slice of a K slot (sb: the slot; tok_k: this lane's ldmatrix row):
-// S^T = K' Q^T as tf32 products m16n8k8 with the 16 tokens on the M rows: the thread's two features of a token (f and
-// f + 1) are the k indices lane % 4 and lane % 4 + 4 of one product, for the key and for the query alike.  The
-// features 64 .. 127 accumulate apart: two shorter chains of products.
+// S^T = K' Q'^T as tf32 products m16n8k8 with the 16 tokens on the M rows (K': keys turned by the fine angle; Q':
+// queries turned back by the slice's coarse angle, coarse_q): the thread's two features of a token (f and f + 1) are
+// the k indices lane % 4 and lane % 4 + 4 of one product, for the key and for the query alike.  The features
+// 64 .. 127 accumulate apart: two shorter chains of products.
 // acc[0], acc[1]: token lane / 4 of the slice, heads qd and qd + 1; acc[2], acc[3]: token lane / 4 + 8 (raw q . k).
 __device__ __forceinline__ void rotated_key_scores(uint32_t sb, int tok_k, const float4* coarse_q,
                                                    const float4* fine_a, const float4* fine_b,
