@@ -256,13 +256,18 @@ def test_layer_step_from_host_memory_matches_device_calls():
     case.close(); other.close()
 
 
-@pytest.mark.parametrize("absorbed", [False, True], ids=["explicit", "absorbed"])
+@pytest.mark.parametrize("absorbed", [False, True, "by_page_order"], ids=["explicit", "absorbed", "by_page_order"])
 def test_layer_step_replayed_from_a_cuda_graph(absorbed):
     # every call only enqueues kernels on the caller's stream, so a whole step can be captured once and replayed
+    # (by_page_order: the kernel family is decided on the device inside the captured step, decode path 5)
     w = synth.C2.replace(batch=2, context=600)
+    if absorbed == "by_page_order":
+        w = synth.C1.replace(batch=2, context=600, random_pages=True)
     case = Case(w, lens=[600, 333], layers=[0, 1])
     ctx, dev = case.ctx, case.ctx.device
-    if absorbed:
+    if absorbed == "by_page_order":
+        assert ctx.decode_path() == 5
+    elif absorbed:
         ctx.enable_absorbed()
     q = {l: case.q[l].to(dev) for l in (0, 1)}
     out = {l: torch.empty(q[l].shape, dtype=torch.float32, device=dev) for l in (0, 1)}
