@@ -1161,6 +1161,26 @@ def run_single(args, rep, peaks, peaks_kind):
     return line
 
 
+def graph_replay_ms(run, rep, steps):
+    """The step captured once in a CUDA graph and replayed: what a serving loop that captures its decode step pays
+    (the launch gaps between the kernels of a short step are what it removes)."""
+    torch = run.torch
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run.step()                                   # (first-use set-up of every kernel stays outside the capture)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            run.step()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        graph.replay()
+    ms_total, _, _ = timed(run, rep, graph.replay, steps, kernel_timing=False)
+    del graph
+    return ms_total / steps
+
+
 def run_sweep(args, rep, peaks, peaks_kind):
     """--workload c4 --sweep: every point of the sweep that fits the device, explicit, absorbed and uncompressed
     steps side by side, each against its own roofline."""
@@ -1186,6 +1206,8 @@ def run_sweep(args, rep, peaks, peaks_kind):
                 for _ in range(3):
                     run.step()
                 ms_exp, timing, _ = timed(run, rep, run.step, steps)
+                small = B * L <= 2 ** 17         # short steps: also replayed from a CUDA graph
+                ms_exp_graph = graph_replay_ms(run, rep, steps) if small else None
                 ref = run.st.out[1].clone()
                 run.full_out = torch.empty_like(ref)
                 for _ in range(3):
@@ -1196,6 +1218,7 @@ def run_sweep(args, rep, peaks, peaks_kind):
                     run.step()
                 ms_abs, _, _ = timed(run, rep, run.step, steps)
                 diff = float((run.st.out[1] - ref).norm() / ref.norm())
+                ms_abs_graph = graph_replay_ms(run, rep, steps) if small else None
                 status = run.ctx.device_status()
                 flops, bytes_ = algorithmic_work(w)
                 recon_ms, recon_n = timing["recon"]
@@ -1211,6 +1234,12 @@ def run_sweep(args, rep, peaks, peaks_kind):
                     "ms_uncompressed": ms_full / steps,
                     "uncompressed_step_frac_of_hbm": full_bytes / (ms_full / steps * 1e-3) / 1e9 / hbm,
                     "rel_l2_absorbed_vs_explicit": diff, "device_status": status})
+                if small:
+                    points[-1].update({
+                        "ms_explicit_graph": ms_exp_graph,
+                        "step_frac_of_burst_peak_graph": flops / (ms_exp_graph * 1e-3) / 1e12 / burst,
+                        "ms_absorbed_graph": ms_abs_graph,
+                        "absorbed_step_frac_of_hbm_graph": bytes_ / (ms_abs_graph * 1e-3) / 1e9 / hbm})
                 run.close()
                 del run, ref
                 torch.cuda.empty_cache()
